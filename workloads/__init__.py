@@ -1,0 +1,8 @@
+"""Seeded synthetic workloads shared by the CPU oracle's tests and the CUDA library's tests.
+
+This package holds no arithmetic of the method: it only describes networks as
+op lists (plain tuples) and draws seeded inputs of the stated shapes.
+"""
+from .resnet_spec import (CONV, BNRELU, ADD, MAXPOOL, HEAD, Op, resnet_v2_cifar, resnet_v2_imagenet,
+                          default_cuts, CONFIGS, config, conv_sweep_shapes)
+from .inputs import draw_inputs, draw_params, tensor_shapes, param_offsets

@@ -1,0 +1,86 @@
+"""Op lists of the pre-activation bottleneck ResNets the benchmark configurations name.
+
+An op is the tuple (kind, src0, src1, c_in, c_out, ksize, stride, pad, eps);
+src = index of the producing op, -1 = the network input.  Inside a block the
+order is BNRELU, CONV1x1, BNRELU, CONV3x3, BNRELU, CONV1x1, [projection CONV1x1], ADD.
+The stride of a down-sampling block sits on its first 1x1 conv and on the
+projection, which reads the raw block input; there is no BN after the stem.
+"""
+from collections import namedtuple
+
+CONV, BNRELU, ADD, MAXPOOL, HEAD = 1, 2, 3, 4, 5
+Op = namedtuple("Op", "kind src0 src1 c_in c_out ksize stride pad eps")
+EPS = 1e-5
+
+
+def _bottleneck_stages(ops, t, c_t, widths, blocks, first_stride):
+    for si, (w, nb) in enumerate(zip(widths, blocks)):
+        for bi in range(nb):
+            s = first_stride[si] if bi == 0 else 1
+            ops.append(Op(BNRELU, t, -1, c_t, c_t, 0, 1, 0, EPS)); a1 = len(ops) - 1
+            ops.append(Op(CONV, a1, -1, c_t, w, 1, s, 0, 0.0)); c1 = len(ops) - 1
+            ops.append(Op(BNRELU, c1, -1, w, w, 0, 1, 0, EPS)); a2 = len(ops) - 1
+            ops.append(Op(CONV, a2, -1, w, w, 3, 1, 1, 0.0)); c2 = len(ops) - 1
+            ops.append(Op(BNRELU, c2, -1, w, w, 0, 1, 0, EPS)); a3 = len(ops) - 1
+            ops.append(Op(CONV, a3, -1, w, 4 * w, 1, 1, 0, 0.0)); c3 = len(ops) - 1
+            short = t
+            if bi == 0:
+                ops.append(Op(CONV, t, -1, c_t, 4 * w, 1, s, 0, 0.0)); short = len(ops) - 1
+            ops.append(Op(ADD, c3, short, 4 * w, 4 * w, 0, 1, 0, 0.0)); t = len(ops) - 1
+            c_t = 4 * w
+    return t, c_t
+
+
+def resnet_v2_cifar(n, widths=(16, 32, 64), n_classes=10, in_ch=3):
+    """Depth 9n+2: 3x3 stem to widths[0] channels, three stages of n bottleneck blocks."""
+    ops = [Op(CONV, -1, -1, in_ch, widths[0], 3, 1, 1, 0.0)]
+    t, c_t = _bottleneck_stages(ops, 0, widths[0], widths, (n,) * len(widths), (1,) + (2,) * (len(widths) - 1))
+    ops.append(Op(BNRELU, t, -1, c_t, c_t, 0, 1, 0, EPS))
+    ops.append(Op(HEAD, len(ops) - 1, -1, c_t, n_classes, 0, 1, 0, 0.0))
+    return ops
+
+
+def resnet_v2_imagenet(blocks=(3, 8, 36, 3), widths=(64, 128, 256, 512), n_classes=1000, in_ch=3):
+    """7x7 stride-2 stem, 3x3 stride-2 max-pool, four bottleneck stages."""
+    ops = [Op(CONV, -1, -1, in_ch, widths[0], 7, 2, 3, 0.0),
+           Op(MAXPOOL, 0, -1, widths[0], widths[0], 3, 2, 1, 0.0)]
+    t, c_t = _bottleneck_stages(ops, 1, widths[0], widths, blocks, (1,) + (2,) * (len(widths) - 1))
+    ops.append(Op(BNRELU, t, -1, c_t, c_t, 0, 1, 0, EPS))
+    ops.append(Op(HEAD, len(ops) - 1, -1, c_t, n_classes, 0, 1, 0, 0.0))
+    return ops
+
+
+def default_cuts(n_ops, P):
+    """Equal op counts per partition: cut p at floor(p*K/P)."""
+    return [(p * n_ops) // P for p in range(1, P)]
+
+
+# name -> (ops builder, input (H, W, C), batch B, micro-batches M, partitions P)
+CONFIGS = {
+    "r11":   (lambda: resnet_v2_cifar(1), (32, 32, 3), 8, 2, 2),
+    "r110":  (lambda: resnet_v2_cifar(12), (32, 32, 3), 128, 4, 4),
+    "r1001": (lambda: resnet_v2_cifar(111), (32, 32, 3), 128, 8, 8),
+    "r152":  (lambda: resnet_v2_imagenet(), (224, 224, 3), 64, 4, 4),
+}
+
+
+def config(name):
+    build, hwc, B, M, P = CONFIGS[name]
+    ops = build()
+    return dict(name=name, ops=ops, in_hwc=hwc, B=B, M=M, P=P, cuts=default_cuts(len(ops), P))
+
+
+def conv_sweep_shapes():
+    """The convolution micro-benchmark sweep: (ksize, stride, c_in, c_out, H) at batch 128.
+
+    The cross product of the channel pair at each resolution for 1x1 and 3x3
+    (pad 1) convolutions, plus the four stride-2 transitions.
+    """
+    out = []
+    for H, (a, b) in ((32, (16, 64)), (16, (32, 128)), (8, (64, 256))):
+        for k in (1, 3):
+            for ci in (a, b):
+                for co in (a, b):
+                    out.append((k, 1, ci, co, H))
+    out += [(1, 2, 64, 32, 32), (1, 2, 64, 128, 32), (1, 2, 128, 64, 16), (1, 2, 128, 256, 16)]
+    return out
