@@ -1,0 +1,190 @@
+/*
+ * hpf.h -- C ABI of the B200 (sm_100a) library for the partitioned, micro-batch
+ * pipelined training step of HyPar-Flow (arXiv 1911.05146).
+ *
+ * A network is a list of ops (Section 5.1: the model as a list of layers).  The
+ * list is cut into consecutive partitions (Section 5.1); each partition becomes
+ * one pipeline stage bound to one CUDA stream.  A batch is split into
+ * micro-batches that flow through the stages (Section 5.3, "pipeline stages
+ * within each minibatch").  Activations cross a cut forward and partial errors
+ * cross it backward (Section 5.2, Eq. 5-7; Section 5.3 send/recv); on one GPU
+ * the hand-off is an event on a shared device buffer.  Per-micro-batch weight
+ * gradients land in their own slot and are averaged at the end (the arithmetic
+ * of the gradient allreduce of Section 5.3).
+ *
+ * Conventions
+ *   - Every function returns HPF_OK (0) or a negative hpf_status.  Nothing
+ *     aborts, nothing throws across this boundary.
+ *   - "d_" arguments are DEVICE pointers, "h_" arguments are HOST pointers,
+ *     everything else is host memory owned by the caller for the duration of
+ *     the call only.
+ *   - The library allocates no device memory (the one exception is stated at
+ *     its declaration): parameters, gradient buffers and the workspace belong
+ *     to the caller, as do the streams.
+ *   - Tensors are fp32, channels innermost: activations [n][h][w][c], conv
+ *     weights [c_out][r][s][c_in].
+ *   - The step calls (forward, backward, grad_average) only enqueue work.
+ *     hpf_loss and hpf_synchronize wait for it.
+ *   - There is no CPU fallback: without a CUDA device the step calls fail with
+ *     HPF_ERR_CUDA.
+ */
+#ifndef HPF_H_
+#define HPF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hpf_model hpf_model; /* opaque, host side */
+
+typedef enum {
+    HPF_OK = 0,
+    HPF_ERR_INVALID = -1,     /* null pointer, bad cut list, B % M != 0, malformed op list, shape mismatch */
+    HPF_ERR_UNSUPPORTED = -2, /* a shape no kernel covers (e.g. BN channels not a multiple of 4) */
+    HPF_ERR_STATE = -3,       /* call order: backward before forward, average before backward, not bound */
+    HPF_ERR_WORKSPACE = -4,   /* workspace too small or misaligned */
+    HPF_ERR_CUDA = -5,        /* a CUDA call failed; text via hpf_last_error */
+    HPF_ERR_TIMEOUT = -6      /* hpf_synchronize deadline passed, or a bounded device-side wait gave up */
+} hpf_status;
+
+typedef enum { HPF_OP_CONV = 1, HPF_OP_BNRELU = 2, HPF_OP_ADD = 3, HPF_OP_MAXPOOL = 4, HPF_OP_HEAD = 5 } hpf_op_kind;
+
+/* One entry of the layer list.
+ *   CONV    cross-correlation, zero padding, no bias: ksize x ksize, stride, pad; c_in -> c_out
+ *   BNRELU  training-mode batch norm over the micro-batch (biased variance) followed by ReLU; c_in == c_out
+ *   ADD     src0 + src1 (residual join)
+ *   MAXPOOL ksize x ksize window, stride, pad (padding never wins)
+ *   HEAD    mean over (h,w), fully connected to c_out classes, softmax cross-entropy, mean over the
+ *           micro-batch (Eq. 2 with the cross-entropy loss).  Must be the last op and only the last. */
+typedef struct {
+    int32_t kind;        /* hpf_op_kind */
+    int32_t src0, src1;  /* index of the producing op, -1 = the network input; src1 only for ADD, else -1 */
+    int32_t c_in, c_out;
+    int32_t ksize, stride, pad;
+    float eps;           /* BNRELU */
+} hpf_op;
+
+/* ---- model (host only; no CUDA call) -------------------------------------------------------------
+ * Section 5.1.  in_shape = {B, H, W, C}.  cuts = P-1 strictly increasing op indices in [1, n_ops-1];
+ * partition p owns ops [cuts[p-1], cuts[p]).  A cut may fall anywhere, also inside a residual block.
+ * n_microbatches = M must divide B (Section 5.3: between 1 and the batch size).
+ * Errors: HPF_ERR_INVALID for a malformed list / cuts / M; HPF_ERR_UNSUPPORTED for a shape outside
+ * the kernels' reach.  *out is set only on success; release it with hpf_model_destroy. */
+int hpf_model_create(const hpf_op *ops, int32_t n_ops, const int32_t in_shape[4], const int32_t *cuts,
+                     int32_t n_cuts, int32_t n_microbatches, hpf_model **out);
+int hpf_model_destroy(hpf_model *model);
+
+/* Options, to be set before hpf_workspace_bytes / hpf_bind.
+ *   HPF_OPT_GRAPH          1 (default): each phase is captured once into a CUDA graph and replayed;
+ *                          0: kernels are enqueued directly on the streams every call.
+ *   HPF_OPT_CONV_PATH      0 (default): tensor-core (tcgen05) convolution kernels wherever the shape
+ *                          allows, CUDA-core kernels for the rest (3-channel stem, odd channel counts);
+ *                          1: CUDA-core kernels everywhere (fp32 FMA; a cross-check, not a fallback).
+ *   HPF_OPT_SINGLE_STREAM  1: all stages on stream 0 (hazard check: results must equal the multi-stream run).
+ *   HPF_OPT_KEEP_MESSAGES  1: every partition copies what it receives across a cut (activations forward,
+ *                          partial errors backward) into message buffers readable with hpf_message_ptr. */
+typedef enum { HPF_OPT_GRAPH = 1, HPF_OPT_CONV_PATH = 2, HPF_OPT_SINGLE_STREAM = 3, HPF_OPT_KEEP_MESSAGES = 4 } hpf_option;
+int hpf_set_option(hpf_model *model, int32_t option, int32_t value);
+
+/* ---- integer bookkeeping (Section 5.1 lists, Section 5.3 pipelining) ----------------------------- */
+int hpf_num_ops(const hpf_model *model, int32_t *n_ops);
+int hpf_num_partitions(const hpf_model *model, int32_t *P);
+int hpf_num_params(const hpf_model *model, int64_t *G);
+/* Offsets (in floats) into the flat parameter / gradient vectors: ops in list order; CONV weights
+ * [c_out][r][s][c_in]; BNRELU gamma[C] then beta[C]; HEAD W[classes][C] then bias[classes]. */
+int hpf_param_layout(const hpf_model *model, int32_t op, int64_t *w_off, int64_t *w_cnt, int64_t *b_off, int64_t *b_cnt);
+int hpf_op_shape(const hpf_model *model, int32_t op, int32_t hwc[3]);
+int hpf_partition_of_op(const hpf_model *model, int32_t op, int32_t *p);
+int hpf_partition_range(const hpf_model *model, int32_t p, int32_t *first_op, int32_t *end_op);
+int hpf_microbatch_range(const hpf_model *model, int32_t m, int32_t *first, int32_t *end);
+/* The tensors crossing cut `cut` (0-based): produced before it, read at or after it (Section 5.3,
+ * Forward/Backward lists), ascending producer index. */
+int hpf_boundary_count(const hpf_model *model, int32_t cut, int32_t *n);
+int hpf_boundary_desc(const hpf_model *model, int32_t cut, int32_t i, int32_t *producer_op, int32_t shape[4] /* b,H,W,C */);
+/* Fill/drain pipeline: forward (p,m) runs at tick p+m, backward (p,m) at tick (P-1-p)+m. */
+int hpf_schedule_tick(const hpf_model *model, int32_t p, int32_t m, int32_t *fwd_tick, int32_t *bwd_tick);
+
+/* ---- device resources ---------------------------------------------------------------------------- */
+int hpf_workspace_bytes(const hpf_model *model, size_t *bytes);
+/* d_params [G], d_grad_slots [M][G] (slot m = dL_m/dtheta), d_grad_avg [G], d_workspace (256-byte
+ * aligned, >= hpf_workspace_bytes): all caller-owned device memory that must outlive the model.
+ * cuda_streams: n_streams >= P cudaStream_t handles (stage p runs on stream p; stream 0 is the one
+ * the phases fork from and join to).  Creates events and tensor-map descriptors; allocates nothing
+ * on the device.  Errors: HPF_ERR_WORKSPACE, HPF_ERR_INVALID, HPF_ERR_CUDA. */
+int hpf_bind(hpf_model *model, float *d_params, float *d_grad_slots, float *d_grad_avg, void *d_workspace,
+             size_t ws_bytes, void *const *cuda_streams, int32_t n_streams);
+
+/* ---- the step ------------------------------------------------------------------------------------ */
+/* Section 5.3 forward pass: every (partition p, micro-batch m) in pipeline order.  d_x [B][H][W][C]
+ * fp32, d_labels [B] int32 in [0, classes); both must already be valid for work ordered after
+ * stream 0's current tail, and stay valid until the backward work has finished. */
+int hpf_forward(hpf_model *model, const float *d_x, const int32_t *d_labels);
+/* Section 5.2 Eq. 5-7: reverse sweep, last partition first; writes slot m of d_grad_slots. */
+int hpf_backward(hpf_model *model);
+/* d_grad_avg = (sum over m ascending of slot m) / M  (Section 5.3: gradients accumulated/averaged). */
+int hpf_grad_average(hpf_model *model);
+/* Waits for the forward work; *h_loss = (1/M) sum_m L_m. */
+int hpf_loss(hpf_model *model, float *h_loss);
+/* The whole step from HOST buffers (pinned memory recommended): copies h_x / h_labels to the device,
+ * runs forward, backward and the average, copies the loss back and waits. */
+int hpf_step_host(hpf_model *model, const float *h_x, const int32_t *h_labels, float *h_loss);
+/* Waits (polling, timeout_ms <= 0: no limit) for all enqueued work; reports a sticky device-side
+ * error flag (bounded waits inside kernels) as HPF_ERR_TIMEOUT. */
+int hpf_synchronize(hpf_model *model, int32_t timeout_ms);
+
+/* ---- inspection for parity tests ----------------------------------------------------------------- */
+/* Output of op `op` for micro-batch m (want_grad = 0) or dL_m/d(output) (want_grad = 1) as left by the
+ * last step.  shape = {b, H, W, C}; the head's output is its logits {b,1,1,classes}. */
+int hpf_tensor_ptr(const hpf_model *model, int32_t op, int32_t m, int32_t want_grad, const float **d_ptr, int32_t shape[4]);
+/* With HPF_OPT_KEEP_MESSAGES: the i-th tensor received across `cut` for micro-batch m, forward
+ * (want_grad = 0: the activation) or backward (want_grad = 1: the partial error, i.e. the sum over
+ * the consumers at or after the cut, Eq. 7). */
+int hpf_message_ptr(const hpf_model *model, int32_t cut, int32_t i, int32_t m, int32_t want_grad, const float **d_ptr);
+/* Per-micro-batch losses L_m (device, M floats). */
+int hpf_loss_slots_ptr(const hpf_model *model, const float **d_ptr);
+/* Kernel launches (graph kernel nodes count as launches) issued by the step calls since bind. */
+int hpf_launch_count(const hpf_model *model, int64_t *n);
+/* How many convolution launch sites per phase use the tensor-core path / the CUDA-core path. */
+int hpf_conv_path_counts(const hpf_model *model, int64_t *n_tensor, int64_t *n_cuda_core);
+
+/* ---- single kernels on caller buffers (convolution sweep, memory-bound kernel benchmarks) --------
+ * All pointers are device pointers, `stream` is a cudaStream_t.  x [N][H][W][C], w [K][R][R][C],
+ * y/dy [N][P][Q][K] with P = (H+2*pad-R)/stride+1.  path: 0 = tensor cores when the shape allows
+ * (else HPF_ERR_UNSUPPORTED), 1 = CUDA cores.  d_scratch: caller-owned scratch of at least
+ * hpf_conv_scratch_bytes(); it is written by the call and holds nothing afterwards. */
+int hpf_conv_scratch_bytes(int32_t N, int32_t H, int32_t W, int32_t C, int32_t K, int32_t R, int32_t stride,
+                           int32_t pad, size_t *bytes);
+int hpf_conv_fwd(const float *d_x, const float *d_w, float *d_y, int32_t N, int32_t H, int32_t W, int32_t C,
+                 int32_t K, int32_t R, int32_t stride, int32_t pad, int32_t path, void *d_scratch, void *stream);
+/* d_wt: the weights rearranged for the data gradient, [C][R][R][K] with the taps rotated by 180 degrees,
+ * written by hpf_conv_dgrad_weights (K*R*R*C floats). */
+int hpf_conv_dgrad_weights(const float *d_w, float *d_wt, int32_t C, int32_t K, int32_t R, void *stream);
+int hpf_conv_dgrad(const float *d_dy, const float *d_w, const float *d_wt, float *d_dx, int32_t N, int32_t H,
+                   int32_t W, int32_t C, int32_t K, int32_t R, int32_t stride, int32_t pad, int32_t path,
+                   void *d_scratch, void *stream);
+int hpf_conv_wgrad(const float *d_x, const float *d_dy, float *d_dw, int32_t N, int32_t H, int32_t W, int32_t C,
+                   int32_t K, int32_t R, int32_t stride, int32_t pad, int32_t path, void *d_scratch, void *stream);
+/* Fused BN(training)+ReLU over x [rows][C]: d_stats receives mean[C] then 1/sqrt(var+eps)[C].
+ * d_scratch: at least hpf_bnrelu_scratch_bytes(rows, C). */
+int hpf_bnrelu_scratch_bytes(int64_t rows, int32_t C, size_t *bytes);
+int hpf_bnrelu_fwd(const float *d_x, const float *d_gamma, const float *d_beta, float eps, float *d_y,
+                   float *d_stats, int64_t rows, int32_t C, void *d_scratch, void *stream);
+/* dx (+= if accumulate) = BN+ReLU backward of dy; d_addend (may be NULL) is added to dx as well
+ * (the shortcut's gradient at a residual fan-out).  d_dgamma / d_dbeta [C] are overwritten. */
+int hpf_bnrelu_bwd(const float *d_x, const float *d_dy, const float *d_gamma, const float *d_beta,
+                   const float *d_stats, float *d_dx, const float *d_addend, int32_t accumulate,
+                   float *d_dgamma, float *d_dbeta, int64_t rows, int32_t C, void *d_scratch, void *stream);
+/* out[j] = (sum_{m ascending} slots[m][j]) / M */
+int hpf_grad_average_flat(const float *d_slots, float *d_out, int32_t M, int64_t G, void *stream);
+
+const char *hpf_strerror(int status);
+/* Text of the most recent failure on the calling thread (CUDA error string and call site). */
+const char *hpf_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HPF_H_ */

@@ -1,0 +1,62 @@
+// Internal launcher interface between the host scheduler and the CUDA kernels.
+// Every launcher only enqueues on `st`, returns the launch status and adds the
+// number of kernels it launched to *n_launch (if non-null).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+namespace hpf {
+
+struct ConvShape {
+    int N, H, W, C;      // input  [N][H][W][C]
+    int K, R, stride, pad;
+    int P, Q;            // output [N][P][Q][K]
+};
+inline ConvShape make_conv_shape(int N, int H, int W, int C, int K, int R, int stride, int pad)
+{
+    ConvShape s{N, H, W, C, K, R, stride, pad, (H + 2 * pad - R) / stride + 1, (W + 2 * pad - R) / stride + 1};
+    return s;
+}
+
+// Device-side status word shared by all kernels that have bounded waits.
+// 0 = fine; anything else = where a wait gave up (see conv_tc.cu).
+struct DeviceStatus { unsigned int code; unsigned int detail; };
+
+// ---------------- memory-bound kernels (kernels_mem.cu) ----------------
+size_t bn_scratch_bytes(int64_t rows, int C);
+// scratch: first 256 bytes hold the block ticket (must be zero before the first use; the kernels
+// leave it zero), the rest holds per-block partial sums.
+cudaError_t bnrelu_fwd(const float* x, const float* gamma, const float* beta, float eps, float* y, float* stats,
+                       int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch);
+cudaError_t bnrelu_bwd(const float* x, const float* dy, const float* gamma, const float* beta, const float* stats,
+                       float* dx, const float* addend, bool accumulate, float* dgamma, float* dbeta,
+                       int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch);
+cudaError_t add_fwd(const float* a, const float* b, float* out, int64_t n, cudaStream_t st, int64_t* n_launch);
+// dst (+)= src
+cudaError_t grad_accumulate(float* dst, const float* src, int64_t n, bool accumulate, cudaStream_t st, int64_t* n_launch);
+cudaError_t grad_average(const float* slots, float* out, int M, int64_t G, cudaStream_t st, int64_t* n_launch);
+cudaError_t loss_average(const float* loss_slots, float* out, int M, cudaStream_t st, int64_t* n_launch);
+cudaError_t maxpool_fwd(const float* x, float* y, ConvShape s, cudaStream_t st, int64_t* n_launch);
+cudaError_t maxpool_bwd(const float* x, const float* dy, float* dx, bool accumulate, ConvShape s, cudaStream_t st,
+                        int64_t* n_launch);
+// head: a [b][HW][C]; pooled scratch [b][C]; persample scratch [b]
+cudaError_t head_fwd(const float* a, const float* Wfc, const float* bias, const int32_t* labels, float* logits,
+                     float* pooled, float* persample, float* loss_slot, int b, int HW, int C, int ncls,
+                     cudaStream_t st, int64_t* n_launch);
+cudaError_t head_bwd(const float* Wfc, const int32_t* labels, const float* logits, const float* pooled,
+                     float* dlogits, float* da, float* dW, float* dbias, int b, int HW, int C, int ncls,
+                     cudaStream_t st, int64_t* n_launch);
+
+// ---------------- CUDA-core convolutions (conv_simt.cu) ----------------
+size_t conv_simt_scratch_bytes(const ConvShape& s);
+// y = conv(x, w) (+ residual)
+cudaError_t conv_fwd_simt(const float* x, const float* w, float* y, const float* residual, const ConvShape& s,
+                          cudaStream_t st, int64_t* n_launch);
+// dx (+= if accumulate) = dgrad(dy, w) (+ addend)
+cudaError_t conv_dgrad_simt(const float* dy, const float* w, float* dx, const float* addend, bool accumulate,
+                            const ConvShape& s, cudaStream_t st, int64_t* n_launch);
+cudaError_t conv_wgrad_simt(const float* x, const float* dy, float* dw, const ConvShape& s, void* scratch,
+                            cudaStream_t st, int64_t* n_launch);
+
+}  // namespace hpf

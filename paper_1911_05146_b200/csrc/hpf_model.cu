@@ -1,0 +1,1067 @@
+// Host side of the library: layer-list validation, partition / micro-batch bookkeeping, the memory
+// plan, the gradient-flow plan, the stream/event (or captured-graph) pipeline scheduler, and the C ABI.
+#include "../../include/hpf.h"
+#include "conv_tc.h"
+#include "hpf_kernels.h"
+
+#include <chrono>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <thread>
+#include <vector>
+
+using namespace hpf;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+int fail(int status, const char* what)
+{
+    g_last_error = what ? what : "";
+    return status;
+}
+
+int cuda_fail(cudaError_t e, const char* where)
+{
+    char buf[512];
+    snprintf(buf, sizeof buf, "%s: %s", where, cudaGetErrorString(e));
+    g_last_error = buf;
+    return HPF_ERR_CUDA;
+}
+
+#define CU(call)                                                   \
+    do {                                                           \
+        cudaError_t e__ = (call);                                  \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #call);      \
+    } while (0)
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+enum Phase { PH_FWD = 0, PH_BWD = 1, PH_AVG = 2, PH_COUNT = 3 };
+enum State { ST_CREATED = 0, ST_BOUND = 1, ST_FWD = 2, ST_BWD = 3 };
+
+struct OpInfo {
+    hpf_op op;
+    int H, W, C;            // output
+    int iH, iW, iC;         // input (src0)
+    int64_t w_off, w_cnt, b_off, b_cnt;
+    int part;
+    std::vector<int> consumers;   // ascending, with multiplicity
+};
+
+// How the backward of op `op` treats its contribution to one source tensor.
+struct GradEdge {
+    int accumulate = 0;     // the kernel adds to what the gradient buffer already holds
+    int addend = -1;        // tensor whose gradient buffer is added on the fly (a residual ADD's output)
+};
+struct AccumAction {        // explicit dst (+)= src over gradient buffers, run at op `at`'s place in the sweep
+    int at, dst, src, accumulate;
+};
+struct MessagePlan {        // how the partial error of a boundary tensor is assembled (debug messages)
+    int tensor;
+    int from_buffer;        // the tensor's own gradient buffer holds contributions of consumers >= cut
+    int pending;            // plus this ADD output's gradient (not folded yet), or -1
+};
+
+}  // namespace
+
+struct hpf_model {
+    std::vector<OpInfo> ops;
+    int n_ops = 0, B = 0, M = 0, b = 0, P = 1;
+    int inH = 0, inW = 0, inC = 0;
+    std::vector<int> cuts;                    // P-1
+    std::vector<int> part_lo, part_hi;        // P
+    std::vector<std::vector<int>> live;       // per cut
+    int64_t G = 0;
+    // options
+    int opt_graph = 1, opt_conv_path = 0, opt_single = 0, opt_messages = 0;
+    // gradient-flow plan
+    std::vector<int> grad_alias;              // tensor -> ADD op whose gradient buffer it shares, or -1
+    std::vector<GradEdge> edge0;              // per op: contribution to src0
+    std::vector<AccumAction> accums;
+    std::vector<std::vector<MessagePlan>> msg_plan;   // per cut
+    // memory plan (byte offsets into the workspace)
+    std::vector<size_t> act_off, grad_off, stats_off;   // [m * n_ops + op]
+    std::vector<size_t> bn_scratch_off, conv_scratch_off;   // per stream
+    std::vector<size_t> pooled_off, persample_off;      // per m
+    std::vector<std::vector<size_t>> fmsg_off, bmsg_off;  // [cut][i*M + m]
+    size_t loss_slots_off = 0, loss_avg_off = 0, wt_off = 0, stage_x_off = 0, stage_lab_off = 0, status_off = 0;
+    size_t zero_lo = 0, zero_hi = 0;          // region that must start zeroed (tickets, status)
+    size_t ws_bytes = 0;
+    bool planned = false;
+    // bound resources
+    float *params = nullptr, *gslots = nullptr, *gavg = nullptr;
+    char* ws = nullptr;
+    std::vector<cudaStream_t> streams;
+    std::vector<cudaEvent_t> ev_fwd, ev_bwd;  // [cut * M + m]
+    std::vector<cudaEvent_t> ev_join;         // per stream
+    cudaEvent_t ev_fork = nullptr, ev_sync = nullptr;
+    // tensor-core plans [m * n_ops + op] per pass
+    std::vector<ConvTcPlan> tc_plan[3];
+    std::vector<char> use_tc[3];              // per op
+    // graphs
+    struct FwdGraph { const float* x = nullptr; const int32_t* labels = nullptr; cudaGraphExec_t exec = nullptr; int64_t nodes = 0; };
+    FwdGraph fwd_graph[2];
+    int fwd_graph_next = 0;
+    cudaGraphExec_t graph[PH_COUNT] = {nullptr, nullptr, nullptr};
+    int64_t graph_nodes[PH_COUNT] = {0, 0, 0};
+    const float* cur_x = nullptr;
+    const int32_t* cur_labels = nullptr;
+    const int32_t* bwd_labels = nullptr;
+    const float* bwd_x = nullptr;
+    int state = ST_CREATED;
+    int64_t launches = 0;
+
+    float* act(int op, int m) const { return reinterpret_cast<float*>(ws + act_off[(size_t)m * n_ops + op]); }
+    float* grad(int op, int m) const { return reinterpret_cast<float*>(ws + grad_off[(size_t)m * n_ops + op]); }
+    float* stats(int op, int m) const { return reinterpret_cast<float*>(ws + stats_off[(size_t)m * n_ops + op]); }
+    int64_t numel(int op) const { const OpInfo& o = ops[op]; return (int64_t)b * o.H * o.W * o.C; }
+    cudaStream_t stream_of(int p) const { return opt_single ? streams[0] : streams[p]; }
+    DeviceStatus* status() const { return reinterpret_cast<DeviceStatus*>(ws + status_off); }
+};
+
+namespace {
+
+// ------------------------------------------------------------------------------------------------
+// validation + bookkeeping (Section 5.1)
+// ------------------------------------------------------------------------------------------------
+int build_ops(hpf_model* mdl, const hpf_op* ops, int n_ops)
+{
+    mdl->ops.resize(n_ops);
+    int64_t at = 0;
+    for (int i = 0; i < n_ops; ++i) {
+        OpInfo& o = mdl->ops[i];
+        o.op = ops[i];
+        const hpf_op& q = ops[i];
+        if (q.src0 < -1 || q.src0 >= i) return fail(HPF_ERR_INVALID, "op source must be an earlier op or -1");
+        if (q.src0 >= 0 && ops[q.src0].kind == HPF_OP_HEAD) return fail(HPF_ERR_INVALID, "the head has no output tensor to read");
+        if (q.src0 < 0) { o.iH = mdl->inH; o.iW = mdl->inW; o.iC = mdl->inC; }
+        else { o.iH = mdl->ops[q.src0].H; o.iW = mdl->ops[q.src0].W; o.iC = mdl->ops[q.src0].C; }
+        int64_t wc = 0, bc = 0;
+        switch (q.kind) {
+        case HPF_OP_CONV:
+        case HPF_OP_MAXPOOL:
+            if (q.c_in != o.iC || q.ksize < 1 || q.stride < 1 || q.pad < 0 || q.c_out < 1)
+                return fail(HPF_ERR_INVALID, "bad convolution / pooling geometry");
+            if (q.kind == HPF_OP_MAXPOOL && q.c_out != o.iC) return fail(HPF_ERR_INVALID, "pooling keeps the channel count");
+            if (o.iH + 2 * q.pad < q.ksize || o.iW + 2 * q.pad < q.ksize) return fail(HPF_ERR_INVALID, "window larger than the padded input");
+            if (q.pad >= q.ksize) return fail(HPF_ERR_UNSUPPORTED, "padding must be smaller than the window");
+            o.H = (o.iH + 2 * q.pad - q.ksize) / q.stride + 1;
+            o.W = (o.iW + 2 * q.pad - q.ksize) / q.stride + 1;
+            o.C = q.c_out;
+            if (q.kind == HPF_OP_CONV) wc = (int64_t)q.c_out * q.ksize * q.ksize * q.c_in;
+            break;
+        case HPF_OP_BNRELU:
+            if (q.c_in != o.iC || q.c_out != o.iC) return fail(HPF_ERR_INVALID, "BN channel count mismatch");
+            if (o.iC % 4) return fail(HPF_ERR_UNSUPPORTED, "BN channel count must be a multiple of 4");
+            if (q.src0 < 0) return fail(HPF_ERR_UNSUPPORTED, "BN directly on the network input");
+            if (!(q.eps > 0.f)) return fail(HPF_ERR_INVALID, "BN eps must be positive");
+            o.H = o.iH; o.W = o.iW; o.C = o.iC;
+            wc = bc = o.iC;
+            break;
+        case HPF_OP_ADD: {
+            if (q.src1 < 0 || q.src1 >= i || q.src0 < 0) return fail(HPF_ERR_INVALID, "ADD needs two earlier ops as sources");
+            if (ops[q.src1].kind == HPF_OP_HEAD) return fail(HPF_ERR_INVALID, "the head has no output tensor to read");
+            const OpInfo& t = mdl->ops[q.src1];
+            if (t.H != o.iH || t.W != o.iW || t.C != o.iC || q.c_out != o.iC) return fail(HPF_ERR_INVALID, "ADD shape mismatch");
+            o.H = o.iH; o.W = o.iW; o.C = o.iC;
+            break;
+        }
+        case HPF_OP_HEAD:
+            if (i != n_ops - 1) return fail(HPF_ERR_INVALID, "the head must be the last op");
+            if (q.c_in != o.iC || q.c_out < 1 || q.src0 < 0) return fail(HPF_ERR_INVALID, "bad head");
+            o.H = 1; o.W = 1; o.C = q.c_out;
+            wc = (int64_t)q.c_out * q.c_in; bc = q.c_out;
+            break;
+        default:
+            return fail(HPF_ERR_INVALID, "unknown op kind");
+        }
+        if (q.kind != HPF_OP_ADD && q.src1 != -1) return fail(HPF_ERR_INVALID, "src1 is only for ADD");
+        o.w_off = at; o.w_cnt = wc; at += wc;
+        o.b_off = at; o.b_cnt = bc; at += bc;
+        if (q.src0 >= 0) mdl->ops[q.src0].consumers.push_back(i);
+        if (q.kind == HPF_OP_ADD) mdl->ops[q.src1].consumers.push_back(i);
+    }
+    if (ops[n_ops - 1].kind != HPF_OP_HEAD) return fail(HPF_ERR_INVALID, "the last op must be the head");
+    for (int i = 0; i < n_ops - 1; ++i)
+        if (mdl->ops[i].consumers.empty()) return fail(HPF_ERR_INVALID, "an op's output is never read");
+    mdl->G = at;
+    return HPF_OK;
+}
+
+int build_partitions(hpf_model* mdl, const int32_t* cuts, int n_cuts)
+{
+    const int n = mdl->n_ops;
+    if (n_cuts < 0 || n_cuts > n - 1) return fail(HPF_ERR_INVALID, "more partitions than ops");
+    if (n_cuts > 0 && !cuts) return fail(HPF_ERR_INVALID, "null cut list");
+    for (int j = 0; j < n_cuts; ++j) {
+        if (cuts[j] < 1 || cuts[j] > n - 1) return fail(HPF_ERR_INVALID, "cut out of range");
+        if (j && cuts[j] <= cuts[j - 1]) return fail(HPF_ERR_INVALID, "cuts must be strictly increasing");
+    }
+    mdl->cuts.assign(cuts, cuts + n_cuts);
+    mdl->P = n_cuts + 1;
+    mdl->part_lo.resize(mdl->P); mdl->part_hi.resize(mdl->P);
+    for (int p = 0; p < mdl->P; ++p) {
+        mdl->part_lo[p] = p == 0 ? 0 : cuts[p - 1];
+        mdl->part_hi[p] = p == mdl->P - 1 ? n : cuts[p];
+        for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i) mdl->ops[i].part = p;
+    }
+    // only the first partition may read the network input
+    for (int i = mdl->part_hi[0]; i < n; ++i)
+        if (mdl->ops[i].op.src0 < 0) return fail(HPF_ERR_INVALID, "the network input is read beyond the first partition");
+    // live sets (Section 5.3: what crosses each cut)
+    mdl->live.assign(n_cuts, {});
+    for (int j = 0; j < n_cuts; ++j)
+        for (int t = 0; t < cuts[j]; ++t)
+            if (!mdl->ops[t].consumers.empty() && mdl->ops[t].consumers.back() >= cuts[j]) mdl->live[j].push_back(t);
+    return HPF_OK;
+}
+
+// Gradient flow: a tensor with several consumers sums their contributions in descending consumer
+// order (the order of the reverse sweep).  A residual ADD contributes its own output gradient
+// unchanged, so it costs no kernel: either the source simply shares the ADD's gradient buffer
+// (sole consumer), or the next consumer's kernel adds it on the fly.
+int build_grad_plan(hpf_model* mdl)
+{
+    const int n = mdl->n_ops;
+    mdl->grad_alias.assign(n, -1);
+    mdl->edge0.assign(n, GradEdge());
+    mdl->accums.clear();
+    for (int t = 0; t < n - 1; ++t) {
+        const std::vector<int>& cs = mdl->ops[t].consumers;
+        if (cs.size() == 1 && mdl->ops[cs[0]].op.kind == HPF_OP_ADD) mdl->grad_alias[t] = cs[0];
+    }
+    std::vector<char> written(n, 0);
+    std::vector<int> pending(n, -1);
+    for (int i = n - 1; i >= 0; --i) {
+        const hpf_op& q = mdl->ops[i].op;
+        const int srcs[2] = {q.src0, q.kind == HPF_OP_ADD ? q.src1 : -1};
+        for (int k = 0; k < 2; ++k) {
+            const int t = srcs[k];
+            if (t < 0) continue;
+            if (q.kind == HPF_OP_ADD) {
+                if (mdl->grad_alias[t] == i) continue;
+                bool lower_kernel = false;
+                for (int c : mdl->ops[t].consumers)
+                    if (c < i && mdl->ops[c].op.kind != HPF_OP_ADD && mdl->ops[c].op.kind != HPF_OP_HEAD &&
+                        mdl->ops[c].op.kind != HPF_OP_MAXPOOL) lower_kernel = true;
+                if (lower_kernel && pending[t] < 0) { pending[t] = i; continue; }
+                mdl->accums.push_back(AccumAction{i, t, i, written[t]});
+                written[t] = 1;
+            } else {
+                if (q.kind == HPF_OP_HEAD || q.kind == HPF_OP_MAXPOOL) {
+                    if (pending[t] >= 0) {      // these kernels take no addend: fold it first
+                        mdl->accums.push_back(AccumAction{i, t, pending[t], written[t]});
+                        written[t] = 1; pending[t] = -1;
+                    }
+                    if (q.kind == HPF_OP_HEAD && written[t]) return fail(HPF_ERR_UNSUPPORTED, "the head's input has a later consumer");
+                }
+                mdl->edge0[i].accumulate = written[t];
+                mdl->edge0[i].addend = pending[t];
+                written[t] = 1; pending[t] = -1;
+            }
+        }
+    }
+    // partial-error assembly per cut (for the optional message copies)
+    mdl->msg_plan.assign(mdl->cuts.size(), {});
+    for (size_t j = 0; j < mdl->cuts.size(); ++j) {
+        const int cut = mdl->cuts[j];
+        for (int t : mdl->live[j]) {
+            MessagePlan mp{t, 0, -1};
+            if (mdl->grad_alias[t] >= 0) { mp.from_buffer = 1; mdl->msg_plan[j].push_back(mp); continue; }
+            // replay the plan for consumers >= cut
+            int pend = -1;
+            std::vector<int> cs(mdl->ops[t].consumers.rbegin(), mdl->ops[t].consumers.rend());
+            for (int c : cs) {
+                if (c < cut) break;
+                const hpf_op& q = mdl->ops[c].op;
+                if (q.kind == HPF_OP_ADD) {
+                    bool explicit_acc = false;
+                    for (const AccumAction& a : mdl->accums) if (a.at == c && a.dst == t && a.src == c) explicit_acc = true;
+                    if (explicit_acc) mp.from_buffer = 1; else pend = c;
+                } else {
+                    mp.from_buffer = 1; pend = -1;   // the kernel folded any pending addend
+                }
+            }
+            mp.pending = pend;
+            mdl->msg_plan[j].push_back(mp);
+        }
+    }
+    return HPF_OK;
+}
+
+ConvShape conv_shape_of(const hpf_model* mdl, int i)
+{
+    const OpInfo& o = mdl->ops[i];
+    return make_conv_shape(mdl->b, o.iH, o.iW, o.iC, o.op.c_out, o.op.ksize, o.op.stride, o.op.pad);
+}
+
+// ------------------------------------------------------------------------------------------------
+// memory plan
+// ------------------------------------------------------------------------------------------------
+void build_memory_plan(hpf_model* mdl)
+{
+    const int n = mdl->n_ops, M = mdl->M, P = mdl->P;
+    size_t at = 0;
+    auto take = [&](size_t bytes) { size_t o = at; at = align_up(at + bytes, 256); return o; };
+    // region that must start as zeros: status word and BN tickets (with their partials)
+    mdl->zero_lo = at;
+    mdl->status_off = take(sizeof(DeviceStatus));
+    mdl->bn_scratch_off.assign(P, 0);
+    mdl->conv_scratch_off.assign(P, 0);
+    for (int p = 0; p < P; ++p) {
+        size_t bn = 256;
+        for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i)
+            if (mdl->ops[i].op.kind == HPF_OP_BNRELU) {
+                const OpInfo& o = mdl->ops[i];
+                size_t need = bn_scratch_bytes((int64_t)mdl->b * o.H * o.W, o.C);
+                if (need > bn) bn = need;
+            }
+        mdl->bn_scratch_off[p] = take(bn);
+    }
+    mdl->zero_hi = at;
+    for (int p = 0; p < P; ++p) {
+        size_t cv = 256;
+        for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i)
+            if (mdl->ops[i].op.kind == HPF_OP_CONV) {
+                const ConvShape s = conv_shape_of(mdl, i);
+                size_t need = conv_simt_scratch_bytes(s);
+                size_t need2 = conv_tc_scratch_bytes(s);
+                if (need2 > need) need = need2;
+                if (need > cv) cv = need;
+            }
+        mdl->conv_scratch_off[p] = take(cv);
+    }
+    mdl->loss_slots_off = take(sizeof(float) * M);
+    mdl->loss_avg_off = take(sizeof(float));
+    mdl->wt_off = take(sizeof(float) * (size_t)mdl->G);
+    mdl->stage_x_off = take(sizeof(float) * (size_t)mdl->B * mdl->inH * mdl->inW * mdl->inC);
+    mdl->stage_lab_off = take(sizeof(int32_t) * (size_t)mdl->B);
+    const int headC = mdl->ops[n - 1].op.c_in;
+    mdl->pooled_off.resize(M); mdl->persample_off.resize(M);
+    for (int m = 0; m < M; ++m) {
+        mdl->pooled_off[m] = take(sizeof(float) * (size_t)mdl->b * headC);
+        mdl->persample_off[m] = take(sizeof(float) * (size_t)mdl->b);
+    }
+    mdl->act_off.assign((size_t)n * M, 0); mdl->grad_off.assign((size_t)n * M, 0); mdl->stats_off.assign((size_t)n * M, 0);
+    for (int m = 0; m < M; ++m) {
+        for (int i = 0; i < n; ++i) mdl->act_off[(size_t)m * n + i] = take(sizeof(float) * (size_t)mdl->numel(i));
+        for (int i = n - 1; i >= 0; --i) {
+            const int a = mdl->grad_alias[i];
+            if (a >= 0) mdl->grad_off[(size_t)m * n + i] = mdl->grad_off[(size_t)m * n + a];   // a > i: already placed
+            else mdl->grad_off[(size_t)m * n + i] = take(sizeof(float) * (size_t)mdl->numel(i));
+        }
+        for (int i = 0; i < n; ++i)
+            if (mdl->ops[i].op.kind == HPF_OP_BNRELU) mdl->stats_off[(size_t)m * n + i] = take(sizeof(float) * 2 * (size_t)mdl->ops[i].C);
+    }
+    mdl->fmsg_off.assign(mdl->cuts.size(), {}); mdl->bmsg_off.assign(mdl->cuts.size(), {});
+    if (mdl->opt_messages)
+        for (size_t j = 0; j < mdl->cuts.size(); ++j) {
+            mdl->fmsg_off[j].resize(mdl->live[j].size() * M); mdl->bmsg_off[j].resize(mdl->live[j].size() * M);
+            for (size_t k = 0; k < mdl->live[j].size(); ++k)
+                for (int m = 0; m < M; ++m) {
+                    mdl->fmsg_off[j][k * M + m] = take(sizeof(float) * (size_t)mdl->numel(mdl->live[j][k]));
+                    mdl->bmsg_off[j][k * M + m] = take(sizeof(float) * (size_t)mdl->numel(mdl->live[j][k]));
+                }
+        }
+    mdl->ws_bytes = at;
+    mdl->planned = true;
+}
+
+bool op_uses_tc(const hpf_model* mdl, int i, int pass)
+{
+    if (mdl->opt_conv_path != 0) return false;
+    if (mdl->ops[i].op.kind != HPF_OP_CONV) return false;
+    return conv_tc_supported(conv_shape_of(mdl, i), pass);
+}
+
+// ------------------------------------------------------------------------------------------------
+// enqueue: the pipeline (Section 5.3)
+// ------------------------------------------------------------------------------------------------
+const float* src_act(const hpf_model* mdl, int src, int m)
+{
+    if (src < 0) return mdl->cur_x + (int64_t)m * mdl->b * mdl->inH * mdl->inW * mdl->inC;
+    return mdl->act(src, m);
+}
+
+int forward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
+{
+    const OpInfo& o = mdl->ops[i];
+    const hpf_op& q = o.op;
+    const float* in0 = src_act(mdl, q.src0, m);
+    float* out = mdl->act(i, m);
+    switch (q.kind) {
+    case HPF_OP_CONV: {
+        if (mdl->use_tc[PASS_FWD][i]) {
+            CU(conv_tc_launch(&mdl->tc_plan[PASS_FWD][(size_t)m * mdl->n_ops + i], mdl->status(), st, &mdl->launches));
+        } else {
+            CU(conv_fwd_simt(in0, mdl->params + o.w_off, out, nullptr, conv_shape_of(mdl, i), st, &mdl->launches));
+        }
+        break;
+    }
+    case HPF_OP_BNRELU:
+        CU(bnrelu_fwd(in0, mdl->params + o.w_off, mdl->params + o.b_off, q.eps, out, mdl->stats(i, m),
+                      (int64_t)mdl->b * o.H * o.W, o.C, mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
+        break;
+    case HPF_OP_ADD:
+        CU(add_fwd(in0, mdl->act(q.src1, m), out, mdl->numel(i), st, &mdl->launches));
+        break;
+    case HPF_OP_MAXPOOL:
+        CU(maxpool_fwd(in0, out, conv_shape_of(mdl, i), st, &mdl->launches));
+        break;
+    case HPF_OP_HEAD:
+        CU(head_fwd(in0, mdl->params + o.w_off, mdl->params + o.b_off, mdl->cur_labels + (int64_t)m * mdl->b, out,
+                    reinterpret_cast<float*>(mdl->ws + mdl->pooled_off[m]),
+                    reinterpret_cast<float*>(mdl->ws + mdl->persample_off[m]),
+                    reinterpret_cast<float*>(mdl->ws + mdl->loss_slots_off) + m, mdl->b, o.iH * o.iW, o.iC, q.c_out, st,
+                    &mdl->launches));
+        break;
+    }
+    return HPF_OK;
+}
+
+int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
+{
+    const OpInfo& o = mdl->ops[i];
+    const hpf_op& q = o.op;
+    const GradEdge& e = mdl->edge0[i];
+    // explicit accumulations scheduled at this op
+    for (const AccumAction& a : mdl->accums)
+        if (a.at == i) CU(grad_accumulate(mdl->grad(a.dst, m), mdl->grad(a.src, m), mdl->numel(a.dst), a.accumulate != 0, st, &mdl->launches));
+    const float* in0 = src_act(mdl, q.src0, m);
+    float* dout = mdl->grad(i, m);
+    float* slot = mdl->gslots + (int64_t)m * mdl->G;
+    const float* addend = e.addend >= 0 ? mdl->grad(e.addend, m) : nullptr;
+    switch (q.kind) {
+    case HPF_OP_CONV: {
+        const ConvShape s = conv_shape_of(mdl, i);
+        if (mdl->use_tc[PASS_WGRAD][i]) {
+            CU(conv_tc_launch(&mdl->tc_plan[PASS_WGRAD][(size_t)m * mdl->n_ops + i], mdl->status(), st, &mdl->launches));
+        } else {
+            CU(conv_wgrad_simt(in0, dout, slot + o.w_off, s, mdl->ws + mdl->conv_scratch_off[p], st, &mdl->launches));
+        }
+        if (q.src0 >= 0) {
+            if (mdl->use_tc[PASS_DGRAD][i]) {
+                CU(conv_tc_launch(&mdl->tc_plan[PASS_DGRAD][(size_t)m * mdl->n_ops + i], mdl->status(), st, &mdl->launches));
+            } else {
+                CU(conv_dgrad_simt(dout, mdl->params + o.w_off, mdl->grad(q.src0, m), addend, e.accumulate != 0, s, st, &mdl->launches));
+            }
+        }
+        break;
+    }
+    case HPF_OP_BNRELU:
+        CU(bnrelu_bwd(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m), addend,
+                      e.accumulate != 0, slot + o.w_off, slot + o.b_off, (int64_t)mdl->b * o.H * o.W, o.C,
+                      mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
+        break;
+    case HPF_OP_ADD:
+        break;   // its contributions are aliases, on-the-fly addends, or the explicit accumulations above
+    case HPF_OP_MAXPOOL:
+        if (q.src0 >= 0)
+            CU(maxpool_bwd(in0, dout, mdl->grad(q.src0, m), e.accumulate != 0, conv_shape_of(mdl, i), st, &mdl->launches));
+        break;
+    case HPF_OP_HEAD:
+        CU(head_bwd(mdl->params + o.w_off, mdl->cur_labels + (int64_t)m * mdl->b, mdl->act(i, m),
+                    reinterpret_cast<float*>(mdl->ws + mdl->pooled_off[m]), dout, mdl->grad(q.src0, m), slot + o.w_off,
+                    slot + o.b_off, mdl->b, o.iH * o.iW, o.iC, q.c_out, st, &mdl->launches));
+        break;
+    }
+    return HPF_OK;
+}
+
+int enqueue_phase(hpf_model* mdl, int phase)
+{
+    const int P = mdl->P, M = mdl->M;
+    cudaStream_t s0 = mdl->streams[0];
+    const bool multi = !mdl->opt_single && P > 1;
+    if (multi) {
+        CU(cudaEventRecord(mdl->ev_fork, s0));
+        for (int p = 1; p < P; ++p) CU(cudaStreamWaitEvent(mdl->streams[p], mdl->ev_fork, 0));
+    }
+    if (phase == PH_FWD) {
+        // tick t: every (p, m) with p + m = t
+        for (int t = 0; t < P + M - 1; ++t)
+            for (int p = 0; p < P; ++p) {
+                const int m = t - p;
+                if (m < 0 || m >= M) continue;
+                cudaStream_t st = mdl->stream_of(p);
+                if (p > 0) {
+                    if (multi) CU(cudaStreamWaitEvent(st, mdl->ev_fwd[(size_t)(p - 1) * M + m], 0));     // recv
+                    if (mdl->opt_messages)
+                        for (size_t k = 0; k < mdl->live[p - 1].size(); ++k)
+                            CU(grad_accumulate(reinterpret_cast<float*>(mdl->ws + mdl->fmsg_off[p - 1][k * M + m]),
+                                               mdl->act(mdl->live[p - 1][k], m), mdl->numel(mdl->live[p - 1][k]), false, st, &mdl->launches));
+                }
+                for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i) {
+                    int rc = forward_op(mdl, i, m, st, p);
+                    if (rc) return rc;
+                }
+                if (p < P - 1 && multi) CU(cudaEventRecord(mdl->ev_fwd[(size_t)p * M + m], st));          // send
+            }
+    } else if (phase == PH_BWD) {
+        // the data gradient of a tensor-core convolution reads rearranged weights: once per step
+        for (int p = 0; p < P; ++p)
+            for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i)
+                if (mdl->use_tc[PASS_DGRAD][i] && mdl->ops[i].op.src0 >= 0) {
+                    const OpInfo& o = mdl->ops[i];
+                    CU(conv_dgrad_weights(mdl->params + o.w_off, reinterpret_cast<float*>(mdl->ws + mdl->wt_off) + o.w_off,
+                                          o.op.c_in, o.op.c_out, o.op.ksize, mdl->stream_of(p), &mdl->launches));
+                }
+        for (int t = 0; t < P + M - 1; ++t)
+            for (int p = P - 1; p >= 0; --p) {
+                const int m = t - (P - 1 - p);
+                if (m < 0 || m >= M) continue;
+                cudaStream_t st = mdl->stream_of(p);
+                if (p < P - 1) {
+                    if (multi) CU(cudaStreamWaitEvent(st, mdl->ev_bwd[(size_t)p * M + m], 0));           // recv partial errors
+                    if (mdl->opt_messages)
+                        for (size_t k = 0; k < mdl->msg_plan[p].size(); ++k) {
+                            const MessagePlan& mp = mdl->msg_plan[p][k];
+                            float* dst = reinterpret_cast<float*>(mdl->ws + mdl->bmsg_off[p][k * M + m]);
+                            if (mp.from_buffer) CU(grad_accumulate(dst, mdl->grad(mp.tensor, m), mdl->numel(mp.tensor), false, st, &mdl->launches));
+                            if (mp.pending >= 0) CU(grad_accumulate(dst, mdl->grad(mp.pending, m), mdl->numel(mp.tensor), mp.from_buffer != 0, st, &mdl->launches));
+                        }
+                }
+                for (int i = mdl->part_hi[p] - 1; i >= mdl->part_lo[p]; --i) {
+                    int rc = backward_op(mdl, i, m, st, p);
+                    if (rc) return rc;
+                }
+                if (p > 0 && multi) CU(cudaEventRecord(mdl->ev_bwd[(size_t)(p - 1) * M + m], st));       // send partial errors
+            }
+    }
+    if (multi)
+        for (int p = 1; p < P; ++p) {
+            CU(cudaEventRecord(mdl->ev_join[p], mdl->streams[p]));
+            CU(cudaStreamWaitEvent(s0, mdl->ev_join[p], 0));
+        }
+    if (phase == PH_FWD)
+        CU(loss_average(reinterpret_cast<float*>(mdl->ws + mdl->loss_slots_off), reinterpret_cast<float*>(mdl->ws + mdl->loss_avg_off), M, s0, &mdl->launches));
+    if (phase == PH_AVG)
+        CU(grad_average(mdl->gslots, mdl->gavg, M, mdl->G, s0, &mdl->launches));
+    return HPF_OK;
+}
+
+int capture_phase(hpf_model* mdl, int phase, cudaGraphExec_t* exec, int64_t* nodes)
+{
+    cudaStream_t s0 = mdl->streams[0];
+    const int64_t before = mdl->launches;
+    CU(cudaStreamBeginCapture(s0, cudaStreamCaptureModeThreadLocal));
+    int rc = enqueue_phase(mdl, phase);
+    cudaGraph_t graph = nullptr;
+    cudaError_t e = cudaStreamEndCapture(s0, &graph);
+    *nodes = mdl->launches - before;
+    mdl->launches = before;
+    if (rc) { if (graph) cudaGraphDestroy(graph); return rc; }
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamEndCapture");
+    e = cudaGraphInstantiate(exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGraphInstantiate");
+    return HPF_OK;
+}
+
+int run_phase(hpf_model* mdl, int phase)
+{
+    if (!mdl->opt_graph) return enqueue_phase(mdl, phase);
+    cudaGraphExec_t exec = nullptr;
+    int64_t nodes = 0;
+    if (phase == PH_FWD) {
+        hpf_model::FwdGraph* slot = nullptr;
+        for (auto& g : mdl->fwd_graph)
+            if (g.exec && g.x == mdl->cur_x && g.labels == mdl->cur_labels) slot = &g;
+        if (!slot) {
+            slot = &mdl->fwd_graph[mdl->fwd_graph_next];
+            mdl->fwd_graph_next ^= 1;
+            if (slot->exec) { cudaGraphExecDestroy(slot->exec); slot->exec = nullptr; }
+            int rc = capture_phase(mdl, phase, &slot->exec, &slot->nodes);
+            if (rc) return rc;
+            slot->x = mdl->cur_x; slot->labels = mdl->cur_labels;
+        }
+        exec = slot->exec; nodes = slot->nodes;
+    } else {
+        if (phase == PH_BWD && mdl->graph[PH_BWD] && (mdl->bwd_labels != mdl->cur_labels || mdl->bwd_x != mdl->cur_x)) {
+            // the captured backward reads the input and the labels it was captured with
+            cudaGraphExecDestroy(mdl->graph[PH_BWD]); mdl->graph[PH_BWD] = nullptr;
+        }
+        if (!mdl->graph[phase]) {
+            int rc = capture_phase(mdl, phase, &mdl->graph[phase], &mdl->graph_nodes[phase]);
+            if (rc) return rc;
+            if (phase == PH_BWD) { mdl->bwd_labels = mdl->cur_labels; mdl->bwd_x = mdl->cur_x; }
+        }
+        exec = mdl->graph[phase]; nodes = mdl->graph_nodes[phase];
+    }
+    CU(cudaGraphLaunch(exec, mdl->streams[0]));
+    mdl->launches += nodes;
+    return HPF_OK;
+}
+
+void release_device_objects(hpf_model* mdl)
+{
+    for (auto& g : mdl->fwd_graph) if (g.exec) { cudaGraphExecDestroy(g.exec); g.exec = nullptr; }
+    for (auto& g : mdl->graph) if (g) { cudaGraphExecDestroy(g); g = nullptr; }
+    for (auto e : mdl->ev_fwd) cudaEventDestroy(e);
+    for (auto e : mdl->ev_bwd) cudaEventDestroy(e);
+    for (auto e : mdl->ev_join) if (e) cudaEventDestroy(e);
+    if (mdl->ev_fork) cudaEventDestroy(mdl->ev_fork);
+    if (mdl->ev_sync) cudaEventDestroy(mdl->ev_sync);
+    mdl->ev_fwd.clear(); mdl->ev_bwd.clear(); mdl->ev_join.clear();
+    mdl->ev_fork = mdl->ev_sync = nullptr;
+}
+
+}  // namespace
+
+// ================================================================================================
+// C ABI
+// ================================================================================================
+extern "C" {
+
+int hpf_model_create(const hpf_op* ops, int32_t n_ops, const int32_t in_shape[4], const int32_t* cuts, int32_t n_cuts,
+                     int32_t n_microbatches, hpf_model** out)
+{
+    if (!ops || !in_shape || !out) return fail(HPF_ERR_INVALID, "null argument");
+    if (n_ops < 1) return fail(HPF_ERR_INVALID, "empty op list");
+    for (int k = 0; k < 4; ++k) if (in_shape[k] < 1) return fail(HPF_ERR_INVALID, "bad input shape");
+    const int B = in_shape[0], M = n_microbatches;
+    if (M < 1 || M > B || B % M) return fail(HPF_ERR_INVALID, "the micro-batch count must divide the batch");
+    hpf_model* mdl = new hpf_model();
+    mdl->n_ops = n_ops; mdl->B = B; mdl->M = M; mdl->b = B / M;
+    mdl->inH = in_shape[1]; mdl->inW = in_shape[2]; mdl->inC = in_shape[3];
+    int rc = build_ops(mdl, ops, n_ops);
+    if (!rc) rc = build_partitions(mdl, cuts, n_cuts);
+    if (!rc) rc = build_grad_plan(mdl);
+    if (rc) { delete mdl; return rc; }
+    *out = mdl;
+    return HPF_OK;
+}
+
+int hpf_model_destroy(hpf_model* mdl)
+{
+    if (!mdl) return fail(HPF_ERR_INVALID, "null model");
+    release_device_objects(mdl);
+    delete mdl;
+    return HPF_OK;
+}
+
+int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
+{
+    if (!mdl) return fail(HPF_ERR_INVALID, "null model");
+    if (mdl->state != ST_CREATED) return fail(HPF_ERR_STATE, "options must be set before hpf_bind");
+    switch (option) {
+    case HPF_OPT_GRAPH: mdl->opt_graph = value != 0; break;
+    case HPF_OPT_CONV_PATH: if (value != 0 && value != 1) return fail(HPF_ERR_INVALID, "bad conv path"); mdl->opt_conv_path = value; break;
+    case HPF_OPT_SINGLE_STREAM: mdl->opt_single = value != 0; break;
+    case HPF_OPT_KEEP_MESSAGES: mdl->opt_messages = value != 0; break;
+    default: return fail(HPF_ERR_INVALID, "unknown option");
+    }
+    mdl->planned = false;
+    return HPF_OK;
+}
+
+int hpf_num_ops(const hpf_model* mdl, int32_t* n) { if (!mdl || !n) return fail(HPF_ERR_INVALID, "null"); *n = mdl->n_ops; return HPF_OK; }
+int hpf_num_partitions(const hpf_model* mdl, int32_t* P) { if (!mdl || !P) return fail(HPF_ERR_INVALID, "null"); *P = mdl->P; return HPF_OK; }
+int hpf_num_params(const hpf_model* mdl, int64_t* G) { if (!mdl || !G) return fail(HPF_ERR_INVALID, "null"); *G = mdl->G; return HPF_OK; }
+
+int hpf_param_layout(const hpf_model* mdl, int32_t op, int64_t* w_off, int64_t* w_cnt, int64_t* b_off, int64_t* b_cnt)
+{
+    if (!mdl || !w_off || !w_cnt || !b_off || !b_cnt) return fail(HPF_ERR_INVALID, "null");
+    if (op < 0 || op >= mdl->n_ops) return fail(HPF_ERR_INVALID, "op out of range");
+    const OpInfo& o = mdl->ops[op];
+    *w_off = o.w_off; *w_cnt = o.w_cnt; *b_off = o.b_off; *b_cnt = o.b_cnt;
+    return HPF_OK;
+}
+
+int hpf_op_shape(const hpf_model* mdl, int32_t op, int32_t hwc[3])
+{
+    if (!mdl || !hwc) return fail(HPF_ERR_INVALID, "null");
+    if (op < 0 || op >= mdl->n_ops) return fail(HPF_ERR_INVALID, "op out of range");
+    hwc[0] = mdl->ops[op].H; hwc[1] = mdl->ops[op].W; hwc[2] = mdl->ops[op].C;
+    return HPF_OK;
+}
+
+int hpf_partition_of_op(const hpf_model* mdl, int32_t op, int32_t* p)
+{
+    if (!mdl || !p) return fail(HPF_ERR_INVALID, "null");
+    if (op < 0 || op >= mdl->n_ops) return fail(HPF_ERR_INVALID, "op out of range");
+    *p = mdl->ops[op].part;
+    return HPF_OK;
+}
+
+int hpf_partition_range(const hpf_model* mdl, int32_t p, int32_t* first_op, int32_t* end_op)
+{
+    if (!mdl || !first_op || !end_op) return fail(HPF_ERR_INVALID, "null");
+    if (p < 0 || p >= mdl->P) return fail(HPF_ERR_INVALID, "partition out of range");
+    *first_op = mdl->part_lo[p]; *end_op = mdl->part_hi[p];
+    return HPF_OK;
+}
+
+int hpf_microbatch_range(const hpf_model* mdl, int32_t m, int32_t* first, int32_t* end)
+{
+    if (!mdl || !first || !end) return fail(HPF_ERR_INVALID, "null");
+    if (m < 0 || m >= mdl->M) return fail(HPF_ERR_INVALID, "micro-batch out of range");
+    *first = m * mdl->b; *end = (m + 1) * mdl->b;
+    return HPF_OK;
+}
+
+int hpf_boundary_count(const hpf_model* mdl, int32_t cut, int32_t* n)
+{
+    if (!mdl || !n) return fail(HPF_ERR_INVALID, "null");
+    if (cut < 0 || cut >= (int)mdl->cuts.size()) return fail(HPF_ERR_INVALID, "cut out of range");
+    *n = (int32_t)mdl->live[cut].size();
+    return HPF_OK;
+}
+
+int hpf_boundary_desc(const hpf_model* mdl, int32_t cut, int32_t i, int32_t* producer_op, int32_t shape[4])
+{
+    if (!mdl || !producer_op || !shape) return fail(HPF_ERR_INVALID, "null");
+    if (cut < 0 || cut >= (int)mdl->cuts.size()) return fail(HPF_ERR_INVALID, "cut out of range");
+    if (i < 0 || i >= (int)mdl->live[cut].size()) return fail(HPF_ERR_INVALID, "boundary tensor out of range");
+    const int t = mdl->live[cut][i];
+    *producer_op = t;
+    shape[0] = mdl->b; shape[1] = mdl->ops[t].H; shape[2] = mdl->ops[t].W; shape[3] = mdl->ops[t].C;
+    return HPF_OK;
+}
+
+int hpf_schedule_tick(const hpf_model* mdl, int32_t p, int32_t m, int32_t* fwd_tick, int32_t* bwd_tick)
+{
+    if (!mdl || !fwd_tick || !bwd_tick) return fail(HPF_ERR_INVALID, "null");
+    if (p < 0 || p >= mdl->P || m < 0 || m >= mdl->M) return fail(HPF_ERR_INVALID, "out of range");
+    *fwd_tick = p + m; *bwd_tick = (mdl->P - 1 - p) + m;
+    return HPF_OK;
+}
+
+int hpf_workspace_bytes(const hpf_model* mdl_c, size_t* bytes)
+{
+    if (!mdl_c || !bytes) return fail(HPF_ERR_INVALID, "null");
+    hpf_model* mdl = const_cast<hpf_model*>(mdl_c);
+    if (!mdl->planned) build_memory_plan(mdl);
+    *bytes = mdl->ws_bytes;
+    return HPF_OK;
+}
+
+int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad_avg, void* d_workspace, size_t ws_bytes,
+             void* const* cuda_streams, int32_t n_streams)
+{
+    if (!mdl || !d_params || !d_grad_slots || !d_grad_avg || !d_workspace || !cuda_streams) return fail(HPF_ERR_INVALID, "null argument");
+    if (mdl->state != ST_CREATED) return fail(HPF_ERR_STATE, "already bound");
+    if (n_streams < mdl->P) return fail(HPF_ERR_INVALID, "one stream per partition is required");
+    if (!mdl->planned) build_memory_plan(mdl);
+    if (ws_bytes < mdl->ws_bytes) return fail(HPF_ERR_WORKSPACE, "workspace too small");
+    if (reinterpret_cast<uintptr_t>(d_workspace) % 256) return fail(HPF_ERR_WORKSPACE, "workspace must be 256-byte aligned");
+    if (reinterpret_cast<uintptr_t>(d_params) % 16 || reinterpret_cast<uintptr_t>(d_grad_slots) % 16 ||
+        reinterpret_cast<uintptr_t>(d_grad_avg) % 16) return fail(HPF_ERR_INVALID, "parameter / gradient buffers must be 16-byte aligned");
+    int ndev = 0;
+    cudaError_t e = cudaGetDeviceCount(&ndev);
+    if (e != cudaSuccess || ndev < 1) { cudaGetLastError(); return cuda_fail(e != cudaSuccess ? e : cudaErrorNoDevice, "cudaGetDeviceCount"); }
+    mdl->params = d_params; mdl->gslots = d_grad_slots; mdl->gavg = d_grad_avg;
+    mdl->ws = reinterpret_cast<char*>(d_workspace);
+    mdl->streams.resize(mdl->P);
+    for (int p = 0; p < mdl->P; ++p) mdl->streams[p] = reinterpret_cast<cudaStream_t>(cuda_streams[p]);
+    const int M = mdl->M, n = mdl->n_ops;
+    CU(cudaEventCreateWithFlags(&mdl->ev_fork, cudaEventDisableTiming));
+    CU(cudaEventCreateWithFlags(&mdl->ev_sync, cudaEventDisableTiming));
+    mdl->ev_join.assign(mdl->P, nullptr);
+    for (int p = 1; p < mdl->P; ++p) CU(cudaEventCreateWithFlags(&mdl->ev_join[p], cudaEventDisableTiming));
+    mdl->ev_fwd.resize(mdl->cuts.size() * M); mdl->ev_bwd.resize(mdl->cuts.size() * M);
+    for (auto& ev : mdl->ev_fwd) CU(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+    for (auto& ev : mdl->ev_bwd) CU(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+    CU(cudaMemsetAsync(mdl->ws + mdl->zero_lo, 0, mdl->zero_hi - mdl->zero_lo, mdl->streams[0]));
+    // tensor-core plans
+    bool any_tc = false;
+    for (int pass = 0; pass < 3; ++pass) {
+        mdl->use_tc[pass].assign(n, 0);
+        for (int i = 0; i < n; ++i) if (op_uses_tc(mdl, i, pass)) { mdl->use_tc[pass][i] = 1; any_tc = true; }
+    }
+    if (any_tc) {
+        CU(conv_tc_init());
+        float* wt = reinterpret_cast<float*>(mdl->ws + mdl->wt_off);
+        for (int pass = 0; pass < 3; ++pass) {
+            mdl->tc_plan[pass].resize((size_t)n * M);
+            for (int m = 0; m < M; ++m)
+                for (int i = 0; i < n; ++i) {
+                    if (!mdl->use_tc[pass][i]) continue;
+                    const OpInfo& o = mdl->ops[i];
+                    const int src = o.op.src0;
+                    // the network input pointer is only known at hpf_forward: tensor-core kernels never read it
+                    if (src < 0) { mdl->use_tc[pass][i] = 0; continue; }
+                    const ConvShape s = conv_shape_of(mdl, i);
+                    const GradEdge& ed = mdl->edge0[i];
+                    ConvTcPlan* pl = &mdl->tc_plan[pass][(size_t)m * n + i];
+                    void* scratch = mdl->ws + mdl->conv_scratch_off[o.part];
+                    if (pass == PASS_FWD)
+                        CU(conv_tc_prepare(pl, s, pass, mdl->act(src, m), nullptr, mdl->params + o.w_off, mdl->act(i, m), nullptr, false, scratch));
+                    else if (pass == PASS_DGRAD)
+                        CU(conv_tc_prepare(pl, s, pass, mdl->grad(i, m), nullptr, wt + o.w_off, mdl->grad(src, m),
+                                           ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch));
+                    else
+                        CU(conv_tc_prepare(pl, s, pass, mdl->grad(i, m), mdl->act(src, m), nullptr,
+                                           mdl->gslots + (int64_t)m * mdl->G + o.w_off, nullptr, false, scratch));
+                }
+        }
+    }
+    CU(cudaStreamSynchronize(mdl->streams[0]));
+    mdl->state = ST_BOUND;
+    return HPF_OK;
+}
+
+int hpf_forward(hpf_model* mdl, const float* d_x, const int32_t* d_labels)
+{
+    if (!mdl || !d_x || !d_labels) return fail(HPF_ERR_INVALID, "null argument");
+    if (mdl->state < ST_BOUND) return fail(HPF_ERR_STATE, "hpf_bind first");
+    mdl->cur_x = d_x; mdl->cur_labels = d_labels;
+    int rc = run_phase(mdl, PH_FWD);
+    if (rc) return rc;
+    mdl->state = ST_FWD;
+    return HPF_OK;
+}
+
+int hpf_backward(hpf_model* mdl)
+{
+    if (!mdl) return fail(HPF_ERR_INVALID, "null model");
+    if (mdl->state != ST_FWD) return fail(HPF_ERR_STATE, "hpf_backward needs a fresh hpf_forward");
+    int rc = run_phase(mdl, PH_BWD);
+    if (rc) return rc;
+    mdl->state = ST_BWD;
+    return HPF_OK;
+}
+
+int hpf_grad_average(hpf_model* mdl)
+{
+    if (!mdl) return fail(HPF_ERR_INVALID, "null model");
+    if (mdl->state != ST_BWD) return fail(HPF_ERR_STATE, "hpf_grad_average needs hpf_backward");
+    return run_phase(mdl, PH_AVG);
+}
+
+int hpf_loss(hpf_model* mdl, float* h_loss)
+{
+    if (!mdl || !h_loss) return fail(HPF_ERR_INVALID, "null argument");
+    if (mdl->state < ST_FWD) return fail(HPF_ERR_STATE, "hpf_loss needs hpf_forward");
+    CU(cudaMemcpyAsync(h_loss, mdl->ws + mdl->loss_avg_off, sizeof(float), cudaMemcpyDeviceToHost, mdl->streams[0]));
+    CU(cudaStreamSynchronize(mdl->streams[0]));
+    return HPF_OK;
+}
+
+int hpf_step_host(hpf_model* mdl, const float* h_x, const int32_t* h_labels, float* h_loss)
+{
+    if (!mdl || !h_x || !h_labels || !h_loss) return fail(HPF_ERR_INVALID, "null argument");
+    if (mdl->state < ST_BOUND) return fail(HPF_ERR_STATE, "hpf_bind first");
+    cudaStream_t s0 = mdl->streams[0];
+    float* dx = reinterpret_cast<float*>(mdl->ws + mdl->stage_x_off);
+    int32_t* dl = reinterpret_cast<int32_t*>(mdl->ws + mdl->stage_lab_off);
+    CU(cudaMemcpyAsync(dx, h_x, sizeof(float) * (size_t)mdl->B * mdl->inH * mdl->inW * mdl->inC, cudaMemcpyHostToDevice, s0));
+    CU(cudaMemcpyAsync(dl, h_labels, sizeof(int32_t) * (size_t)mdl->B, cudaMemcpyHostToDevice, s0));
+    int rc = hpf_forward(mdl, dx, dl);
+    if (!rc) rc = hpf_backward(mdl);
+    if (!rc) rc = hpf_grad_average(mdl);
+    if (rc) return rc;
+    return hpf_loss(mdl, h_loss);
+}
+
+int hpf_synchronize(hpf_model* mdl, int32_t timeout_ms)
+{
+    if (!mdl) return fail(HPF_ERR_INVALID, "null model");
+    if (mdl->state < ST_BOUND) return fail(HPF_ERR_STATE, "hpf_bind first");
+    // every phase joins into stream 0, so its tail covers all stages
+    CU(cudaEventRecord(mdl->ev_sync, mdl->streams[0]));
+    const auto t0 = std::chrono::steady_clock::now();
+    for (;;) {
+        cudaError_t e = cudaEventQuery(mdl->ev_sync);
+        if (e == cudaSuccess) break;
+        if (e != cudaErrorNotReady) return cuda_fail(e, "cudaEventQuery");
+        if (timeout_ms > 0 &&
+            std::chrono::duration_cast<std::chrono::milliseconds>(std::chrono::steady_clock::now() - t0).count() > timeout_ms)
+            return fail(HPF_ERR_TIMEOUT, "hpf_synchronize: deadline passed");
+        std::this_thread::sleep_for(std::chrono::microseconds(50));
+    }
+    DeviceStatus hs{0, 0};
+    CU(cudaMemcpy(&hs, mdl->status(), sizeof hs, cudaMemcpyDeviceToHost));
+    if (hs.code) {
+        char buf[128];
+        snprintf(buf, sizeof buf, "a bounded device-side wait gave up (code %u, detail %u)", hs.code, hs.detail);
+        return fail(HPF_ERR_TIMEOUT, buf);
+    }
+    return HPF_OK;
+}
+
+int hpf_tensor_ptr(const hpf_model* mdl, int32_t op, int32_t m, int32_t want_grad, const float** d_ptr, int32_t shape[4])
+{
+    if (!mdl || !d_ptr || !shape) return fail(HPF_ERR_INVALID, "null");
+    if (mdl->state < ST_BOUND) return fail(HPF_ERR_STATE, "hpf_bind first");
+    if (op < 0 || op >= mdl->n_ops || m < 0 || m >= mdl->M) return fail(HPF_ERR_INVALID, "out of range");
+    *d_ptr = want_grad ? mdl->grad(op, m) : mdl->act(op, m);
+    shape[0] = mdl->b; shape[1] = mdl->ops[op].H; shape[2] = mdl->ops[op].W; shape[3] = mdl->ops[op].C;
+    return HPF_OK;
+}
+
+int hpf_message_ptr(const hpf_model* mdl, int32_t cut, int32_t i, int32_t m, int32_t want_grad, const float** d_ptr)
+{
+    if (!mdl || !d_ptr) return fail(HPF_ERR_INVALID, "null");
+    if (mdl->state < ST_BOUND || !mdl->opt_messages) return fail(HPF_ERR_STATE, "needs HPF_OPT_KEEP_MESSAGES and hpf_bind");
+    if (cut < 0 || cut >= (int)mdl->cuts.size() || m < 0 || m >= mdl->M || i < 0 || i >= (int)mdl->live[cut].size())
+        return fail(HPF_ERR_INVALID, "out of range");
+    const size_t off = want_grad ? mdl->bmsg_off[cut][(size_t)i * mdl->M + m] : mdl->fmsg_off[cut][(size_t)i * mdl->M + m];
+    *d_ptr = reinterpret_cast<const float*>(mdl->ws + off);
+    return HPF_OK;
+}
+
+int hpf_loss_slots_ptr(const hpf_model* mdl, const float** d_ptr)
+{
+    if (!mdl || !d_ptr) return fail(HPF_ERR_INVALID, "null");
+    if (mdl->state < ST_BOUND) return fail(HPF_ERR_STATE, "hpf_bind first");
+    *d_ptr = reinterpret_cast<const float*>(mdl->ws + mdl->loss_slots_off);
+    return HPF_OK;
+}
+
+int hpf_launch_count(const hpf_model* mdl, int64_t* n)
+{
+    if (!mdl || !n) return fail(HPF_ERR_INVALID, "null");
+    *n = mdl->launches;
+    return HPF_OK;
+}
+
+int hpf_conv_path_counts(const hpf_model* mdl, int64_t* n_tensor, int64_t* n_cuda_core)
+{
+    if (!mdl || !n_tensor || !n_cuda_core) return fail(HPF_ERR_INVALID, "null");
+    if (mdl->state < ST_BOUND) return fail(HPF_ERR_STATE, "hpf_bind first");
+    int64_t t = 0, c = 0;
+    for (int i = 0; i < mdl->n_ops; ++i) {
+        if (mdl->ops[i].op.kind != HPF_OP_CONV) continue;
+        for (int pass = 0; pass < 3; ++pass) {
+            if (pass == PASS_DGRAD && mdl->ops[i].op.src0 < 0) continue;
+            if (mdl->use_tc[pass][i]) ++t; else ++c;
+        }
+    }
+    *n_tensor = t; *n_cuda_core = c;
+    return HPF_OK;
+}
+
+// ---- single kernels -----------------------------------------------------------------------------
+static int check_conv_args(int32_t N, int32_t H, int32_t W, int32_t C, int32_t K, int32_t R, int32_t stride, int32_t pad)
+{
+    if (N < 1 || H < 1 || W < 1 || C < 1 || K < 1 || R < 1 || stride < 1 || pad < 0 || pad >= R) return fail(HPF_ERR_INVALID, "bad convolution geometry");
+    if (H + 2 * pad < R || W + 2 * pad < R) return fail(HPF_ERR_INVALID, "window larger than the padded input");
+    return HPF_OK;
+}
+
+int hpf_conv_scratch_bytes(int32_t N, int32_t H, int32_t W, int32_t C, int32_t K, int32_t R, int32_t stride, int32_t pad, size_t* bytes)
+{
+    if (!bytes) return fail(HPF_ERR_INVALID, "null");
+    int rc = check_conv_args(N, H, W, C, K, R, stride, pad);
+    if (rc) return rc;
+    const ConvShape s = make_conv_shape(N, H, W, C, K, R, stride, pad);
+    size_t a = conv_simt_scratch_bytes(s), b = conv_tc_scratch_bytes(s);
+    *bytes = align_up((a > b ? a : b) + 256, 256);
+    return HPF_OK;
+}
+
+static int conv_single(int pass, const float* in, const float* in2, const float* w, const float* wt, float* out,
+                       int32_t N, int32_t H, int32_t W, int32_t C, int32_t K, int32_t R, int32_t stride, int32_t pad,
+                       int32_t path, void* d_scratch, void* stream)
+{
+    int rc = check_conv_args(N, H, W, C, K, R, stride, pad);
+    if (rc) return rc;
+    if (!in || !out || !d_scratch) return fail(HPF_ERR_INVALID, "null argument");
+    const ConvShape s = make_conv_shape(N, H, W, C, K, R, stride, pad);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (path == 1) {
+        if (pass == PASS_FWD) CU(conv_fwd_simt(in, w, out, nullptr, s, st, nullptr));
+        else if (pass == PASS_DGRAD) CU(conv_dgrad_simt(in, w, out, nullptr, false, s, st, nullptr));
+        else CU(conv_wgrad_simt(in2, in, out, s, d_scratch, st, nullptr));
+        return HPF_OK;
+    }
+    if (path != 0) return fail(HPF_ERR_INVALID, "bad path");
+    if (!conv_tc_supported(s, pass)) return fail(HPF_ERR_UNSUPPORTED, "shape outside the tensor-core kernels' reach");
+    CU(conv_tc_init());
+    ConvTcPlan plan;
+    // the last 256 bytes of the scratch hold the device status word of this call
+    size_t sb = 0;
+    hpf_conv_scratch_bytes(N, H, W, C, K, R, stride, pad, &sb);
+    DeviceStatus* status = reinterpret_cast<DeviceStatus*>(reinterpret_cast<char*>(d_scratch) + sb - 256);
+    CU(cudaMemsetAsync(status, 0, sizeof(DeviceStatus), st));
+    CU(conv_tc_prepare(&plan, s, pass, in, in2, pass == PASS_DGRAD ? wt : w, out, nullptr, false, d_scratch));
+    CU(conv_tc_launch(&plan, status, st, nullptr));
+    return HPF_OK;
+}
+
+int hpf_conv_fwd(const float* d_x, const float* d_w, float* d_y, int32_t N, int32_t H, int32_t W, int32_t C, int32_t K,
+                 int32_t R, int32_t stride, int32_t pad, int32_t path, void* d_scratch, void* stream)
+{
+    if (!d_w) return fail(HPF_ERR_INVALID, "null argument");
+    return conv_single(PASS_FWD, d_x, nullptr, d_w, nullptr, d_y, N, H, W, C, K, R, stride, pad, path, d_scratch, stream);
+}
+
+int hpf_conv_dgrad_weights(const float* d_w, float* d_wt, int32_t C, int32_t K, int32_t R, void* stream)
+{
+    if (!d_w || !d_wt || C < 1 || K < 1 || R < 1) return fail(HPF_ERR_INVALID, "bad argument");
+    CU(conv_dgrad_weights(d_w, d_wt, C, K, R, reinterpret_cast<cudaStream_t>(stream), nullptr));
+    return HPF_OK;
+}
+
+int hpf_conv_dgrad(const float* d_dy, const float* d_w, const float* d_wt, float* d_dx, int32_t N, int32_t H, int32_t W,
+                   int32_t C, int32_t K, int32_t R, int32_t stride, int32_t pad, int32_t path, void* d_scratch, void* stream)
+{
+    if (!d_w || (path == 0 && !d_wt)) return fail(HPF_ERR_INVALID, "null argument");
+    return conv_single(PASS_DGRAD, d_dy, nullptr, d_w, d_wt, d_dx, N, H, W, C, K, R, stride, pad, path, d_scratch, stream);
+}
+
+int hpf_conv_wgrad(const float* d_x, const float* d_dy, float* d_dw, int32_t N, int32_t H, int32_t W, int32_t C, int32_t K,
+                   int32_t R, int32_t stride, int32_t pad, int32_t path, void* d_scratch, void* stream)
+{
+    if (!d_x) return fail(HPF_ERR_INVALID, "null argument");
+    return conv_single(PASS_WGRAD, d_dy, d_x, nullptr, nullptr, d_dw, N, H, W, C, K, R, stride, pad, path, d_scratch, stream);
+}
+
+int hpf_bnrelu_scratch_bytes(int64_t rows, int32_t C, size_t* bytes)
+{
+    if (!bytes || rows < 1 || C < 4 || C % 4) return fail(HPF_ERR_INVALID, "bad argument");
+    *bytes = align_up(bn_scratch_bytes(rows, C), 256);
+    return HPF_OK;
+}
+
+int hpf_bnrelu_fwd(const float* d_x, const float* d_gamma, const float* d_beta, float eps, float* d_y, float* d_stats,
+                   int64_t rows, int32_t C, void* d_scratch, void* stream)
+{
+    if (!d_x || !d_gamma || !d_beta || !d_y || !d_stats || !d_scratch) return fail(HPF_ERR_INVALID, "null argument");
+    if (rows < 1 || C < 4 || C % 4) return fail(HPF_ERR_UNSUPPORTED, "channel count must be a multiple of 4");
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    CU(cudaMemsetAsync(d_scratch, 0, 256, st));
+    CU(bnrelu_fwd(d_x, d_gamma, d_beta, eps, d_y, d_stats, rows, C, d_scratch, st, nullptr));
+    return HPF_OK;
+}
+
+int hpf_bnrelu_bwd(const float* d_x, const float* d_dy, const float* d_gamma, const float* d_beta, const float* d_stats,
+                   float* d_dx, const float* d_addend, int32_t accumulate, float* d_dgamma, float* d_dbeta, int64_t rows,
+                   int32_t C, void* d_scratch, void* stream)
+{
+    if (!d_x || !d_dy || !d_gamma || !d_beta || !d_stats || !d_dx || !d_dgamma || !d_dbeta || !d_scratch) return fail(HPF_ERR_INVALID, "null argument");
+    if (rows < 1 || C < 4 || C % 4) return fail(HPF_ERR_UNSUPPORTED, "channel count must be a multiple of 4");
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    CU(cudaMemsetAsync(d_scratch, 0, 256, st));
+    CU(bnrelu_bwd(d_x, d_dy, d_gamma, d_beta, d_stats, d_dx, d_addend, accumulate != 0, d_dgamma, d_dbeta, rows, C, d_scratch, st, nullptr));
+    return HPF_OK;
+}
+
+int hpf_grad_average_flat(const float* d_slots, float* d_out, int32_t M, int64_t G, void* stream)
+{
+    if (!d_slots || !d_out || M < 1 || G < 1) return fail(HPF_ERR_INVALID, "bad argument");
+    CU(grad_average(d_slots, d_out, M, G, reinterpret_cast<cudaStream_t>(stream), nullptr));
+    return HPF_OK;
+}
+
+const char* hpf_strerror(int status)
+{
+    switch (status) {
+    case HPF_OK: return "ok";
+    case HPF_ERR_INVALID: return "invalid argument";
+    case HPF_ERR_UNSUPPORTED: return "unsupported shape";
+    case HPF_ERR_STATE: return "call out of order";
+    case HPF_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case HPF_ERR_CUDA: return "CUDA error";
+    case HPF_ERR_TIMEOUT: return "timeout";
+    default: return "unknown status";
+    }
+}
+
+const char* hpf_last_error(void) { return g_last_error.c_str(); }
+
+}  // extern "C"

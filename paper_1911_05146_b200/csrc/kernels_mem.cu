@@ -1,0 +1,610 @@
+// Memory-bound kernels of the step: fused BN(training)+ReLU forward/backward, residual add,
+// gradient accumulate/average, max-pool and the pool+FC+softmax-CE head.  sm_100a.
+//
+// All tensors are fp32 with channels innermost.  Loads and stores are 128-bit and coalesced:
+// consecutive threads walk consecutive float4 of a row-major [rows][C] tensor.
+#include "hpf_kernels.h"
+
+#include <math.h>
+
+namespace hpf {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kMaxBlocks = 148 * 4;
+
+__host__ __device__ inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// ------------------------------------------------------------------------------------------------
+// BN + ReLU.  z = gamma * ((x - mean) * rstd) + beta, y = max(z, 0).  The same expression is used by
+// the forward and by the backward mask, so both take the ReLU decision on identical fp32 values.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float bn_xhat(float x, float mean, float rstd) { return (x - mean) * rstd; }
+__device__ __forceinline__ float bn_z(float xh, float g, float b) { return fmaf(g, xh, b); }
+
+struct BnPlan {
+    int cg_total;        // float4 column groups = C/4
+    int cgt;             // column groups handled per pass by one block (<= 256)
+    int rl;              // row lanes per block = 256 / cgt
+    int passes;          // ceil(cg_total / cgt)
+    int nblk;
+    int64_t rows_per_blk;
+};
+
+BnPlan bn_plan(int64_t rows, int C)
+{
+    BnPlan p;
+    p.cg_total = C / 4;
+    p.cgt = p.cg_total < kThreads ? p.cg_total : kThreads;
+    p.rl = kThreads / p.cgt;
+    p.passes = (p.cg_total + p.cgt - 1) / p.cgt;
+    int64_t nb = rows / ((int64_t)p.rl * 16);
+    if (nb < 1) nb = 1;
+    if (nb > kMaxBlocks) nb = kMaxBlocks;
+    p.rows_per_blk = ceil_div64(rows, nb);
+    p.nblk = (int)ceil_div64(rows, p.rows_per_blk);
+    return p;
+}
+
+// Per-channel reductions over the rows.
+//   forward  (BWD = false): a = sum (x - shift), b = sum (x - shift)^2 with shift = x[row 0][c]
+//                           -> mean, rstd = 1/sqrt(var + eps)      (shifted sums avoid cancellation)
+//   backward (BWD = true):  a = sum dz, b = sum dz * xhat, dz = dy * [z > 0]
+//                           -> dbeta, dgamma and the two per-row coefficients of the dx formula
+// Each block reduces its slab of rows, writes one partial per channel, and the block that takes the
+// last ticket adds the partials in ascending block order (fp64), so the result does not depend on
+// which block happens to finish last.
+template <bool BWD>
+__global__ void __launch_bounds__(kThreads)
+bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, const float* __restrict__ gamma,
+                 const float* __restrict__ beta, const float* __restrict__ stats, float eps, int64_t rows, int C,
+                 int cgt, int rl, int passes, int64_t rows_per_blk, unsigned int* ticket,
+                 float* __restrict__ partials, float* __restrict__ out_a, float* __restrict__ out_b,
+                 float* __restrict__ coef)
+{
+    __shared__ float sh[kThreads][8];
+    __shared__ int is_last;
+    const int t = threadIdx.x;
+    const int cg_total = C / 4;
+    const int my_rl = t / cgt, my_cg = t % cgt;
+    const int64_t r0 = (int64_t)blockIdx.x * rows_per_blk;
+    int64_t r1 = r0 + rows_per_blk;
+    if (r1 > rows) r1 = rows;
+    const float4* x4 = reinterpret_cast<const float4*>(x);
+    const float4* dy4 = reinterpret_cast<const float4*>(dy);
+
+    for (int pass = 0; pass < passes; ++pass) {
+        const int cg = pass * cgt + my_cg;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+        if (my_rl < rl && cg < cg_total) {
+            float4 p0, p1, gm, bt;
+            if (BWD) {
+                p0 = __ldg(reinterpret_cast<const float4*>(stats) + cg);              // mean
+                p1 = __ldg(reinterpret_cast<const float4*>(stats + C) + cg);          // rstd
+                gm = __ldg(reinterpret_cast<const float4*>(gamma) + cg);
+                bt = __ldg(reinterpret_cast<const float4*>(beta) + cg);
+            } else {
+                p0 = __ldg(x4 + cg);                                                  // shift = first row
+            }
+#pragma unroll 4
+            for (int64_t r = r0 + my_rl; r < r1; r += rl) {
+                const float4 v = __ldg(x4 + r * cg_total + cg);
+                if (BWD) {
+                    const float4 g = __ldg(dy4 + r * cg_total + cg);
+                    float xh, dz;
+                    xh = bn_xhat(v.x, p0.x, p1.x); dz = bn_z(xh, gm.x, bt.x) > 0.f ? g.x : 0.f; a.x += dz; b.x = fmaf(dz, xh, b.x);
+                    xh = bn_xhat(v.y, p0.y, p1.y); dz = bn_z(xh, gm.y, bt.y) > 0.f ? g.y : 0.f; a.y += dz; b.y = fmaf(dz, xh, b.y);
+                    xh = bn_xhat(v.z, p0.z, p1.z); dz = bn_z(xh, gm.z, bt.z) > 0.f ? g.z : 0.f; a.z += dz; b.z = fmaf(dz, xh, b.z);
+                    xh = bn_xhat(v.w, p0.w, p1.w); dz = bn_z(xh, gm.w, bt.w) > 0.f ? g.w : 0.f; a.w += dz; b.w = fmaf(dz, xh, b.w);
+                } else {
+                    float d;
+                    d = v.x - p0.x; a.x += d; b.x = fmaf(d, d, b.x);
+                    d = v.y - p0.y; a.y += d; b.y = fmaf(d, d, b.y);
+                    d = v.z - p0.z; a.z += d; b.z = fmaf(d, d, b.z);
+                    d = v.w - p0.w; a.w += d; b.w = fmaf(d, d, b.w);
+                }
+            }
+        }
+        sh[t][0] = a.x; sh[t][1] = a.y; sh[t][2] = a.z; sh[t][3] = a.w;
+        sh[t][4] = b.x; sh[t][5] = b.y; sh[t][6] = b.z; sh[t][7] = b.w;
+        __syncthreads();
+        // one output per (column group, component): add the row lanes in ascending order
+        for (int o = t; o < cgt * 8; o += kThreads) {
+            const int cgl = o >> 3, comp = o & 7;
+            const int cgo = pass * cgt + cgl;
+            if (cgo < cg_total) {
+                float s = 0.f;
+                for (int l = 0; l < rl; ++l) s += sh[l * cgt + cgl][comp];
+                const int c = cgo * 4 + (comp & 3);
+                partials[((int64_t)blockIdx.x * 2 + (comp >> 2)) * C + c] = s;
+            }
+        }
+        __syncthreads();
+    }
+
+    __threadfence();
+    __syncthreads();
+    if (t == 0) {
+        const unsigned int old = atomicAdd(ticket, 1u);
+        is_last = (old == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const double inv_rows = 1.0 / (double)rows;
+    for (int c = t; c < C; c += kThreads) {
+        double sa = 0.0, sb = 0.0;
+        for (unsigned int k = 0; k < gridDim.x; ++k) {
+            sa += (double)__ldcg(&partials[((int64_t)k * 2 + 0) * C + c]);
+            sb += (double)__ldcg(&partials[((int64_t)k * 2 + 1) * C + c]);
+        }
+        if (BWD) {
+            out_a[c] = (float)sa;                 // dbeta
+            out_b[c] = (float)sb;                 // dgamma
+            coef[c] = (float)(sa * inv_rows);
+            coef[C + c] = (float)(sb * inv_rows);
+        } else {
+            const double shift = (double)__ldg(x + c);
+            const double ms = sa * inv_rows;
+            double var = sb * inv_rows - ms * ms;
+            if (var < 0.0) var = 0.0;
+            out_a[c] = (float)(shift + ms);                       // mean
+            out_b[c] = (float)(1.0 / sqrt(var + (double)eps));    // rstd
+        }
+    }
+    if (t == 0) *ticket = 0u;
+}
+
+__global__ void __launch_bounds__(kThreads)
+bn_apply_fwd_kernel(const float4* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+                    const float* __restrict__ stats, float4* __restrict__ y, int64_t n4, int cg_total, int C)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        const int cg = (int)(i % cg_total);
+        const float4 v = __ldg(x + i);
+        const float4 mu = __ldg(reinterpret_cast<const float4*>(stats) + cg);
+        const float4 rs = __ldg(reinterpret_cast<const float4*>(stats + C) + cg);
+        const float4 g = __ldg(reinterpret_cast<const float4*>(gamma) + cg);
+        const float4 b = __ldg(reinterpret_cast<const float4*>(beta) + cg);
+        float4 o;
+        o.x = fmaxf(bn_z(bn_xhat(v.x, mu.x, rs.x), g.x, b.x), 0.f);
+        o.y = fmaxf(bn_z(bn_xhat(v.y, mu.y, rs.y), g.y, b.y), 0.f);
+        o.z = fmaxf(bn_z(bn_xhat(v.z, mu.z, rs.z), g.z, b.z), 0.f);
+        o.w = fmaxf(bn_z(bn_xhat(v.w, mu.w, rs.w), g.w, b.w), 0.f);
+        y[i] = o;
+    }
+}
+
+__device__ __forceinline__ float bn_dx1(float x, float dy, float mu, float rs, float g, float b, float ca, float cb)
+{
+    const float xh = bn_xhat(x, mu, rs);
+    const float dz = bn_z(xh, g, b) > 0.f ? dy : 0.f;
+    return g * rs * (dz - ca - xh * cb);
+}
+
+template <bool ADDEND, bool ACCUM>
+__global__ void __launch_bounds__(kThreads)
+bn_apply_bwd_kernel(const float4* __restrict__ x, const float4* __restrict__ dy, const float* __restrict__ gamma,
+                    const float* __restrict__ beta, const float* __restrict__ stats, const float* __restrict__ coef,
+                    const float4* __restrict__ addend, float4* __restrict__ dx, int64_t n4, int cg_total, int C)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        const int cg = (int)(i % cg_total);
+        const float4 v = __ldg(x + i);
+        const float4 d = __ldg(dy + i);
+        const float4 mu = __ldg(reinterpret_cast<const float4*>(stats) + cg);
+        const float4 rs = __ldg(reinterpret_cast<const float4*>(stats + C) + cg);
+        const float4 g = __ldg(reinterpret_cast<const float4*>(gamma) + cg);
+        const float4 b = __ldg(reinterpret_cast<const float4*>(beta) + cg);
+        const float4 ca = __ldcg(reinterpret_cast<const float4*>(coef) + cg);
+        const float4 cb = __ldcg(reinterpret_cast<const float4*>(coef + C) + cg);
+        float4 o;
+        o.x = bn_dx1(v.x, d.x, mu.x, rs.x, g.x, b.x, ca.x, cb.x);
+        o.y = bn_dx1(v.y, d.y, mu.y, rs.y, g.y, b.y, ca.y, cb.y);
+        o.z = bn_dx1(v.z, d.z, mu.z, rs.z, g.z, b.z, ca.z, cb.z);
+        o.w = bn_dx1(v.w, d.w, mu.w, rs.w, g.w, b.w, ca.w, cb.w);
+        if (ADDEND) { const float4 e = __ldg(addend + i); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+        if (ACCUM) { const float4 e = dx[i]; o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+        dx[i] = o;
+    }
+}
+
+int ew_blocks(int64_t n_items)
+{
+    int64_t nb = ceil_div64(n_items, kThreads);
+    if (nb > kMaxBlocks * 2) nb = kMaxBlocks * 2;
+    if (nb < 1) nb = 1;
+    return (int)nb;
+}
+
+// ------------------------------------------------------------------------------------------------
+// element-wise
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+add_kernel(const float* __restrict__ a, const float* __restrict__ b, float* __restrict__ out, int64_t n)
+{
+    const int64_t n4 = n / 4;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (int64_t i = t0; i < n4; i += stride) {
+        const float4 u = __ldg(reinterpret_cast<const float4*>(a) + i), v = __ldg(reinterpret_cast<const float4*>(b) + i);
+        reinterpret_cast<float4*>(out)[i] = make_float4(u.x + v.x, u.y + v.y, u.z + v.z, u.w + v.w);
+    }
+    for (int64_t i = n4 * 4 + t0; i < n; i += stride) out[i] = a[i] + b[i];
+}
+
+template <bool ACCUM>
+__global__ void __launch_bounds__(kThreads)
+accumulate_kernel(float* __restrict__ dst, const float* __restrict__ src, int64_t n)
+{
+    const int64_t n4 = n / 4;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (int64_t i = t0; i < n4; i += stride) {
+        float4 v = __ldg(reinterpret_cast<const float4*>(src) + i);
+        if (ACCUM) { const float4 e = reinterpret_cast<float4*>(dst)[i]; v.x += e.x; v.y += e.y; v.z += e.z; v.w += e.w; }
+        reinterpret_cast<float4*>(dst)[i] = v;
+    }
+    for (int64_t i = n4 * 4 + t0; i < n; i += stride) dst[i] = ACCUM ? dst[i] + src[i] : src[i];
+}
+
+// out[j] = (slots[0][j] + slots[1][j] + ... + slots[M-1][j]) / M, ascending m.  Reads M*G floats,
+// writes G: pure streaming, one float4 per slot per thread in flight.
+__global__ void __launch_bounds__(kThreads)
+grad_average_kernel(const float* __restrict__ slots, float* __restrict__ out, int M, int64_t G, float inv_m)
+{
+    const int64_t n4 = G / 4;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool vec = (G % 4 == 0);       // slot m starts at m*G floats: 16-byte aligned only then
+    if (vec) {
+        for (int64_t i = t0; i < n4; i += stride) {
+            float4 s = __ldcs(reinterpret_cast<const float4*>(slots) + i);
+            for (int m = 1; m < M; ++m) {
+                const float4 v = __ldcs(reinterpret_cast<const float4*>(slots + (int64_t)m * G) + i);
+                s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+            }
+            reinterpret_cast<float4*>(out)[i] = make_float4(s.x * inv_m, s.y * inv_m, s.z * inv_m, s.w * inv_m);
+        }
+    } else {
+        for (int64_t i = t0; i < G; i += stride) {
+            float s = slots[i];
+            for (int m = 1; m < M; ++m) s += slots[(int64_t)m * G + i];
+            out[i] = s * inv_m;
+        }
+    }
+}
+
+__global__ void loss_average_kernel(const float* __restrict__ loss_slots, float* __restrict__ out, int M)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        float s = 0.f;
+        for (int m = 0; m < M; ++m) s += loss_slots[m];
+        *out = s / (float)M;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// max-pool (only the 224x224 layout uses it)
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+maxpool_fwd_kernel(const float* __restrict__ x, float* __restrict__ y, ConvShape s)
+{
+    const int64_t total = (int64_t)s.N * s.P * s.Q * s.C;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int c = (int)(i % s.C);
+        int64_t r = i / s.C;
+        const int q = (int)(r % s.Q); r /= s.Q;
+        const int p = (int)(r % s.P);
+        const int n = (int)(r / s.P);
+        float best = -INFINITY;
+        for (int rr = 0; rr < s.R; ++rr) {
+            const int ih = p * s.stride + rr - s.pad;
+            if (ih < 0 || ih >= s.H) continue;
+            for (int ss = 0; ss < s.R; ++ss) {
+                const int iw = q * s.stride + ss - s.pad;
+                if (iw < 0 || iw >= s.W) continue;
+                best = fmaxf(best, __ldg(&x[(((int64_t)n * s.H + ih) * s.W + iw) * s.C + c]));
+            }
+        }
+        y[i] = best;
+    }
+}
+
+// Gather form (no atomics, fixed order): an input position receives dy of every window whose first
+// maximum (row-major window order) it is.
+template <bool ACCUM>
+__global__ void __launch_bounds__(kThreads)
+maxpool_bwd_kernel(const float* __restrict__ x, const float* __restrict__ dy, float* __restrict__ dx, ConvShape s)
+{
+    const int64_t total = (int64_t)s.N * s.H * s.W * s.C;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int c = (int)(i % s.C);
+        int64_t r = i / s.C;
+        const int w = (int)(r % s.W); r /= s.W;
+        const int h = (int)(r % s.H);
+        const int n = (int)(r / s.H);
+        const float mine = __ldg(&x[i]);
+        float acc = 0.f;
+        // windows (p,q) that contain (h,w): p*stride - pad <= h < p*stride - pad + R
+        int p_lo = h + s.pad - s.R + 1; p_lo = p_lo <= 0 ? 0 : (p_lo + s.stride - 1) / s.stride;
+        int p_hi = (h + s.pad) / s.stride; if (p_hi > s.P - 1) p_hi = s.P - 1;
+        int q_lo = w + s.pad - s.R + 1; q_lo = q_lo <= 0 ? 0 : (q_lo + s.stride - 1) / s.stride;
+        int q_hi = (w + s.pad) / s.stride; if (q_hi > s.Q - 1) q_hi = s.Q - 1;
+        for (int p = p_lo; p <= p_hi; ++p) {
+            const int h0 = p * s.stride - s.pad;
+            for (int q = q_lo; q <= q_hi; ++q) {
+                const int w0 = q * s.stride - s.pad;
+                bool first_max = true;
+                for (int rr = 0; rr < s.R && first_max; ++rr) {
+                    const int ih = h0 + rr;
+                    if (ih < 0 || ih >= s.H) continue;
+                    for (int ss = 0; ss < s.R; ++ss) {
+                        const int iw = w0 + ss;
+                        if (iw < 0 || iw >= s.W) continue;
+                        const float v = __ldg(&x[(((int64_t)n * s.H + ih) * s.W + iw) * s.C + c]);
+                        const bool before = (ih < h) || (ih == h && iw < w);
+                        if (v > mine || (before && v == mine)) { first_max = false; break; }
+                    }
+                }
+                if (first_max) acc += __ldg(&dy[(((int64_t)n * s.P + p) * s.Q + q) * s.C + c]);
+            }
+        }
+        dx[i] = ACCUM ? dx[i] + acc : acc;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// head: global average pool + FC + softmax cross-entropy
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ float block_reduce(float v, bool is_max, float* sh)
+{
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    v = is_max ? warp_max(v) : warp_sum(v);
+    __syncthreads();
+    if (lane == 0) sh[wid] = v;
+    __syncthreads();
+    float r = sh[0];
+    for (int k = 1; k < (int)(blockDim.x >> 5); ++k) r = is_max ? fmaxf(r, sh[k]) : r + sh[k];
+    return r;
+}
+
+// one block per sample; dynamic smem: C + ncls floats
+__global__ void __launch_bounds__(kThreads)
+head_fwd_kernel(const float* __restrict__ a, const float* __restrict__ Wfc, const float* __restrict__ bias,
+                const int32_t* __restrict__ labels, float* __restrict__ logits, float* __restrict__ pooled,
+                float* __restrict__ persample, int HW, int C, int ncls)
+{
+    extern __shared__ float smem[];
+    __shared__ float red[32];
+    float* sp = smem;            // pooled [C]
+    float* sl = smem + C;        // logits [ncls]
+    const int n = blockIdx.x, t = threadIdx.x;
+    const float inv = 1.f / (float)HW;
+    for (int c = t; c < C; c += blockDim.x) {
+        float s = 0.f;
+        for (int i = 0; i < HW; ++i) s += __ldg(&a[((int64_t)n * HW + i) * C + c]);
+        const float pv = s * inv;
+        sp[c] = pv;
+        pooled[(int64_t)n * C + c] = pv;
+    }
+    __syncthreads();
+    const int lane = t & 31, wid = t >> 5, nw = blockDim.x >> 5;
+    for (int j = wid; j < ncls; j += nw) {
+        float s = 0.f;
+        for (int c = lane; c < C; c += 32) s = fmaf(sp[c], __ldg(&Wfc[(int64_t)j * C + c]), s);
+        s = warp_sum(s);
+        if (lane == 0) { const float lg = s + __ldg(&bias[j]); sl[j] = lg; logits[(int64_t)n * ncls + j] = lg; }
+    }
+    __syncthreads();
+    float mx = -INFINITY;
+    for (int j = t; j < ncls; j += blockDim.x) mx = fmaxf(mx, sl[j]);
+    mx = block_reduce(mx, true, red);
+    float z = 0.f;
+    for (int j = t; j < ncls; j += blockDim.x) z += expf(sl[j] - mx);
+    z = block_reduce(z, false, red);
+    if (t == 0) persample[n] = -(sl[labels[n]] - mx - logf(z));
+}
+
+__global__ void head_loss_kernel(const float* __restrict__ persample, float* __restrict__ loss_slot, int b)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        float s = 0.f;
+        for (int n = 0; n < b; ++n) s += persample[n];
+        *loss_slot = s / (float)b;
+    }
+}
+
+// one block per sample: dlogits = (softmax - onehot)/b, da[n,i,c] = (dlogits . W[:,c]) / HW
+__global__ void __launch_bounds__(kThreads)
+head_bwd_data_kernel(const float* __restrict__ Wfc, const int32_t* __restrict__ labels, const float* __restrict__ logits,
+                     float* __restrict__ dlogits, float* __restrict__ da, int b, int HW, int C, int ncls)
+{
+    extern __shared__ float smem[];
+    __shared__ float red[32];
+    float* sd = smem;            // dlogits [ncls]
+    const int n = blockIdx.x, t = threadIdx.x;
+    float mx = -INFINITY;
+    for (int j = t; j < ncls; j += blockDim.x) mx = fmaxf(mx, __ldg(&logits[(int64_t)n * ncls + j]));
+    mx = block_reduce(mx, true, red);
+    float z = 0.f;
+    for (int j = t; j < ncls; j += blockDim.x) z += expf(__ldg(&logits[(int64_t)n * ncls + j]) - mx);
+    z = block_reduce(z, false, red);
+    const int lab = labels[n];
+    const float invb = 1.f / (float)b;
+    for (int j = t; j < ncls; j += blockDim.x) {
+        const float p = expf(__ldg(&logits[(int64_t)n * ncls + j]) - mx) / z;
+        const float d = (p - (j == lab ? 1.f : 0.f)) * invb;
+        sd[j] = d;
+        dlogits[(int64_t)n * ncls + j] = d;
+    }
+    __syncthreads();
+    const float inv = 1.f / (float)HW;
+    for (int c = t; c < C; c += blockDim.x) {
+        float s = 0.f;
+        for (int j = 0; j < ncls; ++j) s = fmaf(sd[j], __ldg(&Wfc[(int64_t)j * C + c]), s);
+        s *= inv;
+        for (int i = 0; i < HW; ++i) da[((int64_t)n * HW + i) * C + c] = s;
+    }
+}
+
+// one block per class: dW[j][c] = sum_n dlogits[n][j] * pooled[n][c] (ascending n), dbias[j] = sum_n dlogits[n][j]
+__global__ void __launch_bounds__(kThreads)
+head_bwd_param_kernel(const float* __restrict__ dlogits, const float* __restrict__ pooled, float* __restrict__ dW,
+                      float* __restrict__ dbias, int b, int C, int ncls)
+{
+    const int j = blockIdx.x, t = threadIdx.x;
+    for (int c = t; c < C; c += blockDim.x) {
+        float s = 0.f;
+        for (int n = 0; n < b; ++n) s = fmaf(__ldg(&dlogits[(int64_t)n * ncls + j]), __ldg(&pooled[(int64_t)n * C + c]), s);
+        dW[(int64_t)j * C + c] = s;
+    }
+    if (t == 0) {
+        float s = 0.f;
+        for (int n = 0; n < b; ++n) s += dlogits[(int64_t)n * ncls + j];
+        dbias[j] = s;
+    }
+}
+
+inline void count(int64_t* n_launch, int k) { if (n_launch) *n_launch += k; }
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+// launchers
+// ------------------------------------------------------------------------------------------------
+size_t bn_scratch_bytes(int64_t rows, int C)
+{
+    const BnPlan p = bn_plan(rows, C);
+    return 256 + ((size_t)p.nblk * 2 * C + 2 * (size_t)C) * sizeof(float);
+}
+
+cudaError_t bnrelu_fwd(const float* x, const float* gamma, const float* beta, float eps, float* y, float* stats,
+                       int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch)
+{
+    const BnPlan p = bn_plan(rows, C);
+    unsigned int* ticket = reinterpret_cast<unsigned int*>(scratch);
+    float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + 256);
+    bn_reduce_kernel<false><<<p.nblk, kThreads, 0, st>>>(x, nullptr, gamma, beta, nullptr, eps, rows, C, p.cgt, p.rl,
+                                                         p.passes, p.rows_per_blk, ticket, partials, stats, stats + C,
+                                                         nullptr);
+    const int64_t n4 = rows * (C / 4);
+    bn_apply_fwd_kernel<<<ew_blocks(n4), kThreads, 0, st>>>(reinterpret_cast<const float4*>(x), gamma, beta, stats,
+                                                            reinterpret_cast<float4*>(y), n4, C / 4, C);
+    count(n_launch, 2);
+    return cudaGetLastError();
+}
+
+cudaError_t bnrelu_bwd(const float* x, const float* dy, const float* gamma, const float* beta, const float* stats,
+                       float* dx, const float* addend, bool accumulate, float* dgamma, float* dbeta, int64_t rows,
+                       int C, void* scratch, cudaStream_t st, int64_t* n_launch)
+{
+    const BnPlan p = bn_plan(rows, C);
+    unsigned int* ticket = reinterpret_cast<unsigned int*>(scratch);
+    float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + 256);
+    float* coef = partials + (size_t)p.nblk * 2 * C;
+    bn_reduce_kernel<true><<<p.nblk, kThreads, 0, st>>>(x, dy, gamma, beta, stats, 0.f, rows, C, p.cgt, p.rl, p.passes,
+                                                        p.rows_per_blk, ticket, partials, dbeta, dgamma, coef);
+    const int64_t n4 = rows * (C / 4);
+    const int nb = ew_blocks(n4);
+    const float4* x4 = reinterpret_cast<const float4*>(x);
+    const float4* dy4 = reinterpret_cast<const float4*>(dy);
+    const float4* ad4 = reinterpret_cast<const float4*>(addend);
+    float4* dx4 = reinterpret_cast<float4*>(dx);
+    if (addend && accumulate)
+        bn_apply_bwd_kernel<true, true><<<nb, kThreads, 0, st>>>(x4, dy4, gamma, beta, stats, coef, ad4, dx4, n4, C / 4, C);
+    else if (addend)
+        bn_apply_bwd_kernel<true, false><<<nb, kThreads, 0, st>>>(x4, dy4, gamma, beta, stats, coef, ad4, dx4, n4, C / 4, C);
+    else if (accumulate)
+        bn_apply_bwd_kernel<false, true><<<nb, kThreads, 0, st>>>(x4, dy4, gamma, beta, stats, coef, ad4, dx4, n4, C / 4, C);
+    else
+        bn_apply_bwd_kernel<false, false><<<nb, kThreads, 0, st>>>(x4, dy4, gamma, beta, stats, coef, ad4, dx4, n4, C / 4, C);
+    count(n_launch, 2);
+    return cudaGetLastError();
+}
+
+cudaError_t add_fwd(const float* a, const float* b, float* out, int64_t n, cudaStream_t st, int64_t* n_launch)
+{
+    add_kernel<<<ew_blocks(n / 4 + 1), kThreads, 0, st>>>(a, b, out, n);
+    count(n_launch, 1);
+    return cudaGetLastError();
+}
+
+cudaError_t grad_accumulate(float* dst, const float* src, int64_t n, bool accumulate, cudaStream_t st, int64_t* n_launch)
+{
+    if (accumulate) accumulate_kernel<true><<<ew_blocks(n / 4 + 1), kThreads, 0, st>>>(dst, src, n);
+    else accumulate_kernel<false><<<ew_blocks(n / 4 + 1), kThreads, 0, st>>>(dst, src, n);
+    count(n_launch, 1);
+    return cudaGetLastError();
+}
+
+cudaError_t grad_average(const float* slots, float* out, int M, int64_t G, cudaStream_t st, int64_t* n_launch)
+{
+    grad_average_kernel<<<ew_blocks(G / 4 + 1), kThreads, 0, st>>>(slots, out, M, G, 1.f / (float)M);
+    count(n_launch, 1);
+    return cudaGetLastError();
+}
+
+cudaError_t loss_average(const float* loss_slots, float* out, int M, cudaStream_t st, int64_t* n_launch)
+{
+    loss_average_kernel<<<1, 32, 0, st>>>(loss_slots, out, M);
+    count(n_launch, 1);
+    return cudaGetLastError();
+}
+
+cudaError_t maxpool_fwd(const float* x, float* y, ConvShape s, cudaStream_t st, int64_t* n_launch)
+{
+    maxpool_fwd_kernel<<<ew_blocks((int64_t)s.N * s.P * s.Q * s.C), kThreads, 0, st>>>(x, y, s);
+    count(n_launch, 1);
+    return cudaGetLastError();
+}
+
+cudaError_t maxpool_bwd(const float* x, const float* dy, float* dx, bool accumulate, ConvShape s, cudaStream_t st,
+                        int64_t* n_launch)
+{
+    const int nb = ew_blocks((int64_t)s.N * s.H * s.W * s.C);
+    if (accumulate) maxpool_bwd_kernel<true><<<nb, kThreads, 0, st>>>(x, dy, dx, s);
+    else maxpool_bwd_kernel<false><<<nb, kThreads, 0, st>>>(x, dy, dx, s);
+    count(n_launch, 1);
+    return cudaGetLastError();
+}
+
+cudaError_t head_fwd(const float* a, const float* Wfc, const float* bias, const int32_t* labels, float* logits,
+                     float* pooled, float* persample, float* loss_slot, int b, int HW, int C, int ncls,
+                     cudaStream_t st, int64_t* n_launch)
+{
+    const size_t smem = (size_t)(C + ncls) * sizeof(float);
+    head_fwd_kernel<<<b, kThreads, smem, st>>>(a, Wfc, bias, labels, logits, pooled, persample, HW, C, ncls);
+    head_loss_kernel<<<1, 32, 0, st>>>(persample, loss_slot, b);
+    count(n_launch, 2);
+    return cudaGetLastError();
+}
+
+cudaError_t head_bwd(const float* Wfc, const int32_t* labels, const float* logits, const float* pooled,
+                     float* dlogits, float* da, float* dW, float* dbias, int b, int HW, int C, int ncls,
+                     cudaStream_t st, int64_t* n_launch)
+{
+    head_bwd_data_kernel<<<b, kThreads, (size_t)ncls * sizeof(float), st>>>(Wfc, labels, logits, dlogits, da, b, HW, C, ncls);
+    head_bwd_param_kernel<<<ncls, kThreads, 0, st>>>(dlogits, pooled, dW, dbias, b, C, ncls);
+    count(n_launch, 2);
+    return cudaGetLastError();
+}
+
+}  // namespace hpf

@@ -1,0 +1,53 @@
+"""Full-size configurations in the launch configuration the benchmark times: the whole step runs on
+the GPU, the oracle recomputes sampled micro-batches one by one."""
+import numpy as np
+import pytest
+
+import workloads as wl
+from oracle import reference as ora
+from hpf_testlib import Bound, rel_l2, seeded, TOL_TENSOR, TOL_LOSS
+
+pytestmark = pytest.mark.gpu
+
+
+def _fullsize(name, sample_m):
+    c = wl.config(name)
+    ops, hwc, B, M = c["ops"], c["in_hwc"], c["B"], c["M"]
+    x, labels, theta = seeded(ops, hwc, B)
+    bd = Bound(ops, hwc, B, M, c["cuts"], theta)
+    bd.upload(x, labels)
+    loss = bd.step()
+    b = B // M
+    slots = bd.slots.cpu().numpy()
+    offs, G = wl.param_offsets(ops)
+    losses = bd.loss_slots()
+    assert np.isfinite(slots).all()
+    worst = {"act": 0.0, "dact": 0.0, "g": 0.0}
+    for m in sample_m:
+        r = ora.microbatch(ops, hwc, theta, x[m * b:(m + 1) * b], labels[m * b:(m + 1) * b])
+        assert abs(losses[m] - r["loss"]) <= TOL_LOSS * abs(r["loss"])
+        for i in range(len(ops)):
+            e = rel_l2(bd.tensor(i, m), r["act"][i]); worst["act"] = max(worst["act"], e)
+            assert e <= TOL_TENSOR, ("act", i, m, e)
+            e = rel_l2(bd.tensor(i, m, grad=True), r["dact"][i]); worst["dact"] = max(worst["dact"], e)
+            assert e <= TOL_TENSOR, ("dact", i, m, e)
+        for i, (w_off, w_cnt, b_off, b_cnt) in enumerate(offs):
+            for off, cnt in ((w_off, w_cnt), (b_off, b_cnt)):
+                if cnt:
+                    e = rel_l2(slots[m, off:off + cnt], r["g"][off:off + cnt]); worst["g"] = max(worst["g"], e)
+                    assert e <= TOL_TENSOR, ("g", i, m, e)
+    # properties that hold at any size: the average is the fixed-order mean of the slots
+    acc = slots[0].copy()
+    for m in range(1, M):
+        acc += slots[m]
+    assert np.array_equal(bd.avg.cpu().numpy(), acc * np.float32(1.0 / M))
+    assert abs(loss - float(np.sum(losses.astype(np.float32)) / np.float32(M))) <= 1e-6 * abs(loss)
+    print(name, "worst rel-L2", worst)
+
+
+def test_config3_resnet110_batch128():
+    _fullsize("r110", sample_m=[0, 3])
+
+
+def test_config4_resnet1001_batch128():
+    _fullsize("r1001", sample_m=[7])

@@ -1,0 +1,131 @@
+"""Single kernels through the C ABI against the oracle: the convolution sweep shapes (forward, data
+gradient, weight gradient; tensor-core and CUDA-core paths), BN+ReLU forward/backward on ragged
+sizes, the gradient average."""
+import numpy as np
+import pytest
+import torch
+
+import paper_1911_05146_b200 as hpf
+import workloads as wl
+from oracle import reference as ora
+from hpf_testlib import rel_l2, TOL_TENSOR
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(DEV)
+
+
+def _conv_case(ks, st, ci, co, H, N, path, seed=0):
+    pad = 1 if ks == 3 else (3 if ks == 7 else 0)
+    rng = np.random.Generator(np.random.PCG64(1000 + seed))
+    x = rng.standard_normal((N, H, H, ci)).astype(np.float32)
+    w = (rng.standard_normal((co, ks, ks, ci)) * np.sqrt(2.0 / (ci * ks * ks))).astype(np.float32)
+    P = (H + 2 * pad - ks) // st + 1
+    dy = rng.standard_normal((N, P, P, co)).astype(np.float32)
+    dx_, dw_, dy_ = _dev(x), _dev(w), _dev(dy)
+    scratch = torch.zeros(hpf.conv_scratch_bytes(N, H, H, ci, co, ks, st, pad), dtype=torch.uint8, device=DEV)
+    y = torch.full((N, P, P, co), float("nan"), device=DEV)
+    gx = torch.full((N, H, H, ci), float("nan"), device=DEV)
+    gw = torch.full((co, ks, ks, ci), float("nan"), device=DEV)
+    wt = torch.empty_like(dw_)
+    args = (N, H, H, ci, co, ks, st, pad, path)
+    hpf.conv_fwd(dx_, dw_, y, *args, scratch)
+    hpf.conv_dgrad_weights(dw_, wt, ci, co, ks)
+    hpf.conv_dgrad(dy_, dw_, wt, gx, *args, scratch)
+    hpf.conv_wgrad(dx_, dy_, gw, *args, scratch)
+    torch.cuda.synchronize()
+    e_f = rel_l2(y.cpu().numpy(), ora.conv_fwd(x, w, st, pad))
+    e_d = rel_l2(gx.cpu().numpy(), ora.conv_dgrad(dy, w, x.shape, st, pad))
+    e_w = rel_l2(gw.cpu().numpy(), ora.conv_wgrad(x, dy, ks, st, pad))
+    return e_f, e_d, e_w
+
+
+@pytest.mark.parametrize("shape", wl.conv_sweep_shapes(), ids=lambda s: "k%d_s%d_%dto%d_at%d" % s)
+def test_conv_sweep_tensor_core_path(shape):
+    """Sweep shapes at batch 6 (spans several tiles and a ragged tail of the pixel tiling)."""
+    ks, st, ci, co, H = shape
+    try:
+        e = _conv_case(ks, st, ci, co, H, N=6, path=0)
+    except hpf.HpfError as err:
+        assert err.status == -2
+        pytest.fail("sweep shape not covered by the tensor-core kernels: %s" % (shape,))
+    assert max(e) <= TOL_TENSOR, e
+    assert max(e) > 1e-6 or True
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 16, 64, 32), (3, 1, 32, 32, 16), (1, 2, 128, 64, 16), (3, 1, 3, 16, 32),
+                                   (7, 2, 3, 64, 32), (3, 2, 5, 7, 9), (1, 1, 12, 20, 5)],
+                         ids=lambda s: "k%d_s%d_%dto%d_at%d" % s)
+def test_conv_cuda_core_path(shape):
+    ks, st, ci, co, H = shape
+    e = _conv_case(ks, st, ci, co, H, N=3, path=1)
+    assert max(e) <= 1e-5, e          # fp32 FMA: far inside the tolerance
+
+
+def test_conv_bad_arguments():
+    s = torch.zeros(1024, dtype=torch.uint8, device=DEV)
+    with pytest.raises(hpf.HpfError) as e:
+        hpf.conv_fwd(s, s, s, 1, 4, 4, 3, 8, 5, 1, 0, 1, s)      # window larger than the input
+    assert e.value.status == -1
+    with pytest.raises(hpf.HpfError) as e:
+        hpf.conv_fwd(s, s, s, 1, 8, 8, 3, 8, 3, 1, 1, 0, s)      # 3 channels: no tensor-core kernel
+    assert e.value.status == -2
+
+
+@pytest.mark.parametrize("rows,C", [(1, 4), (7, 12), (1000, 16), (4096 + 37, 64), (16384, 16), (1024, 256), (50, 2048)])
+def test_bnrelu_fwd_bwd(rows, C):
+    rng = np.random.Generator(np.random.PCG64(rows * 7 + C))
+    x = (rng.standard_normal((rows, C)) * 2 + 3).astype(np.float32)       # mean >> 0: the cancellation case
+    dy = rng.standard_normal((rows, C)).astype(np.float32)
+    gamma = (1 + 0.3 * rng.standard_normal(C)).astype(np.float32)
+    beta = (0.3 * rng.standard_normal(C)).astype(np.float32)
+    addend = rng.standard_normal((rows, C)).astype(np.float32)
+    eps = 1e-5
+    scratch = torch.zeros(hpf.bnrelu_scratch_bytes(rows, C), dtype=torch.uint8, device=DEV)
+    dx_, ddy, dg, db, dadd = _dev(x), _dev(dy), _dev(gamma), _dev(beta), _dev(addend)
+    y = torch.empty_like(dx_); stats = torch.empty(2 * C, device=DEV)
+    for _ in range(2):          # twice: the block ticket must be left clean
+        hpf.bnrelu_fwd(dx_, dg, db, eps, y, stats, rows, C, scratch)
+    torch.cuda.synchronize()
+    mean, var = ora.bn_stats(x)
+    if rows > 1:
+        assert rel_l2(stats[:C].cpu().numpy(), mean) <= 1e-5
+        assert rel_l2(stats[C:].cpu().numpy(), 1 / np.sqrt(var + eps)) <= 1e-4
+    y_ref = ora.bnrelu_fwd(x, gamma, beta, eps)
+    assert rel_l2(y.cpu().numpy(), y_ref) <= 1e-4
+    gx = torch.full_like(dx_, float("nan")); ggam = torch.empty(C, device=DEV); gbet = torch.empty(C, device=DEV)
+    hpf.bnrelu_bwd(dx_, ddy, dg, db, stats, gx, None, 0, ggam, gbet, rows, C, scratch)
+    torch.cuda.synchronize()
+    rx, rg, rb = ora.bnrelu_bwd(x, dy, gamma, beta, eps)
+    if rows > 8:
+        assert rel_l2(gx.cpu().numpy(), rx) <= 1e-3
+        assert rel_l2(ggam.cpu().numpy(), rg) <= 1e-3 and rel_l2(gbet.cpu().numpy(), rb) <= 1e-3
+    # accumulate + addend: dx_total = existing + dx + addend
+    base = gx.clone()
+    hpf.bnrelu_bwd(dx_, ddy, dg, db, stats, gx, dadd, 1, ggam, gbet, rows, C, scratch)
+    torch.cuda.synchronize()
+    assert torch.allclose(gx, base + base + dadd, rtol=1e-5, atol=1e-5)
+
+
+def test_bnrelu_rejects_odd_channels():
+    s = torch.zeros(4096, dtype=torch.uint8, device=DEV)
+    with pytest.raises(hpf.HpfError) as e:
+        hpf.bnrelu_fwd(s, s, s, 1e-5, s, s, 10, 6, s)
+    assert e.value.status == -2
+
+
+@pytest.mark.parametrize("M,G", [(1, 5), (3, 1023), (8, 4096 * 33 + 2), (4, 1 << 20)])
+def test_grad_average_flat(M, G):
+    rng = np.random.Generator(np.random.PCG64(M * 100 + 1))
+    slots = rng.standard_normal((M, G)).astype(np.float32)
+    d = _dev(slots); out = torch.empty(G, device=DEV)
+    hpf.grad_average_flat(d, out, M, G)
+    torch.cuda.synchronize()
+    acc = slots[0].copy()
+    for m in range(1, M):
+        acc += slots[m]
+    assert np.array_equal(out.cpu().numpy(), acc * np.float32(1.0 / M))      # fixed ascending order, bit-exact
+    assert rel_l2(out.cpu().numpy(), ora.grad_average(slots)) <= 1e-6

@@ -1,0 +1,161 @@
+"""Parity of the CUDA step against the fp64 oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import paper_1911_05146_b200 as hpf
+import workloads as wl
+from oracle import reference as ora
+from hpf_testlib import Bound, rel_l2, seeded, TOL_TENSOR, TOL_LOSS
+
+pytestmark = pytest.mark.gpu
+
+
+def check_step(ops, in_hwc, B, M, cuts, options=None, seed=0, bn_jitter=0.0, microbatches=None, tensors=True):
+    x, labels, theta = seeded(ops, in_hwc, B, seed, bn_jitter)
+    bd = Bound(ops, in_hwc, B, M, cuts, theta, options)
+    bd.upload(x, labels)
+    loss = bd.step()
+    ref = ora.step(ops, in_hwc, theta, x, labels, M, cuts=list(cuts))
+    assert abs(loss - ref["loss"]) <= TOL_LOSS * abs(ref["loss"]), (loss, ref["loss"])
+    assert np.allclose(bd.loss_slots(), ref["losses"], rtol=TOL_LOSS, atol=0)
+    slots = bd.slots.cpu().numpy()
+    avg = bd.avg.cpu().numpy()
+    assert np.isfinite(slots).all() and np.isfinite(avg).all()     # every parameter got a gradient
+    offs, G = wl.param_offsets(ops)
+    worst = 0.0
+    for i, (w_off, w_cnt, b_off, b_cnt) in enumerate(offs):
+        for off, cnt in ((w_off, w_cnt), (b_off, b_cnt)):
+            if cnt == 0:
+                continue
+            for m in range(M):
+                e = rel_l2(slots[m, off:off + cnt], ref["g_slots"][m, off:off + cnt])
+                worst = max(worst, e)
+                assert e <= TOL_TENSOR, ("slot", m, "op", i, e)
+            e = rel_l2(avg[off:off + cnt], ref["g_avg"][off:off + cnt])
+            assert e <= TOL_TENSOR, ("avg op", i, e)
+    # the average is exactly the fixed-order fp32 sum of the slots over M
+    acc = slots[0].copy()
+    for m in range(1, M):
+        acc += slots[m]
+    assert np.array_equal(avg, acc * np.float32(1.0 / M))
+    if tensors:
+        b = B // M
+        for m in (range(M) if microbatches is None else microbatches):
+            mb = ora.microbatch(ops, in_hwc, theta, x[m * b:(m + 1) * b], labels[m * b:(m + 1) * b])
+            for i in range(len(ops)):
+                e = rel_l2(bd.tensor(i, m), mb["act"][i]); worst = max(worst, e)
+                assert e <= TOL_TENSOR, ("act", i, m, e)
+                e = rel_l2(bd.tensor(i, m, grad=True), mb["dact"][i]); worst = max(worst, e)
+                assert e <= TOL_TENSOR, ("dact", i, m, e)
+    return bd, ref, worst
+
+
+@pytest.mark.parametrize("conv_path", [0, 1])
+@pytest.mark.parametrize("graph", [1, 0])
+def test_config1_resnet11(conv_path, graph):
+    c = wl.config("r11")
+    check_step(c["ops"], c["in_hwc"], c["B"], c["M"], c["cuts"],
+               {hpf.OPT_CONV_PATH: conv_path, hpf.OPT_GRAPH: graph})
+
+
+@pytest.mark.parametrize("cuts", [[], [4], [3, 7, 8], [1, 5, 12, 25]])
+def test_mid_block_cuts_and_jittered_bn(cuts):
+    ops = wl.resnet_v2_cifar(1)
+    check_step(ops, (32, 32, 3), 4, 2, cuts, seed=3, bn_jitter=0.3)
+
+
+def test_odd_widths_run_on_cuda_cores():
+    ops = wl.resnet_v2_cifar(1, widths=(4, 8, 12), n_classes=5)
+    bd, _, _ = check_step(ops, (8, 8, 3), 6, 3, [9], seed=1, bn_jitter=0.2)
+    n_tc, n_cc = bd.model.conv_path_counts()
+    assert n_tc == 0 and n_cc > 0
+
+
+def test_imagenet_layout_small_with_maxpool():
+    ops = wl.resnet_v2_imagenet(blocks=(1, 1), widths=(16, 32), n_classes=7)
+    check_step(ops, (32, 32, 3), 4, 2, [2, 11], seed=2, bn_jitter=0.2)
+
+
+def test_second_step_and_new_inputs_reuse_the_model():
+    c = wl.config("r11")
+    ops = c["ops"]
+    x, labels, theta = seeded(ops, c["in_hwc"], c["B"])
+    bd = Bound(ops, c["in_hwc"], c["B"], c["M"], c["cuts"], theta)
+    bd.upload(x, labels)
+    l1 = bd.step(); s1 = bd.slots.clone()
+    l2 = bd.step()
+    assert l1 == l2 and torch.equal(s1, bd.slots)          # same inputs -> bit-identical, nothing left over
+    x2, labels2, _ = seeded(ops, c["in_hwc"], c["B"], seed=5)
+    bd.upload(x2, labels2)                                   # new device buffers -> the phases are re-captured
+    l3 = bd.step()
+    ref = ora.step(ops, c["in_hwc"], theta, x2, labels2, c["M"], cuts=c["cuts"])
+    assert abs(l3 - ref["loss"]) <= TOL_LOSS * abs(ref["loss"])
+    assert rel_l2(bd.avg.cpu().numpy(), ref["g_avg"]) <= TOL_TENSOR
+    # the host-buffer entry point gives the same numbers
+    hx = torch.from_numpy(x2).pin_memory(); hl = torch.from_numpy(labels2).pin_memory()
+    l4 = bd.model.step_host(hx, hl)
+    bd.model.synchronize(60000)
+    assert l4 == l3
+    assert rel_l2(bd.avg.cpu().numpy(), ref["g_avg"]) <= TOL_TENSOR
+
+
+def test_single_stream_equals_multi_stream_bitwise():
+    """Stream-hazard check: a missing event would show up as a difference."""
+    ops = wl.resnet_v2_cifar(2)
+    x, labels, theta = seeded(ops, (32, 32, 3), 8, seed=4)
+    cuts = wl.default_cuts(len(ops), 4)
+    outs = []
+    for single in (0, 1):
+        bd = Bound(ops, (32, 32, 3), 8, 4, cuts, theta, {hpf.OPT_SINGLE_STREAM: single})
+        bd.upload(x, labels)
+        loss = bd.step()
+        outs.append((loss, bd.slots.clone(), bd.avg.clone()))
+    assert outs[0][0] == outs[1][0]
+    assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
+
+
+def test_messages_across_cuts_match_the_oracle():
+    """Activations sent forward and partial errors sent back (Eq. 7) per cut and micro-batch."""
+    ops = wl.resnet_v2_cifar(1)
+    cuts = [4, 8, 12]          # mid-block, block edge, mid-block
+    B, M = 4, 2
+    x, labels, theta = seeded(ops, (32, 32, 3), B, seed=6, bn_jitter=0.2)
+    bd = Bound(ops, (32, 32, 3), B, M, cuts, theta, {hpf.OPT_KEEP_MESSAGES: 1})
+    bd.upload(x, labels)
+    bd.step()
+    b = B // M
+    for m in range(M):
+        r = ora.microbatch(ops, (32, 32, 3), theta, x[m * b:(m + 1) * b], labels[m * b:(m + 1) * b], cuts=cuts)
+        for (j, k), msg in r["fwd_msg"].items():
+            assert rel_l2(bd.message(j, k, m), msg) <= TOL_TENSOR, ("fwd", j, k, m)
+        for (j, k), msg in r["bwd_msg"].items():
+            assert rel_l2(bd.message(j, k, m, grad=True), msg) <= TOL_TENSOR, ("bwd", j, k, m)
+
+
+def test_state_machine_on_a_bound_model():
+    c = wl.config("r11")
+    x, labels, theta = seeded(c["ops"], c["in_hwc"], c["B"])
+    bd = Bound(c["ops"], c["in_hwc"], c["B"], c["M"], c["cuts"], theta)
+    bd.upload(x, labels)
+    for call in (bd.model.backward, bd.model.grad_average):
+        with pytest.raises(hpf.HpfError) as e:
+            call()
+        assert e.value.status == -3
+    bd.model.forward(bd.x, bd.labels)
+    with pytest.raises(hpf.HpfError):
+        bd.model.grad_average()
+    bd.model.backward()
+    with pytest.raises(hpf.HpfError):
+        bd.model.backward()
+    bd.model.grad_average()
+    bd.model.synchronize(60000)
+    with pytest.raises(hpf.HpfError) as e:
+        bd.model.set_option(hpf.OPT_GRAPH, 0)
+    assert e.value.status == -3
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    m2 = hpf.Model(c["ops"], (c["B"],) + c["in_hwc"], c["cuts"], c["M"])
+    with pytest.raises(hpf.HpfError) as e:
+        m2.bind(bd.params, bd.slots, bd.avg, small, bd.streams)
+    assert e.value.status == -4
+    assert bd.model.launch_count() > 0
