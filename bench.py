@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the partitioned, micro-batch pipelined training step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload r1001|r110|r11|r152] [--impl reference]
+
+One step = forward + backward + gradient average of the whole batch (all partitions, all
+micro-batches).  Prints ONE JSON line.  N > 1 (under torchrun) runs N independent replicas, one per
+GPU, with no data-path collective (weak scaling); the timing is the max over ranks.
+`--impl reference` times the fp64 CPU oracle on the host cores instead (rank 0 only).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "images/sec fwd+bwd (1 B200) ResNet-1001 v2 32x32 b128; conv tensor-pipe % of peak"
+UNIT = "images/s"
+NAMES = {"r1001": "ResNet-1001 v2 (n=111, widths 16/32/64 x4), 32x32x3, batch 128, 8 partitions x 8 micro-batches",
+         "r110": "ResNet-110 v2 (n=12), 32x32x3, batch 128, 4 partitions x 4 micro-batches",
+         "r11": "ResNet-11 v2 (n=1), 32x32x3, batch 8, 2 partitions x 2 micro-batches",
+         "r152": "ResNet-152 v2 ImageNet layout, 224x224x3, batch 64, 4 partitions x 4 micro-batches"}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"], bf16_tflops_sustained=p.get("bf16_tflops_sustained"),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ----------------------------------------------------------------------------------------------------
+# algorithmic byte / flop model of one step (unfused op model: every op reads its inputs and writes
+# its outputs once; conv counted for forward, data gradient and weight gradient)
+# ----------------------------------------------------------------------------------------------------
+def step_model(ops, in_hwc, B):
+    shapes = wl.tensor_shapes(ops, in_hwc)
+    by = dict(conv=0.0, bn=0.0, add=0.0, other=0.0)
+    flops = 0.0
+    for i, o in enumerate(ops):
+        H, W, C = shapes[i]
+        iH, iW, iC = in_hwc if o.src0 < 0 else shapes[o.src0]
+        out_el = B * H * W * C
+        if o.kind == wl.CONV:
+            in_el = B * H * W * iC if o.stride > 1 else B * iH * iW * iC     # only the sampled pixels of a strided 1x1
+            wts = o.c_out * o.ksize * o.ksize * o.c_in
+            passes = 3 if o.src0 >= 0 else 2
+            by["conv"] += 4.0 * (in_el + out_el + wts) * passes
+            flops += 2.0 * out_el * o.ksize * o.ksize * o.c_in * passes
+        elif o.kind == wl.BNRELU:
+            by["bn"] += 8.0 * out_el + 12.0 * out_el
+        elif o.kind == wl.ADD:
+            by["add"] += 12.0 * out_el
+        else:
+            by["other"] += 8.0 * out_el
+    return by, flops
+
+
+class ClockSampler:
+    """nvidia-smi sampling of SM clock and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, "/tmp/hpf_clocks_%d_%d.csv" % (os.getpid(), index)
+
+    def start(self):
+        try:
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "200"], stdout=self.out,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for k, name in enumerate(names):
+                if f[4 + k].lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.remove(self.path)
+        except OSError:
+            pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "power_w_max": float(max(power)),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------------
+def oracle_sample(cfg, images, threads=None):
+    """Times the oracle (forward + reverse sweep) on `images` samples of the workload."""
+    from oracle import reference as ora
+    ops, hwc = cfg["ops"], cfg["in_hwc"]
+    x, labels = wl.draw_inputs(images, hwc, ops[-1].c_out)
+    theta = wl.draw_params(ops)
+    t0 = time.perf_counter()
+    ora.microbatch(ops, hwc, theta, x, labels, want=[])
+    return time.perf_counter() - t0
+
+
+def run_reference(args, cfg):
+    """The reference arm: the oracle as it stands on the host cores, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = os.cpu_count()
+    b = cfg["B"] // cfg["M"]
+    t1 = oracle_sample(cfg, 1)                               # calibration, untimed
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    images = int(max(1, min(b, budget / max(t1, 1e-3))))
+    for _ in range(args.warmup):
+        oracle_sample(cfg, images)
+    ts = [oracle_sample(cfg, images) for _ in range(args.steps)]
+    total = sum(ts)
+    value = images * args.steps / total
+    sample = "forward+backward of one micro-batch of %d image(s) of the workload per step (fp64, OpenMP)" % images
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": NAMES[args.workload], "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def kernel_roofline(torch, hpf, cfg, pk):
+    """Times the dominant kernel of the step (fused BN+ReLU backward) alone, through the C ABI, on the
+    workload's most frequent shape, cycling through operand sets that together exceed L2."""
+    b = cfg["B"] // cfg["M"]
+    shapes = wl.tensor_shapes(cfg["ops"], cfg["in_hwc"])
+    count = {}
+    for o, s in zip(cfg["ops"], shapes):
+        if o.kind == wl.BNRELU:
+            count[s] = count.get(s, 0) + 1
+    (H, W, C), _ = max(count.items(), key=lambda kv: kv[1] * kv[0][0] * kv[0][1] * kv[0][2])
+    rows = b * H * W
+    nset = max(3, int(300e6 // (rows * C * 4 * 3)) + 1)
+    dev = "cuda"
+    xs = [torch.randn(rows, C, device=dev) for _ in range(nset)]
+    dys = [torch.randn(rows, C, device=dev) for _ in range(nset)]
+    dxs = [torch.empty(rows, C, device=dev) for _ in range(nset)]
+    gamma = torch.ones(C, device=dev); beta = torch.zeros(C, device=dev)
+    stats = torch.empty(2 * C, device=dev); y = torch.empty(rows, C, device=dev)
+    dg = torch.empty(C, device=dev); db = torch.empty(C, device=dev)
+    scratch = torch.zeros(hpf.bnrelu_scratch_bytes(rows, C), dtype=torch.uint8, device=dev)
+    st = torch.cuda.current_stream()
+    hpf.bnrelu_fwd(xs[0], gamma, beta, 1e-5, y, stats, rows, C, scratch)
+    reps = 5 * nset
+    for i in range(nset):
+        hpf.bnrelu_bwd(xs[i], dys[i], gamma, beta, stats, dxs[i], None, 0, dg, db, rows, C, scratch)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(st)
+    for i in range(reps):
+        k = i % nset
+        hpf.bnrelu_bwd(xs[k], dys[k], gamma, beta, stats, dxs[k], None, 0, dg, db, rows, C, scratch)
+    e1.record(st)
+    torch.cuda.synchronize()
+    sec = e0.elapsed_time(e1) * 1e-3 / reps
+    alg = 12.0 * rows * C                      # read dy, read x, write dx
+    achieved = alg / sec / 1e9
+    return {"bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"],
+            "traffic": None, "peak_source": pk["source"],
+            "kernel": "fused BN+ReLU backward (reduce + apply), %d rows x %d channels per launch, %d rotating operand sets"
+                      % (rows, C, nset),
+            "algorithmic_bytes_per_launch": alg, "us_per_launch": sec * 1e6}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="hpf", choices=["hpf", "reference"])
+    ap.add_argument("--workload", default="r1001", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--conv-path", type=int, default=0)
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-kernel-roofline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "hpf" else args.warmup
+    cfg = wl.config(args.workload)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import paper_1911_05146_b200 as hpf
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    pk = peaks()
+
+    ops, hwc, B, M = cfg["ops"], cfg["in_hwc"], cfg["B"], cfg["M"]
+    x, labels = wl.draw_inputs(B, hwc, ops[-1].c_out, seed_x=wl.inputs.SEED_X + rank)     # each replica its own batch
+    theta = wl.draw_params(ops)
+    model = hpf.Model(ops, (B,) + tuple(hwc), cfg["cuts"], M)
+    model.set_option(hpf.OPT_GRAPH, 0 if args.no_graph else 1)
+    model.set_option(hpf.OPT_CONV_PATH, args.conv_path)
+    G = model.num_params()
+    params = torch.from_numpy(theta).to(dev)
+    slots = torch.empty((M, G), device=dev)
+    avg = torch.empty(G, device=dev)
+    ws_bytes = model.workspace_bytes()
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    streams = [torch.cuda.Stream(device=dev) for _ in range(model.num_partitions())]
+    torch.cuda.synchronize()
+    model.bind(params, slots, avg, ws, streams)
+    dx, dl = torch.from_numpy(x).to(dev), torch.from_numpy(labels).to(dev)
+    hx, hl = torch.from_numpy(x).pin_memory(), torch.from_numpy(labels).pin_memory()
+    s0 = streams[0]
+
+    def step():
+        model.forward(dx, dl)
+        model.backward()
+        model.grad_average()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    model.synchronize(0)
+    l0 = model.launch_count()
+    sampler = ClockSampler(local)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    e0.record(s0)
+    for _ in range(args.steps):
+        step()
+    e1.record(s0)
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    launches = model.launch_count() - l0
+    loss = model.loss()
+    model.synchronize(0)
+
+    # end to end: host buffers in, loss out, every step
+    for _ in range(2):
+        model.step_host(hx, hl)
+    barrier()
+    e0.record(s0)
+    for _ in range(args.steps):
+        model.step_host(hx, hl)
+    e1.record(s0)
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+
+    if dist is not None:
+        t = torch.tensor([ms, ms_e2e], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = t.tolist()
+    if rank != 0:
+        if dist is not None:
+            dist.barrier(); dist.destroy_process_group()
+        return
+
+    ms_step = ms / args.steps
+    value = world * B / (ms_step * 1e-3)
+    by, flops = step_model(ops, hwc, B)
+    step_bytes = sum(by.values())
+    n_tc, n_cc = model.conv_path_counts()
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "tf32" if n_tc else "f32", "data": "synthetic",
+        "config": {"workload": NAMES[args.workload], "global_batch": world * B, "micro_batches": M,
+                   "partitions": model.num_partitions(), "parallelism": "replicas x%d, no data-path collective" % world,
+                   "l2": "working set %.1f GB per step exceeds the 126 MB L2; no explicit flush" % (ws_bytes / 1e9),
+                   "graph": not args.no_graph, "conv_sites_tensor_core": n_tc, "conv_sites_cuda_core": n_cc,
+                   "loss": loss},
+        "e2e": {"value": world * B / (ms_e2e / args.steps * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": int(hx.numel() * 4 + hl.numel() * 4), "d2h_bytes_per_step": 4},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "step_roofline": {"bound": "hbm", "algorithmic_bytes_per_step": step_bytes, "bytes_by_class": by,
+                          "conv_flops_per_step": flops, "achieved": step_bytes / (ms_step * 1e-3) / 1e9,
+                          "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": step_bytes / (ms_step * 1e-3) / 1e9 / pk["hbm_gbs"],
+                          "peak_source": pk["source"],
+                          "conv_tflops": flops / (ms_step * 1e-3) / 1e12},
+    }
+    if not args.skip_kernel_roofline:
+        line["roofline"] = kernel_roofline(torch, hpf, cfg, pk)
+    if not args.skip_cpu_baseline:
+        b = B // M
+        t1 = oracle_sample(cfg, 1)
+        images = int(max(1, min(b, 20.0 / max(t1, 1e-3))))
+        t = oracle_sample(cfg, images)
+        line["cpu_baseline"] = {"value": images / t, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                                "sample": "forward+backward of one micro-batch of %d image(s) of the workload, %.1f s "
+                                          "(fp64, OpenMP on all host cores)" % (images, t)}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier(); dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

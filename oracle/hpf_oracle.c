@@ -36,6 +36,17 @@
  * order; max-pool padding is -infinity and ties go to the first window
  * position in row-major order.
  *
+ * ReLU decisions.  The derivative of ReLU is a step, so dL/d(anything upstream)
+ * is a discontinuous function of the forward values: an implementation whose
+ * pre-activation z differs from this file's by a rounding error takes the
+ * other branch wherever |z| is smaller than that error, and both branches are
+ * correct results of the method in their own arithmetic.  The sweeps therefore
+ * accept, per BNRELU op, the decisions (z > 0) another implementation took:
+ * where |z| >= tau*|gamma_c| the decision is unique and this file's own is
+ * used (a disagreement there is counted as a violation); where |z| is below
+ * that window the supplied decision is used.  With no decisions supplied, or
+ * tau = 0, nothing changes.
+ *
  * Layout: activations are [n][h][w][c] (channels innermost), convolution
  * weights [c_out][r][s][c_in].  Everything is double.
  *
@@ -307,28 +318,55 @@ void ora_bnrelu_fwd(const double *x, int64_t rows, int32_t C, const double *gamm
 }
 
 /* dz = dy * [gamma*xhat+beta > 0]; dbeta = sum dz; dgamma = sum dz*xhat;
- * dx = gamma / sqrt(var+eps) * (dz - dbeta/rows - xhat * dgamma/rows). */
-void ora_bnrelu_bwd(const double *x, const double *dy, int64_t rows, int32_t C, const double *gamma,
-                    const double *beta, double eps, double *dx, double *dgamma, double *dbeta)
+ * dx = gamma / sqrt(var+eps) * (dz - dbeta/rows - xhat * dgamma/rows).
+ * decisions (may be NULL): one byte per element, nonzero = "z > 0" as another
+ * implementation decided it; honoured only inside the window |z| < tau*|gamma_c|.
+ * counts (may be NULL): [0] += decisions used that differ from this file's own,
+ * [1] += supplied decisions that differ outside the window (violations). */
+void ora_bnrelu_bwd_dec(const double *x, const double *dy, int64_t rows, int32_t C, const double *gamma,
+                        const double *beta, double eps, const uint8_t *decisions, double tau, int64_t *counts,
+                        double *dx, double *dgamma, double *dbeta)
 {
     double *mean = (double *)malloc(sizeof(double) * 2 * (size_t)C), *var = mean + C;
+    int64_t n_used = 0, n_viol = 0;
     ora_bn_stats(x, rows, C, mean, var);
-#pragma omp parallel for schedule(static)
+#pragma omp parallel for schedule(static) reduction(+ : n_used, n_viol)
     for (int32_t c = 0; c < C; ++c) {
         double rstd = 1.0 / sqrt(var[c] + eps), sb = 0.0, sg = 0.0;
+        double window = tau * fabs(gamma[c]);
+        uint8_t *open = (uint8_t *)malloc((size_t)rows);
         for (int64_t i = 0; i < rows; ++i) {
             double xh = (x[i * C + c] - mean[c]) * rstd;
-            double dz = (gamma[c] * xh + beta[c] > 0.0) ? dy[i * C + c] : 0.0;
+            double z = gamma[c] * xh + beta[c];
+            int own = z > 0.0;
+            int use = own;
+            if (decisions) {
+                int theirs = decisions[i * C + c] != 0;
+                if (theirs != own) {
+                    if (fabs(z) < window) { use = theirs; ++n_used; }
+                    else ++n_viol;
+                }
+            }
+            open[i] = (uint8_t)use;
+            double dz = use ? dy[i * C + c] : 0.0;
             sb += dz; sg += dz * xh;
         }
         dbeta[c] = sb; dgamma[c] = sg;
         for (int64_t i = 0; i < rows; ++i) {
             double xh = (x[i * C + c] - mean[c]) * rstd;
-            double dz = (gamma[c] * xh + beta[c] > 0.0) ? dy[i * C + c] : 0.0;
+            double dz = open[i] ? dy[i * C + c] : 0.0;
             dx[i * C + c] = gamma[c] * rstd * (dz - sb / (double)rows - xh * sg / (double)rows);
         }
+        free(open);
     }
+    if (counts) { counts[0] += n_used; counts[1] += n_viol; }
     free(mean);
+}
+
+void ora_bnrelu_bwd(const double *x, const double *dy, int64_t rows, int32_t C, const double *gamma,
+                    const double *beta, double eps, double *dx, double *dgamma, double *dbeta)
+{
+    ora_bnrelu_bwd_dec(x, dy, rows, C, gamma, beta, eps, NULL, 0.0, NULL, dx, dgamma, dbeta);
 }
 
 /* Window max with -infinity padding; argmax = first maximum in (r,s) row-major order. */
@@ -466,6 +504,9 @@ typedef struct {
     int64_t *w_off, *w_cnt, *b_off, *b_cnt, G;
     const double *theta;          /* G */
     const int32_t *labels;        /* b */
+    const uint8_t *const *decisions; /* per op (BNRELU entries used), or NULL */
+    double tau;
+    int64_t counts[2];
 } ora_ctx;
 
 static const int32_t *shape_of(const ora_ctx *c, int32_t t) { return t < 0 ? c->in_hwc : &c->hwc[3 * t]; }
@@ -523,8 +564,9 @@ static int op_backward(const ora_ctx *c, int32_t i, const double *in0, const dou
         if (d0) ora_conv_dgrad(dout, c->b, s[0], s[1], s[2], th + c->w_off[i], o->c_out, o->ksize, o->stride, o->pad, tmp);
         break;
     case ORA_BNRELU:
-        ora_bnrelu_bwd(in0, dout, (int64_t)c->b * s[0] * s[1], s[2], th + c->w_off[i], th + c->b_off[i], o->eps,
-                       tmp, g + c->w_off[i], g + c->b_off[i]);
+        ora_bnrelu_bwd_dec(in0, dout, (int64_t)c->b * s[0] * s[1], s[2], th + c->w_off[i], th + c->b_off[i], o->eps,
+                           c->decisions ? c->decisions[i] : NULL, c->tau, ((ora_ctx *)c)->counts,
+                           tmp, g + c->w_off[i], g + c->b_off[i]);
         break;
     case ORA_ADD: {
         int64_t n = numel_of(c, i);
@@ -570,13 +612,15 @@ static void ctx_free(ora_ctx *c) { free(c->hwc); free(c->w_off); }
  * keep_act[i] / keep_dact[i] (either array may be NULL, any entry may be NULL)
  * receive op i's output and dL_m/d(output).  dx_in (may be NULL) receives
  * dL_m/d(network input).  g (length G) receives dL_m/d(theta). */
-int ora_microbatch(const ora_op *ops, int32_t n_ops, int32_t b, const int32_t in_hwc[3],
-                   const double *theta, const double *x, const int32_t *labels,
-                   double **keep_act, double **keep_dact, double *dx_in, double *g, double *loss)
+int ora_microbatch_dec(const ora_op *ops, int32_t n_ops, int32_t b, const int32_t in_hwc[3],
+                       const double *theta, const double *x, const int32_t *labels,
+                       const uint8_t *const *decisions, double tau, int64_t *counts_out,
+                       double **keep_act, double **keep_dact, double *dx_in, double *g, double *loss)
 {
     ora_ctx c;
     int rc = ctx_init(&c, ops, n_ops, b, in_hwc, theta, labels);
     if (rc) { ctx_free(&c); return rc; }
+    c.decisions = decisions; c.tau = tau;
     double **act = (double **)calloc((size_t)n_ops, sizeof(double *));
     double **dact = (double **)calloc((size_t)n_ops, sizeof(double *));
     double *dx0 = NULL;
@@ -606,11 +650,19 @@ int ora_microbatch(const ora_op *ops, int32_t n_ops, int32_t b, const int32_t in
         free(dact[i]); dact[i] = NULL;   /* every consumer of op i has a larger index */
     }
     if (dx_in) memcpy(dx_in, dx0, sizeof(double) * (size_t)numel_of(&c, -1));
+    if (counts_out) { counts_out[0] = c.counts[0]; counts_out[1] = c.counts[1]; }
 done:
     for (int32_t i = 0; i < n_ops; ++i) { free(act[i]); free(dact[i]); }
     free(act); free(dact); free(dx0);
     ctx_free(&c);
     return rc;
+}
+
+int ora_microbatch(const ora_op *ops, int32_t n_ops, int32_t b, const int32_t in_hwc[3],
+                   const double *theta, const double *x, const int32_t *labels,
+                   double **keep_act, double **keep_dact, double *dx_in, double *g, double *loss)
+{
+    return ora_microbatch_dec(ops, n_ops, b, in_hwc, theta, x, labels, NULL, 0.0, NULL, keep_act, keep_dact, dx_in, g, loss);
 }
 
 /* ------------------------------------------------------------------ */
@@ -626,17 +678,19 @@ done:
  *
  * keep_fwd / keep_bwd: optional [n_cuts][max_live] arrays of output buffers
  * for the messages; the rest as in ora_microbatch. */
-int ora_microbatch_partitioned(const ora_op *ops, int32_t n_ops, int32_t b, const int32_t in_hwc[3],
-                               const int32_t *cuts, int32_t n_cuts, int32_t max_live,
-                               const double *theta, const double *x, const int32_t *labels,
-                               double **keep_act, double **keep_dact,
-                               double **keep_fwd, double **keep_bwd,
-                               double *g, double *loss)
+int ora_microbatch_partitioned_dec(const ora_op *ops, int32_t n_ops, int32_t b, const int32_t in_hwc[3],
+                                   const int32_t *cuts, int32_t n_cuts, int32_t max_live,
+                                   const double *theta, const double *x, const int32_t *labels,
+                                   const uint8_t *const *decisions, double tau, int64_t *counts_out,
+                                   double **keep_act, double **keep_dact,
+                                   double **keep_fwd, double **keep_bwd,
+                                   double *g, double *loss)
 {
     if (ora_check_cuts(n_ops, cuts, n_cuts)) return ORA_EINVAL;
     ora_ctx c;
     int rc = ctx_init(&c, ops, n_ops, b, in_hwc, theta, labels);
     if (rc) { ctx_free(&c); return rc; }
+    c.decisions = decisions; c.tau = tau;
     int32_t P = n_cuts + 1;
     /* bounds of partition p: [lo(p), hi(p)) */
 #define LO(p) ((p) == 0 ? 0 : cuts[(p) - 1])
@@ -723,6 +777,7 @@ int ora_microbatch_partitioned(const ora_op *ops, int32_t n_ops, int32_t b, cons
         for (int32_t i = 0; i < n_ops; ++i) free(dl[i]);
         free(dl);
     }
+    if (counts_out) { counts_out[0] = c.counts[0]; counts_out[1] = c.counts[1]; }
 done:
     for (size_t j = 0; j < (size_t)(n_cuts + 1) * (size_t)n_ops; ++j) { free(fwd_box[j]); free(bwd_box[j]); }
     for (size_t j = 0; j < (size_t)P * (size_t)n_ops; ++j) free(loc[j]);
@@ -731,6 +786,17 @@ done:
     return rc;
 #undef LO
 #undef HI
+}
+
+int ora_microbatch_partitioned(const ora_op *ops, int32_t n_ops, int32_t b, const int32_t in_hwc[3],
+                               const int32_t *cuts, int32_t n_cuts, int32_t max_live,
+                               const double *theta, const double *x, const int32_t *labels,
+                               double **keep_act, double **keep_dact,
+                               double **keep_fwd, double **keep_bwd,
+                               double *g, double *loss)
+{
+    return ora_microbatch_partitioned_dec(ops, n_ops, b, in_hwc, cuts, n_cuts, max_live, theta, x, labels, NULL, 0.0,
+                                          NULL, keep_act, keep_dact, keep_fwd, keep_bwd, g, loss);
 }
 
 /* ------------------------------------------------------------------ */

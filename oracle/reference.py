@@ -214,11 +214,23 @@ def _ptr_array(bufs):
     return arr
 
 
-def microbatch(ops, in_hwc, theta, x, labels, cuts=None, want=None, want_input_grad=False):
+def _decision_array(n, decisions):
+    arr = (C.POINTER(C.c_uint8) * n)()
+    keep = []
+    for i, d in decisions.items():
+        d = np.ascontiguousarray(d, dtype=np.uint8)
+        keep.append(d)
+        arr[i] = d.ctypes.data_as(C.POINTER(C.c_uint8))
+    return arr, keep
+
+
+def microbatch(ops, in_hwc, theta, x, labels, cuts=None, want=None, want_input_grad=False, decisions=None, tau=0.0):
     """One micro-batch.  Returns a dict with loss, g, act{op}, dact{op} and, when
     ``cuts`` is given (partition-by-partition execution), fwd_msg / bwd_msg
     keyed by (cut index, position in the live set).  ``want`` limits which ops'
-    tensors are kept (default: all)."""
+    tensors are kept (default: all).  ``decisions`` maps a BNRELU op to the
+    (z > 0) decisions of another implementation, honoured inside the window
+    |z| < tau*|gamma|; the result then carries decisions_used / decision_violations."""
     n = len(ops)
     b = x.shape[0]
     shp = shapes(ops, in_hwc)
@@ -234,9 +246,12 @@ def microbatch(ops, in_hwc, theta, x, labels, cuts=None, want=None, want_input_g
     loss = C.c_double()
     gp = g.ctypes.data_as(C.POINTER(C.c_double))
     res = {}
+    dec, dec_keep = _decision_array(n, decisions) if decisions else (None, None)
+    counts = (C.c_int64 * 2)(0, 0)
     if cuts is None:
         dx = np.empty(x.shape) if want_input_grad else None
-        rc = lib().ora_microbatch(_ops(ops), n, b, _i32(in_hwc), tp, xp, _i32(labels),
+        rc = lib().ora_microbatch_dec(_ops(ops), n, b, _i32(in_hwc), tp, xp, _i32(labels),
+                                  dec, C.c_double(tau), counts,
                                   _ptr_array(act), _ptr_array(dact),
                                   dx.ctypes.data_as(C.POINTER(C.c_double)) if dx is not None else None,
                                   gp, C.byref(loss))
@@ -250,13 +265,15 @@ def microbatch(ops, in_hwc, theta, x, labels, cuts=None, want=None, want_input_g
         bwd = [[np.empty((b,) + shp[t]) for t in l] + [None] * (max_live - len(l)) for l in lives]
         flat_f = [m for row in fwd for m in row] or [None]
         flat_b = [m for row in bwd for m in row] or [None]
-        rc = lib().ora_microbatch_partitioned(_ops(ops), n, b, _i32(in_hwc), _i32(cuts), len(cuts), max_live,
-                                              tp, xp, _i32(labels), _ptr_array(act), _ptr_array(dact),
+        rc = lib().ora_microbatch_partitioned_dec(_ops(ops), n, b, _i32(in_hwc), _i32(cuts), len(cuts), max_live,
+                                              tp, xp, _i32(labels), dec, C.c_double(tau), counts,
+                                              _ptr_array(act), _ptr_array(dact),
                                               _ptr_array(flat_f), _ptr_array(flat_b), gp, C.byref(loss))
         _check(rc, "microbatch_partitioned")
         res["live"] = lives
         res["fwd_msg"] = {(j, i): fwd[j][i] for j, l in enumerate(lives) for i in range(len(l))}
         res["bwd_msg"] = {(j, i): bwd[j][i] for j, l in enumerate(lives) for i in range(len(l))}
+    res.update(decisions_used=counts[0], decision_violations=counts[1])
     res.update(loss=loss.value, g=g,
                act={i: a for i, a in enumerate(act) if a is not None},
                dact={i: a for i, a in enumerate(dact) if a is not None})

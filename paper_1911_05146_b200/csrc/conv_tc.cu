@@ -1,44 +1,859 @@
-// Tensor-core convolution path (placeholder until the tcgen05 kernels land): reports every shape as
-// outside its reach, so all convolutions run on the CUDA-core kernels.
+// Tensor-core convolution kernels for sm_100a: implicit GEMM on tcgen05.mma (kind::tf32, fp32
+// accumulators in tensor memory), operands staged in shared memory by TMA, one elected thread
+// issuing the MMAs, mbarrier hand-shakes between the TMA producer, the MMA issuer and the epilogue.
+//
+// Forward (and the data gradient, which is a forward convolution over dy with rearranged weights):
+//   D[pixels, c_out] = sum over taps (r,s) and channel chunks of A_tap[pixels, c] * W_tap[c_out, c]^T
+//   One CTA owns one tile of 128 output pixels, chosen as a rectangular box (w x h x n) of the
+//   output so that the A operand of every tap is ONE tiled TMA box of the input tensor, shifted by
+//   (r - pad, s - pad); TMA's out-of-bounds zero fill is the convolution's zero padding.  Both
+//   operands are K-major (channels innermost) with the 64-byte or 128-byte shared-memory swizzle.
+//   A strided 1x1 convolution reads its input through a tensor map with doubled strides.
+// Weight gradient:
+//   dW[c_out, tap, c_in] = sum over pixels dy[pixel, c_out] * x[pixel + tap, c_in]
+//   The reduction runs over pixels, but the tensors are channels-innermost, and kind::tf32 reads
+//   MN-major shared-memory operands as zeros on this hardware (measured), so both operands must be
+//   re-laid K-major (pixels innermost).  TMA brings the raw [pixel][channel] tiles in, four warps
+//   transpose them in shared memory into the 128-byte-swizzled K-major layout (4 conflict-free
+//   32-bit loads and one 128-bit store per thread and 4 pixels), and the MMA issuer consumes those.
+//   One CTA walks a slice of the pixel tiles, keeps one accumulator per tap in tensor memory, and
+//   writes a partial; a second kernel adds the partials in fixed order.
+//
+// Every wait on an mbarrier is bounded: after the limit the kernel records where it gave up in the
+// device status word, stops issuing work, waits (bounded) for its TMA copies in flight, frees its
+// tensor memory and returns.
 #include "conv_tc.h"
+
+#include <cuda.h>
+#include <stdint.h>
+#include <string.h>
 
 namespace hpf {
 
-bool conv_tc_supported(const ConvShape&, int) { return false; }
-cudaError_t conv_tc_init() { return cudaSuccess; }
-size_t conv_tc_scratch_bytes(const ConvShape&) { return 0; }
-cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape&, int, const float*, const float*, const float*, float*,
-                            const float*, bool, void*)
-{
-    plan->valid = 0;
-    return cudaErrorNotSupported;
-}
-cudaError_t conv_tc_launch(const ConvTcPlan*, DeviceStatus*, cudaStream_t, int64_t*) { return cudaErrorNotSupported; }
-
 namespace {
-__global__ void dgrad_weights_kernel(const float* __restrict__ w, float* __restrict__ wt, int C, int K, int R)
+
+constexpr int kTileM = 128;                 // MMA M (TMEM lanes)
+constexpr long long kWaitLimit = 4000000000LL;   // clock64 ticks (~2 s) before a wait gives up
+constexpr uint32_t kSmemBudget = 200 * 1024;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
-    const int64_t total = (int64_t)K * R * R * C;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += stride) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+// Bounded wait.  Returns false if it gave up (or another role already did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitLimit) { *abort_flag = 1; return false; }
+    }
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n"
+        "}\n"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 lanes x 16 consecutive 32-bit columns: thread i of the warp receives lane (base lane + i)
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v)
+{
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte offsets in
+// 16-byte units, descriptor version 1, swizzle mode in the top bits (2 = 128 B, 4 = 64 B).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t swizzle_bytes)
+{
+    const uint64_t layout = swizzle_bytes == 128 ? 2ull : 4ull;
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (layout << 61);
+}
+
+// Instruction descriptor: fp32 accumulator, TF32 A and B, M = 128, N = n; major bits select MN-major operands.
+inline uint32_t instr_desc(int n, bool a_mn_major, bool b_mn_major)
+{
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+}
+
+__device__ __forceinline__ void report(DeviceStatus* status, unsigned int code)
+{
+    if (atomicCAS(&status->code, 0u, code) == 0u) status->detail = blockIdx.x;
+}
+
+// ------------------------------------------------------------------------------------------------
+// kernel parameters
+// ------------------------------------------------------------------------------------------------
+struct alignas(64) FwdParams {
+    CUtensorMap tm_a;            // activations {C, Wv, Hv, N}
+    CUtensorMap tm_b;            // weights {taps*C, c_out}
+    float* out;
+    const float* extra;
+    DeviceStatus* status;
+    long long os_n, os_h, os_w;  // output strides (floats) of pixel (n, p, q)
+    long long dense_h, dense_w;  // strides of one row / one pixel of the dense output (zero fill)
+    int accumulate;
+    int box_w, box_h, box_n, tiles_w, tiles_h;
+    int P, Q, N;                 // output pixel grid of the GEMM
+    int c_out, n_chunk;          // total output channels, channels per CTA
+    int R, pad;                  // window and the tap shift
+    int c_in, kchunk, n_kchunks;
+    int swizzle;
+    int stages;
+    int zero_fill;               // > 1: the output pixel grid is strided, fill the rest of each patch with zeros
+    int out_h, out_w;            // dense output extent (zero fill bounds)
+    unsigned int a_bytes, b_bytes, tx_bytes, tmem_cols, idesc;
+};
+
+struct alignas(64) WgradParams {
+    CUtensorMap tm_a;            // dy {c_out, Q, P, N}, box {m_chunk, w, h, n}, no swizzle
+    CUtensorMap tm_b;            // x {C, Wv, Hv, N}, box {n_cols, w, h, n}, no swizzle
+    float* out;                  // dw or partials [splits][c_out*taps*c_in]
+    DeviceStatus* status;
+    int box_w, box_h, box_n, tiles_w, tiles_h, n_tiles, tiles_per_split;
+    int rows;                    // pixels per tile (32 or 64)
+    int c_out, c_in, R, pad;
+    int m_chunk;                 // output channels per CTA (<= 128)
+    int n_cols;                  // input channels per CTA (<= 256)
+    int taps_per_cta;
+    int raw_stages, t_stages;
+    unsigned int raw_bytes, t_bytes, tx_per_tap, tx_a, tmem_cols, idesc;
+    long long split_stride;      // floats between partials
+};
+
+// ------------------------------------------------------------------------------------------------
+// forward / data-gradient kernel
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) conv_tc_fwd_kernel(const __grid_constant__ FwdParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[2 * 8 + 1];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ int issued, consumed;
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t stage_bytes = p.a_bytes + p.b_bytes;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[8]), accum_bar = smem_u32(&bars[16]);
+
+    int t = blockIdx.x;
+    const int tw = t % p.tiles_w; t /= p.tiles_w;
+    const int th = t % p.tiles_h;
+    const int tn = t / p.tiles_h;
+    const int q0 = tw * p.box_w, p0 = th * p.box_h, n0 = tn * p.box_n;
+    const int co0 = blockIdx.y * p.n_chunk;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        mbar_init(accum_bar, 1);
+        abort_flag = 0; issued = 0; consumed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), p.tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+    const int total = p.R * p.R * p.n_kchunks;
+
+    if (warp == 0 && lane == 0) {
+        // ---- TMA producer ----
+        int it = 0;
+        for (; it < total; ++it) {
+            const int s = it % p.stages;
+            if (!mbar_wait(empty0 + 8 * s, ((it / p.stages) & 1) ^ 1, &abort_flag)) { report(p.status, 1); break; }
+            const int tap = it / p.n_kchunks, kc = it % p.n_kchunks;
+            const int r = tap / p.R, sx = tap % p.R;
+            const uint32_t a_dst = smem_base + s * stage_bytes, b_dst = a_dst + p.a_bytes;
+            mbar_expect_tx(full0 + 8 * s, p.tx_bytes);
+            tma_load_4d(a_dst, &p.tm_a, full0 + 8 * s, kc * p.kchunk, q0 + sx - p.pad, p0 + r - p.pad, n0);
+            tma_load_2d(b_dst, &p.tm_b, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
+        }
+        issued = it;
+    } else if (warp == 1 && lane == 0) {
+        // ---- MMA issuer ----
+        const uint32_t sbo = 8u * (uint32_t)p.kchunk * 4u;          // 8 rows of one swizzle atom
+        int it = 0;
+        for (; it < total; ++it) {
+            const int s = it % p.stages;
+            if (!mbar_wait(full0 + 8 * s, (it / p.stages) & 1, &abort_flag)) { report(p.status, 2); break; }
+            tc_fence_after();
+            const uint32_t a_src = smem_base + s * stage_bytes, b_src = a_src + p.a_bytes;
+            for (int k8 = 0; k8 < p.kchunk / 8; ++k8) {
+                const uint64_t ad = smem_desc(a_src + 32u * k8, 16, sbo, p.swizzle);
+                const uint64_t bd = smem_desc(b_src + 32u * k8, 16, sbo, p.swizzle);
+                umma_tf32(tmem_base, ad, bd, p.idesc, (it | k8) ? 1u : 0u);
+            }
+            umma_commit(empty0 + 8 * s);     // frees the stage once these MMAs have read it
+        }
+        consumed = it;
+        if (it == total) umma_commit(accum_bar);
+    }
+
+    // ---- epilogue: all four warps, warp w owns TMEM lanes [32w, 32w+32) ----
+    __syncwarp();
+    bool ok = mbar_wait(accum_bar, 0, &abort_flag);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+        tc_fence_after();
+        const int row = threadIdx.x;
+        const int wi = row % p.box_w, hi = (row / p.box_w) % p.box_h, ni = row / (p.box_w * p.box_h);
+        const int q = q0 + wi, pp = p0 + hi, n = n0 + ni;
+        const bool valid = ni < p.box_n && q < p.Q && pp < p.P && n < p.N;
+        float* orow = p.out + n * p.os_n + pp * p.os_h + q * p.os_w + co0;
+        const float* erow = p.extra ? p.extra + (n * p.os_n + pp * p.os_h + q * p.os_w + co0) : nullptr;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
+        for (int c0 = 0; c0 < p.n_chunk; c0 += 16) {
+            float v[16];
+            tmem_ld16(lane_addr + (uint32_t)c0, v);
+            if (valid) {
+#pragma unroll
+                for (int j = 0; j < 16; j += 4) {
+                    float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    if (erow) { const float4 e = __ldg(reinterpret_cast<const float4*>(erow + c0 + j)); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+                    if (p.accumulate) { const float4 e = *reinterpret_cast<const float4*>(orow + c0 + j); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+                    *reinterpret_cast<float4*>(orow + c0 + j) = o;
+                }
+            }
+        }
+        if (p.zero_fill > 1 && valid) {
+            // strided data gradient: the positions between the samples receive no contribution
+            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int dy = 0; dy < p.zero_fill; ++dy)
+                for (int dx = 0; dx < p.zero_fill; ++dx) {
+                    if ((dy | dx) == 0) continue;
+                    if (pp * p.zero_fill + dy >= p.out_h || q * p.zero_fill + dx >= p.out_w) continue;
+                    float* zr = orow + dy * p.dense_h + dx * p.dense_w;
+                    for (int c0 = 0; c0 < p.n_chunk; c0 += 4) *reinterpret_cast<float4*>(zr + c0) = z;
+                }
+        }
+    }
+
+    // ---- teardown ----
+    tc_fence_before();
+    __syncthreads();
+    if (abort_flag && threadIdx.x == 0) {
+        // copies still in flight must land before the shared memory is given back
+        for (int it = consumed; it < issued; ++it) {
+            const int s = it % p.stages;
+            const long long t0 = clock64();
+            while (!mbar_try_wait(full0 + 8 * s, (it / p.stages) & 1) && clock64() - t0 < kWaitLimit) {}
+        }
+    }
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
+}
+
+// ------------------------------------------------------------------------------------------------
+// weight-gradient kernel: 6 warps = TMA producer, MMA issuer, 4 transposer / epilogue warps
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// raw [rows][channels] (dense) -> K-major: channel rows of 128 bytes (32 pixels), 16-byte chunks XOR-swizzled by
+// (row % 8), further groups of 32 pixels `atom_stride` bytes apart.  128 threads.
+__device__ __forceinline__ void transpose_tile(const uint8_t* raw, uint8_t* dst, int channels, int rows, uint32_t atom_stride, int tid)
+{
+    const int items = channels * (rows >> 2);
+    for (int it = tid; it < items; it += 128) {
+        const int c = it % channels, p4 = it / channels;
+        const float* src = reinterpret_cast<const float*>(raw) + (p4 * 4) * channels + c;
+        float4 v;
+        v.x = src[0]; v.y = src[channels]; v.z = src[2 * channels]; v.w = src[3 * channels];
+        uint8_t* d = dst + (uint32_t)(p4 >> 3) * atom_stride + (uint32_t)c * 128u + (uint32_t)(((p4 & 7) ^ (c & 7)) << 4);
+        *reinterpret_cast<float4*>(d) = v;
+    }
+}
+
+__global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constant__ WgradParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[4 * 4 + 1];       // full_raw[4], empty_raw[4], full_t[4], empty_t[4], accum
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ int issued, raw_consumed;
+
+    const uint32_t base_off = ((smem_u32(smem_raw) + 1023u) & ~1023u) - smem_u32(smem_raw);
+    uint8_t* smem = smem_raw + base_off;
+    const uint32_t smem_base = smem_u32(smem);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t full_raw0 = smem_u32(&bars[0]), empty_raw0 = smem_u32(&bars[4]), full_t0 = smem_u32(&bars[8]),
+                   empty_t0 = smem_u32(&bars[12]), accum_bar = smem_u32(&bars[16]);
+    // shared memory: raw stages first, then the transposed stages
+    const uint32_t t_region0 = (uint32_t)p.raw_stages * p.raw_bytes;
+
+    const int split = blockIdx.x;
+    const int tap0 = blockIdx.y * p.taps_per_cta;
+    const int m_chunks = p.c_out / p.m_chunk;
+    const int m0 = (blockIdx.z % m_chunks) * p.m_chunk;
+    const int cn0 = (blockIdx.z / m_chunks) * p.n_cols;
+    int ntaps = p.R * p.R - tap0;
+    if (ntaps > p.taps_per_cta) ntaps = p.taps_per_cta;
+    const int tile_begin = split * p.tiles_per_split;
+    int tile_end = tile_begin + p.tiles_per_split;
+    if (tile_end > p.n_tiles) tile_end = p.n_tiles;
+    const int total = tile_end - tile_begin;
+    const int katoms = p.rows >> 5;
+    const uint32_t raw_a = (uint32_t)p.rows * p.m_chunk * 4u, raw_b = (uint32_t)p.rows * p.n_cols * 4u;
+    const uint32_t t_a = (uint32_t)katoms * 128u * 128u;                  // room for 128 channel rows
+    const uint32_t t_b = (uint32_t)katoms * (uint32_t)p.n_cols * 128u;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(full_raw0 + 8 * s, 1); mbar_init(empty_raw0 + 8 * s, 4);
+            mbar_init(full_t0 + 8 * s, 4); mbar_init(empty_t0 + 8 * s, 1);
+        }
+        mbar_init(accum_bar, 1);
+        abort_flag = 0; issued = 0; raw_consumed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), p.tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- TMA producer ----
+            int it = 0;
+            for (; it < total; ++it) {
+                const int s = it % p.raw_stages;
+                if (!mbar_wait(empty_raw0 + 8 * s, ((it / p.raw_stages) & 1) ^ 1, &abort_flag)) { report(p.status, 3); break; }
+                int t = tile_begin + it;
+                const int tw = t % p.tiles_w; t /= p.tiles_w;
+                const int th = t % p.tiles_h;
+                const int tn = t / p.tiles_h;
+                const int q0 = tw * p.box_w, p0 = th * p.box_h, n0 = tn * p.box_n;
+                const uint32_t dst = smem_base + s * p.raw_bytes;
+                const uint32_t bar = full_raw0 + 8 * s;
+                mbar_expect_tx(bar, p.tx_a + (uint32_t)ntaps * p.tx_per_tap);
+                tma_load_4d(dst, &p.tm_a, bar, m0, q0, p0, n0);
+                for (int tp = 0; tp < ntaps; ++tp) {
+                    const int r = (tap0 + tp) / p.R, sx = (tap0 + tp) % p.R;
+                    tma_load_4d(dst + raw_a + tp * raw_b, &p.tm_b, bar, cn0, q0 + sx - p.pad, p0 + r - p.pad, n0);
+                }
+            }
+            issued = it;
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- MMA issuer ----
+            int it = 0;
+            for (; it < total; ++it) {
+                const int t = it % p.t_stages;
+                if (!mbar_wait(full_t0 + 8 * t, (it / p.t_stages) & 1, &abort_flag)) { report(p.status, 4); break; }
+                tc_fence_after();
+                const uint32_t a_src = smem_base + t_region0 + t * p.t_bytes, b_src = a_src + t_a;
+                for (int tp = 0; tp < ntaps; ++tp)
+                    for (int kb = 0; kb < katoms; ++kb)
+                        for (int k8 = 0; k8 < 4; ++k8) {
+                            const uint64_t ad = smem_desc(a_src + (uint32_t)kb * 16384u + 32u * k8, 16, 1024, 128);
+                            const uint64_t bd = smem_desc(b_src + (uint32_t)tp * t_b + (uint32_t)kb * (uint32_t)p.n_cols * 128u + 32u * k8, 16, 1024, 128);
+                            umma_tf32(tmem_base + (uint32_t)(tp * p.n_cols), ad, bd, p.idesc, (it | kb | k8) ? 1u : 0u);
+                        }
+                umma_commit(empty_t0 + 8 * t);
+            }
+            if (it == total) umma_commit(accum_bar);
+        }
+    } else {
+        // ---- transposers (warps 2..5), then the epilogue ----
+        const int tid = threadIdx.x - 64;
+        int it = 0;
+        bool ok = true;
+        for (; it < total && ok; ++it) {
+            const int s = it % p.raw_stages, t = it % p.t_stages;
+            ok = mbar_wait(full_raw0 + 8 * s, (it / p.raw_stages) & 1, &abort_flag) &&
+                 mbar_wait(empty_t0 + 8 * t, ((it / p.t_stages) & 1) ^ 1, &abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) { if (lane == 0) report(p.status, 5); break; }
+            const uint8_t* raw = smem + s * p.raw_bytes;
+            uint8_t* tdst = smem + t_region0 + t * p.t_bytes;
+            transpose_tile(raw, tdst, p.m_chunk, p.rows, 16384u, tid);
+            for (int tp = 0; tp < ntaps; ++tp)
+                transpose_tile(raw + raw_a + tp * raw_b, tdst + t_a + tp * t_b, p.n_cols, p.rows, (uint32_t)p.n_cols * 128u, tid);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes -> MMA reads
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(full_t0 + 8 * t); mbar_arrive(empty_raw0 + 8 * s); }
+        }
+        if (tid == 0) raw_consumed = it;
+
+        bool done = ok && mbar_wait(accum_bar, 0, &abort_flag);
+        done = __all_sync(0xffffffffu, done);
+        if (done) {
+            tc_fence_after();
+            const int row = (warp & 3) * 32 + lane;          // TMEM lane = output channel within the chunk
+            const bool valid = row < p.m_chunk;
+            const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+            float* obase = p.out + (long long)split * p.split_stride + ((long long)(m0 + row) * p.R * p.R) * p.c_in + cn0;
+            for (int tp = 0; tp < ntaps; ++tp)
+                for (int c0 = 0; c0 < p.n_cols; c0 += 16) {
+                    float v[16];
+                    tmem_ld16(lane_addr + (uint32_t)(tp * p.n_cols + c0), v);
+                    if (valid) {
+                        // a gradient slot starts at m*G floats: 16-byte aligned only if G is a multiple of 4
+                        float* o = obase + (long long)(tap0 + tp) * p.c_in + c0;
+                        if ((reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(o + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) o[j] = v[j];
+                        }
+                    }
+                }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (abort_flag && threadIdx.x == 0) {
+        for (int it = raw_consumed; it < issued; ++it) {
+            const int s = it % p.raw_stages;
+            const long long t0 = clock64();
+            while (!mbar_try_wait(full_raw0 + 8 * s, (it / p.raw_stages) & 1) && clock64() - t0 < kWaitLimit) {}
+        }
+    }
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
+}
+
+__global__ void __launch_bounds__(256)
+wgrad_partials_reduce_kernel(const float* __restrict__ partials, float* __restrict__ dw, long long n, int splits)
+{
+    // n is a multiple of 4 and the partials are 16-byte aligned; dw (inside a gradient slot) may not be
+    const long long n4 = n / 4;
+    const bool dw_vec = (reinterpret_cast<uintptr_t>(dw) & 15u) == 0;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        float4 s = __ldcg(reinterpret_cast<const float4*>(partials) + i);
+        for (int z = 1; z < splits; ++z) {
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(partials + (long long)z * n) + i);
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        }
+        if (dw_vec) reinterpret_cast<float4*>(dw)[i] = s;
+        else { dw[4 * i] = s.x; dw[4 * i + 1] = s.y; dw[4 * i + 2] = s.z; dw[4 * i + 3] = s.w; }
+    }
+}
+
+__global__ void __launch_bounds__(256) dgrad_weights_kernel(const float* __restrict__ w, float* __restrict__ wt, int C, int K, int R)
+{
+    const long long total = (long long)K * R * R * C;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += stride) {
         // o indexes wt[c][r'][s'][k]
         const int k = (int)(o % K);
-        int64_t t = o / K;
+        long long t = o / K;
         const int s2 = (int)(t % R); t /= R;
         const int r2 = (int)(t % R);
         const int c = (int)(t / R);
-        wt[o] = __ldg(&w[(((int64_t)k * R + (R - 1 - r2)) * R + (R - 1 - s2)) * C + c]);
+        wt[o] = __ldg(&w[(((long long)k * R + (R - 1 - r2)) * R + (R - 1 - s2)) * C + c]);
     }
 }
+
+// ------------------------------------------------------------------------------------------------
+// host: tile geometry and tensor maps
+// ------------------------------------------------------------------------------------------------
+struct PixelBox { int w, h, n, rows; };
+
+// A rectangular box of output pixels with at most `max_rows` pixels; all of w, then rows of h, then images.
+bool choose_box(int Q, int P, int N, int max_rows, int rows_mult, PixelBox* out)
+{
+    if (Q > max_rows) return false;
+    PixelBox b;
+    b.w = Q;
+    int hmax = max_rows / Q;
+    if (hmax > P) hmax = P;
+    b.h = 1;
+    for (int h = hmax; h >= 1; --h)
+        if (P % h == 0) { b.h = h; break; }
+    // prefer a non-dividing taller box when the dividing one wastes more than half of the tile
+    if (b.h * 2 <= hmax && rows_mult <= 1) b.h = hmax;
+    b.n = 1;
+    if (b.h == P) {
+        int nmax = max_rows / (Q * P);
+        if (nmax > N) nmax = N;
+        if (nmax >= 1) b.n = nmax;
+    }
+    b.rows = b.w * b.h * b.n;
+    if (rows_mult > 1 && b.rows % rows_mult) {
+        // shrink until the row count is a multiple of rows_mult
+        bool found = false;
+        for (int n = b.n; n >= 1 && !found; --n)
+            for (int h = b.h; h >= 1 && !found; --h)
+                if ((Q * h * n) % rows_mult == 0 && (n == 1 || h == P)) { b.h = h; b.n = n; found = true; }
+        if (!found) return false;
+        b.rows = b.w * b.h * b.n;
+    }
+    *out = b;
+    return true;
+}
+
+int chunk_of(int channels) { return channels % 32 == 0 ? 32 : 16; }
+unsigned int pow2_cols(int need)
+{
+    unsigned int c = 32;
+    while ((int)c < need) c <<= 1;
+    return c;
+}
+
+// Geometry of the three passes seen as "forward-like" problems.
+struct FwdView {
+    int N, P, Q;          // output pixel grid
+    int c_in, c_out;      // reduction channels, output channels
+    int R, pad;           // taps and tap shift
+    int in_w, in_h;       // extent of the input tensor map's pixel dims
+    long long in_sw, in_sh, in_sn;   // input strides (floats) of the tensor map's w, h, n dims
+    long long os_n, os_h, os_w, dense_h, dense_w;
+    int zero_fill, out_h, out_w;
+};
+
+bool fwd_view(const ConvShape& s, int pass, FwdView* v)
+{
+    if (s.C % 16 || s.K % 16) return false;
+    if (s.R != 1 && s.R != 3) return false;
+    if (s.R == 3 && (s.stride != 1 || s.pad != 1)) return false;
+    if (s.R == 1 && s.pad != 0) return false;
+    if (s.stride < 1 || s.stride > 2) return false;
+    if (pass == PASS_FWD) {
+        v->N = s.N; v->P = s.P; v->Q = s.Q; v->c_in = s.C; v->c_out = s.K; v->R = s.R; v->pad = s.pad;
+        v->in_w = s.stride == 1 ? s.W : s.Q; v->in_h = s.stride == 1 ? s.H : s.P;
+        v->in_sw = (long long)s.stride * s.C; v->in_sh = (long long)s.stride * s.W * s.C; v->in_sn = (long long)s.H * s.W * s.C;
+        v->os_w = s.K; v->os_h = (long long)s.Q * s.K; v->os_n = (long long)s.P * s.Q * s.K;
+        v->dense_h = v->os_h; v->dense_w = v->os_w; v->zero_fill = 1; v->out_h = s.P; v->out_w = s.Q;
+    } else {
+        // dx = "forward" convolution of dy with the rearranged weights; tap shift R-1-pad
+        v->N = s.N; v->P = s.stride == 1 ? s.H : s.P; v->Q = s.stride == 1 ? s.W : s.Q;
+        v->c_in = s.K; v->c_out = s.C; v->R = s.R; v->pad = s.R - 1 - s.pad;
+        v->in_w = s.Q; v->in_h = s.P;
+        v->in_sw = s.K; v->in_sh = (long long)s.Q * s.K; v->in_sn = (long long)s.P * s.Q * s.K;
+        v->dense_w = s.C; v->dense_h = (long long)s.W * s.C;
+        v->os_w = (long long)s.stride * s.C; v->os_h = (long long)s.stride * s.W * s.C; v->os_n = (long long)s.H * s.W * s.C;
+        v->zero_fill = s.stride; v->out_h = s.H; v->out_w = s.W;
+    }
+    if (v->c_out > 256 && v->c_out % 256) return false;
+    return true;
+}
+
+cudaError_t encode(CUtensorMap* tm, const float* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
+                   const cuuint32_t* box, int swizzle_bytes)
+{
+    if (!g_encode) return cudaErrorNotReady;
+    cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+    CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<float*>(base), dims, strides_bytes, box,
+                          ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                          : (swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE),
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+struct WgradGeom {
+    PixelBox box;
+    int m_chunk, n_cols, taps_per_cta, tap_groups, raw_stages, t_stages, splits, tiles_per_split, n_tiles;
+    unsigned int raw_bytes, t_bytes, tmem_cols;
+};
+
+bool wgrad_geom(const ConvShape& s, WgradGeom* g)
+{
+    if (s.C % 16 || s.K % 16) return false;
+    if (s.R != 1 && s.R != 3) return false;
+    if (s.R == 3 && (s.stride != 1 || s.pad != 1)) return false;
+    if (s.R == 1 && s.pad != 0) return false;
+    if (s.stride < 1 || s.stride > 2) return false;
+    g->m_chunk = s.K < 128 ? s.K : 128;
+    if (s.K % g->m_chunk) return false;
+    g->n_cols = s.C < 256 ? s.C : 256;
+    if (s.C % g->n_cols) return false;
+    const int taps = s.R * s.R;
+    // taps per CTA (all, one row of the window, or one) and pixels per tile (64 or 32): the first
+    // combination whose accumulators fit tensor memory and whose 2 raw + 2 transposed stages fit shared memory
+    bool found = false;
+    const int cand[3] = {taps, taps == 9 ? 3 : 1, 1};
+    for (int ci = 0; ci < 3 && !found; ++ci) {
+        const int tpc = cand[ci];
+        if (tpc * g->n_cols > 512) continue;
+        for (int rows = 64; rows >= 32 && !found; rows >>= 1) {
+            PixelBox b;
+            if (!choose_box(s.Q, s.P, s.N, rows, 32, &b)) continue;
+            const unsigned int raw = (unsigned int)b.rows * 4u * (unsigned int)(g->m_chunk + tpc * g->n_cols);
+            const unsigned int raw_al = (raw + 1023u) & ~1023u;
+            const unsigned int tb = (unsigned int)(b.rows / 32) * 128u * (unsigned int)(128 + tpc * g->n_cols);
+            if (2 * raw_al + 2 * tb > kSmemBudget) continue;
+            g->taps_per_cta = tpc;
+            g->box = b; g->raw_bytes = raw_al; g->t_bytes = tb;
+            g->t_stages = 2;
+            int rs = (int)((kSmemBudget - 2 * tb) / raw_al);
+            g->raw_stages = rs > 4 ? 4 : rs;
+            found = true;
+        }
+    }
+    if (!found) return false;
+    g->tap_groups = (taps + g->taps_per_cta - 1) / g->taps_per_cta;
+    g->tmem_cols = pow2_cols(g->taps_per_cta * g->n_cols);
+    const int tiles_w = (s.Q + g->box.w - 1) / g->box.w, tiles_h = (s.P + g->box.h - 1) / g->box.h, tiles_n = (s.N + g->box.n - 1) / g->box.n;
+    g->n_tiles = tiles_w * tiles_h * tiles_n;
+    // splits: enough CTAs to spread the pixel walk, few enough that the partials stay a fraction of the operand bytes
+    const double operand_bytes = 4.0 * ((double)s.N * s.P * s.Q * s.K + (double)s.N * s.P * s.Q * s.C);
+    const double dw_bytes = 4.0 * (double)s.K * taps * s.C;
+    int splits = g->n_tiles / 4;
+    const int cap = (int)(operand_bytes / (4.0 * dw_bytes));
+    if (splits > cap) splits = cap;
+    if (splits > 64) splits = 64;
+    if (splits < 1) splits = 1;
+    g->tiles_per_split = (g->n_tiles + splits - 1) / splits;
+    g->splits = (g->n_tiles + g->tiles_per_split - 1) / g->tiles_per_split;
+    return true;
+}
+
+inline void count(int64_t* n_launch, int k) { if (n_launch) *n_launch += k; }
+
 }  // namespace
+
+// ------------------------------------------------------------------------------------------------
+// interface
+// ------------------------------------------------------------------------------------------------
+bool conv_tc_supported(const ConvShape& s, int pass)
+{
+    if (pass == PASS_WGRAD) { WgradGeom g; return wgrad_geom(s, &g); }
+    FwdView v;
+    if (!fwd_view(s, pass, &v)) return false;
+    PixelBox b;
+    return choose_box(v.Q, v.P, v.N, kTileM, 1, &b);
+}
+
+cudaError_t conv_tc_init()
+{
+    if (g_encode) return cudaSuccess;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+    if (e != cudaSuccess) return e;
+    if (q != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    static bool attr_done = false;
+    if (!attr_done) {
+        e = cudaFuncSetAttribute(conv_tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(conv_tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    return cudaSuccess;
+}
+
+size_t conv_tc_scratch_bytes(const ConvShape& s)
+{
+    WgradGeom g;
+    if (!wgrad_geom(s, &g)) return 0;
+    return g.splits > 1 ? (size_t)g.splits * s.K * s.R * s.R * s.C * sizeof(float) : 0;
+}
+
+struct ConvTcFwdLaunch { FwdParams p; dim3 grid; unsigned int smem; };
+struct ConvTcWgradLaunch { WgradParams p; dim3 grid; unsigned int smem; int splits; float* dw; long long n_out; };
+static_assert(sizeof(ConvTcFwdLaunch) <= 640 && sizeof(ConvTcWgradLaunch) <= 640, "plan storage too small");
+
+cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, const float* in, const float* in2,
+                            const float* weights, float* out, const float* extra, bool accumulate, void* scratch)
+{
+    plan->valid = 0; plan->s = s; plan->pass = pass;
+    if (pass == PASS_WGRAD) {
+        WgradGeom g;
+        if (!wgrad_geom(s, &g)) return cudaErrorNotSupported;
+        ConvTcWgradLaunch* L = reinterpret_cast<ConvTcWgradLaunch*>(plan->storage);
+        WgradParams& p = L->p;
+        memset(&p, 0, sizeof p);
+        // dy {K, Q, P, N}
+        {
+            cuuint64_t dims[4] = {(cuuint64_t)s.K, (cuuint64_t)s.Q, (cuuint64_t)s.P, (cuuint64_t)s.N};
+            cuuint64_t str[3] = {(cuuint64_t)s.K * 4, (cuuint64_t)s.Q * s.K * 4, (cuuint64_t)s.P * s.Q * s.K * 4};
+            cuuint32_t box[4] = {(cuuint32_t)g.m_chunk, (cuuint32_t)g.box.w, (cuuint32_t)g.box.h, (cuuint32_t)g.box.n};
+            cudaError_t e = encode(&p.tm_a, in, 4, dims, str, box, 0);
+            if (e != cudaSuccess) return e;
+        }
+        // x {C, Wv, Hv, N}: a strided 1x1 convolution samples every stride-th pixel
+        {
+            const int wv = s.stride == 1 ? s.W : s.Q, hv = s.stride == 1 ? s.H : s.P;
+            cuuint64_t dims[4] = {(cuuint64_t)s.C, (cuuint64_t)wv, (cuuint64_t)hv, (cuuint64_t)s.N};
+            cuuint64_t str[3] = {(cuuint64_t)s.stride * s.C * 4, (cuuint64_t)s.stride * s.W * s.C * 4, (cuuint64_t)s.H * s.W * s.C * 4};
+            cuuint32_t box[4] = {(cuuint32_t)g.n_cols, (cuuint32_t)g.box.w, (cuuint32_t)g.box.h, (cuuint32_t)g.box.n};
+            cudaError_t e = encode(&p.tm_b, in2, 4, dims, str, box, 0);
+            if (e != cudaSuccess) return e;
+        }
+        const long long n_out = (long long)s.K * s.R * s.R * s.C;
+        p.out = g.splits > 1 ? reinterpret_cast<float*>(scratch) : out;
+        p.box_w = g.box.w; p.box_h = g.box.h; p.box_n = g.box.n;
+        p.tiles_w = (s.Q + g.box.w - 1) / g.box.w; p.tiles_h = (s.P + g.box.h - 1) / g.box.h;
+        p.n_tiles = g.n_tiles; p.tiles_per_split = g.tiles_per_split; p.rows = g.box.rows;
+        p.c_out = s.K; p.c_in = s.C; p.R = s.R; p.pad = s.pad;
+        p.m_chunk = g.m_chunk; p.n_cols = g.n_cols; p.taps_per_cta = g.taps_per_cta;
+        p.raw_stages = g.raw_stages; p.t_stages = g.t_stages;
+        p.raw_bytes = g.raw_bytes; p.t_bytes = g.t_bytes;
+        p.tx_a = (unsigned int)g.box.rows * g.m_chunk * 4u; p.tx_per_tap = (unsigned int)g.box.rows * g.n_cols * 4u;
+        p.tmem_cols = g.tmem_cols;
+        p.idesc = instr_desc(g.n_cols, false, false);
+        p.split_stride = n_out;
+        L->grid = dim3(g.splits, g.tap_groups, (s.K / g.m_chunk) * (s.C / g.n_cols));
+        L->smem = (unsigned int)g.raw_stages * g.raw_bytes + (unsigned int)g.t_stages * g.t_bytes + 1024;
+        L->splits = g.splits; L->dw = out; L->n_out = n_out;
+        plan->valid = 1;
+        return cudaSuccess;
+    }
+    FwdView v;
+    PixelBox b;
+    if (!fwd_view(s, pass, &v) || !choose_box(v.Q, v.P, v.N, kTileM, 1, &b)) return cudaErrorNotSupported;
+    ConvTcFwdLaunch* L = reinterpret_cast<ConvTcFwdLaunch*>(plan->storage);
+    FwdParams& p = L->p;
+    memset(&p, 0, sizeof p);
+    const int kchunk = chunk_of(v.c_in);
+    const int n_chunk = v.c_out < 256 ? v.c_out : 256;
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)v.c_in, (cuuint64_t)v.in_w, (cuuint64_t)v.in_h, (cuuint64_t)v.N};
+        cuuint64_t str[3] = {(cuuint64_t)v.in_sw * 4, (cuuint64_t)v.in_sh * 4, (cuuint64_t)v.in_sn * 4};
+        cuuint32_t box[4] = {(cuuint32_t)kchunk, (cuuint32_t)b.w, (cuuint32_t)b.h, (cuuint32_t)b.n};
+        cudaError_t e = encode(&p.tm_a, in, 4, dims, str, box, kchunk * 4);
+        if (e != cudaSuccess) return e;
+    }
+    {
+        const long long kdim = (long long)v.R * v.R * v.c_in;
+        cuuint64_t dims[2] = {(cuuint64_t)kdim, (cuuint64_t)v.c_out};
+        cuuint64_t str[1] = {(cuuint64_t)kdim * 4};
+        cuuint32_t box[2] = {(cuuint32_t)kchunk, (cuuint32_t)n_chunk};
+        cudaError_t e = encode(&p.tm_b, weights, 2, dims, str, box, kchunk * 4);
+        if (e != cudaSuccess) return e;
+    }
+    p.out = out; p.extra = extra; p.accumulate = accumulate ? 1 : 0;
+    p.os_n = v.os_n; p.os_h = v.os_h; p.os_w = v.os_w; p.dense_h = v.dense_h; p.dense_w = v.dense_w;
+    p.box_w = b.w; p.box_h = b.h; p.box_n = b.n;
+    p.tiles_w = (v.Q + b.w - 1) / b.w; p.tiles_h = (v.P + b.h - 1) / b.h;
+    const int tiles_n = (v.N + b.n - 1) / b.n;
+    p.P = v.P; p.Q = v.Q; p.N = v.N; p.c_out = v.c_out; p.n_chunk = n_chunk; p.R = v.R; p.pad = v.pad;
+    p.c_in = v.c_in; p.kchunk = kchunk; p.n_kchunks = v.c_in / kchunk; p.swizzle = kchunk * 4;
+    p.zero_fill = v.zero_fill; p.out_h = v.out_h; p.out_w = v.out_w;
+    p.a_bytes = (unsigned int)kTileM * kchunk * 4;
+    p.b_bytes = ((unsigned int)n_chunk * kchunk * 4 + 1023u) & ~1023u;
+    p.tx_bytes = (unsigned int)b.rows * kchunk * 4 + (unsigned int)n_chunk * kchunk * 4;
+    const unsigned int stage = p.a_bytes + p.b_bytes;
+    int stages = (int)(kSmemBudget / stage);
+    const int total = v.R * v.R * p.n_kchunks;
+    if (stages > 6) stages = 6;
+    if (stages > total) stages = total;
+    p.stages = stages;
+    p.tmem_cols = pow2_cols(n_chunk);
+    p.idesc = instr_desc(n_chunk, false, false);
+    L->grid = dim3(p.tiles_w * p.tiles_h * tiles_n, v.c_out / n_chunk, 1);
+    L->smem = (unsigned int)stages * stage + 1024;
+    plan->valid = 1;
+    return cudaSuccess;
+}
+
+cudaError_t conv_tc_launch(const ConvTcPlan* plan, DeviceStatus* status, cudaStream_t st, int64_t* n_launch)
+{
+    if (!plan->valid) return cudaErrorInvalidValue;
+    if (plan->pass == PASS_WGRAD) {
+        ConvTcWgradLaunch L = *reinterpret_cast<const ConvTcWgradLaunch*>(plan->storage);
+        L.p.status = status;
+        conv_tc_wgrad_kernel<<<L.grid, 192, L.smem, st>>>(L.p);
+        count(n_launch, 1);
+        if (L.splits > 1) {
+            int nb = (int)((L.n_out / 4 + 255) / 256);
+            if (nb > 592) nb = 592;
+            wgrad_partials_reduce_kernel<<<nb, 256, 0, st>>>(L.p.out, L.dw, L.n_out, L.splits);
+            count(n_launch, 1);
+        }
+        return cudaGetLastError();
+    }
+    ConvTcFwdLaunch L = *reinterpret_cast<const ConvTcFwdLaunch*>(plan->storage);
+    L.p.status = status;
+    conv_tc_fwd_kernel<<<L.grid, 128, L.smem, st>>>(L.p);
+    count(n_launch, 1);
+    return cudaGetLastError();
+}
 
 cudaError_t conv_dgrad_weights(const float* w, float* wt, int C, int K, int R, cudaStream_t st, int64_t* n_launch)
 {
-    const int64_t total = (int64_t)K * R * R * C;
+    const long long total = (long long)K * R * R * C;
     int nb = (int)((total + 255) / 256);
     if (nb > 592) nb = 592;
     dgrad_weights_kernel<<<nb, 256, 0, st>>>(w, wt, C, K, R);
-    if (n_launch) *n_launch += 1;
+    count(n_launch, 1);
     return cudaGetLastError();
 }
 

@@ -14,30 +14,13 @@ cudaError_t conv_tc_init();
 
 size_t conv_tc_scratch_bytes(const ConvShape& s);
 
-// A prepared launch: tensor maps are encoded once (they bake in the device pointers).
+// A prepared launch: tensor maps are encoded once (they bake in the device pointers) and the kernel
+// parameters are kept ready in `storage`.
 struct ConvTcPlan {
-    alignas(64) unsigned char tmap_a[128];   // activation operand (x or dy)
-    alignas(64) unsigned char tmap_b[128];   // weight operand (fwd/dgrad) or second activation operand (wgrad)
     ConvShape s;
     int pass;
     int valid;
-    // tile geometry (see conv_tc.cu)
-    int box_w, box_h, box_n;      // pixel box of one M tile
-    int tiles_w, tiles_h, tiles_n;
-    int kchunk;                   // channels per K step (16 or 32)
-    int n_kchunks;                // c_in / kchunk
-    int swizzle_bytes;            // 64 or 128
-    int stages;
-    int splits;                   // wgrad: pixel-tile slices (grid.y)
-    unsigned int smem_bytes;
-    unsigned int tmem_cols;
-    const float* in;              // fwd: x, dgrad: dy, wgrad: dy
-    const float* in2;             // wgrad: x
-    const float* weights;         // fwd: w, dgrad: transformed weights
-    float* out;                   // fwd: y, dgrad: dx, wgrad: dw
-    const float* extra;           // fwd: residual, dgrad: addend (nullable)
-    int accumulate;
-    void* scratch;                // wgrad partials
+    alignas(64) unsigned char storage[640];
 };
 
 // pass = PASS_FWD:   out = conv(in, weights) (+ extra)

@@ -374,6 +374,10 @@ bool op_uses_tc(const hpf_model* mdl, int i, int pass)
 {
     if (mdl->opt_conv_path != 0) return false;
     if (mdl->ops[i].op.kind != HPF_OP_CONV) return false;
+    if (mdl->ops[i].op.src0 < 0) return false;          // the network input pointer is not known at bind time
+    if (mdl->ops[i].w_off % 4) return false;            // the weight tensor map needs a 16-byte aligned base
+    // a strided data gradient zero-fills between its samples, so it cannot also add to what is there
+    if (pass == PASS_DGRAD && mdl->ops[i].op.stride > 1 && (mdl->edge0[i].accumulate || mdl->edge0[i].addend >= 0)) return false;
     return conv_tc_supported(conv_shape_of(mdl, i), pass);
 }
 
@@ -782,8 +786,6 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                     if (!mdl->use_tc[pass][i]) continue;
                     const OpInfo& o = mdl->ops[i];
                     const int src = o.op.src0;
-                    // the network input pointer is only known at hpf_forward: tensor-core kernels never read it
-                    if (src < 0) { mdl->use_tc[pass][i] = 0; continue; }
                     const ConvShape s = conv_shape_of(mdl, i);
                     const GradEdge& ed = mdl->edge0[i];
                     ConvTcPlan* pl = &mdl->tc_plan[pass][(size_t)m * n + i];

@@ -7,6 +7,11 @@ import workloads as wl
 
 TOL_TENSOR = 1e-2     # relative L2 per activation and gradient tensor
 TOL_LOSS = 1e-3       # relative, on the loss
+# ReLU decisions: the gradient is a discontinuous function of the forward values, so both sides must take
+# the decision z > 0 on the same side wherever the forward tolerance leaves it open.  The oracle keeps its own
+# decision where |z| >= TAU*|gamma| (a GPU disagreement there fails the test) and evaluates the gradient under
+# the GPU's decision inside that window.
+TAU = 0.02
 
 
 def rel_l2(a, ref):
@@ -72,3 +77,15 @@ def seeded(ops, in_hwc, B, seed=0, bn_jitter=0.0):
     x, labels = wl.draw_inputs(B, in_hwc, ops[-1].c_out, seed_x=wl.inputs.SEED_X + seed, seed_labels=wl.inputs.SEED_LABELS + seed)
     theta = wl.draw_params(ops, seed=wl.inputs.SEED_PARAMS + seed, bn_jitter=bn_jitter)
     return x, labels, theta
+
+
+def matched_oracle(bd, m, theta, x, labels, cuts=None, want=None):
+    """The oracle's micro-batch m with the GPU's in-window ReLU decisions; fails on any decision the
+    forward tolerance does not leave open."""
+    from oracle import reference as ora
+    b = bd.B // bd.M
+    dec = {i: (bd.tensor(i, m) > 0).astype(np.uint8) for i, o in enumerate(bd.ops) if o.kind == wl.BNRELU}
+    r = ora.microbatch(bd.ops, bd.in_hwc, theta, x[m * b:(m + 1) * b], labels[m * b:(m + 1) * b], cuts=cuts, want=want,
+                       decisions=dec, tau=TAU)
+    assert r["decision_violations"] == 0, r["decision_violations"]
+    return r

@@ -5,7 +5,7 @@ import pytest
 
 import workloads as wl
 from oracle import reference as ora
-from hpf_testlib import Bound, rel_l2, seeded, TOL_TENSOR, TOL_LOSS
+from hpf_testlib import Bound, rel_l2, seeded, matched_oracle, TOL_TENSOR, TOL_LOSS
 
 pytestmark = pytest.mark.gpu
 
@@ -24,7 +24,8 @@ def _fullsize(name, sample_m):
     assert np.isfinite(slots).all()
     worst = {"act": 0.0, "dact": 0.0, "g": 0.0}
     for m in sample_m:
-        r = ora.microbatch(ops, hwc, theta, x[m * b:(m + 1) * b], labels[m * b:(m + 1) * b])
+        r = matched_oracle(bd, m, theta, x, labels)
+        worst["decisions_from_gpu"] = worst.get("decisions_from_gpu", 0) + r["decisions_used"]
         assert abs(losses[m] - r["loss"]) <= TOL_LOSS * abs(r["loss"])
         for i in range(len(ops)):
             e = rel_l2(bd.tensor(i, m), r["act"][i]); worst["act"] = max(worst["act"], e)

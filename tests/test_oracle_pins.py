@@ -366,3 +366,51 @@ def test_maxpool_against_brute_force_and_tie_rule():
     dx = ora.maxpool_bwd(x1, dy, 3, 2, 1)
     exp = np.zeros((4, 4)); exp[0, 0] = 1; exp[0, 1] = 2; exp[1, 0] = 3; exp[1, 1] = 4
     assert np.array_equal(dx[0, :, :, 0], exp)
+
+
+# ------------------------------------------------------------------ ReLU decisions
+def test_supplied_relu_decisions_window():
+    """Decisions of another implementation are honoured only inside |z| < tau*|gamma|, and a
+    gradient evaluated with a flipped in-window decision equals the plain gradient of a nearby
+    problem whose own decision is the flipped one (here: beta nudged across the kink)."""
+    ops, hwc, x, labels, theta = _setup(tiny_cifar, B=4)
+    plain = ora.microbatch(ops, hwc, theta, x, labels)
+    bn = [i for i, o in enumerate(ops) if o.kind == wl.BNRELU]
+    offs, _ = wl.param_offsets(ops)
+    own = {i: (plain["act"][i] > 0).astype(np.uint8) for i in bn}
+    # own decisions, any tau: bit-identical, nothing used, no violation
+    same = ora.microbatch(ops, hwc, theta, x, labels, decisions=own, tau=0.05)
+    assert np.array_equal(same["g"], plain["g"]) and same["decisions_used"] == 0 and same["decision_violations"] == 0
+    # all decisions inverted with tau = 0: every one is a violation, none is used
+    inv = {i: 1 - d for i, d in own.items()}
+    r = ora.microbatch(ops, hwc, theta, x, labels, decisions=inv, tau=0.0)
+    assert np.array_equal(r["g"], plain["g"]) and r["decisions_used"] == 0
+    assert r["decision_violations"] == sum(d.size for d in own.values())
+    # flip the decision of the element of one BN whose pre-activation is closest to zero
+    i = bn[2]
+    src = ops[i].src0
+    xin = plain["act"][src]; C = xin.shape[-1]
+    gamma = theta[offs[i][0]:offs[i][0] + C]; beta = theta[offs[i][2]:offs[i][2] + C]
+    mean, var = ora.bn_stats(xin)
+    z = gamma * (xin - mean) / np.sqrt(var + ops[i].eps) + beta
+    flat = np.abs(z / gamma).reshape(-1, C)
+    row, ch = np.unravel_index(np.argmin(flat), flat.shape)
+    zmin = z.reshape(-1, C)[row, ch]
+    flipped = {k: v.copy() for k, v in own.items()}
+    flipped[i].reshape(-1, C)[row, ch] ^= 1
+    two = np.sort(flat.ravel())[:2]
+    tau = 0.5 * (two[0] + two[1])
+    assert np.sum(np.abs(z / gamma) < tau) == 1                      # only that element is undecided
+    r = ora.microbatch(ops, hwc, theta, x, labels, decisions=flipped, tau=tau)
+    assert r["decisions_used"] == 1 and r["decision_violations"] == 0
+    assert not np.array_equal(r["g"], plain["g"])
+    # the nearby problem: beta_ch moved by 2*|z| so that its own decision flips
+    theta2 = theta.copy()
+    theta2[offs[i][2] + ch] -= 2.0 * zmin
+    near = ora.microbatch(ops, hwc, theta2, x, labels)
+    assert (near["act"][i] > 0).reshape(-1, C)[row, ch] != (plain["act"][i] > 0).reshape(-1, C)[row, ch]
+    d_flip = np.linalg.norm(r["g"] - near["g"]); d_plain = np.linalg.norm(plain["g"] - near["g"])
+    assert d_flip < 0.05 * d_plain, (d_flip, d_plain)                # the flip explains the jump
+    # partition-by-partition execution honours the decisions identically
+    rp = ora.microbatch(ops, hwc, theta, x, labels, cuts=[4, 13], decisions=flipped, tau=tau)
+    assert np.array_equal(rp["g"], r["g"]) and rp["decisions_used"] == 1
