@@ -81,8 +81,10 @@ int hpf_model_destroy(hpf_model *model);
  *   HPF_OPT_GRAPH          1 (default): each phase is captured once into a CUDA graph and replayed;
  *                          0: kernels are enqueued directly on the streams every call.
  *   HPF_OPT_CONV_PATH      0 (default): tensor-core (tcgen05) convolution kernels wherever the shape
- *                          allows, CUDA-core kernels for the rest (3-channel stem, odd channel counts);
- *                          1: CUDA-core kernels everywhere (fp32 FMA; a cross-check, not a fallback).
+ *                          allows, error-compensated three-pass TF32 (fp32-class accuracy), CUDA-core
+ *                          kernels for the rest (3-channel stem, odd channel counts);
+ *                          1: CUDA-core kernels everywhere (fp32 FMA; a cross-check, not a fallback);
+ *                          2: as 0 with a single TF32 pass (11-bit operands; error grows with depth).
  *   HPF_OPT_SINGLE_STREAM  1: all stages on stream 0 (hazard check: results must equal the multi-stream run).
  *   HPF_OPT_KEEP_MESSAGES  1: every partition copies what it receives across a cut (activations forward,
  *                          partial errors backward) into message buffers readable with hpf_message_ptr. */
@@ -152,17 +154,19 @@ int hpf_conv_path_counts(const hpf_model *model, int64_t *n_tensor, int64_t *n_c
 
 /* ---- single kernels on caller buffers (convolution sweep, memory-bound kernel benchmarks) --------
  * All pointers are device pointers, `stream` is a cudaStream_t.  x [N][H][W][C], w [K][R][R][C],
- * y/dy [N][P][Q][K] with P = (H+2*pad-R)/stride+1.  path: 0 = tensor cores when the shape allows
- * (else HPF_ERR_UNSUPPORTED), 1 = CUDA cores.  d_scratch: caller-owned scratch of at least
- * hpf_conv_scratch_bytes(); it is written by the call and holds nothing afterwards. */
+ * y/dy [N][P][Q][K] with P = (H+2*pad-R)/stride+1.  path: 0 = tensor cores, three-pass TF32;
+ * 2 = tensor cores, one TF32 pass (both HPF_ERR_UNSUPPORTED when the shape is outside their reach);
+ * 1 = CUDA cores.  d_scratch: caller-owned scratch of at least hpf_conv_scratch_bytes(); it is written
+ * by the call and holds nothing afterwards.
+ * d_wprep: the weights as the tensor-core kernels read them, 4*K*R*R*C floats written by
+ * hpf_conv_prepare_weights ([hi | lo | rearranged-for-dgrad hi | lo]); ignored (may be NULL) for path 1
+ * and by hpf_conv_wgrad. */
 int hpf_conv_scratch_bytes(int32_t N, int32_t H, int32_t W, int32_t C, int32_t K, int32_t R, int32_t stride,
                            int32_t pad, size_t *bytes);
-int hpf_conv_fwd(const float *d_x, const float *d_w, float *d_y, int32_t N, int32_t H, int32_t W, int32_t C,
-                 int32_t K, int32_t R, int32_t stride, int32_t pad, int32_t path, void *d_scratch, void *stream);
-/* d_wt: the weights rearranged for the data gradient, [C][R][R][K] with the taps rotated by 180 degrees,
- * written by hpf_conv_dgrad_weights (K*R*R*C floats). */
-int hpf_conv_dgrad_weights(const float *d_w, float *d_wt, int32_t C, int32_t K, int32_t R, void *stream);
-int hpf_conv_dgrad(const float *d_dy, const float *d_w, const float *d_wt, float *d_dx, int32_t N, int32_t H,
+int hpf_conv_prepare_weights(const float *d_w, float *d_wprep, int32_t C, int32_t K, int32_t R, void *stream);
+int hpf_conv_fwd(const float *d_x, const float *d_w, const float *d_wprep, float *d_y, int32_t N, int32_t H, int32_t W,
+                 int32_t C, int32_t K, int32_t R, int32_t stride, int32_t pad, int32_t path, void *d_scratch, void *stream);
+int hpf_conv_dgrad(const float *d_dy, const float *d_w, const float *d_wprep, float *d_dx, int32_t N, int32_t H,
                    int32_t W, int32_t C, int32_t K, int32_t R, int32_t stride, int32_t pad, int32_t path,
                    void *d_scratch, void *stream);
 int hpf_conv_wgrad(const float *d_x, const float *d_dy, float *d_dw, int32_t N, int32_t H, int32_t W, int32_t C,

@@ -54,8 +54,8 @@ _SIGNATURES = {
     "hpf_launch_count": [_vp, _pi64],
     "hpf_conv_path_counts": [_vp, _pi64, _pi64],
     "hpf_conv_scratch_bytes": [_i32] * 8 + [C.POINTER(C.c_size_t)],
-    "hpf_conv_fwd": [_vp, _vp, _vp] + [_i32] * 9 + [_vp, _vp],
-    "hpf_conv_dgrad_weights": [_vp, _vp, _i32, _i32, _i32, _vp],
+    "hpf_conv_prepare_weights": [_vp, _vp, _i32, _i32, _i32, _vp],
+    "hpf_conv_fwd": [_vp, _vp, _vp, _vp] + [_i32] * 9 + [_vp, _vp],
     "hpf_conv_dgrad": [_vp, _vp, _vp, _vp] + [_i32] * 9 + [_vp, _vp],
     "hpf_conv_wgrad": [_vp, _vp, _vp] + [_i32] * 9 + [_vp, _vp],
     "hpf_bnrelu_scratch_bytes": [_i64, _i32, C.POINTER(C.c_size_t)],
@@ -221,16 +221,17 @@ def conv_scratch_bytes(N, H, W, Cc, K, R, stride, pad):
     n = C.c_size_t(); _check(lib().hpf_conv_scratch_bytes(N, H, W, Cc, K, R, stride, pad, C.byref(n))); return n.value
 
 
-def conv_fwd(x, w, y, N, H, W, Cc, K, R, stride, pad, path, scratch, stream=None):
-    _check(lib().hpf_conv_fwd(_ptr(x), _ptr(w), _ptr(y), N, H, W, Cc, K, R, stride, pad, path, _ptr(scratch), _stream(stream)))
+def conv_prepare_weights(w, wprep, Cc, K, R, stream=None):
+    _check(lib().hpf_conv_prepare_weights(_ptr(w), _ptr(wprep), Cc, K, R, _stream(stream)))
 
 
-def conv_dgrad_weights(w, wt, Cc, K, R, stream=None):
-    _check(lib().hpf_conv_dgrad_weights(_ptr(w), _ptr(wt), Cc, K, R, _stream(stream)))
+def conv_fwd(x, w, wprep, y, N, H, W, Cc, K, R, stride, pad, path, scratch, stream=None):
+    _check(lib().hpf_conv_fwd(_ptr(x), _ptr(w), _ptr(wprep), _ptr(y), N, H, W, Cc, K, R, stride, pad, path, _ptr(scratch),
+                              _stream(stream)))
 
 
-def conv_dgrad(dy, w, wt, dx, N, H, W, Cc, K, R, stride, pad, path, scratch, stream=None):
-    _check(lib().hpf_conv_dgrad(_ptr(dy), _ptr(w), _ptr(wt), _ptr(dx), N, H, W, Cc, K, R, stride, pad, path,
+def conv_dgrad(dy, w, wprep, dx, N, H, W, Cc, K, R, stride, pad, path, scratch, stream=None):
+    _check(lib().hpf_conv_dgrad(_ptr(dy), _ptr(w), _ptr(wprep), _ptr(dx), N, H, W, Cc, K, R, stride, pad, path,
                                 _ptr(scratch), _stream(stream)))
 
 

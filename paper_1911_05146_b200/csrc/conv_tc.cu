@@ -19,6 +19,15 @@
 //   One CTA walks a slice of the pixel tiles, keeps one accumulator per tap in tensor memory, and
 //   writes a partial; a second kernel adds the partials in fixed order.
 //
+// Precision.  One TF32 pass keeps 11 significand bits of each operand; through a thousand layers that error
+// grows past the parity tolerance (measured: 3e-2 relative at depth 1001).  The default is therefore the
+// error-compensated three-pass form: every operand is split x = hi + lo with hi = x with its low 13 significand
+// bits cleared (exactly representable in TF32) and lo = x - hi, and the product is accumulated as
+// hi*hi + lo*hi + hi*lo in the fp32 accumulator (the dropped lo*lo term is below 2^-22).  Weights are split once
+// per step by a preparation kernel; activation tiles are split in shared memory by four warps between the TMA
+// arrival and the MMA (the weight gradient's transposing warps do it in the same pass).  The paths are
+// HBM/latency bound, so the extra tensor work is hidden.  A one-pass mode remains selectable.
+//
 // Every wait on an mbarrier is bounded: after the limit the kernel records where it gave up in the
 // device status word, stops issuing work, waits (bounded) for its TMA copies in flight, frees its
 // tensor memory and returns.
@@ -160,7 +169,8 @@ __device__ __forceinline__ void report(DeviceStatus* status, unsigned int code)
 // ------------------------------------------------------------------------------------------------
 struct alignas(64) FwdParams {
     CUtensorMap tm_a;            // activations {C, Wv, Hv, N}
-    CUtensorMap tm_b;            // weights {taps*C, c_out}
+    CUtensorMap tm_b;            // weights, hi part {taps*C, c_out}
+    CUtensorMap tm_b_lo;         // weights, lo part (three-pass mode)
     float* out;
     const float* extra;
     DeviceStatus* status;
@@ -174,9 +184,10 @@ struct alignas(64) FwdParams {
     int c_in, kchunk, n_kchunks;
     int swizzle;
     int stages;
+    int passes;                  // 1 or 3
     int zero_fill;               // > 1: the output pixel grid is strided, fill the rest of each patch with zeros
     int out_h, out_w;            // dense output extent (zero fill bounds)
-    unsigned int a_bytes, b_bytes, tx_bytes, tmem_cols, idesc;
+    unsigned int a_bytes, b_bytes, stage_bytes, tx_bytes, tmem_cols, idesc;
 };
 
 struct alignas(64) WgradParams {
@@ -191,25 +202,41 @@ struct alignas(64) WgradParams {
     int n_cols;                  // input channels per CTA (<= 256)
     int taps_per_cta;
     int raw_stages, t_stages;
+    int passes;                  // 1 or 3
     unsigned int raw_bytes, t_bytes, tx_per_tap, tx_a, tmem_cols, idesc;
     long long split_stride;      // floats between partials
 };
 
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// x = hi + lo, hi = x with the low 13 significand bits cleared (what a TF32 operand keeps)
+__device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+
 // ------------------------------------------------------------------------------------------------
-// forward / data-gradient kernel
+// forward / data-gradient kernel: 6 warps = TMA producer, MMA issuer, 4 splitter / epilogue warps
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128) conv_tc_fwd_kernel(const __grid_constant__ FwdParams p)
+__global__ void __launch_bounds__(192) conv_tc_fwd_kernel(const __grid_constant__ FwdParams p)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[2 * 8 + 1];
+    __shared__ uint64_t bars[3 * 8 + 1];       // full[8], empty[8], split[8], accum
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int issued, consumed;
 
-    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t stage_bytes = p.a_bytes + p.b_bytes;
+    const uint32_t base_off = ((smem_u32(smem_raw) + 1023u) & ~1023u) - smem_u32(smem_raw);
+    uint8_t* smem = smem_raw + base_off;
+    const uint32_t smem_base = smem_u32(smem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[8]), accum_bar = smem_u32(&bars[16]);
+    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[8]), split0 = smem_u32(&bars[16]),
+                   accum_bar = smem_u32(&bars[24]);
+    // stage layout: A | A_lo | B_hi | B_lo   (the lo parts only in three-pass mode)
+    const uint32_t off_alo = p.a_bytes;
+    const uint32_t off_b = p.passes == 3 ? 2 * p.a_bytes : p.a_bytes;
+    const uint32_t off_blo = off_b + p.b_bytes;
 
     int t = blockIdx.x;
     const int tw = t % p.tiles_w; t /= p.tiles_w;
@@ -219,7 +246,7 @@ __global__ void __launch_bounds__(128) conv_tc_fwd_kernel(const __grid_constant_
     const int co0 = blockIdx.y * p.n_chunk;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); mbar_init(split0 + 8 * s, 4); }
         mbar_init(accum_bar, 1);
         abort_flag = 0; issued = 0; consumed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -231,76 +258,110 @@ __global__ void __launch_bounds__(128) conv_tc_fwd_kernel(const __grid_constant_
     const uint32_t tmem_base = tmem_slot;
     const int total = p.R * p.R * p.n_kchunks;
 
-    if (warp == 0 && lane == 0) {
-        // ---- TMA producer ----
-        int it = 0;
-        for (; it < total; ++it) {
-            const int s = it % p.stages;
-            if (!mbar_wait(empty0 + 8 * s, ((it / p.stages) & 1) ^ 1, &abort_flag)) { report(p.status, 1); break; }
-            const int tap = it / p.n_kchunks, kc = it % p.n_kchunks;
-            const int r = tap / p.R, sx = tap % p.R;
-            const uint32_t a_dst = smem_base + s * stage_bytes, b_dst = a_dst + p.a_bytes;
-            mbar_expect_tx(full0 + 8 * s, p.tx_bytes);
-            tma_load_4d(a_dst, &p.tm_a, full0 + 8 * s, kc * p.kchunk, q0 + sx - p.pad, p0 + r - p.pad, n0);
-            tma_load_2d(b_dst, &p.tm_b, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- TMA producer ----
+            int it = 0;
+            for (; it < total; ++it) {
+                const int s = it % p.stages;
+                if (!mbar_wait(empty0 + 8 * s, ((it / p.stages) & 1) ^ 1, &abort_flag)) { report(p.status, 1); break; }
+                const int tap = it / p.n_kchunks, kc = it % p.n_kchunks;
+                const int r = tap / p.R, sx = tap % p.R;
+                const uint32_t dst = smem_base + s * p.stage_bytes;
+                mbar_expect_tx(full0 + 8 * s, p.tx_bytes);
+                tma_load_4d(dst, &p.tm_a, full0 + 8 * s, kc * p.kchunk, q0 + sx - p.pad, p0 + r - p.pad, n0);
+                tma_load_2d(dst + off_b, &p.tm_b, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
+                if (p.passes == 3) tma_load_2d(dst + off_blo, &p.tm_b_lo, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
+            }
+            issued = it;
         }
-        issued = it;
-    } else if (warp == 1 && lane == 0) {
-        // ---- MMA issuer ----
-        const uint32_t sbo = 8u * (uint32_t)p.kchunk * 4u;          // 8 rows of one swizzle atom
-        int it = 0;
-        for (; it < total; ++it) {
-            const int s = it % p.stages;
-            if (!mbar_wait(full0 + 8 * s, (it / p.stages) & 1, &abort_flag)) { report(p.status, 2); break; }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- MMA issuer ----
+            const uint32_t sbo = 8u * (uint32_t)p.kchunk * 4u;          // 8 rows of one swizzle atom
+            int it = 0;
+            for (; it < total; ++it) {
+                const int s = it % p.stages;
+                const uint32_t par = (it / p.stages) & 1;
+                if (!mbar_wait(full0 + 8 * s, par, &abort_flag)) { report(p.status, 2); break; }
+                if (p.passes == 3 && !mbar_wait(split0 + 8 * s, par, &abort_flag)) { report(p.status, 6); break; }
+                tc_fence_after();
+                const uint32_t st = smem_base + s * p.stage_bytes;
+                for (int k8 = 0; k8 < p.kchunk / 8; ++k8) {
+                    const uint64_t ad = smem_desc(st + 32u * k8, 16, sbo, p.swizzle);
+                    const uint64_t bd = smem_desc(st + off_b + 32u * k8, 16, sbo, p.swizzle);
+                    umma_tf32(tmem_base, ad, bd, p.idesc, (it | k8) ? 1u : 0u);
+                    if (p.passes == 3) {
+                        const uint64_t adl = smem_desc(st + off_alo + 32u * k8, 16, sbo, p.swizzle);
+                        const uint64_t bdl = smem_desc(st + off_blo + 32u * k8, 16, sbo, p.swizzle);
+                        umma_tf32(tmem_base, adl, bd, p.idesc, 1u);
+                        umma_tf32(tmem_base, ad, bdl, p.idesc, 1u);
+                    }
+                }
+                umma_commit(empty0 + 8 * s);     // frees the stage once these MMAs have read it
+            }
+            consumed = it;
+            if (it == total) umma_commit(accum_bar);
+        }
+    } else {
+        // ---- warps 2..5: split the activation tile into hi / lo, then the epilogue ----
+        const int tid = threadIdx.x - 64;
+        bool ok = true;
+        if (p.passes == 3) {
+            const int n4 = (int)(p.a_bytes >> 4);
+            for (int it = 0; it < total; ++it) {
+                const int s = it % p.stages;
+                ok = mbar_wait(full0 + 8 * s, (it / p.stages) & 1, &abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) { if (lane == 0) report(p.status, 7); break; }
+                float4* a = reinterpret_cast<float4*>(smem + s * p.stage_bytes);
+                float4* alo = reinterpret_cast<float4*>(smem + s * p.stage_bytes + off_alo);
+                for (int i = tid; i < n4; i += 128) {
+                    const float4 v = a[i];
+                    const float4 h = make_float4(tf32_hi(v.x), tf32_hi(v.y), tf32_hi(v.z), tf32_hi(v.w));
+                    a[i] = h;
+                    alo[i] = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
+                }
+                fence_async_smem();               // generic-proxy writes -> tensor-core reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(split0 + 8 * s);
+            }
+        }
+        bool done = ok && mbar_wait(accum_bar, 0, &abort_flag);
+        done = __all_sync(0xffffffffu, done);
+        if (done) {
             tc_fence_after();
-            const uint32_t a_src = smem_base + s * stage_bytes, b_src = a_src + p.a_bytes;
-            for (int k8 = 0; k8 < p.kchunk / 8; ++k8) {
-                const uint64_t ad = smem_desc(a_src + 32u * k8, 16, sbo, p.swizzle);
-                const uint64_t bd = smem_desc(b_src + 32u * k8, 16, sbo, p.swizzle);
-                umma_tf32(tmem_base, ad, bd, p.idesc, (it | k8) ? 1u : 0u);
-            }
-            umma_commit(empty0 + 8 * s);     // frees the stage once these MMAs have read it
-        }
-        consumed = it;
-        if (it == total) umma_commit(accum_bar);
-    }
-
-    // ---- epilogue: all four warps, warp w owns TMEM lanes [32w, 32w+32) ----
-    __syncwarp();
-    bool ok = mbar_wait(accum_bar, 0, &abort_flag);
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
-        tc_fence_after();
-        const int row = threadIdx.x;
-        const int wi = row % p.box_w, hi = (row / p.box_w) % p.box_h, ni = row / (p.box_w * p.box_h);
-        const int q = q0 + wi, pp = p0 + hi, n = n0 + ni;
-        const bool valid = ni < p.box_n && q < p.Q && pp < p.P && n < p.N;
-        float* orow = p.out + n * p.os_n + pp * p.os_h + q * p.os_w + co0;
-        const float* erow = p.extra ? p.extra + (n * p.os_n + pp * p.os_h + q * p.os_w + co0) : nullptr;
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
-        for (int c0 = 0; c0 < p.n_chunk; c0 += 16) {
-            float v[16];
-            tmem_ld16(lane_addr + (uint32_t)c0, v);
-            if (valid) {
+            const int row = (warp & 3) * 32 + lane;          // TMEM lane = pixel within the tile
+            const int wi = row % p.box_w, hi = (row / p.box_w) % p.box_h, ni = row / (p.box_w * p.box_h);
+            const int q = q0 + wi, pp = p0 + hi, n = n0 + ni;
+            const bool valid = ni < p.box_n && q < p.Q && pp < p.P && n < p.N;
+            float* orow = p.out + n * p.os_n + pp * p.os_h + q * p.os_w + co0;
+            const float* erow = p.extra ? p.extra + (n * p.os_n + pp * p.os_h + q * p.os_w + co0) : nullptr;
+            const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+            for (int c0 = 0; c0 < p.n_chunk; c0 += 16) {
+                float v[16];
+                tmem_ld16(lane_addr + (uint32_t)c0, v);
+                if (valid) {
 #pragma unroll
-                for (int j = 0; j < 16; j += 4) {
-                    float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                    if (erow) { const float4 e = __ldg(reinterpret_cast<const float4*>(erow + c0 + j)); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
-                    if (p.accumulate) { const float4 e = *reinterpret_cast<const float4*>(orow + c0 + j); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
-                    *reinterpret_cast<float4*>(orow + c0 + j) = o;
+                    for (int j = 0; j < 16; j += 4) {
+                        float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        if (erow) { const float4 e = __ldg(reinterpret_cast<const float4*>(erow + c0 + j)); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+                        if (p.accumulate) { const float4 e = *reinterpret_cast<const float4*>(orow + c0 + j); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+                        *reinterpret_cast<float4*>(orow + c0 + j) = o;
+                    }
                 }
             }
-        }
-        if (p.zero_fill > 1 && valid) {
-            // strided data gradient: the positions between the samples receive no contribution
-            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int dy = 0; dy < p.zero_fill; ++dy)
-                for (int dx = 0; dx < p.zero_fill; ++dx) {
-                    if ((dy | dx) == 0) continue;
-                    if (pp * p.zero_fill + dy >= p.out_h || q * p.zero_fill + dx >= p.out_w) continue;
-                    float* zr = orow + dy * p.dense_h + dx * p.dense_w;
-                    for (int c0 = 0; c0 < p.n_chunk; c0 += 4) *reinterpret_cast<float4*>(zr + c0) = z;
-                }
+            if (p.zero_fill > 1 && valid) {
+                // strided data gradient: the positions between the samples receive no contribution
+                const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int dy = 0; dy < p.zero_fill; ++dy)
+                    for (int dx = 0; dx < p.zero_fill; ++dx) {
+                        if ((dy | dx) == 0) continue;
+                        if (pp * p.zero_fill + dy >= p.out_h || q * p.zero_fill + dx >= p.out_w) continue;
+                        float* zr = orow + dy * p.dense_h + dx * p.dense_w;
+                        for (int c0 = 0; c0 < p.n_chunk; c0 += 4) *reinterpret_cast<float4*>(zr + c0) = z;
+                    }
+            }
         }
     }
 
@@ -322,14 +383,13 @@ __global__ void __launch_bounds__(128) conv_tc_fwd_kernel(const __grid_constant_
 // ------------------------------------------------------------------------------------------------
 // weight-gradient kernel: 6 warps = TMA producer, MMA issuer, 4 transposer / epilogue warps
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
 // raw [rows][channels] (dense) -> K-major: channel rows of 128 bytes (32 pixels), 16-byte chunks XOR-swizzled by
-// (row % 8), further groups of 32 pixels `atom_stride` bytes apart.  128 threads.
-__device__ __forceinline__ void transpose_tile(const uint8_t* raw, uint8_t* dst, int channels, int rows, uint32_t atom_stride, int tid)
+// (row % 8), further groups of 32 pixels `atom_stride` bytes apart.  With SPLIT the hi part goes to dst and the
+// lo part to dst_lo.  128 threads; per 4 pixels a thread issues 4 conflict-free 32-bit loads and one (two)
+// conflict-free 128-bit store(s).
+template <bool SPLIT>
+__device__ __forceinline__ void transpose_tile(const uint8_t* raw, uint8_t* dst, uint8_t* dst_lo, int channels, int rows,
+                                               uint32_t atom_stride, int tid)
 {
     const int items = channels * (rows >> 2);
     for (int it = tid; it < items; it += 128) {
@@ -337,8 +397,14 @@ __device__ __forceinline__ void transpose_tile(const uint8_t* raw, uint8_t* dst,
         const float* src = reinterpret_cast<const float*>(raw) + (p4 * 4) * channels + c;
         float4 v;
         v.x = src[0]; v.y = src[channels]; v.z = src[2 * channels]; v.w = src[3 * channels];
-        uint8_t* d = dst + (uint32_t)(p4 >> 3) * atom_stride + (uint32_t)c * 128u + (uint32_t)(((p4 & 7) ^ (c & 7)) << 4);
-        *reinterpret_cast<float4*>(d) = v;
+        const uint32_t o = (uint32_t)(p4 >> 3) * atom_stride + (uint32_t)c * 128u + (uint32_t)(((p4 & 7) ^ (c & 7)) << 4);
+        if (SPLIT) {
+            const float4 h = make_float4(tf32_hi(v.x), tf32_hi(v.y), tf32_hi(v.z), tf32_hi(v.w));
+            *reinterpret_cast<float4*>(dst + o) = h;
+            *reinterpret_cast<float4*>(dst_lo + o) = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
+        } else {
+            *reinterpret_cast<float4*>(dst + o) = v;
+        }
     }
 }
 
@@ -374,6 +440,8 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
     const uint32_t raw_a = (uint32_t)p.rows * p.m_chunk * 4u, raw_b = (uint32_t)p.rows * p.n_cols * 4u;
     const uint32_t t_a = (uint32_t)katoms * 128u * 128u;                  // room for 128 channel rows
     const uint32_t t_b = (uint32_t)katoms * (uint32_t)p.n_cols * 128u;
+    // transposed stage layout: A_hi | B_hi[taps] | A_lo | B_lo[taps]
+    const uint32_t t_half = t_a + (uint32_t)p.taps_per_cta * t_b;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 4; ++s) {
@@ -425,9 +493,18 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
                 for (int tp = 0; tp < ntaps; ++tp)
                     for (int kb = 0; kb < katoms; ++kb)
                         for (int k8 = 0; k8 < 4; ++k8) {
-                            const uint64_t ad = smem_desc(a_src + (uint32_t)kb * 16384u + 32u * k8, 16, 1024, 128);
-                            const uint64_t bd = smem_desc(b_src + (uint32_t)tp * t_b + (uint32_t)kb * (uint32_t)p.n_cols * 128u + 32u * k8, 16, 1024, 128);
-                            umma_tf32(tmem_base + (uint32_t)(tp * p.n_cols), ad, bd, p.idesc, (it | kb | k8) ? 1u : 0u);
+                            const uint32_t ao = (uint32_t)kb * 16384u + 32u * k8;
+                            const uint32_t bo = (uint32_t)tp * t_b + (uint32_t)kb * (uint32_t)p.n_cols * 128u + 32u * k8;
+                            const uint64_t ad = smem_desc(a_src + ao, 16, 1024, 128);
+                            const uint64_t bd = smem_desc(b_src + bo, 16, 1024, 128);
+                            const uint32_t acc = tmem_base + (uint32_t)(tp * p.n_cols);
+                            umma_tf32(acc, ad, bd, p.idesc, (it | kb | k8) ? 1u : 0u);
+                            if (p.passes == 3) {
+                                const uint64_t adl = smem_desc(a_src + t_half + ao, 16, 1024, 128);
+                                const uint64_t bdl = smem_desc(b_src + t_half + bo, 16, 1024, 128);
+                                umma_tf32(acc, adl, bd, p.idesc, 1u);
+                                umma_tf32(acc, ad, bdl, p.idesc, 1u);
+                            }
                         }
                 umma_commit(empty_t0 + 8 * t);
             }
@@ -446,10 +523,18 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
             if (!ok) { if (lane == 0) report(p.status, 5); break; }
             const uint8_t* raw = smem + s * p.raw_bytes;
             uint8_t* tdst = smem + t_region0 + t * p.t_bytes;
-            transpose_tile(raw, tdst, p.m_chunk, p.rows, 16384u, tid);
-            for (int tp = 0; tp < ntaps; ++tp)
-                transpose_tile(raw + raw_a + tp * raw_b, tdst + t_a + tp * t_b, p.n_cols, p.rows, (uint32_t)p.n_cols * 128u, tid);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes -> MMA reads
+            if (p.passes == 3) {
+                transpose_tile<true>(raw, tdst, tdst + t_half, p.m_chunk, p.rows, 16384u, tid);
+                for (int tp = 0; tp < ntaps; ++tp)
+                    transpose_tile<true>(raw + raw_a + tp * raw_b, tdst + t_a + tp * t_b, tdst + t_half + t_a + tp * t_b, p.n_cols,
+                                         p.rows, (uint32_t)p.n_cols * 128u, tid);
+            } else {
+                transpose_tile<false>(raw, tdst, nullptr, p.m_chunk, p.rows, 16384u, tid);
+                for (int tp = 0; tp < ntaps; ++tp)
+                    transpose_tile<false>(raw + raw_a + tp * raw_b, tdst + t_a + tp * t_b, nullptr, p.n_cols, p.rows,
+                                          (uint32_t)p.n_cols * 128u, tid);
+            }
+            fence_async_smem();     // generic-proxy writes -> tensor-core reads
             __syncwarp();
             if (lane == 0) { mbar_arrive(full_t0 + 8 * t); mbar_arrive(empty_raw0 + 8 * s); }
         }
@@ -513,19 +598,41 @@ wgrad_partials_reduce_kernel(const float* __restrict__ partials, float* __restri
     }
 }
 
-__global__ void __launch_bounds__(256) dgrad_weights_kernel(const float* __restrict__ w, float* __restrict__ wt, int C, int K, int R)
+// Weight preparation, once per step: for every convolution of the table (or the one passed by value), the hi / lo split of the weights
+// ([K][R][R][C], forward operand) and of the weights rearranged for the data gradient
+// (wt[c][R-1-r][R-1-s][k] = w[k][r][s][c]).  blockIdx.x = table entry, blockIdx.y strides over its elements.
+__device__ __forceinline__ void weight_prep_one(const float* __restrict__ params, float* __restrict__ w_hi, float* __restrict__ w_lo,
+                                                float* __restrict__ wt_hi, float* __restrict__ wt_lo, const WeightPrepEntry e)
 {
+    const int C = e.C, K = e.K, R = e.R;
     const long long total = (long long)K * R * R * C;
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += stride) {
+    const long long stride = (long long)gridDim.y * blockDim.x;
+    const float* w = params + e.w_off;
+    for (long long o = (long long)blockIdx.y * blockDim.x + threadIdx.x; o < total; o += stride) {
         // o indexes wt[c][r'][s'][k]
         const int k = (int)(o % K);
         long long t = o / K;
         const int s2 = (int)(t % R); t /= R;
         const int r2 = (int)(t % R);
         const int c = (int)(t / R);
-        wt[o] = __ldg(&w[(((long long)k * R + (R - 1 - r2)) * R + (R - 1 - s2)) * C + c]);
+        const long long src = (((long long)k * R + (R - 1 - r2)) * R + (R - 1 - s2)) * C + c;
+        const float v = __ldg(&w[src]);
+        const float h = tf32_hi(v);
+        wt_hi[e.w_off + o] = h; wt_lo[e.w_off + o] = v - h;
+        w_hi[e.w_off + src] = h; w_lo[e.w_off + src] = v - h;
     }
+}
+__global__ void __launch_bounds__(256)
+weight_prep_kernel(const float* __restrict__ params, float* __restrict__ w_hi, float* __restrict__ w_lo,
+                   float* __restrict__ wt_hi, float* __restrict__ wt_lo, const WeightPrepEntry* __restrict__ table)
+{
+    weight_prep_one(params, w_hi, w_lo, wt_hi, wt_lo, table[blockIdx.x]);
+}
+__global__ void __launch_bounds__(256)
+weight_prep_single_kernel(const float* __restrict__ w, float* __restrict__ w_hi, float* __restrict__ w_lo,
+                          float* __restrict__ wt_hi, float* __restrict__ wt_lo, WeightPrepEntry e)
+{
+    weight_prep_one(w, w_hi, w_lo, wt_hi, wt_lo, e);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -574,7 +681,7 @@ unsigned int pow2_cols(int need)
     return c;
 }
 
-// Geometry of the three passes seen as "forward-like" problems.
+// Geometry of the forward pass and of the data gradient seen as a forward-like problem.
 struct FwdView {
     int N, P, Q;          // output pixel grid
     int c_in, c_out;      // reduction channels, output channels
@@ -631,7 +738,7 @@ struct WgradGeom {
     unsigned int raw_bytes, t_bytes, tmem_cols;
 };
 
-bool wgrad_geom(const ConvShape& s, WgradGeom* g)
+bool wgrad_geom(const ConvShape& s, int passes, WgradGeom* g)
 {
     if (s.C % 16 || s.K % 16) return false;
     if (s.R != 1 && s.R != 3) return false;
@@ -640,29 +747,35 @@ bool wgrad_geom(const ConvShape& s, WgradGeom* g)
     if (s.stride < 1 || s.stride > 2) return false;
     g->m_chunk = s.K < 128 ? s.K : 128;
     if (s.K % g->m_chunk) return false;
-    g->n_cols = s.C < 256 ? s.C : 256;
-    if (s.C % g->n_cols) return false;
     const int taps = s.R * s.R;
-    // taps per CTA (all, one row of the window, or one) and pixels per tile (64 or 32): the first
-    // combination whose accumulators fit tensor memory and whose 2 raw + 2 transposed stages fit shared memory
+    const unsigned int parts = passes == 3 ? 2u : 1u;
+    // input channels per CTA (all up to 256, else 128 or 64), taps per CTA (all, one row of the window, or one)
+    // and pixels per tile (64 or 32): the first combination whose accumulators fit tensor memory and whose
+    // 2 raw + 2 transposed stages fit shared memory
     bool found = false;
+    const int ncand[3] = {s.C < 256 ? s.C : 256, 128, 64};
     const int cand[3] = {taps, taps == 9 ? 3 : 1, 1};
-    for (int ci = 0; ci < 3 && !found; ++ci) {
-        const int tpc = cand[ci];
-        if (tpc * g->n_cols > 512) continue;
-        for (int rows = 64; rows >= 32 && !found; rows >>= 1) {
-            PixelBox b;
-            if (!choose_box(s.Q, s.P, s.N, rows, 32, &b)) continue;
-            const unsigned int raw = (unsigned int)b.rows * 4u * (unsigned int)(g->m_chunk + tpc * g->n_cols);
-            const unsigned int raw_al = (raw + 1023u) & ~1023u;
-            const unsigned int tb = (unsigned int)(b.rows / 32) * 128u * (unsigned int)(128 + tpc * g->n_cols);
-            if (2 * raw_al + 2 * tb > kSmemBudget) continue;
-            g->taps_per_cta = tpc;
-            g->box = b; g->raw_bytes = raw_al; g->t_bytes = tb;
-            g->t_stages = 2;
-            int rs = (int)((kSmemBudget - 2 * tb) / raw_al);
-            g->raw_stages = rs > 4 ? 4 : rs;
-            found = true;
+    for (int ni = 0; ni < 3 && !found; ++ni) {
+        const int n_cols = ncand[ni];
+        if (n_cols > s.C || s.C % n_cols || (ni > 0 && n_cols >= ncand[0])) continue;
+        for (int ci = 0; ci < 3 && !found; ++ci) {
+            const int tpc = cand[ci];
+            if (tpc * n_cols > 512) continue;
+            for (int rows = 64; rows >= 32 && !found; rows >>= 1) {
+                PixelBox b;
+                if (!choose_box(s.Q, s.P, s.N, rows, 32, &b)) continue;
+                const unsigned int raw = (unsigned int)b.rows * 4u * (unsigned int)(g->m_chunk + tpc * n_cols);
+                const unsigned int raw_al = (raw + 1023u) & ~1023u;
+                const unsigned int tb = parts * (unsigned int)(b.rows / 32) * 128u * (unsigned int)(128 + tpc * n_cols);
+                if (2 * raw_al + 2 * tb > kSmemBudget) continue;
+                g->n_cols = n_cols;
+                g->taps_per_cta = tpc;
+                g->box = b; g->raw_bytes = raw_al; g->t_bytes = tb;
+                g->t_stages = 2;
+                int rs = (int)((kSmemBudget - 2 * tb) / raw_al);
+                g->raw_stages = rs > 4 ? 4 : rs;
+                found = true;
+            }
         }
     }
     if (!found) return false;
@@ -692,7 +805,7 @@ inline void count(int64_t* n_launch, int k) { if (n_launch) *n_launch += k; }
 // ------------------------------------------------------------------------------------------------
 bool conv_tc_supported(const ConvShape& s, int pass)
 {
-    if (pass == PASS_WGRAD) { WgradGeom g; return wgrad_geom(s, &g); }
+    if (pass == PASS_WGRAD) { WgradGeom g; return wgrad_geom(s, 3, &g); }
     FwdView v;
     if (!fwd_view(s, pass, &v)) return false;
     PixelBox b;
@@ -707,36 +820,39 @@ cudaError_t conv_tc_init()
     cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
     if (e != cudaSuccess) return e;
     if (q != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+    e = cudaFuncSetAttribute(conv_tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(conv_tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
+    if (e != cudaSuccess) return e;
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
-    static bool attr_done = false;
-    if (!attr_done) {
-        e = cudaFuncSetAttribute(conv_tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(conv_tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
     return cudaSuccess;
 }
 
 size_t conv_tc_scratch_bytes(const ConvShape& s)
 {
-    WgradGeom g;
-    if (!wgrad_geom(s, &g)) return 0;
-    return g.splits > 1 ? (size_t)g.splits * s.K * s.R * s.R * s.C * sizeof(float) : 0;
+    size_t need = 0;
+    for (int passes = 1; passes <= 3; passes += 2) {
+        WgradGeom g;
+        if (!wgrad_geom(s, passes, &g)) continue;
+        const size_t b = g.splits > 1 ? (size_t)g.splits * s.K * s.R * s.R * s.C * sizeof(float) : 0;
+        if (b > need) need = b;
+    }
+    return need;
 }
 
 struct ConvTcFwdLaunch { FwdParams p; dim3 grid; unsigned int smem; };
 struct ConvTcWgradLaunch { WgradParams p; dim3 grid; unsigned int smem; int splits; float* dw; long long n_out; };
-static_assert(sizeof(ConvTcFwdLaunch) <= 640 && sizeof(ConvTcWgradLaunch) <= 640, "plan storage too small");
+static_assert(sizeof(ConvTcFwdLaunch) <= sizeof(((ConvTcPlan*)0)->storage) && sizeof(ConvTcWgradLaunch) <= sizeof(((ConvTcPlan*)0)->storage),
+              "plan storage too small");
 
-cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, const float* in, const float* in2,
-                            const float* weights, float* out, const float* extra, bool accumulate, void* scratch)
+cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int passes, const float* in, const float* in2,
+                            const float* w_hi, const float* w_lo, float* out, const float* extra, bool accumulate, void* scratch)
 {
     plan->valid = 0; plan->s = s; plan->pass = pass;
+    if (passes != 1 && passes != 3) return cudaErrorInvalidValue;
     if (pass == PASS_WGRAD) {
         WgradGeom g;
-        if (!wgrad_geom(s, &g)) return cudaErrorNotSupported;
+        if (!wgrad_geom(s, passes, &g)) return cudaErrorNotSupported;
         ConvTcWgradLaunch* L = reinterpret_cast<ConvTcWgradLaunch*>(plan->storage);
         WgradParams& p = L->p;
         memset(&p, 0, sizeof p);
@@ -764,7 +880,7 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, cons
         p.n_tiles = g.n_tiles; p.tiles_per_split = g.tiles_per_split; p.rows = g.box.rows;
         p.c_out = s.K; p.c_in = s.C; p.R = s.R; p.pad = s.pad;
         p.m_chunk = g.m_chunk; p.n_cols = g.n_cols; p.taps_per_cta = g.taps_per_cta;
-        p.raw_stages = g.raw_stages; p.t_stages = g.t_stages;
+        p.raw_stages = g.raw_stages; p.t_stages = g.t_stages; p.passes = passes;
         p.raw_bytes = g.raw_bytes; p.t_bytes = g.t_bytes;
         p.tx_a = (unsigned int)g.box.rows * g.m_chunk * 4u; p.tx_per_tap = (unsigned int)g.box.rows * g.n_cols * 4u;
         p.tmem_cols = g.tmem_cols;
@@ -796,8 +912,12 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, cons
         cuuint64_t dims[2] = {(cuuint64_t)kdim, (cuuint64_t)v.c_out};
         cuuint64_t str[1] = {(cuuint64_t)kdim * 4};
         cuuint32_t box[2] = {(cuuint32_t)kchunk, (cuuint32_t)n_chunk};
-        cudaError_t e = encode(&p.tm_b, weights, 2, dims, str, box, kchunk * 4);
+        cudaError_t e = encode(&p.tm_b, w_hi, 2, dims, str, box, kchunk * 4);
         if (e != cudaSuccess) return e;
+        if (passes == 3) {
+            e = encode(&p.tm_b_lo, w_lo, 2, dims, str, box, kchunk * 4);
+            if (e != cudaSuccess) return e;
+        }
     }
     p.out = out; p.extra = extra; p.accumulate = accumulate ? 1 : 0;
     p.os_n = v.os_n; p.os_h = v.os_h; p.os_w = v.os_w; p.dense_h = v.dense_h; p.dense_w = v.dense_w;
@@ -806,12 +926,14 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, cons
     const int tiles_n = (v.N + b.n - 1) / b.n;
     p.P = v.P; p.Q = v.Q; p.N = v.N; p.c_out = v.c_out; p.n_chunk = n_chunk; p.R = v.R; p.pad = v.pad;
     p.c_in = v.c_in; p.kchunk = kchunk; p.n_kchunks = v.c_in / kchunk; p.swizzle = kchunk * 4;
+    p.passes = passes;
     p.zero_fill = v.zero_fill; p.out_h = v.out_h; p.out_w = v.out_w;
     p.a_bytes = (unsigned int)kTileM * kchunk * 4;
     p.b_bytes = ((unsigned int)n_chunk * kchunk * 4 + 1023u) & ~1023u;
-    p.tx_bytes = (unsigned int)b.rows * kchunk * 4 + (unsigned int)n_chunk * kchunk * 4;
-    const unsigned int stage = p.a_bytes + p.b_bytes;
-    int stages = (int)(kSmemBudget / stage);
+    const unsigned int parts = passes == 3 ? 2u : 1u;
+    p.stage_bytes = parts * (p.a_bytes + p.b_bytes);
+    p.tx_bytes = (unsigned int)b.rows * kchunk * 4 + parts * (unsigned int)n_chunk * kchunk * 4;
+    int stages = (int)(kSmemBudget / p.stage_bytes);
     const int total = v.R * v.R * p.n_kchunks;
     if (stages > 6) stages = 6;
     if (stages > total) stages = total;
@@ -819,7 +941,7 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, cons
     p.tmem_cols = pow2_cols(n_chunk);
     p.idesc = instr_desc(n_chunk, false, false);
     L->grid = dim3(p.tiles_w * p.tiles_h * tiles_n, v.c_out / n_chunk, 1);
-    L->smem = (unsigned int)stages * stage + 1024;
+    L->smem = (unsigned int)stages * p.stage_bytes + 1024;
     plan->valid = 1;
     return cudaSuccess;
 }
@@ -842,17 +964,25 @@ cudaError_t conv_tc_launch(const ConvTcPlan* plan, DeviceStatus* status, cudaStr
     }
     ConvTcFwdLaunch L = *reinterpret_cast<const ConvTcFwdLaunch*>(plan->storage);
     L.p.status = status;
-    conv_tc_fwd_kernel<<<L.grid, 128, L.smem, st>>>(L.p);
+    conv_tc_fwd_kernel<<<L.grid, 192, L.smem, st>>>(L.p);
     count(n_launch, 1);
     return cudaGetLastError();
 }
 
-cudaError_t conv_dgrad_weights(const float* w, float* wt, int C, int K, int R, cudaStream_t st, int64_t* n_launch)
+cudaError_t conv_weight_prep(const float* params, float* w_hi, float* w_lo, float* wt_hi, float* wt_lo,
+                             const WeightPrepEntry* d_table, int n_entries, cudaStream_t st, int64_t* n_launch)
 {
-    const long long total = (long long)K * R * R * C;
-    int nb = (int)((total + 255) / 256);
-    if (nb > 592) nb = 592;
-    dgrad_weights_kernel<<<nb, 256, 0, st>>>(w, wt, C, K, R);
+    if (n_entries < 1) return cudaSuccess;
+    weight_prep_kernel<<<dim3(n_entries, 4), 256, 0, st>>>(params, w_hi, w_lo, wt_hi, wt_lo, d_table);
+    count(n_launch, 1);
+    return cudaGetLastError();
+}
+
+cudaError_t conv_weight_prep_single(const float* w, float* w_hi, float* w_lo, float* wt_hi, float* wt_lo, int C, int K, int R,
+                                    cudaStream_t st, int64_t* n_launch)
+{
+    WeightPrepEntry e{0, C, K, R, 0};
+    weight_prep_single_kernel<<<dim3(1, 16), 256, 0, st>>>(w, w_hi, w_lo, wt_hi, wt_lo, e);
     count(n_launch, 1);
     return cudaGetLastError();
 }

@@ -20,17 +20,25 @@ struct ConvTcPlan {
     ConvShape s;
     int pass;
     int valid;
-    alignas(64) unsigned char storage[640];
+    alignas(64) unsigned char storage[768];
 };
 
-// pass = PASS_FWD:   out = conv(in, weights) (+ extra)
-// pass = PASS_DGRAD: out (+)= dgrad(in = dy, weights = rearranged weights) (+ extra)
+// passes = 3: error-compensated (hi*hi + lo*hi + hi*lo); passes = 1: single TF32 pass.
+// pass = PASS_FWD:   out = conv(in, w) (+ extra); w_hi / w_lo = split weights [K][R][R][C]
+// pass = PASS_DGRAD: out (+)= dgrad(in = dy) (+ extra); w_hi / w_lo = split rearranged weights [C][R][R][K]
 // pass = PASS_WGRAD: out = wgrad(in = dy, in2 = x)
-cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, const float* in, const float* in2,
-                            const float* weights, float* out, const float* extra, bool accumulate, void* scratch);
+cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int passes, const float* in, const float* in2,
+                            const float* w_hi, const float* w_lo, float* out, const float* extra, bool accumulate, void* scratch);
 cudaError_t conv_tc_launch(const ConvTcPlan* plan, DeviceStatus* status, cudaStream_t st, int64_t* n_launch);
 
-// wt[c][R-1-r][R-1-s][k] = w[k][r][s][c]  (the weights of the data gradient seen as a forward convolution)
-cudaError_t conv_dgrad_weights(const float* w, float* wt, int C, int K, int R, cudaStream_t st, int64_t* n_launch);
+// One convolution's weights inside the flat parameter vector.
+struct WeightPrepEntry { long long w_off; int C, K, R, reserved; };
+// For every table entry (device memory): w_hi/w_lo = hi/lo split of the weights, wt_hi/wt_lo = split of the weights
+// rearranged for the data gradient (wt[c][R-1-r][R-1-s][k] = w[k][r][s][c]); all four use the entry's w_off.
+cudaError_t conv_weight_prep(const float* params, float* w_hi, float* w_lo, float* wt_hi, float* wt_lo,
+                             const WeightPrepEntry* d_table, int n_entries, cudaStream_t st, int64_t* n_launch);
+
+cudaError_t conv_weight_prep_single(const float* w, float* w_hi, float* w_lo, float* wt_hi, float* wt_lo, int C, int K, int R,
+                                    cudaStream_t st, int64_t* n_launch);
 
 }  // namespace hpf

@@ -87,7 +87,9 @@ struct hpf_model {
     std::vector<size_t> bn_scratch_off, conv_scratch_off;   // per stream
     std::vector<size_t> pooled_off, persample_off;      // per m
     std::vector<std::vector<size_t>> fmsg_off, bmsg_off;  // [cut][i*M + m]
-    size_t loss_slots_off = 0, loss_avg_off = 0, wt_off = 0, stage_x_off = 0, stage_lab_off = 0, status_off = 0;
+    size_t loss_slots_off = 0, loss_avg_off = 0, wprep_off = 0, stage_x_off = 0, stage_lab_off = 0, status_off = 0;
+    std::vector<size_t> prep_table_off;       // per partition: WeightPrepEntry[] in the workspace
+    std::vector<std::vector<WeightPrepEntry>> prep_table;   // host copies
     size_t zero_lo = 0, zero_hi = 0;          // region that must start zeroed (tickets, status)
     size_t ws_bytes = 0;
     bool planned = false;
@@ -336,7 +338,9 @@ void build_memory_plan(hpf_model* mdl)
     }
     mdl->loss_slots_off = take(sizeof(float) * M);
     mdl->loss_avg_off = take(sizeof(float));
-    mdl->wt_off = take(sizeof(float) * (size_t)mdl->G);
+    mdl->wprep_off = take(sizeof(float) * 4 * (size_t)((mdl->G + 3) / 4 * 4));   // w_hi | w_lo | wt_hi | wt_lo, parameter offsets
+    mdl->prep_table_off.assign(P, 0);
+    for (int p = 0; p < P; ++p) mdl->prep_table_off[p] = take(sizeof(WeightPrepEntry) * (size_t)(mdl->part_hi[p] - mdl->part_lo[p] + 1));
     mdl->stage_x_off = take(sizeof(float) * (size_t)mdl->B * mdl->inH * mdl->inW * mdl->inC);
     mdl->stage_lab_off = take(sizeof(int32_t) * (size_t)mdl->B);
     const int headC = mdl->ops[n - 1].op.c_in;
@@ -372,7 +376,7 @@ void build_memory_plan(hpf_model* mdl)
 
 bool op_uses_tc(const hpf_model* mdl, int i, int pass)
 {
-    if (mdl->opt_conv_path != 0) return false;
+    if (mdl->opt_conv_path == 1) return false;
     if (mdl->ops[i].op.kind != HPF_OP_CONV) return false;
     if (mdl->ops[i].op.src0 < 0) return false;          // the network input pointer is not known at bind time
     if (mdl->ops[i].w_off % 4) return false;            // the weight tensor map needs a 16-byte aligned base
@@ -485,6 +489,15 @@ int enqueue_phase(hpf_model* mdl, int phase)
         for (int p = 1; p < P; ++p) CU(cudaStreamWaitEvent(mdl->streams[p], mdl->ev_fork, 0));
     }
     if (phase == PH_FWD) {
+        // the tensor-core convolutions read split (and, for the data gradient, rearranged) weights: once per step
+        for (int p = 0; p < P; ++p)
+            if (!mdl->prep_table[p].empty()) {
+                float* wp = reinterpret_cast<float*>(mdl->ws + mdl->wprep_off);
+                const int64_t G4 = (mdl->G + 3) / 4 * 4;      // keeps every array 16-byte aligned
+                CU(conv_weight_prep(mdl->params, wp, wp + G4, wp + 2 * G4, wp + 3 * G4,
+                                    reinterpret_cast<const WeightPrepEntry*>(mdl->ws + mdl->prep_table_off[p]),
+                                    (int)mdl->prep_table[p].size(), mdl->stream_of(p), &mdl->launches));
+            }
         // tick t: every (p, m) with p + m = t
         for (int t = 0; t < P + M - 1; ++t)
             for (int p = 0; p < P; ++p) {
@@ -505,14 +518,6 @@ int enqueue_phase(hpf_model* mdl, int phase)
                 if (p < P - 1 && multi) CU(cudaEventRecord(mdl->ev_fwd[(size_t)p * M + m], st));          // send
             }
     } else if (phase == PH_BWD) {
-        // the data gradient of a tensor-core convolution reads rearranged weights: once per step
-        for (int p = 0; p < P; ++p)
-            for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i)
-                if (mdl->use_tc[PASS_DGRAD][i] && mdl->ops[i].op.src0 >= 0) {
-                    const OpInfo& o = mdl->ops[i];
-                    CU(conv_dgrad_weights(mdl->params + o.w_off, reinterpret_cast<float*>(mdl->ws + mdl->wt_off) + o.w_off,
-                                          o.op.c_in, o.op.c_out, o.op.ksize, mdl->stream_of(p), &mdl->launches));
-                }
         for (int t = 0; t < P + M - 1; ++t)
             for (int p = P - 1; p >= 0; --p) {
                 const int m = t - (P - 1 - p);
@@ -653,7 +658,7 @@ int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
     if (mdl->state != ST_CREATED) return fail(HPF_ERR_STATE, "options must be set before hpf_bind");
     switch (option) {
     case HPF_OPT_GRAPH: mdl->opt_graph = value != 0; break;
-    case HPF_OPT_CONV_PATH: if (value != 0 && value != 1) return fail(HPF_ERR_INVALID, "bad conv path"); mdl->opt_conv_path = value; break;
+    case HPF_OPT_CONV_PATH: if (value < 0 || value > 2) return fail(HPF_ERR_INVALID, "bad conv path"); mdl->opt_conv_path = value; break;
     case HPF_OPT_SINGLE_STREAM: mdl->opt_single = value != 0; break;
     case HPF_OPT_KEEP_MESSAGES: mdl->opt_messages = value != 0; break;
     default: return fail(HPF_ERR_INVALID, "unknown option");
@@ -776,9 +781,21 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
         mdl->use_tc[pass].assign(n, 0);
         for (int i = 0; i < n; ++i) if (op_uses_tc(mdl, i, pass)) { mdl->use_tc[pass][i] = 1; any_tc = true; }
     }
+    mdl->prep_table.assign(mdl->P, {});
     if (any_tc) {
         CU(conv_tc_init());
-        float* wt = reinterpret_cast<float*>(mdl->ws + mdl->wt_off);
+        const int passes = mdl->opt_conv_path == 2 ? 1 : 3;
+        float* wp = reinterpret_cast<float*>(mdl->ws + mdl->wprep_off);
+        const int64_t G = (mdl->G + 3) / 4 * 4;       // stride between the four prepared-weight arrays
+        for (int i = 0; i < n; ++i)
+            if (mdl->use_tc[PASS_FWD][i] || mdl->use_tc[PASS_DGRAD][i]) {
+                const OpInfo& o = mdl->ops[i];
+                mdl->prep_table[o.part].push_back(WeightPrepEntry{o.w_off, o.op.c_in, o.op.c_out, o.op.ksize, 0});
+            }
+        for (int p = 0; p < mdl->P; ++p)
+            if (!mdl->prep_table[p].empty())
+                CU(cudaMemcpyAsync(mdl->ws + mdl->prep_table_off[p], mdl->prep_table[p].data(),
+                                   sizeof(WeightPrepEntry) * mdl->prep_table[p].size(), cudaMemcpyHostToDevice, mdl->streams[0]));
         for (int pass = 0; pass < 3; ++pass) {
             mdl->tc_plan[pass].resize((size_t)n * M);
             for (int m = 0; m < M; ++m)
@@ -791,12 +808,13 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                     ConvTcPlan* pl = &mdl->tc_plan[pass][(size_t)m * n + i];
                     void* scratch = mdl->ws + mdl->conv_scratch_off[o.part];
                     if (pass == PASS_FWD)
-                        CU(conv_tc_prepare(pl, s, pass, mdl->act(src, m), nullptr, mdl->params + o.w_off, mdl->act(i, m), nullptr, false, scratch));
+                        CU(conv_tc_prepare(pl, s, pass, passes, mdl->act(src, m), nullptr, wp + o.w_off, wp + G + o.w_off,
+                                           mdl->act(i, m), nullptr, false, scratch));
                     else if (pass == PASS_DGRAD)
-                        CU(conv_tc_prepare(pl, s, pass, mdl->grad(i, m), nullptr, wt + o.w_off, mdl->grad(src, m),
-                                           ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch));
+                        CU(conv_tc_prepare(pl, s, pass, passes, mdl->grad(i, m), nullptr, wp + 2 * G + o.w_off, wp + 3 * G + o.w_off,
+                                           mdl->grad(src, m), ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch));
                     else
-                        CU(conv_tc_prepare(pl, s, pass, mdl->grad(i, m), mdl->act(src, m), nullptr,
+                        CU(conv_tc_prepare(pl, s, pass, passes, mdl->grad(i, m), mdl->act(src, m), nullptr, nullptr,
                                            mdl->gslots + (int64_t)m * mdl->G + o.w_off, nullptr, false, scratch));
                 }
         }
@@ -956,7 +974,7 @@ int hpf_conv_scratch_bytes(int32_t N, int32_t H, int32_t W, int32_t C, int32_t K
     return HPF_OK;
 }
 
-static int conv_single(int pass, const float* in, const float* in2, const float* w, const float* wt, float* out,
+static int conv_single(int pass, const float* in, const float* in2, const float* w, const float* wprep, float* out,
                        int32_t N, int32_t H, int32_t W, int32_t C, int32_t K, int32_t R, int32_t stride, int32_t pad,
                        int32_t path, void* d_scratch, void* stream)
 {
@@ -966,12 +984,14 @@ static int conv_single(int pass, const float* in, const float* in2, const float*
     const ConvShape s = make_conv_shape(N, H, W, C, K, R, stride, pad);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     if (path == 1) {
+        if (pass != PASS_WGRAD && !w) return fail(HPF_ERR_INVALID, "null argument");
         if (pass == PASS_FWD) CU(conv_fwd_simt(in, w, out, nullptr, s, st, nullptr));
         else if (pass == PASS_DGRAD) CU(conv_dgrad_simt(in, w, out, nullptr, false, s, st, nullptr));
         else CU(conv_wgrad_simt(in2, in, out, s, d_scratch, st, nullptr));
         return HPF_OK;
     }
-    if (path != 0) return fail(HPF_ERR_INVALID, "bad path");
+    if (path != 0 && path != 2) return fail(HPF_ERR_INVALID, "bad path");
+    if (pass != PASS_WGRAD && !wprep) return fail(HPF_ERR_INVALID, "the tensor-core paths need prepared weights");
     if (!conv_tc_supported(s, pass)) return fail(HPF_ERR_UNSUPPORTED, "shape outside the tensor-core kernels' reach");
     CU(conv_tc_init());
     ConvTcPlan plan;
@@ -980,30 +1000,32 @@ static int conv_single(int pass, const float* in, const float* in2, const float*
     hpf_conv_scratch_bytes(N, H, W, C, K, R, stride, pad, &sb);
     DeviceStatus* status = reinterpret_cast<DeviceStatus*>(reinterpret_cast<char*>(d_scratch) + sb - 256);
     CU(cudaMemsetAsync(status, 0, sizeof(DeviceStatus), st));
-    CU(conv_tc_prepare(&plan, s, pass, in, in2, pass == PASS_DGRAD ? wt : w, out, nullptr, false, d_scratch));
+    const int64_t nw = (int64_t)K * R * R * C;
+    const float* hi = wprep ? wprep + (pass == PASS_DGRAD ? 2 * nw : 0) : nullptr;
+    CU(conv_tc_prepare(&plan, s, pass, path == 2 ? 1 : 3, in, in2, hi, hi ? hi + nw : nullptr, out, nullptr, false, d_scratch));
     CU(conv_tc_launch(&plan, status, st, nullptr));
     return HPF_OK;
 }
 
-int hpf_conv_fwd(const float* d_x, const float* d_w, float* d_y, int32_t N, int32_t H, int32_t W, int32_t C, int32_t K,
-                 int32_t R, int32_t stride, int32_t pad, int32_t path, void* d_scratch, void* stream)
+int hpf_conv_prepare_weights(const float* d_w, float* d_wprep, int32_t C, int32_t K, int32_t R, void* stream)
 {
-    if (!d_w) return fail(HPF_ERR_INVALID, "null argument");
-    return conv_single(PASS_FWD, d_x, nullptr, d_w, nullptr, d_y, N, H, W, C, K, R, stride, pad, path, d_scratch, stream);
-}
-
-int hpf_conv_dgrad_weights(const float* d_w, float* d_wt, int32_t C, int32_t K, int32_t R, void* stream)
-{
-    if (!d_w || !d_wt || C < 1 || K < 1 || R < 1) return fail(HPF_ERR_INVALID, "bad argument");
-    CU(conv_dgrad_weights(d_w, d_wt, C, K, R, reinterpret_cast<cudaStream_t>(stream), nullptr));
+    if (!d_w || !d_wprep || C < 1 || K < 1 || R < 1) return fail(HPF_ERR_INVALID, "bad argument");
+    const int64_t nw = (int64_t)K * R * R * C;
+    CU(conv_weight_prep_single(d_w, d_wprep, d_wprep + nw, d_wprep + 2 * nw, d_wprep + 3 * nw, C, K, R,
+                               reinterpret_cast<cudaStream_t>(stream), nullptr));
     return HPF_OK;
 }
 
-int hpf_conv_dgrad(const float* d_dy, const float* d_w, const float* d_wt, float* d_dx, int32_t N, int32_t H, int32_t W,
+int hpf_conv_fwd(const float* d_x, const float* d_w, const float* d_wprep, float* d_y, int32_t N, int32_t H, int32_t W, int32_t C,
+                 int32_t K, int32_t R, int32_t stride, int32_t pad, int32_t path, void* d_scratch, void* stream)
+{
+    return conv_single(PASS_FWD, d_x, nullptr, d_w, d_wprep, d_y, N, H, W, C, K, R, stride, pad, path, d_scratch, stream);
+}
+
+int hpf_conv_dgrad(const float* d_dy, const float* d_w, const float* d_wprep, float* d_dx, int32_t N, int32_t H, int32_t W,
                    int32_t C, int32_t K, int32_t R, int32_t stride, int32_t pad, int32_t path, void* d_scratch, void* stream)
 {
-    if (!d_w || (path == 0 && !d_wt)) return fail(HPF_ERR_INVALID, "null argument");
-    return conv_single(PASS_DGRAD, d_dy, nullptr, d_w, d_wt, d_dx, N, H, W, C, K, R, stride, pad, path, d_scratch, stream);
+    return conv_single(PASS_DGRAD, d_dy, nullptr, d_w, d_wprep, d_dx, N, H, W, C, K, R, stride, pad, path, d_scratch, stream);
 }
 
 int hpf_conv_wgrad(const float* d_x, const float* d_dy, float* d_dw, int32_t N, int32_t H, int32_t W, int32_t C, int32_t K,

@@ -55,7 +55,7 @@ def check_step(ops, in_hwc, B, M, cuts, options=None, seed=0, bn_jitter=0.0, mic
     return bd, ref, worst
 
 
-@pytest.mark.parametrize("conv_path", [0, 1])
+@pytest.mark.parametrize("conv_path", [0, 1, 2])
 @pytest.mark.parametrize("graph", [1, 0])
 def test_config1_resnet11(conv_path, graph):
     c = wl.config("r11")
