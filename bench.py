@@ -198,19 +198,85 @@ def kernel_roofline(torch, hpf, cfg, pk):
             "algorithmic_bytes_per_launch": alg, "us_per_launch": sec * 1e6}
 
 
+def conv_sweep(args):
+    """Configuration 2: the bottleneck convolution shapes at batch 128, forward / data gradient / weight
+    gradient each, through the C ABI on rotating operand sets that together exceed L2.  One JSON line with
+    a row per (shape, pass): microseconds, achieved TFLOP/s and GB/s (algorithmic), and the fraction of
+    min(TF32 peak, arithmetic intensity x HBM bandwidth)."""
+    import torch
+    import paper_1911_05146_b200 as hpf
+    torch.cuda.set_device(0)
+    pk = peaks()
+    tf32_peak = pk["bf16_tflops"] / 2.0            # dense TF32 = half the measured dense BF16 rate
+    N, rows_out = 128, []
+    dev = "cuda"
+    for (ks, st, ci, co, H) in wl.conv_sweep_shapes():
+        pad = 1 if ks == 3 else 0
+        P = (H + 2 * pad - ks) // st + 1
+        x_el, y_el, w_el = N * H * H * ci, N * P * P * co, co * ks * ks * ci
+        in_el = N * P * P * ci if st > 1 else x_el
+        nset = max(2, int(260e6 // (4 * (x_el + y_el))) + 1)
+        xs = [torch.randn(N, H, H, ci, device=dev) for _ in range(nset)]
+        ys = [torch.randn(N, P, P, co, device=dev) for _ in range(nset)]
+        w = torch.randn(co, ks, ks, ci, device=dev) * (2.0 / (ci * ks * ks)) ** 0.5
+        dw = torch.empty_like(w)
+        wprep = torch.empty(4 * w_el, device=dev)
+        scratch = torch.zeros(hpf.conv_scratch_bytes(N, H, H, ci, co, ks, st, pad), dtype=torch.uint8, device=dev)
+        hpf.conv_prepare_weights(w, wprep, ci, co, ks)
+        geo = (N, H, H, ci, co, ks, st, pad, args.conv_path)
+        calls = {
+            "fwd": lambda k: hpf.conv_fwd(xs[k], w, wprep, ys[k], *geo, scratch),
+            "dgrad": lambda k: hpf.conv_dgrad(ys[k], w, wprep, xs[k], *geo, scratch),
+            "wgrad": lambda k: hpf.conv_wgrad(xs[k], ys[k], dw, *geo, scratch),
+        }
+        flops = 2.0 * N * P * P * ci * co * ks * ks
+        nbytes = 4.0 * (in_el + y_el + w_el)
+        for name, fn in calls.items():
+            for k in range(nset):
+                fn(k)
+            reps = max(10, 3 * nset)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for i in range(reps):
+                fn(i % nset)
+            e1.record()
+            torch.cuda.synchronize()
+            sec = e0.elapsed_time(e1) * 1e-3 / reps
+            ceiling = min(tf32_peak, flops / nbytes * pk["hbm_gbs"] / 1e3)     # TFLOP/s
+            rows_out.append({"shape": "%dx%d s%d %d->%d @%d" % (ks, ks, st, ci, co, H), "pass": name, "us": sec * 1e6,
+                             "tflops": flops / sec / 1e12, "gbs": nbytes / sec / 1e9, "ai": flops / nbytes,
+                             "ceiling_tflops": ceiling, "frac_of_ceiling": flops / sec / 1e12 / ceiling})
+        del xs, ys
+    best = max(r["tflops"] for r in rows_out)
+    print(json.dumps({"metric": "conv sweep (configuration 2), batch 128", "unit": "TFLOP/s", "value": best, "n_gpus": 1,
+                      "dtype": "tf32", "data": "synthetic", "config": {"workload": "28 bottleneck conv shapes x {fwd, dgrad, wgrad}",
+                      "conv_path": args.conv_path, "tf32_peak_tflops": tf32_peak, "hbm_gbs": pk["hbm_gbs"], "peak_source": pk["source"]},
+                      "rows": rows_out}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="hpf", choices=["hpf", "reference"])
-    ap.add_argument("--workload", default="r1001", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--workload", default="r1001", choices=sorted(wl.CONFIGS) + ["conv_sweep"])
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--conv-path", type=int, default=0)
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-kernel-roofline", action="store_true")
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--profile", action="store_true",
+                    help="for runs under a profiler: honour --warmup below 3 and skip the side measurements")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "hpf" else args.warmup
+    if args.profile:
+        args.skip_e2e = args.skip_cpu_baseline = args.skip_kernel_roofline = True
+    elif args.impl == "hpf":
+        args.warmup = max(args.warmup, 3)
+    if args.workload == "conv_sweep":
+        conv_sweep(args)
+        return
     cfg = wl.config(args.workload)
     if args.impl == "reference":
         run_reference(args, cfg)
@@ -282,15 +348,17 @@ def main():
     model.synchronize(0)
 
     # end to end: host buffers in, loss out, every step
-    for _ in range(2):
-        model.step_host(hx, hl)
-    barrier()
-    e0.record(s0)
-    for _ in range(args.steps):
-        model.step_host(hx, hl)
-    e1.record(s0)
-    barrier()
-    ms_e2e = e0.elapsed_time(e1)
+    ms_e2e = float("nan")
+    if not args.skip_e2e:
+        for _ in range(2):
+            model.step_host(hx, hl)
+        barrier()
+        e0.record(s0)
+        for _ in range(args.steps):
+            model.step_host(hx, hl)
+        e1.record(s0)
+        barrier()
+        ms_e2e = e0.elapsed_time(e1)
 
     if dist is not None:
         t = torch.tensor([ms, ms_e2e], device=dev, dtype=torch.float64)

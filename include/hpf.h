@@ -87,8 +87,13 @@ int hpf_model_destroy(hpf_model *model);
  *                          2: as 0 with a single TF32 pass (11-bit operands; error grows with depth).
  *   HPF_OPT_SINGLE_STREAM  1: all stages on stream 0 (hazard check: results must equal the multi-stream run).
  *   HPF_OPT_KEEP_MESSAGES  1: every partition copies what it receives across a cut (activations forward,
- *                          partial errors backward) into message buffers readable with hpf_message_ptr. */
-typedef enum { HPF_OPT_GRAPH = 1, HPF_OPT_CONV_PATH = 2, HPF_OPT_SINGLE_STREAM = 3, HPF_OPT_KEEP_MESSAGES = 4 } hpf_option;
+ *                          partial errors backward) into message buffers readable with hpf_message_ptr.
+ *   HPF_OPT_FUSE_ADD       1 (default): a residual ADD is computed in the epilogue of the later of its two
+ *                          producers when that is a convolution nothing else reads, in the same partition;
+ *                          that convolution's own output is then not stored (hpf_tensor_ptr answers
+ *                          HPF_ERR_STATE for it).  0: every op's output is stored. */
+typedef enum { HPF_OPT_GRAPH = 1, HPF_OPT_CONV_PATH = 2, HPF_OPT_SINGLE_STREAM = 3, HPF_OPT_KEEP_MESSAGES = 4,
+               HPF_OPT_FUSE_ADD = 5 } hpf_option;
 int hpf_set_option(hpf_model *model, int32_t option, int32_t value);
 
 /* ---- integer bookkeeping (Section 5.1 lists, Section 5.3 pipelining) ----------------------------- */

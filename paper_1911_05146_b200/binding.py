@@ -5,7 +5,7 @@ import os
 from . import build as _build
 
 CONV, BNRELU, ADD, MAXPOOL, HEAD = 1, 2, 3, 4, 5
-OPT_GRAPH, OPT_CONV_PATH, OPT_SINGLE_STREAM, OPT_KEEP_MESSAGES = 1, 2, 3, 4
+OPT_GRAPH, OPT_CONV_PATH, OPT_SINGLE_STREAM, OPT_KEEP_MESSAGES, OPT_FUSE_ADD = 1, 2, 3, 4, 5
 
 
 class HpfError(RuntimeError):
@@ -254,3 +254,4 @@ def bnrelu_bwd(x, dy, gamma, beta, stats, dx, addend, accumulate, dgamma, dbeta,
 
 def grad_average_flat(slots, out, M, G, stream=None):
     _check(lib().hpf_grad_average_flat(_ptr(slots), _ptr(out), M, G, _stream(stream)))
+

@@ -76,9 +76,11 @@ struct hpf_model {
     std::vector<std::vector<int>> live;       // per cut
     int64_t G = 0;
     // options
-    int opt_graph = 1, opt_conv_path = 0, opt_single = 0, opt_messages = 0;
+    int opt_graph = 1, opt_conv_path = 0, opt_single = 0, opt_messages = 0, opt_fuse_add = 1;
     // gradient-flow plan
     std::vector<int> grad_alias;              // tensor -> ADD op whose gradient buffer it shares, or -1
+    std::vector<int> fused_into;              // conv -> residual ADD computed in its epilogue (its own output is not stored), or -1
+    std::vector<int> add_done_by;             // ADD -> the conv that computes it, or -1
     std::vector<GradEdge> edge0;              // per op: contribution to src0
     std::vector<AccumAction> accums;
     std::vector<std::vector<MessagePlan>> msg_plan;   // per cut
@@ -294,6 +296,27 @@ int build_grad_plan(hpf_model* mdl)
     return HPF_OK;
 }
 
+// Residual ADD fused into the epilogue of the later of its two producers when that producer is a
+// convolution read by nothing else and sits in the same partition: the sum is written straight into the
+// ADD's output tensor and the convolution's own output is never stored.
+void build_fusion_plan(hpf_model* mdl)
+{
+    const int n = mdl->n_ops;
+    mdl->fused_into.assign(n, -1);
+    mdl->add_done_by.assign(n, -1);
+    if (!mdl->opt_fuse_add) return;
+    for (int i = 0; i < n; ++i) {
+        const hpf_op& q = mdl->ops[i].op;
+        if (q.kind != HPF_OP_ADD || q.src0 == q.src1) continue;
+        const int late = q.src0 > q.src1 ? q.src0 : q.src1;
+        const OpInfo& c = mdl->ops[late];
+        if (c.op.kind != HPF_OP_CONV || c.consumers.size() != 1 || c.part != mdl->ops[i].part) continue;
+        if (mdl->opt_messages) continue;      // message copies want every tensor materialised
+        mdl->fused_into[late] = i;
+        mdl->add_done_by[i] = late;
+    }
+}
+
 ConvShape conv_shape_of(const hpf_model* mdl, int i)
 {
     const OpInfo& o = mdl->ops[i];
@@ -305,6 +328,7 @@ ConvShape conv_shape_of(const hpf_model* mdl, int i)
 // ------------------------------------------------------------------------------------------------
 void build_memory_plan(hpf_model* mdl)
 {
+    build_fusion_plan(mdl);
     const int n = mdl->n_ops, M = mdl->M, P = mdl->P;
     size_t at = 0;
     auto take = [&](size_t bytes) { size_t o = at; at = align_up(at + bytes, 256); return o; };
@@ -351,7 +375,11 @@ void build_memory_plan(hpf_model* mdl)
     }
     mdl->act_off.assign((size_t)n * M, 0); mdl->grad_off.assign((size_t)n * M, 0); mdl->stats_off.assign((size_t)n * M, 0);
     for (int m = 0; m < M; ++m) {
-        for (int i = 0; i < n; ++i) mdl->act_off[(size_t)m * n + i] = take(sizeof(float) * (size_t)mdl->numel(i));
+        for (int i = n - 1; i >= 0; --i) {
+            const int f = mdl->fused_into[i];
+            if (f >= 0) mdl->act_off[(size_t)m * n + i] = mdl->act_off[(size_t)m * n + f];   // f > i: already placed
+            else mdl->act_off[(size_t)m * n + i] = take(sizeof(float) * (size_t)mdl->numel(i));
+        }
         for (int i = n - 1; i >= 0; --i) {
             const int a = mdl->grad_alias[i];
             if (a >= 0) mdl->grad_off[(size_t)m * n + i] = mdl->grad_off[(size_t)m * n + a];   // a > i: already placed
@@ -402,10 +430,16 @@ int forward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
     float* out = mdl->act(i, m);
     switch (q.kind) {
     case HPF_OP_CONV: {
+        // with a fused residual ADD, `out` is the ADD's output tensor and the other addend rides in the epilogue
+        const float* residual = nullptr;
+        if (mdl->fused_into[i] >= 0) {
+            const hpf_op& a = mdl->ops[mdl->fused_into[i]].op;
+            residual = mdl->act(a.src0 == i ? a.src1 : a.src0, m);
+        }
         if (mdl->use_tc[PASS_FWD][i]) {
             CU(conv_tc_launch(&mdl->tc_plan[PASS_FWD][(size_t)m * mdl->n_ops + i], mdl->status(), st, &mdl->launches));
         } else {
-            CU(conv_fwd_simt(in0, mdl->params + o.w_off, out, nullptr, conv_shape_of(mdl, i), st, &mdl->launches));
+            CU(conv_fwd_simt(in0, mdl->params + o.w_off, out, residual, conv_shape_of(mdl, i), st, &mdl->launches));
         }
         break;
     }
@@ -414,7 +448,7 @@ int forward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
                       (int64_t)mdl->b * o.H * o.W, o.C, mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
         break;
     case HPF_OP_ADD:
-        CU(add_fwd(in0, mdl->act(q.src1, m), out, mdl->numel(i), st, &mdl->launches));
+        if (mdl->add_done_by[i] < 0) CU(add_fwd(in0, mdl->act(q.src1, m), out, mdl->numel(i), st, &mdl->launches));
         break;
     case HPF_OP_MAXPOOL:
         CU(maxpool_fwd(in0, out, conv_shape_of(mdl, i), st, &mdl->launches));
@@ -661,6 +695,7 @@ int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
     case HPF_OPT_CONV_PATH: if (value < 0 || value > 2) return fail(HPF_ERR_INVALID, "bad conv path"); mdl->opt_conv_path = value; break;
     case HPF_OPT_SINGLE_STREAM: mdl->opt_single = value != 0; break;
     case HPF_OPT_KEEP_MESSAGES: mdl->opt_messages = value != 0; break;
+    case HPF_OPT_FUSE_ADD: mdl->opt_fuse_add = value != 0; break;
     default: return fail(HPF_ERR_INVALID, "unknown option");
     }
     mdl->planned = false;
@@ -807,9 +842,15 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                     const GradEdge& ed = mdl->edge0[i];
                     ConvTcPlan* pl = &mdl->tc_plan[pass][(size_t)m * n + i];
                     void* scratch = mdl->ws + mdl->conv_scratch_off[o.part];
-                    if (pass == PASS_FWD)
+                    if (pass == PASS_FWD) {
+                        const float* residual = nullptr;
+                        if (mdl->fused_into[i] >= 0) {
+                            const hpf_op& a = mdl->ops[mdl->fused_into[i]].op;
+                            residual = mdl->act(a.src0 == i ? a.src1 : a.src0, m);
+                        }
                         CU(conv_tc_prepare(pl, s, pass, passes, mdl->act(src, m), nullptr, wp + o.w_off, wp + G + o.w_off,
-                                           mdl->act(i, m), nullptr, false, scratch));
+                                           mdl->act(i, m), residual, false, scratch));
+                    }
                     else if (pass == PASS_DGRAD)
                         CU(conv_tc_prepare(pl, s, pass, passes, mdl->grad(i, m), nullptr, wp + 2 * G + o.w_off, wp + 3 * G + o.w_off,
                                            mdl->grad(src, m), ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch));
@@ -908,6 +949,7 @@ int hpf_tensor_ptr(const hpf_model* mdl, int32_t op, int32_t m, int32_t want_gra
     if (!mdl || !d_ptr || !shape) return fail(HPF_ERR_INVALID, "null");
     if (mdl->state < ST_BOUND) return fail(HPF_ERR_STATE, "hpf_bind first");
     if (op < 0 || op >= mdl->n_ops || m < 0 || m >= mdl->M) return fail(HPF_ERR_INVALID, "out of range");
+    if (!want_grad && mdl->fused_into[op] >= 0) return fail(HPF_ERR_STATE, "not stored: this convolution's output is fused into the residual add");
     *d_ptr = want_grad ? mdl->grad(op, m) : mdl->act(op, m);
     shape[0] = mdl->b; shape[1] = mdl->ops[op].H; shape[2] = mdl->ops[op].W; shape[3] = mdl->ops[op].C;
     return HPF_OK;

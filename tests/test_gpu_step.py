@@ -6,7 +6,7 @@ import torch
 import paper_1911_05146_b200 as hpf
 import workloads as wl
 from oracle import reference as ora
-from hpf_testlib import Bound, rel_l2, seeded, matched_oracle, TOL_TENSOR, TOL_LOSS
+from hpf_testlib import Bound, rel_l2, seeded, matched_oracle, TOL_TENSOR, TOL_LOSS, TAU, TAU_ONE_PASS
 
 pytestmark = pytest.mark.gpu
 
@@ -30,7 +30,8 @@ def check_step(ops, in_hwc, B, M, cuts, options=None, seed=0, bn_jitter=0.0, mic
     offs, G = wl.param_offsets(ops)
     worst = 0.0
     used = 0
-    mbs = [matched_oracle(bd, m, theta, x, labels, cuts=list(cuts)) for m in range(M)]
+    tau = TAU_ONE_PASS if (options or {}).get(hpf.OPT_CONV_PATH) == 2 else TAU
+    mbs = [matched_oracle(bd, m, theta, x, labels, cuts=list(cuts), tau=tau) for m in range(M)]
     g_avg_ref = ora.grad_average(np.stack([r["g"] for r in mbs]))
     for i, (w_off, w_cnt, b_off, b_cnt) in enumerate(offs):
         for off, cnt in ((w_off, w_cnt), (b_off, b_cnt)):
@@ -47,8 +48,10 @@ def check_step(ops, in_hwc, B, M, cuts, options=None, seed=0, bn_jitter=0.0, mic
             mb = mbs[m]
             used += mb["decisions_used"]
             for i in range(len(ops)):
-                e = rel_l2(bd.tensor(i, m), mb["act"][i]); worst = max(worst, e)
-                assert e <= TOL_TENSOR, ("act", i, m, e)
+                a = bd.tensor_or_none(i, m)          # None: a convolution whose output lives only inside the fused residual add
+                if a is not None:
+                    e = rel_l2(a, mb["act"][i]); worst = max(worst, e)
+                    assert e <= TOL_TENSOR, ("act", i, m, e)
                 e = rel_l2(bd.tensor(i, m, grad=True), mb["dact"][i]); worst = max(worst, e)
                 assert e <= TOL_TENSOR, ("dact", i, m, e)
     print("worst rel-L2 %.3e, in-window ReLU decisions taken from the GPU: %d" % (worst, used))
@@ -64,9 +67,16 @@ def test_config1_resnet11(conv_path, graph):
 
 
 @pytest.mark.parametrize("cuts", [[], [4], [3, 7, 8], [1, 5, 12, 25]])
-def test_mid_block_cuts_and_jittered_bn(cuts):
+@pytest.mark.parametrize("fuse_add", [1, 0])
+def test_mid_block_cuts_and_jittered_bn(cuts, fuse_add):
     ops = wl.resnet_v2_cifar(1)
-    check_step(ops, (32, 32, 3), 4, 2, cuts, seed=3, bn_jitter=0.3)
+    bd, _, _ = check_step(ops, (32, 32, 3), 4, 2, cuts, {hpf.OPT_FUSE_ADD: fuse_add}, seed=3, bn_jitter=0.3)
+    stored = [bd.tensor_or_none(i, 0) is not None for i in range(len(ops))]
+    if fuse_add == 0:
+        assert all(stored)
+    else:
+        # every cut list leaves at least one (projection, ADD) pair inside one partition
+        assert not all(stored)
 
 
 def test_odd_widths_run_on_cuda_cores():
