@@ -186,6 +186,23 @@ int hpf_bnrelu_fwd(const float *d_x, const float *d_gamma, const float *d_beta, 
 int hpf_bnrelu_bwd(const float *d_x, const float *d_dy, const float *d_gamma, const float *d_beta,
                    const float *d_stats, float *d_dx, const float *d_addend, int32_t accumulate,
                    float *d_dgamma, float *d_dbeta, int64_t rows, int32_t C, void *d_scratch, void *stream);
+/* The same BN+ReLU forward for callers that cannot allocate device memory or be handed scratch at the
+ * time of the call (code inside a no-allocation region: a real-time loop, a stream callback, a plug-in
+ * given only its input and output buffers).  The paper has no counterpart; this is a convenience of the
+ * library.  The scratch is a fixed array of hpf_static_scratch_bytes() (2 MiB) inside the library's
+ * device image: every GPU that loads the library holds it until the process exits.  The call allocates
+ * nothing (no cudaMalloc, no cudaFree, no allocating library routine).
+ *   - Sizes whose partial sums exceed the array (hpf_bnrelu_scratch_bytes(rows, C) > 2 MiB) are refused
+ *     with HPF_ERR_WORKSPACE; nothing is launched.
+ *   - The first call on a device looks up the array's device address (that device must be current).
+ *     Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the call
+ *     clears the part that must start at zero.  Two calls whose kernels overlap on the GPU (different
+ *     streams, no ordering between them) race on it: order them.
+ * Inputs and outputs are the caller's, exactly as for hpf_bnrelu_fwd; results are identical to it. */
+int hpf_bnrelu_fwd_static(const float *d_x, const float *d_gamma, const float *d_beta, float eps, float *d_y,
+                          float *d_stats, int64_t rows, int32_t C, void *stream);
+int hpf_static_scratch_bytes(size_t *bytes);
 /* out[j] = (sum_{m ascending} slots[m][j]) / M */
 int hpf_grad_average_flat(const float *d_slots, float *d_out, int32_t M, int64_t G, void *stream);
 

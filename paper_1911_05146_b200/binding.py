@@ -62,6 +62,8 @@ _SIGNATURES = {
     "hpf_bnrelu_fwd": [_vp, _vp, _vp, _f32, _vp, _vp, _i64, _i32, _vp, _vp],
     "hpf_bnrelu_bwd": [_vp] * 7 + [_i32, _vp, _vp, _i64, _i32, _vp, _vp],
     "hpf_grad_average_flat": [_vp, _vp, _i32, _i64, _vp],
+    "hpf_bnrelu_fwd_static": [_vp, _vp, _vp, _f32, _vp, _vp, _i64, _i32, _vp],
+    "hpf_static_scratch_bytes": [C.POINTER(C.c_size_t)],
 }
 EXPORTS = sorted(list(_SIGNATURES) + ["hpf_strerror", "hpf_last_error"])
 
@@ -255,3 +257,11 @@ def bnrelu_bwd(x, dy, gamma, beta, stats, dx, addend, accumulate, dgamma, dbeta,
 def grad_average_flat(slots, out, M, G, stream=None):
     _check(lib().hpf_grad_average_flat(_ptr(slots), _ptr(out), M, G, _stream(stream)))
 
+
+def bnrelu_fwd_static(x, gamma, beta, eps, y, stats, rows, Cc, stream=None):
+    """BN+ReLU forward on the library's built-in scratch: for callers that cannot allocate (see hpf.h)."""
+    _check(lib().hpf_bnrelu_fwd_static(_ptr(x), _ptr(gamma), _ptr(beta), eps, _ptr(y), _ptr(stats), rows, Cc, _stream(stream)))
+
+
+def static_scratch_bytes():
+    n = C.c_size_t(); _check(lib().hpf_static_scratch_bytes(C.byref(n))); return n.value
