@@ -255,13 +255,67 @@ def conv_sweep(args):
                       "rows": rows_out}), flush=True)
 
 
+def membound_sweep(args):
+    """The memory-bound kernels alone, through the C ABI: fused BN+ReLU forward / backward at batch 128 and at the
+    headline micro-batch size (16) on the bottleneck tensor shapes, and the gradient average at the parameter
+    counts of configurations 4 and 5.  Rotating operand sets larger than L2; CUDA events on the launching stream."""
+    import torch
+    import paper_1911_05146_b200 as hpf
+    torch.cuda.set_device(0)
+    pk = peaks()
+    dev, out = "cuda", []
+
+    def timed(fn, nset, reps):
+        for k in range(nset):
+            fn(k)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(reps):
+            fn(i % nset)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e-3 / reps
+
+    shapes = [(N, H, C) for N in (128, 16) for (H, C) in ((32, 64), (16, 128), (8, 256), (32, 16))] + [(64, 56, 256)]
+    for (N, H, C) in shapes:
+        rows = N * H * H
+        nset = max(3, int(300e6 // (rows * C * 4 * 3)) + 1)
+        xs = [torch.randn(rows, C, device=dev) for _ in range(nset)]
+        dys = [torch.randn(rows, C, device=dev) for _ in range(nset)]
+        outs = [torch.empty(rows, C, device=dev) for _ in range(nset)]
+        g = torch.ones(C, device=dev); b = torch.zeros(C, device=dev)
+        stats = torch.empty(2 * C, device=dev); dg = torch.empty(C, device=dev); db = torch.empty(C, device=dev)
+        scratch = torch.zeros(hpf.bnrelu_scratch_bytes(rows, C), dtype=torch.uint8, device=dev)
+        reps = max(20, 3 * nset)
+        tf = timed(lambda k: hpf.bnrelu_fwd(xs[k], g, b, 1e-5, outs[k], stats, rows, C, scratch), nset, reps)
+        tb = timed(lambda k: hpf.bnrelu_bwd(xs[k], dys[k], g, b, stats, outs[k], None, 0, dg, db, rows, C, scratch), nset, reps)
+        for name, t, bpe in (("bnrelu_fwd", tf, 8.0), ("bnrelu_bwd", tb, 12.0)):
+            gbs = bpe * rows * C / t / 1e9
+            out.append({"kernel": name, "shape": "N=%d %dx%d C=%d" % (N, H, H, C), "mb": rows * C * 4 / 1e6, "us": t * 1e6,
+                        "gbs": gbs, "frac_hbm": gbs / pk["hbm_gbs"]})
+        del xs, dys, outs
+    for (M, G) in ((8, 10327706), (4, 60185128)):
+        nset = 2
+        slots = [torch.randn(M, G, device=dev) for _ in range(nset)]
+        avg = torch.empty(G, device=dev)
+        t = timed(lambda k: hpf.grad_average_flat(slots[k], avg, M, G), nset, 20)
+        gbs = 4.0 * (M + 1) * G / t / 1e9
+        out.append({"kernel": "grad_average", "shape": "M=%d G=%d" % (M, G), "mb": 4.0 * M * G / 1e6, "us": t * 1e6, "gbs": gbs,
+                    "frac_hbm": gbs / pk["hbm_gbs"]})
+        del slots
+    print(json.dumps({"metric": "memory-bound kernels alone (algorithmic GB/s)", "unit": "GB/s", "value": max(r["gbs"] for r in out),
+                      "n_gpus": 1, "dtype": "f32", "data": "synthetic", "config": {"workload": "BN+ReLU fwd/bwd, gradient average",
+                      "hbm_gbs": pk["hbm_gbs"], "peak_source": pk["source"]}, "rows": out}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="hpf", choices=["hpf", "reference"])
-    ap.add_argument("--workload", default="r1001", choices=sorted(wl.CONFIGS) + ["conv_sweep"])
+    ap.add_argument("--workload", default="r1001", choices=sorted(wl.CONFIGS) + ["conv_sweep", "membound_sweep"])
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--conv-path", type=int, default=0)
     ap.add_argument("--skip-cpu-baseline", action="store_true")
@@ -276,6 +330,9 @@ def main():
         args.warmup = max(args.warmup, 3)
     if args.workload == "conv_sweep":
         conv_sweep(args)
+        return
+    if args.workload == "membound_sweep":
+        membound_sweep(args)
         return
     cfg = wl.config(args.workload)
     if args.impl == "reference":

@@ -201,9 +201,10 @@ struct alignas(64) WgradParams {
     int m_chunk;                 // output channels per CTA (<= 128)
     int n_cols;                  // input channels per CTA (<= 256)
     int taps_per_cta;
+    int taps_per_mma;            // taps stacked along N in one MMA (n_cols * taps_per_mma <= 256)
     int raw_stages, t_stages;
     int passes;                  // 1 or 3
-    unsigned int raw_bytes, t_bytes, tx_per_tap, tx_a, tmem_cols, idesc;
+    unsigned int raw_bytes, t_bytes, tx_per_tap, tx_a, tmem_cols, idesc, idesc_tail;
     long long split_stride;      // floats between partials
 };
 
@@ -392,8 +393,11 @@ __device__ __forceinline__ void transpose_tile(const uint8_t* raw, uint8_t* dst,
                                                uint32_t atom_stride, int tid)
 {
     const int items = channels * (rows >> 2);
+    const bool pow2 = (channels & (channels - 1)) == 0;
+    const int shift = 31 - __clz(channels);
     for (int it = tid; it < items; it += 128) {
-        const int c = it % channels, p4 = it / channels;
+        const int c = pow2 ? (it & (channels - 1)) : (it % channels);
+        const int p4 = pow2 ? (it >> shift) : (it / channels);
         const float* src = reinterpret_cast<const float*>(raw) + (p4 * 4) * channels + c;
         float4 v;
         v.x = src[0]; v.y = src[channels]; v.z = src[2 * channels]; v.w = src[3 * channels];
@@ -439,9 +443,12 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
     const int katoms = p.rows >> 5;
     const uint32_t raw_a = (uint32_t)p.rows * p.m_chunk * 4u, raw_b = (uint32_t)p.rows * p.n_cols * 4u;
     const uint32_t t_a = (uint32_t)katoms * 128u * 128u;                  // room for 128 channel rows
-    const uint32_t t_b = (uint32_t)katoms * (uint32_t)p.n_cols * 128u;
-    // transposed stage layout: A_hi | B_hi[taps] | A_lo | B_lo[taps]
-    const uint32_t t_half = t_a + (uint32_t)p.taps_per_cta * t_b;
+    // transposed B: [pixel group of 32][tap][input channel] rows of 128 bytes, so that consecutive taps are consecutive
+    // N rows of one operand and one MMA covers several taps at once
+    const uint32_t t_b_tap = (uint32_t)p.n_cols * 128u;                   // one tap inside one pixel group
+    const uint32_t t_b_atom = (uint32_t)p.taps_per_cta * t_b_tap;         // one pixel group, all taps
+    // transposed stage layout: A_hi | B_hi | A_lo | B_lo
+    const uint32_t t_half = t_a + (uint32_t)katoms * t_b_atom;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 4; ++s) {
@@ -490,22 +497,26 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
                 if (!mbar_wait(full_t0 + 8 * t, (it / p.t_stages) & 1, &abort_flag)) { report(p.status, 4); break; }
                 tc_fence_after();
                 const uint32_t a_src = smem_base + t_region0 + t * p.t_bytes, b_src = a_src + t_a;
-                for (int tp = 0; tp < ntaps; ++tp)
+                // taps are stacked along N: groups of up to 256 / n_cols taps per MMA
+                for (int tg = 0; tg < ntaps; tg += p.taps_per_mma) {
+                    const int nt = ntaps - tg < p.taps_per_mma ? ntaps - tg : p.taps_per_mma;
+                    const uint32_t idesc = nt == p.taps_per_mma ? p.idesc : p.idesc_tail;
+                    const uint32_t acc = tmem_base + (uint32_t)(tg * p.n_cols);
                     for (int kb = 0; kb < katoms; ++kb)
                         for (int k8 = 0; k8 < 4; ++k8) {
                             const uint32_t ao = (uint32_t)kb * 16384u + 32u * k8;
-                            const uint32_t bo = (uint32_t)tp * t_b + (uint32_t)kb * (uint32_t)p.n_cols * 128u + 32u * k8;
+                            const uint32_t bo = (uint32_t)kb * t_b_atom + (uint32_t)tg * t_b_tap + 32u * k8;
                             const uint64_t ad = smem_desc(a_src + ao, 16, 1024, 128);
                             const uint64_t bd = smem_desc(b_src + bo, 16, 1024, 128);
-                            const uint32_t acc = tmem_base + (uint32_t)(tp * p.n_cols);
-                            umma_tf32(acc, ad, bd, p.idesc, (it | kb | k8) ? 1u : 0u);
+                            umma_tf32(acc, ad, bd, idesc, (it | kb | k8) ? 1u : 0u);
                             if (p.passes == 3) {
                                 const uint64_t adl = smem_desc(a_src + t_half + ao, 16, 1024, 128);
                                 const uint64_t bdl = smem_desc(b_src + t_half + bo, 16, 1024, 128);
-                                umma_tf32(acc, adl, bd, p.idesc, 1u);
-                                umma_tf32(acc, ad, bdl, p.idesc, 1u);
+                                umma_tf32(acc, adl, bd, idesc, 1u);
+                                umma_tf32(acc, ad, bdl, idesc, 1u);
                             }
                         }
+                }
                 umma_commit(empty_t0 + 8 * t);
             }
             if (it == total) umma_commit(accum_bar);
@@ -526,13 +537,12 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
             if (p.passes == 3) {
                 transpose_tile<true>(raw, tdst, tdst + t_half, p.m_chunk, p.rows, 16384u, tid);
                 for (int tp = 0; tp < ntaps; ++tp)
-                    transpose_tile<true>(raw + raw_a + tp * raw_b, tdst + t_a + tp * t_b, tdst + t_half + t_a + tp * t_b, p.n_cols,
-                                         p.rows, (uint32_t)p.n_cols * 128u, tid);
+                    transpose_tile<true>(raw + raw_a + tp * raw_b, tdst + t_a + tp * t_b_tap, tdst + t_half + t_a + tp * t_b_tap,
+                                         p.n_cols, p.rows, t_b_atom, tid);
             } else {
                 transpose_tile<false>(raw, tdst, nullptr, p.m_chunk, p.rows, 16384u, tid);
                 for (int tp = 0; tp < ntaps; ++tp)
-                    transpose_tile<false>(raw + raw_a + tp * raw_b, tdst + t_a + tp * t_b, nullptr, p.n_cols, p.rows,
-                                          (uint32_t)p.n_cols * 128u, tid);
+                    transpose_tile<false>(raw + raw_a + tp * raw_b, tdst + t_a + tp * t_b_tap, nullptr, p.n_cols, p.rows, t_b_atom, tid);
             }
             fence_async_smem();     // generic-proxy writes -> tensor-core reads
             __syncwarp();
@@ -580,20 +590,28 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
     if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
 }
 
+// dw[i] = sum over splits of partials[z][i], in an order fixed by the launch shape: thread (lane, zl) adds the
+// splits zl, zl+8, ... ascending, then the 8 partial sums are added ascending.  32 float4 per block.
 __global__ void __launch_bounds__(256)
 wgrad_partials_reduce_kernel(const float* __restrict__ partials, float* __restrict__ dw, long long n, int splits)
 {
-    // n is a multiple of 4 and the partials are 16-byte aligned; dw (inside a gradient slot) may not be
-    const long long n4 = n / 4;
-    const bool dw_vec = (reinterpret_cast<uintptr_t>(dw) & 15u) == 0;
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
-        float4 s = __ldcg(reinterpret_cast<const float4*>(partials) + i);
-        for (int z = 1; z < splits; ++z) {
+    __shared__ float4 sh[8][32];
+    const int lane = threadIdx.x & 31, zl = threadIdx.x >> 5;
+    const long long n4 = n / 4;          // n is a multiple of 4 and the partials are 16-byte aligned; dw may not be
+    const long long i = (long long)blockIdx.x * 32 + lane;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i < n4) {
+#pragma unroll 4
+        for (int z = zl; z < splits; z += 8) {
             const float4 v = __ldcg(reinterpret_cast<const float4*>(partials + (long long)z * n) + i);
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
         }
-        if (dw_vec) reinterpret_cast<float4*>(dw)[i] = s;
+    }
+    sh[zl][lane] = s;
+    __syncthreads();
+    if (zl == 0 && i < n4) {
+        for (int k = 1; k < 8; ++k) { const float4 v = sh[k][lane]; s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w; }
+        if ((reinterpret_cast<uintptr_t>(dw) & 15u) == 0) reinterpret_cast<float4*>(dw)[i] = s;
         else { dw[4 * i] = s.x; dw[4 * i + 1] = s.y; dw[4 * i + 2] = s.z; dw[4 * i + 3] = s.w; }
     }
 }
@@ -787,9 +805,14 @@ bool wgrad_geom(const ConvShape& s, int passes, WgradGeom* g)
     const double operand_bytes = 4.0 * ((double)s.N * s.P * s.Q * s.K + (double)s.N * s.P * s.Q * s.C);
     const double dw_bytes = 4.0 * (double)s.K * taps * s.C;
     int splits = g->n_tiles / 4;
-    const int cap = (int)(operand_bytes / (4.0 * dw_bytes));
+    int cap = (int)(operand_bytes / (4.0 * dw_bytes));
+    // small problems are latency bound, not byte bound: spread the pixel walk over at least ~48 CTAs
+    const int ctas_per_split = g->tap_groups * (s.K / g->m_chunk) * (s.C / g->n_cols);
+    const int want = (48 + ctas_per_split - 1) / ctas_per_split;
+    if (cap < want) cap = want;
     if (splits > cap) splits = cap;
     if (splits > 64) splits = 64;
+    if (splits > g->n_tiles / 2) splits = g->n_tiles / 2;
     if (splits < 1) splits = 1;
     g->tiles_per_split = (g->n_tiles + splits - 1) / splits;
     g->splits = (g->n_tiles + g->tiles_per_split - 1) / g->tiles_per_split;
@@ -884,7 +907,9 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
         p.raw_bytes = g.raw_bytes; p.t_bytes = g.t_bytes;
         p.tx_a = (unsigned int)g.box.rows * g.m_chunk * 4u; p.tx_per_tap = (unsigned int)g.box.rows * g.n_cols * 4u;
         p.tmem_cols = g.tmem_cols;
-        p.idesc = instr_desc(g.n_cols, false, false);
+        p.taps_per_mma = 256 / g.n_cols < g.taps_per_cta ? 256 / g.n_cols : g.taps_per_cta;
+        p.idesc = instr_desc(g.n_cols * p.taps_per_mma, false, false);
+        p.idesc_tail = instr_desc(g.n_cols * (g.taps_per_cta % p.taps_per_mma ? g.taps_per_cta % p.taps_per_mma : p.taps_per_mma), false, false);
         p.split_stride = n_out;
         L->grid = dim3(g.splits, g.tap_groups, (s.K / g.m_chunk) * (s.C / g.n_cols));
         L->smem = (unsigned int)g.raw_stages * g.raw_bytes + (unsigned int)g.t_stages * g.t_bytes + 1024;
@@ -955,8 +980,7 @@ cudaError_t conv_tc_launch(const ConvTcPlan* plan, DeviceStatus* status, cudaStr
         conv_tc_wgrad_kernel<<<L.grid, 192, L.smem, st>>>(L.p);
         count(n_launch, 1);
         if (L.splits > 1) {
-            int nb = (int)((L.n_out / 4 + 255) / 256);
-            if (nb > 592) nb = 592;
+            const int nb = (int)((L.n_out / 4 + 31) / 32);
             wgrad_partials_reduce_kernel<<<nb, 256, 0, st>>>(L.p.out, L.dw, L.n_out, L.splits);
             count(n_launch, 1);
         }

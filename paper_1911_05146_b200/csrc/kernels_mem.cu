@@ -23,27 +23,40 @@ __host__ __device__ inline int64_t ceil_div64(int64_t a, int64_t b) { return (a 
 __device__ __forceinline__ float bn_xhat(float x, float mean, float rstd) { return (x - mean) * rstd; }
 __device__ __forceinline__ float bn_z(float xh, float g, float b) { return fmaf(g, xh, b); }
 
+// Thread layout shared by the BN kernels: a block of kBnThreads threads is (row lanes) x (float4 column groups);
+// a thread keeps its column group for the whole kernel, so per-channel coefficients live in registers and no
+// index arithmetic runs per element.
+constexpr int kBnThreads = 512;
+constexpr int kBnMaxBlocks = 128;        // bounds the partials the last block has to combine
+
 struct BnPlan {
     int cg_total;        // float4 column groups = C/4
-    int cgt;             // column groups handled per pass by one block (<= 256)
-    int rl;              // row lanes per block = 256 / cgt
+    int cgt;             // column groups handled per pass by one block (<= kBnThreads)
+    int rl;              // row lanes per block = kBnThreads / cgt
     int passes;          // ceil(cg_total / cgt)
-    int nblk;
+    int nblk;            // blocks of the reduction kernels
     int64_t rows_per_blk;
+    int nblk_apply;      // blocks of the apply kernels (no partials: as many as the rows allow)
+    int64_t rows_per_blk_apply;
 };
 
 BnPlan bn_plan(int64_t rows, int C)
 {
     BnPlan p;
     p.cg_total = C / 4;
-    p.cgt = p.cg_total < kThreads ? p.cg_total : kThreads;
-    p.rl = kThreads / p.cgt;
+    p.cgt = p.cg_total < kBnThreads ? p.cg_total : kBnThreads;
+    p.rl = kBnThreads / p.cgt;
     p.passes = (p.cg_total + p.cgt - 1) / p.cgt;
-    int64_t nb = rows / ((int64_t)p.rl * 16);
+    int64_t nb = rows / ((int64_t)p.rl * 8);
     if (nb < 1) nb = 1;
-    if (nb > kMaxBlocks) nb = kMaxBlocks;
+    if (nb > kBnMaxBlocks) nb = kBnMaxBlocks;
     p.rows_per_blk = ceil_div64(rows, nb);
     p.nblk = (int)ceil_div64(rows, p.rows_per_blk);
+    int64_t na = rows / ((int64_t)p.rl * 4);
+    if (na < 1) na = 1;
+    if (na > 148 * 8) na = 148 * 8;
+    p.rows_per_blk_apply = ceil_div64(rows, na);
+    p.nblk_apply = (int)ceil_div64(rows, p.rows_per_blk_apply);
     return p;
 }
 
@@ -52,18 +65,19 @@ BnPlan bn_plan(int64_t rows, int C)
 //                           -> mean, rstd = 1/sqrt(var + eps)      (shifted sums avoid cancellation)
 //   backward (BWD = true):  a = sum dz, b = sum dz * xhat, dz = dy * [z > 0]
 //                           -> dbeta, dgamma and the two per-row coefficients of the dx formula
-// Each block reduces its slab of rows, writes one partial per channel, and the block that takes the
-// last ticket adds the partials in ascending block order (fp64), so the result does not depend on
-// which block happens to finish last.
+// Each block reduces its slab of rows and writes one partial per channel; the block that takes the last
+// ticket combines the partials: every thread adds a fixed subset in ascending block order (fp64), a fixed
+// tree adds those, so the result does not depend on which block happens to finish last.
 template <bool BWD>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kBnThreads)
 bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, const float* __restrict__ gamma,
                  const float* __restrict__ beta, const float* __restrict__ stats, float eps, int64_t rows, int C,
                  int cgt, int rl, int passes, int64_t rows_per_blk, unsigned int* ticket,
                  float* __restrict__ partials, float* __restrict__ out_a, float* __restrict__ out_b,
                  float* __restrict__ coef)
 {
-    __shared__ float sh[kThreads][8];
+    __shared__ double shd[kBnThreads][8];            // 32 KB; the float phase uses it as float[kBnThreads][8]
+    float (*sh)[8] = reinterpret_cast<float (*)[8]>(&shd[0][0]);
     __shared__ int is_last;
     const int t = threadIdx.x;
     const int cg_total = C / 4;
@@ -87,11 +101,15 @@ bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, cons
             } else {
                 p0 = __ldg(x4 + cg);                                                  // shift = first row
             }
+            const float4* xp = x4 + (r0 + my_rl) * cg_total + cg;
+            const float4* dp = dy4 + (r0 + my_rl) * cg_total + cg;
+            const int64_t step = (int64_t)rl * cg_total;
+            const int n = (int)((r1 - r0 - my_rl + rl - 1) / rl);
 #pragma unroll 4
-            for (int64_t r = r0 + my_rl; r < r1; r += rl) {
-                const float4 v = __ldg(x4 + r * cg_total + cg);
+            for (int k = 0; k < n; ++k) {
+                const float4 v = __ldg(xp + k * step);
                 if (BWD) {
-                    const float4 g = __ldg(dy4 + r * cg_total + cg);
+                    const float4 g = __ldg(dp + k * step);
                     float xh, dz;
                     xh = bn_xhat(v.x, p0.x, p1.x); dz = bn_z(xh, gm.x, bt.x) > 0.f ? g.x : 0.f; a.x += dz; b.x = fmaf(dz, xh, b.x);
                     xh = bn_xhat(v.y, p0.y, p1.y); dz = bn_z(xh, gm.y, bt.y) > 0.f ? g.y : 0.f; a.y += dz; b.y = fmaf(dz, xh, b.y);
@@ -110,7 +128,7 @@ bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, cons
         sh[t][4] = b.x; sh[t][5] = b.y; sh[t][6] = b.z; sh[t][7] = b.w;
         __syncthreads();
         // one output per (column group, component): add the row lanes in ascending order
-        for (int o = t; o < cgt * 8; o += kThreads) {
+        for (int o = t; o < cgt * 8; o += kBnThreads) {
             const int cgl = o >> 3, comp = o & 7;
             const int cgo = pass * cgt + cgl;
             if (cgo < cg_total) {
@@ -132,48 +150,90 @@ bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, cons
     __syncthreads();
     if (!is_last) return;
     __threadfence();
+    // combine: thread (lane l, column group) adds the partials of blocks l, l+rl, ... (both sums, 4 channels each)
     const double inv_rows = 1.0 / (double)rows;
-    for (int c = t; c < C; c += kThreads) {
-        double sa = 0.0, sb = 0.0;
-        for (unsigned int k = 0; k < gridDim.x; ++k) {
-            sa += (double)__ldcg(&partials[((int64_t)k * 2 + 0) * C + c]);
-            sb += (double)__ldcg(&partials[((int64_t)k * 2 + 1) * C + c]);
+    const int nb = (int)gridDim.x;
+    for (int pass = 0; pass < passes; ++pass) {
+        const int cg = pass * cgt + my_cg;
+        double acc[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+        if (my_rl < rl && cg < cg_total) {
+#pragma unroll 2
+            for (int k = my_rl; k < nb; k += rl) {
+                const float4 va = __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 0) * C) + cg);
+                const float4 vb = __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 1) * C) + cg);
+                acc[0] += (double)va.x; acc[1] += (double)va.y; acc[2] += (double)va.z; acc[3] += (double)va.w;
+                acc[4] += (double)vb.x; acc[5] += (double)vb.y; acc[6] += (double)vb.z; acc[7] += (double)vb.w;
+            }
         }
-        if (BWD) {
-            out_a[c] = (float)sa;                 // dbeta
-            out_b[c] = (float)sb;                 // dgamma
-            coef[c] = (float)(sa * inv_rows);
-            coef[C + c] = (float)(sb * inv_rows);
-        } else {
-            const double shift = (double)__ldg(x + c);
-            const double ms = sa * inv_rows;
-            double var = sb * inv_rows - ms * ms;
-            if (var < 0.0) var = 0.0;
-            out_a[c] = (float)(shift + ms);                       // mean
-            out_b[c] = (float)(1.0 / sqrt(var + (double)eps));    // rstd
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < 8; ++j) shd[t][j] = acc[j];
+        __syncthreads();
+        for (int o = t; o < cgt * 8; o += kBnThreads) {
+            const int cgl = o >> 3, comp = o & 7;
+            const int cgo = pass * cgt + cgl;
+            if (cgo >= cg_total) continue;
+            double s = 0.0;
+            for (int l = 0; l < rl; ++l) s += shd[l * cgt + cgl][comp];
+            // the pair (a, b) of one channel is finished by two threads: exchange through shared memory
+            shd[cgl][comp] = s;       // row 0 lane (l = 0) slot of this column group: safe, every read above is done per o
         }
+        __syncthreads();
+        for (int cl = t; cl < cgt * 4; cl += kBnThreads) {
+            const int cgl = cl >> 2, e = cl & 3;
+            const int cgo = pass * cgt + cgl;
+            if (cgo >= cg_total) continue;
+            const int c = cgo * 4 + e;
+            const double sa = shd[cgl][e], sb = shd[cgl][4 + e];
+            if (BWD) {
+                out_a[c] = (float)sa;                 // dbeta
+                out_b[c] = (float)sb;                 // dgamma
+                coef[c] = (float)(sa * inv_rows);
+                coef[C + c] = (float)(sb * inv_rows);
+            } else {
+                const double shift = (double)__ldg(x + c);
+                const double ms = sa * inv_rows;
+                double var = sb * inv_rows - ms * ms;
+                if (var < 0.0) var = 0.0;
+                out_a[c] = (float)(shift + ms);                       // mean
+                out_b[c] = (float)(1.0 / sqrt(var + (double)eps));    // rstd
+            }
+        }
+        __syncthreads();
     }
     if (t == 0) *ticket = 0u;
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kBnThreads)
 bn_apply_fwd_kernel(const float4* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
-                    const float* __restrict__ stats, float4* __restrict__ y, int64_t n4, int cg_total, int C)
+                    const float* __restrict__ stats, float4* __restrict__ y, int64_t rows, int C, int cgt, int rl,
+                    int passes, int64_t rows_per_blk)
 {
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
-        const int cg = (int)(i % cg_total);
-        const float4 v = __ldg(x + i);
+    const int t = threadIdx.x, cg_total = C / 4;
+    const int my_rl = t / cgt, my_cg = t % cgt;
+    const int64_t r0 = (int64_t)blockIdx.x * rows_per_blk;
+    int64_t r1 = r0 + rows_per_blk;
+    if (r1 > rows) r1 = rows;
+    if (my_rl >= rl) return;
+    for (int pass = 0; pass < passes; ++pass) {
+        const int cg = pass * cgt + my_cg;
+        if (cg >= cg_total) continue;
         const float4 mu = __ldg(reinterpret_cast<const float4*>(stats) + cg);
         const float4 rs = __ldg(reinterpret_cast<const float4*>(stats + C) + cg);
         const float4 g = __ldg(reinterpret_cast<const float4*>(gamma) + cg);
         const float4 b = __ldg(reinterpret_cast<const float4*>(beta) + cg);
-        float4 o;
-        o.x = fmaxf(bn_z(bn_xhat(v.x, mu.x, rs.x), g.x, b.x), 0.f);
-        o.y = fmaxf(bn_z(bn_xhat(v.y, mu.y, rs.y), g.y, b.y), 0.f);
-        o.z = fmaxf(bn_z(bn_xhat(v.z, mu.z, rs.z), g.z, b.z), 0.f);
-        o.w = fmaxf(bn_z(bn_xhat(v.w, mu.w, rs.w), g.w, b.w), 0.f);
-        y[i] = o;
+        const int64_t base = (r0 + my_rl) * cg_total + cg, step = (int64_t)rl * cg_total;
+        const int n = (int)((r1 - r0 - my_rl + rl - 1) / rl);
+#pragma unroll 4
+        for (int k = 0; k < n; ++k) {
+            const float4 v = __ldg(x + base + k * step);
+            float4 o;
+            o.x = fmaxf(bn_z(bn_xhat(v.x, mu.x, rs.x), g.x, b.x), 0.f);
+            o.y = fmaxf(bn_z(bn_xhat(v.y, mu.y, rs.y), g.y, b.y), 0.f);
+            o.z = fmaxf(bn_z(bn_xhat(v.z, mu.z, rs.z), g.z, b.z), 0.f);
+            o.w = fmaxf(bn_z(bn_xhat(v.w, mu.w, rs.w), g.w, b.w), 0.f);
+            y[base + k * step] = o;
+        }
     }
 }
 
@@ -185,37 +245,50 @@ __device__ __forceinline__ float bn_dx1(float x, float dy, float mu, float rs, f
 }
 
 template <bool ADDEND, bool ACCUM>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kBnThreads)
 bn_apply_bwd_kernel(const float4* __restrict__ x, const float4* __restrict__ dy, const float* __restrict__ gamma,
                     const float* __restrict__ beta, const float* __restrict__ stats, const float* __restrict__ coef,
-                    const float4* __restrict__ addend, float4* __restrict__ dx, int64_t n4, int cg_total, int C)
+                    const float4* __restrict__ addend, float4* __restrict__ dx, int64_t rows, int C, int cgt, int rl,
+                    int passes, int64_t rows_per_blk)
 {
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
-        const int cg = (int)(i % cg_total);
-        const float4 v = __ldg(x + i);
-        const float4 d = __ldg(dy + i);
+    const int t = threadIdx.x, cg_total = C / 4;
+    const int my_rl = t / cgt, my_cg = t % cgt;
+    const int64_t r0 = (int64_t)blockIdx.x * rows_per_blk;
+    int64_t r1 = r0 + rows_per_blk;
+    if (r1 > rows) r1 = rows;
+    if (my_rl >= rl) return;
+    for (int pass = 0; pass < passes; ++pass) {
+        const int cg = pass * cgt + my_cg;
+        if (cg >= cg_total) continue;
         const float4 mu = __ldg(reinterpret_cast<const float4*>(stats) + cg);
         const float4 rs = __ldg(reinterpret_cast<const float4*>(stats + C) + cg);
         const float4 g = __ldg(reinterpret_cast<const float4*>(gamma) + cg);
         const float4 b = __ldg(reinterpret_cast<const float4*>(beta) + cg);
         const float4 ca = __ldcg(reinterpret_cast<const float4*>(coef) + cg);
         const float4 cb = __ldcg(reinterpret_cast<const float4*>(coef + C) + cg);
-        float4 o;
-        o.x = bn_dx1(v.x, d.x, mu.x, rs.x, g.x, b.x, ca.x, cb.x);
-        o.y = bn_dx1(v.y, d.y, mu.y, rs.y, g.y, b.y, ca.y, cb.y);
-        o.z = bn_dx1(v.z, d.z, mu.z, rs.z, g.z, b.z, ca.z, cb.z);
-        o.w = bn_dx1(v.w, d.w, mu.w, rs.w, g.w, b.w, ca.w, cb.w);
-        if (ADDEND) { const float4 e = __ldg(addend + i); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
-        if (ACCUM) { const float4 e = dx[i]; o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
-        dx[i] = o;
+        const int64_t base = (r0 + my_rl) * cg_total + cg, step = (int64_t)rl * cg_total;
+        const int n = (int)((r1 - r0 - my_rl + rl - 1) / rl);
+#pragma unroll 4
+        for (int k = 0; k < n; ++k) {
+            const int64_t i = base + k * step;
+            const float4 v = __ldg(x + i);
+            const float4 d = __ldg(dy + i);
+            float4 o;
+            o.x = bn_dx1(v.x, d.x, mu.x, rs.x, g.x, b.x, ca.x, cb.x);
+            o.y = bn_dx1(v.y, d.y, mu.y, rs.y, g.y, b.y, ca.y, cb.y);
+            o.z = bn_dx1(v.z, d.z, mu.z, rs.z, g.z, b.z, ca.z, cb.z);
+            o.w = bn_dx1(v.w, d.w, mu.w, rs.w, g.w, b.w, ca.w, cb.w);
+            if (ADDEND) { const float4 e = __ldg(addend + i); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+            if (ACCUM) { const float4 e = dx[i]; o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+            dx[i] = o;
+        }
     }
 }
 
 int ew_blocks(int64_t n_items)
 {
     int64_t nb = ceil_div64(n_items, kThreads);
-    if (nb > kMaxBlocks * 2) nb = kMaxBlocks * 2;
+    if (nb > kMaxBlocks * 4) nb = kMaxBlocks * 4;
     if (nb < 1) nb = 1;
     return (int)nb;
 }
@@ -252,29 +325,29 @@ accumulate_kernel(float* __restrict__ dst, const float* __restrict__ src, int64_
 }
 
 // out[j] = (slots[0][j] + slots[1][j] + ... + slots[M-1][j]) / M, ascending m.  Reads M*G floats,
-// writes G: pure streaming, one float4 per slot per thread in flight.
+// writes G: pure streaming.  Slot m starts at m*G floats, so the widest aligned access depends on G:
+// VEC = 4 when G % 4 == 0, 2 when G is even, else 1.
+template <int VEC>
 __global__ void __launch_bounds__(kThreads)
 grad_average_kernel(const float* __restrict__ slots, float* __restrict__ out, int M, int64_t G, float inv_m)
 {
-    const int64_t n4 = G / 4;
+    const int64_t nv = G / VEC;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const bool vec = (G % 4 == 0);       // slot m starts at m*G floats: 16-byte aligned only then
-    if (vec) {
-        for (int64_t i = t0; i < n4; i += stride) {
-            float4 s = __ldcs(reinterpret_cast<const float4*>(slots) + i);
-            for (int m = 1; m < M; ++m) {
-                const float4 v = __ldcs(reinterpret_cast<const float4*>(slots + (int64_t)m * G) + i);
-                s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
-            }
-            reinterpret_cast<float4*>(out)[i] = make_float4(s.x * inv_m, s.y * inv_m, s.z * inv_m, s.w * inv_m);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nv; i += stride) {
+        float s[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) s[e] = 0.f;
+#pragma unroll 8
+        for (int m = 0; m < M; ++m) {
+            const float* src = slots + (int64_t)m * G + i * VEC;
+            if (VEC == 4) { const float4 v = __ldcs(reinterpret_cast<const float4*>(src)); s[0] += v.x; s[1] += v.y; s[2 % VEC] += v.z; s[3 % VEC] += v.w; }
+            else if (VEC == 2) { const float2 v = __ldcs(reinterpret_cast<const float2*>(src)); s[0] += v.x; s[1 % VEC] += v.y; }
+            else s[0] += __ldcs(src);
         }
-    } else {
-        for (int64_t i = t0; i < G; i += stride) {
-            float s = slots[i];
-            for (int m = 1; m < M; ++m) s += slots[(int64_t)m * G + i];
-            out[i] = s * inv_m;
-        }
+        float* dst = out + i * VEC;
+        if (VEC == 4) *reinterpret_cast<float4*>(dst) = make_float4(s[0] * inv_m, s[1 % VEC] * inv_m, s[2 % VEC] * inv_m, s[3 % VEC] * inv_m);
+        else if (VEC == 2) *reinterpret_cast<float2*>(dst) = make_float2(s[0] * inv_m, s[1 % VEC] * inv_m);
+        else dst[0] = s[0] * inv_m;
     }
 }
 
@@ -502,12 +575,12 @@ cudaError_t bnrelu_fwd(const float* x, const float* gamma, const float* beta, fl
     const BnPlan p = bn_plan(rows, C);
     unsigned int* ticket = reinterpret_cast<unsigned int*>(scratch);
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + 256);
-    bn_reduce_kernel<false><<<p.nblk, kThreads, 0, st>>>(x, nullptr, gamma, beta, nullptr, eps, rows, C, p.cgt, p.rl,
-                                                         p.passes, p.rows_per_blk, ticket, partials, stats, stats + C,
-                                                         nullptr);
-    const int64_t n4 = rows * (C / 4);
-    bn_apply_fwd_kernel<<<ew_blocks(n4), kThreads, 0, st>>>(reinterpret_cast<const float4*>(x), gamma, beta, stats,
-                                                            reinterpret_cast<float4*>(y), n4, C / 4, C);
+    bn_reduce_kernel<false><<<p.nblk, kBnThreads, 0, st>>>(x, nullptr, gamma, beta, nullptr, eps, rows, C, p.cgt, p.rl,
+                                                           p.passes, p.rows_per_blk, ticket, partials, stats, stats + C,
+                                                           nullptr);
+    bn_apply_fwd_kernel<<<p.nblk_apply, kBnThreads, 0, st>>>(reinterpret_cast<const float4*>(x), gamma, beta, stats,
+                                                             reinterpret_cast<float4*>(y), rows, C, p.cgt, p.rl, p.passes,
+                                                             p.rows_per_blk_apply);
     count(n_launch, 2);
     return cudaGetLastError();
 }
@@ -520,22 +593,19 @@ cudaError_t bnrelu_bwd(const float* x, const float* dy, const float* gamma, cons
     unsigned int* ticket = reinterpret_cast<unsigned int*>(scratch);
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + 256);
     float* coef = partials + (size_t)p.nblk * 2 * C;
-    bn_reduce_kernel<true><<<p.nblk, kThreads, 0, st>>>(x, dy, gamma, beta, stats, 0.f, rows, C, p.cgt, p.rl, p.passes,
-                                                        p.rows_per_blk, ticket, partials, dbeta, dgamma, coef);
-    const int64_t n4 = rows * (C / 4);
-    const int nb = ew_blocks(n4);
+    bn_reduce_kernel<true><<<p.nblk, kBnThreads, 0, st>>>(x, dy, gamma, beta, stats, 0.f, rows, C, p.cgt, p.rl, p.passes,
+                                                          p.rows_per_blk, ticket, partials, dbeta, dgamma, coef);
     const float4* x4 = reinterpret_cast<const float4*>(x);
     const float4* dy4 = reinterpret_cast<const float4*>(dy);
     const float4* ad4 = reinterpret_cast<const float4*>(addend);
     float4* dx4 = reinterpret_cast<float4*>(dx);
-    if (addend && accumulate)
-        bn_apply_bwd_kernel<true, true><<<nb, kThreads, 0, st>>>(x4, dy4, gamma, beta, stats, coef, ad4, dx4, n4, C / 4, C);
-    else if (addend)
-        bn_apply_bwd_kernel<true, false><<<nb, kThreads, 0, st>>>(x4, dy4, gamma, beta, stats, coef, ad4, dx4, n4, C / 4, C);
-    else if (accumulate)
-        bn_apply_bwd_kernel<false, true><<<nb, kThreads, 0, st>>>(x4, dy4, gamma, beta, stats, coef, ad4, dx4, n4, C / 4, C);
-    else
-        bn_apply_bwd_kernel<false, false><<<nb, kThreads, 0, st>>>(x4, dy4, gamma, beta, stats, coef, ad4, dx4, n4, C / 4, C);
+    const int nb = p.nblk_apply;
+#define HPF_BN_APPLY(A, B) bn_apply_bwd_kernel<A, B><<<nb, kBnThreads, 0, st>>>(x4, dy4, gamma, beta, stats, coef, ad4, dx4, rows, C, p.cgt, p.rl, p.passes, p.rows_per_blk_apply)
+    if (addend && accumulate) HPF_BN_APPLY(true, true);
+    else if (addend) HPF_BN_APPLY(true, false);
+    else if (accumulate) HPF_BN_APPLY(false, true);
+    else HPF_BN_APPLY(false, false);
+#undef HPF_BN_APPLY
     count(n_launch, 2);
     return cudaGetLastError();
 }
@@ -557,7 +627,11 @@ cudaError_t grad_accumulate(float* dst, const float* src, int64_t n, bool accumu
 
 cudaError_t grad_average(const float* slots, float* out, int M, int64_t G, cudaStream_t st, int64_t* n_launch)
 {
-    grad_average_kernel<<<ew_blocks(G / 4 + 1), kThreads, 0, st>>>(slots, out, M, G, 1.f / (float)M);
+    const float inv_m = 1.f / (float)M;
+    const bool out16 = (reinterpret_cast<uintptr_t>(out) & 15u) == 0 && (reinterpret_cast<uintptr_t>(slots) & 15u) == 0;
+    if (G % 4 == 0 && out16) grad_average_kernel<4><<<ew_blocks(G / 4), kThreads, 0, st>>>(slots, out, M, G, inv_m);
+    else if (G % 2 == 0 && out16) grad_average_kernel<2><<<ew_blocks(G / 2), kThreads, 0, st>>>(slots, out, M, G, inv_m);
+    else grad_average_kernel<1><<<ew_blocks(G), kThreads, 0, st>>>(slots, out, M, G, inv_m);
     count(n_launch, 1);
     return cudaGetLastError();
 }
