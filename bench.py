@@ -367,7 +367,7 @@ def main():
     avg = torch.empty(G, device=dev)
     ws_bytes = model.workspace_bytes()
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
-    streams = [torch.cuda.Stream(device=dev) for _ in range(model.num_partitions())]
+    streams = [torch.cuda.Stream(device=dev) for _ in range(2 * model.num_partitions())]     # stage streams + weight-gradient side streams
     torch.cuda.synchronize()
     model.bind(params, slots, avg, ws, streams)
     dx, dl = torch.from_numpy(x).to(dev), torch.from_numpy(labels).to(dev)

@@ -119,8 +119,9 @@ int hpf_workspace_bytes(const hpf_model *model, size_t *bytes);
 /* d_params [G], d_grad_slots [M][G] (slot m = dL_m/dtheta), d_grad_avg [G], d_workspace (256-byte
  * aligned, >= hpf_workspace_bytes): all caller-owned device memory that must outlive the model.
  * cuda_streams: n_streams >= P cudaStream_t handles (stage p runs on stream p; stream 0 is the one
- * the phases fork from and join to).  Creates events and tensor-map descriptors; allocates nothing
- * on the device.  Errors: HPF_ERR_WORKSPACE, HPF_ERR_INVALID, HPF_ERR_CUDA. */
+ * the phases fork from and join to).  With n_streams >= 2P, stream P+p carries stage p's weight-gradient
+ * kernels, which feed only the final average and so leave the chain of dependent kernels.  Creates
+ * events and tensor-map descriptors; allocates nothing on the device.  Errors: HPF_ERR_WORKSPACE, HPF_ERR_INVALID, HPF_ERR_CUDA. */
 int hpf_bind(hpf_model *model, float *d_params, float *d_grad_slots, float *d_grad_avg, void *d_workspace,
              size_t ws_bytes, void *const *cuda_streams, int32_t n_streams);
 

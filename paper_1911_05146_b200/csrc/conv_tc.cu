@@ -44,6 +44,7 @@ namespace {
 constexpr int kTileM = 128;                 // MMA M (TMEM lanes)
 constexpr long long kWaitLimit = 4000000000LL;   // clock64 ticks (~2 s) before a wait gives up
 constexpr uint32_t kSmemBudget = 200 * 1024;
+constexpr int kFwdMaxStages = 3;              // shallow pipelines leave shared memory for CTAs of other streams
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -791,7 +792,7 @@ bool wgrad_geom(const ConvShape& s, int passes, WgradGeom* g)
                 g->box = b; g->raw_bytes = raw_al; g->t_bytes = tb;
                 g->t_stages = 2;
                 int rs = (int)((kSmemBudget - 2 * tb) / raw_al);
-                g->raw_stages = rs > 4 ? 4 : rs;
+                g->raw_stages = rs > 2 ? 2 : rs;
                 found = true;
             }
         }
@@ -960,7 +961,7 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     p.tx_bytes = (unsigned int)b.rows * kchunk * 4 + parts * (unsigned int)n_chunk * kchunk * 4;
     int stages = (int)(kSmemBudget / p.stage_bytes);
     const int total = v.R * v.R * p.n_kchunks;
-    if (stages > 6) stages = 6;
+    if (stages > kFwdMaxStages) stages = kFwdMaxStages;
     if (stages > total) stages = total;
     p.stages = stages;
     p.tmem_cols = pow2_cols(n_chunk);

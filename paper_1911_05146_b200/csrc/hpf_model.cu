@@ -101,6 +101,8 @@ struct hpf_model {
     std::vector<cudaStream_t> streams;
     std::vector<cudaEvent_t> ev_fwd, ev_bwd;  // [cut * M + m]
     std::vector<cudaEvent_t> ev_join;         // per stream
+    std::vector<cudaStream_t> side;           // per partition: weight-gradient stream (empty: none)
+    std::vector<cudaEvent_t> ev_side, ev_side_join;   // per partition: gradient ready -> side stream; side stream done
     cudaEvent_t ev_fork = nullptr, ev_sync = nullptr;
     // tensor-core plans [m * n_ops + op] per pass
     std::vector<ConvTcPlan> tc_plan[3];
@@ -479,10 +481,18 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
     switch (q.kind) {
     case HPF_OP_CONV: {
         const ConvShape s = conv_shape_of(mdl, i);
+        // The weight gradient feeds nothing but the final average, so it leaves the chain of dependent kernels:
+        // it runs on the partition's side stream once dL/d(output) is ready (everything before this point on st).
+        cudaStream_t wst = st;
+        if (!mdl->side.empty() && !mdl->opt_single) {
+            wst = mdl->side[p];
+            CU(cudaEventRecord(mdl->ev_side[p], st));
+            CU(cudaStreamWaitEvent(wst, mdl->ev_side[p], 0));
+        }
         if (mdl->use_tc[PASS_WGRAD][i]) {
-            CU(conv_tc_launch(&mdl->tc_plan[PASS_WGRAD][(size_t)m * mdl->n_ops + i], mdl->status(), st, &mdl->launches));
+            CU(conv_tc_launch(&mdl->tc_plan[PASS_WGRAD][(size_t)m * mdl->n_ops + i], mdl->status(), wst, &mdl->launches));
         } else {
-            CU(conv_wgrad_simt(in0, dout, slot + o.w_off, s, mdl->ws + mdl->conv_scratch_off[p], st, &mdl->launches));
+            CU(conv_wgrad_simt(in0, dout, slot + o.w_off, s, mdl->ws + mdl->conv_scratch_off[p], wst, &mdl->launches));
         }
         if (q.src0 >= 0) {
             if (mdl->use_tc[PASS_DGRAD][i]) {
@@ -574,6 +584,14 @@ int enqueue_phase(hpf_model* mdl, int phase)
                 if (p > 0 && multi) CU(cudaEventRecord(mdl->ev_bwd[(size_t)(p - 1) * M + m], st));       // send partial errors
             }
     }
+    if (phase == PH_BWD && !mdl->side.empty() && !mdl->opt_single)
+        for (int p = 0; p < P; ++p) {
+            // the side stream holds work only if it was forked during this phase; joining an unforked stream is harmless
+            CU(cudaEventRecord(mdl->ev_side[p], mdl->stream_of(p)));
+            CU(cudaStreamWaitEvent(mdl->side[p], mdl->ev_side[p], 0));
+            CU(cudaEventRecord(mdl->ev_side_join[p], mdl->side[p]));
+            CU(cudaStreamWaitEvent(s0, mdl->ev_side_join[p], 0));
+        }
     if (multi)
         for (int p = 1; p < P; ++p) {
             CU(cudaEventRecord(mdl->ev_join[p], mdl->streams[p]));
@@ -646,6 +664,9 @@ void release_device_objects(hpf_model* mdl)
     for (auto e : mdl->ev_fwd) cudaEventDestroy(e);
     for (auto e : mdl->ev_bwd) cudaEventDestroy(e);
     for (auto e : mdl->ev_join) if (e) cudaEventDestroy(e);
+    for (auto e : mdl->ev_side) if (e) cudaEventDestroy(e);
+    for (auto e : mdl->ev_side_join) if (e) cudaEventDestroy(e);
+    mdl->ev_side.clear(); mdl->ev_side_join.clear();
     if (mdl->ev_fork) cudaEventDestroy(mdl->ev_fork);
     if (mdl->ev_sync) cudaEventDestroy(mdl->ev_sync);
     mdl->ev_fwd.clear(); mdl->ev_bwd.clear(); mdl->ev_join.clear();
@@ -801,6 +822,16 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
     mdl->ws = reinterpret_cast<char*>(d_workspace);
     mdl->streams.resize(mdl->P);
     for (int p = 0; p < mdl->P; ++p) mdl->streams[p] = reinterpret_cast<cudaStream_t>(cuda_streams[p]);
+    mdl->side.clear();
+    if (n_streams >= 2 * mdl->P) {
+        mdl->side.resize(mdl->P);
+        for (int p = 0; p < mdl->P; ++p) mdl->side[p] = reinterpret_cast<cudaStream_t>(cuda_streams[mdl->P + p]);
+        mdl->ev_side.assign(mdl->P, nullptr); mdl->ev_side_join.assign(mdl->P, nullptr);
+        for (int p = 0; p < mdl->P; ++p) {
+            CU(cudaEventCreateWithFlags(&mdl->ev_side[p], cudaEventDisableTiming));
+            CU(cudaEventCreateWithFlags(&mdl->ev_side_join[p], cudaEventDisableTiming));
+        }
+    }
     const int M = mdl->M, n = mdl->n_ops;
     CU(cudaEventCreateWithFlags(&mdl->ev_fork, cudaEventDisableTiming));
     CU(cudaEventCreateWithFlags(&mdl->ev_sync, cudaEventDisableTiming));

@@ -28,7 +28,7 @@ def rel_l2(a, ref):
 class Bound:
     """A model bound to torch-owned device memory."""
 
-    def __init__(self, ops, in_hwc, B, M, cuts, theta, options=None, device="cuda:0"):
+    def __init__(self, ops, in_hwc, B, M, cuts, theta, options=None, device="cuda:0", side_streams=True):
         self.ops, self.in_hwc, self.B, self.M, self.cuts = ops, tuple(in_hwc), B, M, list(cuts)
         self.dev = torch.device(device)
         torch.cuda.set_device(self.dev)
@@ -40,7 +40,8 @@ class Bound:
         self.slots = torch.full((M, self.G), float("nan"), dtype=torch.float32, device=self.dev)
         self.avg = torch.full((self.G,), float("nan"), dtype=torch.float32, device=self.dev)
         self.ws = torch.empty(self.model.workspace_bytes(), dtype=torch.uint8, device=self.dev)
-        self.streams = [torch.cuda.Stream(device=self.dev) for _ in range(self.model.num_partitions())]
+        n_streams = self.model.num_partitions() * (2 if side_streams else 1)
+        self.streams = [torch.cuda.Stream(device=self.dev) for _ in range(n_streams)]
         torch.cuda.synchronize()
         self.model.bind(self.params, self.slots, self.avg, self.ws, self.streams)
 

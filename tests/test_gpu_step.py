@@ -121,13 +121,14 @@ def test_single_stream_equals_multi_stream_bitwise():
     x, labels, theta = seeded(ops, (32, 32, 3), 8, seed=4)
     cuts = wl.default_cuts(len(ops), 4)
     outs = []
-    for single in (0, 1):
-        bd = Bound(ops, (32, 32, 3), 8, 4, cuts, theta, {hpf.OPT_SINGLE_STREAM: single})
+    for single, side in ((0, True), (1, True), (0, False)):
+        bd = Bound(ops, (32, 32, 3), 8, 4, cuts, theta, {hpf.OPT_SINGLE_STREAM: single}, side_streams=side)
         bd.upload(x, labels)
         loss = bd.step()
         outs.append((loss, bd.slots.clone(), bd.avg.clone()))
-    assert outs[0][0] == outs[1][0]
-    assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
+    for o in outs[1:]:
+        assert outs[0][0] == o[0]
+        assert torch.equal(outs[0][1], o[1]) and torch.equal(outs[0][2], o[2])
 
 
 def test_messages_across_cuts_match_the_oracle():
