@@ -155,6 +155,26 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def max_over_ranks(dist, values, device):
+    """Step times of a multi-rank run: the slowest rank counts (all_reduce MAX; no data-path collective)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def replica_inputs(cfg, rank):
+    """Rank r's replica: its own batch (seeded by rank), the same parameters on every rank."""
+    x, labels = wl.draw_inputs(cfg["B"], cfg["in_hwc"], cfg["ops"][-1].c_out, seed_x=wl.inputs.SEED_X + rank,
+                               seed_labels=wl.inputs.SEED_LABELS + rank)
+    return x, labels, wl.draw_params(cfg["ops"])
+
+
+def aggregate_throughput(world, batch_per_rank, ms_per_step):
+    """Whole-job images/s of `world` replicas that each finish a batch every ms_per_step (weak scaling)."""
+    return world * batch_per_rank / (ms_per_step * 1e-3)
+
+
 def kernel_roofline(torch, hpf, cfg, pk):
     """Times the dominant kernel of the step (fused BN+ReLU backward) alone, through the C ABI, on the
     workload's most frequent shape, cycling through operand sets that together exceed L2."""
@@ -211,6 +231,8 @@ def conv_sweep(args):
     N, rows_out = 128, []
     dev = "cuda"
     for (ks, st, ci, co, H) in wl.conv_sweep_shapes():
+        if args.sweep_filter and args.sweep_filter not in "%dx%d s%d %d->%d @%d" % (ks, ks, st, ci, co, H):
+            continue
         pad = 1 if ks == 3 else 0
         P = (H + 2 * pad - ks) // st + 1
         x_el, y_el, w_el = N * H * H * ci, N * P * P * co, co * ks * ks * ci
@@ -234,7 +256,7 @@ def conv_sweep(args):
         for name, fn in calls.items():
             for k in range(nset):
                 fn(k)
-            reps = max(10, 3 * nset)
+            reps = 2 if args.profile else max(10, 3 * nset)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             torch.cuda.synchronize()
             e0.record()
@@ -321,6 +343,7 @@ def main():
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-kernel-roofline", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--sweep-filter", default="", help="conv_sweep: only shapes whose label contains this text")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under a profiler: honour --warmup below 3 and skip the side measurements")
     args = ap.parse_args()
@@ -356,8 +379,7 @@ def main():
     pk = peaks()
 
     ops, hwc, B, M = cfg["ops"], cfg["in_hwc"], cfg["B"], cfg["M"]
-    x, labels = wl.draw_inputs(B, hwc, ops[-1].c_out, seed_x=wl.inputs.SEED_X + rank)     # each replica its own batch
-    theta = wl.draw_params(ops)
+    x, labels, theta = replica_inputs(cfg, rank)          # each replica its own batch, shared parameters
     model = hpf.Model(ops, (B,) + tuple(hwc), cfg["cuts"], M)
     model.set_option(hpf.OPT_GRAPH, 0 if args.no_graph else 1)
     model.set_option(hpf.OPT_CONV_PATH, args.conv_path)
@@ -418,16 +440,14 @@ def main():
         ms_e2e = e0.elapsed_time(e1)
 
     if dist is not None:
-        t = torch.tensor([ms, ms_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = t.tolist()
+        ms, ms_e2e = max_over_ranks(dist, [ms, ms_e2e], dev)
     if rank != 0:
         if dist is not None:
             dist.barrier(); dist.destroy_process_group()
         return
 
     ms_step = ms / args.steps
-    value = world * B / (ms_step * 1e-3)
+    value = aggregate_throughput(world, B, ms_step)
     by, flops = step_model(ops, hwc, B)
     step_bytes = sum(by.values())
     n_tc, n_cc = model.conv_path_counts()

@@ -31,7 +31,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     procs = []
     for src in _sources():
         obj = os.path.join(CSRC, os.path.basename(src)[:-3] + ".o")
-        cmd = [nvcc] + [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")] + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
+        extra = os.environ.get("HPF_NVCC_EXTRA", "").split()          # e.g. -DHPF_TC_TIMELINE for latency studies
+        cmd = [nvcc] + [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")] + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
         procs.append((cmd, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     for cmd, p in procs:

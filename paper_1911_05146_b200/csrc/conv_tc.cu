@@ -44,7 +44,7 @@ namespace {
 constexpr int kTileM = 128;                 // MMA M (TMEM lanes)
 constexpr long long kWaitLimit = 4000000000LL;   // clock64 ticks (~2 s) before a wait gives up
 constexpr uint32_t kSmemBudget = 200 * 1024;
-constexpr int kFwdMaxStages = 3;              // shallow pipelines leave shared memory for CTAs of other streams
+constexpr int kFwdMaxStages = 4;
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -144,6 +144,25 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v)
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// The same without the wait, so that several loads can be in flight before one tmem_ld_wait().
+__device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, float* v)
+{
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void prefetch_tmap(const void* tmap)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
+}
+
 // Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte offsets in
 // 16-byte units, descriptor version 1, swizzle mode in the top bits (2 = 128 B, 4 = 64 B).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t swizzle_bytes)
@@ -160,6 +179,20 @@ inline uint32_t instr_desc(int n, bool a_mn_major, bool b_mn_major)
            ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
 }
 
+// Optional timeline of CTA (0,0) for latency studies: globaltimer stamps behind the status word (debug builds only).
+#ifdef HPF_TC_TIMELINE
+#define HPF_TL(slot)                                                                                      \
+    do {                                                                                                  \
+        if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {                                      \
+            unsigned long long t_;                                                                        \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                        \
+            reinterpret_cast<unsigned long long*>(p.status)[2 + (slot)] = t_;                             \
+        }                                                                                                 \
+    } while (0)
+#else
+#define HPF_TL(slot) do {} while (0)
+#endif
+
 __device__ __forceinline__ void report(DeviceStatus* status, unsigned int code)
 {
     if (atomicCAS(&status->code, 0u, code) == 0u) status->detail = blockIdx.x;
@@ -168,10 +201,10 @@ __device__ __forceinline__ void report(DeviceStatus* status, unsigned int code)
 // ------------------------------------------------------------------------------------------------
 // kernel parameters
 // ------------------------------------------------------------------------------------------------
-struct alignas(64) FwdParams {
-    CUtensorMap tm_a;            // activations {C, Wv, Hv, N}
-    CUtensorMap tm_b;            // weights, hi part {taps*C, c_out}
-    CUtensorMap tm_b_lo;         // weights, lo part (three-pass mode)
+// The scalar part of the parameters is copied to shared memory by the first warps at kernel start: a kernel
+// parameter block of this size spans several constant-cache lines, and first touches from the single-thread
+// roles (producer, MMA issuer) and from the epilogue would each pay a serialised miss on the critical path.
+struct FwdScalars {
     float* out;
     const float* extra;
     DeviceStatus* status;
@@ -186,14 +219,19 @@ struct alignas(64) FwdParams {
     int swizzle;
     int stages;
     int passes;                  // 1 or 3
+    int stacked;                 // three-pass: hi*hi and hi*lo come from one MMA over [B_hi; B_lo] (needs 2*n_chunk <= 256)
     int zero_fill;               // > 1: the output pixel grid is strided, fill the rest of each patch with zeros
     int out_h, out_w;            // dense output extent (zero fill bounds)
-    unsigned int a_bytes, b_bytes, stage_bytes, tx_bytes, tmem_cols, idesc;
+    unsigned int a_bytes, b_bytes, stage_bytes, tx_bytes, tmem_cols, idesc, idesc2, stg_pitch;
+};
+struct alignas(64) FwdParams {
+    CUtensorMap tm_a;            // activations {C, Wv, Hv, N}
+    CUtensorMap tm_b;            // weights, hi part {taps*C, c_out}
+    CUtensorMap tm_b_lo;         // weights, lo part (three-pass mode)
+    FwdScalars s;
 };
 
-struct alignas(64) WgradParams {
-    CUtensorMap tm_a;            // dy {c_out, Q, P, N}, box {m_chunk, w, h, n}, no swizzle
-    CUtensorMap tm_b;            // x {C, Wv, Hv, N}, box {n_cols, w, h, n}, no swizzle
+struct WgradScalars {
     float* out;                  // dw or partials [splits][c_out*taps*c_in]
     DeviceStatus* status;
     int box_w, box_h, box_n, tiles_w, tiles_h, n_tiles, tiles_per_split;
@@ -208,6 +246,19 @@ struct alignas(64) WgradParams {
     unsigned int raw_bytes, t_bytes, tx_per_tap, tx_a, tmem_cols, idesc, idesc_tail;
     long long split_stride;      // floats between partials
 };
+struct alignas(64) WgradParams {
+    CUtensorMap tm_a;            // dy {c_out, Q, P, N}, box {m_chunk, w, h, n}, no swizzle
+    CUtensorMap tm_b;            // x {C, Wv, Hv, N}, box {n_cols, w, h, n}, no swizzle
+    WgradScalars s;
+};
+
+template <class T>
+__device__ __forceinline__ void load_scalars(T* dst, const T* src)
+{
+    static_assert(sizeof(T) % 4 == 0, "scalar block must be a whole number of words");
+    const uint32_t* w = reinterpret_cast<const uint32_t*>(src);
+    for (int i = threadIdx.x; i < (int)(sizeof(T) / 4); i += blockDim.x) reinterpret_cast<uint32_t*>(dst)[i] = w[i];
+}
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
@@ -219,10 +270,13 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 
 // ------------------------------------------------------------------------------------------------
-// forward / data-gradient kernel: 6 warps = TMA producer, MMA issuer, 4 splitter / epilogue warps
+// forward / data-gradient kernel: 10 warps = TMA producer, MMA issuer, 8 splitter / epilogue warps
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(192) conv_tc_fwd_kernel(const __grid_constant__ FwdParams p)
+__global__ void __launch_bounds__(320) conv_tc_fwd_kernel(const __grid_constant__ FwdParams gp)
 {
+    __shared__ FwdScalars p;                 // scalar parameters, see load_scalars
+    load_scalars(&p, &gp.s);
+    __syncthreads();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[3 * 8 + 1];       // full[8], empty[8], split[8], accum
     __shared__ uint32_t tmem_slot;
@@ -247,18 +301,21 @@ __global__ void __launch_bounds__(192) conv_tc_fwd_kernel(const __grid_constant_
     const int q0 = tw * p.box_w, p0 = th * p.box_h, n0 = tn * p.box_n;
     const int co0 = blockIdx.y * p.n_chunk;
 
+    if (threadIdx.x == 0) HPF_TL(0);
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); mbar_init(split0 + 8 * s, 4); }
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); mbar_init(split0 + 8 * s, 8); }
         mbar_init(accum_bar, 1);
         abort_flag = 0; issued = 0; consumed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (threadIdx.x == 32) { prefetch_tmap(&gp.tm_a); prefetch_tmap(&gp.tm_b); if (p.passes == 3) prefetch_tmap(&gp.tm_b_lo); }
     if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), p.tmem_cols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
     const int total = p.R * p.R * p.n_kchunks;
+    if (threadIdx.x == 0) HPF_TL(1);
 
     if (warp == 0) {
         if (lane == 0) {
@@ -271,102 +328,198 @@ __global__ void __launch_bounds__(192) conv_tc_fwd_kernel(const __grid_constant_
                 const int r = tap / p.R, sx = tap % p.R;
                 const uint32_t dst = smem_base + s * p.stage_bytes;
                 mbar_expect_tx(full0 + 8 * s, p.tx_bytes);
-                tma_load_4d(dst, &p.tm_a, full0 + 8 * s, kc * p.kchunk, q0 + sx - p.pad, p0 + r - p.pad, n0);
-                tma_load_2d(dst + off_b, &p.tm_b, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
-                if (p.passes == 3) tma_load_2d(dst + off_blo, &p.tm_b_lo, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
+                tma_load_4d(dst, &gp.tm_a, full0 + 8 * s, kc * p.kchunk, q0 + sx - p.pad, p0 + r - p.pad, n0);
+                tma_load_2d(dst + off_b, &gp.tm_b, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
+                if (p.passes == 3) tma_load_2d(dst + off_blo, &gp.tm_b_lo, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
+                if (it == 0) HPF_TL(2);
             }
             issued = it;
         }
     } else if (warp == 1) {
         if (lane == 0) {
             // ---- MMA issuer ----
+            // One thread issues every MMA, so the loop is kept to a few instructions per MMA: the descriptor's
+            // constant part is built once and only its 14-bit address field is advanced (32 bytes = 2 units per K step).
             const uint32_t sbo = 8u * (uint32_t)p.kchunk * 4u;          // 8 rows of one swizzle atom
-            int it = 0;
+            const uint64_t desc_hi = smem_desc(0, 16, sbo, p.swizzle);
+            const uint32_t idesc = p.idesc, idesc2 = p.idesc2, stage_bytes = p.stage_bytes;
+            const bool stacked = p.stacked != 0;
+            const int stages = p.stages, k8n = p.kchunk / 8;
+            const bool three = p.passes == 3;
+            int it = 0, s = 0;
+            uint32_t par = 0;
             for (; it < total; ++it) {
-                const int s = it % p.stages;
-                const uint32_t par = (it / p.stages) & 1;
                 if (!mbar_wait(full0 + 8 * s, par, &abort_flag)) { report(p.status, 2); break; }
-                if (p.passes == 3 && !mbar_wait(split0 + 8 * s, par, &abort_flag)) { report(p.status, 6); break; }
+                if (three && !mbar_wait(split0 + 8 * s, par, &abort_flag)) { report(p.status, 6); break; }
                 tc_fence_after();
-                const uint32_t st = smem_base + s * p.stage_bytes;
-                for (int k8 = 0; k8 < p.kchunk / 8; ++k8) {
-                    const uint64_t ad = smem_desc(st + 32u * k8, 16, sbo, p.swizzle);
-                    const uint64_t bd = smem_desc(st + off_b + 32u * k8, 16, sbo, p.swizzle);
-                    umma_tf32(tmem_base, ad, bd, p.idesc, (it | k8) ? 1u : 0u);
-                    if (p.passes == 3) {
-                        const uint64_t adl = smem_desc(st + off_alo + 32u * k8, 16, sbo, p.swizzle);
-                        const uint64_t bdl = smem_desc(st + off_blo + 32u * k8, 16, sbo, p.swizzle);
-                        umma_tf32(tmem_base, adl, bd, p.idesc, 1u);
-                        umma_tf32(tmem_base, ad, bdl, p.idesc, 1u);
+                if (it == 0) HPF_TL(5);
+                const uint32_t st = smem_base + s * stage_bytes;
+                const uint64_t a0 = desc_hi | (uint64_t)((st & 0x3FFFFu) >> 4);
+                const uint64_t b0 = desc_hi | (uint64_t)(((st + off_b) & 0x3FFFFu) >> 4);
+                const uint64_t al0 = desc_hi | (uint64_t)(((st + off_alo) & 0x3FFFFu) >> 4);
+                const uint64_t bl0 = desc_hi | (uint64_t)(((st + off_blo) & 0x3FFFFu) >> 4);
+                if (three && stacked) {
+                    // B_lo follows B_hi in shared memory: A_hi x [B_hi; B_lo] in one MMA of twice the width
+                    // (columns [0,n) = hi*hi, [n,2n) = hi*lo, added in the epilogue), then A_lo x B_hi.
+#pragma unroll 4
+                    for (int k8 = 0; k8 < k8n; ++k8) {
+                        umma_tf32(tmem_base, a0 + 2 * k8, b0 + 2 * k8, idesc2, (it | k8) ? 1u : 0u);
+                        umma_tf32(tmem_base, al0 + 2 * k8, b0 + 2 * k8, idesc, 1u);
                     }
+                } else if (three) {
+#pragma unroll 4
+                    for (int k8 = 0; k8 < k8n; ++k8) {
+                        umma_tf32(tmem_base, a0 + 2 * k8, b0 + 2 * k8, idesc, (it | k8) ? 1u : 0u);
+                        umma_tf32(tmem_base, al0 + 2 * k8, b0 + 2 * k8, idesc, 1u);
+                        umma_tf32(tmem_base, a0 + 2 * k8, bl0 + 2 * k8, idesc, 1u);
+                    }
+                } else {
+#pragma unroll 4
+                    for (int k8 = 0; k8 < k8n; ++k8) umma_tf32(tmem_base, a0 + 2 * k8, b0 + 2 * k8, idesc, (it | k8) ? 1u : 0u);
                 }
                 umma_commit(empty0 + 8 * s);     // frees the stage once these MMAs have read it
+                if (++s == stages) { s = 0; par ^= 1u; }
             }
             consumed = it;
             if (it == total) umma_commit(accum_bar);
+            HPF_TL(6);
         }
     } else {
-        // ---- warps 2..5: split the activation tile into hi / lo, then the epilogue ----
-        const int tid = threadIdx.x - 64;
+        // ---- warps 2..9: split the activation tile into hi / lo, then the epilogue ----
+        const int tid = threadIdx.x - 64;               // 0..255
         bool ok = true;
         if (p.passes == 3) {
-            const int n4 = (int)(p.a_bytes >> 4);
+            const int per = (int)(p.a_bytes >> 12);     // float4 per thread: a_bytes / 16 / 256 = 2 or 4
             for (int it = 0; it < total; ++it) {
                 const int s = it % p.stages;
                 ok = mbar_wait(full0 + 8 * s, (it / p.stages) & 1, &abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) { if (lane == 0) report(p.status, 7); break; }
+                if (it == 0 && tid == 0) HPF_TL(3);
                 float4* a = reinterpret_cast<float4*>(smem + s * p.stage_bytes);
                 float4* alo = reinterpret_cast<float4*>(smem + s * p.stage_bytes + off_alo);
-                for (int i = tid; i < n4; i += 128) {
-                    const float4 v = a[i];
-                    const float4 h = make_float4(tf32_hi(v.x), tf32_hi(v.y), tf32_hi(v.z), tf32_hi(v.w));
-                    a[i] = h;
-                    alo[i] = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
-                }
+                float4 v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) if (j < per) v[j] = a[tid + 256 * j];
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (j < per) {
+                        const float4 h = make_float4(tf32_hi(v[j].x), tf32_hi(v[j].y), tf32_hi(v[j].z), tf32_hi(v[j].w));
+                        a[tid + 256 * j] = h;
+                        alo[tid + 256 * j] = make_float4(v[j].x - h.x, v[j].y - h.y, v[j].z - h.z, v[j].w - h.w);
+                    }
                 fence_async_smem();               // generic-proxy writes -> tensor-core reads
                 __syncwarp();
                 if (lane == 0) mbar_arrive(split0 + 8 * s);
+                if (it == 0 && tid == 0) HPF_TL(4);
             }
         }
-        bool done = ok && mbar_wait(accum_bar, 0, &abort_flag);
-        done = __all_sync(0xffffffffu, done);
-        if (done) {
-            tc_fence_after();
-            const int row = (warp & 3) * 32 + lane;          // TMEM lane = pixel within the tile
-            const int wi = row % p.box_w, hi = (row / p.box_w) % p.box_h, ni = row / (p.box_w * p.box_h);
+        (void)ok;
+        mbar_wait(accum_bar, 0, &abort_flag);
+        // every pipeline buffer is idle now (all MMAs completed, all copies landed): the tile is staged there
+        // so that the write-out is coalesced (a TMEM lane is a pixel: thread-per-row stores would touch 32 lines each)
+        __shared__ long long row_off[kTileM];
+        __shared__ int row_fill[kTileM];               // strided data gradient: which neighbours of the sample exist
+        if (tid < kTileM) {
+            const int wi = tid % p.box_w, hi = (tid / p.box_w) % p.box_h, ni = tid / (p.box_w * p.box_h);
             const int q = q0 + wi, pp = p0 + hi, n = n0 + ni;
             const bool valid = ni < p.box_n && q < p.Q && pp < p.P && n < p.N;
-            float* orow = p.out + n * p.os_n + pp * p.os_h + q * p.os_w + co0;
-            const float* erow = p.extra ? p.extra + (n * p.os_n + pp * p.os_h + q * p.os_w + co0) : nullptr;
+            row_off[tid] = valid ? (n * p.os_n + pp * p.os_h + q * p.os_w + co0) : -1;
+            int fill = 0;                              // bit (dy*4 + dx) set: position (pp*s+dy, q*s+dx) gets zeros
+            for (int dy = 0; dy < p.zero_fill; ++dy)
+                for (int dx = 0; dx < p.zero_fill; ++dx)
+                    if ((dy | dx) && pp * p.zero_fill + dy < p.out_h && q * p.zero_fill + dx < p.out_w) fill |= 1 << (dy * 4 + dx);
+            row_fill[tid] = (valid && p.zero_fill > 1 && p.zero_fill <= 4) ? fill : 0;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        const bool done = abort_flag == 0;             // uniform over the 8 warps after the barrier
+        if (done) {
+            tc_fence_after();
+            if (tid == 0) HPF_TL(7);
+            // TMEM lane = pixel within the tile.  Two warps share each group of 32 lanes (a warp reaches lanes
+            // 32*(warp%4) ..): they take alternate groups of 32 output channels.
+            const int row = (warp & 3) * 32 + lane;
+            const int half = (warp - 2) >> 2;
+            float* stg = reinterpret_cast<float*>(smem);
             const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-            for (int c0 = 0; c0 < p.n_chunk; c0 += 16) {
-                float v[16];
-                tmem_ld16(lane_addr + (uint32_t)c0, v);
-                if (valid) {
+            for (int g0 = half * 32; g0 < p.n_chunk; g0 += 64) {
+                const int ncols = p.n_chunk - g0 < 32 ? p.n_chunk - g0 : 32;      // 16 or 32
+                float v[32];
+                tmem_ld16_nowait(lane_addr + (uint32_t)g0, v);
+                if (ncols > 16) tmem_ld16_nowait(lane_addr + (uint32_t)(g0 + 16), v + 16);
+                tmem_ld_wait();
+                if (p.stacked) {
+                    float u[32];
+                    tmem_ld16_nowait(lane_addr + (uint32_t)(p.n_chunk + g0), u);
+                    if (ncols > 16) tmem_ld16_nowait(lane_addr + (uint32_t)(p.n_chunk + g0 + 16), u + 16);
+                    tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 16; j += 4) {
-                        float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                        if (erow) { const float4 e = __ldg(reinterpret_cast<const float4*>(erow + c0 + j)); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
-                        if (p.accumulate) { const float4 e = *reinterpret_cast<const float4*>(orow + c0 + j); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
-                        *reinterpret_cast<float4*>(orow + c0 + j) = o;
+                    for (int j = 0; j < 32; ++j) if (j < ncols) v[j] += u[j];
+                }
+                float4* dst = reinterpret_cast<float4*>(stg + (size_t)row * p.stg_pitch + g0);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) if (4 * j < ncols) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            }
+            if (tid == 0) HPF_TL(10);
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (tid == 0) HPF_TL(11);
+            // write-out: consecutive threads write consecutive float4 of a pixel's channel row.  Eight warps cannot
+            // hide latency by occupancy, so four independent float4 are in flight per thread and nothing is re-read.
+            const int c4n = p.n_chunk >> 2;
+            const int total4 = kTileM * c4n;
+            const int sh = (c4n & (c4n - 1)) == 0 ? 31 - __clz(c4n) : -1;
+            const float* extra = p.extra;
+            float* outp = p.out;
+            const bool accumulate = p.accumulate != 0;
+            const unsigned int pitch = p.stg_pitch;
+            const long long dense_h = p.dense_h, dense_w = p.dense_w;
+            for (int base = tid; base < total4; base += 1024) {
+                float4 o[4];
+                long long off[4];
+                int fill[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int idx = base + 256 * u;
+                    off[u] = -1; fill[u] = 0;
+                    if (idx < total4) {
+                        const int r = sh >= 0 ? (idx >> sh) : (idx / c4n);
+                        const int c4 = idx - r * c4n;
+                        const long long ro = row_off[r];
+                        if (ro >= 0) {
+                            off[u] = ro + 4 * c4;
+                            fill[u] = row_fill[r];
+                            o[u] = *reinterpret_cast<const float4*>(stg + (size_t)r * pitch + 4 * c4);
+                        }
                     }
                 }
-            }
-            if (p.zero_fill > 1 && valid) {
-                // strided data gradient: the positions between the samples receive no contribution
-                const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int dy = 0; dy < p.zero_fill; ++dy)
-                    for (int dx = 0; dx < p.zero_fill; ++dx) {
-                        if ((dy | dx) == 0) continue;
-                        if (pp * p.zero_fill + dy >= p.out_h || q * p.zero_fill + dx >= p.out_w) continue;
-                        float* zr = orow + dy * p.dense_h + dx * p.dense_w;
-                        for (int c0 = 0; c0 < p.n_chunk; c0 += 4) *reinterpret_cast<float4*>(zr + c0) = z;
+                if (extra) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (off[u] >= 0) { const float4 e = __ldg(reinterpret_cast<const float4*>(extra + off[u])); o[u].x += e.x; o[u].y += e.y; o[u].z += e.z; o[u].w += e.w; }
+                }
+                if (accumulate) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (off[u] >= 0) { const float4 e = *reinterpret_cast<const float4*>(outp + off[u]); o[u].x += e.x; o[u].y += e.y; o[u].z += e.z; o[u].w += e.w; }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (off[u] < 0) continue;
+                    float* optr = outp + off[u];
+                    *reinterpret_cast<float4*>(optr) = o[u];
+                    if (fill[u]) {
+                        // strided data gradient: the positions between the samples receive no contribution
+                        const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int dy = 0; dy < 4; ++dy)
+                            for (int dx = 0; dx < 4; ++dx)
+                                if (fill[u] & (1 << (dy * 4 + dx))) *reinterpret_cast<float4*>(optr + dy * dense_h + dx * dense_w) = z;
                     }
+                }
             }
         }
     }
 
+    if (threadIdx.x == 64) HPF_TL(8);
     // ---- teardown ----
     tc_fence_before();
     __syncthreads();
@@ -380,6 +533,7 @@ __global__ void __launch_bounds__(192) conv_tc_fwd_kernel(const __grid_constant_
     }
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
+    if (threadIdx.x == 0) HPF_TL(9);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -413,8 +567,11 @@ __device__ __forceinline__ void transpose_tile(const uint8_t* raw, uint8_t* dst,
     }
 }
 
-__global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constant__ WgradParams p)
+__global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constant__ WgradParams gp)
 {
+    __shared__ WgradScalars p;                 // scalar parameters, see load_scalars
+    load_scalars(&p, &gp.s);
+    __syncthreads();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[4 * 4 + 1];       // full_raw[4], empty_raw[4], full_t[4], empty_t[4], accum
     __shared__ uint32_t tmem_slot;
@@ -481,10 +638,10 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
                 const uint32_t dst = smem_base + s * p.raw_bytes;
                 const uint32_t bar = full_raw0 + 8 * s;
                 mbar_expect_tx(bar, p.tx_a + (uint32_t)ntaps * p.tx_per_tap);
-                tma_load_4d(dst, &p.tm_a, bar, m0, q0, p0, n0);
+                tma_load_4d(dst, &gp.tm_a, bar, m0, q0, p0, n0);
                 for (int tp = 0; tp < ntaps; ++tp) {
                     const int r = (tap0 + tp) / p.R, sx = (tap0 + tp) % p.R;
-                    tma_load_4d(dst + raw_a + tp * raw_b, &p.tm_b, bar, cn0, q0 + sx - p.pad, p0 + r - p.pad, n0);
+                    tma_load_4d(dst + raw_a + tp * raw_b, &gp.tm_b, bar, cn0, q0 + sx - p.pad, p0 + r - p.pad, n0);
                 }
             }
             issued = it;
@@ -878,14 +1035,15 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
         WgradGeom g;
         if (!wgrad_geom(s, passes, &g)) return cudaErrorNotSupported;
         ConvTcWgradLaunch* L = reinterpret_cast<ConvTcWgradLaunch*>(plan->storage);
-        WgradParams& p = L->p;
-        memset(&p, 0, sizeof p);
+        WgradParams& P = L->p;
+        memset(&P, 0, sizeof P);
+        WgradScalars& p = P.s;
         // dy {K, Q, P, N}
         {
             cuuint64_t dims[4] = {(cuuint64_t)s.K, (cuuint64_t)s.Q, (cuuint64_t)s.P, (cuuint64_t)s.N};
             cuuint64_t str[3] = {(cuuint64_t)s.K * 4, (cuuint64_t)s.Q * s.K * 4, (cuuint64_t)s.P * s.Q * s.K * 4};
             cuuint32_t box[4] = {(cuuint32_t)g.m_chunk, (cuuint32_t)g.box.w, (cuuint32_t)g.box.h, (cuuint32_t)g.box.n};
-            cudaError_t e = encode(&p.tm_a, in, 4, dims, str, box, 0);
+            cudaError_t e = encode(&P.tm_a, in, 4, dims, str, box, 0);
             if (e != cudaSuccess) return e;
         }
         // x {C, Wv, Hv, N}: a strided 1x1 convolution samples every stride-th pixel
@@ -894,7 +1052,7 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
             cuuint64_t dims[4] = {(cuuint64_t)s.C, (cuuint64_t)wv, (cuuint64_t)hv, (cuuint64_t)s.N};
             cuuint64_t str[3] = {(cuuint64_t)s.stride * s.C * 4, (cuuint64_t)s.stride * s.W * s.C * 4, (cuuint64_t)s.H * s.W * s.C * 4};
             cuuint32_t box[4] = {(cuuint32_t)g.n_cols, (cuuint32_t)g.box.w, (cuuint32_t)g.box.h, (cuuint32_t)g.box.n};
-            cudaError_t e = encode(&p.tm_b, in2, 4, dims, str, box, 0);
+            cudaError_t e = encode(&P.tm_b, in2, 4, dims, str, box, 0);
             if (e != cudaSuccess) return e;
         }
         const long long n_out = (long long)s.K * s.R * s.R * s.C;
@@ -922,15 +1080,16 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     PixelBox b;
     if (!fwd_view(s, pass, &v) || !choose_box(v.Q, v.P, v.N, kTileM, 1, &b)) return cudaErrorNotSupported;
     ConvTcFwdLaunch* L = reinterpret_cast<ConvTcFwdLaunch*>(plan->storage);
-    FwdParams& p = L->p;
-    memset(&p, 0, sizeof p);
+    FwdParams& P = L->p;
+    memset(&P, 0, sizeof P);
+    FwdScalars& p = P.s;
     const int kchunk = chunk_of(v.c_in);
     const int n_chunk = v.c_out < 256 ? v.c_out : 256;
     {
         cuuint64_t dims[4] = {(cuuint64_t)v.c_in, (cuuint64_t)v.in_w, (cuuint64_t)v.in_h, (cuuint64_t)v.N};
         cuuint64_t str[3] = {(cuuint64_t)v.in_sw * 4, (cuuint64_t)v.in_sh * 4, (cuuint64_t)v.in_sn * 4};
         cuuint32_t box[4] = {(cuuint32_t)kchunk, (cuuint32_t)b.w, (cuuint32_t)b.h, (cuuint32_t)b.n};
-        cudaError_t e = encode(&p.tm_a, in, 4, dims, str, box, kchunk * 4);
+        cudaError_t e = encode(&P.tm_a, in, 4, dims, str, box, kchunk * 4);
         if (e != cudaSuccess) return e;
     }
     {
@@ -938,10 +1097,10 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
         cuuint64_t dims[2] = {(cuuint64_t)kdim, (cuuint64_t)v.c_out};
         cuuint64_t str[1] = {(cuuint64_t)kdim * 4};
         cuuint32_t box[2] = {(cuuint32_t)kchunk, (cuuint32_t)n_chunk};
-        cudaError_t e = encode(&p.tm_b, w_hi, 2, dims, str, box, kchunk * 4);
+        cudaError_t e = encode(&P.tm_b, w_hi, 2, dims, str, box, kchunk * 4);
         if (e != cudaSuccess) return e;
         if (passes == 3) {
-            e = encode(&p.tm_b_lo, w_lo, 2, dims, str, box, kchunk * 4);
+            e = encode(&P.tm_b_lo, w_lo, 2, dims, str, box, kchunk * 4);
             if (e != cudaSuccess) return e;
         }
     }
@@ -964,10 +1123,15 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     if (stages > kFwdMaxStages) stages = kFwdMaxStages;
     if (stages > total) stages = total;
     p.stages = stages;
-    p.tmem_cols = pow2_cols(n_chunk);
+    p.stacked = (passes == 3 && 2 * n_chunk <= 256) ? 1 : 0;
+    p.tmem_cols = pow2_cols(p.stacked ? 2 * n_chunk : n_chunk);
     p.idesc = instr_desc(n_chunk, false, false);
+    p.idesc2 = instr_desc(p.stacked ? 2 * n_chunk : n_chunk, false, false);
+    p.stg_pitch = (unsigned int)n_chunk + 4u;
     L->grid = dim3(p.tiles_w * p.tiles_h * tiles_n, v.c_out / n_chunk, 1);
-    L->smem = (unsigned int)stages * p.stage_bytes + 1024;
+    L->smem = (unsigned int)stages * p.stage_bytes;
+    if (L->smem < (unsigned int)kTileM * p.stg_pitch * 4u) L->smem = (unsigned int)kTileM * p.stg_pitch * 4u;   // epilogue staging
+    L->smem += 1024;
     plan->valid = 1;
     return cudaSuccess;
 }
@@ -977,19 +1141,19 @@ cudaError_t conv_tc_launch(const ConvTcPlan* plan, DeviceStatus* status, cudaStr
     if (!plan->valid) return cudaErrorInvalidValue;
     if (plan->pass == PASS_WGRAD) {
         ConvTcWgradLaunch L = *reinterpret_cast<const ConvTcWgradLaunch*>(plan->storage);
-        L.p.status = status;
+        L.p.s.status = status;
         conv_tc_wgrad_kernel<<<L.grid, 192, L.smem, st>>>(L.p);
         count(n_launch, 1);
         if (L.splits > 1) {
             const int nb = (int)((L.n_out / 4 + 31) / 32);
-            wgrad_partials_reduce_kernel<<<nb, 256, 0, st>>>(L.p.out, L.dw, L.n_out, L.splits);
+            wgrad_partials_reduce_kernel<<<nb, 256, 0, st>>>(L.p.s.out, L.dw, L.n_out, L.splits);
             count(n_launch, 1);
         }
         return cudaGetLastError();
     }
     ConvTcFwdLaunch L = *reinterpret_cast<const ConvTcFwdLaunch*>(plan->storage);
-    L.p.status = status;
-    conv_tc_fwd_kernel<<<L.grid, 192, L.smem, st>>>(L.p);
+    L.p.s.status = status;
+    conv_tc_fwd_kernel<<<L.grid, 320, L.smem, st>>>(L.p);
     count(n_launch, 1);
     return cudaGetLastError();
 }
