@@ -275,6 +275,7 @@ __device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__flo
 __global__ void __launch_bounds__(320) conv_tc_fwd_kernel(const __grid_constant__ FwdParams gp)
 {
     __shared__ FwdScalars p;                 // scalar parameters, see load_scalars
+    pdl_launch_dependents();
     load_scalars(&p, &gp.s);
     __syncthreads();
     extern __shared__ uint8_t smem_raw[];
@@ -313,6 +314,7 @@ __global__ void __launch_bounds__(320) conv_tc_fwd_kernel(const __grid_constant_
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_wait();              // everything above touched only parameters, shared and tensor memory
     const uint32_t tmem_base = tmem_slot;
     const int total = p.R * p.R * p.n_kchunks;
     if (threadIdx.x == 0) HPF_TL(1);
@@ -570,6 +572,7 @@ __device__ __forceinline__ void transpose_tile(const uint8_t* raw, uint8_t* dst,
 __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constant__ WgradParams gp)
 {
     __shared__ WgradScalars p;                 // scalar parameters, see load_scalars
+    pdl_launch_dependents();
     load_scalars(&p, &gp.s);
     __syncthreads();
     extern __shared__ uint8_t smem_raw[];
@@ -621,6 +624,7 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_wait();              // everything above touched only parameters, shared and tensor memory
     const uint32_t tmem_base = tmem_slot;
 
     if (warp == 0) {
@@ -754,6 +758,8 @@ __global__ void __launch_bounds__(256)
 wgrad_partials_reduce_kernel(const float* __restrict__ partials, float* __restrict__ dw, long long n, int splits)
 {
     __shared__ float4 sh[8][32];
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31, zl = threadIdx.x >> 5;
     const long long n4 = n / 4;          // n is a multiple of 4 and the partials are 16-byte aligned; dw may not be
     const long long i = (long long)blockIdx.x * 32 + lane;
@@ -1142,18 +1148,18 @@ cudaError_t conv_tc_launch(const ConvTcPlan* plan, DeviceStatus* status, cudaStr
     if (plan->pass == PASS_WGRAD) {
         ConvTcWgradLaunch L = *reinterpret_cast<const ConvTcWgradLaunch*>(plan->storage);
         L.p.s.status = status;
-        conv_tc_wgrad_kernel<<<L.grid, 192, L.smem, st>>>(L.p);
+        launch_pdl(conv_tc_wgrad_kernel, L.grid, dim3(192), L.smem, st, L.p);
         count(n_launch, 1);
         if (L.splits > 1) {
             const int nb = (int)((L.n_out / 4 + 31) / 32);
-            wgrad_partials_reduce_kernel<<<nb, 256, 0, st>>>(L.p.s.out, L.dw, L.n_out, L.splits);
+            launch_pdl(wgrad_partials_reduce_kernel, dim3(nb), dim3(256), 0, st, (const float*)L.p.s.out, L.dw, L.n_out, L.splits);
             count(n_launch, 1);
         }
         return cudaGetLastError();
     }
     ConvTcFwdLaunch L = *reinterpret_cast<const ConvTcFwdLaunch*>(plan->storage);
     L.p.s.status = status;
-    conv_tc_fwd_kernel<<<L.grid, 320, L.smem, st>>>(L.p);
+    launch_pdl(conv_tc_fwd_kernel, L.grid, dim3(320), L.smem, st, L.p);
     count(n_launch, 1);
     return cudaGetLastError();
 }

@@ -19,6 +19,29 @@ inline ConvShape make_conv_shape(int N, int H, int W, int C, int K, int R, int s
     return s;
 }
 
+// Programmatic dependent launch.  The step is a long chain of small dependent kernels, so the gap between the end
+// of one and the start of the next is a sizeable part of the critical path.  Hot kernels are launched with the
+// programmatic-serialisation attribute: such a kernel may be scheduled while its predecessor in the stream is
+// still running, executes its prologue (barrier and tensor-memory set-up, parameter and descriptor fetches), and
+// blocks in pdl_wait() until the predecessor has completed and its writes are visible.  Every kernel launched
+// this way calls pdl_wait() before its first read or write of global data.
+extern bool g_pdl_enabled;
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = g_pdl_enabled ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
 // Device-side status word shared by all kernels that have bounded waits.
 // 0 = fine; anything else = where a wait gave up (see conv_tc.cu).
 struct DeviceStatus { unsigned int code; unsigned int detail; };

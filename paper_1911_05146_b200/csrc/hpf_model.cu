@@ -717,6 +717,7 @@ int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
     case HPF_OPT_SINGLE_STREAM: mdl->opt_single = value != 0; break;
     case HPF_OPT_KEEP_MESSAGES: mdl->opt_messages = value != 0; break;
     case HPF_OPT_FUSE_ADD: mdl->opt_fuse_add = value != 0; break;
+    case HPF_OPT_PDL: hpf::g_pdl_enabled = value != 0; break;
     default: return fail(HPF_ERR_INVALID, "unknown option");
     }
     mdl->planned = false;

@@ -9,6 +9,8 @@
 
 namespace hpf {
 
+bool g_pdl_enabled = true;
+
 namespace {
 
 constexpr int kThreads = 256;
@@ -78,6 +80,8 @@ bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, cons
 {
     __shared__ double shd[kBnThreads][8];            // 32 KB; the float phase uses it as float[kBnThreads][8]
     float (*sh)[8] = reinterpret_cast<float (*)[8]>(&shd[0][0]);
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ int is_last;
     const int t = threadIdx.x;
     const int cg_total = C / 4;
@@ -209,6 +213,8 @@ bn_apply_fwd_kernel(const float4* __restrict__ x, const float* __restrict__ gamm
                     const float* __restrict__ stats, float4* __restrict__ y, int64_t rows, int C, int cgt, int rl,
                     int passes, int64_t rows_per_blk)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int t = threadIdx.x, cg_total = C / 4;
     const int my_rl = t / cgt, my_cg = t % cgt;
     const int64_t r0 = (int64_t)blockIdx.x * rows_per_blk;
@@ -251,6 +257,8 @@ bn_apply_bwd_kernel(const float4* __restrict__ x, const float4* __restrict__ dy,
                     const float4* __restrict__ addend, float4* __restrict__ dx, int64_t rows, int C, int cgt, int rl,
                     int passes, int64_t rows_per_blk)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int t = threadIdx.x, cg_total = C / 4;
     const int my_rl = t / cgt, my_cg = t % cgt;
     const int64_t r0 = (int64_t)blockIdx.x * rows_per_blk;
@@ -299,6 +307,8 @@ int ew_blocks(int64_t n_items)
 __global__ void __launch_bounds__(kThreads)
 add_kernel(const float* __restrict__ a, const float* __restrict__ b, float* __restrict__ out, int64_t n)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int64_t n4 = n / 4;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -313,6 +323,8 @@ template <bool ACCUM>
 __global__ void __launch_bounds__(kThreads)
 accumulate_kernel(float* __restrict__ dst, const float* __restrict__ src, int64_t n)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int64_t n4 = n / 4;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -575,10 +587,10 @@ cudaError_t bnrelu_fwd(const float* x, const float* gamma, const float* beta, fl
     const BnPlan p = bn_plan(rows, C);
     unsigned int* ticket = reinterpret_cast<unsigned int*>(scratch);
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + 256);
-    bn_reduce_kernel<false><<<p.nblk, kBnThreads, 0, st>>>(x, nullptr, gamma, beta, nullptr, eps, rows, C, p.cgt, p.rl,
+    launch_pdl(bn_reduce_kernel<false>, p.nblk, kBnThreads, 0, st, x, (const float*)nullptr, gamma, beta, (const float*)nullptr, eps, rows, C, p.cgt, p.rl,
                                                            p.passes, p.rows_per_blk, ticket, partials, stats, stats + C,
-                                                           nullptr);
-    bn_apply_fwd_kernel<<<p.nblk_apply, kBnThreads, 0, st>>>(reinterpret_cast<const float4*>(x), gamma, beta, stats,
+                                                           (float*)nullptr);
+    launch_pdl(bn_apply_fwd_kernel, p.nblk_apply, kBnThreads, 0, st, reinterpret_cast<const float4*>(x), gamma, beta, stats,
                                                              reinterpret_cast<float4*>(y), rows, C, p.cgt, p.rl, p.passes,
                                                              p.rows_per_blk_apply);
     count(n_launch, 2);
@@ -593,14 +605,14 @@ cudaError_t bnrelu_bwd(const float* x, const float* dy, const float* gamma, cons
     unsigned int* ticket = reinterpret_cast<unsigned int*>(scratch);
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + 256);
     float* coef = partials + (size_t)p.nblk * 2 * C;
-    bn_reduce_kernel<true><<<p.nblk, kBnThreads, 0, st>>>(x, dy, gamma, beta, stats, 0.f, rows, C, p.cgt, p.rl, p.passes,
+    launch_pdl(bn_reduce_kernel<true>, p.nblk, kBnThreads, 0, st, x, dy, gamma, beta, stats, 0.f, rows, C, p.cgt, p.rl, p.passes,
                                                           p.rows_per_blk, ticket, partials, dbeta, dgamma, coef);
     const float4* x4 = reinterpret_cast<const float4*>(x);
     const float4* dy4 = reinterpret_cast<const float4*>(dy);
     const float4* ad4 = reinterpret_cast<const float4*>(addend);
     float4* dx4 = reinterpret_cast<float4*>(dx);
     const int nb = p.nblk_apply;
-#define HPF_BN_APPLY(A, B) bn_apply_bwd_kernel<A, B><<<nb, kBnThreads, 0, st>>>(x4, dy4, gamma, beta, stats, coef, ad4, dx4, rows, C, p.cgt, p.rl, p.passes, p.rows_per_blk_apply)
+#define HPF_BN_APPLY(A, B) launch_pdl(bn_apply_bwd_kernel<A, B>, nb, kBnThreads, 0, st, x4, dy4, gamma, beta, stats, coef, ad4, dx4, rows, C, p.cgt, p.rl, p.passes, p.rows_per_blk_apply)
     if (addend && accumulate) HPF_BN_APPLY(true, true);
     else if (addend) HPF_BN_APPLY(true, false);
     else if (accumulate) HPF_BN_APPLY(false, true);
@@ -612,15 +624,15 @@ cudaError_t bnrelu_bwd(const float* x, const float* dy, const float* gamma, cons
 
 cudaError_t add_fwd(const float* a, const float* b, float* out, int64_t n, cudaStream_t st, int64_t* n_launch)
 {
-    add_kernel<<<ew_blocks(n / 4 + 1), kThreads, 0, st>>>(a, b, out, n);
+    launch_pdl(add_kernel, ew_blocks(n / 4 + 1), kThreads, 0, st, a, b, out, n);
     count(n_launch, 1);
     return cudaGetLastError();
 }
 
 cudaError_t grad_accumulate(float* dst, const float* src, int64_t n, bool accumulate, cudaStream_t st, int64_t* n_launch)
 {
-    if (accumulate) accumulate_kernel<true><<<ew_blocks(n / 4 + 1), kThreads, 0, st>>>(dst, src, n);
-    else accumulate_kernel<false><<<ew_blocks(n / 4 + 1), kThreads, 0, st>>>(dst, src, n);
+    if (accumulate) launch_pdl(accumulate_kernel<true>, ew_blocks(n / 4 + 1), kThreads, 0, st, dst, src, n);
+    else launch_pdl(accumulate_kernel<false>, ew_blocks(n / 4 + 1), kThreads, 0, st, dst, src, n);
     count(n_launch, 1);
     return cudaGetLastError();
 }
