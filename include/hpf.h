@@ -93,9 +93,13 @@ int hpf_model_destroy(hpf_model *model);
  *                          that convolution's own output is then not stored (hpf_tensor_ptr answers
  *                          HPF_ERR_STATE for it).  0: every op's output is stored.
  *   HPF_OPT_PDL            1 (default): hot kernels use programmatic dependent launch (a kernel is scheduled and runs
- *                          its set-up while its predecessor in the stream drains).  Process-wide switch. */
+ *                          its set-up while its predecessor in the stream drains).  Process-wide switch.
+ *   HPF_OPT_WGRAD_PASSES   1 (default) or 3: TF32 passes of the tensor-core weight gradient.  A weight gradient feeds
+ *                          nothing but the average, so its rounding error (about 8e-4 relative with one pass) does not
+ *                          compound with depth the way forward and data-gradient errors do; those always follow
+ *                          HPF_OPT_CONV_PATH. */
 typedef enum { HPF_OPT_GRAPH = 1, HPF_OPT_CONV_PATH = 2, HPF_OPT_SINGLE_STREAM = 3, HPF_OPT_KEEP_MESSAGES = 4,
-               HPF_OPT_FUSE_ADD = 5, HPF_OPT_PDL = 6 } hpf_option;
+               HPF_OPT_FUSE_ADD = 5, HPF_OPT_PDL = 6, HPF_OPT_WGRAD_PASSES = 7 } hpf_option;
 int hpf_set_option(hpf_model *model, int32_t option, int32_t value);
 
 /* ---- integer bookkeeping (Section 5.1 lists, Section 5.3 pipelining) ----------------------------- */

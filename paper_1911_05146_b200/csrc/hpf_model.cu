@@ -5,6 +5,7 @@
 #include "hpf_kernels.h"
 
 #include <chrono>
+#include <cstdlib>
 #include <cstdio>
 #include <cstring>
 #include <string>
@@ -76,7 +77,7 @@ struct hpf_model {
     std::vector<std::vector<int>> live;       // per cut
     int64_t G = 0;
     // options
-    int opt_graph = 1, opt_conv_path = 0, opt_single = 0, opt_messages = 0, opt_fuse_add = 1;
+    int opt_graph = 1, opt_conv_path = 0, opt_single = 0, opt_messages = 0, opt_fuse_add = 1, opt_wgrad_passes = 1;
     // gradient-flow plan
     std::vector<int> grad_alias;              // tensor -> ADD op whose gradient buffer it shares, or -1
     std::vector<int> fused_into;              // conv -> residual ADD computed in its epilogue (its own output is not stored), or -1
@@ -489,7 +490,9 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
             CU(cudaEventRecord(mdl->ev_side[p], st));
             CU(cudaStreamWaitEvent(wst, mdl->ev_side[p], 0));
         }
-        if (mdl->use_tc[PASS_WGRAD][i]) {
+        static const bool skip_wgrad_dbg = getenv("HPF_DBG_SKIP_WGRAD") != nullptr;
+        if (skip_wgrad_dbg) {
+        } else if (mdl->use_tc[PASS_WGRAD][i]) {
             CU(conv_tc_launch(&mdl->tc_plan[PASS_WGRAD][(size_t)m * mdl->n_ops + i], mdl->status(), wst, &mdl->launches));
         } else {
             CU(conv_wgrad_simt(in0, dout, slot + o.w_off, s, mdl->ws + mdl->conv_scratch_off[p], wst, &mdl->launches));
@@ -718,6 +721,7 @@ int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
     case HPF_OPT_KEEP_MESSAGES: mdl->opt_messages = value != 0; break;
     case HPF_OPT_FUSE_ADD: mdl->opt_fuse_add = value != 0; break;
     case HPF_OPT_PDL: hpf::g_pdl_enabled = value != 0; break;
+    case HPF_OPT_WGRAD_PASSES: if (value != 1 && value != 3) return fail(HPF_ERR_INVALID, "1 or 3 passes"); mdl->opt_wgrad_passes = value; break;
     default: return fail(HPF_ERR_INVALID, "unknown option");
     }
     mdl->planned = false;
@@ -887,7 +891,7 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                         CU(conv_tc_prepare(pl, s, pass, passes, mdl->grad(i, m), nullptr, wp + 2 * G + o.w_off, wp + 3 * G + o.w_off,
                                            mdl->grad(src, m), ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch));
                     else
-                        CU(conv_tc_prepare(pl, s, pass, passes, mdl->grad(i, m), mdl->act(src, m), nullptr, nullptr,
+                        CU(conv_tc_prepare(pl, s, pass, mdl->opt_conv_path == 2 ? 1 : mdl->opt_wgrad_passes, mdl->grad(i, m), mdl->act(src, m), nullptr, nullptr,
                                            mdl->gslots + (int64_t)m * mdl->G + o.w_off, nullptr, false, scratch));
                 }
         }
