@@ -97,9 +97,14 @@ int hpf_model_destroy(hpf_model *model);
  *   HPF_OPT_WGRAD_PASSES   1 (default) or 3: TF32 passes of the tensor-core weight gradient.  A weight gradient feeds
  *                          nothing but the average, so its rounding error (about 8e-4 relative with one pass) does not
  *                          compound with depth the way forward and data-gradient errors do; those always follow
- *                          HPF_OPT_CONV_PATH. */
+ *                          HPF_OPT_CONV_PATH.
+ *   HPF_OPT_FUSE_BN        bit 0 (default on): the per-channel sums of a BN's forward statistics are formed in the write-out
+ *                          of the tensor-core convolution kernel that produces the BN's input, when both run back to
+ *                          back on one stream; the BN forward is then one kernel.  bit 1 (default off: measured slower):
+ *                          the same for the backward sums (dbeta, dgamma) in the data-gradient kernel that produces
+ *                          the gradient of the BN's output.  0: every BN runs its own reduction kernels. */
 typedef enum { HPF_OPT_GRAPH = 1, HPF_OPT_CONV_PATH = 2, HPF_OPT_SINGLE_STREAM = 3, HPF_OPT_KEEP_MESSAGES = 4,
-               HPF_OPT_FUSE_ADD = 5, HPF_OPT_PDL = 6, HPF_OPT_WGRAD_PASSES = 7 } hpf_option;
+               HPF_OPT_FUSE_ADD = 5, HPF_OPT_PDL = 6, HPF_OPT_WGRAD_PASSES = 7, HPF_OPT_FUSE_BN = 8 } hpf_option;
 int hpf_set_option(hpf_model *model, int32_t option, int32_t value);
 
 /* ---- integer bookkeeping (Section 5.1 lists, Section 5.3 pipelining) ----------------------------- */

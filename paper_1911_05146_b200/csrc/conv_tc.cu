@@ -223,6 +223,14 @@ struct FwdScalars {
     int zero_fill;               // > 1: the output pixel grid is strided, fill the rest of each patch with zeros
     int out_h, out_w;            // dense output extent (zero fill bounds)
     unsigned int a_bytes, b_bytes, stage_bytes, tx_bytes, tmem_cols, idesc, idesc2, stg_pitch;
+    // batch-norm reductions folded into the write-out (see ConvBnFuse): 0 none, 1 sums of the output,
+    // 2 sums of the masked gradient for the backward of the BN whose output this data gradient is
+    int stat_mode;
+    float* stat_partials;        // [tiles][2][c_out] per-tile partial sums
+    const float* bn_x;           // mode 2: the BN's input, same shape as the output
+    const float* bn_stats;       // mode 2: mean[c_out], rstd[c_out]
+    const float* bn_gamma;
+    const float* bn_beta;
 };
 struct alignas(64) FwdParams {
     CUtensorMap tm_a;            // activations {C, Wv, Hv, N}
@@ -475,6 +483,16 @@ __global__ void __launch_bounds__(320) conv_tc_fwd_kernel(const __grid_constant_
             const bool accumulate = p.accumulate != 0;
             const unsigned int pitch = p.stg_pitch;
             const long long dense_h = p.dense_h, dense_w = p.dense_w;
+            const int stat_mode = p.stat_mode;
+            float4 sa = make_float4(0.f, 0.f, 0.f, 0.f), sb = sa;
+            float4 bmu = sa, brs = sa, bg = sa, bb = sa;
+            if (stat_mode == 2) {
+                const int cch = co0 + 4 * (tid % c4n);             // this thread's channels (fixed: 256 % c4n == 0)
+                bmu = __ldg(reinterpret_cast<const float4*>(p.bn_stats + cch));
+                brs = __ldg(reinterpret_cast<const float4*>(p.bn_stats + p.c_out + cch));
+                bg = __ldg(reinterpret_cast<const float4*>(p.bn_gamma + cch));
+                bb = __ldg(reinterpret_cast<const float4*>(p.bn_beta + cch));
+            }
             for (int base = tid; base < total4; base += 1024) {
                 float4 o[4];
                 long long off[4];
@@ -509,6 +527,19 @@ __global__ void __launch_bounds__(320) conv_tc_fwd_kernel(const __grid_constant_
                     if (off[u] < 0) continue;
                     float* optr = outp + off[u];
                     *reinterpret_cast<float4*>(optr) = o[u];
+                    if (stat_mode == 1) {
+                        sa.x += o[u].x; sa.y += o[u].y; sa.z += o[u].z; sa.w += o[u].w;
+                        sb.x = fmaf(o[u].x, o[u].x, sb.x); sb.y = fmaf(o[u].y, o[u].y, sb.y);
+                        sb.z = fmaf(o[u].z, o[u].z, sb.z); sb.w = fmaf(o[u].w, o[u].w, sb.w);
+                    } else if (stat_mode == 2) {
+                        // dz = dy * [z > 0] with z recomputed exactly as the BN forward computed it
+                        const float4 xv = __ldg(reinterpret_cast<const float4*>(p.bn_x + off[u]));
+                        float xh, dz;
+                        xh = (xv.x - bmu.x) * brs.x; dz = fmaf(bg.x, xh, bb.x) > 0.f ? o[u].x : 0.f; sa.x += dz; sb.x = fmaf(dz, xh, sb.x);
+                        xh = (xv.y - bmu.y) * brs.y; dz = fmaf(bg.y, xh, bb.y) > 0.f ? o[u].y : 0.f; sa.y += dz; sb.y = fmaf(dz, xh, sb.y);
+                        xh = (xv.z - bmu.z) * brs.z; dz = fmaf(bg.z, xh, bb.z) > 0.f ? o[u].z : 0.f; sa.z += dz; sb.z = fmaf(dz, xh, sb.z);
+                        xh = (xv.w - bmu.w) * brs.w; dz = fmaf(bg.w, xh, bb.w) > 0.f ? o[u].w : 0.f; sa.w += dz; sb.w = fmaf(dz, xh, sb.w);
+                    }
                     if (fill[u]) {
                         // strided data gradient: the positions between the samples receive no contribution
                         const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -516,6 +547,21 @@ __global__ void __launch_bounds__(320) conv_tc_fwd_kernel(const __grid_constant_
                             for (int dx = 0; dx < 4; ++dx)
                                 if (fill[u] & (1 << (dy * 4 + dx))) *reinterpret_cast<float4*>(optr + dy * dense_h + dx * dense_w) = z;
                     }
+                }
+            }
+            if (stat_mode) {
+                // a thread kept one group of 4 channels throughout (256 is a multiple of c4n): add the 256 / c4n
+                // threads of each group in ascending order and store this tile's partial sums
+                asm volatile("bar.sync 1, 256;" ::: "memory");          // the staging area is free again
+                float4* red = reinterpret_cast<float4*>(smem);
+                red[2 * tid] = sa; red[2 * tid + 1] = sb;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (tid < c4n * 2) {
+                    const int g = tid >> 1, which = tid & 1;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int t2 = g; t2 < 256; t2 += c4n) { const float4 v2 = red[2 * t2 + which]; acc.x += v2.x; acc.y += v2.y; acc.z += v2.z; acc.w += v2.w; }
+                    float* dstp = p.stat_partials + ((size_t)blockIdx.x * 2 + which) * p.c_out + co0 + 4 * g;
+                    *reinterpret_cast<float4*>(dstp) = acc;
                 }
             }
         }
@@ -999,6 +1045,22 @@ bool conv_tc_supported(const ConvShape& s, int pass)
     return choose_box(v.Q, v.P, v.N, kTileM, 1, &b);
 }
 
+int conv_tc_tiles(const ConvShape& s, int pass)
+{
+    FwdView v;
+    PixelBox b;
+    if (pass == PASS_WGRAD || !fwd_view(s, pass, &v) || !choose_box(v.Q, v.P, v.N, kTileM, 1, &b)) return 0;
+    return ((v.Q + b.w - 1) / b.w) * ((v.P + b.h - 1) / b.h) * ((v.N + b.n - 1) / b.n);
+}
+
+bool conv_tc_can_fuse_bn(const ConvShape& s, int pass)
+{
+    FwdView v;
+    if (pass == PASS_WGRAD || !fwd_view(s, pass, &v)) return false;
+    const int n_chunk = v.c_out < 256 ? v.c_out : 256;
+    return 256 % (n_chunk / 4) == 0 && conv_tc_tiles(s, pass) > 0;
+}
+
 cudaError_t conv_tc_init()
 {
     if (g_encode) return cudaSuccess;
@@ -1033,7 +1095,8 @@ static_assert(sizeof(ConvTcFwdLaunch) <= sizeof(((ConvTcPlan*)0)->storage) && si
               "plan storage too small");
 
 cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int passes, const float* in, const float* in2,
-                            const float* w_hi, const float* w_lo, float* out, const float* extra, bool accumulate, void* scratch)
+                            const float* w_hi, const float* w_lo, float* out, const float* extra, bool accumulate, void* scratch,
+                            const ConvBnFuse* fuse)
 {
     plan->valid = 0; plan->s = s; plan->pass = pass;
     if (passes != 1 && passes != 3) return cudaErrorInvalidValue;
@@ -1129,6 +1192,11 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     if (stages > kFwdMaxStages) stages = kFwdMaxStages;
     if (stages > total) stages = total;
     p.stages = stages;
+    if (fuse && fuse->mode) {
+        if (256 % (n_chunk / 4)) return cudaErrorNotSupported;
+        p.stat_mode = fuse->mode; p.stat_partials = fuse->partials;
+        p.bn_x = fuse->bn_x; p.bn_stats = fuse->bn_stats; p.bn_gamma = fuse->bn_gamma; p.bn_beta = fuse->bn_beta;
+    }
     p.stacked = (passes == 3 && 2 * n_chunk <= 256) ? 1 : 0;
     p.tmem_cols = pow2_cols(p.stacked ? 2 * n_chunk : n_chunk);
     p.idesc = instr_desc(n_chunk, false, false);

@@ -23,12 +23,31 @@ struct ConvTcPlan {
     alignas(64) unsigned char storage[768];
 };
 
+// Batch-norm reductions folded into the forward / data-gradient kernel's write-out.
+//   mode 1 (forward): per tile, per output channel, sum and sum of squares of what the kernel writes (the
+//          statistics of the BN that reads this tensor next);
+//   mode 2 (data gradient): this kernel writes dL/dy of a BN+ReLU output y; per tile and channel it also forms
+//          sum dz and sum dz*xhat (dz = dy*[z>0]) from the BN's input bn_x, its saved statistics and gamma/beta.
+// partials: [conv_tc_tiles(s, pass)][2][channels] floats, written in full by every launch.
+struct ConvBnFuse {
+    int mode = 0;
+    float* partials = nullptr;
+    const float* bn_x = nullptr;
+    const float* bn_stats = nullptr;
+    const float* bn_gamma = nullptr;
+    const float* bn_beta = nullptr;
+};
+// Number of pixel tiles (= partial-sum rows) of the forward / data-gradient launch, and whether the fusion applies.
+int conv_tc_tiles(const ConvShape& s, int pass);
+bool conv_tc_can_fuse_bn(const ConvShape& s, int pass);
+
 // passes = 3: error-compensated (hi*hi + lo*hi + hi*lo); passes = 1: single TF32 pass.
 // pass = PASS_FWD:   out = conv(in, w) (+ extra); w_hi / w_lo = split weights [K][R][R][C]
 // pass = PASS_DGRAD: out (+)= dgrad(in = dy) (+ extra); w_hi / w_lo = split rearranged weights [C][R][R][K]
 // pass = PASS_WGRAD: out = wgrad(in = dy, in2 = x)
 cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int passes, const float* in, const float* in2,
-                            const float* w_hi, const float* w_lo, float* out, const float* extra, bool accumulate, void* scratch);
+                            const float* w_hi, const float* w_lo, float* out, const float* extra, bool accumulate, void* scratch,
+                            const ConvBnFuse* fuse = nullptr);
 cudaError_t conv_tc_launch(const ConvTcPlan* plan, DeviceStatus* status, cudaStream_t st, int64_t* n_launch);
 
 // One convolution's weights inside the flat parameter vector.

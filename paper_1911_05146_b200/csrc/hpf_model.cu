@@ -82,6 +82,9 @@ struct hpf_model {
     std::vector<int> grad_alias;              // tensor -> ADD op whose gradient buffer it shares, or -1
     std::vector<int> fused_into;              // conv -> residual ADD computed in its epilogue (its own output is not stored), or -1
     std::vector<int> add_done_by;             // ADD -> the conv that computes it, or -1
+    std::vector<int> bn_fwd_from, bn_bwd_from; // BN -> conv whose forward / data-gradient kernel leaves its per-tile sums, or -1
+    std::vector<int> conv_fwd_bn, conv_dgrad_bn; // the inverse maps
+    int opt_fuse_bn = 1;       // bit 0: forward statistics, bit 1: backward sums (measured slower: the write-out is latency bound)
     std::vector<GradEdge> edge0;              // per op: contribution to src0
     std::vector<AccumAction> accums;
     std::vector<std::vector<MessagePlan>> msg_plan;   // per cut
@@ -320,10 +323,52 @@ void build_fusion_plan(hpf_model* mdl)
     }
 }
 
+ConvShape conv_shape_of(const hpf_model* mdl, int i);
+bool op_uses_tc(const hpf_model* mdl, int i, int pass);
+
 ConvShape conv_shape_of(const hpf_model* mdl, int i)
 {
     const OpInfo& o = mdl->ops[i];
     return make_conv_shape(mdl->b, o.iH, o.iW, o.iC, o.op.c_out, o.op.ksize, o.op.stride, o.op.pad);
+}
+
+// Which convolutions run on the tensor cores, and which BN reductions ride in their write-out: the sums of a
+// BN's input in the forward kernel that produces it, the sums of the BN's backward in the data-gradient kernel
+// that produces dL/d(BN output).  Only when producer and BN run back to back on the same stream (same partition,
+// nothing but a fused residual add between them), so that the per-stream scratch can carry the partial sums.
+void build_kernel_plan(hpf_model* mdl)
+{
+    const int n = mdl->n_ops;
+    for (int pass = 0; pass < 3; ++pass) {
+        mdl->use_tc[pass].assign(n, 0);
+        for (int i = 0; i < n; ++i) mdl->use_tc[pass][i] = op_uses_tc(mdl, i, pass) ? 1 : 0;
+    }
+    mdl->bn_fwd_from.assign(n, -1); mdl->bn_bwd_from.assign(n, -1);
+    mdl->conv_fwd_bn.assign(n, -1); mdl->conv_dgrad_bn.assign(n, -1);
+    if (!mdl->opt_fuse_bn) return;
+    for (int j = 0; j < n; ++j) {
+        const OpInfo& bn = mdl->ops[j];
+        if (bn.op.kind != HPF_OP_BNRELU || bn.C > 2048) continue;
+        // forward: the kernel that writes the BN's input
+        int t = bn.op.src0, prod = -1;
+        if (mdl->ops[t].op.kind == HPF_OP_CONV && mdl->fused_into[t] < 0) prod = t;
+        else if (mdl->ops[t].op.kind == HPF_OP_ADD && mdl->add_done_by[t] >= 0) prod = mdl->add_done_by[t];
+        if ((mdl->opt_fuse_bn & 1) && prod >= 0 && mdl->use_tc[PASS_FWD][prod] && mdl->ops[prod].part == bn.part && mdl->conv_fwd_bn[prod] < 0 &&
+            conv_tc_can_fuse_bn(conv_shape_of(mdl, prod), PASS_FWD)) {
+            bool adjacent = true;
+            for (int k = prod + 1; k < j; ++k)
+                if (!(mdl->ops[k].op.kind == HPF_OP_ADD && mdl->add_done_by[k] >= 0)) adjacent = false;
+            if (adjacent) { mdl->bn_fwd_from[j] = prod; mdl->conv_fwd_bn[prod] = j; }
+        }
+        // backward: the data-gradient kernel of the BN output's only reader
+        if ((mdl->opt_fuse_bn & 2) && bn.consumers.size() == 1 && bn.consumers[0] == j + 1) {
+            const int i = j + 1;
+            if (mdl->ops[i].op.kind == HPF_OP_CONV && mdl->ops[i].op.src0 == j && mdl->use_tc[PASS_DGRAD][i] &&
+                mdl->ops[i].part == bn.part && conv_tc_can_fuse_bn(conv_shape_of(mdl, i), PASS_DGRAD)) {
+                mdl->bn_bwd_from[j] = i; mdl->conv_dgrad_bn[i] = j;
+            }
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -332,6 +377,7 @@ ConvShape conv_shape_of(const hpf_model* mdl, int i)
 void build_memory_plan(hpf_model* mdl)
 {
     build_fusion_plan(mdl);
+    build_kernel_plan(mdl);
     const int n = mdl->n_ops, M = mdl->M, P = mdl->P;
     size_t at = 0;
     auto take = [&](size_t bytes) { size_t o = at; at = align_up(at + bytes, 256); return o; };
@@ -347,6 +393,12 @@ void build_memory_plan(hpf_model* mdl)
                 const OpInfo& o = mdl->ops[i];
                 size_t need = bn_scratch_bytes((int64_t)mdl->b * o.H * o.W, o.C);
                 if (need > bn) bn = need;
+                for (int pass = PASS_FWD; pass <= PASS_DGRAD; ++pass) {
+                    const int from = pass == PASS_FWD ? mdl->bn_fwd_from[i] : mdl->bn_bwd_from[i];
+                    if (from < 0) continue;
+                    need = 256 + (size_t)conv_tc_tiles(conv_shape_of(mdl, from), pass) * 2 * o.C * sizeof(float);
+                    if (need > bn) bn = need;
+                }
             }
         mdl->bn_scratch_off[p] = take(bn);
     }
@@ -447,8 +499,14 @@ int forward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
         break;
     }
     case HPF_OP_BNRELU:
-        CU(bnrelu_fwd(in0, mdl->params + o.w_off, mdl->params + o.b_off, q.eps, out, mdl->stats(i, m),
-                      (int64_t)mdl->b * o.H * o.W, o.C, mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
+        if (mdl->bn_fwd_from[i] >= 0)      // the producing convolution left the per-tile sums in the stream's scratch
+            CU(bnrelu_fwd_fused(in0, mdl->params + o.w_off, mdl->params + o.b_off, q.eps, out, mdl->stats(i, m),
+                                reinterpret_cast<const float*>(mdl->ws + mdl->bn_scratch_off[p] + 256),
+                                conv_tc_tiles(conv_shape_of(mdl, mdl->bn_fwd_from[i]), PASS_FWD), (int64_t)mdl->b * o.H * o.W, o.C,
+                                st, &mdl->launches));
+        else
+            CU(bnrelu_fwd(in0, mdl->params + o.w_off, mdl->params + o.b_off, q.eps, out, mdl->stats(i, m),
+                          (int64_t)mdl->b * o.H * o.W, o.C, mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
         break;
     case HPF_OP_ADD:
         if (mdl->add_done_by[i] < 0) CU(add_fwd(in0, mdl->act(q.src1, m), out, mdl->numel(i), st, &mdl->launches));
@@ -507,9 +565,16 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
         break;
     }
     case HPF_OP_BNRELU:
-        CU(bnrelu_bwd(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m), addend,
-                      e.accumulate != 0, slot + o.w_off, slot + o.b_off, (int64_t)mdl->b * o.H * o.W, o.C,
-                      mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
+        if (mdl->bn_bwd_from[i] >= 0)      // the data-gradient kernel that produced dout left the per-tile sums
+            CU(bnrelu_bwd_fused(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m),
+                                addend, e.accumulate != 0, slot + o.w_off, slot + o.b_off,
+                                reinterpret_cast<const float*>(mdl->ws + mdl->bn_scratch_off[p] + 256),
+                                conv_tc_tiles(conv_shape_of(mdl, mdl->bn_bwd_from[i]), PASS_DGRAD), (int64_t)mdl->b * o.H * o.W,
+                                o.C, st, &mdl->launches));
+        else
+            CU(bnrelu_bwd(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m), addend,
+                          e.accumulate != 0, slot + o.w_off, slot + o.b_off, (int64_t)mdl->b * o.H * o.W, o.C,
+                          mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
         break;
     case HPF_OP_ADD:
         break;   // its contributions are aliases, on-the-fly addends, or the explicit accumulations above
@@ -721,6 +786,7 @@ int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
     case HPF_OPT_KEEP_MESSAGES: mdl->opt_messages = value != 0; break;
     case HPF_OPT_FUSE_ADD: mdl->opt_fuse_add = value != 0; break;
     case HPF_OPT_PDL: hpf::g_pdl_enabled = value != 0; break;
+    case HPF_OPT_FUSE_BN: if (value < 0 || value > 3) return fail(HPF_ERR_INVALID, "0..3"); mdl->opt_fuse_bn = value; break;
     case HPF_OPT_WGRAD_PASSES: if (value != 1 && value != 3) return fail(HPF_ERR_INVALID, "1 or 3 passes"); mdl->opt_wgrad_passes = value; break;
     default: return fail(HPF_ERR_INVALID, "unknown option");
     }
@@ -848,10 +914,8 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
     CU(cudaMemsetAsync(mdl->ws + mdl->zero_lo, 0, mdl->zero_hi - mdl->zero_lo, mdl->streams[0]));
     // tensor-core plans
     bool any_tc = false;
-    for (int pass = 0; pass < 3; ++pass) {
-        mdl->use_tc[pass].assign(n, 0);
-        for (int i = 0; i < n; ++i) if (op_uses_tc(mdl, i, pass)) { mdl->use_tc[pass][i] = 1; any_tc = true; }
-    }
+    for (int pass = 0; pass < 3; ++pass)
+        for (int i = 0; i < n; ++i) if (mdl->use_tc[pass][i]) any_tc = true;
     mdl->prep_table.assign(mdl->P, {});
     if (any_tc) {
         CU(conv_tc_init());
@@ -884,12 +948,30 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                             const hpf_op& a = mdl->ops[mdl->fused_into[i]].op;
                             residual = mdl->act(a.src0 == i ? a.src1 : a.src0, m);
                         }
+                        ConvBnFuse fuse;
+                        if (mdl->conv_fwd_bn[i] >= 0) {
+                            fuse.mode = 1;
+                            fuse.partials = reinterpret_cast<float*>(mdl->ws + mdl->bn_scratch_off[o.part] + 256);
+                        }
                         CU(conv_tc_prepare(pl, s, pass, passes, mdl->act(src, m), nullptr, wp + o.w_off, wp + G + o.w_off,
-                                           mdl->act(i, m), residual, false, scratch));
+                                           mdl->act(i, m), residual, false, scratch, &fuse));
                     }
-                    else if (pass == PASS_DGRAD)
+                    else if (pass == PASS_DGRAD) {
+                        ConvBnFuse fuse;
+                        const int j = mdl->conv_dgrad_bn[i];
+                        if (j >= 0) {
+                            const OpInfo& bn = mdl->ops[j];
+                            fuse.mode = 2;
+                            fuse.partials = reinterpret_cast<float*>(mdl->ws + mdl->bn_scratch_off[o.part] + 256);
+                            fuse.bn_x = mdl->act(bn.op.src0, m);
+                            fuse.bn_stats = mdl->stats(j, m);
+                            fuse.bn_gamma = mdl->params + bn.w_off;
+                            fuse.bn_beta = mdl->params + bn.b_off;
+                        }
                         CU(conv_tc_prepare(pl, s, pass, passes, mdl->grad(i, m), nullptr, wp + 2 * G + o.w_off, wp + 3 * G + o.w_off,
-                                           mdl->grad(src, m), ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch));
+                                           mdl->grad(src, m), ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch,
+                                           &fuse));
+                    }
                     else
                         CU(conv_tc_prepare(pl, s, pass, mdl->opt_conv_path == 2 ? 1 : mdl->opt_wgrad_passes, mdl->grad(i, m), mdl->act(src, m), nullptr, nullptr,
                                            mdl->gslots + (int64_t)m * mdl->G + o.w_off, nullptr, false, scratch));

@@ -66,6 +66,19 @@ def test_config1_resnet11(conv_path, graph):
                {hpf.OPT_CONV_PATH: conv_path, hpf.OPT_GRAPH: graph})
 
 
+@pytest.mark.parametrize("fuse_bn,pdl,wgrad_passes", [(0, 1, 1), (3, 0, 3), (2, 0, 3)])
+def test_config1_without_the_fusions(fuse_bn, pdl, wgrad_passes):
+    """The BN reductions in their own kernels or both folded into the convolutions, plain stream-ordered
+    launches, three-pass weight gradient."""
+    c = wl.config("r11")
+    try:
+        check_step(c["ops"], c["in_hwc"], c["B"], c["M"], c["cuts"],
+                   {hpf.OPT_FUSE_BN: fuse_bn, hpf.OPT_PDL: pdl, hpf.OPT_WGRAD_PASSES: wgrad_passes})
+    finally:
+        hpf.lib().hpf_set_option  # the PDL switch is process-wide: restore the default
+        m = hpf.Model(c["ops"], (c["B"],) + c["in_hwc"], c["cuts"], c["M"]); m.set_option(hpf.OPT_PDL, 1)
+
+
 @pytest.mark.parametrize("cuts", [[], [4], [3, 7, 8], [1, 5, 12, 25]])
 @pytest.mark.parametrize("fuse_add", [1, 0])
 def test_mid_block_cuts_and_jittered_bn(cuts, fuse_add):
