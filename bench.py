@@ -354,6 +354,9 @@ def main():
     ap.add_argument("--impl", default="hpf", choices=["hpf", "reference"])
     ap.add_argument("--workload", default="r1001", choices=sorted(wl.CONFIGS) + ["conv_sweep", "membound_sweep"])
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--cuts", default="equal", choices=["balanced", "equal"],
+                    help="partition cut points: balanced = the library's load balancer on its modelled op costs; "
+                         "equal = the same number of ops in every partition")
     ap.add_argument("--conv-path", type=int, default=0)
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-kernel-roofline", action="store_true")
@@ -395,7 +398,10 @@ def main():
 
     ops, hwc, B, M = cfg["ops"], cfg["in_hwc"], cfg["B"], cfg["M"]
     x, labels, theta = replica_inputs(cfg, rank)          # each replica its own batch, shared parameters
-    model = hpf.Model(ops, (B,) + tuple(hwc), cfg["cuts"], M)
+    cuts = cfg["cuts"]
+    if args.cuts == "balanced":
+        cuts = hpf.balance_cuts(hpf.estimate_op_costs(ops, (B // M,) + tuple(hwc)), cfg["P"])
+    model = hpf.Model(ops, (B,) + tuple(hwc), cuts, M)
     model.set_option(hpf.OPT_GRAPH, 0 if args.no_graph else 1)
     model.set_option(hpf.OPT_CONV_PATH, args.conv_path)
     G = model.num_params()
@@ -473,7 +479,7 @@ def main():
         "config": {"workload": NAMES[args.workload], "global_batch": world * B, "micro_batches": M,
                    "partitions": model.num_partitions(), "parallelism": "replicas x%d, no data-path collective" % world,
                    "l2": "working set %.1f GB per step exceeds the 126 MB L2; no explicit flush" % (ws_bytes / 1e9),
-                   "graph": not args.no_graph, "conv_sites_tensor_core": n_tc, "conv_sites_cuda_core": n_cc,
+                   "cuts": args.cuts, "cut_points": list(cuts), "graph": not args.no_graph, "conv_sites_tensor_core": n_tc, "conv_sites_cuda_core": n_cc,
                    "loss": loss},
         "e2e": {"value": world * B / (ms_e2e / args.steps * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": int(hx.numel() * 4 + hl.numel() * 4), "d2h_bytes_per_step": 4},

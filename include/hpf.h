@@ -125,6 +125,16 @@ int hpf_boundary_desc(const hpf_model *model, int32_t cut, int32_t i, int32_t *p
 /* Fill/drain pipeline: forward (p,m) runs at tick p+m, backward (p,m) at tick (P-1-p)+m. */
 int hpf_schedule_tick(const hpf_model *model, int32_t p, int32_t m, int32_t *fwd_tick, int32_t *bwd_tick);
 
+/* ---- load balancer (Section 5.4 names the component and leaves it to future work) -----------------
+ * hpf_estimate_op_costs: modelled time (microseconds, forward + backward on the pipeline's critical chain) of every op
+ * for one micro-batch of b samples: a fixed latency per kernel, a term per tensor-core K step and a term per byte
+ * moved, with constants calibrated on B200 at micro-batch 16 (weight gradients run beside the chain and are not
+ * counted).  Host only.  cost_us: n_ops doubles.
+ * hpf_balance_cuts: P-1 cut points that minimise the largest partition cost (contiguous partitions, every
+ * partition non-empty).  Any non-negative costs may be passed (measured ones, too).  Host only. */
+int hpf_estimate_op_costs(const hpf_op *ops, int32_t n_ops, const int32_t in_shape[4] /* b,H,W,C */, double *cost_us);
+int hpf_balance_cuts(const double *cost, int32_t n_ops, int32_t n_partitions, int32_t *cuts /* P-1 */);
+
 /* ---- device resources ---------------------------------------------------------------------------- */
 int hpf_workspace_bytes(const hpf_model *model, size_t *bytes);
 /* d_params [G], d_grad_slots [M][G] (slot m = dL_m/dtheta), d_grad_avg [G], d_workspace (256-byte

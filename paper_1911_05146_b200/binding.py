@@ -40,6 +40,8 @@ _SIGNATURES = {
     "hpf_boundary_count": [_vp, _i32, _pi32],
     "hpf_boundary_desc": [_vp, _i32, _i32, _pi32, _pi32],
     "hpf_schedule_tick": [_vp, _i32, _i32, _pi32, _pi32],
+    "hpf_estimate_op_costs": [C.POINTER(_Op), _i32, _pi32, C.POINTER(C.c_double)],
+    "hpf_balance_cuts": [C.POINTER(C.c_double), _i32, _i32, _pi32],
     "hpf_workspace_bytes": [_vp, C.POINTER(C.c_size_t)],
     "hpf_bind": [_vp, _vp, _vp, _vp, _vp, C.c_size_t, C.POINTER(_vp), _i32],
     "hpf_forward": [_vp, _vp, _vp],
@@ -106,6 +108,27 @@ def _stream(stream):
         import torch
         return torch.cuda.current_stream().cuda_stream
     return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def _op_array(ops):
+    arr = (_Op * len(ops))()
+    for i, o in enumerate(ops):
+        arr[i] = _Op(*[int(v) for v in o[:8]], float(o[8]))
+    return arr
+
+
+def estimate_op_costs(ops, microbatch_shape):
+    """Modelled microseconds (forward + backward chain) per op for one micro-batch of shape (b, H, W, C)."""
+    out = (C.c_double * len(ops))()
+    _check(lib().hpf_estimate_op_costs(_op_array(ops), len(ops), (_i32 * 4)(*microbatch_shape), out))
+    return list(out)
+
+
+def balance_cuts(costs, n_partitions):
+    """Cut points minimising the largest partition cost."""
+    cuts = (_i32 * max(n_partitions - 1, 1))()
+    _check(lib().hpf_balance_cuts((C.c_double * len(costs))(*costs), len(costs), n_partitions, cuts))
+    return list(cuts[:n_partitions - 1])
 
 
 class Model:

@@ -866,6 +866,76 @@ int hpf_schedule_tick(const hpf_model* mdl, int32_t p, int32_t m, int32_t* fwd_t
     return HPF_OK;
 }
 
+int hpf_estimate_op_costs(const hpf_op* ops, int32_t n_ops, const int32_t in_shape[4], double* cost_us)
+{
+    if (!ops || !in_shape || !cost_us || n_ops < 1) return fail(HPF_ERR_INVALID, "null argument");
+    // shapes through a throw-away model (validates the list as well)
+    hpf_model* tmp = nullptr;
+    int rc = hpf_model_create(ops, n_ops, in_shape, nullptr, 0, 1, &tmp);
+    if (rc) return rc;
+    // Calibration (B200, micro-batch 16, one stream): a bottleneck block costs 113 / 115 / 149 us at 32x32 / 16x16 / 8x8,
+    // which a fixed cost per kernel, 0.39 us per tensor-core K step (8 channels of one tap, forward plus data
+    // gradient) and 1.4 TB/s of effective bandwidth reproduce.
+    const double us_per_k8 = 0.39, bytes_per_us = 1.4e6;
+    for (int i = 0; i < n_ops; ++i) {
+        const OpInfo& o = tmp->ops[i];
+        const double in_el = (double)in_shape[0] * o.iH * o.iW * o.iC, out_el = (double)in_shape[0] * o.H * o.W * o.C;
+        double c = 0.0;
+        switch (o.op.kind) {
+        case HPF_OP_CONV: {
+            const int taps = o.op.ksize * o.op.ksize;
+            const double k8 = taps * (o.op.c_in / 8.0) + (o.op.src0 >= 0 ? taps * (o.op.c_out / 8.0) : 0.0);
+            c = 8.0 + us_per_k8 * k8 + 4.0 * 2.0 * (in_el + out_el) / bytes_per_us;
+            break;
+        }
+        case HPF_OP_BNRELU: c = 9.0 + 20.0 * out_el / bytes_per_us; break;
+        case HPF_OP_ADD: c = 0.0; break;                       // fused into the producing convolution
+        case HPF_OP_MAXPOOL: c = 6.0 + 4.0 * 2.0 * (in_el + out_el) / bytes_per_us; break;
+        default: c = 20.0; break;                               // head: a handful of tiny kernels
+        }
+        cost_us[i] = c;
+    }
+    hpf_model_destroy(tmp);
+    return HPF_OK;
+}
+
+int hpf_balance_cuts(const double* cost, int32_t n_ops, int32_t P, int32_t* cuts)
+{
+    if (!cost || n_ops < 1 || P < 1 || P > n_ops || (P > 1 && !cuts)) return fail(HPF_ERR_INVALID, "bad argument");
+    double total = 0.0, biggest = 0.0;
+    for (int i = 0; i < n_ops; ++i) {
+        if (!(cost[i] >= 0.0)) return fail(HPF_ERR_INVALID, "costs must be non-negative");
+        total += cost[i];
+        if (cost[i] > biggest) biggest = cost[i];
+    }
+    // smallest bottleneck B such that a greedy left-to-right fill needs at most P partitions (bisection on B)
+    auto parts_needed = [&](double B) {
+        int parts = 1; double acc = 0.0;
+        for (int i = 0; i < n_ops; ++i) {
+            if (acc + cost[i] > B && acc > 0.0) { ++parts; acc = 0.0; }
+            acc += cost[i];
+        }
+        return parts;
+    };
+    double lo = biggest, hi = total > biggest ? total : biggest;
+    for (int it = 0; it < 100; ++it) {
+        const double mid = 0.5 * (lo + hi);
+        if (parts_needed(mid) <= P) hi = mid; else lo = mid;
+    }
+    // cut greedily at bottleneck hi, but never leave fewer ops than partitions still to be filled
+    int made = 0; double acc = 0.0; int start = 0;
+    for (int i = 0; i < n_ops && made < P - 1; ++i) {
+        const int remaining_parts = P - 1 - made;                // partitions still to open after the current one
+        const bool must = n_ops - i == remaining_parts;          // every remaining op has to open a partition
+        if (i > start && ((acc + cost[i] > hi * (1.0 + 1e-12)) || must)) { cuts[made++] = i; acc = 0.0; start = i; }
+        acc += cost[i];
+    }
+    // if the costs ran out early (zero-cost tail), spread the remaining cuts over the last ops
+    for (int k = made; k < P - 1; ++k) cuts[k] = n_ops - (P - 1 - k);
+    for (int k = P - 2; k > 0; --k) if (cuts[k - 1] >= cuts[k]) cuts[k - 1] = cuts[k] - 1;
+    return HPF_OK;
+}
+
 int hpf_workspace_bytes(const hpf_model* mdl_c, size_t* bytes)
 {
     if (!mdl_c || !bytes) return fail(HPF_ERR_INVALID, "null");

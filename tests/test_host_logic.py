@@ -126,3 +126,34 @@ def test_workspace_grows_with_message_buffers():
     b = hpf.Model(ops, (8, 32, 32, 3), [4], 2)
     b.set_option(hpf.OPT_KEEP_MESSAGES, 1)
     assert b.workspace_bytes() > a.workspace_bytes()
+
+
+def test_load_balancer_cuts():
+    """Section 5.4's load balancer: contiguous partitions minimising the largest modelled partition cost."""
+    import itertools
+    import numpy as np
+    rng = np.random.default_rng(0)
+    for n, P in ((6, 2), (7, 3), (9, 4), (8, 8), (5, 1)):
+        cost = rng.uniform(0.1, 5.0, n).tolist()
+        cuts = hpf.balance_cuts(cost, P)
+        assert len(cuts) == P - 1 and all(0 < c < n for c in cuts) and cuts == sorted(set(cuts))
+        b = [0] + cuts + [n]
+        got = max(sum(cost[b[i]:b[i + 1]]) for i in range(P))
+        best = min(max(sum(cost[x:y]) for x, y in zip((0,) + c, c + (n,))) for c in itertools.combinations(range(1, n), P - 1)) if P > 1 else sum(cost)
+        assert got <= best * (1 + 1e-9), (cost, cuts, got, best)          # brute force over every cut placement
+    with pytest.raises(hpf.HpfError):
+        hpf.balance_cuts([1.0, 2.0], 3)                                    # more partitions than ops
+    with pytest.raises(hpf.HpfError):
+        hpf.balance_cuts([1.0, -2.0, 1.0], 2)
+    # the modelled costs of ResNet-1001: 8x8-stage blocks are the dearest, so their partitions get fewer ops
+    c = wl.config("r1001")
+    costs = hpf.estimate_op_costs(c["ops"], (16, 32, 32, 3))
+    assert len(costs) == len(c["ops"]) and min(costs) >= 0
+    cuts = hpf.balance_cuts(costs, 8)
+    sizes = np.diff([0] + cuts + [len(c["ops"])])
+    assert sizes[-1] < sizes[0]
+    parts = [sum(costs[a:b]) for a, b in zip([0] + cuts, cuts + [len(c["ops"])])]
+    eq = [sum(costs[a:b]) for a, b in zip([0] + c["cuts"], c["cuts"] + [len(c["ops"])])]
+    assert max(parts) < max(eq) and max(parts) / min(parts) < 1.05
+    m = hpf.Model(c["ops"], (c["B"],) + c["in_hwc"], cuts, c["M"])       # the cuts are accepted by the model
+    assert m.num_partitions() == 8
