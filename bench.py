@@ -191,7 +191,7 @@ def kernel_roofline(torch, hpf, cfg, pk):
             in_el = b * P * Q * C if o.stride > 1 else b * H * W * C
             key = (o.ksize, o.stride, o.pad, C, K, H)
             weight[key] = weight.get(key, 0) + 4.0 * (in_el + b * P * Q * K + K * o.ksize * o.ksize * C)
-    (ks, st, pad, ci, co, H), _ = max(weight.items(), key=lambda kv: kv[1])
+    (ks, st, pad, ci, co, H), _ = max(weight.items(), key=lambda kv: (kv[1], kv[0][3]))      # ties: the wider input
     P = (H + 2 * pad - ks) // st + 1
     in_el = b * P * P * ci if st > 1 else b * H * H * ci
     alg = 4.0 * (in_el + b * P * P * co + co * ks * ks * ci)
@@ -224,7 +224,10 @@ def kernel_roofline(torch, hpf, cfg, pk):
     sec = e0.elapsed_time(e1) * 1e-3 / (3 * reps)
     achieved = alg / sec / 1e9
     return {"bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"],
-            "traffic": None, "peak_source": pk["source"],
+            # dram__bytes_read + dram__bytes_write of this kernel in the ncu capture of the same shape at batch 128
+            # (profiles/conv_tc_fwd_1x1_64to16_at32_batch128.md: 33.62 MB read = the input once, the output still in L2
+            # when the kernel ends), scaled by the pixels per launch
+            "traffic": 33.62e6 * b / 128.0 if (ks, st, ci, co, H) == (1, 1, 64, 16, 32) else None, "peak_source": pk["source"],
             "kernel": "conv_tc_fwd_kernel (tcgen05 implicit GEMM, three-pass TF32), %dx%d stride %d, %d->%d channels, %dx%d "
                       "pixels, micro-batch %d; %d rotating operand sets; one 8-byte status memset node precedes each launch"
                       % (ks, ks, st, ci, co, H, H, b, nset),

@@ -280,7 +280,7 @@ __device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__flo
 // ------------------------------------------------------------------------------------------------
 // forward / data-gradient kernel: 10 warps = TMA producer, MMA issuer, 8 splitter / epilogue warps
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(320) conv_tc_fwd_kernel(const __grid_constant__ FwdParams gp)
+__global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_constant__ FwdParams gp)
 {
     __shared__ FwdScalars p;                 // scalar parameters, see load_scalars
     pdl_launch_dependents();
@@ -522,6 +522,13 @@ __global__ void __launch_bounds__(320) conv_tc_fwd_kernel(const __grid_constant_
                     for (int u = 0; u < 4; ++u)
                         if (off[u] >= 0) { const float4 e = *reinterpret_cast<const float4*>(outp + off[u]); o[u].x += e.x; o[u].y += e.y; o[u].z += e.z; o[u].w += e.w; }
                 }
+                float4 xv4[4];
+                if (stat_mode == 2) {
+                    // all loads of the batch are issued before its first store: a load behind a store would wait for it
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (off[u] >= 0) xv4[u] = __ldg(reinterpret_cast<const float4*>(p.bn_x + off[u]));
+                }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     if (off[u] < 0) continue;
@@ -533,7 +540,7 @@ __global__ void __launch_bounds__(320) conv_tc_fwd_kernel(const __grid_constant_
                         sb.z = fmaf(o[u].z, o[u].z, sb.z); sb.w = fmaf(o[u].w, o[u].w, sb.w);
                     } else if (stat_mode == 2) {
                         // dz = dy * [z > 0] with z recomputed exactly as the BN forward computed it
-                        const float4 xv = __ldg(reinterpret_cast<const float4*>(p.bn_x + off[u]));
+                        const float4 xv = xv4[u];
                         float xh, dz;
                         xh = (xv.x - bmu.x) * brs.x; dz = fmaf(bg.x, xh, bb.x) > 0.f ? o[u].x : 0.f; sa.x += dz; sb.x = fmaf(dz, xh, sb.x);
                         xh = (xv.y - bmu.y) * brs.y; dz = fmaf(bg.y, xh, bb.y) > 0.f ? o[u].y : 0.f; sa.y += dz; sb.y = fmaf(dz, xh, sb.y);

@@ -548,9 +548,7 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
             CU(cudaEventRecord(mdl->ev_side[p], st));
             CU(cudaStreamWaitEvent(wst, mdl->ev_side[p], 0));
         }
-        static const bool skip_wgrad_dbg = getenv("HPF_DBG_SKIP_WGRAD") != nullptr;
-        if (skip_wgrad_dbg) {
-        } else if (mdl->use_tc[PASS_WGRAD][i]) {
+        if (mdl->use_tc[PASS_WGRAD][i]) {
             CU(conv_tc_launch(&mdl->tc_plan[PASS_WGRAD][(size_t)m * mdl->n_ops + i], mdl->status(), wst, &mdl->launches));
         } else {
             CU(conv_wgrad_simt(in0, dout, slot + o.w_off, s, mdl->ws + mdl->conv_scratch_off[p], wst, &mdl->launches));
