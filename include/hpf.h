@@ -102,9 +102,16 @@ int hpf_model_destroy(hpf_model *model);
  *                          of the tensor-core convolution kernel that produces the BN's input, when both run back to
  *                          back on one stream; the BN forward is then one kernel.  bit 1 (default off: measured slower):
  *                          the same for the backward sums (dbeta, dgamma) in the data-gradient kernel that produces
- *                          the gradient of the BN's output.  0: every BN runs its own reduction kernels. */
+ *                          the gradient of the BN's output.  bit 2 (default on; needs bit 0): a BN+ReLU whose output only the
+ *                          next op reads, a stride-1 tensor-core convolution of the same partition, has no kernel of
+ *                          its own: that convolution derives the statistics from the per-tile sums, applies the BN+ReLU
+ *                          to its input tile on the way to the tensor core and stores the BN's output and statistics as
+ *                          a by-product.  0: every BN runs its own reduction kernels.  Default 5.
+ *   HPF_OPT_CELL_TIMES     1: a one-thread kernel stores the device's nanosecond timer at the start and at the end of
+ *                          every (partition, micro-batch) cell of the forward and backward schedules (Section 5.3's
+ *                          pipeline, as it really ran); read them with hpf_cell_times.  Default 0. */
 typedef enum { HPF_OPT_GRAPH = 1, HPF_OPT_CONV_PATH = 2, HPF_OPT_SINGLE_STREAM = 3, HPF_OPT_KEEP_MESSAGES = 4,
-               HPF_OPT_FUSE_ADD = 5, HPF_OPT_PDL = 6, HPF_OPT_WGRAD_PASSES = 7, HPF_OPT_FUSE_BN = 8 } hpf_option;
+               HPF_OPT_FUSE_ADD = 5, HPF_OPT_PDL = 6, HPF_OPT_WGRAD_PASSES = 7, HPF_OPT_FUSE_BN = 8, HPF_OPT_CELL_TIMES = 9 } hpf_option;
 int hpf_set_option(hpf_model *model, int32_t option, int32_t value);
 
 /* ---- integer bookkeeping (Section 5.1 lists, Section 5.3 pipelining) ----------------------------- */
@@ -174,6 +181,11 @@ int hpf_tensor_ptr(const hpf_model *model, int32_t op, int32_t m, int32_t want_g
 int hpf_message_ptr(const hpf_model *model, int32_t cut, int32_t i, int32_t m, int32_t want_grad, const float **d_ptr);
 /* Per-micro-batch losses L_m (device, M floats). */
 int hpf_loss_slots_ptr(const hpf_model *model, const float **d_ptr);
+/* Pipeline timeline (needs HPF_OPT_CELL_TIMES=1 and the phase to have run): h_ns[(p*M + m)*2 + {0,1}] = device
+ * timer in nanoseconds at the start / end of cell (partition p, micro-batch m) of the last forward (phase 0) or
+ * backward (phase 1).  h_ns: host, 2*P*M values.  Synchronises.  HPF_ERR_STATE if the option is off. */
+int hpf_cell_times(hpf_model *model, int32_t phase, int64_t *h_ns);
+
 /* Kernel launches (graph kernel nodes count as launches) issued by the step calls since bind. */
 int hpf_launch_count(const hpf_model *model, int64_t *n);
 /* How many convolution launch sites per phase use the tensor-core path / the CUDA-core path. */

@@ -5,7 +5,7 @@ import os
 from . import build as _build
 
 CONV, BNRELU, ADD, MAXPOOL, HEAD = 1, 2, 3, 4, 5
-OPT_GRAPH, OPT_CONV_PATH, OPT_SINGLE_STREAM, OPT_KEEP_MESSAGES, OPT_FUSE_ADD, OPT_PDL, OPT_WGRAD_PASSES, OPT_FUSE_BN = 1, 2, 3, 4, 5, 6, 7, 8
+OPT_GRAPH, OPT_CONV_PATH, OPT_SINGLE_STREAM, OPT_KEEP_MESSAGES, OPT_FUSE_ADD, OPT_PDL, OPT_WGRAD_PASSES, OPT_FUSE_BN, OPT_CELL_TIMES = 1, 2, 3, 4, 5, 6, 7, 8, 9
 
 
 class HpfError(RuntimeError):
@@ -54,6 +54,7 @@ _SIGNATURES = {
     "hpf_message_ptr": [_vp, _i32, _i32, _i32, _i32, C.POINTER(_vp)],
     "hpf_loss_slots_ptr": [_vp, C.POINTER(_vp)],
     "hpf_launch_count": [_vp, _pi64],
+    "hpf_cell_times": [_vp, _i32, _pi64],
     "hpf_conv_path_counts": [_vp, _pi64, _pi64],
     "hpf_conv_scratch_bytes": [_i32] * 8 + [C.POINTER(C.c_size_t)],
     "hpf_conv_prepare_weights": [_vp, _vp, _i32, _i32, _i32, _vp],
@@ -233,6 +234,12 @@ class Model:
 
     def loss_slots_ptr(self):
         p = _vp(); _check(lib().hpf_loss_slots_ptr(self._h, C.byref(p))); return p.value
+
+    def cell_times(self, phase):
+        """ns timestamps [p][m] = (start, end) of every cell of the last forward (0) / backward (1)."""
+        P = self.num_partitions()
+        buf = (_i64 * (P * self.M * 2))(); _check(lib().hpf_cell_times(self._h, int(phase), buf))
+        return [[(buf[(p * self.M + m) * 2], buf[(p * self.M + m) * 2 + 1]) for m in range(self.M)] for p in range(P)]
 
     def launch_count(self):
         n = _i64(); _check(lib().hpf_launch_count(self._h, C.byref(n))); return n.value

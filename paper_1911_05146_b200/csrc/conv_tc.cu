@@ -32,6 +32,7 @@
 // device status word, stops issuing work, waits (bounded) for its TMA copies in flight, frees its
 // tensor memory and returns.
 #include "conv_tc.h"
+#include <cstdlib>
 
 #include <cuda.h>
 #include <stdint.h>
@@ -231,6 +232,17 @@ struct FwdScalars {
     const float* bn_stats;       // mode 2: mean[c_out], rstd[c_out]
     const float* bn_gamma;
     const float* bn_beta;
+    // BN+ReLU applied to the activation operand on its way to the tensor core (see ConvBnFuse::in_mode)
+    int bn_in;
+    int bn_in_tiles;             // rows of bn_in_partials
+    int in_w, in_h;              // extent of the input pixel grid (the padding mask)
+    float bn_in_eps;
+    double bn_in_inv_rows;       // 1 / (pixels the statistics run over)
+    const float* bn_in_partials; // [bn_in_tiles][2][c_in] per-tile sums of x and x*x
+    const float* bn_in_gamma;
+    const float* bn_in_beta;
+    float* bn_in_stats;          // mean[c_in], rstd[c_in], written by the first CTA
+    float* bn_in_y;              // relu(bn(x)), dense [N][in_h][in_w][c_in], written by the CTAs of the first channel slice
 };
 struct alignas(64) FwdParams {
     CUtensorMap tm_a;            // activations {C, Wv, Hv, N}
@@ -356,11 +368,12 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             const bool stacked = p.stacked != 0;
             const int stages = p.stages, k8n = p.kchunk / 8;
             const bool three = p.passes == 3;
+            const bool split_first = three || p.bn_in != 0;   // the splitter warps rewrite the tile before it is read
             int it = 0, s = 0;
             uint32_t par = 0;
             for (; it < total; ++it) {
                 if (!mbar_wait(full0 + 8 * s, par, &abort_flag)) { report(p.status, 2); break; }
-                if (three && !mbar_wait(split0 + 8 * s, par, &abort_flag)) { report(p.status, 6); break; }
+                if (split_first && !mbar_wait(split0 + 8 * s, par, &abort_flag)) { report(p.status, 6); break; }
                 tc_fence_after();
                 if (it == 0) HPF_TL(5);
                 const uint32_t st = smem_base + s * stage_bytes;
@@ -398,7 +411,107 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
         // ---- warps 2..9: split the activation tile into hi / lo, then the epilogue ----
         const int tid = threadIdx.x - 64;               // 0..255
         bool ok = true;
-        if (p.passes == 3) {
+        if (p.bn_in) {
+            // ---- BN+ReLU on the way in: the tile holds the BN's input x; the operand is relu(gamma*xhat+beta) ----
+            // Statistics: every CTA adds the producer's per-tile sums in the same fixed order (fp64), so all CTAs
+            // hold identical mean / rstd; the first CTA stores them for the backward pass.
+            __shared__ double bn_red[256][4];
+            __shared__ __align__(16) float bn_par[4][256];      // mean, rstd, gamma, beta per input channel
+            const int C = p.c_in, ncol4 = C >> 1;              // float4 columns of one tile's [2][C] sums (256 % ncol4 == 0)
+            {
+                const int col4 = tid % ncol4, ln = tid / ncol4, L = 256 / ncol4;
+                const float4* part = reinterpret_cast<const float4*>(p.bn_in_partials);
+                double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+#pragma unroll 4
+                for (int k = ln; k < p.bn_in_tiles; k += L) {
+                    const float4 v = __ldcg(part + (size_t)k * ncol4 + col4);
+                    a0 += (double)v.x; a1 += (double)v.y; a2 += (double)v.z; a3 += (double)v.w;
+                }
+                bn_red[tid][0] = a0; bn_red[tid][1] = a1; bn_red[tid][2] = a2; bn_red[tid][3] = a3;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (tid < ncol4) {
+                    // rows tid, tid + ncol4, ... are read by this thread alone, so the total can go back into row tid
+                    double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
+                    for (int l = 0; l < L; ++l) {
+                        const double* r = bn_red[l * ncol4 + tid];
+                        t0 += r[0]; t1 += r[1]; t2 += r[2]; t3 += r[3];
+                    }
+                    bn_red[tid][0] = t0; bn_red[tid][1] = t1; bn_red[tid][2] = t2; bn_red[tid][3] = t3;
+                }
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                const double* tot = &bn_red[0][0];              // [2][C]: sums, then sums of squares
+                for (int c = tid; c < C; c += 256) {
+                    const double mean = tot[c] * p.bn_in_inv_rows;
+                    double var = tot[C + c] * p.bn_in_inv_rows - mean * mean;
+                    if (var < 0.0) var = 0.0;
+                    const float mu = (float)mean, rs = (float)(1.0 / sqrt(var + (double)p.bn_in_eps));
+                    bn_par[0][c] = mu; bn_par[1][c] = rs;
+                    bn_par[2][c] = __ldg(p.bn_in_gamma + c); bn_par[3][c] = __ldg(p.bn_in_beta + c);
+                    if (blockIdx.x == 0 && blockIdx.y == 0) { p.bn_in_stats[c] = mu; p.bn_in_stats[C + c] = rs; }
+                }
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+            }
+            // A thread owns one 16-byte column of the (swizzled) tile rows tid/f4row + j*(256/f4row): its four
+            // channels within the K chunk are fixed, and so are the pixels of its rows.
+            const int f4row = p.kchunk >> 2;                    // 4 or 8 float4 per tile row
+            const int per = (int)(p.a_bytes >> 12);             // rows per thread: 2 or 4
+            const int row0 = tid / f4row, rstep = 256 / f4row;
+            const int cph = tid % f4row;
+            const int clog = p.kchunk == 32 ? (cph ^ (row0 & 7)) : (cph ^ ((row0 >> 1) & 3));
+            int px[4], py[4], pn[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int r = row0 + j * rstep;
+                const int wi = r % p.box_w, hi = (r / p.box_w) % p.box_h, ni = r / (p.box_w * p.box_h);
+                px[j] = q0 + wi; py[j] = p0 + hi;
+                pn[j] = (j < per && ni < p.box_n && n0 + ni < p.N) ? n0 + ni : -1;
+            }
+            const bool three = p.passes == 3;
+            const bool writer = blockIdx.y == 0;
+            for (int it = 0; it < total; ++it) {
+                const int s = it % p.stages;
+                ok = mbar_wait(full0 + 8 * s, (it / p.stages) & 1, &abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) { if (lane == 0) report(p.status, 7); break; }
+                if (it == 0 && tid == 0) HPF_TL(3);
+                const int tap = it / p.n_kchunks, kc = it - tap * p.n_kchunks;
+                const int dyy = tap / p.R - p.pad, dxx = tap % p.R - p.pad;
+                const int ch = kc * p.kchunk + 4 * clog;
+                const float4 mu = *reinterpret_cast<const float4*>(&bn_par[0][ch]);
+                const float4 rs = *reinterpret_cast<const float4*>(&bn_par[1][ch]);
+                const float4 g = *reinterpret_cast<const float4*>(&bn_par[2][ch]);
+                const float4 b = *reinterpret_cast<const float4*>(&bn_par[3][ch]);
+                float4* a = reinterpret_cast<float4*>(smem + s * p.stage_bytes);
+                float4* alo = reinterpret_cast<float4*>(smem + s * p.stage_bytes + off_alo);
+                float4 v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) if (j < per) v[j] = a[tid + 256 * j];
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (j < per) {
+                        const int xx = px[j] + dxx, yy = py[j] + dyy;
+                        const bool inside = pn[j] >= 0 && (unsigned)xx < (unsigned)p.in_w && (unsigned)yy < (unsigned)p.in_h;
+                        float4 y;       // the padding ring is zero AFTER the activation
+                        y.x = inside ? fmaxf(fmaf(g.x, (v[j].x - mu.x) * rs.x, b.x), 0.f) : 0.f;
+                        y.y = inside ? fmaxf(fmaf(g.y, (v[j].y - mu.y) * rs.y, b.y), 0.f) : 0.f;
+                        y.z = inside ? fmaxf(fmaf(g.z, (v[j].z - mu.z) * rs.z, b.z), 0.f) : 0.f;
+                        y.w = inside ? fmaxf(fmaf(g.w, (v[j].w - mu.w) * rs.w, b.w), 0.f) : 0.f;
+                        if (writer && inside && dxx == 0 && dyy == 0)     // each pixel is some tile's centre tap exactly once
+                            *reinterpret_cast<float4*>(p.bn_in_y + (((size_t)pn[j] * p.in_h + yy) * p.in_w + xx) * C + ch) = y;
+                        if (three) {
+                            const float4 h = make_float4(tf32_hi(y.x), tf32_hi(y.y), tf32_hi(y.z), tf32_hi(y.w));
+                            a[tid + 256 * j] = h;
+                            alo[tid + 256 * j] = make_float4(y.x - h.x, y.y - h.y, y.z - h.z, y.w - h.w);
+                        } else {
+                            a[tid + 256 * j] = y;
+                        }
+                    }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(split0 + 8 * s);
+                if (it == 0 && tid == 0) HPF_TL(4);
+            }
+        } else if (p.passes == 3) {
             const int per = (int)(p.a_bytes >> 12);     // float4 per thread: a_bytes / 16 / 256 = 2 or 4
             for (int it = 0; it < total; ++it) {
                 const int s = it % p.stages;
@@ -1068,6 +1181,14 @@ bool conv_tc_can_fuse_bn(const ConvShape& s, int pass)
     return 256 % (n_chunk / 4) == 0 && conv_tc_tiles(s, pass) > 0;
 }
 
+bool conv_tc_can_fuse_bn_input(const ConvShape& s)
+{
+    FwdView v;
+    if (!fwd_view(s, PASS_FWD, &v) || s.stride != 1) return false;
+    const int C = s.C;
+    return C >= 16 && C <= 256 && (C & (C - 1)) == 0 && conv_tc_tiles(s, PASS_FWD) > 0;
+}
+
 cudaError_t conv_tc_init()
 {
     if (g_encode) return cudaSuccess;
@@ -1198,11 +1319,26 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     const int total = v.R * v.R * p.n_kchunks;
     if (stages > kFwdMaxStages) stages = kFwdMaxStages;
     if (stages > total) stages = total;
+    {
+        static const int target = getenv("HPF_DBG_SMEM_TARGET") ? atoi(getenv("HPF_DBG_SMEM_TARGET")) : 0;
+        if (target > 0) {
+            int occ = target / (int)p.stage_bytes;
+            if (occ < 1) occ = 1;
+            if (stages > occ) stages = occ;
+        }
+    }
     p.stages = stages;
     if (fuse && fuse->mode) {
         if (256 % (n_chunk / 4)) return cudaErrorNotSupported;
         p.stat_mode = fuse->mode; p.stat_partials = fuse->partials;
         p.bn_x = fuse->bn_x; p.bn_stats = fuse->bn_stats; p.bn_gamma = fuse->bn_gamma; p.bn_beta = fuse->bn_beta;
+    }
+    if (fuse && fuse->in_mode) {
+        if (pass != PASS_FWD || !conv_tc_can_fuse_bn_input(s) || fuse->in_tiles < 1 || fuse->in_rows < 1) return cudaErrorNotSupported;
+        p.bn_in = 1; p.bn_in_tiles = fuse->in_tiles; p.in_w = v.in_w; p.in_h = v.in_h; p.bn_in_eps = fuse->in_eps;
+        p.bn_in_inv_rows = 1.0 / (double)fuse->in_rows;
+        p.bn_in_partials = fuse->in_partials; p.bn_in_gamma = fuse->in_gamma; p.bn_in_beta = fuse->in_beta;
+        p.bn_in_stats = fuse->in_stats; p.bn_in_y = fuse->in_y;
     }
     p.stacked = (passes == 3 && 2 * n_chunk <= 256) ? 1 : 0;
     p.tmem_cols = pow2_cols(p.stacked ? 2 * n_chunk : n_chunk);

@@ -20,7 +20,7 @@ struct ConvTcPlan {
     ConvShape s;
     int pass;
     int valid;
-    alignas(64) unsigned char storage[768];
+    alignas(64) unsigned char storage[896];
 };
 
 // Batch-norm reductions folded into the forward / data-gradient kernel's write-out.
@@ -36,7 +36,23 @@ struct ConvBnFuse {
     const float* bn_stats = nullptr;
     const float* bn_gamma = nullptr;
     const float* bn_beta = nullptr;
+    // Input side (forward pass only), in_mode 1: the kernel's input tensor is the INPUT x of a BN+ReLU op whose
+    // output only this convolution reads.  The kernel derives mean / rstd from the per-tile sums the producer of x
+    // left (in_partials, [in_tiles][2][C]), applies y = relu(gamma*(x-mean)*rstd+beta) to the activation tile on
+    // its way to the tensor core (the padding ring stays zero), and stores y (in_y, needed by the backward pass)
+    // and the statistics (in_stats) as a by-product: the BN+ReLU needs no kernel of its own.
+    int in_mode = 0;
+    const float* in_partials = nullptr;
+    int in_tiles = 0;
+    long long in_rows = 0;
+    float in_eps = 0.f;
+    const float* in_gamma = nullptr;
+    const float* in_beta = nullptr;
+    float* in_stats = nullptr;
+    float* in_y = nullptr;
 };
+// Whether in_mode 1 applies to this convolution.
+bool conv_tc_can_fuse_bn_input(const ConvShape& s);
 // Number of pixel tiles (= partial-sum rows) of the forward / data-gradient launch, and whether the fusion applies.
 int conv_tc_tiles(const ConvShape& s, int pass);
 bool conv_tc_can_fuse_bn(const ConvShape& s, int pass);

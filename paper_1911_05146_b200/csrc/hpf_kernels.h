@@ -66,6 +66,8 @@ cudaError_t add_fwd(const float* a, const float* b, float* out, int64_t n, cudaS
 // dst (+)= src
 cudaError_t grad_accumulate(float* dst, const float* src, int64_t n, bool accumulate, cudaStream_t st, int64_t* n_launch);
 cudaError_t grad_average(const float* slots, float* out, int M, int64_t G, cudaStream_t st, int64_t* n_launch);
+// writes the device's nanosecond timer to *slot (one thread)
+cudaError_t stamp_time(unsigned long long* slot, cudaStream_t st, int64_t* n_launch);
 cudaError_t loss_average(const float* loss_slots, float* out, int M, cudaStream_t st, int64_t* n_launch);
 cudaError_t maxpool_fwd(const float* x, float* y, ConvShape s, cudaStream_t st, int64_t* n_launch);
 cudaError_t maxpool_bwd(const float* x, const float* dy, float* dx, bool accumulate, ConvShape s, cudaStream_t st,

@@ -84,7 +84,12 @@ struct hpf_model {
     std::vector<int> add_done_by;             // ADD -> the conv that computes it, or -1
     std::vector<int> bn_fwd_from, bn_bwd_from; // BN -> conv whose forward / data-gradient kernel leaves its per-tile sums, or -1
     std::vector<int> conv_fwd_bn, conv_dgrad_bn; // the inverse maps
-    int opt_fuse_bn = 1;       // bit 0: forward statistics, bit 1: backward sums (measured slower: the write-out is latency bound)
+    std::vector<int> bn_into, conv_in_bn;      // BN -> the convolution that applies it to its own input operand (no BN kernel), and the inverse
+    std::vector<int> bn_buf;                   // BN -> which of the stream's two partial-sum buffers carries its sums
+    std::vector<size_t> bn_part_bytes;         // per partition: size of one partial-sum buffer
+    int opt_cell_times = 0;    // record a device timestamp at the start and end of every (partition, micro-batch) cell
+    size_t cell_times_off = 0;
+    int opt_fuse_bn = 5;       // bit 0: forward statistics, bit 1: backward sums (measured slower), bit 2: BN+ReLU applied by the reading convolution
     std::vector<GradEdge> edge0;              // per op: contribution to src0
     std::vector<AccumAction> accums;
     std::vector<std::vector<MessagePlan>> msg_plan;   // per cut
@@ -127,6 +132,16 @@ struct hpf_model {
     float* act(int op, int m) const { return reinterpret_cast<float*>(ws + act_off[(size_t)m * n_ops + op]); }
     float* grad(int op, int m) const { return reinterpret_cast<float*>(ws + grad_off[(size_t)m * n_ops + op]); }
     float* stats(int op, int m) const { return reinterpret_cast<float*>(ws + stats_off[(size_t)m * n_ops + op]); }
+    unsigned long long* cell_time_slot(int phase, int p, int m) const
+    {
+        return reinterpret_cast<unsigned long long*>(ws + cell_times_off) + 2 * (((size_t)(phase == PH_BWD) * P + p) * M + m);
+    }
+    // per-tile partial sums of BN op `bn` left by the convolution kernel that produced its input
+    float* bn_partials(int bn) const
+    {
+        const int p = ops[bn].part;
+        return reinterpret_cast<float*>(ws + bn_scratch_off[p] + 256 + (size_t)bn_buf[bn] * bn_part_bytes[p]);
+    }
     int64_t numel(int op) const { const OpInfo& o = ops[op]; return (int64_t)b * o.H * o.W * o.C; }
     cudaStream_t stream_of(int p) const { return opt_single ? streams[0] : streams[p]; }
     DeviceStatus* status() const { return reinterpret_cast<DeviceStatus*>(ws + status_off); }
@@ -345,7 +360,9 @@ void build_kernel_plan(hpf_model* mdl)
     }
     mdl->bn_fwd_from.assign(n, -1); mdl->bn_bwd_from.assign(n, -1);
     mdl->conv_fwd_bn.assign(n, -1); mdl->conv_dgrad_bn.assign(n, -1);
+    mdl->bn_into.assign(n, -1); mdl->conv_in_bn.assign(n, -1); mdl->bn_buf.assign(n, 0);
     if (!mdl->opt_fuse_bn) return;
+    std::vector<int> n_fused(mdl->P, 0);
     for (int j = 0; j < n; ++j) {
         const OpInfo& bn = mdl->ops[j];
         if (bn.op.kind != HPF_OP_BNRELU || bn.C > 2048) continue;
@@ -358,7 +375,20 @@ void build_kernel_plan(hpf_model* mdl)
             bool adjacent = true;
             for (int k = prod + 1; k < j; ++k)
                 if (!(mdl->ops[k].op.kind == HPF_OP_ADD && mdl->add_done_by[k] >= 0)) adjacent = false;
-            if (adjacent) { mdl->bn_fwd_from[j] = prod; mdl->conv_fwd_bn[prod] = j; }
+            if (adjacent) {
+                mdl->bn_fwd_from[j] = prod; mdl->conv_fwd_bn[prod] = j;
+                // A convolution that applies BN j reads the sums while its own write-out already produces the next
+                // BN's: successive fused BNs of a stream alternate between two buffers.
+                mdl->bn_buf[j] = n_fused[bn.part]++ & 1;
+            }
+        }
+        // the BN+ReLU itself: applied by its only reader, the next op, a stride-1 tensor-core convolution
+        if ((mdl->opt_fuse_bn & 4) && mdl->bn_fwd_from[j] >= 0 && bn.consumers.size() == 1 && bn.consumers[0] == j + 1) {
+            const int i = j + 1;
+            if (mdl->ops[i].op.kind == HPF_OP_CONV && mdl->ops[i].op.src0 == j && mdl->use_tc[PASS_FWD][i] &&
+                mdl->ops[i].part == bn.part && conv_tc_can_fuse_bn_input(conv_shape_of(mdl, i))) {
+                mdl->bn_into[j] = i; mdl->conv_in_bn[i] = j;
+            }
         }
         // backward: the data-gradient kernel of the BN output's only reader
         if ((mdl->opt_fuse_bn & 2) && bn.consumers.size() == 1 && bn.consumers[0] == j + 1) {
@@ -386,8 +416,9 @@ void build_memory_plan(hpf_model* mdl)
     mdl->status_off = take(sizeof(DeviceStatus));
     mdl->bn_scratch_off.assign(P, 0);
     mdl->conv_scratch_off.assign(P, 0);
+    mdl->bn_part_bytes.assign(P, 0);
     for (int p = 0; p < P; ++p) {
-        size_t bn = 256;
+        size_t bn = 256, part = 0;
         for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i)
             if (mdl->ops[i].op.kind == HPF_OP_BNRELU) {
                 const OpInfo& o = mdl->ops[i];
@@ -396,10 +427,12 @@ void build_memory_plan(hpf_model* mdl)
                 for (int pass = PASS_FWD; pass <= PASS_DGRAD; ++pass) {
                     const int from = pass == PASS_FWD ? mdl->bn_fwd_from[i] : mdl->bn_bwd_from[i];
                     if (from < 0) continue;
-                    need = 256 + (size_t)conv_tc_tiles(conv_shape_of(mdl, from), pass) * 2 * o.C * sizeof(float);
-                    if (need > bn) bn = need;
+                    need = align_up((size_t)conv_tc_tiles(conv_shape_of(mdl, from), pass) * 2 * o.C * sizeof(float), 256);
+                    if (need > part) part = need;
                 }
             }
+        mdl->bn_part_bytes[p] = part;
+        if (256 + 2 * part > bn) bn = 256 + 2 * part;
         mdl->bn_scratch_off[p] = take(bn);
     }
     mdl->zero_hi = at;
@@ -415,6 +448,7 @@ void build_memory_plan(hpf_model* mdl)
             }
         mdl->conv_scratch_off[p] = take(cv);
     }
+    mdl->cell_times_off = take(sizeof(unsigned long long) * 2 * 2 * (size_t)P * M);
     mdl->loss_slots_off = take(sizeof(float) * M);
     mdl->loss_avg_off = take(sizeof(float));
     mdl->wprep_off = take(sizeof(float) * 4 * (size_t)((mdl->G + 3) / 4 * 4));   // w_hi | w_lo | wt_hi | wt_lo, parameter offsets
@@ -499,9 +533,10 @@ int forward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
         break;
     }
     case HPF_OP_BNRELU:
+        if (mdl->bn_into[i] >= 0) break;   // the convolution that reads this BN applies it (and stores `out` and the statistics)
         if (mdl->bn_fwd_from[i] >= 0)      // the producing convolution left the per-tile sums in the stream's scratch
             CU(bnrelu_fwd_fused(in0, mdl->params + o.w_off, mdl->params + o.b_off, q.eps, out, mdl->stats(i, m),
-                                reinterpret_cast<const float*>(mdl->ws + mdl->bn_scratch_off[p] + 256),
+                                mdl->bn_partials(i),
                                 conv_tc_tiles(conv_shape_of(mdl, mdl->bn_fwd_from[i]), PASS_FWD), (int64_t)mdl->b * o.H * o.W, o.C,
                                 st, &mdl->launches));
         else
@@ -621,10 +656,12 @@ int enqueue_phase(hpf_model* mdl, int phase)
                             CU(grad_accumulate(reinterpret_cast<float*>(mdl->ws + mdl->fmsg_off[p - 1][k * M + m]),
                                                mdl->act(mdl->live[p - 1][k], m), mdl->numel(mdl->live[p - 1][k]), false, st, &mdl->launches));
                 }
+                if (mdl->opt_cell_times) CU(stamp_time(mdl->cell_time_slot(PH_FWD, p, m), st, &mdl->launches));
                 for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i) {
                     int rc = forward_op(mdl, i, m, st, p);
                     if (rc) return rc;
                 }
+                if (mdl->opt_cell_times) CU(stamp_time(mdl->cell_time_slot(PH_FWD, p, m) + 1, st, &mdl->launches));
                 if (p < P - 1 && multi) CU(cudaEventRecord(mdl->ev_fwd[(size_t)p * M + m], st));          // send
             }
     } else if (phase == PH_BWD) {
@@ -643,10 +680,12 @@ int enqueue_phase(hpf_model* mdl, int phase)
                             if (mp.pending >= 0) CU(grad_accumulate(dst, mdl->grad(mp.pending, m), mdl->numel(mp.tensor), mp.from_buffer != 0, st, &mdl->launches));
                         }
                 }
+                if (mdl->opt_cell_times) CU(stamp_time(mdl->cell_time_slot(PH_BWD, p, m), st, &mdl->launches));
                 for (int i = mdl->part_hi[p] - 1; i >= mdl->part_lo[p]; --i) {
                     int rc = backward_op(mdl, i, m, st, p);
                     if (rc) return rc;
                 }
+                if (mdl->opt_cell_times) CU(stamp_time(mdl->cell_time_slot(PH_BWD, p, m) + 1, st, &mdl->launches));
                 if (p > 0 && multi) CU(cudaEventRecord(mdl->ev_bwd[(size_t)(p - 1) * M + m], st));       // send partial errors
             }
     }
@@ -784,7 +823,8 @@ int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
     case HPF_OPT_KEEP_MESSAGES: mdl->opt_messages = value != 0; break;
     case HPF_OPT_FUSE_ADD: mdl->opt_fuse_add = value != 0; break;
     case HPF_OPT_PDL: hpf::g_pdl_enabled = value != 0; break;
-    case HPF_OPT_FUSE_BN: if (value < 0 || value > 3) return fail(HPF_ERR_INVALID, "0..3"); mdl->opt_fuse_bn = value; break;
+    case HPF_OPT_FUSE_BN: if (value < 0 || value > 7) return fail(HPF_ERR_INVALID, "0..7"); mdl->opt_fuse_bn = value; break;
+    case HPF_OPT_CELL_TIMES: mdl->opt_cell_times = value != 0; break;
     case HPF_OPT_WGRAD_PASSES: if (value != 1 && value != 3) return fail(HPF_ERR_INVALID, "1 or 3 passes"); mdl->opt_wgrad_passes = value; break;
     default: return fail(HPF_ERR_INVALID, "unknown option");
     }
@@ -1019,9 +1059,22 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                         ConvBnFuse fuse;
                         if (mdl->conv_fwd_bn[i] >= 0) {
                             fuse.mode = 1;
-                            fuse.partials = reinterpret_cast<float*>(mdl->ws + mdl->bn_scratch_off[o.part] + 256);
+                            fuse.partials = mdl->bn_partials(mdl->conv_fwd_bn[i]);
                         }
-                        CU(conv_tc_prepare(pl, s, pass, passes, mdl->act(src, m), nullptr, wp + o.w_off, wp + G + o.w_off,
+                        const float* in = mdl->act(src, m);
+                        const int jb = mdl->conv_in_bn[i];
+                        if (jb >= 0) {
+                            const OpInfo& bn = mdl->ops[jb];
+                            in = mdl->act(bn.op.src0, m);          // the BN's input; its output is a by-product of this kernel
+                            fuse.in_mode = 1;
+                            fuse.in_partials = mdl->bn_partials(jb);
+                            fuse.in_tiles = conv_tc_tiles(conv_shape_of(mdl, mdl->bn_fwd_from[jb]), PASS_FWD);
+                            fuse.in_rows = (long long)mdl->b * bn.H * bn.W;
+                            fuse.in_eps = bn.op.eps;
+                            fuse.in_gamma = mdl->params + bn.w_off; fuse.in_beta = mdl->params + bn.b_off;
+                            fuse.in_stats = mdl->stats(jb, m); fuse.in_y = mdl->act(jb, m);
+                        }
+                        CU(conv_tc_prepare(pl, s, pass, passes, in, nullptr, wp + o.w_off, wp + G + o.w_off,
                                            mdl->act(i, m), residual, false, scratch, &fuse));
                     }
                     else if (pass == PASS_DGRAD) {
@@ -1157,6 +1210,19 @@ int hpf_loss_slots_ptr(const hpf_model* mdl, const float** d_ptr)
     if (!mdl || !d_ptr) return fail(HPF_ERR_INVALID, "null");
     if (mdl->state < ST_BOUND) return fail(HPF_ERR_STATE, "hpf_bind first");
     *d_ptr = reinterpret_cast<const float*>(mdl->ws + mdl->loss_slots_off);
+    return HPF_OK;
+}
+
+int hpf_cell_times(hpf_model* mdl, int32_t phase, int64_t* h_ns)
+{
+    if (!mdl || !h_ns) return fail(HPF_ERR_INVALID, "null");
+    if (phase != 0 && phase != 1) return fail(HPF_ERR_INVALID, "phase is 0 (forward) or 1 (backward)");
+    if (mdl->state < ST_FWD || (phase == 1 && mdl->state < ST_BWD)) return fail(HPF_ERR_STATE, "run the phase first");
+    if (!mdl->opt_cell_times) return fail(HPF_ERR_STATE, "HPF_OPT_CELL_TIMES is off");
+    int rc = hpf_synchronize(mdl, 0);
+    if (rc) return rc;
+    static_assert(sizeof(unsigned long long) == sizeof(int64_t), "timestamp width");
+    CU(cudaMemcpy(h_ns, mdl->cell_time_slot(phase ? PH_BWD : PH_FWD, 0, 0), sizeof(int64_t) * 2 * (size_t)mdl->P * mdl->M, cudaMemcpyDeviceToHost));
     return HPF_OK;
 }
 

@@ -471,6 +471,13 @@ grad_average_kernel(const float* __restrict__ slots, float* __restrict__ out, in
     }
 }
 
+__global__ void stamp_kernel(unsigned long long* slot)
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    *slot = t;
+}
+
 __global__ void loss_average_kernel(const float* __restrict__ loss_slots, float* __restrict__ out, int M)
 {
     if (threadIdx.x == 0 && blockIdx.x == 0) {
@@ -782,6 +789,13 @@ cudaError_t grad_average(const float* slots, float* out, int M, int64_t G, cudaS
     if (G % 4 == 0 && out16) grad_average_kernel<4><<<ew_blocks(G / 4), kThreads, 0, st>>>(slots, out, M, G, inv_m);
     else if (G % 2 == 0 && out16) grad_average_kernel<2><<<ew_blocks(G / 2), kThreads, 0, st>>>(slots, out, M, G, inv_m);
     else grad_average_kernel<1><<<ew_blocks(G), kThreads, 0, st>>>(slots, out, M, G, inv_m);
+    count(n_launch, 1);
+    return cudaGetLastError();
+}
+
+cudaError_t stamp_time(unsigned long long* slot, cudaStream_t st, int64_t* n_launch)
+{
+    stamp_kernel<<<1, 1, 0, st>>>(slot);
     count(n_launch, 1);
     return cudaGetLastError();
 }
