@@ -98,15 +98,13 @@ int hpf_model_destroy(hpf_model *model);
  *                          nothing but the average, so its rounding error (about 8e-4 relative with one pass) does not
  *                          compound with depth the way forward and data-gradient errors do; those always follow
  *                          HPF_OPT_CONV_PATH.
- *   HPF_OPT_FUSE_BN        bit 0 (default on): the per-channel sums of a BN's forward statistics are formed in the write-out
- *                          of the tensor-core convolution kernel that produces the BN's input, when both run back to
- *                          back on one stream; the BN forward is then one kernel.  bit 1 (default off: measured slower):
- *                          the same for the backward sums (dbeta, dgamma) in the data-gradient kernel that produces
- *                          the gradient of the BN's output.  bit 2 (default on; needs bit 0): a BN+ReLU whose output only the
- *                          next op reads, a stride-1 tensor-core convolution of the same partition, has no kernel of
- *                          its own: that convolution derives the statistics from the per-tile sums, applies the BN+ReLU
- *                          to its input tile on the way to the tensor core and stores the BN's output and statistics as
- *                          a by-product.  0: every BN runs its own reduction kernels.  Default 5.
+ *   HPF_OPT_FUSE_BN        bit 0: the per-channel sums of a BN's forward statistics are formed in the write-out of the
+ *                          tensor-core convolution kernel that produces the BN's input, when both run back to back on
+ *                          one stream; the BN forward is then one kernel.  bit 1 (needs bit 0): a BN+ReLU whose output
+ *                          only the next op reads, a stride-1 tensor-core convolution of the same partition, has no
+ *                          kernel of its own: that convolution derives the statistics from the per-tile sums, applies
+ *                          the BN+ReLU to its input tile on the way to the tensor core and stores the BN's output and
+ *                          statistics as a by-product.  0: every BN runs its own kernels.  Default 3.
  *   HPF_OPT_CELL_TIMES     1: a one-thread kernel stores the device's nanosecond timer at the start and at the end of
  *                          every (partition, micro-batch) cell of the forward and backward schedules (Section 5.3's
  *                          pipeline, as it really ran); read them with hpf_cell_times.  Default 0. */

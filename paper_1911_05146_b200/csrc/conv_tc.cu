@@ -180,8 +180,18 @@ inline uint32_t instr_desc(int n, bool a_mn_major, bool b_mn_major)
            ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
 }
 
-// Optional timeline of CTA (0,0) for latency studies: globaltimer stamps behind the status word (debug builds only).
-#ifdef HPF_TC_TIMELINE
+// Optional timelines for latency studies (debug builds only).  HPF_TC_TIMELINE=2: every CTA of the forward kernel
+// stamps its milestones in shared memory and adds the elapsed times to per-class totals (class = window size and
+// grid size), read back with hpf_debug_timeline.  Otherwise: globaltimer stamps of CTA (0,0) behind the status word.
+#if defined(HPF_TC_TIMELINE) && HPF_TC_TIMELINE == 2
+__device__ unsigned long long g_tl_acc[8][16];
+#define HPF_TL(slot)                                                                                      \
+    do {                                                                                                  \
+        unsigned long long t_;                                                                            \
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                            \
+        tl_s[(slot)] = t_;                                                                                \
+    } while (0)
+#elif defined(HPF_TC_TIMELINE)
 #define HPF_TL(slot)                                                                                      \
     do {                                                                                                  \
         if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {                                      \
@@ -224,24 +234,19 @@ struct FwdScalars {
     int zero_fill;               // > 1: the output pixel grid is strided, fill the rest of each patch with zeros
     int out_h, out_w;            // dense output extent (zero fill bounds)
     unsigned int a_bytes, b_bytes, stage_bytes, tx_bytes, tmem_cols, idesc, idesc2, stg_pitch;
-    // batch-norm reductions folded into the write-out (see ConvBnFuse): 0 none, 1 sums of the output,
-    // 2 sums of the masked gradient for the backward of the BN whose output this data gradient is
+    // batch-norm statistics folded into the write-out (see ConvBnFuse): 0 none, 1 sums of the output and its square
     int stat_mode;
     float* stat_partials;        // [tiles][2][c_out] per-tile partial sums
-    const float* bn_x;           // mode 2: the BN's input, same shape as the output
-    const float* bn_stats;       // mode 2: mean[c_out], rstd[c_out]
-    const float* bn_gamma;
-    const float* bn_beta;
+    unsigned int* stat_ticket;   // counts finished CTAs; zero between launches
+    float* stat_out;             // mean[c_out], rstd[c_out], written by the CTA that finishes last
+    float stat_eps;
+    double stat_inv_rows;        // 1 / (pixels the statistics run over)
     // BN+ReLU applied to the activation operand on its way to the tensor core (see ConvBnFuse::in_mode)
     int bn_in;
-    int bn_in_tiles;             // rows of bn_in_partials
     int in_w, in_h;              // extent of the input pixel grid (the padding mask)
-    float bn_in_eps;
-    double bn_in_inv_rows;       // 1 / (pixels the statistics run over)
-    const float* bn_in_partials; // [bn_in_tiles][2][c_in] per-tile sums of x and x*x
     const float* bn_in_gamma;
     const float* bn_in_beta;
-    float* bn_in_stats;          // mean[c_in], rstd[c_in], written by the first CTA
+    const float* bn_in_stats;    // mean[c_in], rstd[c_in] (left by the kernel that produced x)
     float* bn_in_y;              // relu(bn(x)), dense [N][in_h][in_w][c_in], written by the CTAs of the first channel slice
 };
 struct alignas(64) FwdParams {
@@ -295,6 +300,10 @@ __device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__flo
 __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_constant__ FwdParams gp)
 {
     __shared__ FwdScalars p;                 // scalar parameters, see load_scalars
+#if defined(HPF_TC_TIMELINE) && HPF_TC_TIMELINE == 2
+    __shared__ unsigned long long tl_s[16];
+    if (threadIdx.x < 16) tl_s[threadIdx.x] = 0;
+#endif
     pdl_launch_dependents();
     load_scalars(&p, &gp.s);
     __syncthreads();
@@ -413,44 +422,13 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
         bool ok = true;
         if (p.bn_in) {
             // ---- BN+ReLU on the way in: the tile holds the BN's input x; the operand is relu(gamma*xhat+beta) ----
-            // Statistics: every CTA adds the producer's per-tile sums in the same fixed order (fp64), so all CTAs
-            // hold identical mean / rstd; the first CTA stores them for the backward pass.
-            __shared__ double bn_red[256][4];
             __shared__ __align__(16) float bn_par[4][256];      // mean, rstd, gamma, beta per input channel
-            const int C = p.c_in, ncol4 = C >> 1;              // float4 columns of one tile's [2][C] sums (256 % ncol4 == 0)
-            {
-                const int col4 = tid % ncol4, ln = tid / ncol4, L = 256 / ncol4;
-                const float4* part = reinterpret_cast<const float4*>(p.bn_in_partials);
-                double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-#pragma unroll 4
-                for (int k = ln; k < p.bn_in_tiles; k += L) {
-                    const float4 v = __ldcg(part + (size_t)k * ncol4 + col4);
-                    a0 += (double)v.x; a1 += (double)v.y; a2 += (double)v.z; a3 += (double)v.w;
-                }
-                bn_red[tid][0] = a0; bn_red[tid][1] = a1; bn_red[tid][2] = a2; bn_red[tid][3] = a3;
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (tid < ncol4) {
-                    // rows tid, tid + ncol4, ... are read by this thread alone, so the total can go back into row tid
-                    double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
-                    for (int l = 0; l < L; ++l) {
-                        const double* r = bn_red[l * ncol4 + tid];
-                        t0 += r[0]; t1 += r[1]; t2 += r[2]; t3 += r[3];
-                    }
-                    bn_red[tid][0] = t0; bn_red[tid][1] = t1; bn_red[tid][2] = t2; bn_red[tid][3] = t3;
-                }
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                const double* tot = &bn_red[0][0];              // [2][C]: sums, then sums of squares
-                for (int c = tid; c < C; c += 256) {
-                    const double mean = tot[c] * p.bn_in_inv_rows;
-                    double var = tot[C + c] * p.bn_in_inv_rows - mean * mean;
-                    if (var < 0.0) var = 0.0;
-                    const float mu = (float)mean, rs = (float)(1.0 / sqrt(var + (double)p.bn_in_eps));
-                    bn_par[0][c] = mu; bn_par[1][c] = rs;
-                    bn_par[2][c] = __ldg(p.bn_in_gamma + c); bn_par[3][c] = __ldg(p.bn_in_beta + c);
-                    if (blockIdx.x == 0 && blockIdx.y == 0) { p.bn_in_stats[c] = mu; p.bn_in_stats[C + c] = rs; }
-                }
-                asm volatile("bar.sync 1, 256;" ::: "memory");
+            const int C = p.c_in;
+            if (tid < C) {
+                bn_par[0][tid] = __ldg(p.bn_in_stats + tid); bn_par[1][tid] = __ldg(p.bn_in_stats + C + tid);
+                bn_par[2][tid] = __ldg(p.bn_in_gamma + tid); bn_par[3][tid] = __ldg(p.bn_in_beta + tid);
             }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             // A thread owns one 16-byte column of the (swizzled) tile rows tid/f4row + j*(256/f4row): its four
             // channels within the K chunk are fixed, and so are the pixels of its rows.
             const int f4row = p.kchunk >> 2;                    // 4 or 8 float4 per tile row
@@ -541,13 +519,13 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
         mbar_wait(accum_bar, 0, &abort_flag);
         // every pipeline buffer is idle now (all MMAs completed, all copies landed): the tile is staged there
         // so that the write-out is coalesced (a TMEM lane is a pixel: thread-per-row stores would touch 32 lines each)
-        __shared__ long long row_off[kTileM];
+        __shared__ int row_off[kTileM];                // offset (floats) of the pixel's channel row in the output, or -1
         __shared__ int row_fill[kTileM];               // strided data gradient: which neighbours of the sample exist
         if (tid < kTileM) {
             const int wi = tid % p.box_w, hi = (tid / p.box_w) % p.box_h, ni = tid / (p.box_w * p.box_h);
             const int q = q0 + wi, pp = p0 + hi, n = n0 + ni;
             const bool valid = ni < p.box_n && q < p.Q && pp < p.P && n < p.N;
-            row_off[tid] = valid ? (n * p.os_n + pp * p.os_h + q * p.os_w + co0) : -1;
+            row_off[tid] = valid ? (int)(n * p.os_n + pp * p.os_h + q * p.os_w + co0) : -1;
             int fill = 0;                              // bit (dy*4 + dx) set: position (pp*s+dy, q*s+dx) gets zeros
             for (int dy = 0; dy < p.zero_fill; ++dy)
                 for (int dx = 0; dx < p.zero_fill; ++dx)
@@ -560,28 +538,26 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             tc_fence_after();
             if (tid == 0) HPF_TL(7);
             // TMEM lane = pixel within the tile.  Two warps share each group of 32 lanes (a warp reaches lanes
-            // 32*(warp%4) ..): they take alternate groups of 32 output channels.
+            // 32*(warp%4) ..): they take alternate groups of 16 output channels.
             const int row = (warp & 3) * 32 + lane;
             const int half = (warp - 2) >> 2;
             float* stg = reinterpret_cast<float*>(smem);
             const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-            for (int g0 = half * 32; g0 < p.n_chunk; g0 += 64) {
-                const int ncols = p.n_chunk - g0 < 32 ? p.n_chunk - g0 : 32;      // 16 or 32
-                float v[32];
+            for (int g0 = half * 16; g0 < p.n_chunk; g0 += 32) {
+                float v[16];
                 tmem_ld16_nowait(lane_addr + (uint32_t)g0, v);
-                if (ncols > 16) tmem_ld16_nowait(lane_addr + (uint32_t)(g0 + 16), v + 16);
-                tmem_ld_wait();
                 if (p.stacked) {
-                    float u[32];
+                    float u[16];
                     tmem_ld16_nowait(lane_addr + (uint32_t)(p.n_chunk + g0), u);
-                    if (ncols > 16) tmem_ld16_nowait(lane_addr + (uint32_t)(p.n_chunk + g0 + 16), u + 16);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) if (j < ncols) v[j] += u[j];
+                    for (int j = 0; j < 16; ++j) v[j] += u[j];
+                } else {
+                    tmem_ld_wait();
                 }
                 float4* dst = reinterpret_cast<float4*>(stg + (size_t)row * p.stg_pitch + g0);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) if (4 * j < ncols) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
             }
             if (tid == 0) HPF_TL(10);
             asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -598,17 +574,9 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             const long long dense_h = p.dense_h, dense_w = p.dense_w;
             const int stat_mode = p.stat_mode;
             float4 sa = make_float4(0.f, 0.f, 0.f, 0.f), sb = sa;
-            float4 bmu = sa, brs = sa, bg = sa, bb = sa;
-            if (stat_mode == 2) {
-                const int cch = co0 + 4 * (tid % c4n);             // this thread's channels (fixed: 256 % c4n == 0)
-                bmu = __ldg(reinterpret_cast<const float4*>(p.bn_stats + cch));
-                brs = __ldg(reinterpret_cast<const float4*>(p.bn_stats + p.c_out + cch));
-                bg = __ldg(reinterpret_cast<const float4*>(p.bn_gamma + cch));
-                bb = __ldg(reinterpret_cast<const float4*>(p.bn_beta + cch));
-            }
             for (int base = tid; base < total4; base += 1024) {
                 float4 o[4];
-                long long off[4];
+                int off[4];
                 int fill[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -617,7 +585,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     if (idx < total4) {
                         const int r = sh >= 0 ? (idx >> sh) : (idx / c4n);
                         const int c4 = idx - r * c4n;
-                        const long long ro = row_off[r];
+                        const int ro = row_off[r];
                         if (ro >= 0) {
                             off[u] = ro + 4 * c4;
                             fill[u] = row_fill[r];
@@ -635,30 +603,15 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     for (int u = 0; u < 4; ++u)
                         if (off[u] >= 0) { const float4 e = *reinterpret_cast<const float4*>(outp + off[u]); o[u].x += e.x; o[u].y += e.y; o[u].z += e.z; o[u].w += e.w; }
                 }
-                float4 xv4[4];
-                if (stat_mode == 2) {
-                    // all loads of the batch are issued before its first store: a load behind a store would wait for it
-#pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        if (off[u] >= 0) xv4[u] = __ldg(reinterpret_cast<const float4*>(p.bn_x + off[u]));
-                }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     if (off[u] < 0) continue;
                     float* optr = outp + off[u];
                     *reinterpret_cast<float4*>(optr) = o[u];
-                    if (stat_mode == 1) {
+                    if (stat_mode) {
                         sa.x += o[u].x; sa.y += o[u].y; sa.z += o[u].z; sa.w += o[u].w;
                         sb.x = fmaf(o[u].x, o[u].x, sb.x); sb.y = fmaf(o[u].y, o[u].y, sb.y);
                         sb.z = fmaf(o[u].z, o[u].z, sb.z); sb.w = fmaf(o[u].w, o[u].w, sb.w);
-                    } else if (stat_mode == 2) {
-                        // dz = dy * [z > 0] with z recomputed exactly as the BN forward computed it
-                        const float4 xv = xv4[u];
-                        float xh, dz;
-                        xh = (xv.x - bmu.x) * brs.x; dz = fmaf(bg.x, xh, bb.x) > 0.f ? o[u].x : 0.f; sa.x += dz; sb.x = fmaf(dz, xh, sb.x);
-                        xh = (xv.y - bmu.y) * brs.y; dz = fmaf(bg.y, xh, bb.y) > 0.f ? o[u].y : 0.f; sa.y += dz; sb.y = fmaf(dz, xh, sb.y);
-                        xh = (xv.z - bmu.z) * brs.z; dz = fmaf(bg.z, xh, bb.z) > 0.f ? o[u].z : 0.f; sa.z += dz; sb.z = fmaf(dz, xh, sb.z);
-                        xh = (xv.w - bmu.w) * brs.w; dz = fmaf(bg.w, xh, bb.w) > 0.f ? o[u].w : 0.f; sa.w += dz; sb.w = fmaf(dz, xh, sb.w);
                     }
                     if (fill[u]) {
                         // strided data gradient: the positions between the samples receive no contribution
@@ -682,6 +635,51 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     for (int t2 = g; t2 < 256; t2 += c4n) { const float4 v2 = red[2 * t2 + which]; acc.x += v2.x; acc.y += v2.y; acc.z += v2.z; acc.w += v2.w; }
                     float* dstp = p.stat_partials + ((size_t)blockIdx.x * 2 + which) * p.c_out + co0 + 4 * g;
                     *reinterpret_cast<float4*>(dstp) = acc;
+                    __threadfence();
+                }
+                // The CTA that finishes last turns the per-tile sums into mean and 1/sigma: tiles are added in a fixed
+                // order in fp64, so the result does not depend on which CTA that is.
+                __shared__ int is_last;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (tid == 0) {
+                    const unsigned int done_before = atomicAdd(p.stat_ticket, 1u);
+                    is_last = done_before == gridDim.x * gridDim.y - 1;
+                }
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (is_last) {
+                    __threadfence();
+                    const int C = p.c_out, ncol4 = C >> 1;          // float4 columns of one tile's [2][C] sums (256 % ncol4 == 0)
+                    const int n_tiles = gridDim.x;
+                    double (*bn_red)[4] = reinterpret_cast<double (*)[4]>(smem);
+                    const int col4 = tid % ncol4, ln = tid / ncol4, L = 256 / ncol4;
+                    const float4* part = reinterpret_cast<const float4*>(p.stat_partials);
+                    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+#pragma unroll 8
+                    for (int k = ln; k < n_tiles; k += L) {
+                        const float4 v = __ldcg(part + (size_t)k * ncol4 + col4);
+                        a0 += (double)v.x; a1 += (double)v.y; a2 += (double)v.z; a3 += (double)v.w;
+                    }
+                    bn_red[tid][0] = a0; bn_red[tid][1] = a1; bn_red[tid][2] = a2; bn_red[tid][3] = a3;
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                    if (tid < ncol4) {
+                        // rows tid, tid + ncol4, ... are read by this thread alone, so the total can go back into row tid
+                        double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
+                        for (int l = 0; l < L; ++l) {
+                            const double* r = bn_red[l * ncol4 + tid];
+                            t0 += r[0]; t1 += r[1]; t2 += r[2]; t3 += r[3];
+                        }
+                        bn_red[tid][0] = t0; bn_red[tid][1] = t1; bn_red[tid][2] = t2; bn_red[tid][3] = t3;
+                    }
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                    const double* tot = &bn_red[0][0];              // [2][C]: sums, then sums of squares
+                    if (tid < C) {
+                        const double mean = tot[tid] * p.stat_inv_rows;
+                        double var = tot[C + tid] * p.stat_inv_rows - mean * mean;
+                        if (var < 0.0) var = 0.0;
+                        p.stat_out[tid] = (float)mean;
+                        p.stat_out[C + tid] = (float)(1.0 / sqrt(var + (double)p.stat_eps));
+                    }
+                    if (tid == 0) *p.stat_ticket = 0u;
                 }
             }
         }
@@ -702,6 +700,15 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
     if (threadIdx.x == 0) HPF_TL(9);
+#if defined(HPF_TC_TIMELINE) && HPF_TC_TIMELINE == 2
+    __syncthreads();
+    if (threadIdx.x < 16) {
+        const int tiles = gridDim.x;
+        const int cls = (p.R == 3 ? 1 : 0) + 2 * (tiles >= 128 ? 0 : (tiles >= 32 ? 1 : 2)) + (p.bn_in ? 0 : 0);
+        if (threadIdx.x == 0) atomicAdd(&g_tl_acc[cls][0], 1ull);
+        else if (tl_s[threadIdx.x] > tl_s[0]) atomicAdd(&g_tl_acc[cls][threadIdx.x], tl_s[threadIdx.x] - tl_s[0]);
+    }
+#endif
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1280,7 +1287,8 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     FwdParams& P = L->p;
     memset(&P, 0, sizeof P);
     FwdScalars& p = P.s;
-    const int kchunk = chunk_of(v.c_in);
+    static const int dbg_kchunk = getenv("HPF_DBG_KCHUNK") ? atoi(getenv("HPF_DBG_KCHUNK")) : 0;
+    const int kchunk = dbg_kchunk == 16 ? 16 : chunk_of(v.c_in);
     const int n_chunk = v.c_out < 256 ? v.c_out : 256;
     {
         cuuint64_t dims[4] = {(cuuint64_t)v.c_in, (cuuint64_t)v.in_w, (cuuint64_t)v.in_h, (cuuint64_t)v.N};
@@ -1301,6 +1309,7 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
             if (e != cudaSuccess) return e;
         }
     }
+    if ((long long)v.N * v.os_n >= (1LL << 31)) return cudaErrorNotSupported;      // the write-out keeps 32-bit offsets
     p.out = out; p.extra = extra; p.accumulate = accumulate ? 1 : 0;
     p.os_n = v.os_n; p.os_h = v.os_h; p.os_w = v.os_w; p.dense_h = v.dense_h; p.dense_w = v.dense_w;
     p.box_w = b.w; p.box_h = b.h; p.box_n = b.n;
@@ -1317,7 +1326,8 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     p.tx_bytes = (unsigned int)b.rows * kchunk * 4 + parts * (unsigned int)n_chunk * kchunk * 4;
     int stages = (int)(kSmemBudget / p.stage_bytes);
     const int total = v.R * v.R * p.n_kchunks;
-    if (stages > kFwdMaxStages) stages = kFwdMaxStages;
+    static const int dbg_max_stages = getenv("HPF_DBG_MAX_STAGES") ? atoi(getenv("HPF_DBG_MAX_STAGES")) : kFwdMaxStages;
+    if (stages > dbg_max_stages) stages = dbg_max_stages;
     if (stages > total) stages = total;
     {
         static const int target = getenv("HPF_DBG_SMEM_TARGET") ? atoi(getenv("HPF_DBG_SMEM_TARGET")) : 0;
@@ -1330,14 +1340,14 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     p.stages = stages;
     if (fuse && fuse->mode) {
         if (256 % (n_chunk / 4)) return cudaErrorNotSupported;
-        p.stat_mode = fuse->mode; p.stat_partials = fuse->partials;
-        p.bn_x = fuse->bn_x; p.bn_stats = fuse->bn_stats; p.bn_gamma = fuse->bn_gamma; p.bn_beta = fuse->bn_beta;
+        if (fuse->mode != 1 || pass != PASS_FWD || !conv_tc_can_fuse_bn(s, pass) || fuse->rows < 1) return cudaErrorNotSupported;
+        p.stat_mode = 1; p.stat_partials = fuse->partials;
+        p.stat_ticket = fuse->ticket; p.stat_out = fuse->stats_out; p.stat_eps = fuse->eps; p.stat_inv_rows = 1.0 / (double)fuse->rows;
     }
     if (fuse && fuse->in_mode) {
-        if (pass != PASS_FWD || !conv_tc_can_fuse_bn_input(s) || fuse->in_tiles < 1 || fuse->in_rows < 1) return cudaErrorNotSupported;
-        p.bn_in = 1; p.bn_in_tiles = fuse->in_tiles; p.in_w = v.in_w; p.in_h = v.in_h; p.bn_in_eps = fuse->in_eps;
-        p.bn_in_inv_rows = 1.0 / (double)fuse->in_rows;
-        p.bn_in_partials = fuse->in_partials; p.bn_in_gamma = fuse->in_gamma; p.bn_in_beta = fuse->in_beta;
+        if (pass != PASS_FWD || !conv_tc_can_fuse_bn_input(s)) return cudaErrorNotSupported;
+        p.bn_in = 1; p.in_w = v.in_w; p.in_h = v.in_h;
+        p.bn_in_gamma = fuse->in_gamma; p.bn_in_beta = fuse->in_beta;
         p.bn_in_stats = fuse->in_stats; p.bn_in_y = fuse->in_y;
     }
     p.stacked = (passes == 3 && 2 * n_chunk <= 256) ? 1 : 0;
@@ -1394,3 +1404,16 @@ cudaError_t conv_weight_prep_single(const float* w, float* w_hi, float* w_lo, fl
 }
 
 }  // namespace hpf
+
+#if defined(HPF_TC_TIMELINE) && HPF_TC_TIMELINE == 2
+extern "C" int hpf_debug_timeline(unsigned long long* h_out, int reset)
+{
+    cudaDeviceSynchronize();
+    if (h_out && cudaMemcpyFromSymbol(h_out, hpf::g_tl_acc, sizeof(unsigned long long) * 8 * 16) != cudaSuccess) return -1;
+    if (reset) {
+        static unsigned long long zeros[8 * 16];
+        if (cudaMemcpyToSymbol(hpf::g_tl_acc, zeros, sizeof zeros) != cudaSuccess) return -1;
+    }
+    return 0;
+}
+#endif

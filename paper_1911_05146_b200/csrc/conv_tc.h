@@ -23,32 +23,26 @@ struct ConvTcPlan {
     alignas(64) unsigned char storage[896];
 };
 
-// Batch-norm reductions folded into the forward / data-gradient kernel's write-out.
-//   mode 1 (forward): per tile, per output channel, sum and sum of squares of what the kernel writes (the
-//          statistics of the BN that reads this tensor next);
-//   mode 2 (data gradient): this kernel writes dL/dy of a BN+ReLU output y; per tile and channel it also forms
-//          sum dz and sum dz*xhat (dz = dy*[z>0]) from the BN's input bn_x, its saved statistics and gamma/beta.
-// partials: [conv_tc_tiles(s, pass)][2][channels] floats, written in full by every launch.
+// Batch-norm work folded into the forward kernel.
+//   mode 1 (output side): the kernel's output is the input of a BN.  Per tile and output channel the write-out forms
+//   the sum and the sum of squares of what it stores (partials, [conv_tc_tiles(s, PASS_FWD)][2][channels] floats); the
+//   CTA that finishes last (ticket: one zeroed word, left zero) adds them in a fixed order and stores mean[C], rstd[C]
+//   of the `rows` pixels to stats_out.
+//   in_mode 1 (input side): the kernel's input tensor is the INPUT x of a BN+ReLU op whose output only this convolution
+//   reads, and in_stats holds that BN's mean / rstd.  The kernel applies y = relu(gamma*(x-mean)*rstd+beta) to the
+//   activation tile on its way to the tensor core (the padding ring stays zero) and stores y (in_y, needed by the
+//   backward pass) as a by-product: the BN+ReLU needs no kernel of its own.
 struct ConvBnFuse {
     int mode = 0;
     float* partials = nullptr;
-    const float* bn_x = nullptr;
-    const float* bn_stats = nullptr;
-    const float* bn_gamma = nullptr;
-    const float* bn_beta = nullptr;
-    // Input side (forward pass only), in_mode 1: the kernel's input tensor is the INPUT x of a BN+ReLU op whose
-    // output only this convolution reads.  The kernel derives mean / rstd from the per-tile sums the producer of x
-    // left (in_partials, [in_tiles][2][C]), applies y = relu(gamma*(x-mean)*rstd+beta) to the activation tile on
-    // its way to the tensor core (the padding ring stays zero), and stores y (in_y, needed by the backward pass)
-    // and the statistics (in_stats) as a by-product: the BN+ReLU needs no kernel of its own.
+    unsigned int* ticket = nullptr;
+    float* stats_out = nullptr;
+    long long rows = 0;
+    float eps = 0.f;
     int in_mode = 0;
-    const float* in_partials = nullptr;
-    int in_tiles = 0;
-    long long in_rows = 0;
-    float in_eps = 0.f;
     const float* in_gamma = nullptr;
     const float* in_beta = nullptr;
-    float* in_stats = nullptr;
+    const float* in_stats = nullptr;
     float* in_y = nullptr;
 };
 // Whether in_mode 1 applies to this convolution.

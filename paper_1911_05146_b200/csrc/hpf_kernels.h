@@ -55,13 +55,9 @@ cudaError_t bnrelu_fwd(const float* x, const float* gamma, const float* beta, fl
 cudaError_t bnrelu_bwd(const float* x, const float* dy, const float* gamma, const float* beta, const float* stats,
                        float* dx, const float* addend, bool accumulate, float* dgamma, float* dbeta,
                        int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch);
-// The same with the per-channel sums supplied as per-tile partials [n_tiles][2][C] by the producing convolution
-// kernel (forward: sum x, sum x^2; backward: sum dz, sum dz*xhat): one kernel, no separate reduction.
-cudaError_t bnrelu_fwd_fused(const float* x, const float* gamma, const float* beta, float eps, float* y, float* stats,
-                             const float* partials, int n_tiles, int64_t rows, int C, cudaStream_t st, int64_t* n_launch);
-cudaError_t bnrelu_bwd_fused(const float* x, const float* dy, const float* gamma, const float* beta, const float* stats,
-                             float* dx, const float* addend, bool accumulate, float* dgamma, float* dbeta,
-                             const float* partials, int n_tiles, int64_t rows, int C, cudaStream_t st, int64_t* n_launch);
+// The forward's second half alone: the statistics (mean[C], rstd[C]) were left by the convolution kernel that produced x.
+cudaError_t bnrelu_fwd_apply(const float* x, const float* gamma, const float* beta, const float* stats, float* y,
+                             int64_t rows, int C, cudaStream_t st, int64_t* n_launch);
 cudaError_t add_fwd(const float* a, const float* b, float* out, int64_t n, cudaStream_t st, int64_t* n_launch);
 // dst (+)= src
 cudaError_t grad_accumulate(float* dst, const float* src, int64_t n, bool accumulate, cudaStream_t st, int64_t* n_launch);

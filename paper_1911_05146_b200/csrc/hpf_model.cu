@@ -82,14 +82,12 @@ struct hpf_model {
     std::vector<int> grad_alias;              // tensor -> ADD op whose gradient buffer it shares, or -1
     std::vector<int> fused_into;              // conv -> residual ADD computed in its epilogue (its own output is not stored), or -1
     std::vector<int> add_done_by;             // ADD -> the conv that computes it, or -1
-    std::vector<int> bn_fwd_from, bn_bwd_from; // BN -> conv whose forward / data-gradient kernel leaves its per-tile sums, or -1
-    std::vector<int> conv_fwd_bn, conv_dgrad_bn; // the inverse maps
+    std::vector<int> bn_fwd_from;              // BN -> conv whose forward kernel leaves the per-tile sums of the BN's input, or -1
+    std::vector<int> conv_fwd_bn;              // the inverse map
     std::vector<int> bn_into, conv_in_bn;      // BN -> the convolution that applies it to its own input operand (no BN kernel), and the inverse
-    std::vector<int> bn_buf;                   // BN -> which of the stream's two partial-sum buffers carries its sums
-    std::vector<size_t> bn_part_bytes;         // per partition: size of one partial-sum buffer
     int opt_cell_times = 0;    // record a device timestamp at the start and end of every (partition, micro-batch) cell
     size_t cell_times_off = 0;
-    int opt_fuse_bn = 5;       // bit 0: forward statistics, bit 1: backward sums (measured slower), bit 2: BN+ReLU applied by the reading convolution
+    int opt_fuse_bn = 3;       // bit 0: BN statistics in the producing convolution's write-out, bit 1: BN+ReLU applied by the reading convolution
     std::vector<GradEdge> edge0;              // per op: contribution to src0
     std::vector<AccumAction> accums;
     std::vector<std::vector<MessagePlan>> msg_plan;   // per cut
@@ -135,12 +133,6 @@ struct hpf_model {
     unsigned long long* cell_time_slot(int phase, int p, int m) const
     {
         return reinterpret_cast<unsigned long long*>(ws + cell_times_off) + 2 * (((size_t)(phase == PH_BWD) * P + p) * M + m);
-    }
-    // per-tile partial sums of BN op `bn` left by the convolution kernel that produced its input
-    float* bn_partials(int bn) const
-    {
-        const int p = ops[bn].part;
-        return reinterpret_cast<float*>(ws + bn_scratch_off[p] + 256 + (size_t)bn_buf[bn] * bn_part_bytes[p]);
     }
     int64_t numel(int op) const { const OpInfo& o = ops[op]; return (int64_t)b * o.H * o.W * o.C; }
     cudaStream_t stream_of(int p) const { return opt_single ? streams[0] : streams[p]; }
@@ -358,11 +350,10 @@ void build_kernel_plan(hpf_model* mdl)
         mdl->use_tc[pass].assign(n, 0);
         for (int i = 0; i < n; ++i) mdl->use_tc[pass][i] = op_uses_tc(mdl, i, pass) ? 1 : 0;
     }
-    mdl->bn_fwd_from.assign(n, -1); mdl->bn_bwd_from.assign(n, -1);
-    mdl->conv_fwd_bn.assign(n, -1); mdl->conv_dgrad_bn.assign(n, -1);
-    mdl->bn_into.assign(n, -1); mdl->conv_in_bn.assign(n, -1); mdl->bn_buf.assign(n, 0);
+    mdl->bn_fwd_from.assign(n, -1);
+    mdl->conv_fwd_bn.assign(n, -1);
+    mdl->bn_into.assign(n, -1); mdl->conv_in_bn.assign(n, -1);
     if (!mdl->opt_fuse_bn) return;
-    std::vector<int> n_fused(mdl->P, 0);
     for (int j = 0; j < n; ++j) {
         const OpInfo& bn = mdl->ops[j];
         if (bn.op.kind != HPF_OP_BNRELU || bn.C > 2048) continue;
@@ -375,27 +366,14 @@ void build_kernel_plan(hpf_model* mdl)
             bool adjacent = true;
             for (int k = prod + 1; k < j; ++k)
                 if (!(mdl->ops[k].op.kind == HPF_OP_ADD && mdl->add_done_by[k] >= 0)) adjacent = false;
-            if (adjacent) {
-                mdl->bn_fwd_from[j] = prod; mdl->conv_fwd_bn[prod] = j;
-                // A convolution that applies BN j reads the sums while its own write-out already produces the next
-                // BN's: successive fused BNs of a stream alternate between two buffers.
-                mdl->bn_buf[j] = n_fused[bn.part]++ & 1;
-            }
+            if (adjacent) { mdl->bn_fwd_from[j] = prod; mdl->conv_fwd_bn[prod] = j; }
         }
         // the BN+ReLU itself: applied by its only reader, the next op, a stride-1 tensor-core convolution
-        if ((mdl->opt_fuse_bn & 4) && mdl->bn_fwd_from[j] >= 0 && bn.consumers.size() == 1 && bn.consumers[0] == j + 1) {
+        if ((mdl->opt_fuse_bn & 2) && mdl->bn_fwd_from[j] >= 0 && bn.consumers.size() == 1 && bn.consumers[0] == j + 1) {
             const int i = j + 1;
             if (mdl->ops[i].op.kind == HPF_OP_CONV && mdl->ops[i].op.src0 == j && mdl->use_tc[PASS_FWD][i] &&
                 mdl->ops[i].part == bn.part && conv_tc_can_fuse_bn_input(conv_shape_of(mdl, i))) {
                 mdl->bn_into[j] = i; mdl->conv_in_bn[i] = j;
-            }
-        }
-        // backward: the data-gradient kernel of the BN output's only reader
-        if ((mdl->opt_fuse_bn & 2) && bn.consumers.size() == 1 && bn.consumers[0] == j + 1) {
-            const int i = j + 1;
-            if (mdl->ops[i].op.kind == HPF_OP_CONV && mdl->ops[i].op.src0 == j && mdl->use_tc[PASS_DGRAD][i] &&
-                mdl->ops[i].part == bn.part && conv_tc_can_fuse_bn(conv_shape_of(mdl, i), PASS_DGRAD)) {
-                mdl->bn_bwd_from[j] = i; mdl->conv_dgrad_bn[i] = j;
             }
         }
     }
@@ -416,23 +394,19 @@ void build_memory_plan(hpf_model* mdl)
     mdl->status_off = take(sizeof(DeviceStatus));
     mdl->bn_scratch_off.assign(P, 0);
     mdl->conv_scratch_off.assign(P, 0);
-    mdl->bn_part_bytes.assign(P, 0);
     for (int p = 0; p < P; ++p) {
-        size_t bn = 256, part = 0;
+        size_t bn = 256;
         for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i)
             if (mdl->ops[i].op.kind == HPF_OP_BNRELU) {
                 const OpInfo& o = mdl->ops[i];
                 size_t need = bn_scratch_bytes((int64_t)mdl->b * o.H * o.W, o.C);
                 if (need > bn) bn = need;
-                for (int pass = PASS_FWD; pass <= PASS_DGRAD; ++pass) {
-                    const int from = pass == PASS_FWD ? mdl->bn_fwd_from[i] : mdl->bn_bwd_from[i];
-                    if (from < 0) continue;
-                    need = align_up((size_t)conv_tc_tiles(conv_shape_of(mdl, from), pass) * 2 * o.C * sizeof(float), 256);
-                    if (need > part) part = need;
+                const int from = mdl->bn_fwd_from[i];
+                if (from >= 0) {
+                    need = 256 + (size_t)conv_tc_tiles(conv_shape_of(mdl, from), PASS_FWD) * 2 * o.C * sizeof(float);
+                    if (need > bn) bn = need;
                 }
             }
-        mdl->bn_part_bytes[p] = part;
-        if (256 + 2 * part > bn) bn = 256 + 2 * part;
         mdl->bn_scratch_off[p] = take(bn);
     }
     mdl->zero_hi = at;
@@ -534,11 +508,9 @@ int forward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
     }
     case HPF_OP_BNRELU:
         if (mdl->bn_into[i] >= 0) break;   // the convolution that reads this BN applies it (and stores `out` and the statistics)
-        if (mdl->bn_fwd_from[i] >= 0)      // the producing convolution left the per-tile sums in the stream's scratch
-            CU(bnrelu_fwd_fused(in0, mdl->params + o.w_off, mdl->params + o.b_off, q.eps, out, mdl->stats(i, m),
-                                mdl->bn_partials(i),
-                                conv_tc_tiles(conv_shape_of(mdl, mdl->bn_fwd_from[i]), PASS_FWD), (int64_t)mdl->b * o.H * o.W, o.C,
-                                st, &mdl->launches));
+        if (mdl->bn_fwd_from[i] >= 0)      // the producing convolution left mean and 1/sigma
+            CU(bnrelu_fwd_apply(in0, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), out,
+                                (int64_t)mdl->b * o.H * o.W, o.C, st, &mdl->launches));
         else
             CU(bnrelu_fwd(in0, mdl->params + o.w_off, mdl->params + o.b_off, q.eps, out, mdl->stats(i, m),
                           (int64_t)mdl->b * o.H * o.W, o.C, mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
@@ -598,16 +570,9 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
         break;
     }
     case HPF_OP_BNRELU:
-        if (mdl->bn_bwd_from[i] >= 0)      // the data-gradient kernel that produced dout left the per-tile sums
-            CU(bnrelu_bwd_fused(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m),
-                                addend, e.accumulate != 0, slot + o.w_off, slot + o.b_off,
-                                reinterpret_cast<const float*>(mdl->ws + mdl->bn_scratch_off[p] + 256),
-                                conv_tc_tiles(conv_shape_of(mdl, mdl->bn_bwd_from[i]), PASS_DGRAD), (int64_t)mdl->b * o.H * o.W,
-                                o.C, st, &mdl->launches));
-        else
-            CU(bnrelu_bwd(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m), addend,
-                          e.accumulate != 0, slot + o.w_off, slot + o.b_off, (int64_t)mdl->b * o.H * o.W, o.C,
-                          mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
+        CU(bnrelu_bwd(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m), addend,
+                      e.accumulate != 0, slot + o.w_off, slot + o.b_off, (int64_t)mdl->b * o.H * o.W, o.C,
+                      mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
         break;
     case HPF_OP_ADD:
         break;   // its contributions are aliases, on-the-fly addends, or the explicit accumulations above
@@ -823,7 +788,7 @@ int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
     case HPF_OPT_KEEP_MESSAGES: mdl->opt_messages = value != 0; break;
     case HPF_OPT_FUSE_ADD: mdl->opt_fuse_add = value != 0; break;
     case HPF_OPT_PDL: hpf::g_pdl_enabled = value != 0; break;
-    case HPF_OPT_FUSE_BN: if (value < 0 || value > 7) return fail(HPF_ERR_INVALID, "0..7"); mdl->opt_fuse_bn = value; break;
+    case HPF_OPT_FUSE_BN: if (value < 0 || value > 3) return fail(HPF_ERR_INVALID, "0..3"); mdl->opt_fuse_bn = value; break;
     case HPF_OPT_CELL_TIMES: mdl->opt_cell_times = value != 0; break;
     case HPF_OPT_WGRAD_PASSES: if (value != 1 && value != 3) return fail(HPF_ERR_INVALID, "1 or 3 passes"); mdl->opt_wgrad_passes = value; break;
     default: return fail(HPF_ERR_INVALID, "unknown option");
@@ -1058,8 +1023,14 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                         }
                         ConvBnFuse fuse;
                         if (mdl->conv_fwd_bn[i] >= 0) {
+                            const int jn = mdl->conv_fwd_bn[i];
+                            const OpInfo& bn = mdl->ops[jn];
                             fuse.mode = 1;
-                            fuse.partials = mdl->bn_partials(mdl->conv_fwd_bn[i]);
+                            fuse.ticket = reinterpret_cast<unsigned int*>(mdl->ws + mdl->bn_scratch_off[o.part]);
+                            fuse.partials = reinterpret_cast<float*>(mdl->ws + mdl->bn_scratch_off[o.part] + 256);
+                            fuse.stats_out = mdl->stats(jn, m);
+                            fuse.rows = (long long)mdl->b * bn.H * bn.W;
+                            fuse.eps = bn.op.eps;
                         }
                         const float* in = mdl->act(src, m);
                         const int jb = mdl->conv_in_bn[i];
@@ -1067,10 +1038,6 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                             const OpInfo& bn = mdl->ops[jb];
                             in = mdl->act(bn.op.src0, m);          // the BN's input; its output is a by-product of this kernel
                             fuse.in_mode = 1;
-                            fuse.in_partials = mdl->bn_partials(jb);
-                            fuse.in_tiles = conv_tc_tiles(conv_shape_of(mdl, mdl->bn_fwd_from[jb]), PASS_FWD);
-                            fuse.in_rows = (long long)mdl->b * bn.H * bn.W;
-                            fuse.in_eps = bn.op.eps;
                             fuse.in_gamma = mdl->params + bn.w_off; fuse.in_beta = mdl->params + bn.b_off;
                             fuse.in_stats = mdl->stats(jb, m); fuse.in_y = mdl->act(jb, m);
                         }
@@ -1078,20 +1045,8 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                                            mdl->act(i, m), residual, false, scratch, &fuse));
                     }
                     else if (pass == PASS_DGRAD) {
-                        ConvBnFuse fuse;
-                        const int j = mdl->conv_dgrad_bn[i];
-                        if (j >= 0) {
-                            const OpInfo& bn = mdl->ops[j];
-                            fuse.mode = 2;
-                            fuse.partials = reinterpret_cast<float*>(mdl->ws + mdl->bn_scratch_off[o.part] + 256);
-                            fuse.bn_x = mdl->act(bn.op.src0, m);
-                            fuse.bn_stats = mdl->stats(j, m);
-                            fuse.bn_gamma = mdl->params + bn.w_off;
-                            fuse.bn_beta = mdl->params + bn.b_off;
-                        }
                         CU(conv_tc_prepare(pl, s, pass, passes, mdl->grad(i, m), nullptr, wp + 2 * G + o.w_off, wp + 3 * G + o.w_off,
-                                           mdl->grad(src, m), ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch,
-                                           &fuse));
+                                           mdl->grad(src, m), ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch));
                     }
                     else
                         CU(conv_tc_prepare(pl, s, pass, mdl->opt_conv_path == 2 ? 1 : mdl->opt_wgrad_passes, mdl->grad(i, m), mdl->act(src, m), nullptr, nullptr,

@@ -293,114 +293,6 @@ bn_apply_bwd_kernel(const float4* __restrict__ x, const float4* __restrict__ dy,
     }
 }
 
-// BN+ReLU forward / backward when the per-channel sums already exist as per-tile partials written by the
-// producing convolution kernel (partials[tile][0][C] and partials[tile][1][C]).  Every block first adds the
-// partials of its own channels (thread (lane, column group) takes tiles lane, lane+rl, ... ascending in fp64, the
-// lanes are then added ascending: the same fixed order in every block), then streams its rows.
-//   forward:  sums are sum x and sum x^2          -> mean, rstd (block 0 stores them for the backward pass)
-//   backward: sums are sum dz and sum dz*xhat     -> dbeta, dgamma (block 0 stores them) and the dx coefficients
-template <bool BWD, bool ADDEND, bool ACCUM>
-__global__ void __launch_bounds__(kBnThreads)
-bn_apply_fused_kernel(const float4* __restrict__ x, const float4* __restrict__ dy, const float* __restrict__ gamma,
-                      const float* __restrict__ beta, float* __restrict__ stats, const float* __restrict__ partials,
-                      int n_tiles, float eps, float4* __restrict__ out, const float4* __restrict__ addend,
-                      float* __restrict__ dgamma, float* __restrict__ dbeta, int64_t rows, int C, int cgt, int rl,
-                      int64_t rows_per_blk)
-{
-    __shared__ double shd[kBnThreads][8];
-    pdl_launch_dependents();
-    pdl_wait();
-    const int t = threadIdx.x, cg_total = C / 4;
-    const int my_rl = t / cgt, my_cg = t % cgt;
-    double acc[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
-    if (my_rl < rl && my_cg < cg_total) {
-#pragma unroll 2
-        for (int k = my_rl; k < n_tiles; k += rl) {
-            const float4 va = __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 0) * C) + my_cg);
-            const float4 vb = __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 1) * C) + my_cg);
-            acc[0] += (double)va.x; acc[1] += (double)va.y; acc[2] += (double)va.z; acc[3] += (double)va.w;
-            acc[4] += (double)vb.x; acc[5] += (double)vb.y; acc[6] += (double)vb.z; acc[7] += (double)vb.w;
-        }
-    }
-#pragma unroll
-    for (int j = 0; j < 8; ++j) shd[t][j] = acc[j];
-    __syncthreads();
-    double fin = 0.0;
-    const bool owner = t < cgt * 8;                 // one thread per (column group, component)
-    if (owner) {
-        const int cgl = t >> 3, comp = t & 7;
-        for (int l = 0; l < rl; ++l) fin += shd[l * cgt + cgl][comp];
-    }
-    __syncthreads();
-    if (owner) shd[t >> 3][t & 7] = fin;            // cgt * 8 <= kBnThreads * 8 / rl: rows 0..cgt-1 hold the totals
-    __syncthreads();
-    if (my_rl >= rl || my_cg >= cg_total) return;
-    const double inv_rows = 1.0 / (double)rows;
-    float4 c0, c1;       // forward: mean, rstd; backward: dbeta/rows, dgamma/rows
-    {
-        double a4[4], b4[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) { a4[e] = shd[my_cg][e]; b4[e] = shd[my_cg][4 + e]; }
-        if (BWD) {
-            c0 = make_float4((float)(a4[0] * inv_rows), (float)(a4[1] * inv_rows), (float)(a4[2] * inv_rows), (float)(a4[3] * inv_rows));
-            c1 = make_float4((float)(b4[0] * inv_rows), (float)(b4[1] * inv_rows), (float)(b4[2] * inv_rows), (float)(b4[3] * inv_rows));
-            if (blockIdx.x == 0 && my_rl == 0) {
-                // scalar stores: a gradient slot starts at m*G floats, which need not be 16-byte aligned
-#pragma unroll
-                for (int e = 0; e < 4; ++e) { dbeta[4 * my_cg + e] = (float)a4[e]; dgamma[4 * my_cg + e] = (float)b4[e]; }
-            }
-        } else {
-            float m_[4], r_[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const double mean = a4[e] * inv_rows;
-                double var = b4[e] * inv_rows - mean * mean;
-                if (var < 0.0) var = 0.0;
-                m_[e] = (float)mean; r_[e] = (float)(1.0 / sqrt(var + (double)eps));
-            }
-            c0 = make_float4(m_[0], m_[1], m_[2], m_[3]);
-            c1 = make_float4(r_[0], r_[1], r_[2], r_[3]);
-            if (blockIdx.x == 0 && my_rl == 0) {
-                reinterpret_cast<float4*>(stats)[my_cg] = c0;
-                reinterpret_cast<float4*>(stats + C)[my_cg] = c1;
-            }
-        }
-    }
-    const int64_t r0 = (int64_t)blockIdx.x * rows_per_blk;
-    int64_t r1 = r0 + rows_per_blk;
-    if (r1 > rows) r1 = rows;
-    const float4 g = __ldg(reinterpret_cast<const float4*>(gamma) + my_cg);
-    const float4 b = __ldg(reinterpret_cast<const float4*>(beta) + my_cg);
-    float4 mu = c0, rs = c1;
-    if (BWD) {
-        mu = __ldg(reinterpret_cast<const float4*>(stats) + my_cg);
-        rs = __ldg(reinterpret_cast<const float4*>(stats + C) + my_cg);
-    }
-    const int64_t base = (r0 + my_rl) * cg_total + my_cg, step = (int64_t)rl * cg_total;
-    const int n = (int)((r1 - r0 - my_rl + rl - 1) / rl);
-#pragma unroll 4
-    for (int k = 0; k < n; ++k) {
-        const int64_t i = base + k * step;
-        const float4 v = __ldg(x + i);
-        float4 o;
-        if (BWD) {
-            const float4 d = __ldg(dy + i);
-            o.x = bn_dx1(v.x, d.x, mu.x, rs.x, g.x, b.x, c0.x, c1.x);
-            o.y = bn_dx1(v.y, d.y, mu.y, rs.y, g.y, b.y, c0.y, c1.y);
-            o.z = bn_dx1(v.z, d.z, mu.z, rs.z, g.z, b.z, c0.z, c1.z);
-            o.w = bn_dx1(v.w, d.w, mu.w, rs.w, g.w, b.w, c0.w, c1.w);
-            if (ADDEND) { const float4 e = __ldg(addend + i); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
-            if (ACCUM) { const float4 e = out[i]; o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
-        } else {
-            o.x = fmaxf(bn_z(bn_xhat(v.x, mu.x, rs.x), g.x, b.x), 0.f);
-            o.y = fmaxf(bn_z(bn_xhat(v.y, mu.y, rs.y), g.y, b.y), 0.f);
-            o.z = fmaxf(bn_z(bn_xhat(v.z, mu.z, rs.z), g.z, b.z), 0.f);
-            o.w = fmaxf(bn_z(bn_xhat(v.w, mu.w, rs.w), g.w, b.w), 0.f);
-        }
-        out[i] = o;
-    }
-}
-
 int ew_blocks(int64_t n_items)
 {
     int64_t nb = ceil_div64(n_items, kThreads);
@@ -737,32 +629,12 @@ cudaError_t bnrelu_bwd(const float* x, const float* dy, const float* gamma, cons
     return cudaGetLastError();
 }
 
-cudaError_t bnrelu_fwd_fused(const float* x, const float* gamma, const float* beta, float eps, float* y, float* stats,
-                             const float* partials, int n_tiles, int64_t rows, int C, cudaStream_t st, int64_t* n_launch)
+cudaError_t bnrelu_fwd_apply(const float* x, const float* gamma, const float* beta, const float* stats, float* y,
+                             int64_t rows, int C, cudaStream_t st, int64_t* n_launch)
 {
     const BnPlan p = bn_plan(rows, C);
-    if (p.passes != 1) return cudaErrorNotSupported;
-    launch_pdl(bn_apply_fused_kernel<false, false, false>, p.nblk_apply, kBnThreads, 0, st, reinterpret_cast<const float4*>(x),
-               (const float4*)nullptr, gamma, beta, stats, partials, n_tiles, eps, reinterpret_cast<float4*>(y), (const float4*)nullptr,
-               (float*)nullptr, (float*)nullptr, rows, C, p.cgt, p.rl, p.rows_per_blk_apply);
-    count(n_launch, 1);
-    return cudaGetLastError();
-}
-
-cudaError_t bnrelu_bwd_fused(const float* x, const float* dy, const float* gamma, const float* beta, const float* stats,
-                             float* dx, const float* addend, bool accumulate, float* dgamma, float* dbeta,
-                             const float* partials, int n_tiles, int64_t rows, int C, cudaStream_t st, int64_t* n_launch)
-{
-    const BnPlan p = bn_plan(rows, C);
-    if (p.passes != 1) return cudaErrorNotSupported;
-#define HPF_BN_FUSED(A, B) launch_pdl(bn_apply_fused_kernel<true, A, B>, p.nblk_apply, kBnThreads, 0, st, reinterpret_cast<const float4*>(x), \
-        reinterpret_cast<const float4*>(dy), gamma, beta, const_cast<float*>(stats), partials, n_tiles, 0.f, reinterpret_cast<float4*>(dx),   \
-        reinterpret_cast<const float4*>(addend), dgamma, dbeta, rows, C, p.cgt, p.rl, p.rows_per_blk_apply)
-    if (addend && accumulate) HPF_BN_FUSED(true, true);
-    else if (addend) HPF_BN_FUSED(true, false);
-    else if (accumulate) HPF_BN_FUSED(false, true);
-    else HPF_BN_FUSED(false, false);
-#undef HPF_BN_FUSED
+    launch_pdl(bn_apply_fwd_kernel, p.nblk_apply, kBnThreads, 0, st, reinterpret_cast<const float4*>(x), gamma, beta, stats,
+               reinterpret_cast<float4*>(y), rows, C, p.cgt, p.rl, p.passes, p.rows_per_blk_apply);
     count(n_launch, 1);
     return cudaGetLastError();
 }

@@ -66,7 +66,7 @@ def test_config1_resnet11(conv_path, graph):
                {hpf.OPT_CONV_PATH: conv_path, hpf.OPT_GRAPH: graph})
 
 
-@pytest.mark.parametrize("fuse_bn,pdl,wgrad_passes", [(0, 1, 1), (3, 0, 3), (2, 0, 3)])
+@pytest.mark.parametrize("fuse_bn,pdl,wgrad_passes", [(0, 1, 1), (1, 0, 3), (3, 0, 3)])
 def test_config1_without_the_fusions(fuse_bn, pdl, wgrad_passes):
     """The BN reductions in their own kernels or both folded into the convolutions, plain stream-ordered
     launches, three-pass weight gradient."""
