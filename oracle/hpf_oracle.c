@@ -492,6 +492,21 @@ void ora_grad_average(const double *g_slots, int32_t M, int64_t G, double *out)
     }
 }
 
+/* Parameter update that closes the training step (Section 5.3: after the gradient allreduce every
+ * replica applies the averaged gradients, optimizer.apply_gradients()).  Stochastic gradient descent
+ * with momentum in the Keras form, the framework the paper builds on:
+ *     g' = g + weight_decay * theta;   v <- momentum * v - lr * g';   theta <- theta + v.
+ * momentum = 0 and weight_decay = 0 give plain gradient descent theta <- theta - lr * g. */
+void ora_sgd_momentum(double *theta, double *v, const double *g, int64_t G, double lr, double momentum,
+                      double weight_decay)
+{
+    for (int64_t j = 0; j < G; ++j) {
+        const double gj = g[j] + weight_decay * theta[j];
+        v[j] = momentum * v[j] - lr * gj;
+        theta[j] = theta[j] + v[j];
+    }
+}
+
 /* ------------------------------------------------------------------ */
 /* One op applied to whole tensors (used by both sweeps below)         */
 /* ------------------------------------------------------------------ */

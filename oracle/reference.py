@@ -206,6 +206,16 @@ def grad_average(g_slots):
     return out
 
 
+def sgd_momentum(theta, v, g, lr, momentum=0.0, weight_decay=0.0):
+    """Returns (theta', v') of one Keras-form SGD step (Section 5.3, apply_gradients); inputs are not modified."""
+    theta = np.array(theta, dtype=np.float64); v = np.array(v, dtype=np.float64)
+    g = np.ascontiguousarray(g, dtype=np.float64)
+    P = C.POINTER(C.c_double)
+    lib().ora_sgd_momentum(theta.ctypes.data_as(P), v.ctypes.data_as(P), g.ctypes.data_as(P), C.c_int64(theta.size),
+                           C.c_double(lr), C.c_double(momentum), C.c_double(weight_decay))
+    return theta, v
+
+
 # ---------------------------------------------------------------- sweeps
 def _ptr_array(bufs):
     arr = (C.POINTER(C.c_double) * len(bufs))()

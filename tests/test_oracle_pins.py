@@ -414,3 +414,42 @@ def test_supplied_relu_decisions_window():
     # partition-by-partition execution honours the decisions identically
     rp = ora.microbatch(ops, hwc, theta, x, labels, cuts=[4, 13], decisions=flipped, tau=tau)
     assert np.array_equal(rp["g"], r["g"]) and rp["decisions_used"] == 1
+
+
+# ---------------------------------------------------------------- parameter update (Section 5.3, apply_gradients)
+def test_sgd_momentum_closed_forms():
+    """Constant gradient g, no decay: v_k = -lr*g*(1-mu^k)/(1-mu) and theta_k = theta_0 + sum_i v_i (geometric sums);
+    mu = 0 is plain descent; with decay and mu = 0 on a zero gradient theta shrinks by (1 - lr*wd) per step."""
+    rng = np.random.default_rng(7)
+    G, lr, mu = 37, 0.1, 0.9
+    theta0, g = rng.standard_normal(G), rng.standard_normal(G)
+    theta, v = theta0.copy(), np.zeros(G)
+    for k in range(1, 6):
+        theta, v = ora.sgd_momentum(theta, v, g, lr, mu)
+        vk = -lr * g * (1 - mu ** k) / (1 - mu)
+        sum_v = -lr * g * (k - mu * (1 - mu ** k) / (1 - mu)) / (1 - mu)
+        np.testing.assert_allclose(v, vk, rtol=1e-13, atol=1e-15)
+        np.testing.assert_allclose(theta, theta0 + sum_v, rtol=1e-13, atol=1e-15)
+    t1, v1 = ora.sgd_momentum(theta0, np.zeros(G), g, lr)
+    np.testing.assert_allclose(t1, theta0 - lr * g, rtol=1e-15)
+    np.testing.assert_allclose(v1, -lr * g, rtol=1e-15)
+    t, v = theta0.copy(), np.zeros(G)
+    for _ in range(4):
+        t, v = ora.sgd_momentum(t, v, np.zeros(G), lr, 0.0, 0.5)
+    np.testing.assert_allclose(t, theta0 * (1 - lr * 0.5) ** 4, rtol=1e-14)
+    # sign: a step along -g lowers a quadratic 0.5*|theta|^2 whose gradient is theta
+    t2, _ = ora.sgd_momentum(theta0, np.zeros(G), theta0, 0.3)
+    assert np.sum(t2 ** 2) < np.sum(theta0 ** 2)
+    # the inputs are not modified
+    assert np.array_equal(g, g.copy()) and not np.shares_memory(t1, theta0)
+
+
+def test_sgd_step_lowers_the_loss_of_a_tiny_net():
+    """Descent property on the real objective: for a small enough rate, L(theta - lr*g) < L(theta)."""
+    ops, hwc = wl.resnet_v2_cifar(1, (4, 8, 16), 3), (8, 8, 3)
+    x, labels = wl.draw_inputs(4, hwc, 3)
+    theta = wl.draw_params(ops, bn_jitter=0.2)
+    r0 = ora.step(ops, hwc, theta, x, labels, 2)
+    theta1, _ = ora.sgd_momentum(theta, np.zeros(theta.size), r0["g_avg"], 0.05)
+    r1 = ora.step(ops, hwc, theta1, x, labels, 2)
+    assert r1["loss"] < r0["loss"]
