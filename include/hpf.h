@@ -160,6 +160,14 @@ int hpf_forward(hpf_model *model, const float *d_x, const int32_t *d_labels);
 int hpf_backward(hpf_model *model);
 /* d_grad_avg = (sum over m ascending of slot m) / M  (Section 5.3: gradients accumulated/averaged). */
 int hpf_grad_average(hpf_model *model);
+/* The gradient average fused with the parameter update that closes the training step (Section 5.3: the averaged
+ * gradients are applied, optimizer.apply_gradients()).  SGD with momentum in the Keras form:
+ *     gbar = (sum_m g_m)/M;  g' = gbar + weight_decay*theta;  v <- momentum*v - lr*g';  theta <- theta + v.
+ * Reads the bound gradient slots, writes gbar to the bound d_grad_avg and updates the bound d_params and d_velocity
+ * (device, G floats, caller-owned, zero before the first step) in place, in one kernel enqueued behind the backward
+ * phase.  Needs hpf_backward (HPF_ERR_STATE otherwise); use it INSTEAD of hpf_grad_average.  Hyper-parameters must
+ * be >= 0 (HPF_ERR_INVALID). */
+int hpf_sgd_momentum_step(hpf_model *model, float *d_velocity, float lr, float momentum, float weight_decay);
 /* Waits for the forward work; *h_loss = (1/M) sum_m L_m. */
 int hpf_loss(hpf_model *model, float *h_loss);
 /* The whole step from HOST buffers (pinned memory recommended): copies h_x / h_labels to the device,
@@ -237,6 +245,9 @@ int hpf_bnrelu_fwd_static(const float *d_x, const float *d_gamma, const float *d
 int hpf_static_scratch_bytes(size_t *bytes);
 /* out[j] = (sum_{m ascending} slots[m][j]) / M */
 int hpf_grad_average_flat(const float *d_slots, float *d_out, int32_t M, int64_t G, void *stream);
+/* The same update on caller buffers: d_slots [M][G]; d_grad_avg [G] or NULL; d_params, d_velocity [G] updated in place. */
+int hpf_sgd_momentum_flat(const float *d_slots, float *d_grad_avg, float *d_params, float *d_velocity, int32_t M, int64_t G,
+                          float lr, float momentum, float weight_decay, void *stream);
 
 const char *hpf_strerror(int status);
 /* Text of the most recent failure on the calling thread (CUDA error string and call site). */

@@ -53,6 +53,8 @@ _SIGNATURES = {
     "hpf_tensor_ptr": [_vp, _i32, _i32, _i32, C.POINTER(_vp), _pi32],
     "hpf_message_ptr": [_vp, _i32, _i32, _i32, _i32, C.POINTER(_vp)],
     "hpf_loss_slots_ptr": [_vp, C.POINTER(_vp)],
+    "hpf_sgd_momentum_step": [_vp, _vp, _f32, _f32, _f32],
+    "hpf_sgd_momentum_flat": [_vp, _vp, _vp, _vp, _i32, _i64, _f32, _f32, _f32, _vp],
     "hpf_launch_count": [_vp, _pi64],
     "hpf_cell_times": [_vp, _i32, _pi64],
     "hpf_conv_path_counts": [_vp, _pi64, _pi64],
@@ -215,6 +217,9 @@ class Model:
     def grad_average(self):
         _check(lib().hpf_grad_average(self._h))
 
+    def sgd_momentum_step(self, velocity, lr, momentum=0.0, weight_decay=0.0):
+        _check(lib().hpf_sgd_momentum_step(self._h, _ptr(velocity), lr, momentum, weight_decay))
+
     def loss(self):
         v = _f32(); _check(lib().hpf_loss(self._h, C.byref(v))); return v.value
 
@@ -286,6 +291,11 @@ def bnrelu_bwd(x, dy, gamma, beta, stats, dx, addend, accumulate, dgamma, dbeta,
 
 def grad_average_flat(slots, out, M, G, stream=None):
     _check(lib().hpf_grad_average_flat(_ptr(slots), _ptr(out), M, G, _stream(stream)))
+
+
+def sgd_momentum_flat(slots, grad_avg, params, velocity, M, G, lr, momentum=0.0, weight_decay=0.0, stream=None):
+    _check(lib().hpf_sgd_momentum_flat(_ptr(slots), _ptr(grad_avg) if grad_avg is not None else None, _ptr(params), _ptr(velocity),
+                                       M, G, lr, momentum, weight_decay, _stream(stream)))
 
 
 def bnrelu_fwd_static(x, gamma, beta, eps, y, stats, rows, Cc, stream=None):

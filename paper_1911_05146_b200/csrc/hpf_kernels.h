@@ -62,6 +62,9 @@ cudaError_t add_fwd(const float* a, const float* b, float* out, int64_t n, cudaS
 // dst (+)= src
 cudaError_t grad_accumulate(float* dst, const float* src, int64_t n, bool accumulate, cudaStream_t st, int64_t* n_launch);
 cudaError_t grad_average(const float* slots, float* out, int M, int64_t G, cudaStream_t st, int64_t* n_launch);
+// gbar = average of the M slots (stored to gavg unless null); v <- mu*v - lr*(gbar + wd*theta); theta <- theta + v
+cudaError_t sgd_momentum(const float* slots, float* gavg, float* theta, float* vel, int M, int64_t G, float lr, float mu,
+                         float wd, cudaStream_t st, int64_t* n_launch);
 // writes the device's nanosecond timer to *slot (one thread)
 cudaError_t stamp_time(unsigned long long* slot, cudaStream_t st, int64_t* n_launch);
 cudaError_t loss_average(const float* loss_slots, float* out, int M, cudaStream_t st, int64_t* n_launch);

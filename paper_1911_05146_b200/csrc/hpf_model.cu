@@ -1087,6 +1087,17 @@ int hpf_grad_average(hpf_model* mdl)
     return run_phase(mdl, PH_AVG);
 }
 
+int hpf_sgd_momentum_step(hpf_model* mdl, float* d_velocity, float lr, float momentum, float weight_decay)
+{
+    if (!mdl || !d_velocity) return fail(HPF_ERR_INVALID, "null argument");
+    if (mdl->state != ST_BWD) return fail(HPF_ERR_STATE, "hpf_sgd_momentum_step needs hpf_backward");
+    if (!(lr >= 0.f) || !(momentum >= 0.f) || !(weight_decay >= 0.f)) return fail(HPF_ERR_INVALID, "negative or NaN hyper-parameter");
+    // stream 0 carries the tail of the backward phase: the update is ordered behind every gradient
+    CU(sgd_momentum(mdl->gslots, mdl->gavg, mdl->params, d_velocity, mdl->M, mdl->G, lr, momentum, weight_decay,
+                    mdl->streams[0], &mdl->launches));
+    return HPF_OK;
+}
+
 int hpf_loss(hpf_model* mdl, float* h_loss)
 {
     if (!mdl || !h_loss) return fail(HPF_ERR_INVALID, "null argument");
@@ -1311,6 +1322,14 @@ int hpf_bnrelu_bwd(const float* d_x, const float* d_dy, const float* d_gamma, co
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     CU(cudaMemsetAsync(d_scratch, 0, 256, st));
     CU(bnrelu_bwd(d_x, d_dy, d_gamma, d_beta, d_stats, d_dx, d_addend, accumulate != 0, d_dgamma, d_dbeta, rows, C, d_scratch, st, nullptr));
+    return HPF_OK;
+}
+
+int hpf_sgd_momentum_flat(const float* d_slots, float* d_grad_avg, float* d_params, float* d_velocity, int32_t M, int64_t G,
+                          float lr, float momentum, float weight_decay, void* stream)
+{
+    if (!d_slots || !d_params || !d_velocity || M < 1 || G < 1) return fail(HPF_ERR_INVALID, "bad argument");
+    CU(sgd_momentum(d_slots, d_grad_avg, d_params, d_velocity, M, G, lr, momentum, weight_decay, reinterpret_cast<cudaStream_t>(stream), nullptr));
     return HPF_OK;
 }
 

@@ -29,7 +29,9 @@ __device__ __forceinline__ float bn_z(float xh, float g, float b) { return fmaf(
 // a thread keeps its column group for the whole kernel, so per-channel coefficients live in registers and no
 // index arithmetic runs per element.
 constexpr int kBnThreads = 512;
-constexpr int kBnMaxBlocks = 128;        // bounds the partials the last block has to combine
+constexpr int kBnMaxBlocks = 128;        // bounds the partials the last block has to combine (micro-batch sized tensors)
+constexpr int kBnMaxBlocksLarge = 296;   // tensors beyond L2-resident sizes need more loads in flight: two blocks per SM
+constexpr int64_t kBnLargeElems = 2 << 20;
 
 struct BnPlan {
     int cg_total;        // float4 column groups = C/4
@@ -51,7 +53,8 @@ BnPlan bn_plan(int64_t rows, int C)
     p.passes = (p.cg_total + p.cgt - 1) / p.cgt;
     int64_t nb = rows / ((int64_t)p.rl * 8);
     if (nb < 1) nb = 1;
-    if (nb > kBnMaxBlocks) nb = kBnMaxBlocks;
+    const int cap = rows * C > kBnLargeElems ? kBnMaxBlocksLarge : kBnMaxBlocks;
+    if (nb > cap) nb = cap;
     p.rows_per_blk = ceil_div64(rows, nb);
     p.nblk = (int)ceil_div64(rows, p.rows_per_blk);
     int64_t na = rows / ((int64_t)p.rl * 4);
@@ -363,6 +366,48 @@ grad_average_kernel(const float* __restrict__ slots, float* __restrict__ out, in
     }
 }
 
+// Gradient average fused with the parameter update (Section 5.3: averaged gradients, then apply_gradients):
+//   gbar = (sum_m g_m) / M (ascending m);  g' = gbar + wd * theta;  v <- mu * v - lr * g';  theta <- theta + v.
+// One pass over the flat buffers: reads M slots + theta + v, writes gbar (optional) + theta + v.
+template <int VEC>
+__global__ void __launch_bounds__(kThreads)
+sgd_momentum_kernel(const float* __restrict__ slots, float* __restrict__ gavg, float* __restrict__ theta,
+                    float* __restrict__ vel, int M, int64_t G, float inv_m, float lr, float mu, float wd)
+{
+    const int64_t nv = G / VEC;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nv; i += stride) {
+        float s[VEC], th[VEC], v[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) s[e] = 0.f;
+#pragma unroll 8
+        for (int m = 0; m < M; ++m) {
+            const float* src = slots + (int64_t)m * G + i * VEC;
+            if (VEC == 4) { const float4 q = __ldcs(reinterpret_cast<const float4*>(src)); s[0] += q.x; s[1 % VEC] += q.y; s[2 % VEC] += q.z; s[3 % VEC] += q.w; }
+            else s[0] += __ldcs(src);
+        }
+        if (VEC == 4) {
+            const float4 a = *reinterpret_cast<const float4*>(theta + i * 4), b = *reinterpret_cast<const float4*>(vel + i * 4);
+            th[0] = a.x; th[1 % VEC] = a.y; th[2 % VEC] = a.z; th[3 % VEC] = a.w; v[0] = b.x; v[1 % VEC] = b.y; v[2 % VEC] = b.z; v[3 % VEC] = b.w;
+        } else { th[0] = theta[i]; v[0] = vel[i]; }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            s[e] *= inv_m;
+            const float g = fmaf(wd, th[e], s[e]);
+            v[e] = fmaf(mu, v[e], -lr * g);
+            th[e] += v[e];
+        }
+        if (VEC == 4) {
+            if (gavg) *reinterpret_cast<float4*>(gavg + i * 4) = make_float4(s[0], s[1 % VEC], s[2 % VEC], s[3 % VEC]);
+            *reinterpret_cast<float4*>(theta + i * 4) = make_float4(th[0], th[1 % VEC], th[2 % VEC], th[3 % VEC]);
+            *reinterpret_cast<float4*>(vel + i * 4) = make_float4(v[0], v[1 % VEC], v[2 % VEC], v[3 % VEC]);
+        } else {
+            if (gavg) gavg[i] = s[0];
+            theta[i] = th[0]; vel[i] = v[0];
+        }
+    }
+}
+
 __global__ void stamp_kernel(unsigned long long* slot)
 {
     unsigned long long t;
@@ -661,6 +706,18 @@ cudaError_t grad_average(const float* slots, float* out, int M, int64_t G, cudaS
     if (G % 4 == 0 && out16) grad_average_kernel<4><<<ew_blocks(G / 4), kThreads, 0, st>>>(slots, out, M, G, inv_m);
     else if (G % 2 == 0 && out16) grad_average_kernel<2><<<ew_blocks(G / 2), kThreads, 0, st>>>(slots, out, M, G, inv_m);
     else grad_average_kernel<1><<<ew_blocks(G), kThreads, 0, st>>>(slots, out, M, G, inv_m);
+    count(n_launch, 1);
+    return cudaGetLastError();
+}
+
+cudaError_t sgd_momentum(const float* slots, float* gavg, float* theta, float* vel, int M, int64_t G, float lr, float mu,
+                         float wd, cudaStream_t st, int64_t* n_launch)
+{
+    const float inv_m = 1.f / (float)M;
+    const uintptr_t all = reinterpret_cast<uintptr_t>(slots) | reinterpret_cast<uintptr_t>(gavg) | reinterpret_cast<uintptr_t>(theta) |
+                          reinterpret_cast<uintptr_t>(vel);
+    if (G % 4 == 0 && (all & 15u) == 0) sgd_momentum_kernel<4><<<ew_blocks(G / 4), kThreads, 0, st>>>(slots, gavg, theta, vel, M, G, inv_m, lr, mu, wd);
+    else sgd_momentum_kernel<1><<<ew_blocks(G), kThreads, 0, st>>>(slots, gavg, theta, vel, M, G, inv_m, lr, mu, wd);
     count(n_launch, 1);
     return cudaGetLastError();
 }

@@ -134,3 +134,28 @@ def test_grad_average_flat(M, G):
         acc += slots[m]
     assert np.array_equal(out.cpu().numpy(), acc * np.float32(1.0 / M))      # fixed ascending order, bit-exact
     assert rel_l2(out.cpu().numpy(), ora.grad_average(slots)) <= 1e-6
+
+
+@pytest.mark.parametrize("M,G", [(1, 7), (8, 4096 * 33 + 2), (4, 1 << 20)])
+@pytest.mark.parametrize("mu,wd", [(0.0, 0.0), (0.9, 1e-4)])
+def test_sgd_momentum_flat(M, G, mu, wd):
+    """Average + parameter update in one kernel (Section 5.3, apply_gradients) against the fp64 oracle, two steps."""
+    rng = np.random.Generator(np.random.PCG64(M * 10 + G % 97))
+    theta = rng.standard_normal(G).astype(np.float32)
+    vel = np.zeros(G, dtype=np.float32)
+    d_theta, d_vel, d_avg = _dev(theta), _dev(vel), torch.empty(G, device=DEV)
+    th_ref, v_ref = theta.astype(np.float64), np.zeros(G)
+    for step in range(2):
+        slots = rng.standard_normal((M, G)).astype(np.float32)
+        hpf.sgd_momentum_flat(_dev(slots), d_avg, d_theta, d_vel, M, G, 0.05, mu, wd)
+        torch.cuda.synchronize()
+        gbar = ora.grad_average(slots)
+        th_ref, v_ref = ora.sgd_momentum(th_ref, v_ref, gbar, 0.05, mu, wd)
+        assert rel_l2(d_avg.cpu().numpy(), gbar) <= 1e-6
+        assert rel_l2(d_theta.cpu().numpy(), th_ref) <= 1e-6
+        assert rel_l2(d_vel.cpu().numpy(), v_ref) <= 1e-5
+    # gbar may be omitted
+    before = d_theta.clone()
+    hpf.sgd_momentum_flat(_dev(np.zeros((M, G), dtype=np.float32)), None, d_theta, torch.zeros(G, device=DEV), M, G, 0.05, 0.0, 0.0)
+    torch.cuda.synchronize()
+    assert torch.equal(before, d_theta)          # zero gradient, no decay, no velocity: nothing moves

@@ -188,3 +188,34 @@ def test_state_machine_on_a_bound_model():
         m2.bind(bd.params, bd.slots, bd.avg, small, bd.streams)
     assert e.value.status == -4
     assert bd.model.launch_count() > 0
+
+
+def test_training_steps_follow_the_oracle_and_lower_the_loss():
+    """Forward + backward + (average and SGD-momentum update), several steps on one batch: the parameters follow the
+    oracle's trajectory and the loss falls (the step of Section 5.3 closed by apply_gradients)."""
+    c = wl.config("r11")
+    ops, hwc, B, M, cuts = c["ops"], c["in_hwc"], c["B"], c["M"], c["cuts"]
+    x, labels = wl.draw_inputs(B, hwc, 10)
+    theta = wl.draw_params(ops, bn_jitter=0.1)
+    bd = Bound(ops, hwc, B, M, cuts, theta)
+    bd.upload(x, labels)
+    vel = torch.zeros(bd.G, device=bd.dev)
+    lr, mu, wd = 0.05, 0.9, 1e-4
+    th_ref, v_ref = theta.astype(np.float64), np.zeros(theta.size)
+    losses = []
+    with pytest.raises(hpf.HpfError):
+        bd.model.sgd_momentum_step(vel, lr, mu, wd)          # no backward yet
+    for step in range(4):
+        bd.model.forward(bd.x, bd.labels)
+        bd.model.backward()
+        bd.model.sgd_momentum_step(vel, lr, mu, wd)
+        losses.append(bd.model.loss())
+        bd.model.synchronize(60000)
+        r = ora.step(ops, hwc, th_ref, x, labels, M)
+        assert abs(losses[-1] - r["loss"]) <= 5e-3 * abs(r["loss"]), (step, losses[-1], r["loss"])
+        th_ref, v_ref = ora.sgd_momentum(th_ref, v_ref, r["g_avg"], lr, mu, wd)
+        # trajectories drift apart through the ReLU decisions both sides take on their own, so the bound is loose
+        assert rel_l2(bd.params.cpu().numpy(), th_ref) <= 2e-3, (step, rel_l2(bd.params.cpu().numpy(), th_ref))
+    assert losses[-1] < losses[0], losses
+    with pytest.raises(hpf.HpfError):
+        bd.model.sgd_momentum_step(vel, -1.0, mu, wd)
