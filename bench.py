@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the partitioned, micro-batch pipelined training step on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload r1001|r110|r11|r152] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload r1001|r110|r11|r152|r1001k] [--impl reference]
 
 One step = forward + backward + gradient average of the whole batch (all partitions, all
 micro-batches).  Prints ONE JSON line.  N > 1 (under torchrun) runs N independent replicas, one per
@@ -28,7 +28,10 @@ UNIT = "images/s"
 NAMES = {"r1001": "ResNet-1001 v2 (n=111, widths 16/32/64 x4), 32x32x3, batch 128, 8 partitions x 8 micro-batches",
          "r110": "ResNet-110 v2 (n=12), 32x32x3, batch 128, 4 partitions x 4 micro-batches",
          "r11": "ResNet-11 v2 (n=1), 32x32x3, batch 8, 2 partitions x 2 micro-batches",
-         "r152": "ResNet-152 v2 ImageNet layout, 224x224x3, batch 64, 4 partitions x 4 micro-batches"}
+         "r152": "ResNet-152 v2 ImageNet layout, 224x224x3, batch 64, 4 partitions x 4 micro-batches",
+         "r1001k": "ResNet-1001 v2 with the Keras example's widths (16/64/128 -> 64/128/256, 30.25 M parameters), 32x32x3, batch 128, "
+                   "8 partitions x 8 micro-batches",
+         "r20k": "ResNet-20 v2 with the Keras example's widths, 32x32x3, batch 16, 2 partitions x 2 micro-batches"}
 
 
 def peaks():

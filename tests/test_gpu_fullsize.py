@@ -54,3 +54,13 @@ def test_config3_resnet110_batch128():
 
 def test_config4_resnet1001_batch128():
     _fullsize("r1001", sample_m=[7])
+
+
+def test_keras_width_variant_short_net():
+    """The Keras example's widths (bottleneck 16/64/128, outputs 64/128/256: the ~30 M-parameter ResNet-1001 of the
+    paper's evaluation) at depth 20: every micro-batch against the oracle."""
+    _fullsize("r20k", sample_m=[0, 1])
+
+
+def test_keras_width_variant_resnet1001_batch128():
+    _fullsize("r1001k", sample_m=[3])

@@ -38,6 +38,25 @@ def test_depth_and_counts_of_resnet1001():
     assert ora.param_layout(ops)[4] == G == 10327706
 
 
+def test_keras_width_variant_has_the_parameter_count_the_paper_quotes():
+    """With the Keras example's chaining rule (a stage's bottleneck width = the previous stage's output channels:
+    16/64/128 -> 64/128/256) the 1001-layer net has the ~30 M parameters the paper states; closed form, independent
+    of the op loop."""
+    n = 111
+    ops = wl.config("r1001k")["ops"]
+    def block(c_t, w, co, first):
+        return c_t * w + 9 * w * w + w * co + (c_t * co if first else 0) + 2 * (c_t + w + w)
+    G = 3 * 9 * 16
+    c_t = 16
+    for w, co in ((16, 64), (64, 128), (128, 256)):
+        G += block(c_t, w, co, True) + (n - 1) * block(co, w, co, False)
+        c_t = co
+    G += 2 * 256 + 256 * 10 + 10
+    assert ora.param_layout(ops)[4] == G == 30251290
+    assert round(G / 1e6) == int(_facts()["resnet1001_params_millions"])
+    assert len(ops) == 21 * n + 6
+
+
 def test_param_layout_is_dense_and_ordered():
     ops = wl.resnet_v2_imagenet(blocks=(1, 1), widths=(4, 8), n_classes=7)
     w_off, w_cnt, b_off, b_cnt, G = ora.param_layout(ops)

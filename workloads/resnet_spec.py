@@ -13,8 +13,10 @@ Op = namedtuple("Op", "kind src0 src1 c_in c_out ksize stride pad eps")
 EPS = 1e-5
 
 
-def _bottleneck_stages(ops, t, c_t, widths, blocks, first_stride):
+def _bottleneck_stages(ops, t, c_t, widths, blocks, first_stride, outs=None):
+    """widths = bottleneck channels per stage; outs = block output channels per stage (default 4 x width)."""
     for si, (w, nb) in enumerate(zip(widths, blocks)):
+        co = 4 * w if outs is None else outs[si]
         for bi in range(nb):
             s = first_stride[si] if bi == 0 else 1
             ops.append(Op(BNRELU, t, -1, c_t, c_t, 0, 1, 0, EPS)); a1 = len(ops) - 1
@@ -22,19 +24,23 @@ def _bottleneck_stages(ops, t, c_t, widths, blocks, first_stride):
             ops.append(Op(BNRELU, c1, -1, w, w, 0, 1, 0, EPS)); a2 = len(ops) - 1
             ops.append(Op(CONV, a2, -1, w, w, 3, 1, 1, 0.0)); c2 = len(ops) - 1
             ops.append(Op(BNRELU, c2, -1, w, w, 0, 1, 0, EPS)); a3 = len(ops) - 1
-            ops.append(Op(CONV, a3, -1, w, 4 * w, 1, 1, 0, 0.0)); c3 = len(ops) - 1
+            ops.append(Op(CONV, a3, -1, w, co, 1, 1, 0, 0.0)); c3 = len(ops) - 1
             short = t
             if bi == 0:
-                ops.append(Op(CONV, t, -1, c_t, 4 * w, 1, s, 0, 0.0)); short = len(ops) - 1
-            ops.append(Op(ADD, c3, short, 4 * w, 4 * w, 0, 1, 0, 0.0)); t = len(ops) - 1
-            c_t = 4 * w
+                ops.append(Op(CONV, t, -1, c_t, co, 1, s, 0, 0.0)); short = len(ops) - 1
+            ops.append(Op(ADD, c3, short, co, co, 0, 1, 0, 0.0)); t = len(ops) - 1
+            c_t = co
     return t, c_t
 
 
-def resnet_v2_cifar(n, widths=(16, 32, 64), n_classes=10, in_ch=3):
-    """Depth 9n+2: 3x3 stem to widths[0] channels, three stages of n bottleneck blocks."""
+def resnet_v2_cifar(n, widths=(16, 32, 64), n_classes=10, in_ch=3, outs=None):
+    """Depth 9n+2: 3x3 stem to widths[0] channels, three stages of n bottleneck blocks.
+
+    outs = block output channels per stage.  The default (4 x width: 64/128/256 from widths 16/32/64) is the
+    benchmark's instance; widths (16, 64, 128) with outs (64, 128, 256) is the chaining rule of the Keras example
+    the paper takes its definitions from (a stage's bottleneck width = the previous stage's output)."""
     ops = [Op(CONV, -1, -1, in_ch, widths[0], 3, 1, 1, 0.0)]
-    t, c_t = _bottleneck_stages(ops, 0, widths[0], widths, (n,) * len(widths), (1,) + (2,) * (len(widths) - 1))
+    t, c_t = _bottleneck_stages(ops, 0, widths[0], widths, (n,) * len(widths), (1,) + (2,) * (len(widths) - 1), outs)
     ops.append(Op(BNRELU, t, -1, c_t, c_t, 0, 1, 0, EPS))
     ops.append(Op(HEAD, len(ops) - 1, -1, c_t, n_classes, 0, 1, 0, 0.0))
     return ops
@@ -61,6 +67,9 @@ CONFIGS = {
     "r110":  (lambda: resnet_v2_cifar(12), (32, 32, 3), 128, 4, 4),
     "r1001": (lambda: resnet_v2_cifar(111), (32, 32, 3), 128, 8, 8),
     "r152":  (lambda: resnet_v2_imagenet(), (224, 224, 3), 64, 4, 4),
+    # the ~30 M-parameter width variant of ResNet-1001 (Section 6.3 quotes that size) and a short net of the same widths
+    "r1001k": (lambda: resnet_v2_cifar(111, (16, 64, 128), outs=(64, 128, 256)), (32, 32, 3), 128, 8, 8),
+    "r20k":   (lambda: resnet_v2_cifar(2, (16, 64, 128), outs=(64, 128, 256)), (32, 32, 3), 16, 2, 2),
 }
 
 
