@@ -219,3 +219,13 @@ def test_training_steps_follow_the_oracle_and_lower_the_loss():
     assert losses[-1] < losses[0], losses
     with pytest.raises(hpf.HpfError):
         bd.model.sgd_momentum_step(vel, -1.0, mu, wd)
+
+
+def test_microbatch_tuner_returns_the_fastest_candidate():
+    from paper_1911_05146_b200.tuner import tune_microbatches, halving_candidates
+    c = wl.config("r11")
+    theta = torch.from_numpy(wl.draw_params(c["ops"]))
+    best, tried = tune_microbatches(c["ops"], (c["B"],) + tuple(c["in_hwc"]), c["cuts"], theta, patience=8, steps=2)
+    assert set(tried) == set(halving_candidates(c["B"]))
+    assert best in tried and tried[best] == min(tried.values())
+    assert all(ms > 0 for ms in tried.values())

@@ -157,3 +157,14 @@ def test_load_balancer_cuts():
     assert max(parts) < max(eq) and max(parts) / min(parts) < 1.05
     m = hpf.Model(c["ops"], (c["B"],) + c["in_hwc"], cuts, c["M"])       # the cuts are accepted by the model
     assert m.num_partitions() == 8
+
+
+def test_microbatch_tuner_search_order():
+    """Section 5.3: pipeline stages range from 1 to the batch size; the search starts at the batch size and halves."""
+    from paper_1911_05146_b200.tuner import halving_candidates
+    assert halving_candidates(128) == [128, 64, 32, 16, 8, 4, 2, 1]
+    assert halving_candidates(12) == [12, 6, 3, 1]
+    assert halving_candidates(96, smallest=8) == [96, 48, 24, 12]
+    assert halving_candidates(1) == [1]
+    for b in (7, 30, 128):
+        assert all(b % m == 0 for m in halving_candidates(b))
