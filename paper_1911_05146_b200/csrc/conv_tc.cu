@@ -260,7 +260,8 @@ struct WgradScalars {
     float* out;                  // dw or partials [splits][c_out*taps*c_in]
     DeviceStatus* status;
     int box_w, box_h, box_n, tiles_w, tiles_h, n_tiles, tiles_per_split;
-    int rows;                    // pixels per tile (32 or 64)
+    int rows;                    // pixel rows of a tile in shared memory (32 or 64)
+    int box_rows;                // pixels the copy delivers (<= rows); the rest stays zero
     int c_out, c_in, R, pad;
     int m_chunk;                 // output channels per CTA (<= 128)
     int n_cols;                  // input channels per CTA (<= 256)
@@ -651,7 +652,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     const int C = p.c_out, ncol4 = C >> 1;          // float4 columns of one tile's [2][C] sums (256 % ncol4 == 0)
                     const int n_tiles = gridDim.x;
                     double (*bn_red)[4] = reinterpret_cast<double (*)[4]>(smem);
-                    const int col4 = tid % ncol4, ln = tid / ncol4, L = 256 / ncol4;
+                    const int col4 = tid % ncol4, ln = tid / ncol4, L = ncol4 <= 256 ? 256 / ncol4 : 1;   // C <= 256 (checked on the host)
                     const float4* part = reinterpret_cast<const float4*>(p.stat_partials);
                     double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
 #pragma unroll 8
@@ -794,6 +795,19 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), p.tmem_cols);
+    if (p.box_rows < p.rows) {
+        // A pixel box whose size is not a multiple of 32 leaves the last rows of every raw tile untouched by the
+        // copies: they are zeroed once and add nothing to the sums over pixels.
+        const int pad_rows = p.rows - p.box_rows;
+        for (int s = 0; s < p.raw_stages; ++s) {
+            float* st = reinterpret_cast<float*>(smem + s * p.raw_bytes);
+            for (int i = threadIdx.x; i < pad_rows * p.m_chunk; i += blockDim.x) st[p.box_rows * p.m_chunk + i] = 0.f;
+            for (int tp = 0; tp < ntaps; ++tp) {
+                float* bt = reinterpret_cast<float*>(smem + s * p.raw_bytes + raw_a + tp * raw_b);
+                for (int i = threadIdx.x; i < pad_rows * p.n_cols; i += blockDim.x) bt[p.box_rows * p.n_cols + i] = 0.f;
+            }
+        }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -995,11 +1009,21 @@ weight_prep_single_kernel(const float* __restrict__ w, float* __restrict__ w_hi,
 // ------------------------------------------------------------------------------------------------
 struct PixelBox { int w, h, n, rows; };
 
-// A rectangular box of output pixels with at most `max_rows` pixels; all of w, then rows of h, then images.
+// A rectangular box of output pixels with at most `max_rows` pixels: all of w (or, for maps wider than a tile, a
+// divisor of w), then rows of h, then images.
 bool choose_box(int Q, int P, int N, int max_rows, int rows_mult, PixelBox* out)
 {
-    if (Q > max_rows) return false;
     PixelBox b;
+    if (Q > max_rows) {
+        // a row of the map does not fit one tile: the widest divisor of the row that does
+        int w = 0;
+        for (int d = max_rows; d >= 4 && !w; --d)
+            if (Q % d == 0 && (rows_mult <= 1 || d % rows_mult == 0)) w = d;
+        if (!w) return false;
+        b.w = w; b.h = 1; b.n = 1; b.rows = w;
+        *out = b;
+        return true;
+    }
     b.w = Q;
     int hmax = max_rows / Q;
     if (hmax > P) hmax = P;
@@ -1089,7 +1113,7 @@ cudaError_t encode(CUtensorMap* tm, const float* base, int rank, const cuuint64_
 
 struct WgradGeom {
     PixelBox box;
-    int m_chunk, n_cols, taps_per_cta, tap_groups, raw_stages, t_stages, splits, tiles_per_split, n_tiles;
+    int m_chunk, n_cols, taps_per_cta, tap_groups, raw_stages, t_stages, splits, tiles_per_split, n_tiles, rows_padded;
     unsigned int raw_bytes, t_bytes, tmem_cols;
 };
 
@@ -1118,14 +1142,15 @@ bool wgrad_geom(const ConvShape& s, int passes, WgradGeom* g)
             if (tpc * n_cols > 512) continue;
             for (int rows = 64; rows >= 32 && !found; rows >>= 1) {
                 PixelBox b;
-                if (!choose_box(s.Q, s.P, s.N, rows, 32, &b)) continue;
-                const unsigned int raw = (unsigned int)b.rows * 4u * (unsigned int)(g->m_chunk + tpc * n_cols);
+                if (!choose_box(s.Q, s.P, s.N, rows, 1, &b)) continue;
+                const int padded = (b.rows + 31) / 32 * 32;       // shared-memory rows: whole groups of 32 pixels
+                const unsigned int raw = (unsigned int)padded * 4u * (unsigned int)(g->m_chunk + tpc * n_cols);
                 const unsigned int raw_al = (raw + 1023u) & ~1023u;
-                const unsigned int tb = parts * (unsigned int)(b.rows / 32) * 128u * (unsigned int)(128 + tpc * n_cols);
+                const unsigned int tb = parts * (unsigned int)(padded / 32) * 128u * (unsigned int)(128 + tpc * n_cols);
                 if (2 * raw_al + 2 * tb > kSmemBudget) continue;
                 g->n_cols = n_cols;
                 g->taps_per_cta = tpc;
-                g->box = b; g->raw_bytes = raw_al; g->t_bytes = tb;
+                g->box = b; g->rows_padded = padded; g->raw_bytes = raw_al; g->t_bytes = tb;
                 g->t_stages = 2;
                 int rs = (int)((kSmemBudget - 2 * tb) / raw_al);
                 g->raw_stages = rs > 2 ? 2 : rs;
@@ -1184,8 +1209,10 @@ bool conv_tc_can_fuse_bn(const ConvShape& s, int pass)
 {
     FwdView v;
     if (pass == PASS_WGRAD || !fwd_view(s, pass, &v)) return false;
-    const int n_chunk = v.c_out < 256 ? v.c_out : 256;
-    return 256 % (n_chunk / 4) == 0 && conv_tc_tiles(s, pass) > 0;
+    // the write-out keeps one group of 4 channels per thread and the last CTA combines 2*C columns with 256 threads:
+    // a power of two between 16 and 256 channels, all in one channel slice
+    const int C = v.c_out;
+    return C >= 16 && C <= 256 && (C & (C - 1)) == 0 && conv_tc_tiles(s, pass) > 0;
 }
 
 bool conv_tc_can_fuse_bn_input(const ConvShape& s)
@@ -1263,7 +1290,7 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
         p.out = g.splits > 1 ? reinterpret_cast<float*>(scratch) : out;
         p.box_w = g.box.w; p.box_h = g.box.h; p.box_n = g.box.n;
         p.tiles_w = (s.Q + g.box.w - 1) / g.box.w; p.tiles_h = (s.P + g.box.h - 1) / g.box.h;
-        p.n_tiles = g.n_tiles; p.tiles_per_split = g.tiles_per_split; p.rows = g.box.rows;
+        p.n_tiles = g.n_tiles; p.tiles_per_split = g.tiles_per_split; p.rows = g.rows_padded; p.box_rows = g.box.rows;
         p.c_out = s.K; p.c_in = s.C; p.R = s.R; p.pad = s.pad;
         p.m_chunk = g.m_chunk; p.n_cols = g.n_cols; p.taps_per_cta = g.taps_per_cta;
         p.raw_stages = g.raw_stages; p.t_stages = g.t_stages; p.passes = passes;

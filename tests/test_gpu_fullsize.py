@@ -64,3 +64,7 @@ def test_keras_width_variant_short_net():
 
 def test_keras_width_variant_resnet1001_batch128():
     _fullsize("r1001k", sample_m=[3])
+
+
+def test_config5_resnet152_imagenet_layout_batch64():
+    _fullsize("r152", sample_m=[2])

@@ -61,6 +61,19 @@ def test_conv_sweep_tensor_core_path(shape, path):
         assert min(e) > 1e-5          # it really is the 11-bit path
 
 
+@pytest.mark.parametrize("shape", [(3, 1, 64, 64, 56), (1, 1, 256, 64, 56), (1, 2, 256, 128, 56), (3, 1, 128, 128, 28),
+                                   (1, 1, 128, 512, 28), (3, 1, 256, 256, 14), (1, 2, 1024, 512, 14), (3, 1, 512, 512, 7),
+                                   (1, 1, 512, 2048, 7), (1, 1, 2048, 512, 7)],
+                         ids=lambda s: "k%d_s%d_%dto%d_at%d" % s)
+def test_conv_imagenet_layout_map_sizes_on_the_tensor_core_path(shape):
+    """Feature maps 56, 28, 14 and 7 pixels wide (the 224x224 layout): pixel boxes that are not multiples of 32 pixels
+    (weight gradient: zero-padded tile rows) and ragged box rows."""
+    ks, st, ci, co, H = shape
+    e = _conv_case(ks, st, ci, co, H, N=3, path=0)
+    # fp32 accumulation over up to 9*512 products: the error grows with the length of the sum (3e-5 at K = 4608)
+    assert max(e) <= 5e-5, e
+
+
 @pytest.mark.parametrize("shape", [(1, 1, 16, 64, 32), (3, 1, 32, 32, 16), (1, 2, 128, 64, 16), (3, 1, 3, 16, 32),
                                    (7, 2, 3, 64, 32), (3, 2, 5, 7, 9), (1, 1, 12, 20, 5)],
                          ids=lambda s: "k%d_s%d_%dto%d_at%d" % s)

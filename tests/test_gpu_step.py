@@ -104,6 +104,13 @@ def test_imagenet_layout_small_with_maxpool():
     check_step(ops, (32, 32, 3), 4, 2, [2, 11], seed=2, bn_jitter=0.2)
 
 
+def test_imagenet_layout_wide_channels():
+    """Channel counts beyond 256 (512 and 1024 block outputs, 3x3 at 128 and 256): convolutions, BN and the fusions that
+    apply only up to 256 channels side by side."""
+    ops = wl.resnet_v2_imagenet(blocks=(2, 1), widths=(128, 256), n_classes=9)
+    check_step(ops, (32, 32, 3), 4, 2, [9, 20], seed=3, bn_jitter=0.2)
+
+
 def test_second_step_and_new_inputs_reuse_the_model():
     c = wl.config("r11")
     ops = c["ops"]
