@@ -32,7 +32,6 @@
 // device status word, stops issuing work, waits (bounded) for its TMA copies in flight, frees its
 // tensor memory and returns.
 #include "conv_tc.h"
-#include <cstdlib>
 
 #include <cuda.h>
 #include <stdint.h>
@@ -1314,8 +1313,7 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     FwdParams& P = L->p;
     memset(&P, 0, sizeof P);
     FwdScalars& p = P.s;
-    static const int dbg_kchunk = getenv("HPF_DBG_KCHUNK") ? atoi(getenv("HPF_DBG_KCHUNK")) : 0;
-    const int kchunk = dbg_kchunk == 16 ? 16 : chunk_of(v.c_in);
+    const int kchunk = chunk_of(v.c_in);
     const int n_chunk = v.c_out < 256 ? v.c_out : 256;
     {
         cuuint64_t dims[4] = {(cuuint64_t)v.c_in, (cuuint64_t)v.in_w, (cuuint64_t)v.in_h, (cuuint64_t)v.N};
@@ -1353,17 +1351,8 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     p.tx_bytes = (unsigned int)b.rows * kchunk * 4 + parts * (unsigned int)n_chunk * kchunk * 4;
     int stages = (int)(kSmemBudget / p.stage_bytes);
     const int total = v.R * v.R * p.n_kchunks;
-    static const int dbg_max_stages = getenv("HPF_DBG_MAX_STAGES") ? atoi(getenv("HPF_DBG_MAX_STAGES")) : kFwdMaxStages;
-    if (stages > dbg_max_stages) stages = dbg_max_stages;
+    if (stages > kFwdMaxStages) stages = kFwdMaxStages;      // measured: more stages cost more in residency than they hide
     if (stages > total) stages = total;
-    {
-        static const int target = getenv("HPF_DBG_SMEM_TARGET") ? atoi(getenv("HPF_DBG_SMEM_TARGET")) : 0;
-        if (target > 0) {
-            int occ = target / (int)p.stage_bytes;
-            if (occ < 1) occ = 1;
-            if (stages > occ) stages = occ;
-        }
-    }
     p.stages = stages;
     if (fuse && fuse->mode) {
         if (256 % (n_chunk / 4)) return cudaErrorNotSupported;
