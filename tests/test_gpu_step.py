@@ -92,6 +92,18 @@ def test_mid_block_cuts_and_jittered_bn(cuts, fuse_add):
         assert not all(stored)
 
 
+@pytest.mark.parametrize("B,M,cuts", [(4, 1, []), (4, 4, [9]), (3, 3, "every op"), (6, 2, "every op")],
+                         ids=["one_partition_one_microbatch", "microbatches_of_one_sample", "one_op_per_partition_b1", "one_op_per_partition"])
+def test_degenerate_partitionings(B, M, cuts):
+    """The ends of the ranges the method allows (Section 5.3: 1..batch size micro-batches; Section 7: at most one layer
+    per partition): no pipelining at all, micro-batches of a single sample, and every op its own partition."""
+    ops = wl.resnet_v2_cifar(1)
+    if cuts == "every op":
+        cuts = list(range(1, len(ops)))
+    bd, _, _ = check_step(ops, (32, 32, 3), B, M, cuts, seed=4, bn_jitter=0.2)
+    assert bd.model.num_partitions() == len(cuts) + 1
+
+
 def test_odd_widths_run_on_cuda_cores():
     ops = wl.resnet_v2_cifar(1, widths=(4, 8, 12), n_classes=5)
     bd, _, _ = check_step(ops, (8, 8, 3), 6, 3, [9], seed=1, bn_jitter=0.2)
