@@ -140,8 +140,8 @@ def run_reference(args, cfg):
     cores = os.cpu_count()
     b = cfg["B"] // cfg["M"]
     t1 = oracle_sample(cfg, 1)                               # calibration, untimed
-    budget = 150.0 / max(1, args.steps + args.warmup)
-    images = int(max(1, min(b, budget / max(t1, 1e-3))))
+    per_step_s = 150.0 / max(1, args.steps + args.warmup)
+    images = int(max(1, min(b, per_step_s / max(t1, 1e-3))))
     for _ in range(args.warmup):
         oracle_sample(cfg, images)
     ts = [oracle_sample(cfg, images) for _ in range(args.steps)]

@@ -82,7 +82,7 @@ struct hpf_model {
     std::vector<int> grad_alias;              // tensor -> ADD op whose gradient buffer it shares, or -1
     std::vector<int> fused_into;              // conv -> residual ADD computed in its epilogue (its own output is not stored), or -1
     std::vector<int> add_done_by;             // ADD -> the conv that computes it, or -1
-    std::vector<int> bn_fwd_from;              // BN -> conv whose forward kernel leaves the per-tile sums of the BN's input, or -1
+    std::vector<int> bn_fwd_from;              // BN -> conv whose forward kernel also produces the statistics of the BN (its input), or -1
     std::vector<int> conv_fwd_bn;              // the inverse map
     std::vector<int> bn_into, conv_in_bn;      // BN -> the convolution that applies it to its own input operand (no BN kernel), and the inverse
     int opt_cell_times = 0;    // record a device timestamp at the start and end of every (partition, micro-batch) cell
@@ -339,10 +339,10 @@ ConvShape conv_shape_of(const hpf_model* mdl, int i)
     return make_conv_shape(mdl->b, o.iH, o.iW, o.iC, o.op.c_out, o.op.ksize, o.op.stride, o.op.pad);
 }
 
-// Which convolutions run on the tensor cores, and which BN reductions ride in their write-out: the sums of a
-// BN's input in the forward kernel that produces it, the sums of the BN's backward in the data-gradient kernel
-// that produces dL/d(BN output).  Only when producer and BN run back to back on the same stream (same partition,
-// nothing but a fused residual add between them), so that the per-stream scratch can carry the partial sums.
+// Which convolutions run on the tensor cores, and which BN work rides inside them: the statistics of a BN in the
+// forward kernel that produces its input (only when producer and BN run back to back on the same stream: same
+// partition, nothing but a fused residual add between them, so that the per-stream scratch can carry the per-tile
+// sums), and the BN+ReLU itself on the operand path of the convolution that reads it.
 void build_kernel_plan(hpf_model* mdl)
 {
     const int n = mdl->n_ops;
