@@ -245,7 +245,13 @@ struct FwdScalars {
     int in_w, in_h;              // extent of the input pixel grid (the padding mask)
     const float* bn_in_gamma;
     const float* bn_in_beta;
-    const float* bn_in_stats;    // mean[c_in], rstd[c_in] (left by the kernel that produced x)
+    const float* bn_in_stats;    // bn_in 1: mean[c_in], rstd[c_in] (left by the kernel that produced x)
+    // bn_in 2: the statistics are derived here from the producer's per-tile sums and stored by the first CTA
+    const float* bn_in_partials; // [bn_in_tiles][2][c_in]
+    float* bn_in_stats_out;
+    int bn_in_tiles;
+    float bn_in_eps;
+    double bn_in_inv_rows;
     float* bn_in_y;              // relu(bn(x)), dense [N][in_h][in_w][c_in], written by the CTAs of the first channel slice
 };
 struct alignas(64) FwdParams {
@@ -293,6 +299,44 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 
 // x = hi + lo, hi = x with the low 13 significand bits cleared (what a TF32 operand keeps)
 __device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+
+// BN statistics from per-tile sums [n_tiles][2][C] (sum x, sum x*x): the tiles are added in a fixed order in fp64, so
+// every caller gets the same bits.  Called by 256 threads (tid 0..255) that share named barrier 1; C is a power of
+// two in 16..256; bn_red: 256 x 4 doubles of shared memory.  On return thread tid < C holds its channel's mean and
+// 1/sqrt(var + eps).
+__device__ __forceinline__ void bn_combine_partials(const float* partials, int n_tiles, int C, double inv_rows, float eps,
+                                                    double (*bn_red)[4], int tid, float* mean, float* rstd)
+{
+    const int ncol4 = C >> 1;                          // float4 columns of one tile's [2][C] sums; 256 % ncol4 == 0
+    const int col4 = tid % ncol4, ln = tid / ncol4, L = 256 / ncol4;
+    const float4* part = reinterpret_cast<const float4*>(partials);
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+#pragma unroll 8
+    for (int k = ln; k < n_tiles; k += L) {
+        const float4 v = __ldcg(part + (size_t)k * ncol4 + col4);
+        a0 += (double)v.x; a1 += (double)v.y; a2 += (double)v.z; a3 += (double)v.w;
+    }
+    bn_red[tid][0] = a0; bn_red[tid][1] = a1; bn_red[tid][2] = a2; bn_red[tid][3] = a3;
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (tid < ncol4) {
+        // rows tid, tid + ncol4, ... are read by this thread alone, so the total can go back into row tid
+        double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
+        for (int l = 0; l < L; ++l) {
+            const double* r = bn_red[l * ncol4 + tid];
+            t0 += r[0]; t1 += r[1]; t2 += r[2]; t3 += r[3];
+        }
+        bn_red[tid][0] = t0; bn_red[tid][1] = t1; bn_red[tid][2] = t2; bn_red[tid][3] = t3;
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    const double* tot = &bn_red[0][0];                  // [2][C]: sums, then sums of squares
+    if (tid < C) {
+        const double m = tot[tid] * inv_rows;
+        double var = tot[C + tid] * inv_rows - m * m;
+        if (var < 0.0) var = 0.0;
+        *mean = (float)m;
+        *rstd = (float)(1.0 / sqrt(var + (double)eps));
+    }
+}
 
 // ------------------------------------------------------------------------------------------------
 // forward / data-gradient kernel: 10 warps = TMA producer, MMA issuer, 8 splitter / epilogue warps
@@ -424,7 +468,19 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             // ---- BN+ReLU on the way in: the tile holds the BN's input x; the operand is relu(gamma*xhat+beta) ----
             __shared__ __align__(16) float bn_par[4][256];      // mean, rstd, gamma, beta per input channel
             const int C = p.c_in;
-            if (tid < C) {
+            if (p.bn_in == 2) {
+                // The producer left only its per-tile sums (few enough that adding them here, under the first copy's
+                // latency, is cheaper than a ticket at the producer's end): every CTA adds them in the same fixed order,
+                // so all CTAs hold identical statistics; the first CTA stores them for the backward pass.
+                __shared__ double bn_red[256][4];
+                float gam = 0.f, bet = 0.f, mu = 0.f, rs = 0.f;
+                if (tid < C) { gam = __ldg(p.bn_in_gamma + tid); bet = __ldg(p.bn_in_beta + tid); }   // travel with the sums
+                bn_combine_partials(p.bn_in_partials, p.bn_in_tiles, C, p.bn_in_inv_rows, p.bn_in_eps, bn_red, tid, &mu, &rs);
+                if (tid < C) {
+                    bn_par[0][tid] = mu; bn_par[1][tid] = rs; bn_par[2][tid] = gam; bn_par[3][tid] = bet;
+                    if (blockIdx.x == 0 && blockIdx.y == 0) { p.bn_in_stats_out[tid] = mu; p.bn_in_stats_out[C + tid] = rs; }
+                }
+            } else if (tid < C) {
                 bn_par[0][tid] = __ldg(p.bn_in_stats + tid); bn_par[1][tid] = __ldg(p.bn_in_stats + C + tid);
                 bn_par[2][tid] = __ldg(p.bn_in_gamma + tid); bn_par[3][tid] = __ldg(p.bn_in_beta + tid);
             }
@@ -635,50 +691,24 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     for (int t2 = g; t2 < 256; t2 += c4n) { const float4 v2 = red[2 * t2 + which]; acc.x += v2.x; acc.y += v2.y; acc.z += v2.z; acc.w += v2.w; }
                     float* dstp = p.stat_partials + ((size_t)blockIdx.x * 2 + which) * p.c_out + co0 + 4 * g;
                     *reinterpret_cast<float4*>(dstp) = acc;
-                    __threadfence();
+                    if (stat_mode == 1) __threadfence();
                 }
-                // The CTA that finishes last turns the per-tile sums into mean and 1/sigma: tiles are added in a fixed
-                // order in fp64, so the result does not depend on which CTA that is.
+                // stat_mode 1: the CTA that finishes last turns the per-tile sums into mean and 1/sigma (tiles are added in
+                // a fixed order in fp64, so the result does not depend on which CTA that is).  stat_mode 3: the reading
+                // convolution adds the few per-tile sums itself, and this kernel ends without a ticket.
                 __shared__ int is_last;
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (tid == 0) {
+                if (stat_mode == 1) asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (stat_mode == 1 && tid == 0) {
                     const unsigned int done_before = atomicAdd(p.stat_ticket, 1u);
                     is_last = done_before == gridDim.x * gridDim.y - 1;
                 }
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (is_last) {
+                if (stat_mode == 1) asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (stat_mode == 1 && is_last) {
                     __threadfence();
-                    const int C = p.c_out, ncol4 = C >> 1;          // float4 columns of one tile's [2][C] sums (256 % ncol4 == 0)
-                    const int n_tiles = gridDim.x;
-                    double (*bn_red)[4] = reinterpret_cast<double (*)[4]>(smem);
-                    const int col4 = tid % ncol4, ln = tid / ncol4, L = ncol4 <= 256 ? 256 / ncol4 : 1;   // C <= 256 (checked on the host)
-                    const float4* part = reinterpret_cast<const float4*>(p.stat_partials);
-                    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-#pragma unroll 8
-                    for (int k = ln; k < n_tiles; k += L) {
-                        const float4 v = __ldcg(part + (size_t)k * ncol4 + col4);
-                        a0 += (double)v.x; a1 += (double)v.y; a2 += (double)v.z; a3 += (double)v.w;
-                    }
-                    bn_red[tid][0] = a0; bn_red[tid][1] = a1; bn_red[tid][2] = a2; bn_red[tid][3] = a3;
-                    asm volatile("bar.sync 1, 256;" ::: "memory");
-                    if (tid < ncol4) {
-                        // rows tid, tid + ncol4, ... are read by this thread alone, so the total can go back into row tid
-                        double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
-                        for (int l = 0; l < L; ++l) {
-                            const double* r = bn_red[l * ncol4 + tid];
-                            t0 += r[0]; t1 += r[1]; t2 += r[2]; t3 += r[3];
-                        }
-                        bn_red[tid][0] = t0; bn_red[tid][1] = t1; bn_red[tid][2] = t2; bn_red[tid][3] = t3;
-                    }
-                    asm volatile("bar.sync 1, 256;" ::: "memory");
-                    const double* tot = &bn_red[0][0];              // [2][C]: sums, then sums of squares
-                    if (tid < C) {
-                        const double mean = tot[tid] * p.stat_inv_rows;
-                        double var = tot[C + tid] * p.stat_inv_rows - mean * mean;
-                        if (var < 0.0) var = 0.0;
-                        p.stat_out[tid] = (float)mean;
-                        p.stat_out[C + tid] = (float)(1.0 / sqrt(var + (double)p.stat_eps));
-                    }
+                    float mu = 0.f, rs = 0.f;
+                    bn_combine_partials(p.stat_partials, (int)gridDim.x, p.c_out, p.stat_inv_rows, p.stat_eps,
+                                        reinterpret_cast<double (*)[4]>(smem), tid, &mu, &rs);
+                    if (tid < p.c_out) { p.stat_out[tid] = mu; p.stat_out[p.c_out + tid] = rs; }
                     if (tid == 0) *p.stat_ticket = 0u;
                 }
             }
@@ -1356,15 +1386,19 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     p.stages = stages;
     if (fuse && fuse->mode) {
         if (256 % (n_chunk / 4)) return cudaErrorNotSupported;
-        if (fuse->mode != 1 || pass != PASS_FWD || !conv_tc_can_fuse_bn(s, pass) || fuse->rows < 1) return cudaErrorNotSupported;
-        p.stat_mode = 1; p.stat_partials = fuse->partials;
+        if ((fuse->mode != 1 && fuse->mode != 3) || pass != PASS_FWD || !conv_tc_can_fuse_bn(s, pass) || fuse->rows < 1) return cudaErrorNotSupported;
+        p.stat_mode = fuse->mode; p.stat_partials = fuse->partials;
         p.stat_ticket = fuse->ticket; p.stat_out = fuse->stats_out; p.stat_eps = fuse->eps; p.stat_inv_rows = 1.0 / (double)fuse->rows;
     }
     if (fuse && fuse->in_mode) {
         if (pass != PASS_FWD || !conv_tc_can_fuse_bn_input(s)) return cudaErrorNotSupported;
-        p.bn_in = 1; p.in_w = v.in_w; p.in_h = v.in_h;
+        if (fuse->in_mode != 1 && fuse->in_mode != 2) return cudaErrorInvalidValue;
+        if (fuse->in_mode == 2 && (fuse->in_tiles < 1 || fuse->in_rows < 1 || !fuse->in_partials)) return cudaErrorInvalidValue;
+        p.bn_in = fuse->in_mode; p.in_w = v.in_w; p.in_h = v.in_h;
         p.bn_in_gamma = fuse->in_gamma; p.bn_in_beta = fuse->in_beta;
         p.bn_in_stats = fuse->in_stats; p.bn_in_y = fuse->in_y;
+        p.bn_in_partials = fuse->in_partials; p.bn_in_stats_out = fuse->in_stats; p.bn_in_tiles = fuse->in_tiles;
+        p.bn_in_eps = fuse->in_eps; p.bn_in_inv_rows = fuse->in_rows > 0 ? 1.0 / (double)fuse->in_rows : 0.0;
     }
     p.stacked = (passes == 3 && 2 * n_chunk <= 256) ? 1 : 0;
     p.tmem_cols = pow2_cols(p.stacked ? 2 * n_chunk : n_chunk);

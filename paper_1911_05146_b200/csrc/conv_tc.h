@@ -24,14 +24,17 @@ struct ConvTcPlan {
 };
 
 // Batch-norm work folded into the forward kernel.
-//   mode 1 (output side): the kernel's output is the input of a BN.  Per tile and output channel the write-out forms
-//   the sum and the sum of squares of what it stores (partials, [conv_tc_tiles(s, PASS_FWD)][2][channels] floats); the
-//   CTA that finishes last (ticket: one zeroed word, left zero) adds them in a fixed order and stores mean[C], rstd[C]
-//   of the `rows` pixels to stats_out.
-//   in_mode 1 (input side): the kernel's input tensor is the INPUT x of a BN+ReLU op whose output only this convolution
-//   reads, and in_stats holds that BN's mean / rstd.  The kernel applies y = relu(gamma*(x-mean)*rstd+beta) to the
-//   activation tile on its way to the tensor core (the padding ring stays zero) and stores y (in_y, needed by the
-//   backward pass) as a by-product: the BN+ReLU needs no kernel of its own.
+//   Output side: the kernel's output is the input of a BN.  Per tile and output channel the write-out forms the sum and
+//   the sum of squares of what it stores (partials, [conv_tc_tiles(s, PASS_FWD)][2][channels] floats).
+//     mode 1: the CTA that finishes last (ticket: one zeroed word, left zero) adds them in a fixed order and stores
+//             mean[C], rstd[C] of the `rows` pixels to stats_out;
+//     mode 3: the kernel leaves the partials only; the convolution that applies the BN adds them (in_mode 2).
+//   Input side: the kernel's input tensor is the INPUT x of a BN+ReLU op whose output only this convolution reads.  The
+//   kernel applies y = relu(gamma*(x-mean)*rstd+beta) to the activation tile on its way to the tensor core (the padding
+//   ring stays zero) and stores y (in_y, needed by the backward pass) as a by-product: the BN+ReLU needs no kernel.
+//     in_mode 1: in_stats holds mean / rstd (the producer ran mode 1);
+//     in_mode 2: every CTA adds the producer's per-tile sums (in_partials, in_tiles rows, statistics over in_rows
+//                pixels) in the same fixed order and the first CTA stores mean / rstd to in_stats.
 struct ConvBnFuse {
     int mode = 0;
     float* partials = nullptr;
@@ -42,10 +45,14 @@ struct ConvBnFuse {
     int in_mode = 0;
     const float* in_gamma = nullptr;
     const float* in_beta = nullptr;
-    const float* in_stats = nullptr;
+    float* in_stats = nullptr;
     float* in_y = nullptr;
+    const float* in_partials = nullptr;
+    int in_tiles = 0;
+    long long in_rows = 0;
+    float in_eps = 0.f;
 };
-// Whether in_mode 1 applies to this convolution.
+// Whether the input-side fusion applies to this convolution.
 bool conv_tc_can_fuse_bn_input(const ConvShape& s);
 // Number of pixel tiles (= partial-sum rows) of the forward / data-gradient launch, and whether the fusion applies.
 int conv_tc_tiles(const ConvShape& s, int pass);

@@ -85,6 +85,10 @@ struct hpf_model {
     std::vector<int> bn_fwd_from;              // BN -> conv whose forward kernel also produces the statistics of the BN (its input), or -1
     std::vector<int> conv_fwd_bn;              // the inverse map
     std::vector<int> bn_into, conv_in_bn;      // BN -> the convolution that applies it to its own input operand (no BN kernel), and the inverse
+    std::vector<int> bn_late;                  // BN -> 1: the applying convolution derives the statistics from the per-tile sums itself
+    std::vector<int> bn_buf;                   // BN -> which of the stream's two per-tile-sum buffers carries its sums
+    std::vector<size_t> bn_part_bytes;         // per partition: size of one per-tile-sum buffer
+    int opt_bn_late_floats = 8192;             // largest [tiles][2][C] block of per-tile sums a reading convolution adds itself
     int opt_cell_times = 0;    // record a device timestamp at the start and end of every (partition, micro-batch) cell
     size_t cell_times_off = 0;
     int opt_fuse_bn = 3;       // bit 0: BN statistics in the producing convolution's write-out, bit 1: BN+ReLU applied by the reading convolution
@@ -130,6 +134,11 @@ struct hpf_model {
     float* act(int op, int m) const { return reinterpret_cast<float*>(ws + act_off[(size_t)m * n_ops + op]); }
     float* grad(int op, int m) const { return reinterpret_cast<float*>(ws + grad_off[(size_t)m * n_ops + op]); }
     float* stats(int op, int m) const { return reinterpret_cast<float*>(ws + stats_off[(size_t)m * n_ops + op]); }
+    float* bn_partials(int bn) const
+    {
+        const int p = ops[bn].part;
+        return reinterpret_cast<float*>(ws + bn_scratch_off[p] + 256 + (size_t)bn_buf[bn] * bn_part_bytes[p]);
+    }
     unsigned long long* cell_time_slot(int phase, int p, int m) const
     {
         return reinterpret_cast<unsigned long long*>(ws + cell_times_off) + 2 * (((size_t)(phase == PH_BWD) * P + p) * M + m);
@@ -352,7 +361,8 @@ void build_kernel_plan(hpf_model* mdl)
     }
     mdl->bn_fwd_from.assign(n, -1);
     mdl->conv_fwd_bn.assign(n, -1);
-    mdl->bn_into.assign(n, -1); mdl->conv_in_bn.assign(n, -1);
+    mdl->bn_into.assign(n, -1); mdl->conv_in_bn.assign(n, -1); mdl->bn_late.assign(n, 0); mdl->bn_buf.assign(n, 0);
+    std::vector<int> n_fused(mdl->P, 0);
     if (!mdl->opt_fuse_bn) return;
     for (int j = 0; j < n; ++j) {
         const OpInfo& bn = mdl->ops[j];
@@ -366,7 +376,12 @@ void build_kernel_plan(hpf_model* mdl)
             bool adjacent = true;
             for (int k = prod + 1; k < j; ++k)
                 if (!(mdl->ops[k].op.kind == HPF_OP_ADD && mdl->add_done_by[k] >= 0)) adjacent = false;
-            if (adjacent) { mdl->bn_fwd_from[j] = prod; mdl->conv_fwd_bn[prod] = j; }
+            if (adjacent) {
+                mdl->bn_fwd_from[j] = prod; mdl->conv_fwd_bn[prod] = j;
+                // A convolution that reads BN j's sums may still be reading them while its own write-out already
+                // produces the next BN's: successive fused BNs of a stream alternate between two buffers.
+                mdl->bn_buf[j] = n_fused[bn.part]++ & 1;
+            }
         }
         // the BN+ReLU itself: applied by its only reader, the next op, a stride-1 tensor-core convolution
         if ((mdl->opt_fuse_bn & 2) && mdl->bn_fwd_from[j] >= 0 && bn.consumers.size() == 1 && bn.consumers[0] == j + 1) {
@@ -374,6 +389,10 @@ void build_kernel_plan(hpf_model* mdl)
             if (mdl->ops[i].op.kind == HPF_OP_CONV && mdl->ops[i].op.src0 == j && mdl->use_tc[PASS_FWD][i] &&
                 mdl->ops[i].part == bn.part && conv_tc_can_fuse_bn_input(conv_shape_of(mdl, i))) {
                 mdl->bn_into[j] = i; mdl->conv_in_bn[i] = j;
+                // Few per-tile sums: the reading convolution adds them under the latency of its first copy and the
+                // producer ends without a ticket.  Many: the producer's last CTA adds them once.
+                const long long floats = (long long)conv_tc_tiles(conv_shape_of(mdl, mdl->bn_fwd_from[j]), PASS_FWD) * 2 * bn.C;
+                mdl->bn_late[j] = floats <= mdl->opt_bn_late_floats ? 1 : 0;
             }
         }
     }
@@ -394,8 +413,9 @@ void build_memory_plan(hpf_model* mdl)
     mdl->status_off = take(sizeof(DeviceStatus));
     mdl->bn_scratch_off.assign(P, 0);
     mdl->conv_scratch_off.assign(P, 0);
+    mdl->bn_part_bytes.assign(P, 0);
     for (int p = 0; p < P; ++p) {
-        size_t bn = 256;
+        size_t bn = 256, part = 0;
         for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i)
             if (mdl->ops[i].op.kind == HPF_OP_BNRELU) {
                 const OpInfo& o = mdl->ops[i];
@@ -403,10 +423,12 @@ void build_memory_plan(hpf_model* mdl)
                 if (need > bn) bn = need;
                 const int from = mdl->bn_fwd_from[i];
                 if (from >= 0) {
-                    need = 256 + (size_t)conv_tc_tiles(conv_shape_of(mdl, from), PASS_FWD) * 2 * o.C * sizeof(float);
-                    if (need > bn) bn = need;
+                    need = align_up((size_t)conv_tc_tiles(conv_shape_of(mdl, from), PASS_FWD) * 2 * o.C * sizeof(float), 256);
+                    if (need > part) part = need;
                 }
             }
+        mdl->bn_part_bytes[p] = part;
+        if (256 + 2 * part > bn) bn = 256 + 2 * part;
         mdl->bn_scratch_off[p] = take(bn);
     }
     mdl->zero_hi = at;
@@ -1025,9 +1047,9 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                         if (mdl->conv_fwd_bn[i] >= 0) {
                             const int jn = mdl->conv_fwd_bn[i];
                             const OpInfo& bn = mdl->ops[jn];
-                            fuse.mode = 1;
+                            fuse.mode = mdl->bn_late[jn] ? 3 : 1;
                             fuse.ticket = reinterpret_cast<unsigned int*>(mdl->ws + mdl->bn_scratch_off[o.part]);
-                            fuse.partials = reinterpret_cast<float*>(mdl->ws + mdl->bn_scratch_off[o.part] + 256);
+                            fuse.partials = mdl->bn_partials(jn);
                             fuse.stats_out = mdl->stats(jn, m);
                             fuse.rows = (long long)mdl->b * bn.H * bn.W;
                             fuse.eps = bn.op.eps;
@@ -1037,7 +1059,11 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                         if (jb >= 0) {
                             const OpInfo& bn = mdl->ops[jb];
                             in = mdl->act(bn.op.src0, m);          // the BN's input; its output is a by-product of this kernel
-                            fuse.in_mode = 1;
+                            fuse.in_mode = mdl->bn_late[jb] ? 2 : 1;
+                            fuse.in_partials = mdl->bn_partials(jb);
+                            fuse.in_tiles = conv_tc_tiles(conv_shape_of(mdl, mdl->bn_fwd_from[jb]), PASS_FWD);
+                            fuse.in_rows = (long long)mdl->b * bn.H * bn.W;
+                            fuse.in_eps = bn.op.eps;
                             fuse.in_gamma = mdl->params + bn.w_off; fuse.in_beta = mdl->params + bn.b_off;
                             fuse.in_stats = mdl->stats(jb, m); fuse.in_y = mdl->act(jb, m);
                         }
