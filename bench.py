@@ -227,10 +227,11 @@ def kernel_roofline(torch, hpf, cfg, pk):
     sec = e0.elapsed_time(e1) * 1e-3 / (3 * reps)
     achieved = alg / sec / 1e9
     return {"bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"],
-            # dram__bytes_read + dram__bytes_write of this kernel in the ncu capture of the same shape at batch 128
-            # (profiles/conv_tc_fwd_1x1_64to16_at32_batch128.md: 33.62 MB read = the input once, the output still in L2
-            # when the kernel ends), scaled by the pixels per launch
-            "traffic": 33.62e6 * b / 128.0 if (ks, st, ci, co, H) == (1, 1, 64, 16, 32) else None, "peak_source": pk["source"],
+            # dram__bytes_read + dram__bytes_write of this kernel in the ncu captures of the same shape at batch 128
+            # (profiles/conv_tc_fwd_1x1_*_at32_batch128.md: the input is read once, 33.62 MB / 8.47 MB, and the output is
+            # still in L2 when the kernel ends), scaled by the pixels per launch
+            "traffic": {(1, 1, 64, 16, 32): 33.62e6, (1, 1, 16, 64, 32): 8.47e6}.get((ks, st, ci, co, H), 0.0) * b / 128.0 or None,
+            "peak_source": pk["source"],
             "kernel": "conv_tc_fwd_kernel (tcgen05 implicit GEMM, three-pass TF32), %dx%d stride %d, %d->%d channels, %dx%d "
                       "pixels, micro-batch %d; %d rotating operand sets; one 8-byte status memset node precedes each launch"
                       % (ks, ks, st, ci, co, H, H, b, nset),
