@@ -1202,7 +1202,7 @@ bool wgrad_geom(const ConvShape& s, int passes, WgradGeom* g)
     const int want = (48 + ctas_per_split - 1) / ctas_per_split;
     if (cap < want) cap = want;
     if (splits > cap) splits = cap;
-    if (splits > 64) splits = 64;
+    if (splits > 296) splits = 296;          // two CTAs per SM
     if (splits > g->n_tiles / 2) splits = g->n_tiles / 2;
     if (splits < 1) splits = 1;
     g->tiles_per_split = (g->n_tiles + splits - 1) / splits;
