@@ -45,6 +45,7 @@ constexpr int kTileM = 128;                 // MMA M (TMEM lanes)
 constexpr long long kWaitLimit = 4000000000LL;   // clock64 ticks (~2 s) before a wait gives up
 constexpr uint32_t kSmemBudget = 200 * 1024;
 constexpr int kFwdMaxStages = 4;
+constexpr unsigned int kWgradSlack = 16384;   // an MMA reads 128 operand rows (16 KB) from a base that may be the last one in use
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -806,7 +807,11 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
     const int total = tile_end - tile_begin;
     const int katoms = p.rows >> 5;
     const uint32_t raw_a = (uint32_t)p.rows * p.m_chunk * 4u, raw_b = (uint32_t)p.rows * p.n_cols * 4u;
-    const uint32_t t_a = (uint32_t)katoms * 128u * 128u;                  // room for 128 channel rows
+    // The transposed dy operand keeps only its m_chunk channel rows per pixel group.  An MMA always reads 128 rows from
+    // the operand's base: the rows beyond m_chunk come from whatever follows in shared memory (the other operand, the
+    // next stage, the slack after the last stage) and land in accumulator lanes that the epilogue never reads.
+    const uint32_t a_atom = (uint32_t)p.m_chunk * 128u;                   // one pixel group of the dy operand
+    const uint32_t t_a = (uint32_t)katoms * a_atom;
     // transposed B: [pixel group of 32][tap][input channel] rows of 128 bytes, so that consecutive taps are consecutive
     // N rows of one operand and one MMA covers several taps at once
     const uint32_t t_b_tap = (uint32_t)p.n_cols * 128u;                   // one tap inside one pixel group
@@ -882,7 +887,7 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
                     const uint32_t acc = tmem_base + (uint32_t)(tg * p.n_cols);
                     for (int kb = 0; kb < katoms; ++kb)
                         for (int k8 = 0; k8 < 4; ++k8) {
-                            const uint32_t ao = (uint32_t)kb * 16384u + 32u * k8;
+                            const uint32_t ao = (uint32_t)kb * a_atom + 32u * k8;
                             const uint32_t bo = (uint32_t)kb * t_b_atom + (uint32_t)tg * t_b_tap + 32u * k8;
                             const uint64_t ad = smem_desc(a_src + ao, 16, 1024, 128);
                             const uint64_t bd = smem_desc(b_src + bo, 16, 1024, 128);
@@ -913,12 +918,12 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
             const uint8_t* raw = smem + s * p.raw_bytes;
             uint8_t* tdst = smem + t_region0 + t * p.t_bytes;
             if (p.passes == 3) {
-                transpose_tile<true>(raw, tdst, tdst + t_half, p.m_chunk, p.rows, 16384u, tid);
+                transpose_tile<true>(raw, tdst, tdst + t_half, p.m_chunk, p.rows, a_atom, tid);
                 for (int tp = 0; tp < ntaps; ++tp)
                     transpose_tile<true>(raw + raw_a + tp * raw_b, tdst + t_a + tp * t_b_tap, tdst + t_half + t_a + tp * t_b_tap,
                                          p.n_cols, p.rows, t_b_atom, tid);
             } else {
-                transpose_tile<false>(raw, tdst, nullptr, p.m_chunk, p.rows, 16384u, tid);
+                transpose_tile<false>(raw, tdst, nullptr, p.m_chunk, p.rows, a_atom, tid);
                 for (int tp = 0; tp < ntaps; ++tp)
                     transpose_tile<false>(raw + raw_a + tp * raw_b, tdst + t_a + tp * t_b_tap, nullptr, p.n_cols, p.rows, t_b_atom, tid);
             }
@@ -1175,13 +1180,14 @@ bool wgrad_geom(const ConvShape& s, int passes, WgradGeom* g)
                 const int padded = (b.rows + 31) / 32 * 32;       // shared-memory rows: whole groups of 32 pixels
                 const unsigned int raw = (unsigned int)padded * 4u * (unsigned int)(g->m_chunk + tpc * n_cols);
                 const unsigned int raw_al = (raw + 1023u) & ~1023u;
-                const unsigned int tb = parts * (unsigned int)(padded / 32) * 128u * (unsigned int)(128 + tpc * n_cols);
-                if (2 * raw_al + 2 * tb > kSmemBudget) continue;
+                const unsigned int tb = parts * (unsigned int)(padded / 32) * 128u * (unsigned int)(g->m_chunk + tpc * n_cols);
+                const unsigned int slack = g->m_chunk < 128 ? kWgradSlack : 0u;     // no over-read with 128 channel rows
+                if (2 * raw_al + 2 * tb + slack > kSmemBudget) continue;
                 g->n_cols = n_cols;
                 g->taps_per_cta = tpc;
                 g->box = b; g->rows_padded = padded; g->raw_bytes = raw_al; g->t_bytes = tb;
                 g->t_stages = 2;
-                int rs = (int)((kSmemBudget - 2 * tb) / raw_al);
+                int rs = (int)((kSmemBudget - slack - 2 * tb) / raw_al);
                 g->raw_stages = rs > 2 ? 2 : rs;
                 found = true;
             }
@@ -1331,7 +1337,7 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
         p.idesc_tail = instr_desc(g.n_cols * (g.taps_per_cta % p.taps_per_mma ? g.taps_per_cta % p.taps_per_mma : p.taps_per_mma), false, false);
         p.split_stride = n_out;
         L->grid = dim3(g.splits, g.tap_groups, (s.K / g.m_chunk) * (s.C / g.n_cols));
-        L->smem = (unsigned int)g.raw_stages * g.raw_bytes + (unsigned int)g.t_stages * g.t_bytes + 1024;
+        L->smem = (unsigned int)g.raw_stages * g.raw_bytes + (unsigned int)g.t_stages * g.t_bytes + (g.m_chunk < 128 ? kWgradSlack : 0u) + 1024;
         L->splits = g.splits; L->dw = out; L->n_out = n_out;
         plan->valid = 1;
         return cudaSuccess;
