@@ -44,6 +44,7 @@ namespace {
 constexpr int kTileM = 128;                 // MMA M (TMEM lanes)
 constexpr long long kWaitLimit = 4000000000LL;   // clock64 ticks (~2 s) before a wait gives up
 constexpr uint32_t kSmemBudget = 200 * 1024;
+constexpr uint32_t kWgradSmemBudget = 220 * 1024;   // the weight-gradient kernel has next to no static shared memory
 constexpr int kFwdMaxStages = 4;
 constexpr unsigned int kWgradSlack = 16384;   // an MMA reads 128 operand rows (16 KB) from a base that may be the last one in use
 
@@ -1182,12 +1183,12 @@ bool wgrad_geom(const ConvShape& s, int passes, WgradGeom* g)
                 const unsigned int raw_al = (raw + 1023u) & ~1023u;
                 const unsigned int tb = parts * (unsigned int)(padded / 32) * 128u * (unsigned int)(g->m_chunk + tpc * n_cols);
                 const unsigned int slack = g->m_chunk < 128 ? kWgradSlack : 0u;     // no over-read with 128 channel rows
-                if (2 * raw_al + 2 * tb + slack > kSmemBudget) continue;
+                if (2 * raw_al + 2 * tb + slack > kWgradSmemBudget) continue;
                 g->n_cols = n_cols;
                 g->taps_per_cta = tpc;
                 g->box = b; g->rows_padded = padded; g->raw_bytes = raw_al; g->t_bytes = tb;
                 g->t_stages = 2;
-                int rs = (int)((kSmemBudget - slack - 2 * tb) / raw_al);
+                int rs = (int)((kWgradSmemBudget - slack - 2 * tb) / raw_al);
                 g->raw_stages = rs > 2 ? 2 : rs;
                 found = true;
             }
@@ -1268,7 +1269,7 @@ cudaError_t conv_tc_init()
     if (q != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
     e = cudaFuncSetAttribute(conv_tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(conv_tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
+    e = cudaFuncSetAttribute(conv_tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWgradSmemBudget + 2048);
     if (e != cudaSuccess) return e;
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
     return cudaSuccess;
