@@ -1351,7 +1351,14 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     memset(&P, 0, sizeof P);
     FwdScalars& p = P.s;
     const int kchunk = chunk_of(v.c_in);
-    const int n_chunk = v.c_out < 256 ? v.c_out : 256;
+    int n_chunk = v.c_out < 256 ? v.c_out : 256;
+    {
+        // A launch with few pixel tiles leaves most SMs idle: twice as many channel slices of 128 (each CTA issues the
+        // same number of MMAs at half the width) fill them.  Not when BN work rides in the kernel (one slice there).
+        const int tiles = ((v.Q + b.w - 1) / b.w) * ((v.P + b.h - 1) / b.h) * ((v.N + b.n - 1) / b.n);
+        const bool fused = fuse && (fuse->mode || fuse->in_mode);
+        if (!fused && v.c_out % 256 == 0 && tiles * (v.c_out / 256) <= 74) n_chunk = 128;
+    }
     {
         cuuint64_t dims[4] = {(cuuint64_t)v.c_in, (cuuint64_t)v.in_w, (cuuint64_t)v.in_h, (cuuint64_t)v.N};
         cuuint64_t str[3] = {(cuuint64_t)v.in_sw * 4, (cuuint64_t)v.in_sh * 4, (cuuint64_t)v.in_sn * 4};
