@@ -93,7 +93,7 @@ int hpf_model_destroy(hpf_model *model);
  *                          that convolution's own output is then not stored (hpf_tensor_ptr answers
  *                          HPF_ERR_STATE for it).  0: every op's output is stored.
  *   HPF_OPT_PDL            1 (default): hot kernels use programmatic dependent launch (a kernel is scheduled and runs
- *                          its set-up while its predecessor in the stream drains).  Process-wide switch.
+ *                          its set-up while its predecessor in the stream drains).  0: plain stream-ordered launches.
  *   HPF_OPT_WGRAD_PASSES   1 (default) or 3: TF32 passes of the tensor-core weight gradient.  A weight gradient feeds
  *                          nothing but the average, so its rounding error (about 8e-4 relative with one pass) does not
  *                          compound with depth the way forward and data-gradient errors do; those always follow

@@ -25,7 +25,15 @@ inline ConvShape make_conv_shape(int N, int H, int W, int C, int K, int R, int s
 // still running, executes its prologue (barrier and tensor-memory set-up, parameter and descriptor fetches), and
 // blocks in pdl_wait() until the predecessor has completed and its writes are visible.  Every kernel launched
 // this way calls pdl_wait() before its first read or write of global data.
-extern bool g_pdl_enabled;
+// Per host thread: the model whose phase is being enqueued sets it for the duration of the enqueue (PdlScope).
+extern thread_local bool g_pdl_enabled;
+struct PdlScope {
+    bool saved;
+    explicit PdlScope(bool on) : saved(g_pdl_enabled) { g_pdl_enabled = on; }
+    ~PdlScope() { g_pdl_enabled = saved; }
+    PdlScope(const PdlScope&) = delete;
+    PdlScope& operator=(const PdlScope&) = delete;
+};
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
 {

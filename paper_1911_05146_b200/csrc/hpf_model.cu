@@ -89,6 +89,7 @@ struct hpf_model {
     std::vector<int> bn_buf;                   // BN -> which of the stream's two per-tile-sum buffers carries its sums
     std::vector<size_t> bn_part_bytes;         // per partition: size of one per-tile-sum buffer
     int opt_bn_late_floats = 8192;             // largest [tiles][2][C] block of per-tile sums a reading convolution adds itself
+    bool opt_pdl = true;       // programmatic dependent launch for this model's kernels
     int opt_cell_times = 0;    // record a device timestamp at the start and end of every (partition, micro-batch) cell
     size_t cell_times_off = 0;
     int opt_fuse_bn = 3;       // bit 0: BN statistics in the producing convolution's write-out, bit 1: BN+ReLU applied by the reading convolution
@@ -613,6 +614,7 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
 
 int enqueue_phase(hpf_model* mdl, int phase)
 {
+    const PdlScope pdl_scope(mdl->opt_pdl);
     const int P = mdl->P, M = mdl->M;
     cudaStream_t s0 = mdl->streams[0];
     const bool multi = !mdl->opt_single && P > 1;
@@ -809,7 +811,7 @@ int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
     case HPF_OPT_SINGLE_STREAM: mdl->opt_single = value != 0; break;
     case HPF_OPT_KEEP_MESSAGES: mdl->opt_messages = value != 0; break;
     case HPF_OPT_FUSE_ADD: mdl->opt_fuse_add = value != 0; break;
-    case HPF_OPT_PDL: hpf::g_pdl_enabled = value != 0; break;
+    case HPF_OPT_PDL: mdl->opt_pdl = value != 0; break;
     case HPF_OPT_FUSE_BN: if (value < 0 || value > 3) return fail(HPF_ERR_INVALID, "0..3"); mdl->opt_fuse_bn = value; break;
     case HPF_OPT_CELL_TIMES: mdl->opt_cell_times = value != 0; break;
     case HPF_OPT_WGRAD_PASSES: if (value != 1 && value != 3) return fail(HPF_ERR_INVALID, "1 or 3 passes"); mdl->opt_wgrad_passes = value; break;

@@ -9,7 +9,7 @@
 
 namespace hpf {
 
-bool g_pdl_enabled = true;
+thread_local bool g_pdl_enabled = true;
 
 namespace {
 

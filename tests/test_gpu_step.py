@@ -71,12 +71,8 @@ def test_config1_without_the_fusions(fuse_bn, pdl, wgrad_passes):
     """The BN reductions in their own kernels or both folded into the convolutions, plain stream-ordered
     launches, three-pass weight gradient."""
     c = wl.config("r11")
-    try:
-        check_step(c["ops"], c["in_hwc"], c["B"], c["M"], c["cuts"],
-                   {hpf.OPT_FUSE_BN: fuse_bn, hpf.OPT_PDL: pdl, hpf.OPT_WGRAD_PASSES: wgrad_passes})
-    finally:
-        hpf.lib().hpf_set_option  # the PDL switch is process-wide: restore the default
-        m = hpf.Model(c["ops"], (c["B"],) + c["in_hwc"], c["cuts"], c["M"]); m.set_option(hpf.OPT_PDL, 1)
+    check_step(c["ops"], c["in_hwc"], c["B"], c["M"], c["cuts"],
+               {hpf.OPT_FUSE_BN: fuse_bn, hpf.OPT_PDL: pdl, hpf.OPT_WGRAD_PASSES: wgrad_passes})
 
 
 @pytest.mark.parametrize("cuts", [[], [4], [3, 7, 8], [1, 5, 12, 25]])
