@@ -46,6 +46,7 @@ constexpr long long kWaitLimit = 4000000000LL;   // clock64 ticks (~2 s) before 
 constexpr uint32_t kSmemBudget = 200 * 1024;
 constexpr uint32_t kWgradSmemBudget = 220 * 1024;   // the weight-gradient kernel has next to no static shared memory
 constexpr int kFwdMaxStages = 4;
+constexpr int kMultiTileFrom = 2 * 296;     // CTAs (two per SM) beyond which a forward / data-gradient launch gives each CTA two tiles
 constexpr unsigned int kWgradSlack = 16384;   // an MMA reads 128 operand rows (16 KB) from a base that may be the last one in use
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -243,6 +244,12 @@ struct FwdScalars {
     float stat_eps;
     double stat_inv_rows;        // 1 / (pixels the statistics run over)
     // BN+ReLU applied to the activation operand on its way to the tensor core (see ConvBnFuse::in_mode)
+    // several tiles per CTA (MULTI kernel; tile j of CTA b is tile b*tiles_per_cta + j): tile j+1's loads, split and MMAs
+    // run under tile j's write-out, each tile has its own accumulator columns, and the write-out is staged in a region
+    // of its own
+    int n_tiles, tiles_per_cta;
+    unsigned int acc_cols;       // tensor-memory columns of one tile's accumulator
+    unsigned int stg_off;        // byte offset of the write-out staging area (0: it reuses the idle pipeline buffers)
     int bn_in;
     int in_w, in_h;              // extent of the input pixel grid (the padding mask)
     const float* bn_in_gamma;
@@ -343,6 +350,10 @@ __device__ __forceinline__ void bn_combine_partials(const float* partials, int n
 // ------------------------------------------------------------------------------------------------
 // forward / data-gradient kernel: 10 warps = TMA producer, MMA issuer, 8 splitter / epilogue warps
 // ------------------------------------------------------------------------------------------------
+// MULTI = false: one 128-pixel tile per CTA (the shortest launch; what a launch of up to one wave wants).
+// MULTI = true: p.tiles_per_cta tiles per CTA for launches of several waves: fewer CTAs, and a tile's write-out hides
+// the next tile's loads, split and MMAs.
+template <bool MULTI>
 __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_constant__ FwdParams gp)
 {
     __shared__ FwdScalars p;                 // scalar parameters, see load_scalars
@@ -354,7 +365,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
     load_scalars(&p, &gp.s);
     __syncthreads();
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[3 * 8 + 1];       // full[8], empty[8], split[8], accum
+    __shared__ uint64_t bars[3 * 8 + 4];       // full[8], empty[8], split[8], accum[4] (one per tile of this CTA)
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int issued, consumed;
@@ -370,17 +381,25 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
     const uint32_t off_b = p.passes == 3 ? 2 * p.a_bytes : p.a_bytes;
     const uint32_t off_blo = off_b + p.b_bytes;
 
-    int t = blockIdx.x;
-    const int tw = t % p.tiles_w; t /= p.tiles_w;
-    const int th = t % p.tiles_h;
-    const int tn = t / p.tiles_h;
-    const int q0 = tw * p.box_w, p0 = th * p.box_h, n0 = tn * p.box_n;
+    const int tiles_per_cta = MULTI ? p.tiles_per_cta : 1;
+    const int tile0 = blockIdx.x * tiles_per_cta;
+    const int my_tiles = MULTI ? (p.n_tiles - tile0 < tiles_per_cta ? p.n_tiles - tile0 : tiles_per_cta) : 1;
+    const uint32_t acc_cols = MULTI ? p.acc_cols : 0u;
+    const uint32_t stg_off = MULTI ? p.stg_off : 0u;
     const int co0 = blockIdx.y * p.n_chunk;
+    // first pixel (q0, p0, n0) of tile t
+#define HPF_TILE_ORIGIN(t_)                                                          \
+    int q0, p0, n0;                                                                   \
+    {                                                                                 \
+        int t__ = (t_);                                                               \
+        const int tw__ = t__ % p.tiles_w; t__ /= p.tiles_w;                           \
+        q0 = tw__ * p.box_w; p0 = (t__ % p.tiles_h) * p.box_h; n0 = (t__ / p.tiles_h) * p.box_n; \
+    }
 
     if (threadIdx.x == 0) HPF_TL(0);
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); mbar_init(split0 + 8 * s, 8); }
-        mbar_init(accum_bar, 1);
+        for (int j = 0; j < 4; ++j) mbar_init(accum_bar + 8 * j, 1);
         abort_flag = 0; issued = 0; consumed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -398,17 +417,21 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
         if (lane == 0) {
             // ---- TMA producer ----
             int it = 0;
-            for (; it < total; ++it) {
-                const int s = it % p.stages;
-                if (!mbar_wait(empty0 + 8 * s, ((it / p.stages) & 1) ^ 1, &abort_flag)) { report(p.status, 1); break; }
-                const int tap = it / p.n_kchunks, kc = it % p.n_kchunks;
-                const int r = tap / p.R, sx = tap % p.R;
-                const uint32_t dst = smem_base + s * p.stage_bytes;
-                mbar_expect_tx(full0 + 8 * s, p.tx_bytes);
-                tma_load_4d(dst, &gp.tm_a, full0 + 8 * s, kc * p.kchunk, q0 + sx - p.pad, p0 + r - p.pad, n0);
-                tma_load_2d(dst + off_b, &gp.tm_b, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
-                if (p.passes == 3) tma_load_2d(dst + off_blo, &gp.tm_b_lo, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
-                if (it == 0) HPF_TL(2);
+            bool live = true;
+            for (int j = 0; j < my_tiles && live; ++j) {
+                HPF_TILE_ORIGIN(tile0 + j);
+                for (int k = 0; k < total; ++k, ++it) {
+                    const int s = it % p.stages;
+                    if (!mbar_wait(empty0 + 8 * s, ((it / p.stages) & 1) ^ 1, &abort_flag)) { report(p.status, 1); live = false; break; }
+                    const int tap = k / p.n_kchunks, kc = k % p.n_kchunks;
+                    const int r = tap / p.R, sx = tap % p.R;
+                    const uint32_t dst = smem_base + s * p.stage_bytes;
+                    mbar_expect_tx(full0 + 8 * s, p.tx_bytes);
+                    tma_load_4d(dst, &gp.tm_a, full0 + 8 * s, kc * p.kchunk, q0 + sx - p.pad, p0 + r - p.pad, n0);
+                    tma_load_2d(dst + off_b, &gp.tm_b, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
+                    if (p.passes == 3) tma_load_2d(dst + off_blo, &gp.tm_b_lo, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
+                    if (it == 0) HPF_TL(2);
+                }
             }
             issued = it;
         }
@@ -426,9 +449,12 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             const bool split_first = three || p.bn_in != 0;   // the splitter warps rewrite the tile before it is read
             int it = 0, s = 0;
             uint32_t par = 0;
-            for (; it < total; ++it) {
-                if (!mbar_wait(full0 + 8 * s, par, &abort_flag)) { report(p.status, 2); break; }
-                if (split_first && !mbar_wait(split0 + 8 * s, par, &abort_flag)) { report(p.status, 6); break; }
+            bool live = true;
+            for (int j = 0; j < my_tiles && live; ++j) {
+              const uint32_t acc = tmem_base + (uint32_t)j * acc_cols;
+              for (int k = 0; k < total; ++k, ++it) {
+                if (!mbar_wait(full0 + 8 * s, par, &abort_flag)) { report(p.status, 2); live = false; break; }
+                if (split_first && !mbar_wait(split0 + 8 * s, par, &abort_flag)) { report(p.status, 6); live = false; break; }
                 tc_fence_after();
                 if (it == 0) HPF_TL(5);
                 const uint32_t st = smem_base + s * stage_bytes;
@@ -441,25 +467,26 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     // (columns [0,n) = hi*hi, [n,2n) = hi*lo, added in the epilogue), then A_lo x B_hi.
 #pragma unroll 4
                     for (int k8 = 0; k8 < k8n; ++k8) {
-                        umma_tf32(tmem_base, a0 + 2 * k8, b0 + 2 * k8, idesc2, (it | k8) ? 1u : 0u);
-                        umma_tf32(tmem_base, al0 + 2 * k8, b0 + 2 * k8, idesc, 1u);
+                        umma_tf32(acc, a0 + 2 * k8, b0 + 2 * k8, idesc2, (k | k8) ? 1u : 0u);
+                        umma_tf32(acc, al0 + 2 * k8, b0 + 2 * k8, idesc, 1u);
                     }
                 } else if (three) {
 #pragma unroll 4
                     for (int k8 = 0; k8 < k8n; ++k8) {
-                        umma_tf32(tmem_base, a0 + 2 * k8, b0 + 2 * k8, idesc, (it | k8) ? 1u : 0u);
-                        umma_tf32(tmem_base, al0 + 2 * k8, b0 + 2 * k8, idesc, 1u);
-                        umma_tf32(tmem_base, a0 + 2 * k8, bl0 + 2 * k8, idesc, 1u);
+                        umma_tf32(acc, a0 + 2 * k8, b0 + 2 * k8, idesc, (k | k8) ? 1u : 0u);
+                        umma_tf32(acc, al0 + 2 * k8, b0 + 2 * k8, idesc, 1u);
+                        umma_tf32(acc, a0 + 2 * k8, bl0 + 2 * k8, idesc, 1u);
                     }
                 } else {
 #pragma unroll 4
-                    for (int k8 = 0; k8 < k8n; ++k8) umma_tf32(tmem_base, a0 + 2 * k8, b0 + 2 * k8, idesc, (it | k8) ? 1u : 0u);
+                    for (int k8 = 0; k8 < k8n; ++k8) umma_tf32(acc, a0 + 2 * k8, b0 + 2 * k8, idesc, (k | k8) ? 1u : 0u);
                 }
                 umma_commit(empty0 + 8 * s);     // frees the stage once these MMAs have read it
                 if (++s == stages) { s = 0; par ^= 1u; }
+              }
+              if (live) umma_commit(accum_bar + 8 * j);      // tile j's accumulator is complete once these MMAs retire
             }
             consumed = it;
-            if (it == total) umma_commit(accum_bar);
             HPF_TL(6);
         }
     } else {
@@ -494,23 +521,26 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             const int row0 = tid / f4row, rstep = 256 / f4row;
             const int cph = tid % f4row;
             const int clog = p.kchunk == 32 ? (cph ^ (row0 & 7)) : (cph ^ ((row0 >> 1) & 3));
-            int px[4], py[4], pn[4];
+            const bool three = p.passes == 3;
+            const bool writer = blockIdx.y == 0;
+            int it = 0;
+            for (int tj = 0; tj < my_tiles && ok; ++tj) {
+              HPF_TILE_ORIGIN(tile0 + tj);
+              int px[4], py[4], pn[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+              for (int j = 0; j < 4; ++j) {
                 const int r = row0 + j * rstep;
                 const int wi = r % p.box_w, hi = (r / p.box_w) % p.box_h, ni = r / (p.box_w * p.box_h);
                 px[j] = q0 + wi; py[j] = p0 + hi;
                 pn[j] = (j < per && ni < p.box_n && n0 + ni < p.N) ? n0 + ni : -1;
-            }
-            const bool three = p.passes == 3;
-            const bool writer = blockIdx.y == 0;
-            for (int it = 0; it < total; ++it) {
+              }
+              for (int k = 0; k < total; ++k, ++it) {
                 const int s = it % p.stages;
                 ok = mbar_wait(full0 + 8 * s, (it / p.stages) & 1, &abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) { if (lane == 0) report(p.status, 7); break; }
                 if (it == 0 && tid == 0) HPF_TL(3);
-                const int tap = it / p.n_kchunks, kc = it - tap * p.n_kchunks;
+                const int tap = k / p.n_kchunks, kc = k - tap * p.n_kchunks;
                 const int dyy = tap / p.R - p.pad, dxx = tap % p.R - p.pad;
                 const int ch = kc * p.kchunk + 4 * clog;
                 const float4 mu = *reinterpret_cast<const float4*>(&bn_par[0][ch]);
@@ -546,10 +576,12 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                 __syncwarp();
                 if (lane == 0) mbar_arrive(split0 + 8 * s);
                 if (it == 0 && tid == 0) HPF_TL(4);
+              }
             }
         } else if (p.passes == 3) {
             const int per = (int)(p.a_bytes >> 12);     // float4 per thread: a_bytes / 16 / 256 = 2 or 4
-            for (int it = 0; it < total; ++it) {
+            const int all = my_tiles * total;
+            for (int it = 0; it < all; ++it) {
                 const int s = it % p.stages;
                 ok = mbar_wait(full0 + 8 * s, (it / p.stages) & 1, &abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
@@ -574,11 +606,17 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             }
         }
         (void)ok;
-        mbar_wait(accum_bar, 0, &abort_flag);
-        // every pipeline buffer is idle now (all MMAs completed, all copies landed): the tile is staged there
-        // so that the write-out is coalesced (a TMEM lane is a pixel: thread-per-row stores would touch 32 lines each)
+        // The write-out is staged through shared memory so that it is coalesced (a TMEM lane is a pixel: thread-per-row
+        // stores would touch 32 lines each).  With one tile per CTA the staging area is the pipeline itself, idle once
+        // the accumulator is complete; with several tiles it is a region of its own, because the next tile's loads and
+        // MMAs are in flight while this tile is written out.
         __shared__ int row_off[kTileM];                // offset (floats) of the pixel's channel row in the output, or -1
         __shared__ int row_fill[kTileM];               // strided data gradient: which neighbours of the sample exist
+        float* const stg = reinterpret_cast<float*>(smem + stg_off);
+        bool all_done = true;
+        for (int tj = 0; tj < my_tiles; ++tj) {
+        HPF_TILE_ORIGIN(tile0 + tj);
+        mbar_wait(accum_bar + 8 * tj, 0, &abort_flag);
         if (tid < kTileM) {
             const int wi = tid % p.box_w, hi = (tid / p.box_w) % p.box_h, ni = tid / (p.box_w * p.box_h);
             const int q = q0 + wi, pp = p0 + hi, n = n0 + ni;
@@ -592,15 +630,15 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
         const bool done = abort_flag == 0;             // uniform over the 8 warps after the barrier
+        all_done = all_done && done;
         if (done) {
             tc_fence_after();
-            if (tid == 0) HPF_TL(7);
+            if (tid == 0 && tj == 0) HPF_TL(7);
             // TMEM lane = pixel within the tile.  Two warps share each group of 32 lanes (a warp reaches lanes
             // 32*(warp%4) ..): they take alternate groups of 16 output channels.
             const int row = (warp & 3) * 32 + lane;
             const int half = (warp - 2) >> 2;
-            float* stg = reinterpret_cast<float*>(smem);
-            const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+            const uint32_t lane_addr = tmem_base + (uint32_t)tj * acc_cols + ((uint32_t)((warp & 3) * 32) << 16);
             for (int g0 = half * 16; g0 < p.n_chunk; g0 += 32) {
                 float v[16];
                 tmem_ld16_nowait(lane_addr + (uint32_t)g0, v);
@@ -617,9 +655,9 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
 #pragma unroll
                 for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
             }
-            if (tid == 0) HPF_TL(10);
+            if (tid == 0 && tj == 0) HPF_TL(10);
             asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (tid == 0) HPF_TL(11);
+            if (tid == 0 && tj == 0) HPF_TL(11);
             // write-out: consecutive threads write consecutive float4 of a pixel's channel row.  Eight warps cannot
             // hide latency by occupancy, so four independent float4 are in flight per thread and nothing is re-read.
             const int c4n = p.n_chunk >> 2;
@@ -684,17 +722,24 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                 // a thread kept one group of 4 channels throughout (256 is a multiple of c4n): add the 256 / c4n
                 // threads of each group in ascending order and store this tile's partial sums
                 asm volatile("bar.sync 1, 256;" ::: "memory");          // the staging area is free again
-                float4* red = reinterpret_cast<float4*>(smem);
+                float4* red = reinterpret_cast<float4*>(stg);
                 red[2 * tid] = sa; red[2 * tid + 1] = sb;
                 asm volatile("bar.sync 1, 256;" ::: "memory");
                 if (tid < c4n * 2) {
                     const int g = tid >> 1, which = tid & 1;
                     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                     for (int t2 = g; t2 < 256; t2 += c4n) { const float4 v2 = red[2 * t2 + which]; acc.x += v2.x; acc.y += v2.y; acc.z += v2.z; acc.w += v2.w; }
-                    float* dstp = p.stat_partials + ((size_t)blockIdx.x * 2 + which) * p.c_out + co0 + 4 * g;
+                    float* dstp = p.stat_partials + ((size_t)(tile0 + tj) * 2 + which) * p.c_out + co0 + 4 * g;
                     *reinterpret_cast<float4*>(dstp) = acc;
                     if (stat_mode == 1) __threadfence();
                 }
+            }
+        }
+        if (MULTI) asm volatile("bar.sync 1, 256;" ::: "memory");      // the staging area and the row tables serve the next tile
+        }   // tiles of this CTA
+        {
+            const int stat_mode = p.stat_mode;
+            if (stat_mode && all_done) {
                 // stat_mode 1: the CTA that finishes last turns the per-tile sums into mean and 1/sigma (tiles are added in
                 // a fixed order in fp64, so the result does not depend on which CTA that is).  stat_mode 3: the reading
                 // convolution adds the few per-tile sums itself, and this kernel ends without a ticket.
@@ -708,8 +753,8 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                 if (stat_mode == 1 && is_last) {
                     __threadfence();
                     float mu = 0.f, rs = 0.f;
-                    bn_combine_partials(p.stat_partials, (int)gridDim.x, p.c_out, p.stat_inv_rows, p.stat_eps,
-                                        reinterpret_cast<double (*)[4]>(smem), tid, &mu, &rs);
+                    bn_combine_partials(p.stat_partials, MULTI ? p.n_tiles : (int)gridDim.x, p.c_out, p.stat_inv_rows, p.stat_eps,
+                                        reinterpret_cast<double (*)[4]>(stg), tid, &mu, &rs);
                     if (tid < p.c_out) { p.stat_out[tid] = mu; p.stat_out[p.c_out + tid] = rs; }
                     if (tid == 0) *p.stat_ticket = 0u;
                 }
@@ -1267,7 +1312,9 @@ cudaError_t conv_tc_init()
     cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
     if (e != cudaSuccess) return e;
     if (q != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
-    e = cudaFuncSetAttribute(conv_tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
+    e = cudaFuncSetAttribute(conv_tc_fwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(conv_tc_fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(conv_tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWgradSmemBudget + 2048);
     if (e != cudaSuccess) return e;
@@ -1415,13 +1462,23 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
         p.bn_in_eps = fuse->in_eps; p.bn_in_inv_rows = fuse->in_rows > 0 ? 1.0 / (double)fuse->in_rows : 0.0;
     }
     p.stacked = (passes == 3 && 2 * n_chunk <= 256) ? 1 : 0;
-    p.tmem_cols = pow2_cols(p.stacked ? 2 * n_chunk : n_chunk);
+    p.acc_cols = (unsigned int)(p.stacked ? 2 * n_chunk : n_chunk);
     p.idesc = instr_desc(n_chunk, false, false);
     p.idesc2 = instr_desc(p.stacked ? 2 * n_chunk : n_chunk, false, false);
     p.stg_pitch = (unsigned int)n_chunk + 4u;
-    L->grid = dim3(p.tiles_w * p.tiles_h * tiles_n, v.c_out / n_chunk, 1);
-    L->smem = (unsigned int)stages * p.stage_bytes;
-    if (L->smem < (unsigned int)kTileM * p.stg_pitch * 4u) L->smem = (unsigned int)kTileM * p.stg_pitch * 4u;   // epilogue staging
+    p.n_tiles = p.tiles_w * p.tiles_h * tiles_n;
+    const unsigned int pipe_bytes = (unsigned int)stages * p.stage_bytes;
+    const unsigned int stg_bytes = (unsigned int)kTileM * p.stg_pitch * 4u;
+    // Two tiles per CTA when the launch is several waves long anyway: half as many CTAs, and the second tile's loads and
+    // MMAs hide under the first tile's write-out.  Needs twice the accumulator columns (two such CTAs must still fit
+    // the 512 columns of an SM) and a staging area beside the pipeline.  A launch of about a wave keeps one tile per
+    // CTA: there the duration of the launch is one CTA's own chain.
+    p.tiles_per_cta = 1;
+    if (p.n_tiles * (v.c_out / n_chunk) >= kMultiTileFrom && 2 * p.acc_cols <= 256 && pipe_bytes + stg_bytes <= 110u * 1024u) p.tiles_per_cta = 2;
+    p.tmem_cols = pow2_cols((int)p.acc_cols * p.tiles_per_cta);
+    p.stg_off = p.tiles_per_cta > 1 ? pipe_bytes : 0u;
+    L->grid = dim3((p.n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta, v.c_out / n_chunk, 1);
+    L->smem = p.tiles_per_cta > 1 ? pipe_bytes + stg_bytes : (pipe_bytes > stg_bytes ? pipe_bytes : stg_bytes);
     L->smem += 1024;
     plan->valid = 1;
     return cudaSuccess;
@@ -1444,7 +1501,8 @@ cudaError_t conv_tc_launch(const ConvTcPlan* plan, DeviceStatus* status, cudaStr
     }
     ConvTcFwdLaunch L = *reinterpret_cast<const ConvTcFwdLaunch*>(plan->storage);
     L.p.s.status = status;
-    launch_pdl(conv_tc_fwd_kernel, L.grid, dim3(320), L.smem, st, L.p);
+    if (L.p.s.tiles_per_cta > 1) launch_pdl(conv_tc_fwd_kernel<true>, L.grid, dim3(320), L.smem, st, L.p);
+    else launch_pdl(conv_tc_fwd_kernel<false>, L.grid, dim3(320), L.smem, st, L.p);
     count(n_launch, 1);
     return cudaGetLastError();
 }

@@ -61,6 +61,16 @@ def test_conv_sweep_tensor_core_path(shape, path):
         assert min(e) > 1e-5          # it really is the 11-bit path
 
 
+@pytest.mark.parametrize("shape", [(1, 1, 64, 16, 32), (3, 1, 16, 16, 32), (1, 1, 16, 64, 32), (1, 2, 64, 32, 32)],
+                         ids=lambda s: "k%d_s%d_%dto%d_at%d" % s)
+def test_conv_launches_of_several_waves_use_two_tiles_per_cta(shape):
+    """Batch 80 at 32x32: 640 pixel tiles, more than two CTAs per SM can hold at once, so the forward and data-gradient
+    launches give each CTA two tiles (the second tile's loads under the first tile's write-out)."""
+    ks, st, ci, co, H = shape
+    e = _conv_case(ks, st, ci, co, H, N=80, path=0)
+    assert max(e) <= 2e-5, e
+
+
 @pytest.mark.parametrize("shape", [(3, 1, 64, 64, 56), (1, 1, 256, 64, 56), (1, 2, 256, 128, 56), (3, 1, 128, 128, 28),
                                    (1, 1, 128, 512, 28), (3, 1, 256, 256, 14), (1, 2, 1024, 512, 14), (3, 1, 512, 512, 7),
                                    (1, 1, 512, 2048, 7), (1, 1, 2048, 512, 7)],
