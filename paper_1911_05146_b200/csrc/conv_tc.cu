@@ -1474,7 +1474,12 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     // the 512 columns of an SM) and a staging area beside the pipeline.  A launch of about a wave keeps one tile per
     // CTA: there the duration of the launch is one CTA's own chain.
     p.tiles_per_cta = 1;
-    if (p.n_tiles * (v.c_out / n_chunk) >= kMultiTileFrom && 2 * p.acc_cols <= 256 && pipe_bytes + stg_bytes <= 110u * 1024u) p.tiles_per_cta = 2;
+    if (p.n_tiles * (v.c_out / n_chunk) >= kMultiTileFrom && 2 * p.acc_cols <= 256 && pipe_bytes + stg_bytes <= 110u * 1024u) {
+        int t = (p.n_tiles * (v.c_out / n_chunk) + 295) / 296;            // tiles per CTA that bring the launch down to one wave
+        if (t > 4) t = 4;                                                 // accumulator barriers
+        while (t > 2 && (unsigned int)t * p.acc_cols > 256u) --t;
+        p.tiles_per_cta = t < 2 ? 2 : t;
+    }
     p.tmem_cols = pow2_cols((int)p.acc_cols * p.tiles_per_cta);
     p.stg_off = p.tiles_per_cta > 1 ? pipe_bytes : 0u;
     L->grid = dim3((p.n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta, v.c_out / n_chunk, 1);
