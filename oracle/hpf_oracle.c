@@ -60,7 +60,9 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { ORA_CONV = 1, ORA_BNRELU = 2, ORA_ADD = 3, ORA_MAXPOOL = 4, ORA_HEAD = 5 };
+/* BN = batch normalisation without the activation, RELU = the activation alone: the post-activation (v1) residual
+ * block is conv-BN-RELU-conv-BN, ADD with the shortcut, RELU. */
+enum { ORA_CONV = 1, ORA_BNRELU = 2, ORA_ADD = 3, ORA_MAXPOOL = 4, ORA_HEAD = 5, ORA_BN = 6, ORA_RELU = 7 };
 enum { ORA_OK = 0, ORA_EINVAL = -1, ORA_ENOMEM = -2 };
 
 typedef struct {
@@ -97,6 +99,8 @@ int ora_shapes(const ora_op *ops, int32_t n_ops, const int32_t in_hwc[3], int32_
             d[2] = o->c_out;
             break;
         case ORA_BNRELU:
+        case ORA_BN:
+        case ORA_RELU:
             if (o->c_in != C || o->c_out != C) return ORA_EINVAL;
             d[0] = H; d[1] = W; d[2] = C;
             break;
@@ -129,7 +133,7 @@ int ora_param_layout(const ora_op *ops, int32_t n_ops, int64_t *w_off, int64_t *
         const ora_op *o = &ops[i];
         int64_t wc = 0, bc = 0;
         if (o->kind == ORA_CONV) wc = (int64_t)o->c_out * o->ksize * o->ksize * o->c_in;
-        else if (o->kind == ORA_BNRELU) { wc = o->c_in; bc = o->c_in; }
+        else if (o->kind == ORA_BNRELU || o->kind == ORA_BN) { wc = o->c_in; bc = o->c_in; }
         else if (o->kind == ORA_HEAD) { wc = (int64_t)o->c_out * o->c_in; bc = o->c_out; }
         w_off[i] = at; w_cnt[i] = wc; at += wc;
         b_off[i] = at; b_cnt[i] = bc; at += bc;
@@ -369,6 +373,65 @@ void ora_bnrelu_bwd(const double *x, const double *dy, int64_t rows, int32_t C, 
     ora_bnrelu_bwd_dec(x, dy, rows, C, gamma, beta, eps, NULL, 0.0, NULL, dx, dgamma, dbeta);
 }
 
+/* Batch normalisation alone: y = gamma * (x - mean) / sqrt(var + eps) + beta (per-micro-batch statistics, biased
+ * variance), and its backward dx = gamma / sqrt(var+eps) * (dy - mean(dy) - xhat * mean(dy*xhat)). */
+void ora_bn_fwd(const double *x, int64_t rows, int32_t C, const double *gamma, const double *beta, double eps, double *y)
+{
+    double *mean = (double *)malloc(sizeof(double) * 2 * (size_t)C), *var = mean + C;
+    ora_bn_stats(x, rows, C, mean, var);
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < rows; ++i)
+        for (int32_t c = 0; c < C; ++c)
+            y[i * C + c] = gamma[c] * ((x[i * C + c] - mean[c]) / sqrt(var[c] + eps)) + beta[c];
+    free(mean);
+}
+
+void ora_bn_bwd(const double *x, const double *dy, int64_t rows, int32_t C, const double *gamma, double eps,
+                double *dx, double *dgamma, double *dbeta)
+{
+    double *mean = (double *)malloc(sizeof(double) * 2 * (size_t)C), *var = mean + C;
+    ora_bn_stats(x, rows, C, mean, var);
+#pragma omp parallel for schedule(static)
+    for (int32_t c = 0; c < C; ++c) {
+        double rstd = 1.0 / sqrt(var[c] + eps), sb = 0.0, sg = 0.0;
+        for (int64_t i = 0; i < rows; ++i) {
+            double xh = (x[i * C + c] - mean[c]) * rstd;
+            sb += dy[i * C + c]; sg += dy[i * C + c] * xh;
+        }
+        dbeta[c] = sb; dgamma[c] = sg;
+        for (int64_t i = 0; i < rows; ++i) {
+            double xh = (x[i * C + c] - mean[c]) * rstd;
+            dx[i * C + c] = gamma[c] * rstd * (dy[i * C + c] - sb / (double)rows - xh * sg / (double)rows);
+        }
+    }
+    free(mean);
+}
+
+/* y = max(x, 0) and dx = dy * [x > 0] (derivative 0 at 0).  decisions / tau / counts as in ora_bnrelu_bwd_dec,
+ * the window being |x| < tau. */
+void ora_relu_fwd(const double *x, int64_t n, double *y)
+{
+    for (int64_t i = 0; i < n; ++i) y[i] = x[i] > 0.0 ? x[i] : 0.0;
+}
+
+void ora_relu_bwd_dec(const double *x, const double *dy, int64_t n, const uint8_t *decisions, double tau,
+                      int64_t *counts, double *dx)
+{
+    int64_t n_used = 0, n_viol = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        int own = x[i] > 0.0, use = own;
+        if (decisions) {
+            int theirs = decisions[i] != 0;
+            if (theirs != own) {
+                if (fabs(x[i]) < tau) { use = theirs; ++n_used; }
+                else ++n_viol;
+            }
+        }
+        dx[i] = use ? dy[i] : 0.0;
+    }
+    if (counts) { counts[0] += n_used; counts[1] += n_viol; }
+}
+
 /* Window max with -infinity padding; argmax = first maximum in (r,s) row-major order. */
 void ora_maxpool_fwd(const double *x, int32_t N, int32_t H, int32_t W, int32_t C, int32_t R, int32_t st,
                      int32_t pad, double *y)
@@ -549,6 +612,12 @@ static void op_forward(const ora_ctx *c, int32_t i, const double *in0, const dou
         for (int64_t j = 0; j < n; ++j) out[j] = in0[j] + in1[j];
         break;
     }
+    case ORA_BN:
+        ora_bn_fwd(in0, (int64_t)c->b * s[0] * s[1], s[2], th + c->w_off[i], th + c->b_off[i], o->eps, out);
+        break;
+    case ORA_RELU:
+        ora_relu_fwd(in0, numel_of(c, i), out);
+        break;
     case ORA_MAXPOOL:
         ora_maxpool_fwd(in0, c->b, s[0], s[1], s[2], o->ksize, o->stride, o->pad, out);
         break;
@@ -589,6 +658,12 @@ static int op_backward(const ora_ctx *c, int32_t i, const double *in0, const dou
         if (d1) for (int64_t j = 0; j < n; ++j) d1[j] += dout[j];
         return ORA_OK;
     }
+    case ORA_BN:
+        ora_bn_bwd(in0, dout, (int64_t)c->b * s[0] * s[1], s[2], th + c->w_off[i], o->eps, tmp, g + c->w_off[i], g + c->b_off[i]);
+        break;
+    case ORA_RELU:
+        ora_relu_bwd_dec(in0, dout, n_in, c->decisions ? c->decisions[i] : NULL, c->tau, ((ora_ctx *)c)->counts, tmp);
+        break;
     case ORA_MAXPOOL:
         ora_maxpool_bwd(in0, dout, c->b, s[0], s[1], s[2], o->ksize, o->stride, o->pad, tmp);
         break;

@@ -13,7 +13,7 @@ import numpy as np
 
 from . import build as _build
 
-CONV, BNRELU, ADD, MAXPOOL, HEAD = 1, 2, 3, 4, 5
+CONV, BNRELU, ADD, MAXPOOL, HEAD, BN, RELU = 1, 2, 3, 4, 5, 6, 7
 
 
 class _Op(C.Structure):
@@ -238,9 +238,9 @@ def microbatch(ops, in_hwc, theta, x, labels, cuts=None, want=None, want_input_g
     """One micro-batch.  Returns a dict with loss, g, act{op}, dact{op} and, when
     ``cuts`` is given (partition-by-partition execution), fwd_msg / bwd_msg
     keyed by (cut index, position in the live set).  ``want`` limits which ops'
-    tensors are kept (default: all).  ``decisions`` maps a BNRELU op to the
+    tensors are kept (default: all).  ``decisions`` maps a BNRELU (or RELU) op to the
     (z > 0) decisions of another implementation, honoured inside the window
-    |z| < tau*|gamma|; the result then carries decisions_used / decision_violations."""
+    |z| < tau*|gamma| (RELU: |x| < tau); the result then carries decisions_used / decision_violations."""
     n = len(ops)
     b = x.shape[0]
     shp = shapes(ops, in_hwc)

@@ -20,6 +20,11 @@ def tiny_imagenet():
     return wl.resnet_v2_imagenet(blocks=(1, 1), widths=(4, 8), n_classes=7), (16, 16, 3)
 
 
+def tiny_v1():
+    """Post-activation basic blocks (BN without ReLU, ADD, ReLU), with a strided 3x3 and a projection shortcut."""
+    return wl.resnet_v1_cifar(1, widths=(4, 8), n_classes=5), (8, 8, 3)
+
+
 def _setup(builder, B, seed=0):
     ops, hwc = builder()
     x, labels = wl.draw_inputs(B, hwc, ops[-1].c_out, seed_x=100 + seed, seed_labels=200 + seed)
@@ -28,7 +33,7 @@ def _setup(builder, B, seed=0):
 
 
 # ------------------------------------------------------------------ P1
-@pytest.mark.parametrize("builder", [tiny_cifar, tiny_imagenet])
+@pytest.mark.parametrize("builder", [tiny_cifar, tiny_imagenet, tiny_v1])
 def test_finite_differences_every_backward_formula(builder):
     """Central differences of the step loss against the averaged gradient: pins
     every backward formula, the BN coupling across samples and the 1/M."""
@@ -84,7 +89,7 @@ def test_finite_differences_input_gradient():
 
 
 # ------------------------------------------------------------------ P2
-@pytest.mark.parametrize("builder", [tiny_cifar, tiny_imagenet])
+@pytest.mark.parametrize("builder", [tiny_cifar, tiny_imagenet, tiny_v1])
 def test_partition_count_invariance_bit_exact(builder):
     """Section 6.1's claim, partitioned == sequential, as a bit-exact identity:
     0, 1, 2 and 4 cuts, block-aligned and mid-block, give identical fp64 results."""
@@ -297,6 +302,10 @@ def _torch_step(ops, hwc, theta, x, labels, M):
             elif o.kind == wl.BNRELU:
                 y = F.relu(F.batch_norm(s0, None, None, t[w_off:w_off + w_cnt], t[b_off:b_off + b_cnt],
                                         training=True, eps=o.eps))
+            elif o.kind == wl.BN:
+                y = F.batch_norm(s0, None, None, t[w_off:w_off + w_cnt], t[b_off:b_off + b_cnt], training=True, eps=o.eps)
+            elif o.kind == wl.RELU:
+                y = F.relu(s0)
             elif o.kind == wl.ADD:
                 y = s0 + out[o.src1]
             elif o.kind == wl.MAXPOOL:
@@ -314,7 +323,7 @@ def _torch_step(ops, hwc, theta, x, labels, M):
     return np.array(slots), np.array(losses), acts, dacts
 
 
-@pytest.mark.parametrize("builder,B,M", [(tiny_cifar, 4, 2), (tiny_imagenet, 4, 2)])
+@pytest.mark.parametrize("builder,B,M", [(tiny_cifar, 4, 2), (tiny_imagenet, 4, 2), (tiny_v1, 4, 2)])
 def test_against_torch_autograd_small(builder, B, M):
     ops, hwc, x, labels, theta = _setup(builder, B=B, seed=1)
     slots, losses, acts, dacts = _torch_step(ops, hwc, theta, x, labels, M)
@@ -414,6 +423,36 @@ def test_supplied_relu_decisions_window():
     # partition-by-partition execution honours the decisions identically
     rp = ora.microbatch(ops, hwc, theta, x, labels, cuts=[4, 13], decisions=flipped, tau=tau)
     assert np.array_equal(rp["g"], r["g"]) and rp["decisions_used"] == 1
+
+
+def test_supplied_decisions_of_a_stand_alone_relu():
+    """The same rule for the RELU op of the post-activation block: the window is |x| < tau on the op's input, an
+    in-window flip changes exactly that element's gate (dx = dy there instead of 0, or the reverse)."""
+    ops, hwc, x, labels, theta = _setup(tiny_v1, B=4)
+    plain = ora.microbatch(ops, hwc, theta, x, labels)
+    relus = [i for i, o in enumerate(ops) if o.kind == wl.RELU]
+    assert relus
+    own = {i: (plain["act"][ops[i].src0] > 0).astype(np.uint8) for i in relus}
+    same = ora.microbatch(ops, hwc, theta, x, labels, decisions=own, tau=0.1)
+    assert np.array_equal(same["g"], plain["g"]) and same["decisions_used"] == 0 and same["decision_violations"] == 0
+    inv = {i: 1 - d for i, d in own.items()}
+    r = ora.microbatch(ops, hwc, theta, x, labels, decisions=inv, tau=0.0)
+    assert np.array_equal(r["g"], plain["g"]) and r["decision_violations"] == sum(d.size for d in own.values())
+    i = relus[-1]
+    xin = plain["act"][ops[i].src0]
+    flat = np.abs(xin).ravel()
+    j = int(np.argmin(flat))
+    two = np.sort(flat)[:2]
+    tau = 0.5 * (two[0] + two[1])
+    flipped = {k: v.copy() for k, v in own.items()}
+    flipped[i].reshape(-1)[j] ^= 1
+    r = ora.microbatch(ops, hwc, theta, x, labels, decisions=flipped, tau=tau)
+    assert r["decisions_used"] == 1 and r["decision_violations"] == 0
+    d_plain, d_flip, dy = plain["dact"][ops[i].src0].ravel(), r["dact"][ops[i].src0].ravel(), plain["dact"][i].ravel()
+    # the op's input has the RELU as its only reader here, so its gradient is the gated dy
+    if len([o for o in ops if o.src0 == ops[i].src0 or o.src1 == ops[i].src0]) == 1:
+        assert d_flip[j] == (dy[j] if flipped[i].reshape(-1)[j] else 0.0)
+        assert np.array_equal(np.delete(d_flip, j), np.delete(d_plain, j))
 
 
 # ---------------------------------------------------------------- parameter update (Section 5.3, apply_gradients)

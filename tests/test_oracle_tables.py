@@ -57,6 +57,23 @@ def test_keras_width_variant_has_the_parameter_count_the_paper_quotes():
     assert len(ops) == 21 * n + 6
 
 
+def test_depth_and_counts_of_resnet110_v1():
+    """The paper's ResNet-110 is the post-activation basic-block net: depth 6n+2 with n = 18 (Section 6.1 names the
+    model); closed-form parameter count, independent of the op loop."""
+    n = 18
+    ops = wl.resnet_v1_cifar(n)
+    weight_layers = sum(1 for o in ops if o.kind == wl.CONV and o.ksize == 3) + 1      # 3x3 convolutions + FC
+    assert weight_layers == 6 * n + 2 == 110
+    G = 3 * 9 * 16 + 2 * 16
+    c_t = 16
+    for w in (16, 32, 64):
+        first = 9 * c_t * w + 2 * w + 9 * w * w + 2 * w + (c_t * w if c_t != w else 0)
+        G += first + (n - 1) * (2 * (9 * w * w + 2 * w))
+        c_t = w
+    G += 64 * 10 + 10
+    assert ora.param_layout(ops)[4] == G == wl.param_offsets(ops)[1]
+
+
 def test_param_layout_is_dense_and_ordered():
     ops = wl.resnet_v2_imagenet(blocks=(1, 1), widths=(4, 8), n_classes=7)
     w_off, w_cnt, b_off, b_cnt, G = ora.param_layout(ops)

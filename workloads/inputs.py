@@ -8,7 +8,7 @@ beta = 0, FC weights ~ N(0, 2/C) and FC bias = 0.
 """
 import numpy as np
 
-from .resnet_spec import CONV, BNRELU, HEAD, MAXPOOL
+from .resnet_spec import CONV, BNRELU, BN, HEAD, MAXPOOL
 
 SEED_X, SEED_LABELS, SEED_PARAMS = 1911, 5146, 2020
 
@@ -34,7 +34,7 @@ def param_offsets(ops):
         wc = bc = 0
         if o.kind == CONV:
             wc = o.c_out * o.ksize * o.ksize * o.c_in
-        elif o.kind == BNRELU:
+        elif o.kind in (BNRELU, BN):
             wc = bc = o.c_in
         elif o.kind == HEAD:
             wc, bc = o.c_out * o.c_in, o.c_out
@@ -59,7 +59,7 @@ def draw_params(ops, seed=SEED_PARAMS, bn_jitter=0.0):
         if o.kind == CONV:
             fan_in = o.c_in * o.ksize * o.ksize
             theta[w_off:w_off + w_cnt] = (rng.standard_normal(w_cnt) * np.sqrt(2.0 / fan_in)).astype(np.float32)
-        elif o.kind == BNRELU:
+        elif o.kind in (BNRELU, BN):
             theta[w_off:w_off + w_cnt] = 1.0
             if bn_jitter:
                 theta[w_off:w_off + w_cnt] += (bn_jitter * rng.standard_normal(w_cnt)).astype(np.float32)

@@ -8,7 +8,7 @@ projection, which reads the raw block input; there is no BN after the stem.
 """
 from collections import namedtuple
 
-CONV, BNRELU, ADD, MAXPOOL, HEAD = 1, 2, 3, 4, 5
+CONV, BNRELU, ADD, MAXPOOL, HEAD, BN, RELU = 1, 2, 3, 4, 5, 6, 7
 Op = namedtuple("Op", "kind src0 src1 c_in c_out ksize stride pad eps")
 EPS = 1e-5
 
@@ -46,6 +46,31 @@ def resnet_v2_cifar(n, widths=(16, 32, 64), n_classes=10, in_ch=3, outs=None):
     return ops
 
 
+def resnet_v1_cifar(n, widths=(16, 32, 64), n_classes=10, in_ch=3):
+    """Post-activation (v1) basic-block ResNet of depth 6n+2, the Keras example's definition: 3x3 stem conv, BN, ReLU;
+    per block conv3x3 (stride 2 in the first block of stages 2 and 3), BN, ReLU, conv3x3, BN, ADD with the shortcut
+    (a 1x1 stride-2 convolution of the block input where the shape changes, identity elsewhere), ReLU; then the head.
+    Convolution biases are left out: in front of a BN they are absorbed by its shift."""
+    ops = [Op(CONV, -1, -1, in_ch, widths[0], 3, 1, 1, 0.0)]
+    ops.append(Op(BNRELU, 0, -1, widths[0], widths[0], 0, 1, 0, EPS))
+    t, c_t = 1, widths[0]
+    for si, w in enumerate(widths):
+        for bi in range(n):
+            s = 2 if (si > 0 and bi == 0) else 1
+            ops.append(Op(CONV, t, -1, c_t, w, 3, s, 1, 0.0)); c1 = len(ops) - 1
+            ops.append(Op(BNRELU, c1, -1, w, w, 0, 1, 0, EPS)); a1 = len(ops) - 1
+            ops.append(Op(CONV, a1, -1, w, w, 3, 1, 1, 0.0)); c2 = len(ops) - 1
+            ops.append(Op(BN, c2, -1, w, w, 0, 1, 0, EPS)); b2 = len(ops) - 1
+            short = t
+            if s != 1 or c_t != w:
+                ops.append(Op(CONV, t, -1, c_t, w, 1, s, 0, 0.0)); short = len(ops) - 1
+            ops.append(Op(ADD, b2, short, w, w, 0, 1, 0, 0.0)); ad = len(ops) - 1
+            ops.append(Op(RELU, ad, -1, w, w, 0, 1, 0, 0.0)); t = len(ops) - 1
+            c_t = w
+    ops.append(Op(HEAD, t, -1, c_t, n_classes, 0, 1, 0, 0.0))
+    return ops
+
+
 def resnet_v2_imagenet(blocks=(3, 8, 36, 3), widths=(64, 128, 256, 512), n_classes=1000, in_ch=3):
     """7x7 stride-2 stem, 3x3 stride-2 max-pool, four bottleneck stages."""
     ops = [Op(CONV, -1, -1, in_ch, widths[0], 7, 2, 3, 0.0),
@@ -70,6 +95,9 @@ CONFIGS = {
     # the ~30 M-parameter width variant of ResNet-1001 (Section 6.3 quotes that size) and a short net of the same widths
     "r1001k": (lambda: resnet_v2_cifar(111, (16, 64, 128), outs=(64, 128, 256)), (32, 32, 3), 128, 8, 8),
     "r20k":   (lambda: resnet_v2_cifar(2, (16, 64, 128), outs=(64, 128, 256)), (32, 32, 3), 16, 2, 2),
+    # the paper's ResNet-110 is the post-activation (v1) basic-block net, depth 6n+2 with n = 18; a short one for tests
+    "r110v1": (lambda: resnet_v1_cifar(18), (32, 32, 3), 128, 4, 4),
+    "r8v1":   (lambda: resnet_v1_cifar(1), (32, 32, 3), 8, 2, 2),
 }
 
 
