@@ -50,11 +50,14 @@ typedef enum {
     HPF_ERR_TIMEOUT = -6      /* hpf_synchronize deadline passed, or a bounded device-side wait gave up */
 } hpf_status;
 
-typedef enum { HPF_OP_CONV = 1, HPF_OP_BNRELU = 2, HPF_OP_ADD = 3, HPF_OP_MAXPOOL = 4, HPF_OP_HEAD = 5 } hpf_op_kind;
+typedef enum { HPF_OP_CONV = 1, HPF_OP_BNRELU = 2, HPF_OP_ADD = 3, HPF_OP_MAXPOOL = 4, HPF_OP_HEAD = 5, HPF_OP_BN = 6,
+               HPF_OP_RELU = 7 } hpf_op_kind;
 
 /* One entry of the layer list.
  *   CONV    cross-correlation, zero padding, no bias: ksize x ksize, stride, pad; c_in -> c_out
  *   BNRELU  training-mode batch norm over the micro-batch (biased variance) followed by ReLU; c_in == c_out
+ *   BN      the same batch norm without the activation, RELU the activation alone (max(x, 0), derivative 0 at 0): the
+ *           post-activation residual block is CONV BNRELU CONV BN, ADD with the shortcut, RELU; c_in == c_out
  *   ADD     src0 + src1 (residual join)
  *   MAXPOOL ksize x ksize window, stride, pad (padding never wins)
  *   HEAD    mean over (h,w), fully connected to c_out classes, softmax cross-entropy, mean over the

@@ -58,11 +58,16 @@ struct DeviceStatus { unsigned int code; unsigned int detail; };
 size_t bn_scratch_bytes(int64_t rows, int C);
 // scratch: first 256 bytes hold the block ticket (must be zero before the first use; the kernels
 // leave it zero), the rest holds per-block partial sums.
+// relu = false: batch normalisation without the activation (the post-activation block's second BN)
 cudaError_t bnrelu_fwd(const float* x, const float* gamma, const float* beta, float eps, float* y, float* stats,
-                       int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch);
+                       int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch, bool relu = true);
 cudaError_t bnrelu_bwd(const float* x, const float* dy, const float* gamma, const float* beta, const float* stats,
                        float* dx, const float* addend, bool accumulate, float* dgamma, float* dbeta,
-                       int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch);
+                       int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch, bool relu = true);
+// stand-alone ReLU: y = max(x, 0); dx (+= if accumulate) = dy * [x > 0] (+ addend)
+cudaError_t relu_fwd(const float* x, float* y, int64_t n, cudaStream_t st, int64_t* n_launch);
+cudaError_t relu_bwd(const float* x, const float* dy, float* dx, const float* addend, bool accumulate, int64_t n, cudaStream_t st,
+                     int64_t* n_launch);
 // The forward's second half alone: the statistics (mean[C], rstd[C]) were left by the convolution kernel that produced x.
 cudaError_t bnrelu_fwd_apply(const float* x, const float* gamma, const float* beta, const float* stats, float* y,
                              int64_t rows, int C, cudaStream_t st, int64_t* n_launch);

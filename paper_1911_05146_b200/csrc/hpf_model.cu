@@ -180,7 +180,13 @@ int build_ops(hpf_model* mdl, const hpf_op* ops, int n_ops)
             o.C = q.c_out;
             if (q.kind == HPF_OP_CONV) wc = (int64_t)q.c_out * q.ksize * q.ksize * q.c_in;
             break;
+        case HPF_OP_RELU:
+            if (q.c_in != o.iC || q.c_out != o.iC) return fail(HPF_ERR_INVALID, "RELU channel count mismatch");
+            if (q.src0 < 0) return fail(HPF_ERR_UNSUPPORTED, "RELU directly on the network input");
+            o.H = o.iH; o.W = o.iW; o.C = o.iC;
+            break;
         case HPF_OP_BNRELU:
+        case HPF_OP_BN:
             if (q.c_in != o.iC || q.c_out != o.iC) return fail(HPF_ERR_INVALID, "BN channel count mismatch");
             if (o.iC % 4) return fail(HPF_ERR_UNSUPPORTED, "BN channel count must be a multiple of 4");
             if (q.src0 < 0) return fail(HPF_ERR_UNSUPPORTED, "BN directly on the network input");
@@ -418,7 +424,7 @@ void build_memory_plan(hpf_model* mdl)
     for (int p = 0; p < P; ++p) {
         size_t bn = 256, part = 0;
         for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i)
-            if (mdl->ops[i].op.kind == HPF_OP_BNRELU) {
+            if (mdl->ops[i].op.kind == HPF_OP_BNRELU || mdl->ops[i].op.kind == HPF_OP_BN) {
                 const OpInfo& o = mdl->ops[i];
                 size_t need = bn_scratch_bytes((int64_t)mdl->b * o.H * o.W, o.C);
                 if (need > bn) bn = need;
@@ -472,7 +478,8 @@ void build_memory_plan(hpf_model* mdl)
             else mdl->grad_off[(size_t)m * n + i] = take(sizeof(float) * (size_t)mdl->numel(i));
         }
         for (int i = 0; i < n; ++i)
-            if (mdl->ops[i].op.kind == HPF_OP_BNRELU) mdl->stats_off[(size_t)m * n + i] = take(sizeof(float) * 2 * (size_t)mdl->ops[i].C);
+            if (mdl->ops[i].op.kind == HPF_OP_BNRELU || mdl->ops[i].op.kind == HPF_OP_BN)
+                mdl->stats_off[(size_t)m * n + i] = take(sizeof(float) * 2 * (size_t)mdl->ops[i].C);
     }
     mdl->fmsg_off.assign(mdl->cuts.size(), {}); mdl->bmsg_off.assign(mdl->cuts.size(), {});
     if (mdl->opt_messages)
@@ -538,6 +545,13 @@ int forward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
             CU(bnrelu_fwd(in0, mdl->params + o.w_off, mdl->params + o.b_off, q.eps, out, mdl->stats(i, m),
                           (int64_t)mdl->b * o.H * o.W, o.C, mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
         break;
+    case HPF_OP_BN:                        // batch normalisation without the activation
+        CU(bnrelu_fwd(in0, mdl->params + o.w_off, mdl->params + o.b_off, q.eps, out, mdl->stats(i, m),
+                      (int64_t)mdl->b * o.H * o.W, o.C, mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches, false));
+        break;
+    case HPF_OP_RELU:
+        CU(relu_fwd(in0, out, mdl->numel(i), st, &mdl->launches));
+        break;
     case HPF_OP_ADD:
         if (mdl->add_done_by[i] < 0) CU(add_fwd(in0, mdl->act(q.src1, m), out, mdl->numel(i), st, &mdl->launches));
         break;
@@ -596,6 +610,14 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
         CU(bnrelu_bwd(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m), addend,
                       e.accumulate != 0, slot + o.w_off, slot + o.b_off, (int64_t)mdl->b * o.H * o.W, o.C,
                       mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
+        break;
+    case HPF_OP_BN:
+        CU(bnrelu_bwd(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m), addend,
+                      e.accumulate != 0, slot + o.w_off, slot + o.b_off, (int64_t)mdl->b * o.H * o.W, o.C,
+                      mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches, false));
+        break;
+    case HPF_OP_RELU:
+        CU(relu_bwd(in0, dout, mdl->grad(q.src0, m), addend, e.accumulate != 0, mdl->numel(i), st, &mdl->launches));
         break;
     case HPF_OP_ADD:
         break;   // its contributions are aliases, on-the-fly addends, or the explicit accumulations above
@@ -916,6 +938,8 @@ int hpf_estimate_op_costs(const hpf_op* ops, int32_t n_ops, const int32_t in_sha
             break;
         }
         case HPF_OP_BNRELU: c = 9.0 + 20.0 * out_el / bytes_per_us; break;
+        case HPF_OP_BN: c = 18.0 + 20.0 * out_el / bytes_per_us; break;        // its own reduce + apply kernels, both ways
+        case HPF_OP_RELU: c = 6.0 + 20.0 * out_el / bytes_per_us; break;
         case HPF_OP_ADD: c = 0.0; break;                       // fused into the producing convolution
         case HPF_OP_MAXPOOL: c = 6.0 + 4.0 * 2.0 * (in_el + out_el) / bytes_per_us; break;
         default: c = 20.0; break;                               // head: a handful of tiny kernels

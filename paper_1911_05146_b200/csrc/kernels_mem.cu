@@ -19,8 +19,9 @@ constexpr int kMaxBlocks = 148 * 4;
 __host__ __device__ inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
 // ------------------------------------------------------------------------------------------------
-// BN + ReLU.  z = gamma * ((x - mean) * rstd) + beta, y = max(z, 0).  The same expression is used by
-// the forward and by the backward mask, so both take the ReLU decision on identical fp32 values.
+// BN + ReLU.  z = gamma * ((x - mean) * rstd) + beta, y = max(z, floor).  The same expression is used by
+// the forward and by the backward mask (z > floor), so both take the ReLU decision on identical fp32 values.
+// floor = 0 is BN+ReLU; floor = -infinity is batch normalisation without the activation (every element passes).
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ float bn_xhat(float x, float mean, float rstd) { return (x - mean) * rstd; }
 __device__ __forceinline__ float bn_z(float xh, float g, float b) { return fmaf(g, xh, b); }
@@ -79,7 +80,7 @@ bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, cons
                  const float* __restrict__ beta, const float* __restrict__ stats, float eps, int64_t rows, int C,
                  int cgt, int rl, int passes, int64_t rows_per_blk, unsigned int* ticket,
                  float* __restrict__ partials, float* __restrict__ out_a, float* __restrict__ out_b,
-                 float* __restrict__ coef)
+                 float* __restrict__ coef, float floor)
 {
     __shared__ double shd[kBnThreads][8];            // 32 KB; the float phase uses it as float[kBnThreads][8]
     float (*sh)[8] = reinterpret_cast<float (*)[8]>(&shd[0][0]);
@@ -118,10 +119,10 @@ bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, cons
                 if (BWD) {
                     const float4 g = __ldg(dp + k * step);
                     float xh, dz;
-                    xh = bn_xhat(v.x, p0.x, p1.x); dz = bn_z(xh, gm.x, bt.x) > 0.f ? g.x : 0.f; a.x += dz; b.x = fmaf(dz, xh, b.x);
-                    xh = bn_xhat(v.y, p0.y, p1.y); dz = bn_z(xh, gm.y, bt.y) > 0.f ? g.y : 0.f; a.y += dz; b.y = fmaf(dz, xh, b.y);
-                    xh = bn_xhat(v.z, p0.z, p1.z); dz = bn_z(xh, gm.z, bt.z) > 0.f ? g.z : 0.f; a.z += dz; b.z = fmaf(dz, xh, b.z);
-                    xh = bn_xhat(v.w, p0.w, p1.w); dz = bn_z(xh, gm.w, bt.w) > 0.f ? g.w : 0.f; a.w += dz; b.w = fmaf(dz, xh, b.w);
+                    xh = bn_xhat(v.x, p0.x, p1.x); dz = bn_z(xh, gm.x, bt.x) > floor ? g.x : 0.f; a.x += dz; b.x = fmaf(dz, xh, b.x);
+                    xh = bn_xhat(v.y, p0.y, p1.y); dz = bn_z(xh, gm.y, bt.y) > floor ? g.y : 0.f; a.y += dz; b.y = fmaf(dz, xh, b.y);
+                    xh = bn_xhat(v.z, p0.z, p1.z); dz = bn_z(xh, gm.z, bt.z) > floor ? g.z : 0.f; a.z += dz; b.z = fmaf(dz, xh, b.z);
+                    xh = bn_xhat(v.w, p0.w, p1.w); dz = bn_z(xh, gm.w, bt.w) > floor ? g.w : 0.f; a.w += dz; b.w = fmaf(dz, xh, b.w);
                 } else {
                     float d;
                     d = v.x - p0.x; a.x += d; b.x = fmaf(d, d, b.x);
@@ -214,7 +215,7 @@ bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, cons
 __global__ void __launch_bounds__(kBnThreads)
 bn_apply_fwd_kernel(const float4* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
                     const float* __restrict__ stats, float4* __restrict__ y, int64_t rows, int C, int cgt, int rl,
-                    int passes, int64_t rows_per_blk)
+                    int passes, int64_t rows_per_blk, float floor)
 {
     pdl_launch_dependents();
     pdl_wait();
@@ -237,19 +238,19 @@ bn_apply_fwd_kernel(const float4* __restrict__ x, const float* __restrict__ gamm
         for (int k = 0; k < n; ++k) {
             const float4 v = __ldg(x + base + k * step);
             float4 o;
-            o.x = fmaxf(bn_z(bn_xhat(v.x, mu.x, rs.x), g.x, b.x), 0.f);
-            o.y = fmaxf(bn_z(bn_xhat(v.y, mu.y, rs.y), g.y, b.y), 0.f);
-            o.z = fmaxf(bn_z(bn_xhat(v.z, mu.z, rs.z), g.z, b.z), 0.f);
-            o.w = fmaxf(bn_z(bn_xhat(v.w, mu.w, rs.w), g.w, b.w), 0.f);
+            o.x = fmaxf(bn_z(bn_xhat(v.x, mu.x, rs.x), g.x, b.x), floor);
+            o.y = fmaxf(bn_z(bn_xhat(v.y, mu.y, rs.y), g.y, b.y), floor);
+            o.z = fmaxf(bn_z(bn_xhat(v.z, mu.z, rs.z), g.z, b.z), floor);
+            o.w = fmaxf(bn_z(bn_xhat(v.w, mu.w, rs.w), g.w, b.w), floor);
             y[base + k * step] = o;
         }
     }
 }
 
-__device__ __forceinline__ float bn_dx1(float x, float dy, float mu, float rs, float g, float b, float ca, float cb)
+__device__ __forceinline__ float bn_dx1(float x, float dy, float mu, float rs, float g, float b, float ca, float cb, float floor)
 {
     const float xh = bn_xhat(x, mu, rs);
-    const float dz = bn_z(xh, g, b) > 0.f ? dy : 0.f;
+    const float dz = bn_z(xh, g, b) > floor ? dy : 0.f;
     return g * rs * (dz - ca - xh * cb);
 }
 
@@ -258,7 +259,7 @@ __global__ void __launch_bounds__(kBnThreads)
 bn_apply_bwd_kernel(const float4* __restrict__ x, const float4* __restrict__ dy, const float* __restrict__ gamma,
                     const float* __restrict__ beta, const float* __restrict__ stats, const float* __restrict__ coef,
                     const float4* __restrict__ addend, float4* __restrict__ dx, int64_t rows, int C, int cgt, int rl,
-                    int passes, int64_t rows_per_blk)
+                    int passes, int64_t rows_per_blk, float floor)
 {
     pdl_launch_dependents();
     pdl_wait();
@@ -285,10 +286,10 @@ bn_apply_bwd_kernel(const float4* __restrict__ x, const float4* __restrict__ dy,
             const float4 v = __ldg(x + i);
             const float4 d = __ldg(dy + i);
             float4 o;
-            o.x = bn_dx1(v.x, d.x, mu.x, rs.x, g.x, b.x, ca.x, cb.x);
-            o.y = bn_dx1(v.y, d.y, mu.y, rs.y, g.y, b.y, ca.y, cb.y);
-            o.z = bn_dx1(v.z, d.z, mu.z, rs.z, g.z, b.z, ca.z, cb.z);
-            o.w = bn_dx1(v.w, d.w, mu.w, rs.w, g.w, b.w, ca.w, cb.w);
+            o.x = bn_dx1(v.x, d.x, mu.x, rs.x, g.x, b.x, ca.x, cb.x, floor);
+            o.y = bn_dx1(v.y, d.y, mu.y, rs.y, g.y, b.y, ca.y, cb.y, floor);
+            o.z = bn_dx1(v.z, d.z, mu.z, rs.z, g.z, b.z, ca.z, cb.z, floor);
+            o.w = bn_dx1(v.w, d.w, mu.w, rs.w, g.w, b.w, ca.w, cb.w, floor);
             if (ADDEND) { const float4 e = __ldg(addend + i); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
             if (ACCUM) { const float4 e = dx[i]; o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
             dx[i] = o;
@@ -320,6 +321,47 @@ add_kernel(const float* __restrict__ a, const float* __restrict__ b, float* __re
         reinterpret_cast<float4*>(out)[i] = make_float4(u.x + v.x, u.y + v.y, u.z + v.z, u.w + v.w);
     }
     for (int64_t i = n4 * 4 + t0; i < n; i += stride) out[i] = a[i] + b[i];
+}
+
+// Stand-alone ReLU (the post-activation residual block ends in one): y = max(x, 0); dx = dy * [x > 0] (+ addend) (+= dx).
+__global__ void __launch_bounds__(kThreads)
+relu_fwd_kernel(const float* __restrict__ x, float* __restrict__ y, int64_t n)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int64_t n4 = n / 4;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (int64_t i = t0; i < n4; i += stride) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(x) + i);
+        reinterpret_cast<float4*>(y)[i] = make_float4(fmaxf(v.x, 0.f), fmaxf(v.y, 0.f), fmaxf(v.z, 0.f), fmaxf(v.w, 0.f));
+    }
+    for (int64_t i = n4 * 4 + t0; i < n; i += stride) y[i] = fmaxf(x[i], 0.f);
+}
+
+template <bool ADDEND, bool ACCUM>
+__global__ void __launch_bounds__(kThreads)
+relu_bwd_kernel(const float* __restrict__ x, const float* __restrict__ dy, const float* __restrict__ addend,
+                float* __restrict__ dx, int64_t n)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int64_t n4 = n / 4;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (int64_t i = t0; i < n4; i += stride) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(x) + i), d = __ldg(reinterpret_cast<const float4*>(dy) + i);
+        float4 o = make_float4(v.x > 0.f ? d.x : 0.f, v.y > 0.f ? d.y : 0.f, v.z > 0.f ? d.z : 0.f, v.w > 0.f ? d.w : 0.f);
+        if (ADDEND) { const float4 e = __ldg(reinterpret_cast<const float4*>(addend) + i); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+        if (ACCUM) { const float4 e = reinterpret_cast<const float4*>(dx)[i]; o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+        reinterpret_cast<float4*>(dx)[i] = o;
+    }
+    for (int64_t i = n4 * 4 + t0; i < n; i += stride) {
+        float o = x[i] > 0.f ? dy[i] : 0.f;
+        if (ADDEND) o += addend[i];
+        if (ACCUM) o += dx[i];
+        dx[i] = o;
+    }
 }
 
 template <bool ACCUM>
@@ -634,37 +676,39 @@ size_t bn_scratch_bytes(int64_t rows, int C)
 }
 
 cudaError_t bnrelu_fwd(const float* x, const float* gamma, const float* beta, float eps, float* y, float* stats,
-                       int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch)
+                       int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch, bool relu)
 {
     const BnPlan p = bn_plan(rows, C);
+    const float floor = relu ? 0.f : -INFINITY;
     unsigned int* ticket = reinterpret_cast<unsigned int*>(scratch);
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + 256);
     launch_pdl(bn_reduce_kernel<false>, p.nblk, kBnThreads, 0, st, x, (const float*)nullptr, gamma, beta, (const float*)nullptr, eps, rows, C, p.cgt, p.rl,
                                                            p.passes, p.rows_per_blk, ticket, partials, stats, stats + C,
-                                                           (float*)nullptr);
+                                                           (float*)nullptr, floor);
     launch_pdl(bn_apply_fwd_kernel, p.nblk_apply, kBnThreads, 0, st, reinterpret_cast<const float4*>(x), gamma, beta, stats,
                                                              reinterpret_cast<float4*>(y), rows, C, p.cgt, p.rl, p.passes,
-                                                             p.rows_per_blk_apply);
+                                                             p.rows_per_blk_apply, floor);
     count(n_launch, 2);
     return cudaGetLastError();
 }
 
 cudaError_t bnrelu_bwd(const float* x, const float* dy, const float* gamma, const float* beta, const float* stats,
                        float* dx, const float* addend, bool accumulate, float* dgamma, float* dbeta, int64_t rows,
-                       int C, void* scratch, cudaStream_t st, int64_t* n_launch)
+                       int C, void* scratch, cudaStream_t st, int64_t* n_launch, bool relu)
 {
     const BnPlan p = bn_plan(rows, C);
+    const float floor = relu ? 0.f : -INFINITY;
     unsigned int* ticket = reinterpret_cast<unsigned int*>(scratch);
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + 256);
     float* coef = partials + (size_t)p.nblk * 2 * C;
     launch_pdl(bn_reduce_kernel<true>, p.nblk, kBnThreads, 0, st, x, dy, gamma, beta, stats, 0.f, rows, C, p.cgt, p.rl, p.passes,
-                                                          p.rows_per_blk, ticket, partials, dbeta, dgamma, coef);
+                                                          p.rows_per_blk, ticket, partials, dbeta, dgamma, coef, floor);
     const float4* x4 = reinterpret_cast<const float4*>(x);
     const float4* dy4 = reinterpret_cast<const float4*>(dy);
     const float4* ad4 = reinterpret_cast<const float4*>(addend);
     float4* dx4 = reinterpret_cast<float4*>(dx);
     const int nb = p.nblk_apply;
-#define HPF_BN_APPLY(A, B) launch_pdl(bn_apply_bwd_kernel<A, B>, nb, kBnThreads, 0, st, x4, dy4, gamma, beta, stats, coef, ad4, dx4, rows, C, p.cgt, p.rl, p.passes, p.rows_per_blk_apply)
+#define HPF_BN_APPLY(A, B) launch_pdl(bn_apply_bwd_kernel<A, B>, nb, kBnThreads, 0, st, x4, dy4, gamma, beta, stats, coef, ad4, dx4, rows, C, p.cgt, p.rl, p.passes, p.rows_per_blk_apply, floor)
     if (addend && accumulate) HPF_BN_APPLY(true, true);
     else if (addend) HPF_BN_APPLY(true, false);
     else if (accumulate) HPF_BN_APPLY(false, true);
@@ -679,7 +723,26 @@ cudaError_t bnrelu_fwd_apply(const float* x, const float* gamma, const float* be
 {
     const BnPlan p = bn_plan(rows, C);
     launch_pdl(bn_apply_fwd_kernel, p.nblk_apply, kBnThreads, 0, st, reinterpret_cast<const float4*>(x), gamma, beta, stats,
-               reinterpret_cast<float4*>(y), rows, C, p.cgt, p.rl, p.passes, p.rows_per_blk_apply);
+               reinterpret_cast<float4*>(y), rows, C, p.cgt, p.rl, p.passes, p.rows_per_blk_apply, 0.f);
+    count(n_launch, 1);
+    return cudaGetLastError();
+}
+
+cudaError_t relu_fwd(const float* x, float* y, int64_t n, cudaStream_t st, int64_t* n_launch)
+{
+    launch_pdl(relu_fwd_kernel, ew_blocks(n / 4 + 1), kThreads, 0, st, x, y, n);
+    count(n_launch, 1);
+    return cudaGetLastError();
+}
+
+cudaError_t relu_bwd(const float* x, const float* dy, float* dx, const float* addend, bool accumulate, int64_t n, cudaStream_t st,
+                     int64_t* n_launch)
+{
+    const int nb = ew_blocks(n / 4 + 1);
+    if (addend && accumulate) launch_pdl(relu_bwd_kernel<true, true>, nb, kThreads, 0, st, x, dy, addend, dx, n);
+    else if (addend) launch_pdl(relu_bwd_kernel<true, false>, nb, kThreads, 0, st, x, dy, addend, dx, n);
+    else if (accumulate) launch_pdl(relu_bwd_kernel<false, true>, nb, kThreads, 0, st, x, dy, addend, dx, n);
+    else launch_pdl(relu_bwd_kernel<false, false>, nb, kThreads, 0, st, x, dy, addend, dx, n);
     count(n_launch, 1);
     return cudaGetLastError();
 }

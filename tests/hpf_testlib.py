@@ -95,7 +95,7 @@ def matched_oracle(bd, m, theta, x, labels, cuts=None, want=None, tau=TAU):
     forward tolerance does not leave open."""
     from oracle import reference as ora
     b = bd.B // bd.M
-    dec = {i: (bd.tensor(i, m) > 0).astype(np.uint8) for i, o in enumerate(bd.ops) if o.kind == wl.BNRELU}
+    dec = {i: (bd.tensor(i, m) > 0).astype(np.uint8) for i, o in enumerate(bd.ops) if o.kind in (wl.BNRELU, wl.RELU)}
     r = ora.microbatch(bd.ops, bd.in_hwc, theta, x[m * b:(m + 1) * b], labels[m * b:(m + 1) * b], cuts=cuts, want=want,
                        decisions=dec, tau=tau)
     assert r["decision_violations"] == 0, r["decision_violations"]

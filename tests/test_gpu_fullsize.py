@@ -68,3 +68,8 @@ def test_keras_width_variant_resnet1001_batch128():
 
 def test_config5_resnet152_imagenet_layout_batch64():
     _fullsize("r152", sample_m=[2])
+
+
+def test_resnet110_v1_batch128():
+    """The paper's ResNet-110 (post-activation basic blocks, depth 6*18+2), batch 128, 4 partitions x 4 micro-batches."""
+    _fullsize("r110v1", sample_m=[1])

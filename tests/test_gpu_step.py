@@ -100,6 +100,15 @@ def test_degenerate_partitionings(B, M, cuts):
     assert bd.model.num_partitions() == len(cuts) + 1
 
 
+@pytest.mark.parametrize("cuts", [[11], [4, 9, 16]])
+def test_post_activation_basic_blocks(cuts):
+    """ResNet v1 blocks (CONV BNRELU CONV BN, ADD with the shortcut, RELU), with a strided 3x3 convolution and a
+    projection shortcut: the paper's ResNet-110 family at depth 8."""
+    c = wl.config("r8v1")
+    bd, _, _ = check_step(c["ops"], c["in_hwc"], c["B"], c["M"], cuts, seed=6, bn_jitter=0.2)
+    assert bd.model.num_partitions() == len(cuts) + 1
+
+
 def test_odd_widths_run_on_cuda_cores():
     ops = wl.resnet_v2_cifar(1, widths=(4, 8, 12), n_classes=5)
     bd, _, _ = check_step(ops, (8, 8, 3), 6, 3, [9], seed=1, bn_jitter=0.2)
