@@ -25,6 +25,11 @@ def tiny_v1():
     return wl.resnet_v1_cifar(1, widths=(4, 8), n_classes=5), (8, 8, 3)
 
 
+def tiny_vgg():
+    """Convolution + ReLU groups with 2x2 max-pools and hidden fully connected layers, no batch norm."""
+    return wl.vgg16_cifar(widths=(4, 8, 8), convs=(2, 1, 2), fc=12, n_classes=5), (8, 8, 3)
+
+
 def _setup(builder, B, seed=0):
     ops, hwc = builder()
     x, labels = wl.draw_inputs(B, hwc, ops[-1].c_out, seed_x=100 + seed, seed_labels=200 + seed)
@@ -33,7 +38,7 @@ def _setup(builder, B, seed=0):
 
 
 # ------------------------------------------------------------------ P1
-@pytest.mark.parametrize("builder", [tiny_cifar, tiny_imagenet, tiny_v1])
+@pytest.mark.parametrize("builder", [tiny_cifar, tiny_imagenet, tiny_v1, tiny_vgg])
 def test_finite_differences_every_backward_formula(builder):
     """Central differences of the step loss against the averaged gradient: pins
     every backward formula, the BN coupling across samples and the 1/M."""
@@ -89,7 +94,7 @@ def test_finite_differences_input_gradient():
 
 
 # ------------------------------------------------------------------ P2
-@pytest.mark.parametrize("builder", [tiny_cifar, tiny_imagenet, tiny_v1])
+@pytest.mark.parametrize("builder", [tiny_cifar, tiny_imagenet, tiny_v1, tiny_vgg])
 def test_partition_count_invariance_bit_exact(builder):
     """Section 6.1's claim, partitioned == sequential, as a bit-exact identity:
     0, 1, 2 and 4 cuts, block-aligned and mid-block, give identical fp64 results."""
@@ -323,7 +328,7 @@ def _torch_step(ops, hwc, theta, x, labels, M):
     return np.array(slots), np.array(losses), acts, dacts
 
 
-@pytest.mark.parametrize("builder,B,M", [(tiny_cifar, 4, 2), (tiny_imagenet, 4, 2), (tiny_v1, 4, 2)])
+@pytest.mark.parametrize("builder,B,M", [(tiny_cifar, 4, 2), (tiny_imagenet, 4, 2), (tiny_v1, 4, 2), (tiny_vgg, 4, 2)])
 def test_against_torch_autograd_small(builder, B, M):
     ops, hwc, x, labels, theta = _setup(builder, B=B, seed=1)
     slots, losses, acts, dacts = _torch_step(ops, hwc, theta, x, labels, M)

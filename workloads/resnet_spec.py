@@ -71,6 +71,26 @@ def resnet_v1_cifar(n, widths=(16, 32, 64), n_classes=10, in_ch=3):
     return ops
 
 
+def vgg16_cifar(widths=(64, 128, 256, 512, 512), convs=(2, 2, 3, 3, 3), fc=4096, n_classes=10, in_ch=3):
+    """VGG-16 laid out for 32x32 inputs: five groups of 3x3 convolutions (pad 1) each followed by ReLU, a 2x2 stride-2
+    max-pool after every group (32 -> 1 pixel), two hidden fully connected layers with ReLU (1x1 convolutions on the 1x1
+    map) and the classifier (the head's mean over one pixel is the identity).  13 + 3 weight layers, no batch norm.
+    Biases are left out: the op list has no bias term for convolutions."""
+    ops, t, c_t = [], -1, in_ch
+    for w, k in zip(widths, convs):
+        for _ in range(k):
+            ops.append(Op(CONV, t, -1, c_t, w, 3, 1, 1, 0.0)); t = len(ops) - 1
+            ops.append(Op(RELU, t, -1, w, w, 0, 1, 0, 0.0)); t = len(ops) - 1
+            c_t = w
+        ops.append(Op(MAXPOOL, t, -1, c_t, c_t, 2, 2, 0, 0.0)); t = len(ops) - 1
+    for _ in range(2):
+        ops.append(Op(CONV, t, -1, c_t, fc, 1, 1, 0, 0.0)); t = len(ops) - 1
+        ops.append(Op(RELU, t, -1, fc, fc, 0, 1, 0, 0.0)); t = len(ops) - 1
+        c_t = fc
+    ops.append(Op(HEAD, t, -1, c_t, n_classes, 0, 1, 0, 0.0))
+    return ops
+
+
 def resnet_v2_imagenet(blocks=(3, 8, 36, 3), widths=(64, 128, 256, 512), n_classes=1000, in_ch=3):
     """7x7 stride-2 stem, 3x3 stride-2 max-pool, four bottleneck stages."""
     ops = [Op(CONV, -1, -1, in_ch, widths[0], 7, 2, 3, 0.0),
@@ -98,6 +118,9 @@ CONFIGS = {
     # the paper's ResNet-110 is the post-activation (v1) basic-block net, depth 6n+2 with n = 18; a short one for tests
     "r110v1": (lambda: resnet_v1_cifar(18), (32, 32, 3), 128, 4, 4),
     "r8v1":   (lambda: resnet_v1_cifar(1), (32, 32, 3), 8, 2, 2),
+    # the paper's third model and a narrow copy of it for tests
+    "vgg16":  (lambda: vgg16_cifar(), (32, 32, 3), 128, 4, 4),
+    "vgg16s": (lambda: vgg16_cifar(widths=(16, 16, 32, 32, 64), fc=64), (32, 32, 3), 8, 2, 2),
 }
 
 
