@@ -33,7 +33,9 @@ NAMES = {"r1001": "ResNet-1001 v2 (n=111, widths 16/32/64 x4), 32x32x3, batch 12
                    "8 partitions x 8 micro-batches",
          "r20k": "ResNet-20 v2 with the Keras example's widths, 32x32x3, batch 16, 2 partitions x 2 micro-batches",
          "r110v1": "ResNet-110 v1 (post-activation basic blocks, n=18), 32x32x3, batch 128, 4 partitions x 4 micro-batches",
-         "r8v1": "ResNet-8 v1, 32x32x3, batch 8, 2 partitions x 2 micro-batches"}
+         "r8v1": "ResNet-8 v1, 32x32x3, batch 8, 2 partitions x 2 micro-batches",
+         "vgg16": "VGG-16 for 32x32 inputs (13 conv + 2 hidden FC + classifier, no biases), batch 128, 4 partitions x 4 micro-batches",
+         "vgg16s": "VGG-16 layout at reduced width, 32x32x3, batch 8, 2 partitions x 2 micro-batches"}
 
 
 def peaks():

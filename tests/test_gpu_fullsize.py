@@ -73,3 +73,7 @@ def test_config5_resnet152_imagenet_layout_batch64():
 def test_resnet110_v1_batch128():
     """The paper's ResNet-110 (post-activation basic blocks, depth 6*18+2), batch 128, 4 partitions x 4 micro-batches."""
     _fullsize("r110v1", sample_m=[1])
+
+
+def test_vgg16_batch128():
+    _fullsize("vgg16", sample_m=[2])

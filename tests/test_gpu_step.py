@@ -109,6 +109,13 @@ def test_post_activation_basic_blocks(cuts):
     assert bd.model.num_partitions() == len(cuts) + 1
 
 
+def test_vgg_style_net_without_batch_norm():
+    """Convolution + ReLU groups, 2x2 max-pools down to one pixel, hidden fully connected layers as 1x1 convolutions:
+    the paper's VGG-16 layout at reduced width."""
+    c = wl.config("vgg16s")
+    check_step(c["ops"], c["in_hwc"], c["B"], c["M"], c["cuts"], seed=8)
+
+
 def test_odd_widths_run_on_cuda_cores():
     ops = wl.resnet_v2_cifar(1, widths=(4, 8, 12), n_classes=5)
     bd, _, _ = check_step(ops, (8, 8, 3), 6, 3, [9], seed=1, bn_jitter=0.2)
