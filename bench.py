@@ -237,7 +237,7 @@ def kernel_roofline(torch, hpf, cfg, pk):
             "traffic": {(1, 1, 64, 16, 32): 33.62e6, (1, 1, 16, 64, 32): 8.47e6}.get((ks, st, ci, co, H), 0.0) * b / 128.0 or None,
             "peak_source": pk["source"],
             "kernel": "conv_tc_fwd_kernel (tcgen05 implicit GEMM, three-pass TF32), %dx%d stride %d, %d->%d channels, %dx%d "
-                      "pixels, micro-batch %d; %d rotating operand sets; one 8-byte status memset node precedes each launch"
+                      "pixels, micro-batch %d; %d rotating operand sets, kernel nodes only, launched with programmatic dependent launch as in the step"
                       % (ks, ks, st, ci, co, H, H, b, nset),
             "algorithmic_bytes_per_launch": alg, "us_per_launch": sec * 1e6,
             "note": "at the micro-batch size the kernel is latency bound (one 128-pixel tile per CTA, %d CTAs); "

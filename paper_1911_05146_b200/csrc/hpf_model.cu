@@ -1307,11 +1307,11 @@ static int conv_single(int pass, const float* in, const float* in2, const float*
     if (!conv_tc_supported(s, pass)) return fail(HPF_ERR_UNSUPPORTED, "shape outside the tensor-core kernels' reach");
     CU(conv_tc_init());
     ConvTcPlan plan;
-    // the last 256 bytes of the scratch hold the device status word of this call
+    // The last 256 bytes of the scratch hold the device status word.  The caller zeroes it once; the kernels only ever
+    // set it (first failure wins), so a call adds no memset to the stream and back-to-back calls stay kernel after kernel.
     size_t sb = 0;
     hpf_conv_scratch_bytes(N, H, W, C, K, R, stride, pad, &sb);
     DeviceStatus* status = reinterpret_cast<DeviceStatus*>(reinterpret_cast<char*>(d_scratch) + sb - 256);
-    CU(cudaMemsetAsync(status, 0, sizeof(DeviceStatus), st));
     const int64_t nw = (int64_t)K * R * R * C;
     const float* hi = wprep ? wprep + (pass == PASS_DGRAD ? 2 * nw : 0) : nullptr;
     CU(conv_tc_prepare(&plan, s, pass, path == 2 ? 1 : 3, in, in2, hi, hi ? hi + nw : nullptr, out, nullptr, false, d_scratch));
