@@ -222,7 +222,8 @@ int hpf_conv_dgrad(const float *d_dy, const float *d_w, const float *d_wprep, fl
 int hpf_conv_wgrad(const float *d_x, const float *d_dy, float *d_dw, int32_t N, int32_t H, int32_t W, int32_t C,
                    int32_t K, int32_t R, int32_t stride, int32_t pad, int32_t path, void *d_scratch, void *stream);
 /* Fused BN(training)+ReLU over x [rows][C]: d_stats receives mean[C] then 1/sqrt(var+eps)[C].
- * d_scratch: at least hpf_bnrelu_scratch_bytes(rows, C). */
+ * d_scratch: at least hpf_bnrelu_scratch_bytes(rows, C); the caller zeroes its first 256 bytes once (a ticket the
+ * kernels count on and leave at zero), the calls enqueue kernels only. */
 int hpf_bnrelu_scratch_bytes(int64_t rows, int32_t C, size_t *bytes);
 int hpf_bnrelu_fwd(const float *d_x, const float *d_gamma, const float *d_beta, float eps, float *d_y,
                    float *d_stats, int64_t rows, int32_t C, void *d_scratch, void *stream);

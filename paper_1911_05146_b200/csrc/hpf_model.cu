@@ -1360,7 +1360,6 @@ int hpf_bnrelu_fwd(const float* d_x, const float* d_gamma, const float* d_beta, 
     if (!d_x || !d_gamma || !d_beta || !d_y || !d_stats || !d_scratch) return fail(HPF_ERR_INVALID, "null argument");
     if (rows < 1 || C < 4 || C % 4) return fail(HPF_ERR_UNSUPPORTED, "channel count must be a multiple of 4");
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    CU(cudaMemsetAsync(d_scratch, 0, 256, st));
     CU(bnrelu_fwd(d_x, d_gamma, d_beta, eps, d_y, d_stats, rows, C, d_scratch, st, nullptr));
     return HPF_OK;
 }
@@ -1372,7 +1371,6 @@ int hpf_bnrelu_bwd(const float* d_x, const float* d_dy, const float* d_gamma, co
     if (!d_x || !d_dy || !d_gamma || !d_beta || !d_stats || !d_dx || !d_dgamma || !d_dbeta || !d_scratch) return fail(HPF_ERR_INVALID, "null argument");
     if (rows < 1 || C < 4 || C % 4) return fail(HPF_ERR_UNSUPPORTED, "channel count must be a multiple of 4");
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    CU(cudaMemsetAsync(d_scratch, 0, 256, st));
     CU(bnrelu_bwd(d_x, d_dy, d_gamma, d_beta, d_stats, d_dx, d_addend, accumulate != 0, d_dgamma, d_dbeta, rows, C, d_scratch, st, nullptr));
     return HPF_OK;
 }
