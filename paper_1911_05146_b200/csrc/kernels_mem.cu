@@ -95,6 +95,8 @@ bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, cons
     if (r1 > rows) r1 = rows;
     const float4* x4 = reinterpret_cast<const float4*>(x);
     const float4* dy4 = reinterpret_cast<const float4*>(dy);
+    // all column groups in one pass, a power-of-two count of at most 16: the reductions over row lanes use warp shuffles
+    const bool narrow = passes == 1 && cgt == cg_total && cgt <= 16 && (cgt & (cgt - 1)) == 0 && cgt * rl == kBnThreads;
 
     for (int pass = 0; pass < passes; ++pass) {
         const int cg = pass * cgt + my_cg;
@@ -131,6 +133,32 @@ bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, cons
                     d = v.w - p0.w; a.w += d; b.w = fmaf(d, d, b.w);
                 }
             }
+        }
+        if (narrow) {
+            // Few column groups (cgt a power of two <= 16, so 32 / cgt row lanes of a group sit in one warp): a fixed
+            // butterfly over the warp's row lanes, then the 16 warps' totals are added in ascending order.
+            for (int off = 16; off >= cgt; off >>= 1) {
+                a.x += __shfl_xor_sync(0xffffffffu, a.x, off); a.y += __shfl_xor_sync(0xffffffffu, a.y, off);
+                a.z += __shfl_xor_sync(0xffffffffu, a.z, off); a.w += __shfl_xor_sync(0xffffffffu, a.w, off);
+                b.x += __shfl_xor_sync(0xffffffffu, b.x, off); b.y += __shfl_xor_sync(0xffffffffu, b.y, off);
+                b.z += __shfl_xor_sync(0xffffffffu, b.z, off); b.w += __shfl_xor_sync(0xffffffffu, b.w, off);
+            }
+            const int warp = t >> 5, lane = t & 31;
+            if (lane < cgt) {
+                float* d = sh[warp * cgt + lane];
+                d[0] = a.x; d[1] = a.y; d[2] = a.z; d[3] = a.w; d[4] = b.x; d[5] = b.y; d[6] = b.z; d[7] = b.w;
+            }
+            __syncthreads();
+            if (t < cgt * 8) {
+                const int cgl = t >> 3, comp = t & 7;
+                if (cgl < cg_total) {
+                    float s = 0.f;
+                    for (int w = 0; w < kBnThreads / 32; ++w) s += sh[w * cgt + cgl][comp];
+                    partials[((int64_t)blockIdx.x * 2 + (comp >> 2)) * C + cgl * 4 + (comp & 3)] = s;
+                }
+            }
+            __syncthreads();
+            continue;
         }
         sh[t][0] = a.x; sh[t][1] = a.y; sh[t][2] = a.z; sh[t][3] = a.w;
         sh[t][4] = b.x; sh[t][5] = b.y; sh[t][6] = b.z; sh[t][7] = b.w;
@@ -174,6 +202,25 @@ bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, cons
             }
         }
         __syncthreads();
+        if (narrow) {
+            for (int off = 16; off >= cgt; off >>= 1) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], off);
+            }
+            const int warp = t >> 5, lane = t & 31;
+            double (*wsum)[8] = shd + kBnThreads / 2;       // upper half of the buffer: [warp * cgt + column group][8]
+            if (lane < cgt) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) wsum[warp * cgt + lane][j] = acc[j];
+            }
+            __syncthreads();
+            if (t < cgt * 8) {
+                const int cgl = t >> 3, comp = t & 7;
+                double s = 0.0;
+                for (int w = 0; w < kBnThreads / 32; ++w) s += wsum[w * cgt + cgl][comp];
+                shd[cgl][comp] = s;                         // lower half: the totals, read below
+            }
+        } else {
 #pragma unroll
         for (int j = 0; j < 8; ++j) shd[t][j] = acc[j];
         __syncthreads();
@@ -185,6 +232,7 @@ bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, cons
             for (int l = 0; l < rl; ++l) s += shd[l * cgt + cgl][comp];
             // the pair (a, b) of one channel is finished by two threads: exchange through shared memory
             shd[cgl][comp] = s;       // row 0 lane (l = 0) slot of this column group: safe, every read above is done per o
+        }
         }
         __syncthreads();
         for (int cl = t; cl < cgt * 4; cl += kBnThreads) {
