@@ -616,7 +616,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
         bool all_done = true;
         for (int tj = 0; tj < my_tiles; ++tj) {
         HPF_TILE_ORIGIN(tile0 + tj);
-        mbar_wait(accum_bar + 8 * tj, 0, &abort_flag);
+        // the row tables do not depend on the accumulator: they are built while the MMAs still run
         if (tid < kTileM) {
             const int wi = tid % p.box_w, hi = (tid / p.box_w) % p.box_h, ni = tid / (p.box_w * p.box_h);
             const int q = q0 + wi, pp = p0 + hi, n = n0 + ni;
@@ -628,6 +628,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     if ((dy | dx) && pp * p.zero_fill + dy < p.out_h && q * p.zero_fill + dx < p.out_w) fill |= 1 << (dy * 4 + dx);
             row_fill[tid] = (valid && p.zero_fill > 1 && p.zero_fill <= 4) ? fill : 0;
         }
+        mbar_wait(accum_bar + 8 * tj, 0, &abort_flag);
         asm volatile("bar.sync 1, 256;" ::: "memory");
         const bool done = abort_flag == 0;             // uniform over the 8 warps after the barrier
         all_done = all_done && done;
@@ -723,12 +724,25 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                 // threads of each group in ascending order and store this tile's partial sums
                 asm volatile("bar.sync 1, 256;" ::: "memory");          // the staging area is free again
                 float4* red = reinterpret_cast<float4*>(stg);
-                red[2 * tid] = sa; red[2 * tid + 1] = sb;
+                int n_rows = 256;                                       // rows of `red` per group stride c4n
+                if (c4n <= 16) {
+                    // the 32 / c4n threads of a group inside a warp first: a fixed butterfly, then one row per warp
+                    for (int off = 16; off >= c4n; off >>= 1) {
+                        sa.x += __shfl_xor_sync(0xffffffffu, sa.x, off); sa.y += __shfl_xor_sync(0xffffffffu, sa.y, off);
+                        sa.z += __shfl_xor_sync(0xffffffffu, sa.z, off); sa.w += __shfl_xor_sync(0xffffffffu, sa.w, off);
+                        sb.x += __shfl_xor_sync(0xffffffffu, sb.x, off); sb.y += __shfl_xor_sync(0xffffffffu, sb.y, off);
+                        sb.z += __shfl_xor_sync(0xffffffffu, sb.z, off); sb.w += __shfl_xor_sync(0xffffffffu, sb.w, off);
+                    }
+                    if (lane < c4n) { const int r = (tid >> 5) * c4n + lane; red[2 * r] = sa; red[2 * r + 1] = sb; }
+                    n_rows = 8 * c4n;
+                } else {
+                    red[2 * tid] = sa; red[2 * tid + 1] = sb;
+                }
                 asm volatile("bar.sync 1, 256;" ::: "memory");
                 if (tid < c4n * 2) {
                     const int g = tid >> 1, which = tid & 1;
                     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int t2 = g; t2 < 256; t2 += c4n) { const float4 v2 = red[2 * t2 + which]; acc.x += v2.x; acc.y += v2.y; acc.z += v2.z; acc.w += v2.w; }
+                    for (int t2 = g; t2 < n_rows; t2 += c4n) { const float4 v2 = red[2 * t2 + which]; acc.x += v2.x; acc.y += v2.y; acc.z += v2.z; acc.w += v2.w; }
                     float* dstp = p.stat_partials + ((size_t)(tile0 + tj) * 2 + which) * p.c_out + co0 + 4 * g;
                     *reinterpret_cast<float4*>(dstp) = acc;
                     if (stat_mode == 1) __threadfence();
