@@ -1457,6 +1457,8 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     int stages = (int)(kSmemBudget / p.stage_bytes);
     const int total = v.R * v.R * p.n_kchunks;
     if (stages > kFwdMaxStages) stages = kFwdMaxStages;      // measured: more stages cost more in residency than they hide
+    // one more where two CTAs still fit an SM: nine taps then take two rounds of the ring instead of three
+    if (total > kFwdMaxStages && (unsigned int)(kFwdMaxStages + 1) * p.stage_bytes <= 92u * 1024u) stages = kFwdMaxStages + 1;
     if (stages > total) stages = total;
     p.stages = stages;
     if (fuse && fuse->mode) {
