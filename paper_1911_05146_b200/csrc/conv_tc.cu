@@ -325,6 +325,26 @@ __device__ __forceinline__ void bn_combine_partials(const float* partials, int n
         const float4 v = __ldcg(part + (size_t)k * ncol4 + col4);
         a0 += (double)v.x; a1 += (double)v.y; a2 += (double)v.z; a3 += (double)v.w;
     }
+    if (ncol4 <= 16) {
+        // several lanes of a column sit in one warp: a fixed butterfly first, then the eight warps in ascending order
+        for (int off = 16; off >= ncol4; off >>= 1) {
+            a0 += __shfl_xor_sync(0xffffffffu, a0, off); a1 += __shfl_xor_sync(0xffffffffu, a1, off);
+            a2 += __shfl_xor_sync(0xffffffffu, a2, off); a3 += __shfl_xor_sync(0xffffffffu, a3, off);
+        }
+        const int warp = tid >> 5, lane = tid & 31;
+        double (*wsum)[4] = bn_red + 128;                   // [warp * ncol4 + column]; rows 0..127 stay free for the totals
+        if (lane < ncol4) { double* d = wsum[warp * ncol4 + lane]; d[0] = a0; d[1] = a1; d[2] = a2; d[3] = a3; }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (tid < ncol4) {
+            double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
+            for (int w = 0; w < 8; ++w) {
+                const double* r = wsum[w * ncol4 + tid];
+                t0 += r[0]; t1 += r[1]; t2 += r[2]; t3 += r[3];
+            }
+            bn_red[tid][0] = t0; bn_red[tid][1] = t1; bn_red[tid][2] = t2; bn_red[tid][3] = t3;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+    } else {
     bn_red[tid][0] = a0; bn_red[tid][1] = a1; bn_red[tid][2] = a2; bn_red[tid][3] = a3;
     asm volatile("bar.sync 1, 256;" ::: "memory");
     if (tid < ncol4) {
@@ -337,6 +357,7 @@ __device__ __forceinline__ void bn_combine_partials(const float* partials, int n
         bn_red[tid][0] = t0; bn_red[tid][1] = t1; bn_red[tid][2] = t2; bn_red[tid][3] = t3;
     }
     asm volatile("bar.sync 1, 256;" ::: "memory");
+    }
     const double* tot = &bn_red[0][0];                  // [2][C]: sums, then sums of squares
     if (tid < C) {
         const double m = tot[tid] * inv_rows;
