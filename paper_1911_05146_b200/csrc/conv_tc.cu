@@ -1232,7 +1232,7 @@ struct WgradGeom {
     unsigned int raw_bytes, t_bytes, tmem_cols;
 };
 
-bool wgrad_geom(const ConvShape& s, int passes, WgradGeom* g)
+bool wgrad_geom(const ConvShape& s, int passes, WgradGeom* g, int max_ctas = 0)
 {
     if (s.C % 16 || s.K % 16) return false;
     if (s.R != 1 && s.R != 3) return false;
@@ -1284,12 +1284,18 @@ bool wgrad_geom(const ConvShape& s, int passes, WgradGeom* g)
     const double dw_bytes = 4.0 * (double)s.K * taps * s.C;
     int splits = g->n_tiles / 4;
     int cap = (int)(operand_bytes / (4.0 * dw_bytes));
-    // small problems are latency bound, not byte bound: spread the pixel walk over at least ~48 CTAs
+    // small problems are latency bound, not byte bound: spread the pixel walk over several dozen CTAs
     const int ctas_per_split = g->tap_groups * (s.K / g->m_chunk) * (s.C / g->n_cols);
     const int want = (48 + ctas_per_split - 1) / ctas_per_split;
     if (cap < want) cap = want;
     if (splits > cap) splits = cap;
     if (splits > 296) splits = 296;          // two CTAs per SM
+    if (max_ctas > 0) {
+        // the caller wants the launch to take little SM time (CTAs x (fixed cost + tiles)) rather than to be short
+        int ms = max_ctas / ctas_per_split;
+        if (ms < 1) ms = 1;
+        if (splits > ms) splits = ms;
+    }
     if (splits > g->n_tiles / 2) splits = g->n_tiles / 2;
     if (splits < 1) splits = 1;
     g->tiles_per_split = (g->n_tiles + splits - 1) / splits;
@@ -1382,7 +1388,7 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     if (passes != 1 && passes != 3) return cudaErrorInvalidValue;
     if (pass == PASS_WGRAD) {
         WgradGeom g;
-        if (!wgrad_geom(s, passes, &g)) return cudaErrorNotSupported;
+        if (!wgrad_geom(s, passes, &g, fuse ? fuse->wgrad_max_ctas : 0)) return cudaErrorNotSupported;
         ConvTcWgradLaunch* L = reinterpret_cast<ConvTcWgradLaunch*>(plan->storage);
         WgradParams& P = L->p;
         memset(&P, 0, sizeof P);

@@ -47,6 +47,9 @@ struct ConvBnFuse {
     const float* in_beta = nullptr;
     float* in_stats = nullptr;
     float* in_y = nullptr;
+    // weight gradient only: > 0 caps the CTAs of the launch (fewer pixel splits, each walking more tiles): less SM time
+    // at a longer duration, for launches that run beside a chain of latency-bound kernels
+    int wgrad_max_ctas = 0;
     const float* in_partials = nullptr;
     int in_tiles = 0;
     long long in_rows = 0;

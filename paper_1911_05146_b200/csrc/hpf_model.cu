@@ -1100,9 +1100,16 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                         CU(conv_tc_prepare(pl, s, pass, passes, mdl->grad(i, m), nullptr, wp + 2 * G + o.w_off, wp + 3 * G + o.w_off,
                                            mdl->grad(src, m), ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch));
                     }
-                    else
+                    else {
+                        // Weight gradients run on the side streams, beside the stages' chains of dependent kernels and feeding
+                        // nothing but the final average.  With many stages busy the SM time a launch takes counts, not its
+                        // duration: about 32 CTAs is the measured optimum for eight stages (fewer and the weight gradients
+                        // fall behind the chain; with four stages the uncapped launch measured faster).
+                        ConvBnFuse hint;
+                        hint.wgrad_max_ctas = (mdl->P >= 6 && !mdl->side.empty()) ? 32 : 0;
                         CU(conv_tc_prepare(pl, s, pass, mdl->opt_conv_path == 2 ? 1 : mdl->opt_wgrad_passes, mdl->grad(i, m), mdl->act(src, m), nullptr, nullptr,
-                                           mdl->gslots + (int64_t)m * mdl->G + o.w_off, nullptr, false, scratch));
+                                           mdl->gslots + (int64_t)m * mdl->G + o.w_off, nullptr, false, scratch, &hint));
+                    }
                 }
         }
     }
