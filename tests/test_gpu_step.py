@@ -116,6 +116,13 @@ def test_vgg_style_net_without_batch_norm():
     check_step(c["ops"], c["in_hwc"], c["B"], c["M"], c["cuts"], seed=8)
 
 
+def test_large_microbatch_uses_the_multi_tile_convolutions_with_the_bn_fusions():
+    """A micro-batch of 80 images at 32x32 is 640 pixel tiles per convolution: the launches give each CTA several tiles,
+    with the BN statistics and the BN+ReLU-on-the-way-in riding in the same kernels."""
+    c = wl.config("r11")
+    check_step(c["ops"], c["in_hwc"], 80, 1, c["cuts"], seed=9, bn_jitter=0.1, microbatches=[0])
+
+
 def test_odd_widths_run_on_cuda_cores():
     ops = wl.resnet_v2_cifar(1, widths=(4, 8, 12), n_classes=5)
     bd, _, _ = check_step(ops, (8, 8, 3), 6, 3, [9], seed=1, bn_jitter=0.2)
