@@ -52,13 +52,16 @@ BnPlan bn_plan(int64_t rows, int C)
     p.cgt = p.cg_total < kBnThreads ? p.cg_total : kBnThreads;
     p.rl = kBnThreads / p.cgt;
     p.passes = (p.cg_total + p.cgt - 1) / p.cgt;
-    int64_t nb = rows / ((int64_t)p.rl * 4);      // four rows per thread: one batch of loads in flight, one memory round trip
+    // Four rows per thread (one batch of loads in flight, one memory round trip) while that keeps the partials few;
+    // eight beyond, where the last block's combine and the ticket traffic would outweigh the shorter row loop.
+    int64_t nb = rows / ((int64_t)p.rl * 4);
+    if (nb > kBnMaxBlocks) nb = rows / ((int64_t)p.rl * 8) > kBnMaxBlocks ? rows / ((int64_t)p.rl * 8) : kBnMaxBlocks;
     if (nb < 1) nb = 1;
     const int cap = rows * C > kBnLargeElems ? kBnMaxBlocksLarge : kBnMaxBlocks;
     if (nb > cap) nb = cap;
     p.rows_per_blk = ceil_div64(rows, nb);
     p.nblk = (int)ceil_div64(rows, p.rows_per_blk);
-    int64_t na = rows / ((int64_t)p.rl * 8);
+    int64_t na = rows / ((int64_t)p.rl * 4);
     if (na < 1) na = 1;
     if (na > 148 * 8) na = 148 * 8;
     p.rows_per_blk_apply = ceil_div64(rows, na);
