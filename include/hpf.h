@@ -110,9 +110,13 @@ int hpf_model_destroy(hpf_model *model);
  *                          statistics as a by-product.  0: every BN runs its own kernels.  Default 3.
  *   HPF_OPT_CELL_TIMES     1: a one-thread kernel stores the device's nanosecond timer at the start and at the end of
  *                          every (partition, micro-batch) cell of the forward and backward schedules (Section 5.3's
- *                          pipeline, as it really ran); read them with hpf_cell_times.  Default 0. */
+ *                          pipeline, as it really ran); read them with hpf_cell_times.  Default 0.
+ *   HPF_OPT_BN_CLUSTER     1 (default): the backward of a BN whose micro-batch tensor is small enough to sit in the
+ *                          registers of a few thread-block clusters is one launch (the CTAs of a cluster exchange their
+ *                          per-channel sums through distributed shared memory); 0: always the reduce + apply pair. */
 typedef enum { HPF_OPT_GRAPH = 1, HPF_OPT_CONV_PATH = 2, HPF_OPT_SINGLE_STREAM = 3, HPF_OPT_KEEP_MESSAGES = 4,
-               HPF_OPT_FUSE_ADD = 5, HPF_OPT_PDL = 6, HPF_OPT_WGRAD_PASSES = 7, HPF_OPT_FUSE_BN = 8, HPF_OPT_CELL_TIMES = 9 } hpf_option;
+               HPF_OPT_FUSE_ADD = 5, HPF_OPT_PDL = 6, HPF_OPT_WGRAD_PASSES = 7, HPF_OPT_FUSE_BN = 8, HPF_OPT_CELL_TIMES = 9,
+               HPF_OPT_BN_CLUSTER = 10 } hpf_option;
 int hpf_set_option(hpf_model *model, int32_t option, int32_t value);
 
 /* ---- integer bookkeeping (Section 5.1 lists, Section 5.3 pipelining) ----------------------------- */

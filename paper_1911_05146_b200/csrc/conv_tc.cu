@@ -531,7 +531,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     if (blockIdx.x == 0 && blockIdx.y == 0) { p.bn_in_stats_out[tid] = mu; p.bn_in_stats_out[C + tid] = rs; }
                 }
             } else if (tid < C) {
-                bn_par[0][tid] = __ldg(p.bn_in_stats + tid); bn_par[1][tid] = __ldg(p.bn_in_stats + C + tid);
+                bn_par[0][tid] = __ldcg(p.bn_in_stats + tid); bn_par[1][tid] = __ldcg(p.bn_in_stats + C + tid);   // written by the kernel before: not the read-only path
                 bn_par[2][tid] = __ldg(p.bn_in_gamma + tid); bn_par[3][tid] = __ldg(p.bn_in_beta + tid);
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -714,7 +714,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                 if (extra) {
 #pragma unroll
                     for (int u = 0; u < 4; ++u)
-                        if (off[u] >= 0) { const float4 e = __ldg(reinterpret_cast<const float4*>(extra + off[u])); o[u].x += e.x; o[u].y += e.y; o[u].z += e.z; o[u].w += e.w; }
+                        if (off[u] >= 0) { const float4 e = __ldcg(reinterpret_cast<const float4*>(extra + off[u])); o[u].x += e.x; o[u].y += e.y; o[u].z += e.z; o[u].w += e.w; }
                 }
                 if (accumulate) {
 #pragma unroll

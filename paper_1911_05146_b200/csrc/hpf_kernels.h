@@ -63,7 +63,18 @@ cudaError_t bnrelu_fwd(const float* x, const float* gamma, const float* beta, fl
                        int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch, bool relu = true);
 cudaError_t bnrelu_bwd(const float* x, const float* dy, const float* gamma, const float* beta, const float* stats,
                        float* dx, const float* addend, bool accumulate, float* dgamma, float* dbeta,
-                       int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch, bool relu = true);
+                       int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch, bool relu = true,
+                       bool x_is_old = false);
+// x_is_old: x, stats, gamma and beta were complete before the kernels just ahead of this call in the stream were
+// enqueued (forward results read by a backward pass), so the kernel may fetch them while its predecessor still runs.
+extern thread_local bool g_bn_cluster;   // single-launch cluster kernel for micro-batch sized BN backward (default on)
+struct BnClusterScope {
+    bool saved;
+    explicit BnClusterScope(bool on) : saved(g_bn_cluster) { g_bn_cluster = on; }
+    ~BnClusterScope() { g_bn_cluster = saved; }
+    BnClusterScope(const BnClusterScope&) = delete;
+    BnClusterScope& operator=(const BnClusterScope&) = delete;
+};
 // stand-alone ReLU: y = max(x, 0); dx (+= if accumulate) = dy * [x > 0] (+ addend)
 cudaError_t relu_fwd(const float* x, float* y, int64_t n, cudaStream_t st, int64_t* n_launch);
 cudaError_t relu_bwd(const float* x, const float* dy, float* dx, const float* addend, bool accumulate, int64_t n, cudaStream_t st,

@@ -90,6 +90,7 @@ struct hpf_model {
     std::vector<size_t> bn_part_bytes;         // per partition: size of one per-tile-sum buffer
     int opt_bn_late_floats = 8192;             // largest [tiles][2][C] block of per-tile sums a reading convolution adds itself
     bool opt_pdl = true;       // programmatic dependent launch for this model's kernels
+    bool opt_bn_cluster = true; // BN backward of micro-batch sized tensors as one thread-block-cluster launch
     int opt_cell_times = 0;    // record a device timestamp at the start and end of every (partition, micro-batch) cell
     size_t cell_times_off = 0;
     int opt_fuse_bn = 3;       // bit 0: BN statistics in the producing convolution's write-out, bit 1: BN+ReLU applied by the reading convolution
@@ -609,12 +610,12 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
     case HPF_OP_BNRELU:
         CU(bnrelu_bwd(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m), addend,
                       e.accumulate != 0, slot + o.w_off, slot + o.b_off, (int64_t)mdl->b * o.H * o.W, o.C,
-                      mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
+                      mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches, true, true));
         break;
     case HPF_OP_BN:
         CU(bnrelu_bwd(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m), addend,
                       e.accumulate != 0, slot + o.w_off, slot + o.b_off, (int64_t)mdl->b * o.H * o.W, o.C,
-                      mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches, false));
+                      mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches, false, true));
         break;
     case HPF_OP_RELU:
         CU(relu_bwd(in0, dout, mdl->grad(q.src0, m), addend, e.accumulate != 0, mdl->numel(i), st, &mdl->launches));
@@ -637,6 +638,7 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
 int enqueue_phase(hpf_model* mdl, int phase)
 {
     const PdlScope pdl_scope(mdl->opt_pdl);
+    const BnClusterScope bn_cluster_scope(mdl->opt_bn_cluster);
     const int P = mdl->P, M = mdl->M;
     cudaStream_t s0 = mdl->streams[0];
     const bool multi = !mdl->opt_single && P > 1;
@@ -836,6 +838,7 @@ int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
     case HPF_OPT_PDL: mdl->opt_pdl = value != 0; break;
     case HPF_OPT_FUSE_BN: if (value < 0 || value > 3) return fail(HPF_ERR_INVALID, "0..3"); mdl->opt_fuse_bn = value; break;
     case HPF_OPT_CELL_TIMES: mdl->opt_cell_times = value != 0; break;
+    case HPF_OPT_BN_CLUSTER: mdl->opt_bn_cluster = value != 0; break;
     case HPF_OPT_WGRAD_PASSES: if (value != 1 && value != 3) return fail(HPF_ERR_INVALID, "1 or 3 passes"); mdl->opt_wgrad_passes = value; break;
     default: return fail(HPF_ERR_INVALID, "unknown option");
     }

@@ -5,11 +5,13 @@
 // consecutive threads walk consecutive float4 of a row-major [rows][C] tensor.
 #include "hpf_kernels.h"
 
+#include <cooperative_groups.h>
 #include <math.h>
 
 namespace hpf {
 
 thread_local bool g_pdl_enabled = true;
+thread_local bool g_bn_cluster = true;
 
 namespace {
 
@@ -346,6 +348,504 @@ bn_apply_bwd_kernel(const float4* __restrict__ x, const float4* __restrict__ dy,
             dx[i] = o;
         }
     }
+}
+
+// BN(+ReLU) backward of a micro-batch sized tensor in ONE launch: thread-block clusters instead of the reduce / apply pair.
+// A cluster of kBnCluster CTAs owns cgc float4 column groups (channels never mix, so clusters are independent); its CTAs
+// split the rows.  Every thread keeps its NV rows of x and dy in registers, the CTA reduces sum dz and sum dz*xhat per
+// channel (warp butterfly over the row lanes, then the warps in ascending order), the cluster's CTAs read each other's
+// per-channel sums through distributed shared memory in ascending rank order (fp64), and dx is computed from the registers:
+// one trip to memory for the operands, no partials in global memory, no ticket, no second kernel.
+// early_x: x, the statistics and the BN parameters are not produced by the kernels just before this one (they are forward
+// results), so they are fetched before the wait on the preceding kernel and only dy after it.
+constexpr int kBnCluster = 8;
+constexpr int kBnClusterMaxCgc = 16;
+constexpr int kBnClusterMaxActive = 14;   // clusters of 8 one-per-SM CTAs that are resident together (15 measured); more would run as a second wave
+
+template <int NV, bool ADDEND, bool ACCUM>
+__global__ void __launch_bounds__(kBnThreads)
+bn_bwd_cluster_kernel(const float4* __restrict__ x, const float4* __restrict__ dy, const float* __restrict__ gamma,
+                      const float* __restrict__ beta, const float* __restrict__ stats, const float4* __restrict__ addend,
+                      float4* __restrict__ dx, float* __restrict__ dgamma, float* __restrict__ dbeta, int64_t rows, int C,
+                      int cgc, int64_t rows_per_cta, float floor, int early_x)
+{
+    namespace cgr = cooperative_groups;
+    cgr::cluster_group cluster = cgr::this_cluster();
+    __shared__ float wpart[kBnThreads / 32][kBnClusterMaxCgc * 8];
+    __shared__ float part[kBnClusterMaxCgc * 8];
+    __shared__ float coefs[kBnClusterMaxCgc * 8];
+    pdl_launch_dependents();
+    const int t = threadIdx.x;
+    const unsigned int rank = cluster.block_rank();
+    const int cl = blockIdx.x / kBnCluster;
+    const int cg_total = C / 4;
+    const int rl = kBnThreads / cgc;
+    const int my_cg = t % cgc, my_rl = t / cgc;
+    const int cg = cl * cgc + my_cg;
+    const int64_t r0 = (int64_t)rank * rows_per_cta;
+    int64_t r1 = r0 + rows_per_cta;
+    if (r1 > rows) r1 = rows;
+    int n = r1 > r0 + my_rl ? (int)((r1 - r0 - my_rl + rl - 1) / rl) : 0;
+    if (n > NV) n = NV;                                     // the launcher sizes NV so that this never cuts
+    const int64_t base = (r0 + my_rl) * cg_total + cg, step = (int64_t)rl * cg_total;
+
+    if (!early_x) pdl_wait();
+    const float4 mu = __ldg(reinterpret_cast<const float4*>(stats) + cg);
+    const float4 rs = __ldg(reinterpret_cast<const float4*>(stats + C) + cg);
+    const float4 gm = __ldg(reinterpret_cast<const float4*>(gamma) + cg);
+    const float4 bt = __ldg(reinterpret_cast<const float4*>(beta) + cg);
+    float4 xv[NV], dv[NV];
+#pragma unroll
+    for (int k = 0; k < NV; ++k) if (k < n) xv[k] = __ldg(x + base + k * step);
+    if (early_x) pdl_wait();
+#pragma unroll
+    for (int k = 0; k < NV; ++k) if (k < n) dv[k] = __ldcg(dy + base + k * step);   // not the read-only path: such a load may be moved above the wait
+
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+        if (k < n) {
+            float xh, dz;
+            xh = bn_xhat(xv[k].x, mu.x, rs.x); dz = bn_z(xh, gm.x, bt.x) > floor ? dv[k].x : 0.f; a.x += dz; b.x = fmaf(dz, xh, b.x);
+            xv[k].x = xh; dv[k].x = dz;
+            xh = bn_xhat(xv[k].y, mu.y, rs.y); dz = bn_z(xh, gm.y, bt.y) > floor ? dv[k].y : 0.f; a.y += dz; b.y = fmaf(dz, xh, b.y);
+            xv[k].y = xh; dv[k].y = dz;
+            xh = bn_xhat(xv[k].z, mu.z, rs.z); dz = bn_z(xh, gm.z, bt.z) > floor ? dv[k].z : 0.f; a.z += dz; b.z = fmaf(dz, xh, b.z);
+            xv[k].z = xh; dv[k].z = dz;
+            xh = bn_xhat(xv[k].w, mu.w, rs.w); dz = bn_z(xh, gm.w, bt.w) > floor ? dv[k].w : 0.f; a.w += dz; b.w = fmaf(dz, xh, b.w);
+            xv[k].w = xh; dv[k].w = dz;
+        }
+    }
+    // row lanes of one column group inside a warp: fixed butterfly; then the warps in ascending order
+    for (int off = 16; off >= cgc; off >>= 1) {
+        a.x += __shfl_xor_sync(0xffffffffu, a.x, off); a.y += __shfl_xor_sync(0xffffffffu, a.y, off);
+        a.z += __shfl_xor_sync(0xffffffffu, a.z, off); a.w += __shfl_xor_sync(0xffffffffu, a.w, off);
+        b.x += __shfl_xor_sync(0xffffffffu, b.x, off); b.y += __shfl_xor_sync(0xffffffffu, b.y, off);
+        b.z += __shfl_xor_sync(0xffffffffu, b.z, off); b.w += __shfl_xor_sync(0xffffffffu, b.w, off);
+    }
+    const int warp = t >> 5, lane = t & 31;
+    if (lane < cgc) {
+        float* d = &wpart[warp][lane * 8];
+        d[0] = a.x; d[1] = a.y; d[2] = a.z; d[3] = a.w; d[4] = b.x; d[5] = b.y; d[6] = b.z; d[7] = b.w;
+    }
+    __syncthreads();
+    if (t < cgc * 8) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < kBnThreads / 32; ++w) s += wpart[w][t];
+        part[t] = s;
+    }
+    cluster.sync();
+    if (t < cgc * 8) {
+        double s = 0.0;
+#pragma unroll
+        for (unsigned int r = 0; r < (unsigned int)kBnCluster; ++r) s += (double)*cluster.map_shared_rank(&part[t], r);
+        coefs[t] = (float)(s * (1.0 / (double)rows));
+        if (rank == 0) {
+            const int c = (cl * cgc + (t >> 3)) * 4 + (t & 3);
+            if (t & 4) dgamma[c] = (float)s; else dbeta[c] = (float)s;
+        }
+    }
+    __syncthreads();
+    cluster.barrier_arrive();                               // this CTA no longer reads the others' shared memory
+    const float4 ca = *reinterpret_cast<const float4*>(&coefs[my_cg * 8]);
+    const float4 cb = *reinterpret_cast<const float4*>(&coefs[my_cg * 8 + 4]);
+    const float4 sc = make_float4(gm.x * rs.x, gm.y * rs.y, gm.z * rs.z, gm.w * rs.w);
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+        if (k < n) {
+            const int64_t i = base + k * step;
+            float4 o;
+            o.x = sc.x * (dv[k].x - ca.x - xv[k].x * cb.x);
+            o.y = sc.y * (dv[k].y - ca.y - xv[k].y * cb.y);
+            o.z = sc.z * (dv[k].z - ca.z - xv[k].z * cb.z);
+            o.w = sc.w * (dv[k].w - ca.w - xv[k].w * cb.w);
+            if (ADDEND) { const float4 e = __ldcg(addend + i); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+            if (ACCUM) { const float4 e = dx[i]; o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+            dx[i] = o;
+        }
+    }
+    cluster.barrier_wait();                                 // shared memory stays alive until every CTA has read it
+}
+
+struct BnClusterPlan { bool ok; int cgc, n_clusters, nv; int64_t rows_per_cta; };
+
+// Eligible: micro-batch sized tensors whose rows fit the registers of kBnCluster CTAs per column-group slice.  Prefers few
+// rows per thread (more CTAs pulling on memory), then wide slices (longer contiguous segments per row).
+BnClusterPlan bn_cluster_plan(int64_t rows, int C)
+{
+    BnClusterPlan p = {false, 0, 0, 0, 0};
+    if (C % 4 != 0 || rows < 1 || rows * C > (int64_t)(2 << 20)) return p;
+    const int cg_total = C / 4;
+    const int64_t rpc = ceil_div64(rows, kBnCluster);
+    static const int prefs[3] = {2, 4, 8};
+    for (int pi = 0; pi < 3; ++pi) {
+        for (int cgc = kBnClusterMaxCgc; cgc >= 2; cgc >>= 1) {
+            if (cg_total % cgc != 0) continue;
+            const int n_clusters = cg_total / cgc;
+            if (n_clusters > kBnClusterMaxActive) continue;
+            const int64_t nv = ceil_div64(rpc, kBnThreads / cgc);
+            if (nv > prefs[pi]) continue;
+            p.ok = true; p.cgc = cgc; p.n_clusters = n_clusters; p.rows_per_cta = rpc;
+            p.nv = nv <= 1 ? 1 : nv <= 2 ? 2 : nv <= 4 ? 4 : 8;
+            return p;
+        }
+    }
+    return p;
+}
+
+// ------------------------------------------------------------------------------------------------
+// BN on tensors of 8 MB and more (batch-sized tensors, 56x56 maps): bandwidth, not latency, is the limit.
+//   reduce: one resident wave of CTAs streams the rows (eight 128-bit loads in flight per thread); the CTAs of a cluster
+//           add their per-channel sums through distributed shared memory, so that only a few dozen partial rows reach
+//           global memory and no CTA stays behind to combine hundreds of them;
+//   apply:  every CTA adds those few partials itself (fp64, fixed order) in its prologue - no ticket, no fence, no
+//           statistics round trip between the two kernels - then streams its rows; CTA 0 stores the statistics /
+//           parameter gradients.  The apply kernel walks its slab from the end: the rows the reduce kernel read last
+//           are the ones still in L2.
+// ------------------------------------------------------------------------------------------------
+constexpr int kBnBigCluster = 8;
+#ifndef HPF_BN_NB_F
+#define HPF_BN_NB_F 4           // rows per batch of loads: forward kernels (one operand)
+#endif
+#ifndef HPF_BN_NB_B
+#define HPF_BN_NB_B 2           // backward kernels (two operands)
+#endif
+constexpr int kBnBigMaxPartials = 37;            // 296 CTAs in clusters of 8
+
+template <bool BWD>
+__global__ void __launch_bounds__(kBnThreads, 2)
+bn_reduce_big_kernel(const float4* __restrict__ x4, const float4* __restrict__ dy4, const float* __restrict__ gamma,
+                     const float* __restrict__ beta, const float* __restrict__ stats, int64_t rows, int C, int cgt, int rl,
+                     int64_t rows_per_blk, float* __restrict__ partials, float floor)
+{
+    namespace cgr = cooperative_groups;
+    cgr::cluster_group cluster = cgr::this_cluster();
+    __shared__ float sh[kBnThreads][8];
+    __shared__ float part[kBnThreads * 8];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int t = threadIdx.x;
+    const int cg_total = C / 4;                  // == cgt: one pass
+    const int my_rl = t / cgt, my_cg = t % cgt;
+    const int64_t r0 = (int64_t)blockIdx.x * rows_per_blk;
+    int64_t r1 = r0 + rows_per_blk;
+    if (r1 > rows) r1 = rows;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+    {
+        float4 p0, p1, gm, bt;
+        if (BWD) {
+            p0 = __ldg(reinterpret_cast<const float4*>(stats) + my_cg);
+            p1 = __ldg(reinterpret_cast<const float4*>(stats + C) + my_cg);
+            gm = __ldg(reinterpret_cast<const float4*>(gamma) + my_cg);
+            bt = __ldg(reinterpret_cast<const float4*>(beta) + my_cg);
+        } else {
+            p0 = __ldg(x4 + my_cg);                                                   // shift = first row
+        }
+        const float4* xp = x4 + (r0 + my_rl) * cg_total + my_cg;
+        const float4* dp = dy4 + (r0 + my_rl) * cg_total + my_cg;
+        const int64_t step = (int64_t)rl * cg_total;
+        const int n = r1 > r0 + my_rl ? (int)((r1 - r0 - my_rl + rl - 1) / rl) : 0;
+        // batches of predicated loads: every load of a batch is in flight before the first use (a scalar remainder
+        // loop would pay one memory round trip per row)
+        constexpr int NB = BWD ? HPF_BN_NB_B : HPF_BN_NB_F;
+        for (int k0 = 0; k0 < n; k0 += NB) {
+            float4 v[NB], g[BWD ? NB : 1];
+#pragma unroll
+            for (int j = 0; j < NB; ++j) if (k0 + j < n) v[j] = __ldg(xp + (k0 + j) * step);
+            if (BWD) {
+#pragma unroll
+                for (int j = 0; j < NB; ++j) if (k0 + j < n) g[j] = __ldg(dp + (k0 + j) * step);
+            }
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                if (k0 + j < n) {
+                    if (BWD) {
+                        float xh, dz;
+                        xh = bn_xhat(v[j].x, p0.x, p1.x); dz = bn_z(xh, gm.x, bt.x) > floor ? g[j].x : 0.f; a.x += dz; b.x = fmaf(dz, xh, b.x);
+                        xh = bn_xhat(v[j].y, p0.y, p1.y); dz = bn_z(xh, gm.y, bt.y) > floor ? g[j].y : 0.f; a.y += dz; b.y = fmaf(dz, xh, b.y);
+                        xh = bn_xhat(v[j].z, p0.z, p1.z); dz = bn_z(xh, gm.z, bt.z) > floor ? g[j].z : 0.f; a.z += dz; b.z = fmaf(dz, xh, b.z);
+                        xh = bn_xhat(v[j].w, p0.w, p1.w); dz = bn_z(xh, gm.w, bt.w) > floor ? g[j].w : 0.f; a.w += dz; b.w = fmaf(dz, xh, b.w);
+                    } else {
+                        float d;
+                        d = v[j].x - p0.x; a.x += d; b.x = fmaf(d, d, b.x);
+                        d = v[j].y - p0.y; a.y += d; b.y = fmaf(d, d, b.y);
+                        d = v[j].z - p0.z; a.z += d; b.z = fmaf(d, d, b.z);
+                        d = v[j].w - p0.w; a.w += d; b.w = fmaf(d, d, b.w);
+                    }
+                }
+            }
+        }
+    }
+    // the CTA's sums per channel: row lanes in a fixed order
+    if (cgt <= 16) {
+        for (int off = 16; off >= cgt; off >>= 1) {
+            a.x += __shfl_xor_sync(0xffffffffu, a.x, off); a.y += __shfl_xor_sync(0xffffffffu, a.y, off);
+            a.z += __shfl_xor_sync(0xffffffffu, a.z, off); a.w += __shfl_xor_sync(0xffffffffu, a.w, off);
+            b.x += __shfl_xor_sync(0xffffffffu, b.x, off); b.y += __shfl_xor_sync(0xffffffffu, b.y, off);
+            b.z += __shfl_xor_sync(0xffffffffu, b.z, off); b.w += __shfl_xor_sync(0xffffffffu, b.w, off);
+        }
+        const int warp = t >> 5, lane = t & 31;
+        if (lane < cgt) {
+            float* d = sh[warp * cgt + lane];
+            d[0] = a.x; d[1] = a.y; d[2] = a.z; d[3] = a.w; d[4] = b.x; d[5] = b.y; d[6] = b.z; d[7] = b.w;
+        }
+        __syncthreads();
+        if (t < cgt * 8) {
+            const int cgl = t >> 3, comp = t & 7;
+            float s = 0.f;
+#pragma unroll
+            for (int w = 0; w < kBnThreads / 32; ++w) s += sh[w * cgt + cgl][comp];
+            part[t] = s;
+        }
+    } else {
+        sh[t][0] = a.x; sh[t][1] = a.y; sh[t][2] = a.z; sh[t][3] = a.w;
+        sh[t][4] = b.x; sh[t][5] = b.y; sh[t][6] = b.z; sh[t][7] = b.w;
+        __syncthreads();
+        for (int o = t; o < cgt * 8; o += kBnThreads) {
+            const int cgl = o >> 3, comp = o & 7;
+            float s = 0.f;
+            for (int l = 0; l < rl; ++l) s += sh[l * cgt + cgl][comp];
+            part[o] = s;
+        }
+    }
+    cluster.sync();
+    // rank r adds the cluster's CTAs (ascending) for its eighth of the (channel group, component) pairs
+    const unsigned int rank = cluster.block_rank();
+    const int cl = blockIdx.x / kBnBigCluster;
+    for (int o = (int)rank * cgt + t; o < ((int)rank + 1) * cgt; o += kBnThreads) {
+        float s = 0.f;
+#pragma unroll
+        for (unsigned int r = 0; r < (unsigned int)kBnBigCluster; ++r) s += *cluster.map_shared_rank(&part[o], r);
+        const int cgl = o >> 3, comp = o & 7;
+        partials[((int64_t)cl * 2 + (comp >> 2)) * C + cgl * 4 + (comp & 3)] = s;
+    }
+    cluster.sync();
+}
+
+// Prologue of the big apply kernels: per-channel totals of the n_part partial rows (fp64, ascending), then the forward
+// statistics (mean, rstd) or the backward coefficients (sum dz / rows, sum dz*xhat / rows) into fin[0][c], fin[1][c].
+template <bool BWD>
+__device__ __forceinline__ void bn_big_finalise(const float* __restrict__ partials, int n_part, int64_t rows, int C, int cgt, int rl,
+                                                float eps, const float* __restrict__ x, float* __restrict__ out_a,
+                                                float* __restrict__ out_b, bool write_out, double (*shd)[8], float* fin)
+{
+    const int t = threadIdx.x;
+    const int my_rl = t / cgt, my_cg = t % cgt;
+    double acc[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+#pragma unroll 4
+    for (int k = my_rl; k < n_part; k += rl) {
+        const float4 va = __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 0) * C) + my_cg);
+        const float4 vb = __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 1) * C) + my_cg);
+        acc[0] += (double)va.x; acc[1] += (double)va.y; acc[2] += (double)va.z; acc[3] += (double)va.w;
+        acc[4] += (double)vb.x; acc[5] += (double)vb.y; acc[6] += (double)vb.z; acc[7] += (double)vb.w;
+    }
+    if (cgt <= 16) {
+        for (int off = 16; off >= cgt; off >>= 1) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], off);
+        }
+        const int warp = t >> 5, lane = t & 31;
+        double (*wsum)[8] = shd + kBnThreads / 2;
+        if (lane < cgt) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) wsum[warp * cgt + lane][j] = acc[j];
+        }
+        __syncthreads();
+        if (t < cgt * 8) {
+            const int cgl = t >> 3, comp = t & 7;
+            double s = 0.0;
+            for (int w = 0; w < kBnThreads / 32; ++w) s += wsum[w * cgt + cgl][comp];
+            shd[cgl][comp] = s;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) shd[t][j] = acc[j];
+        __syncthreads();
+        double s[8];
+        const bool mine = t < cgt;                 // thread t < cgt totals column group t (all eight components)
+        if (mine) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s[j] = 0.0;
+            for (int l = 0; l < rl; ++l) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) s[j] += shd[l * cgt + t][j];
+            }
+        }
+        __syncthreads();
+        if (mine) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) shd[t][j] = s[j];
+        }
+    }
+    __syncthreads();
+    const double inv_rows = 1.0 / (double)rows;
+    for (int cl = t; cl < cgt * 4; cl += kBnThreads) {
+        const int cgl = cl >> 2, e = cl & 3;
+        const double sa = shd[cgl][e], sb = shd[cgl][4 + e];
+        if (BWD) {
+            fin[cl] = (float)(sa * inv_rows);
+            fin[C + cl] = (float)(sb * inv_rows);
+            if (write_out) { out_a[cl] = (float)sa; out_b[cl] = (float)sb; }        // dbeta, dgamma
+        } else {
+            const double shift = (double)__ldg(x + cl);
+            const double ms = sa * inv_rows;
+            double var = sb * inv_rows - ms * ms;
+            if (var < 0.0) var = 0.0;
+            const float mean = (float)(shift + ms), rstd = (float)(1.0 / sqrt(var + (double)eps));
+            fin[cl] = mean; fin[C + cl] = rstd;
+            if (write_out) { out_a[cl] = mean; out_b[cl] = rstd; }
+        }
+    }
+    __syncthreads();
+}
+
+// dynamic shared memory of the big apply kernels: [512][8] doubles for the prologue, then 2*C floats
+inline size_t bn_big_apply_smem(int C) { return (size_t)kBnThreads * 8 * sizeof(double) + 2 * (size_t)C * sizeof(float); }
+
+__global__ void __launch_bounds__(kBnThreads, 2)
+bn_apply_big_fwd_kernel(const float4* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+                        const float* __restrict__ partials, int n_part, float eps, float* __restrict__ stats,
+                        float4* __restrict__ y, int64_t rows, int C, int cgt, int rl, int64_t rows_per_blk, float floor, int stream_out)
+{
+    extern __shared__ __align__(16) unsigned char bn_big_smem[];
+    double (*shd)[8] = reinterpret_cast<double (*)[8]>(bn_big_smem);
+    float* fin = reinterpret_cast<float*>(bn_big_smem + (size_t)kBnThreads * 8 * sizeof(double));
+    pdl_launch_dependents();
+    pdl_wait();
+    bn_big_finalise<false>(partials, n_part, rows, C, cgt, rl, eps, reinterpret_cast<const float*>(x), stats, stats + C,
+                           blockIdx.x == 0, shd, fin);
+    const int t = threadIdx.x, cg_total = C / 4;
+    const int my_rl = t / cgt, my_cg = t % cgt;
+    const int64_t r0 = (int64_t)blockIdx.x * rows_per_blk;
+    int64_t r1 = r0 + rows_per_blk;
+    if (r1 > rows) r1 = rows;
+    const float4 mu = *reinterpret_cast<const float4*>(fin + my_cg * 4);
+    const float4 rs = *reinterpret_cast<const float4*>(fin + C + my_cg * 4);
+    const float4 g = __ldg(reinterpret_cast<const float4*>(gamma) + my_cg);
+    const float4 b = __ldg(reinterpret_cast<const float4*>(beta) + my_cg);
+    const int64_t base = (r0 + my_rl) * cg_total + my_cg, step = (int64_t)rl * cg_total;
+    const int n = r1 > r0 + my_rl ? (int)((r1 - r0 - my_rl + rl - 1) / rl) : 0;
+    constexpr int NB = HPF_BN_NB_F;
+    for (int k0 = n - 1; k0 >= 0; k0 -= NB) {              // from the end of the slab, in batches of predicated loads
+        float4 v[NB];
+#pragma unroll
+        for (int j = 0; j < NB; ++j) if (k0 - j >= 0) v[j] = __ldg(x + base + (k0 - j) * step);
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+            if (k0 - j >= 0) {
+                float4 o;
+                o.x = fmaxf(bn_z(bn_xhat(v[j].x, mu.x, rs.x), g.x, b.x), floor);
+                o.y = fmaxf(bn_z(bn_xhat(v[j].y, mu.y, rs.y), g.y, b.y), floor);
+                o.z = fmaxf(bn_z(bn_xhat(v[j].z, mu.z, rs.z), g.z, b.z), floor);
+                o.w = fmaxf(bn_z(bn_xhat(v[j].w, mu.w, rs.w), g.w, b.w), floor);
+                if (stream_out) __stcs(y + base + (k0 - j) * step, o); else y[base + (k0 - j) * step] = o;
+            }
+        }
+    }
+}
+
+template <bool ADDEND, bool ACCUM>
+__global__ void __launch_bounds__(kBnThreads, 2)
+bn_apply_big_bwd_kernel(const float4* __restrict__ x, const float4* __restrict__ dy, const float* __restrict__ gamma,
+                        const float* __restrict__ beta, const float* __restrict__ stats, const float* __restrict__ partials,
+                        int n_part, float* __restrict__ dgamma, float* __restrict__ dbeta, const float4* __restrict__ addend,
+                        float4* __restrict__ dx, int64_t rows, int C, int cgt, int rl, int64_t rows_per_blk, float floor, int stream_out)
+{
+    extern __shared__ __align__(16) unsigned char bn_big_smem[];
+    double (*shd)[8] = reinterpret_cast<double (*)[8]>(bn_big_smem);
+    float* fin = reinterpret_cast<float*>(bn_big_smem + (size_t)kBnThreads * 8 * sizeof(double));
+    pdl_launch_dependents();
+    pdl_wait();
+    bn_big_finalise<true>(partials, n_part, rows, C, cgt, rl, 0.f, nullptr, dbeta, dgamma, blockIdx.x == 0, shd, fin);
+    const int t = threadIdx.x, cg_total = C / 4;
+    const int my_rl = t / cgt, my_cg = t % cgt;
+    const int64_t r0 = (int64_t)blockIdx.x * rows_per_blk;
+    int64_t r1 = r0 + rows_per_blk;
+    if (r1 > rows) r1 = rows;
+    const float4 ca = *reinterpret_cast<const float4*>(fin + my_cg * 4);
+    const float4 cb = *reinterpret_cast<const float4*>(fin + C + my_cg * 4);
+    const float4 mu = __ldg(reinterpret_cast<const float4*>(stats) + my_cg);
+    const float4 rs = __ldg(reinterpret_cast<const float4*>(stats + C) + my_cg);
+    const float4 g = __ldg(reinterpret_cast<const float4*>(gamma) + my_cg);
+    const float4 b = __ldg(reinterpret_cast<const float4*>(beta) + my_cg);
+    const int64_t base = (r0 + my_rl) * cg_total + my_cg, step = (int64_t)rl * cg_total;
+    const int n = r1 > r0 + my_rl ? (int)((r1 - r0 - my_rl + rl - 1) / rl) : 0;
+    constexpr int NB = HPF_BN_NB_B;
+    for (int k0 = n - 1; k0 >= 0; k0 -= NB) {
+        float4 v[NB], d[NB];
+#pragma unroll
+        for (int j = 0; j < NB; ++j) if (k0 - j >= 0) { v[j] = __ldg(x + base + (k0 - j) * step); d[j] = __ldg(dy + base + (k0 - j) * step); }
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+            if (k0 - j >= 0) {
+                const int64_t i = base + (k0 - j) * step;
+                float4 o;
+                o.x = bn_dx1(v[j].x, d[j].x, mu.x, rs.x, g.x, b.x, ca.x, cb.x, floor);
+                o.y = bn_dx1(v[j].y, d[j].y, mu.y, rs.y, g.y, b.y, ca.y, cb.y, floor);
+                o.z = bn_dx1(v[j].z, d[j].z, mu.z, rs.z, g.z, b.z, ca.z, cb.z, floor);
+                o.w = bn_dx1(v[j].w, d[j].w, mu.w, rs.w, g.w, b.w, ca.w, cb.w, floor);
+                if (ADDEND) { const float4 e = __ldg(addend + i); o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+                if (ACCUM) { const float4 e = dx[i]; o.x += e.x; o.y += e.y; o.z += e.z; o.w += e.w; }
+                if (stream_out) __stcs(dx + i, o); else dx[i] = o;
+            }
+        }
+    }
+}
+
+struct BnBigPlan { bool ok; int n_clusters, nblk_apply, stream_out; int64_t rows_per_blk, rows_per_blk_apply; };
+
+// Clusters of the reduce kernel that are resident together on this device (asked once per kernel).
+template <bool BWD>
+int bn_big_max_clusters()
+{
+    static int cached = -1;
+    if (cached >= 0) return cached;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kBnBigCluster * kBnBigMaxPartials); cfg.blockDim = dim3(kBnThreads);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kBnBigCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, bn_reduce_big_kernel<BWD>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+    cached = n;
+    return n;
+}
+
+template <bool BWD>
+BnBigPlan bn_big_plan(int64_t rows, int C, const BnPlan& p)
+{
+    BnBigPlan b = {false, 0, 0, 0, 0, 0};
+    if (!g_bn_cluster || C % 4 != 0 || p.passes != 1 || (p.cgt & (p.cgt - 1)) != 0 || rows * C < kBnLargeElems) return b;   // power of two: cgt * rl == block
+    int ncl = bn_big_max_clusters<BWD>();
+    if (ncl > kBnBigMaxPartials) ncl = kBnBigMaxPartials;
+    const int64_t want = rows / ((int64_t)p.rl * 8 * kBnBigCluster);          // at least eight rows per thread
+    if (want < ncl) ncl = (int)want;
+    if (ncl < 2 || ncl > p.nblk) return b;                                    // the scratch holds p.nblk partial rows
+    b.ok = true; b.n_clusters = ncl;
+    b.rows_per_blk = ceil_div64(rows, (int64_t)ncl * kBnBigCluster);
+    int64_t na = rows / ((int64_t)p.rl * 8);
+    if (na > 2 * 148) na = 2 * 148;
+    if (na < 1) na = 1;
+    b.rows_per_blk_apply = ceil_div64(rows, na);
+    b.nblk_apply = (int)ceil_div64(rows, b.rows_per_blk_apply);
+    b.stream_out = rows * C * (int64_t)sizeof(float) > (int64_t)(48 << 20) ? 1 : 0;   // input + output beyond L2: do not keep the output   // input + output beyond L2: do not keep the output
+    return b;
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_cluster_pdl(void (*kernel)(KArgs...), int grid, int block, int cluster, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = g_pdl_enabled ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 int ew_blocks(int64_t n_items)
@@ -733,6 +1233,20 @@ cudaError_t bnrelu_fwd(const float* x, const float* gamma, const float* beta, fl
     const float floor = relu ? 0.f : -INFINITY;
     unsigned int* ticket = reinterpret_cast<unsigned int*>(scratch);
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + 256);
+    const BnBigPlan bp = bn_big_plan<false>(rows, C, p);
+    if (bp.ok) {
+        static bool attr_set = false;
+        const size_t smem = bn_big_apply_smem(C);
+        if (!attr_set) { cudaFuncSetAttribute(bn_apply_big_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bn_big_apply_smem(2048)); attr_set = true; }
+        launch_cluster_pdl(bn_reduce_big_kernel<false>, bp.n_clusters * kBnBigCluster, kBnThreads, kBnBigCluster, st,
+                           reinterpret_cast<const float4*>(x), (const float4*)nullptr, gamma, beta, (const float*)nullptr, rows, C,
+                           p.cgt, p.rl, bp.rows_per_blk, partials, floor);
+        launch_pdl(bn_apply_big_fwd_kernel, bp.nblk_apply, kBnThreads, smem, st, reinterpret_cast<const float4*>(x), gamma, beta,
+                   (const float*)partials, bp.n_clusters, eps, stats, reinterpret_cast<float4*>(y), rows, C, p.cgt, p.rl,
+                   bp.rows_per_blk_apply, floor, bp.stream_out);
+        count(n_launch, 2);
+        return cudaGetLastError();
+    }
     launch_pdl(bn_reduce_kernel<false>, p.nblk, kBnThreads, 0, st, x, (const float*)nullptr, gamma, beta, (const float*)nullptr, eps, rows, C, p.cgt, p.rl,
                                                            p.passes, p.rows_per_blk, ticket, partials, stats, stats + C,
                                                            (float*)nullptr, floor);
@@ -745,13 +1259,65 @@ cudaError_t bnrelu_fwd(const float* x, const float* gamma, const float* beta, fl
 
 cudaError_t bnrelu_bwd(const float* x, const float* dy, const float* gamma, const float* beta, const float* stats,
                        float* dx, const float* addend, bool accumulate, float* dgamma, float* dbeta, int64_t rows,
-                       int C, void* scratch, cudaStream_t st, int64_t* n_launch, bool relu)
+                       int C, void* scratch, cudaStream_t st, int64_t* n_launch, bool relu, bool x_is_old)
 {
     const BnPlan p = bn_plan(rows, C);
     const float floor = relu ? 0.f : -INFINITY;
+    const BnClusterPlan cp = g_bn_cluster ? bn_cluster_plan(rows, C) : BnClusterPlan{false, 0, 0, 0, 0};
+    if (cp.ok) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(cp.n_clusters * kBnCluster); cfg.blockDim = dim3(kBnThreads); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = kBnCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = g_pdl_enabled ? 2 : 1;
+        const float4* x4 = reinterpret_cast<const float4*>(x);
+        const float4* dy4 = reinterpret_cast<const float4*>(dy);
+        const float4* ad4 = reinterpret_cast<const float4*>(addend);
+        float4* dx4 = reinterpret_cast<float4*>(dx);
+        const int early = x_is_old ? 1 : 0;
+        cudaError_t e;
+#define HPF_BN_CL(NV, A, B) e = cudaLaunchKernelEx(&cfg, bn_bwd_cluster_kernel<NV, A, B>, x4, dy4, gamma, beta, stats, ad4, dx4, dgamma, dbeta, rows, C, cp.cgc, cp.rows_per_cta, floor, early)
+#define HPF_BN_CL_NV(NV) do { if (addend && accumulate) HPF_BN_CL(NV, true, true); else if (addend) HPF_BN_CL(NV, true, false); \
+                              else if (accumulate) HPF_BN_CL(NV, false, true); else HPF_BN_CL(NV, false, false); } while (0)
+        if (cp.nv == 1) HPF_BN_CL_NV(1); else if (cp.nv == 2) HPF_BN_CL_NV(2); else if (cp.nv == 4) HPF_BN_CL_NV(4); else HPF_BN_CL_NV(8);
+#undef HPF_BN_CL_NV
+#undef HPF_BN_CL
+        count(n_launch, 1);
+        return e;
+    }
     unsigned int* ticket = reinterpret_cast<unsigned int*>(scratch);
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + 256);
     float* coef = partials + (size_t)p.nblk * 2 * C;
+    const BnBigPlan bp = bn_big_plan<true>(rows, C, p);
+    if (bp.ok) {
+        static bool attr_set = false;
+        const size_t smem = bn_big_apply_smem(C);
+        if (!attr_set) {
+            const int mx = (int)bn_big_apply_smem(2048);
+            cudaFuncSetAttribute(bn_apply_big_bwd_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx);
+            cudaFuncSetAttribute(bn_apply_big_bwd_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx);
+            cudaFuncSetAttribute(bn_apply_big_bwd_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx);
+            cudaFuncSetAttribute(bn_apply_big_bwd_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx);
+            attr_set = true;
+        }
+        const float4* x4 = reinterpret_cast<const float4*>(x);
+        const float4* dy4 = reinterpret_cast<const float4*>(dy);
+        const float4* ad4 = reinterpret_cast<const float4*>(addend);
+        float4* dx4 = reinterpret_cast<float4*>(dx);
+        launch_cluster_pdl(bn_reduce_big_kernel<true>, bp.n_clusters * kBnBigCluster, kBnThreads, kBnBigCluster, st, x4, dy4, gamma, beta,
+                           stats, rows, C, p.cgt, p.rl, bp.rows_per_blk, partials, floor);
+#define HPF_BN_BIG(A, B) launch_pdl(bn_apply_big_bwd_kernel<A, B>, bp.nblk_apply, kBnThreads, smem, st, x4, dy4, gamma, beta, stats, (const float*)partials, bp.n_clusters, dgamma, dbeta, ad4, dx4, rows, C, p.cgt, p.rl, bp.rows_per_blk_apply, floor, bp.stream_out)
+        if (addend && accumulate) HPF_BN_BIG(true, true);
+        else if (addend) HPF_BN_BIG(true, false);
+        else if (accumulate) HPF_BN_BIG(false, true);
+        else HPF_BN_BIG(false, false);
+#undef HPF_BN_BIG
+        count(n_launch, 2);
+        return cudaGetLastError();
+    }
     launch_pdl(bn_reduce_kernel<true>, p.nblk, kBnThreads, 0, st, x, dy, gamma, beta, stats, 0.f, rows, C, p.cgt, p.rl, p.passes,
                                                           p.rows_per_blk, ticket, partials, dbeta, dgamma, coef, floor);
     const float4* x4 = reinterpret_cast<const float4*>(x);
