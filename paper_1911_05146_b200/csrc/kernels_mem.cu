@@ -468,6 +468,106 @@ bn_bwd_cluster_kernel(const float4* __restrict__ x, const float4* __restrict__ d
     cluster.barrier_wait();                                 // shared memory stays alive until every CTA has read it
 }
 
+// The forward twin: statistics and y = max(gamma * xhat + beta, floor) in one launch, x read once into registers.
+// Sums are shifted by the tensor's first row (the same shift in every CTA, so the partial sums add up).
+template <int NV>
+__global__ void __launch_bounds__(kBnThreads)
+bn_fwd_cluster_kernel(const float4* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta, float eps,
+                      float4* __restrict__ y, float* __restrict__ stats, int64_t rows, int C, int cgc, int64_t rows_per_cta,
+                      float floor)
+{
+    namespace cgr = cooperative_groups;
+    cgr::cluster_group cluster = cgr::this_cluster();
+    __shared__ float wpart[kBnThreads / 32][kBnClusterMaxCgc * 8];
+    __shared__ float part[kBnClusterMaxCgc * 8];
+    __shared__ float coefs[kBnClusterMaxCgc * 8];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int t = threadIdx.x;
+    const unsigned int rank = cluster.block_rank();
+    const int cl = blockIdx.x / kBnCluster;
+    const int cg_total = C / 4;
+    const int rl = kBnThreads / cgc;
+    const int my_cg = t % cgc, my_rl = t / cgc;
+    const int cg = cl * cgc + my_cg;
+    const int64_t r0 = (int64_t)rank * rows_per_cta;
+    int64_t r1 = r0 + rows_per_cta;
+    if (r1 > rows) r1 = rows;
+    int n = r1 > r0 + my_rl ? (int)((r1 - r0 - my_rl + rl - 1) / rl) : 0;
+    if (n > NV) n = NV;
+    const int64_t base = (r0 + my_rl) * cg_total + cg, step = (int64_t)rl * cg_total;
+    const float4 p0 = __ldcg(x + cg);                                              // shift = first row
+    const float4 gm = __ldg(reinterpret_cast<const float4*>(gamma) + cg);
+    const float4 bt = __ldg(reinterpret_cast<const float4*>(beta) + cg);
+    float4 xv[NV];
+#pragma unroll
+    for (int k = 0; k < NV; ++k) if (k < n) xv[k] = __ldcg(x + base + k * step);
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+        if (k < n) {
+            float d;
+            d = xv[k].x - p0.x; a.x += d; b.x = fmaf(d, d, b.x);
+            d = xv[k].y - p0.y; a.y += d; b.y = fmaf(d, d, b.y);
+            d = xv[k].z - p0.z; a.z += d; b.z = fmaf(d, d, b.z);
+            d = xv[k].w - p0.w; a.w += d; b.w = fmaf(d, d, b.w);
+        }
+    }
+    for (int off = 16; off >= cgc; off >>= 1) {
+        a.x += __shfl_xor_sync(0xffffffffu, a.x, off); a.y += __shfl_xor_sync(0xffffffffu, a.y, off);
+        a.z += __shfl_xor_sync(0xffffffffu, a.z, off); a.w += __shfl_xor_sync(0xffffffffu, a.w, off);
+        b.x += __shfl_xor_sync(0xffffffffu, b.x, off); b.y += __shfl_xor_sync(0xffffffffu, b.y, off);
+        b.z += __shfl_xor_sync(0xffffffffu, b.z, off); b.w += __shfl_xor_sync(0xffffffffu, b.w, off);
+    }
+    const int warp = t >> 5, lane = t & 31;
+    if (lane < cgc) {
+        float* d = &wpart[warp][lane * 8];
+        d[0] = a.x; d[1] = a.y; d[2] = a.z; d[3] = a.w; d[4] = b.x; d[5] = b.y; d[6] = b.z; d[7] = b.w;
+    }
+    __syncthreads();
+    if (t < cgc * 8) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < kBnThreads / 32; ++w) s += wpart[w][t];
+        part[t] = s;
+    }
+    cluster.sync();
+    if (t < cgc * 4) {                                      // one thread per channel of the slice: (group, element)
+        const int cgl = t >> 2, e = t & 3;
+        double sa = 0.0, sb = 0.0;
+#pragma unroll
+        for (unsigned int r = 0; r < (unsigned int)kBnCluster; ++r) {
+            const float* rp = cluster.map_shared_rank(&part[cgl * 8], r);
+            sa += (double)rp[e]; sb += (double)rp[4 + e];
+        }
+        const int c = (cl * cgc + cgl) * 4 + e;
+        const double inv_rows = 1.0 / (double)rows;
+        const double shift = (double)__ldcg(reinterpret_cast<const float*>(x) + c);
+        const double ms = sa * inv_rows;
+        double var = sb * inv_rows - ms * ms;
+        if (var < 0.0) var = 0.0;
+        const float mean = (float)(shift + ms), rstd = (float)(1.0 / sqrt(var + (double)eps));
+        coefs[cgl * 8 + e] = mean; coefs[cgl * 8 + 4 + e] = rstd;
+        if (rank == 0) { stats[c] = mean; stats[C + c] = rstd; }
+    }
+    __syncthreads();
+    cluster.barrier_arrive();
+    const float4 mu = *reinterpret_cast<const float4*>(&coefs[my_cg * 8]);
+    const float4 rs = *reinterpret_cast<const float4*>(&coefs[my_cg * 8 + 4]);
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+        if (k < n) {
+            float4 o;
+            o.x = fmaxf(bn_z(bn_xhat(xv[k].x, mu.x, rs.x), gm.x, bt.x), floor);
+            o.y = fmaxf(bn_z(bn_xhat(xv[k].y, mu.y, rs.y), gm.y, bt.y), floor);
+            o.z = fmaxf(bn_z(bn_xhat(xv[k].z, mu.z, rs.z), gm.z, bt.z), floor);
+            o.w = fmaxf(bn_z(bn_xhat(xv[k].w, mu.w, rs.w), gm.w, bt.w), floor);
+            y[base + k * step] = o;
+        }
+    }
+    cluster.barrier_wait();
+}
+
 struct BnClusterPlan { bool ok; int cgc, n_clusters, nv; int64_t rows_per_cta; };
 
 // Eligible: micro-batch sized tensors whose rows fit the registers of kBnCluster CTAs per column-group slice.  Prefers few
@@ -1233,6 +1333,19 @@ cudaError_t bnrelu_fwd(const float* x, const float* gamma, const float* beta, fl
     const float floor = relu ? 0.f : -INFINITY;
     unsigned int* ticket = reinterpret_cast<unsigned int*>(scratch);
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + 256);
+    const BnClusterPlan cp = g_bn_cluster ? bn_cluster_plan(rows, C) : BnClusterPlan{false, 0, 0, 0, 0};
+    if (cp.ok) {
+        const float4* x4 = reinterpret_cast<const float4*>(x);
+        float4* y4 = reinterpret_cast<float4*>(y);
+        const int grid = cp.n_clusters * kBnCluster;
+        cudaError_t e;
+        if (cp.nv == 1) e = launch_cluster_pdl(bn_fwd_cluster_kernel<1>, grid, kBnThreads, kBnCluster, st, x4, gamma, beta, eps, y4, stats, rows, C, cp.cgc, cp.rows_per_cta, floor);
+        else if (cp.nv == 2) e = launch_cluster_pdl(bn_fwd_cluster_kernel<2>, grid, kBnThreads, kBnCluster, st, x4, gamma, beta, eps, y4, stats, rows, C, cp.cgc, cp.rows_per_cta, floor);
+        else if (cp.nv == 4) e = launch_cluster_pdl(bn_fwd_cluster_kernel<4>, grid, kBnThreads, kBnCluster, st, x4, gamma, beta, eps, y4, stats, rows, C, cp.cgc, cp.rows_per_cta, floor);
+        else e = launch_cluster_pdl(bn_fwd_cluster_kernel<8>, grid, kBnThreads, kBnCluster, st, x4, gamma, beta, eps, y4, stats, rows, C, cp.cgc, cp.rows_per_cta, floor);
+        count(n_launch, 1);
+        return e;
+    }
     const BnBigPlan bp = bn_big_plan<false>(rows, C, p);
     if (bp.ok) {
         static bool attr_set = false;
