@@ -1084,26 +1084,44 @@ wgrad_partials_reduce_kernel(const float* __restrict__ partials, float* __restri
 
 // Weight preparation, once per step: for every convolution of the table (or the one passed by value), the hi / lo split of the weights
 // ([K][R][R][C], forward operand) and of the weights rearranged for the data gradient
-// (wt[c][R-1-r][R-1-s][k] = w[k][r][s][c]).  blockIdx.x = table entry, blockIdx.y strides over its elements.
+// (wt[c][R-1-r][R-1-s][k] = w[k][r][s][c]).  blockIdx.x = table entry; blockIdx.y strides over 32 x 32 tiles of the (k, c)
+// matrix of one filter tap, transposed through shared memory so that reads and all four writes are coalesced.
 __device__ __forceinline__ void weight_prep_one(const float* __restrict__ params, float* __restrict__ w_hi, float* __restrict__ w_lo,
                                                 float* __restrict__ wt_hi, float* __restrict__ wt_lo, const WeightPrepEntry e)
 {
+    __shared__ float sm[32][33];
     const int C = e.C, K = e.K, R = e.R;
-    const long long total = (long long)K * R * R * C;
-    const long long stride = (long long)gridDim.y * blockDim.x;
+    const int ct = (C + 31) / 32, kt = (K + 31) / 32;
+    const int n_tiles = R * R * ct * kt;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;          // 32 x 8 threads
     const float* w = params + e.w_off;
-    for (long long o = (long long)blockIdx.y * blockDim.x + threadIdx.x; o < total; o += stride) {
-        // o indexes wt[c][r'][s'][k]
-        const int k = (int)(o % K);
-        long long t = o / K;
-        const int s2 = (int)(t % R); t /= R;
-        const int r2 = (int)(t % R);
-        const int c = (int)(t / R);
-        const long long src = (((long long)k * R + (R - 1 - r2)) * R + (R - 1 - s2)) * C + c;
-        const float v = __ldg(&w[src]);
-        const float h = tf32_hi(v);
-        wt_hi[e.w_off + o] = h; wt_lo[e.w_off + o] = v - h;
-        w_hi[e.w_off + src] = h; w_lo[e.w_off + src] = v - h;
+    for (int tile = blockIdx.y; tile < n_tiles; tile += gridDim.y) {
+        const int rs = tile / (ct * kt), rem = tile % (ct * kt);
+        const int k0 = (rem / ct) * 32, c0 = (rem % ct) * 32;
+        const int r = rs / R, s2 = rs % R;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int k = k0 + ty + 8 * j, c = c0 + tx;
+            if (k < K && c < C) {
+                const long long src = (((long long)k * R + r) * R + s2) * C + c;
+                const float v = __ldg(&w[src]);
+                const float h = tf32_hi(v);
+                w_hi[e.w_off + src] = h; w_lo[e.w_off + src] = v - h;
+                sm[ty + 8 * j][tx] = v;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = c0 + ty + 8 * j, k = k0 + tx;
+            if (c < C && k < K) {
+                const float v = sm[tx][ty + 8 * j];
+                const float h = tf32_hi(v);
+                const long long dst = (((long long)c * R + (R - 1 - r)) * R + (R - 1 - s2)) * K + k;
+                wt_hi[e.w_off + dst] = h; wt_lo[e.w_off + dst] = v - h;
+            }
+        }
+        __syncthreads();
     }
 }
 __global__ void __launch_bounds__(256)
@@ -1555,11 +1573,16 @@ cudaError_t conv_tc_launch(const ConvTcPlan* plan, DeviceStatus* status, cudaStr
     return cudaGetLastError();
 }
 
+int conv_weight_prep_tiles(int C, int K, int R) { return R * R * ((C + 31) / 32) * ((K + 31) / 32); }
+
 cudaError_t conv_weight_prep(const float* params, float* w_hi, float* w_lo, float* wt_hi, float* wt_lo,
-                             const WeightPrepEntry* d_table, int n_entries, cudaStream_t st, int64_t* n_launch)
+                             const WeightPrepEntry* d_table, int n_entries, int max_tiles, cudaStream_t st, int64_t* n_launch)
 {
     if (n_entries < 1) return cudaSuccess;
-    weight_prep_kernel<<<dim3(n_entries, 4), 256, 0, st>>>(params, w_hi, w_lo, wt_hi, wt_lo, d_table);
+    int gy = max_tiles < 1 ? 1 : max_tiles;                  // tiles of the largest entry; smaller entries leave blocks idle
+    const int cap = n_entries >= 16 ? 64 : 2048;
+    if (gy > cap) gy = cap;
+    weight_prep_kernel<<<dim3(n_entries, gy), 256, 0, st>>>(params, w_hi, w_lo, wt_hi, wt_lo, d_table);
     count(n_launch, 1);
     return cudaGetLastError();
 }
@@ -1568,7 +1591,9 @@ cudaError_t conv_weight_prep_single(const float* w, float* w_hi, float* w_lo, fl
                                     cudaStream_t st, int64_t* n_launch)
 {
     WeightPrepEntry e{0, C, K, R, 0};
-    weight_prep_single_kernel<<<dim3(1, 16), 256, 0, st>>>(w, w_hi, w_lo, wt_hi, wt_lo, e);
+    int gy = conv_weight_prep_tiles(C, K, R);
+    if (gy > 2048) gy = 2048;
+    weight_prep_single_kernel<<<dim3(1, gy), 256, 0, st>>>(w, w_hi, w_lo, wt_hi, wt_lo, e);
     count(n_launch, 1);
     return cudaGetLastError();
 }

@@ -75,7 +75,9 @@ struct WeightPrepEntry { long long w_off; int C, K, R, reserved; };
 // For every table entry (device memory): w_hi/w_lo = hi/lo split of the weights, wt_hi/wt_lo = split of the weights
 // rearranged for the data gradient (wt[c][R-1-r][R-1-s][k] = w[k][r][s][c]); all four use the entry's w_off.
 cudaError_t conv_weight_prep(const float* params, float* w_hi, float* w_lo, float* wt_hi, float* wt_lo,
-                             const WeightPrepEntry* d_table, int n_entries, cudaStream_t st, int64_t* n_launch);
+                             const WeightPrepEntry* d_table, int n_entries, int max_tiles, cudaStream_t st, int64_t* n_launch);
+// 32 x 32 tiles the preparation kernel walks for one convolution (max_tiles above = the largest of the table)
+int conv_weight_prep_tiles(int C, int K, int R);
 
 cudaError_t conv_weight_prep_single(const float* w, float* w_hi, float* w_lo, float* wt_hi, float* wt_lo, int C, int K, int R,
                                     cudaStream_t st, int64_t* n_launch);

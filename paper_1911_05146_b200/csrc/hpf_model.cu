@@ -4,6 +4,7 @@
 #include "conv_tc.h"
 #include "hpf_kernels.h"
 
+#include <algorithm>
 #include <chrono>
 #include <cstdlib>
 #include <cstdio>
@@ -652,9 +653,11 @@ int enqueue_phase(hpf_model* mdl, int phase)
             if (!mdl->prep_table[p].empty()) {
                 float* wp = reinterpret_cast<float*>(mdl->ws + mdl->wprep_off);
                 const int64_t G4 = (mdl->G + 3) / 4 * 4;      // keeps every array 16-byte aligned
+                int max_tiles = 1;
+                for (const WeightPrepEntry& e : mdl->prep_table[p]) max_tiles = std::max(max_tiles, conv_weight_prep_tiles(e.C, e.K, e.R));
                 CU(conv_weight_prep(mdl->params, wp, wp + G4, wp + 2 * G4, wp + 3 * G4,
                                     reinterpret_cast<const WeightPrepEntry*>(mdl->ws + mdl->prep_table_off[p]),
-                                    (int)mdl->prep_table[p].size(), mdl->stream_of(p), &mdl->launches));
+                                    (int)mdl->prep_table[p].size(), max_tiles, mdl->stream_of(p), &mdl->launches));
             }
         // tick t: every (p, m) with p + m = t
         for (int t = 0; t < P + M - 1; ++t)
