@@ -1459,11 +1459,13 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     const int kchunk = chunk_of(v.c_in);
     int n_chunk = v.c_out < 256 ? v.c_out : 256;
     {
-        // A launch with few pixel tiles leaves most SMs idle: twice as many channel slices of 128 (each CTA issues the
-        // same number of MMAs at half the width) fill them.  Not when BN work rides in the kernel (one slice there).
+        // A launch with few pixel tiles leaves most SMs idle: twice as many channel slices of 128 (two MMAs of the stacked
+        // width per K step instead of three) fill them.  When BN work rides in the kernel every slice repeats the BN on its
+        // copy of the activation tile, which only pays when the K loop is long (the wide convolutions of the ImageNet layout).
         const int tiles = ((v.Q + b.w - 1) / b.w) * ((v.P + b.h - 1) / b.h) * ((v.N + b.n - 1) / b.n);
         const bool fused = fuse && (fuse->mode || fuse->in_mode);
-        if (!fused && v.c_out % 256 == 0 && tiles * (v.c_out / 256) <= 74) n_chunk = 128;
+        const int ksteps = v.R * v.R * v.c_in / 8;
+        if ((!fused || ksteps >= 64) && v.c_out % 256 == 0 && tiles * (v.c_out / 256) <= 74) n_chunk = 128;
     }
     {
         cuuint64_t dims[4] = {(cuuint64_t)v.c_in, (cuuint64_t)v.in_w, (cuuint64_t)v.in_h, (cuuint64_t)v.N};
