@@ -1313,6 +1313,127 @@ head_bwd_param_kernel(const float* __restrict__ dlogits, const float* __restrict
     }
 }
 
+// ---- wide heads (ImageNet layout: 2048 channels x 1000 classes): the same arithmetic spread over the GPU ----
+// pooled[n][c] = mean over the map; grid (ceil(C/256), b)
+__global__ void __launch_bounds__(kThreads)
+head_pool_kernel(const float* __restrict__ a, float* __restrict__ pooled, int HW, int C)
+{
+    const int c = blockIdx.x * kThreads + threadIdx.x, n = blockIdx.y;
+    if (c >= C) return;
+    float s = 0.f;
+    for (int i = 0; i < HW; ++i) s += __ldg(&a[((int64_t)n * HW + i) * C + c]);
+    pooled[(int64_t)n * C + c] = s * (1.f / (float)HW);
+}
+
+// logits[n][j] = pooled[n] . W[j] + bias[j]: one warp per class (a row of W is read once for eight samples at a time)
+__global__ void __launch_bounds__(kThreads)
+head_logits_kernel(const float* __restrict__ pooled, const float* __restrict__ Wfc, const float* __restrict__ bias,
+                   float* __restrict__ logits, int b, int C, int ncls)
+{
+    const int lane = threadIdx.x & 31, j = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    if (j >= ncls) return;
+    for (int n0 = 0; n0 < b; n0 += 8) {
+        float acc[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) acc[q] = 0.f;
+        for (int c = lane; c < C; c += 32) {
+            const float w = __ldg(&Wfc[(int64_t)j * C + c]);
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (n0 + q < b) acc[q] = fmaf(pooled[(int64_t)(n0 + q) * C + c], w, acc[q]);
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float sum = warp_sum(acc[q]);
+            if (lane == 0 && n0 + q < b) logits[(int64_t)(n0 + q) * ncls + j] = sum + __ldg(&bias[j]);
+        }
+    }
+}
+
+// per-sample loss from the logits; one block per sample
+__global__ void __launch_bounds__(kThreads)
+head_softmax_loss_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, float* __restrict__ persample, int ncls)
+{
+    __shared__ float red[32];
+    const int n = blockIdx.x, t = threadIdx.x;
+    const float* lg = logits + (int64_t)n * ncls;
+    float mx = -INFINITY;
+    for (int j = t; j < ncls; j += blockDim.x) mx = fmaxf(mx, lg[j]);
+    mx = block_reduce(mx, true, red);
+    float z = 0.f;
+    for (int j = t; j < ncls; j += blockDim.x) z += expf(lg[j] - mx);
+    z = block_reduce(z, false, red);
+    if (t == 0) persample[n] = -(lg[labels[n]] - mx - logf(z));
+}
+
+// dlogits = (softmax - onehot) / b; one block per sample
+__global__ void __launch_bounds__(kThreads)
+head_dlogits_kernel(const int32_t* __restrict__ labels, const float* __restrict__ logits, float* __restrict__ dlogits, int b, int ncls)
+{
+    __shared__ float red[32];
+    const int n = blockIdx.x, t = threadIdx.x;
+    const float* lg = logits + (int64_t)n * ncls;
+    float mx = -INFINITY;
+    for (int j = t; j < ncls; j += blockDim.x) mx = fmaxf(mx, __ldg(&lg[j]));
+    mx = block_reduce(mx, true, red);
+    float z = 0.f;
+    for (int j = t; j < ncls; j += blockDim.x) z += expf(__ldg(&lg[j]) - mx);
+    z = block_reduce(z, false, red);
+    const int lab = labels[n];
+    const float invb = 1.f / (float)b;
+    for (int j = t; j < ncls; j += blockDim.x) {
+        const float p = expf(__ldg(&lg[j]) - mx) / z;
+        dlogits[(int64_t)n * ncls + j] = (p - (j == lab ? 1.f : 0.f)) * invb;
+    }
+}
+
+// da[n][i][c] = (dlogits[n] . W[:, c]) / HW for every pixel i.  A block owns 64 channels and 8 samples; its 256 threads are
+// 64 channels x 4 interleaved class slices (added in slice order).  grid (ceil(C/64), ceil(b/8)); dynamic smem 8*ncls floats.
+__global__ void __launch_bounds__(kThreads)
+head_bwd_pool_kernel(const float* __restrict__ Wfc, const float* __restrict__ dlogits, float* __restrict__ da, int b, int HW,
+                     int C, int ncls)
+{
+    extern __shared__ float sd[];                      // [8][ncls]
+    __shared__ float red[4][8][64];
+    __shared__ float res[8][64];
+    const int t = threadIdx.x, cl = t & 63, js = t >> 6;
+    const int c0 = blockIdx.x * 64, n0 = blockIdx.y * 8;
+    for (int idx = t; idx < 8 * ncls; idx += kThreads) {
+        const int q = idx / ncls, j = idx - q * ncls;
+        sd[idx] = n0 + q < b ? __ldg(&dlogits[(int64_t)(n0 + q) * ncls + j]) : 0.f;
+    }
+    __syncthreads();
+    float acc[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) acc[q] = 0.f;
+    const int c = c0 + cl;
+    if (c < C) {
+#pragma unroll 4
+        for (int j = js; j < ncls; j += 4) {
+            const float w = __ldg(&Wfc[(int64_t)j * C + c]);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc[q] = fmaf(sd[q * ncls + j], w, acc[q]);
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) red[js][q][cl] = acc[q];
+    __syncthreads();
+    const float inv = 1.f / (float)HW;
+    for (int o = t; o < 8 * 64; o += kThreads) {
+        const int q = o >> 6, k = o & 63;
+        res[q][k] = (((red[0][q][k] + red[1][q][k]) + red[2][q][k]) + red[3][q][k]) * inv;
+    }
+    __syncthreads();
+    const int total = 8 * HW * 64;
+    for (int idx = t; idx < total; idx += kThreads) {
+        const int k = idx & 63, rest = idx >> 6;
+        const int i = rest % HW, q = rest / HW;
+        if (n0 + q < b && c0 + k < C) da[((int64_t)(n0 + q) * HW + i) * C + c0 + k] = res[q][k];
+    }
+}
+
+inline bool head_is_wide(int C, int ncls) { return ncls >= 64 && (int64_t)C * ncls >= 32768; }   // one warp per class: needs many classes
+
 inline void count(int64_t* n_launch, int k) { if (n_launch) *n_launch += k; }
 
 }  // namespace
@@ -1550,6 +1671,14 @@ cudaError_t head_fwd(const float* a, const float* Wfc, const float* bias, const 
                      float* pooled, float* persample, float* loss_slot, int b, int HW, int C, int ncls,
                      cudaStream_t st, int64_t* n_launch)
 {
+    if (head_is_wide(C, ncls)) {
+        head_pool_kernel<<<dim3((C + kThreads - 1) / kThreads, b), kThreads, 0, st>>>(a, pooled, HW, C);
+        head_logits_kernel<<<(ncls + kThreads / 32 - 1) / (kThreads / 32), kThreads, 0, st>>>(pooled, Wfc, bias, logits, b, C, ncls);
+        head_softmax_loss_kernel<<<b, kThreads, 0, st>>>(logits, labels, persample, ncls);
+        head_loss_kernel<<<1, 32, 0, st>>>(persample, loss_slot, b);
+        count(n_launch, 4);
+        return cudaGetLastError();
+    }
     const size_t smem = (size_t)(C + ncls) * sizeof(float);
     head_fwd_kernel<<<b, kThreads, smem, st>>>(a, Wfc, bias, labels, logits, pooled, persample, HW, C, ncls);
     head_loss_kernel<<<1, 32, 0, st>>>(persample, loss_slot, b);
@@ -1561,6 +1690,13 @@ cudaError_t head_bwd(const float* Wfc, const int32_t* labels, const float* logit
                      float* dlogits, float* da, float* dW, float* dbias, int b, int HW, int C, int ncls,
                      cudaStream_t st, int64_t* n_launch)
 {
+    if (head_is_wide(C, ncls) && (size_t)8 * ncls * sizeof(float) <= 40 * 1024) {
+        head_dlogits_kernel<<<b, kThreads, 0, st>>>(labels, logits, dlogits, b, ncls);
+        head_bwd_pool_kernel<<<dim3((C + 63) / 64, (b + 7) / 8), kThreads, (size_t)8 * ncls * sizeof(float), st>>>(Wfc, dlogits, da, b, HW, C, ncls);
+        head_bwd_param_kernel<<<ncls, kThreads, 0, st>>>(dlogits, pooled, dW, dbias, b, C, ncls);
+        count(n_launch, 3);
+        return cudaGetLastError();
+    }
     head_bwd_data_kernel<<<b, kThreads, (size_t)ncls * sizeof(float), st>>>(Wfc, labels, logits, dlogits, da, b, HW, C, ncls);
     head_bwd_param_kernel<<<ncls, kThreads, 0, st>>>(dlogits, pooled, dW, dbias, b, C, ncls);
     count(n_launch, 2);

@@ -142,6 +142,13 @@ def test_imagenet_layout_wide_channels():
     check_step(ops, (32, 32, 3), 4, 2, [9, 20], seed=3, bn_jitter=0.2)
 
 
+def test_many_class_head_on_ragged_sizes():
+    """The head kernels for many classes (one warp per class, 64-channel x 8-sample blocks in the backward): 350 classes on
+    96 channels with micro-batches of 3 samples, so that no block or warp loop is full."""
+    ops = wl.resnet_v2_imagenet(blocks=(1, 1), widths=(16, 24), n_classes=350)
+    check_step(ops, (32, 32, 3), 6, 2, [7], seed=11, bn_jitter=0.2)
+
+
 def test_second_step_and_new_inputs_reuse_the_model():
     c = wl.config("r11")
     ops = c["ops"]
