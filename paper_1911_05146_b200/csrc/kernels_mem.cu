@@ -1189,6 +1189,59 @@ maxpool_bwd_kernel(const float* __restrict__ x, const float* __restrict__ dy, fl
     }
 }
 
+// The same routing, four channels per thread (C a multiple of 4): a quarter of the load instructions.
+template <bool ACCUM>
+__global__ void __launch_bounds__(kThreads)
+maxpool_bwd_vec4_kernel(const float4* __restrict__ x, const float4* __restrict__ dy, float4* __restrict__ dx, ConvShape s)
+{
+    const int C4 = s.C / 4;
+    const int64_t total = (int64_t)s.N * s.H * s.W * C4;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int c = (int)(i % C4);
+        int64_t r = i / C4;
+        const int w = (int)(r % s.W); r /= s.W;
+        const int h = (int)(r % s.H);
+        const int n = (int)(r / s.H);
+        const float4 mine = __ldg(&x[i]);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        int p_lo = h + s.pad - s.R + 1; p_lo = p_lo <= 0 ? 0 : (p_lo + s.stride - 1) / s.stride;
+        int p_hi = (h + s.pad) / s.stride; if (p_hi > s.P - 1) p_hi = s.P - 1;
+        int q_lo = w + s.pad - s.R + 1; q_lo = q_lo <= 0 ? 0 : (q_lo + s.stride - 1) / s.stride;
+        int q_hi = (w + s.pad) / s.stride; if (q_hi > s.Q - 1) q_hi = s.Q - 1;
+        for (int p = p_lo; p <= p_hi; ++p) {
+            const int h0 = p * s.stride - s.pad;
+            for (int q = q_lo; q <= q_hi; ++q) {
+                const int w0 = q * s.stride - s.pad;
+                bool f0 = true, f1 = true, f2 = true, f3 = true;          // still the first maximum of this window
+                for (int rr = 0; rr < s.R; ++rr) {
+                    const int ih = h0 + rr;
+                    if (ih < 0 || ih >= s.H) continue;
+                    for (int ss = 0; ss < s.R; ++ss) {
+                        const int iw = w0 + ss;
+                        if (iw < 0 || iw >= s.W) continue;
+                        const float4 v = __ldg(&x[(((int64_t)n * s.H + ih) * s.W + iw) * C4 + c]);
+                        const bool before = (ih < h) || (ih == h && iw < w);
+                        f0 = f0 && !(v.x > mine.x || (before && v.x == mine.x));
+                        f1 = f1 && !(v.y > mine.y || (before && v.y == mine.y));
+                        f2 = f2 && !(v.z > mine.z || (before && v.z == mine.z));
+                        f3 = f3 && !(v.w > mine.w || (before && v.w == mine.w));
+                    }
+                }
+                if (f0 || f1 || f2 || f3) {
+                    const float4 g = __ldg(&dy[(((int64_t)n * s.P + p) * s.Q + q) * C4 + c]);
+                    if (f0) acc.x += g.x;
+                    if (f1) acc.y += g.y;
+                    if (f2) acc.z += g.z;
+                    if (f3) acc.w += g.w;
+                }
+            }
+        }
+        if (ACCUM) { const float4 e = dx[i]; acc.x += e.x; acc.y += e.y; acc.z += e.z; acc.w += e.w; }
+        dx[i] = acc;
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // head: global average pool + FC + softmax cross-entropy
 // ------------------------------------------------------------------------------------------------
@@ -1660,6 +1713,17 @@ cudaError_t maxpool_fwd(const float* x, float* y, ConvShape s, cudaStream_t st, 
 cudaError_t maxpool_bwd(const float* x, const float* dy, float* dx, bool accumulate, ConvShape s, cudaStream_t st,
                         int64_t* n_launch)
 {
+    const bool vec4 = s.C % 4 == 0 && ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(dy) | reinterpret_cast<uintptr_t>(dx)) & 15u) == 0;
+    if (vec4) {
+        const int nb = ew_blocks((int64_t)s.N * s.H * s.W * (s.C / 4));
+        const float4* x4 = reinterpret_cast<const float4*>(x);
+        const float4* dy4 = reinterpret_cast<const float4*>(dy);
+        float4* dx4 = reinterpret_cast<float4*>(dx);
+        if (accumulate) maxpool_bwd_vec4_kernel<true><<<nb, kThreads, 0, st>>>(x4, dy4, dx4, s);
+        else maxpool_bwd_vec4_kernel<false><<<nb, kThreads, 0, st>>>(x4, dy4, dx4, s);
+        count(n_launch, 1);
+        return cudaGetLastError();
+    }
     const int nb = ew_blocks((int64_t)s.N * s.H * s.W * s.C);
     if (accumulate) maxpool_bwd_kernel<true><<<nb, kThreads, 0, st>>>(x, dy, dx, s);
     else maxpool_bwd_kernel<false><<<nb, kThreads, 0, st>>>(x, dy, dx, s);
