@@ -46,6 +46,10 @@ constexpr long long kWaitLimit = 4000000000LL;   // clock64 ticks (~2 s) before 
 constexpr uint32_t kSmemBudget = 200 * 1024;
 constexpr uint32_t kWgradSmemBudget = 220 * 1024;   // the weight-gradient kernel has next to no static shared memory
 constexpr int kFwdMaxStages = 4;
+#ifndef HPF_WGRAD_WANT
+#define HPF_WGRAD_WANT 96
+#endif
+constexpr int kWgradWantCtas = HPF_WGRAD_WANT;   // CTAs a weight-gradient launch spreads its pixel walk over at least
 constexpr int kMultiTileFrom = 2 * 296;     // CTAs (two per SM) beyond which a forward / data-gradient launch gives each CTA two tiles
 constexpr unsigned int kWgradSlack = 16384;   // an MMA reads 128 operand rows (16 KB) from a base that may be the last one in use
 
@@ -1304,7 +1308,7 @@ bool wgrad_geom(const ConvShape& s, int passes, WgradGeom* g, int max_ctas = 0)
     int cap = (int)(operand_bytes / (4.0 * dw_bytes));
     // small problems are latency bound, not byte bound: spread the pixel walk over several dozen CTAs
     const int ctas_per_split = g->tap_groups * (s.K / g->m_chunk) * (s.C / g->n_cols);
-    const int want = (48 + ctas_per_split - 1) / ctas_per_split;
+    const int want = (kWgradWantCtas + ctas_per_split - 1) / ctas_per_split;
     if (cap < want) cap = want;
     if (splits > cap) splits = cap;
     if (splits > 296) splits = 296;          // two CTAs per SM
