@@ -917,7 +917,10 @@ template <bool BWD>
 BnBigPlan bn_big_plan(int64_t rows, int C, const BnPlan& p)
 {
     BnBigPlan b = {false, 0, 0, 0, 0, 0};
-    if (!g_bn_cluster || C % 4 != 0 || p.passes != 1 || (p.cgt & (p.cgt - 1)) != 0 || rows * C < kBnLargeElems) return b;   // power of two: cgt * rl == block
+    if (!g_bn_cluster || C % 4 != 0 || p.passes != 1 || (p.cgt & (p.cgt - 1)) != 0) return b;   // power of two: cgt * rl == block
+    // large tensors, and wide ones (2048 channels: one row lane per block, so the last block of the ticket scheme would
+    // add its hundred partial rows one after the other)
+    if (rows * C < kBnLargeElems && p.nblk <= 16 * p.rl) return b;
     int ncl = bn_big_max_clusters<BWD>();
     if (ncl > kBnBigMaxPartials) ncl = kBnBigMaxPartials;
     const int64_t want = rows / ((int64_t)p.rl * 8 * kBnBigCluster);          // at least eight rows per thread
