@@ -580,7 +580,7 @@ BnClusterPlan bn_cluster_plan(int64_t rows, int C)
     const int64_t rpc = ceil_div64(rows, kBnCluster);
     static const int prefs[3] = {2, 4, 8};
     for (int pi = 0; pi < 3; ++pi) {
-        for (int cgc = kBnClusterMaxCgc; cgc >= 2; cgc >>= 1) {
+        for (int cgc = kBnClusterMaxCgc; cgc >= 2; cgc >>= 1) {       // a slice of one 16-byte group per row was tried: slower (half-used sectors)
             if (cg_total % cgc != 0) continue;
             const int n_clusters = cg_total / cgc;
             if (n_clusters > kBnClusterMaxActive) continue;
