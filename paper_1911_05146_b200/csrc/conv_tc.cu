@@ -266,6 +266,11 @@ struct FwdScalars {
     float bn_in_eps;
     double bn_in_inv_rows;
     float* bn_in_y;              // relu(bn(x)), dense [N][in_h][in_w][c_in], written by the CTAs of the first channel slice
+    // K loop split over gridDim.z CTAs (launches of a few tiles with a long K loop): every CTA stores its partial tile, the
+    // one that takes the last ticket of its (tile, channel slice) adds them in split order and writes the output
+    int ksplit;
+    float* splitk_partials;      // [(tile * slices + slice) * ksplit + z][128][n_chunk]
+    unsigned int* splitk_ticket; // one per (tile, slice); zero between launches
 };
 struct alignas(64) FwdParams {
     CUtensorMap tm_a;            // activations {C, Wv, Hv, N}
@@ -378,7 +383,7 @@ __device__ __forceinline__ void bn_combine_partials(const float* partials, int n
 // MULTI = false: one 128-pixel tile per CTA (the shortest launch; what a launch of up to one wave wants).
 // MULTI = true: p.tiles_per_cta tiles per CTA for launches of several waves: fewer CTAs, and a tile's write-out hides
 // the next tile's loads, split and MMAs.
-template <bool MULTI>
+template <bool MULTI, bool KSPLIT = false>
 __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_constant__ FwdParams gp)
 {
     __shared__ FwdScalars p;                 // scalar parameters, see load_scalars
@@ -436,6 +441,9 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
     pdl_wait();              // everything above touched only parameters, shared and tensor memory
     const uint32_t tmem_base = tmem_slot;
     const int total = p.R * p.R * p.n_kchunks;
+    // this CTA's share of the K loop (all of it unless the launch splits K over gridDim.z)
+    const int kb = KSPLIT ? (int)(((long long)total * blockIdx.z) / p.ksplit) : 0;
+    const int ke = KSPLIT ? (int)(((long long)total * (blockIdx.z + 1)) / p.ksplit) : total;
     if (threadIdx.x == 0) HPF_TL(1);
 
     if (warp == 0) {
@@ -445,7 +453,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             bool live = true;
             for (int j = 0; j < my_tiles && live; ++j) {
                 HPF_TILE_ORIGIN(tile0 + j);
-                for (int k = 0; k < total; ++k, ++it) {
+                for (int k = kb; k < ke; ++k, ++it) {
                     const int s = it % p.stages;
                     if (!mbar_wait(empty0 + 8 * s, ((it / p.stages) & 1) ^ 1, &abort_flag)) { report(p.status, 1); live = false; break; }
                     const int tap = k / p.n_kchunks, kc = k % p.n_kchunks;
@@ -477,7 +485,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             bool live = true;
             for (int j = 0; j < my_tiles && live; ++j) {
               const uint32_t acc = tmem_base + (uint32_t)j * acc_cols;
-              for (int k = 0; k < total; ++k, ++it) {
+              for (int k = kb; k < ke; ++k, ++it) {
                 if (!mbar_wait(full0 + 8 * s, par, &abort_flag)) { report(p.status, 2); live = false; break; }
                 if (split_first && !mbar_wait(split0 + 8 * s, par, &abort_flag)) { report(p.status, 6); live = false; break; }
                 tc_fence_after();
@@ -492,19 +500,19 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     // (columns [0,n) = hi*hi, [n,2n) = hi*lo, added in the epilogue), then A_lo x B_hi.
 #pragma unroll 4
                     for (int k8 = 0; k8 < k8n; ++k8) {
-                        umma_tf32(acc, a0 + 2 * k8, b0 + 2 * k8, idesc2, (k | k8) ? 1u : 0u);
+                        umma_tf32(acc, a0 + 2 * k8, b0 + 2 * k8, idesc2, ((k - kb) | k8) ? 1u : 0u);
                         umma_tf32(acc, al0 + 2 * k8, b0 + 2 * k8, idesc, 1u);
                     }
                 } else if (three) {
 #pragma unroll 4
                     for (int k8 = 0; k8 < k8n; ++k8) {
-                        umma_tf32(acc, a0 + 2 * k8, b0 + 2 * k8, idesc, (k | k8) ? 1u : 0u);
+                        umma_tf32(acc, a0 + 2 * k8, b0 + 2 * k8, idesc, ((k - kb) | k8) ? 1u : 0u);
                         umma_tf32(acc, al0 + 2 * k8, b0 + 2 * k8, idesc, 1u);
                         umma_tf32(acc, a0 + 2 * k8, bl0 + 2 * k8, idesc, 1u);
                     }
                 } else {
 #pragma unroll 4
-                    for (int k8 = 0; k8 < k8n; ++k8) umma_tf32(acc, a0 + 2 * k8, b0 + 2 * k8, idesc, (k | k8) ? 1u : 0u);
+                    for (int k8 = 0; k8 < k8n; ++k8) umma_tf32(acc, a0 + 2 * k8, b0 + 2 * k8, idesc, ((k - kb) | k8) ? 1u : 0u);
                 }
                 umma_commit(empty0 + 8 * s);     // frees the stage once these MMAs have read it
                 if (++s == stages) { s = 0; par ^= 1u; }
@@ -559,7 +567,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                 px[j] = q0 + wi; py[j] = p0 + hi;
                 pn[j] = (j < per && ni < p.box_n && n0 + ni < p.N) ? n0 + ni : -1;
               }
-              for (int k = 0; k < total; ++k, ++it) {
+              for (int k = kb; k < ke; ++k, ++it) {
                 const int s = it % p.stages;
                 ok = mbar_wait(full0 + 8 * s, (it / p.stages) & 1, &abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
@@ -605,7 +613,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             }
         } else if (p.passes == 3) {
             const int per = (int)(p.a_bytes >> 12);     // float4 per thread: a_bytes / 16 / 256 = 2 or 4
-            const int all = my_tiles * total;
+            const int all = my_tiles * (ke - kb);
             for (int it = 0; it < all; ++it) {
                 const int s = it % p.stages;
                 ok = mbar_wait(full0 + 8 * s, (it / p.stages) & 1, &abort_flag);
@@ -684,6 +692,42 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             if (tid == 0 && tj == 0) HPF_TL(10);
             asm volatile("bar.sync 1, 256;" ::: "memory");
             if (tid == 0 && tj == 0) HPF_TL(11);
+            bool write_out = true;
+            if (KSPLIT) {
+                // split K: the staged tile is this CTA's partial sum.  Store it; the CTA that takes the last ticket of this
+                // (tile, channel slice) adds all partial tiles in split order (so the sum does not depend on which CTA that
+                // is) and goes on to the write-out; the others are done.
+                __shared__ int last_of_unit;
+                const int c4n_ = p.n_chunk >> 2, tile_f4 = kTileM * c4n_;
+                const unsigned int unit = blockIdx.x * gridDim.y + blockIdx.y;
+                float4* mine = reinterpret_cast<float4*>(p.splitk_partials) + ((size_t)unit * p.ksplit + blockIdx.z) * tile_f4;
+                for (int idx = tid; idx < tile_f4; idx += 256) {
+                    const int r = idx / c4n_, c4 = idx - r * c4n_;
+                    mine[idx] = *reinterpret_cast<const float4*>(stg + (size_t)r * p.stg_pitch + 4 * c4);
+                }
+                __threadfence();
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (tid == 0) last_of_unit = atomicAdd(p.splitk_ticket + unit, 1u) == (unsigned int)p.ksplit - 1u;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                write_out = last_of_unit != 0;
+                if (write_out) {
+                    __threadfence();
+                    const float4* all = reinterpret_cast<const float4*>(p.splitk_partials) + (size_t)unit * p.ksplit * tile_f4;
+                    for (int idx = tid; idx < tile_f4; idx += 256) {
+                        float4 a4 = __ldcg(all + idx);
+                        for (int z = 1; z < p.ksplit; ++z) {
+                            const float4 b4 = __ldcg(all + (size_t)z * tile_f4 + idx);
+                            a4.x += b4.x; a4.y += b4.y; a4.z += b4.z; a4.w += b4.w;
+                        }
+                        const int r = idx / c4n_, c4 = idx - r * c4n_;
+                        *reinterpret_cast<float4*>(stg + (size_t)r * p.stg_pitch + 4 * c4) = a4;
+                    }
+                    if (tid == 0) p.splitk_ticket[unit] = 0u;
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                }
+            }
+            float4 sa = make_float4(0.f, 0.f, 0.f, 0.f), sb = sa;
+            if (write_out) {
             // write-out: consecutive threads write consecutive float4 of a pixel's channel row.  Eight warps cannot
             // hide latency by occupancy, so four independent float4 are in flight per thread and nothing is re-read.
             const int c4n = p.n_chunk >> 2;
@@ -695,7 +739,6 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             const unsigned int pitch = p.stg_pitch;
             const long long dense_h = p.dense_h, dense_w = p.dense_w;
             const int stat_mode = p.stat_mode;
-            float4 sa = make_float4(0.f, 0.f, 0.f, 0.f), sb = sa;
             for (int base = tid; base < total4; base += 1024) {
                 float4 o[4];
                 int off[4];
@@ -744,7 +787,10 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     }
                 }
             }
-            if (stat_mode) {
+            }   // write_out
+            if (p.stat_mode) {
+                const int c4n = p.n_chunk >> 2;
+                const int stat_mode = p.stat_mode;
                 // a thread kept one group of 4 channels throughout (256 is a multiple of c4n): add the 256 / c4n
                 // threads of each group in ascending order and store this tile's partial sums
                 asm volatile("bar.sync 1, 256;" ::: "memory");          // the staging area is free again
@@ -1379,10 +1425,55 @@ cudaError_t conv_tc_init()
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(conv_tc_fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(conv_tc_fwd_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
+    if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(conv_tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWgradSmemBudget + 2048);
     if (e != cudaSuccess) return e;
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
     return cudaSuccess;
+}
+
+namespace {
+
+// How many CTAs share one tile's K loop.  Launches of a few tiles whose K loop is long (512-channel 3x3 convolutions on 7x7 or
+// 2x2 maps, fully connected layers) are bound by one CTA's MMA issue (about 0.1 us per K step of 8): splitting the loop
+// shortens it, at the price of one partial tile per split kept in L2.
+int splitk_factor(int tiles, int slices, int total_iters, int k8n)
+{
+    const int ctas = tiles * slices;
+    if (ctas > 32) return 1;                     // more CTAs than that already spread over the GPU; splitting them cost more than it gave
+    const int ksteps = total_iters * k8n;
+    if (ksteps < 128) return 1;
+    int S = 296 / ctas;
+    if (S > 8) S = 8;
+    if (S > ksteps / 32) S = ksteps / 32;        // at least 32 K steps per CTA
+    if (S > total_iters) S = total_iters;
+    return S < 2 ? 1 : S;
+}
+
+// Channel slice width of an unfused forward / data-gradient launch (see conv_tc_prepare).
+int unfused_n_chunk(int c_out, int tiles)
+{
+    int n_chunk = c_out < 256 ? c_out : 256;
+    if (c_out % 256 == 0 && tiles * (c_out / 256) <= 74) n_chunk = 128;
+    return n_chunk;
+}
+
+}  // namespace
+
+size_t conv_tc_splitk_bytes(const ConvShape& s, int pass, int passes)
+{
+    FwdView v;
+    PixelBox b;
+    if (pass == PASS_WGRAD || !fwd_view(s, pass, &v) || !choose_box(v.Q, v.P, v.N, kTileM, 1, &b)) return 0;
+    (void)passes;
+    const int tiles = ((v.Q + b.w - 1) / b.w) * ((v.P + b.h - 1) / b.h) * ((v.N + b.n - 1) / b.n);
+    const int n_chunk = unfused_n_chunk(v.c_out, tiles);
+    if (v.c_out % n_chunk) return 0;
+    const int kchunk = chunk_of(v.c_in);
+    const int S = splitk_factor(tiles, v.c_out / n_chunk, v.R * v.R * (v.c_in / kchunk), kchunk / 8);
+    if (S < 2) return 0;
+    return kSplitKTicketBytes + (size_t)tiles * (v.c_out / n_chunk) * S * kTileM * n_chunk * sizeof(float);
 }
 
 size_t conv_tc_scratch_bytes(const ConvShape& s)
@@ -1547,9 +1638,21 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
         while (t > 2 && (unsigned int)t * p.acc_cols > 256u) --t;
         p.tiles_per_cta = t < 2 ? 2 : t;
     }
+    p.ksplit = 1;
+    if (fuse && fuse->splitk && !fuse->mode && !fuse->in_mode && p.tiles_per_cta == 1) {
+        const int S = splitk_factor(p.n_tiles, v.c_out / n_chunk, total, kchunk / 8);
+        const size_t need = kSplitKTicketBytes + (size_t)p.n_tiles * (v.c_out / n_chunk) * S * kTileM * n_chunk * sizeof(float);
+        if (S > 1 && need <= fuse->splitk_bytes) {
+            p.ksplit = S;
+            p.splitk_ticket = reinterpret_cast<unsigned int*>(fuse->splitk);
+            p.splitk_partials = reinterpret_cast<float*>(reinterpret_cast<char*>(fuse->splitk) + kSplitKTicketBytes);
+            const int per_cta = total / S;                   // the shortest share of the K loop
+            if (p.stages > per_cta) p.stages = per_cta < 1 ? 1 : per_cta;
+        }
+    }
     p.tmem_cols = pow2_cols((int)p.acc_cols * p.tiles_per_cta);
     p.stg_off = p.tiles_per_cta > 1 ? pipe_bytes : 0u;
-    L->grid = dim3((p.n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta, v.c_out / n_chunk, 1);
+    L->grid = dim3((p.n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta, v.c_out / n_chunk, p.ksplit);
     L->smem = p.tiles_per_cta > 1 ? pipe_bytes + stg_bytes : (pipe_bytes > stg_bytes ? pipe_bytes : stg_bytes);
     L->smem += 1024;
     plan->valid = 1;
@@ -1573,7 +1676,8 @@ cudaError_t conv_tc_launch(const ConvTcPlan* plan, DeviceStatus* status, cudaStr
     }
     ConvTcFwdLaunch L = *reinterpret_cast<const ConvTcFwdLaunch*>(plan->storage);
     L.p.s.status = status;
-    if (L.p.s.tiles_per_cta > 1) launch_pdl(conv_tc_fwd_kernel<true>, L.grid, dim3(320), L.smem, st, L.p);
+    if (L.p.s.ksplit > 1) launch_pdl(conv_tc_fwd_kernel<false, true>, L.grid, dim3(320), L.smem, st, L.p);
+    else if (L.p.s.tiles_per_cta > 1) launch_pdl(conv_tc_fwd_kernel<true>, L.grid, dim3(320), L.smem, st, L.p);
     else launch_pdl(conv_tc_fwd_kernel<false>, L.grid, dim3(320), L.smem, st, L.p);
     count(n_launch, 1);
     return cudaGetLastError();

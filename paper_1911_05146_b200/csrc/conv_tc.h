@@ -54,7 +54,14 @@ struct ConvBnFuse {
     int in_tiles = 0;
     long long in_rows = 0;
     float in_eps = 0.f;
+    // forward / data gradient without BN work: room for splitting a long K loop over several CTAs (conv_tc_splitk_bytes;
+    // the first kSplitKTicketBytes hold tickets, zero before the first use and left zero).  nullptr: never split.
+    void* splitk = nullptr;
+    size_t splitk_bytes = 0;
 };
+constexpr size_t kSplitKTicketBytes = 4096;
+// Bytes a forward (or data-gradient) launch of this shape wants for splitting its K loop; 0 when it would not split.
+size_t conv_tc_splitk_bytes(const ConvShape& s, int pass, int passes);
 // Whether the input-side fusion applies to this convolution.
 bool conv_tc_can_fuse_bn_input(const ConvShape& s);
 // Number of pixel tiles (= partial-sum rows) of the forward / data-gradient launch, and whether the fusion applies.

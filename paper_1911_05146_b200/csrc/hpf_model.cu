@@ -101,6 +101,7 @@ struct hpf_model {
     // memory plan (byte offsets into the workspace)
     std::vector<size_t> act_off, grad_off, stats_off;   // [m * n_ops + op]
     std::vector<size_t> bn_scratch_off, conv_scratch_off;   // per stream
+    std::vector<size_t> splitk_off, splitk_bytes;            // per stream: tickets + partial tiles of K-split convolutions (zeroed at bind)
     std::vector<size_t> pooled_off, persample_off;      // per m
     std::vector<std::vector<size_t>> fmsg_off, bmsg_off;  // [cut][i*M + m]
     size_t loss_slots_off = 0, loss_avg_off = 0, wprep_off = 0, stage_x_off = 0, stage_lab_off = 0, status_off = 0;
@@ -439,6 +440,18 @@ void build_memory_plan(hpf_model* mdl)
         mdl->bn_part_bytes[p] = part;
         if (256 + 2 * part > bn) bn = 256 + 2 * part;
         mdl->bn_scratch_off[p] = take(bn);
+    }
+    mdl->splitk_off.assign(P, 0); mdl->splitk_bytes.assign(P, 0);
+    for (int p = 0; p < P; ++p) {
+        size_t need = 0;
+        if (mdl->opt_conv_path != 1)
+            for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i)
+                if (mdl->ops[i].op.kind == HPF_OP_CONV) {
+                    const ConvShape s = conv_shape_of(mdl, i);
+                    need = std::max(need, std::max(conv_tc_splitk_bytes(s, PASS_FWD, 3), conv_tc_splitk_bytes(s, PASS_DGRAD, 3)));
+                }
+        mdl->splitk_bytes[p] = need;
+        mdl->splitk_off[p] = take(need ? need : 16);
     }
     mdl->zero_hi = at;
     for (int p = 0; p < P; ++p) {
@@ -1076,6 +1089,7 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                             residual = mdl->act(a.src0 == i ? a.src1 : a.src0, m);
                         }
                         ConvBnFuse fuse;
+                        if (mdl->splitk_bytes[o.part]) { fuse.splitk = mdl->ws + mdl->splitk_off[o.part]; fuse.splitk_bytes = mdl->splitk_bytes[o.part]; }
                         if (mdl->conv_fwd_bn[i] >= 0) {
                             const int jn = mdl->conv_fwd_bn[i];
                             const OpInfo& bn = mdl->ops[jn];
@@ -1103,8 +1117,11 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                                            mdl->act(i, m), residual, false, scratch, &fuse));
                     }
                     else if (pass == PASS_DGRAD) {
+                        ConvBnFuse dsplit;
+                        if (mdl->splitk_bytes[o.part]) { dsplit.splitk = mdl->ws + mdl->splitk_off[o.part]; dsplit.splitk_bytes = mdl->splitk_bytes[o.part]; }
                         CU(conv_tc_prepare(pl, s, pass, passes, mdl->grad(i, m), nullptr, wp + 2 * G + o.w_off, wp + 3 * G + o.w_off,
-                                           mdl->grad(src, m), ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch));
+                                           mdl->grad(src, m), ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch,
+                                           &dsplit));
                     }
                     else {
                         // Weight gradients run on the side streams, beside the stages' chains of dependent kernels and feeding

@@ -142,6 +142,13 @@ def test_imagenet_layout_wide_channels():
     check_step(ops, (32, 32, 3), 4, 2, [9, 20], seed=3, bn_jitter=0.2)
 
 
+def test_long_k_loops_split_over_ctas():
+    """A 3x3 convolution on 512 channels over a 4x4 map: one pixel tile, 576 K steps, no BN fusion beyond 256 channels, so
+    the forward and the data gradient split their K loop over several CTAs (partial tiles, ticket, ordered sum)."""
+    ops = wl.resnet_v2_imagenet(blocks=(1, 1), widths=(64, 512), n_classes=9)
+    check_step(ops, (32, 32, 3), 4, 2, [11], seed=13, bn_jitter=0.2)
+
+
 def test_many_class_head_on_ragged_sizes():
     """The head kernels for many classes (one warp per class, 64-channel x 8-sample blocks in the backward): 350 classes on
     96 channels with micro-batches of 3 samples, so that no block or warp loop is full."""
