@@ -208,10 +208,11 @@ int hpf_conv_path_counts(const hpf_model *model, int64_t *n_tensor, int64_t *n_c
  * All pointers are device pointers, `stream` is a cudaStream_t.  x [N][H][W][C], w [K][R][R][C],
  * y/dy [N][P][Q][K] with P = (H+2*pad-R)/stride+1.  path: 0 = tensor cores, three-pass TF32;
  * 2 = tensor cores, one TF32 pass (both HPF_ERR_UNSUPPORTED when the shape is outside their reach);
- * 1 = CUDA cores.  d_scratch: caller-owned scratch of at least hpf_conv_scratch_bytes().  Its last 256 bytes are the
- * device status of the tensor-core kernels: the caller zeroes them once (e.g. allocates the scratch zeroed); a kernel
- * whose bounded wait gives up stores a non-zero code there (first failure wins) and nothing ever clears it.  The rest
- * is written by the call and holds nothing afterwards.
+ * 1 = CUDA cores.  d_scratch: caller-owned scratch of at least hpf_conv_scratch_bytes(), zeroed ONCE by the caller (e.g.
+ * allocated zeroed) and used by one stream at a time.  Its last 256 bytes are the device status of the tensor-core
+ * kernels: a kernel whose bounded wait gives up stores a non-zero code there (first failure wins) and nothing ever
+ * clears it.  Launches that split a long K loop over several CTAs keep their tickets in it and leave them at zero.
+ * Everything else is written by the call and holds nothing afterwards.
  * d_wprep: the weights as the tensor-core kernels read them, 4*K*R*R*C floats written by
  * hpf_conv_prepare_weights ([hi | lo | rearranged-for-dgrad hi | lo]); ignored (may be NULL) for path 1
  * and by hpf_conv_wgrad. */

@@ -1312,7 +1312,8 @@ int hpf_conv_scratch_bytes(int32_t N, int32_t H, int32_t W, int32_t C, int32_t K
     if (rc) return rc;
     const ConvShape s = make_conv_shape(N, H, W, C, K, R, stride, pad);
     size_t a = conv_simt_scratch_bytes(s), b = conv_tc_scratch_bytes(s);
-    *bytes = align_up((a > b ? a : b) + 256, 256);
+    // [weight-gradient partials | K-split tickets and partial tiles | device status (256 bytes)]
+    *bytes = align_up(a > b ? a : b, 256) + align_up(std::max(conv_tc_splitk_bytes(s, PASS_FWD, 3), conv_tc_splitk_bytes(s, PASS_DGRAD, 3)), 256) + 256;
     return HPF_OK;
 }
 
@@ -1344,7 +1345,13 @@ static int conv_single(int pass, const float* in, const float* in2, const float*
     DeviceStatus* status = reinterpret_cast<DeviceStatus*>(reinterpret_cast<char*>(d_scratch) + sb - 256);
     const int64_t nw = (int64_t)K * R * R * C;
     const float* hi = wprep ? wprep + (pass == PASS_DGRAD ? 2 * nw : 0) : nullptr;
-    CU(conv_tc_prepare(&plan, s, pass, path == 2 ? 1 : 3, in, in2, hi, hi ? hi + nw : nullptr, out, nullptr, false, d_scratch));
+    ConvBnFuse split;
+    if (pass != PASS_WGRAD) {
+        const size_t a = conv_simt_scratch_bytes(s), b = conv_tc_scratch_bytes(s);
+        split.splitk_bytes = conv_tc_splitk_bytes(s, pass, 3);
+        if (split.splitk_bytes) split.splitk = reinterpret_cast<char*>(d_scratch) + align_up(a > b ? a : b, 256);
+    }
+    CU(conv_tc_prepare(&plan, s, pass, path == 2 ? 1 : 3, in, in2, hi, hi ? hi + nw : nullptr, out, nullptr, false, d_scratch, &split));
     CU(conv_tc_launch(&plan, status, st, nullptr));
     return HPF_OK;
 }
