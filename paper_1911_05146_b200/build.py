@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhpf.so")
-SOURCES = ["hpf_model.cu", "kernels_mem.cu", "conv_simt.cu", "conv_tc.cu", "no_alloc.cu"]
+SOURCES = ["hpf_model.cu", "kernels_mem.cu", "conv_simt.cu", "conv_tc.cu", "no_alloc.cu", "bn_resident.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--use_fast_math=false"]
 

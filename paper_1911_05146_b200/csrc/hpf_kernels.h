@@ -67,6 +67,14 @@ cudaError_t bnrelu_bwd(const float* x, const float* dy, const float* gamma, cons
                        bool x_is_old = false);
 // x_is_old: x, stats, gamma and beta were complete before the kernels just ahead of this call in the stream were
 // enqueued (forward results read by a backward pass), so the kernel may fetch them while its predecessor still runs.
+// The forward from an on-chip copy of the tensor (bn_resident.cu): one cooperative launch that holds every SM, for
+// single-op calls on tensors of 8 MB and more that fit the chip.  cudaErrorNotSupported = not applicable, nothing
+// launched.  Same scratch convention; words 1 and 2 of the scratch are used besides the ticket.
+cudaError_t bnrelu_fwd_resident(const float* x, const float* gamma, const float* beta, float eps, float* y, float* stats,
+                                int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch, bool relu = true);
+cudaError_t bnrelu_bwd_resident(const float* x, const float* dy, const float* gamma, const float* beta, const float* stats,
+                                float* dx, const float* addend, bool accumulate, float* dgamma, float* dbeta, int64_t rows, int C,
+                                void* scratch, cudaStream_t st, int64_t* n_launch, bool relu = true);
 extern thread_local bool g_bn_cluster;   // single-launch cluster kernel for micro-batch sized BN backward (default on)
 struct BnClusterScope {
     bool saved;

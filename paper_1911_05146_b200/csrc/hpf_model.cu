@@ -1391,12 +1391,21 @@ int hpf_bnrelu_scratch_bytes(int64_t rows, int32_t C, size_t* bytes)
     return HPF_OK;
 }
 
+// HPF_BN_RESIDENT=0 in the environment keeps single-op BN calls on the two-kernel path (comparison runs).
+static const bool g_bn_resident = [] { const char* v = getenv("HPF_BN_RESIDENT"); return !v || atoi(v) != 0; }();
+
 int hpf_bnrelu_fwd(const float* d_x, const float* d_gamma, const float* d_beta, float eps, float* d_y, float* d_stats,
                    int64_t rows, int32_t C, void* d_scratch, void* stream)
 {
     if (!d_x || !d_gamma || !d_beta || !d_y || !d_stats || !d_scratch) return fail(HPF_ERR_INVALID, "null argument");
     if (rows < 1 || C < 4 || C % 4) return fail(HPF_ERR_UNSUPPORTED, "channel count must be a multiple of 4");
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    // a single-op call has the GPU to itself: tensors that fit the chip are read once and held between the two steps
+    const cudaError_t res = g_bn_resident ? bnrelu_fwd_resident(d_x, d_gamma, d_beta, eps, d_y, d_stats, rows, C, d_scratch, st, nullptr)
+                                          : cudaErrorNotSupported;
+    if (res == cudaSuccess) return HPF_OK;
+    if (res != cudaErrorNotSupported) CU(res);
+    (void)cudaGetLastError();
     CU(bnrelu_fwd(d_x, d_gamma, d_beta, eps, d_y, d_stats, rows, C, d_scratch, st, nullptr));
     return HPF_OK;
 }
@@ -1408,6 +1417,12 @@ int hpf_bnrelu_bwd(const float* d_x, const float* d_dy, const float* d_gamma, co
     if (!d_x || !d_dy || !d_gamma || !d_beta || !d_stats || !d_dx || !d_dgamma || !d_dbeta || !d_scratch) return fail(HPF_ERR_INVALID, "null argument");
     if (rows < 1 || C < 4 || C % 4) return fail(HPF_ERR_UNSUPPORTED, "channel count must be a multiple of 4");
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const cudaError_t res = g_bn_resident ? bnrelu_bwd_resident(d_x, d_dy, d_gamma, d_beta, d_stats, d_dx, d_addend, accumulate != 0,
+                                                                 d_dgamma, d_dbeta, rows, C, d_scratch, st, nullptr)
+                                          : cudaErrorNotSupported;
+    if (res == cudaSuccess) return HPF_OK;
+    if (res != cudaErrorNotSupported) CU(res);
+    (void)cudaGetLastError();
     CU(bnrelu_bwd(d_x, d_dy, d_gamma, d_beta, d_stats, d_dx, d_addend, accumulate != 0, d_dgamma, d_dbeta, rows, C, d_scratch, st, nullptr));
     return HPF_OK;
 }

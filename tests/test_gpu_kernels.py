@@ -105,7 +105,8 @@ def test_conv_bad_arguments():
 
 @pytest.mark.parametrize("rows,C", [(1, 4), (7, 12), (5, 16), (1000, 16), (4096 + 37, 64), (16384, 16), (16384, 64), (4096, 32),
                                     (4096, 128), (1024, 64), (1024, 256), (50, 2048), (131072, 16), (8192, 256), (65536 + 11, 64),
-                                    (3000, 2048), (40000, 96), (784, 2048), (200, 1024), (32768, 16), (999, 4)])
+                                    (3000, 2048), (40000, 96), (784, 2048), (200, 1024), (32768, 16), (999, 4),
+                                    (131072, 64), (60000 + 3, 128), (262144 + 5, 32), (16384 + 1, 512)])
 def test_bnrelu_fwd_bwd(rows, C):
     rng = np.random.Generator(np.random.PCG64(rows * 7 + C))
     x = (rng.standard_normal((rows, C)) * 2 + 3).astype(np.float32)       # mean >> 0: the cancellation case
