@@ -17,6 +17,14 @@ namespace hpf {
 
 namespace {
 
+// -DHPF_RES_TIMELINE: thread 0 of every CTA stamps the nanosecond timer at the phase boundaries of the forward kernel
+// into the scratch behind the partial rows (8 stamps per CTA), for latency studies.
+#ifdef HPF_RES_TIMELINE
+#define RES_STAMP(k) do { if (threadIdx.x == 0) tl[blockIdx.x * 8 + (k)] = res_timer(); } while (0)
+#else
+#define RES_STAMP(k) do { } while (0)
+#endif
+
 constexpr int kResThreads = 1024;
 constexpr int kResRegV = 6;                       // float4 per thread kept in registers
 constexpr int kResSmemV = 11;                     // float4 per thread kept in shared memory, at most
@@ -97,6 +105,9 @@ __device__ __forceinline__ float4 res_dx(const float4& dz, const float4& xh, con
 __device__ __forceinline__ bool res_exchange(float4 a, float4 b, int C4, unsigned int* sync, unsigned int gen0, float* partials,
                                              double* dred, double* dtot)
 {
+#ifdef HPF_RES_TIMELINE
+    unsigned long long* tl = reinterpret_cast<unsigned long long*>(partials + (size_t)gridDim.x * 8 * C4);
+#endif
     __shared__ int s_fail;
     float* red = reinterpret_cast<float*>(dred);
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
@@ -127,17 +138,19 @@ __device__ __forceinline__ bool res_exchange(float4 a, float4 b, int C4, unsigne
         __stcg(partials + (size_t)blockIdx.x * nval + t, s);
     }
 
-    // grid-wide barrier: the last CTA to arrive clears the count and advances the generation.  The CTA barrier orders
-    // the partial sums of all threads before thread 0's fence, which publishes them ahead of the arrival.
+    // grid-wide barrier.  The CTA barrier orders the partial sums of all threads before thread 0's fence, which publishes
+    // them ahead of the arrival.  The last CTA to arrive advances the generation at once and clears the count afterwards:
+    // nobody reads the count again before the next launch.
     __syncthreads();
+    RES_STAMP(6);
     if (t == 0) {
         int fail = 0;
         __threadfence();
         const unsigned int old = atomicAdd(sync, 1u);
         if (old == gridDim.x - 1) {
-            atomicExch(sync, 0u);
             __threadfence();
             atomicAdd(sync + 1, 1u);
+            atomicExch(sync, 0u);
         } else {
             const unsigned long long t0 = res_timer();
             unsigned int polls = 0;
@@ -145,31 +158,42 @@ __device__ __forceinline__ bool res_exchange(float4 a, float4 b, int C4, unsigne
                 if ((++polls & 1023u) == 0 && res_timer() - t0 > kResWaitNs) { atomicExch(sync + 2, 1u); fail = 1; break; }
             }
         }
-        __threadfence();
         s_fail = fail;
     }
     __syncthreads();
     if (s_fail) return false;
+    RES_STAMP(7);
 
-    // every CTA adds the partial rows itself, 128 bits per load so that a thread has only a few loads, all in flight
-    // together: G thread groups take the rows g, g + G, ... in ascending order (fp64), then the groups are added in
-    // ascending order
+    // every CTA adds the partial rows itself: G thread groups take the rows g, g + G, ... in ascending order (fp64), then
+    // the groups are added in ascending order.  A thread fetches its rows eight at a time, 128 bits each, all in flight
+    // together: a loop that waited for each load in turn would pay an L2 round trip per row.
     {
         const int nv4 = nval >> 2;                   // float4 per partial row, <= 256
-        const int G = kResThreads / nv4, g = t / nv4, v4 = t - g * nv4;
+        int G = kResThreads / nv4;
+        const int g_want = ((int)gridDim.x + 7) >> 3;
+        if (G > g_want) G = g_want;
+        const int g = t / nv4, v4 = t - g * nv4;
         double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-        const float4* prow = reinterpret_cast<const float4*>(partials) + v4;
-#pragma unroll 8
-        for (int bI = g; bI < (int)gridDim.x; bI += G) {
-            const float4 pv = __ldcg(prow + (size_t)bI * nv4);
-            s0 += (double)pv.x; s1 += (double)pv.y; s2 += (double)pv.z; s3 += (double)pv.w;
+        if (g < G) {
+            const float4* prow = reinterpret_cast<const float4*>(partials) + v4;
+            for (int b0 = g; b0 < (int)gridDim.x; b0 += 8 * G) {
+                float4 pv[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const int bI = b0 + k * G;
+                    pv[k] = bI < (int)gridDim.x ? __ldcg(prow + (size_t)bI * nv4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int k = 0; k < 8; ++k) { s0 += (double)pv[k].x; s1 += (double)pv[k].y; s2 += (double)pv[k].z; s3 += (double)pv[k].w; }
+            }
+            // group sums: [g][value], value = 4 * v4 + component
+            dred[g * nval + 4 * v4 + 0] = s0; dred[g * nval + 4 * v4 + 1] = s1;
+            dred[g * nval + 4 * v4 + 2] = s2; dred[g * nval + 4 * v4 + 3] = s3;
         }
-        // group sums: [g][value], value = 4 * v4 + component
-        dred[g * nval + 4 * v4 + 0] = s0; dred[g * nval + 4 * v4 + 1] = s1;
-        dred[g * nval + 4 * v4 + 2] = s2; dred[g * nval + 4 * v4 + 3] = s3;
         __syncthreads();
         if (t < nval) {
             double tot = 0.0;
+#pragma unroll 4
             for (int g2 = 0; g2 < G; ++g2) tot += dred[g2 * nval + t];
             dtot[t] = tot;
         }
@@ -202,6 +226,10 @@ bn_fwd_resident_kernel(const float4* __restrict__ x4, const float* __restrict__ 
 
     pdl_launch_dependents();
     pdl_wait();
+#ifdef HPF_RES_TIMELINE
+    unsigned long long* tl = reinterpret_cast<unsigned long long*>(partials + (size_t)gridDim.x * 8 * C4);
+#endif
+    RES_STAMP(0);
     unsigned int gen0 = 0;
     if (t == 0) gen0 = res_ld_acquire(sync + 1);
 
@@ -211,6 +239,7 @@ bn_fwd_resident_kernel(const float4* __restrict__ x4, const float* __restrict__ 
         if (i < cta_end) res_cp_async16(&held[(j - kResRegV) * kResThreads + t], x4 + i);
     }
     const float4 sh = __ldg(x4 + q);                 // shift = row 0 (shifted sums avoid cancellation)
+    const float shift_c = t < C ? __ldg(reinterpret_cast<const float*>(x4) + t) : 0.f;   // for the finalisation of channel t
     float4 r[kResRegV];
 #pragma unroll
     for (int j = 0; j < kResRegV; ++j) {
@@ -220,12 +249,15 @@ bn_fwd_resident_kernel(const float4* __restrict__ x4, const float* __restrict__ 
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
 #pragma unroll
     for (int j = 0; j < kResRegV; ++j) res_acc(a, b, r[j], sh);
+    RES_STAMP(1);
     res_cp_async_wait_all();
+    RES_STAMP(2);
     for (int j = kResRegV; j < iters; ++j) {
         const long long i = base + (long long)j * kResThreads;
         if (i < cta_end) res_acc(a, b, held[(j - kResRegV) * kResThreads + t], sh);
     }
 
+    RES_STAMP(3);
     if (!res_exchange(a, b, C4, sync, gen0, partials, dred, dtot)) {   // no sums: poison the statistics, store no output
         if (blockIdx.x == 0) for (int c = t; c < 2 * C; c += kResThreads) stats[c] = nanf("");
         return;
@@ -234,7 +266,7 @@ bn_fwd_resident_kernel(const float4* __restrict__ x4, const float* __restrict__ 
     if (t < C) {
         const int qq = t >> 2, k = t & 3;
         const double inv_rows = 1.0 / (double)rows;
-        const double shift = (double)__ldg(reinterpret_cast<const float*>(x4) + t);
+        const double shift = (double)shift_c;
         const double m1 = dtot[k * C4 + qq] * inv_rows;
         double var = dtot[(4 + k) * C4 + qq] * inv_rows - m1 * m1;
         if (var < 0.0) var = 0.0;
@@ -244,6 +276,7 @@ bn_fwd_resident_kernel(const float4* __restrict__ x4, const float* __restrict__ 
         if (blockIdx.x == 0) { stats[t] = mean; stats[C + t] = rstd; }
     }
     __syncthreads();
+    RES_STAMP(4);
     const float4 mu = reinterpret_cast<const float4*>(s_mean)[q];
     const float4 rs = reinterpret_cast<const float4*>(s_rstd)[q];
     const float4 gm = __ldg(reinterpret_cast<const float4*>(gamma) + q);
@@ -257,6 +290,7 @@ bn_fwd_resident_kernel(const float4* __restrict__ x4, const float* __restrict__ 
         const long long i = base + (long long)j * kResThreads;
         if (i < cta_end) __stcs(y4 + i, res_apply(held[(j - kResRegV) * kResThreads + t], mu, rs, gm, bt, floor));
     }
+    RES_STAMP(5);
 }
 
 // Backward: dz = dy * [z > floor]; a = sum dz (dbeta), b = sum dz * xhat (dgamma);
