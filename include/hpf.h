@@ -227,8 +227,14 @@ int hpf_conv_dgrad(const float *d_dy, const float *d_w, const float *d_wprep, fl
 int hpf_conv_wgrad(const float *d_x, const float *d_dy, float *d_dw, int32_t N, int32_t H, int32_t W, int32_t C,
                    int32_t K, int32_t R, int32_t stride, int32_t pad, int32_t path, void *d_scratch, void *stream);
 /* Fused BN(training)+ReLU over x [rows][C]: d_stats receives mean[C] then 1/sqrt(var+eps)[C].
- * d_scratch: at least hpf_bnrelu_scratch_bytes(rows, C); the caller zeroes its first 256 bytes once (a ticket the
- * kernels count on and leave at zero), the calls enqueue kernels only. */
+ * d_scratch: at least hpf_bnrelu_scratch_bytes(rows, C); the caller zeroes its first 256 bytes once (word 0 is a ticket
+ * the kernels count on and leave at zero), the calls enqueue kernels only.
+ * Tensors of 16 MB and more that fit the registers and shared memory of the whole GPU (16...512 channels, a power of two)
+ * are processed by ONE cooperative launch that keeps the tensor on chip between the statistics and the apply step; it
+ * occupies every SM while it runs.  That launch synchronises its CTAs through words 0-1 of the scratch; the wait is
+ * bounded (2 s): if it ever gives up, word 2 of the scratch becomes 1, d_stats (forward) or d_dgamma / d_dbeta
+ * (backward) are NaN and the output is not written.  HPF_BN_RESIDENT=0 in the environment keeps all sizes on the
+ * two-kernel path. */
 int hpf_bnrelu_scratch_bytes(int64_t rows, int32_t C, size_t *bytes);
 int hpf_bnrelu_fwd(const float *d_x, const float *d_gamma, const float *d_beta, float eps, float *d_y,
                    float *d_stats, int64_t rows, int32_t C, void *d_scratch, void *stream);
@@ -250,7 +256,7 @@ int hpf_bnrelu_bwd(const float *d_x, const float *d_dy, const float *d_gamma, co
  *   - All calls on a device share the one array, which keeps the previous call's contents; the call
  *     clears the part that must start at zero.  Two calls whose kernels overlap on the GPU (different
  *     streams, no ordering between them) race on it: order them.
- * Inputs and outputs are the caller's, exactly as for hpf_bnrelu_fwd; results are identical to it. */
+ * Inputs and outputs are the caller's, exactly as for hpf_bnrelu_fwd; results are those of its two-kernel path. */
 int hpf_bnrelu_fwd_static(const float *d_x, const float *d_gamma, const float *d_beta, float eps, float *d_y,
                           float *d_stats, int64_t rows, int32_t C, void *stream);
 int hpf_static_scratch_bytes(size_t *bytes);
