@@ -152,6 +152,7 @@ wgrad_reduce_kernel(const float* __restrict__ partials, float* __restrict__ dw, 
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
         float s = 0.f;
+#pragma unroll 8
         for (int z = 0; z < splits; ++z) s += __ldcg(&partials[(int64_t)z * n + i]);
         dw[i] = s;
     }
@@ -165,7 +166,7 @@ WgradSplit wgrad_split(const ConvShape& s)
     int64_t splits = pixels / 1024;                       // >= 1024 pixels per slice
     const int64_t cap = (int64_t)(32 << 20) / (outs * 4) ;  // partials <= 32 MiB
     if (splits > cap) splits = cap;
-    if (splits > 64) splits = 64;
+    if (splits > 256) splits = 256;                       // few output tiles (the 7x7 stem: 3): the slices are what fills the GPU
     if (splits < 1) splits = 1;
     int64_t kps = (pixels + splits - 1) / splits;
     kps = (kps + BK - 1) / BK * BK;
