@@ -427,6 +427,19 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
     }
 
     if (threadIdx.x == 0) HPF_TL(0);
+    const int total = p.R * p.R * p.n_kchunks;
+    // this CTA's share of the K loop (all of it unless the launch splits K over gridDim.z)
+    const int kb = KSPLIT ? (int)(((long long)total * blockIdx.z) / p.ksplit) : 0;
+    const int ke = KSPLIT ? (int)(((long long)total * (blockIdx.z + 1)) / p.ksplit) : total;
+    // Thread 0 is the TMA producer.  The origin of its first tile and its first K step are a chain of dependent
+    // shared-memory reads and integer divisions in ONE thread (most of a microsecond): worked out here, while the CTA
+    // still waits for tensor memory and for the preceding kernel, not between that wait and the first copy.
+    int f_q0 = 0, f_p0 = 0, f_n0 = 0, f_tap = 0, f_kc = 0, f_r = 0, f_sx = 0;
+    if (threadIdx.x == 0) {
+        HPF_TILE_ORIGIN(tile0);
+        f_q0 = q0; f_p0 = p0; f_n0 = n0;
+        if (KSPLIT) { f_tap = kb / p.n_kchunks; f_kc = kb % p.n_kchunks; f_r = f_tap / p.R; f_sx = f_tap % p.R; }
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); mbar_init(split0 + 8 * s, 8); }
         for (int j = 0; j < 4; ++j) mbar_init(accum_bar + 8 * j, 1);
@@ -438,34 +451,45 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    pdl_wait();              // everything above touched only parameters, shared and tensor memory
+    // Everything above touched only parameters, shared and tensor memory.  The TMA producer (thread 0) first works out
+    // its first tile's coordinates - a chain of dependent shared-memory reads and integer divisions of most of a
+    // microsecond - and waits for the preceding kernel only then, right before its first copy.
+    if (threadIdx.x != 0) pdl_wait();
     const uint32_t tmem_base = tmem_slot;
-    const int total = p.R * p.R * p.n_kchunks;
-    // this CTA's share of the K loop (all of it unless the launch splits K over gridDim.z)
-    const int kb = KSPLIT ? (int)(((long long)total * blockIdx.z) / p.ksplit) : 0;
-    const int ke = KSPLIT ? (int)(((long long)total * (blockIdx.z + 1)) / p.ksplit) : total;
-    if (threadIdx.x == 0) HPF_TL(1);
 
     if (warp == 0) {
         if (lane == 0) {
             // ---- TMA producer ----
-            int it = 0;
+            // no division in the loop: stage, parity, tap and K chunk are counters
+            int it = 0, st = 0;
+            uint32_t par = 1u;
             bool live = true;
+            const int stages = p.stages, nkc = p.n_kchunks, R = p.R, pad = p.pad, kchunk = p.kchunk, c_in = p.c_in;
+            const uint32_t tx = p.tx_bytes, stage_bytes = p.stage_bytes;
+            const bool three = p.passes == 3;
             for (int j = 0; j < my_tiles && live; ++j) {
-                HPF_TILE_ORIGIN(tile0 + j);
+                int q0 = f_q0, p0 = f_p0, n0 = f_n0;
+                if (j > 0) {
+                    int t__ = tile0 + j;
+                    const int tw__ = t__ % p.tiles_w; t__ /= p.tiles_w;
+                    q0 = tw__ * p.box_w; p0 = (t__ % p.tiles_h) * p.box_h; n0 = (t__ / p.tiles_h) * p.box_n;
+                }
+                int tap = f_tap, kc = f_kc, r = f_r, sx = f_sx;
                 for (int k = kb; k < ke; ++k, ++it) {
-                    const int s = it % p.stages;
-                    if (!mbar_wait(empty0 + 8 * s, ((it / p.stages) & 1) ^ 1, &abort_flag)) { report(p.status, 1); live = false; break; }
-                    const int tap = k / p.n_kchunks, kc = k % p.n_kchunks;
-                    const int r = tap / p.R, sx = tap % p.R;
-                    const uint32_t dst = smem_base + s * p.stage_bytes;
-                    mbar_expect_tx(full0 + 8 * s, p.tx_bytes);
-                    tma_load_4d(dst, &gp.tm_a, full0 + 8 * s, kc * p.kchunk, q0 + sx - p.pad, p0 + r - p.pad, n0);
-                    tma_load_2d(dst + off_b, &gp.tm_b, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
-                    if (p.passes == 3) tma_load_2d(dst + off_blo, &gp.tm_b_lo, full0 + 8 * s, tap * p.c_in + kc * p.kchunk, co0);
+                    if (!mbar_wait(empty0 + 8 * st, par, &abort_flag)) { report(p.status, 1); live = false; break; }
+                    const uint32_t dst = smem_base + st * stage_bytes;
+                    const int cx = kc * kchunk, cq = q0 + sx - pad, cp = p0 + r - pad, cb = tap * c_in + cx;
+                    if (it == 0) { pdl_wait(); HPF_TL(1); }
+                    mbar_expect_tx(full0 + 8 * st, tx);
+                    tma_load_4d(dst, &gp.tm_a, full0 + 8 * st, cx, cq, cp, n0);
+                    tma_load_2d(dst + off_b, &gp.tm_b, full0 + 8 * st, cb, co0);
+                    if (three) tma_load_2d(dst + off_blo, &gp.tm_b_lo, full0 + 8 * st, cb, co0);
                     if (it == 0) HPF_TL(2);
+                    if (++kc == nkc) { kc = 0; ++tap; if (++sx == R) { sx = 0; ++r; } }
+                    if (++st == stages) { st = 0; par ^= 1u; }
                 }
             }
+            if (it == 0) pdl_wait();         // nothing to copy: still ordered behind the preceding kernel
             issued = it;
         }
     } else if (warp == 1) {
@@ -542,11 +566,14 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     bn_par[0][tid] = mu; bn_par[1][tid] = rs; bn_par[2][tid] = gam; bn_par[3][tid] = bet;
                     if (blockIdx.x == 0 && blockIdx.y == 0) { p.bn_in_stats_out[tid] = mu; p.bn_in_stats_out[C + tid] = rs; }
                 }
-            } else if (tid < C) {
-                bn_par[0][tid] = __ldcg(p.bn_in_stats + tid); bn_par[1][tid] = __ldcg(p.bn_in_stats + C + tid);   // written by the kernel before: not the read-only path
-                bn_par[2][tid] = __ldg(p.bn_in_gamma + tid); bn_par[3][tid] = __ldg(p.bn_in_beta + tid);
             }
-            asm volatile("bar.sync 1, 256;" ::: "memory");
+            // the statistics written by the kernel before (not the read-only path) and the parameters: fetched now, used
+            // after the index arithmetic below, which runs under their latency
+            float ld_mu = 0.f, ld_rs = 0.f, ld_g = 0.f, ld_b = 0.f;
+            if (p.bn_in != 2 && tid < C) {
+                ld_mu = __ldcg(p.bn_in_stats + tid); ld_rs = __ldcg(p.bn_in_stats + C + tid);
+                ld_g = __ldg(p.bn_in_gamma + tid); ld_b = __ldg(p.bn_in_beta + tid);
+            }
             // A thread owns one 16-byte column of the (swizzled) tile rows tid/f4row + j*(256/f4row): its four
             // channels within the K chunk are fixed, and so are the pixels of its rows.
             const int f4row = p.kchunk >> 2;                    // 4 or 8 float4 per tile row
@@ -556,25 +583,34 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             const int clog = p.kchunk == 32 ? (cph ^ (row0 & 7)) : (cph ^ ((row0 >> 1) & 3));
             const bool three = p.passes == 3;
             const bool writer = blockIdx.y == 0;
-            int it = 0;
+            const int stages = p.stages, nkc = p.n_kchunks, R = p.R, pad = p.pad;
+            // position of row r of the pixel box (the same for every tile)
+            int rw[4], rh[4], rn[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int r = row0 + j * rstep;
+                rw[j] = r % p.box_w; rh[j] = (r / p.box_w) % p.box_h; rn[j] = r / (p.box_w * p.box_h);
+            }
+            const int tap_b = kb / nkc, kc_b = kb - tap_b * nkc, ry_b = tap_b / R, sx_b = tap_b - ry_b * R;
+            if (p.bn_in != 2 && tid < C) { bn_par[0][tid] = ld_mu; bn_par[1][tid] = ld_rs; bn_par[2][tid] = ld_g; bn_par[3][tid] = ld_b; }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            int it = 0, s = 0;
+            uint32_t par = 0;
             for (int tj = 0; tj < my_tiles && ok; ++tj) {
               HPF_TILE_ORIGIN(tile0 + tj);
               int px[4], py[4], pn[4];
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
-                const int r = row0 + j * rstep;
-                const int wi = r % p.box_w, hi = (r / p.box_w) % p.box_h, ni = r / (p.box_w * p.box_h);
-                px[j] = q0 + wi; py[j] = p0 + hi;
-                pn[j] = (j < per && ni < p.box_n && n0 + ni < p.N) ? n0 + ni : -1;
+                px[j] = q0 + rw[j]; py[j] = p0 + rh[j];
+                pn[j] = (j < per && rn[j] < p.box_n && n0 + rn[j] < p.N) ? n0 + rn[j] : -1;
               }
+              int kc = kc_b, ry = ry_b, sx = sx_b;
               for (int k = kb; k < ke; ++k, ++it) {
-                const int s = it % p.stages;
-                ok = mbar_wait(full0 + 8 * s, (it / p.stages) & 1, &abort_flag);
+                ok = mbar_wait(full0 + 8 * s, par, &abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) { if (lane == 0) report(p.status, 7); break; }
                 if (it == 0 && tid == 0) HPF_TL(3);
-                const int tap = k / p.n_kchunks, kc = k - tap * p.n_kchunks;
-                const int dyy = tap / p.R - p.pad, dxx = tap % p.R - p.pad;
+                const int dyy = ry - pad, dxx = sx - pad;
                 const int ch = kc * p.kchunk + 4 * clog;
                 const float4 mu = *reinterpret_cast<const float4*>(&bn_par[0][ch]);
                 const float4 rs = *reinterpret_cast<const float4*>(&bn_par[1][ch]);
@@ -609,14 +645,18 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                 __syncwarp();
                 if (lane == 0) mbar_arrive(split0 + 8 * s);
                 if (it == 0 && tid == 0) HPF_TL(4);
+                if (++kc == nkc) { kc = 0; if (++sx == R) { sx = 0; ++ry; } }
+                if (++s == stages) { s = 0; par ^= 1u; }
               }
             }
         } else if (p.passes == 3) {
             const int per = (int)(p.a_bytes >> 12);     // float4 per thread: a_bytes / 16 / 256 = 2 or 4
             const int all = my_tiles * (ke - kb);
+            const int stages = p.stages;
+            int s = 0;
+            uint32_t par = 0;
             for (int it = 0; it < all; ++it) {
-                const int s = it % p.stages;
-                ok = mbar_wait(full0 + 8 * s, (it / p.stages) & 1, &abort_flag);
+                ok = mbar_wait(full0 + 8 * s, par, &abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) { if (lane == 0) report(p.status, 7); break; }
                 if (it == 0 && tid == 0) HPF_TL(3);
@@ -636,6 +676,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                 __syncwarp();
                 if (lane == 0) mbar_arrive(split0 + 8 * s);
                 if (it == 0 && tid == 0) HPF_TL(4);
+                if (++s == stages) { s = 0; par ^= 1u; }
             }
         }
         (void)ok;
