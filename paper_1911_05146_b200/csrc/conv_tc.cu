@@ -329,10 +329,17 @@ __device__ __forceinline__ void bn_combine_partials(const float* partials, int n
     const int col4 = tid % ncol4, ln = tid / ncol4, L = 256 / ncol4;
     const float4* part = reinterpret_cast<const float4*>(partials);
     double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-#pragma unroll 8
-    for (int k = ln; k < n_tiles; k += L) {
-        const float4 v = __ldcg(part + (size_t)k * ncol4 + col4);
-        a0 += (double)v.x; a1 += (double)v.y; a2 += (double)v.z; a3 += (double)v.w;
+    // eight rows per batch, all eight loads in flight together (a loop that used each load before issuing the next would
+    // pay an L2 round trip per row); rows beyond the last add zero
+    for (int k0 = ln; k0 < n_tiles; k0 += 8 * L) {
+        float4 v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int k = k0 + j * L;
+            v[j] = k < n_tiles ? __ldcg(part + (size_t)k * ncol4 + col4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { a0 += (double)v[j].x; a1 += (double)v[j].y; a2 += (double)v[j].z; a3 += (double)v[j].w; }
     }
     if (ncol4 <= 16) {
         // several lanes of a column sit in one warp: a fixed butterfly first, then the eight warps in ascending order
