@@ -1030,33 +1030,40 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
     if (warp == 0) {
         if (lane == 0) {
             // ---- TMA producer ----
-            int it = 0;
+            // no division in the loop: the stage, its parity, the tile's position and the taps' offsets are counters
+            const int raw_stages = p.raw_stages, tiles_w = p.tiles_w, tiles_h = p.tiles_h, R = p.R, pad = p.pad;
+            const int box_w = p.box_w, box_h = p.box_h, box_n = p.box_n;
+            const uint32_t raw_bytes = p.raw_bytes, tx = p.tx_a + (uint32_t)ntaps * p.tx_per_tap;
+            int tw, th, tn;
+            { int t = tile_begin; tw = t % tiles_w; t /= tiles_w; th = t % tiles_h; tn = t / tiles_h; }
+            const int r_first = tap0 / R, sx_first = tap0 - r_first * R;
+            int it = 0, s = 0;
+            uint32_t par = 1u;
             for (; it < total; ++it) {
-                const int s = it % p.raw_stages;
-                if (!mbar_wait(empty_raw0 + 8 * s, ((it / p.raw_stages) & 1) ^ 1, &abort_flag)) { report(p.status, 3); break; }
-                int t = tile_begin + it;
-                const int tw = t % p.tiles_w; t /= p.tiles_w;
-                const int th = t % p.tiles_h;
-                const int tn = t / p.tiles_h;
-                const int q0 = tw * p.box_w, p0 = th * p.box_h, n0 = tn * p.box_n;
-                const uint32_t dst = smem_base + s * p.raw_bytes;
+                if (!mbar_wait(empty_raw0 + 8 * s, par, &abort_flag)) { report(p.status, 3); break; }
+                const int q0 = tw * box_w, p0 = th * box_h, n0 = tn * box_n;
+                const uint32_t dst = smem_base + s * raw_bytes;
                 const uint32_t bar = full_raw0 + 8 * s;
-                mbar_expect_tx(bar, p.tx_a + (uint32_t)ntaps * p.tx_per_tap);
+                mbar_expect_tx(bar, tx);
                 tma_load_4d(dst, &gp.tm_a, bar, m0, q0, p0, n0);
+                int r = r_first, sx = sx_first;
                 for (int tp = 0; tp < ntaps; ++tp) {
-                    const int r = (tap0 + tp) / p.R, sx = (tap0 + tp) % p.R;
-                    tma_load_4d(dst + raw_a + tp * raw_b, &gp.tm_b, bar, cn0, q0 + sx - p.pad, p0 + r - p.pad, n0);
+                    tma_load_4d(dst + raw_a + tp * raw_b, &gp.tm_b, bar, cn0, q0 + sx - pad, p0 + r - pad, n0);
+                    if (++sx == R) { sx = 0; ++r; }
                 }
+                if (++tw == tiles_w) { tw = 0; if (++th == tiles_h) { th = 0; ++tn; } }
+                if (++s == raw_stages) { s = 0; par ^= 1u; }
             }
             issued = it;
         }
     } else if (warp == 1) {
         if (lane == 0) {
             // ---- MMA issuer ----
-            int it = 0;
+            const int t_stages = p.t_stages;
+            int it = 0, t = 0;
+            uint32_t tpar = 0;
             for (; it < total; ++it) {
-                const int t = it % p.t_stages;
-                if (!mbar_wait(full_t0 + 8 * t, (it / p.t_stages) & 1, &abort_flag)) { report(p.status, 4); break; }
+                if (!mbar_wait(full_t0 + 8 * t, tpar, &abort_flag)) { report(p.status, 4); break; }
                 tc_fence_after();
                 const uint32_t a_src = smem_base + t_region0 + t * p.t_bytes, b_src = a_src + t_a;
                 // taps are stacked along N: groups of up to 256 / n_cols taps per MMA
@@ -1080,18 +1087,20 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
                         }
                 }
                 umma_commit(empty_t0 + 8 * t);
+                if (++t == t_stages) { t = 0; tpar ^= 1u; }
             }
             if (it == total) umma_commit(accum_bar);
         }
     } else {
         // ---- transposers (warps 2..5), then the epilogue ----
         const int tid = threadIdx.x - 64;
-        int it = 0;
+        int it = 0, s = 0, t = 0;
+        uint32_t spar = 0, tpar = 1u;
+        const int raw_stages = p.raw_stages, t_stages = p.t_stages;
         bool ok = true;
         for (; it < total && ok; ++it) {
-            const int s = it % p.raw_stages, t = it % p.t_stages;
-            ok = mbar_wait(full_raw0 + 8 * s, (it / p.raw_stages) & 1, &abort_flag) &&
-                 mbar_wait(empty_t0 + 8 * t, ((it / p.t_stages) & 1) ^ 1, &abort_flag);
+            ok = mbar_wait(full_raw0 + 8 * s, spar, &abort_flag) &&
+                 mbar_wait(empty_t0 + 8 * t, tpar, &abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) { if (lane == 0) report(p.status, 5); break; }
             const uint8_t* raw = smem + s * p.raw_bytes;
@@ -1109,6 +1118,8 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
             fence_async_smem();     // generic-proxy writes -> tensor-core reads
             __syncwarp();
             if (lane == 0) { mbar_arrive(full_t0 + 8 * t); mbar_arrive(empty_raw0 + 8 * s); }
+            if (++s == raw_stages) { s = 0; spar ^= 1u; }
+            if (++t == t_stages) { t = 0; tpar ^= 1u; }
         }
         if (tid == 0) raw_consumed = it;
 
