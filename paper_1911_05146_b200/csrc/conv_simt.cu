@@ -164,9 +164,13 @@ WgradSplit wgrad_split(const ConvShape& s)
     const int64_t pixels = (int64_t)s.N * s.P * s.Q;
     const int64_t outs = (int64_t)s.K * s.R * s.R * s.C;
     int64_t splits = pixels / 1024;                       // >= 1024 pixels per slice
+    // few output tiles (a stem convolution: one to three): the slices are what fills the GPU, down to 128 pixels each
+    const int64_t out_tiles = (int64_t)((s.K + BM - 1) / BM) * ((s.R * s.R * s.C + BN - 1) / BN);
+    if (splits * out_tiles < 296) splits = (296 + out_tiles - 1) / out_tiles;
+    if (splits > pixels / 128) splits = pixels / 128;
     const int64_t cap = (int64_t)(32 << 20) / (outs * 4) ;  // partials <= 32 MiB
     if (splits > cap) splits = cap;
-    if (splits > 256) splits = 256;                       // few output tiles (the 7x7 stem: 3): the slices are what fills the GPU
+    if (splits > 256) splits = 256;
     if (splits < 1) splits = 1;
     int64_t kps = (pixels + splits - 1) / splits;
     kps = (kps + BK - 1) / BK * BK;

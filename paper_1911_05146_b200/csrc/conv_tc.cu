@@ -1176,10 +1176,16 @@ wgrad_partials_reduce_kernel(const float* __restrict__ partials, float* __restri
     const long long i = (long long)blockIdx.x * 32 + lane;
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
     if (i < n4) {
-#pragma unroll 4
-        for (int z = zl; z < splits; z += 8) {
-            const float4 v = __ldcg(reinterpret_cast<const float4*>(partials + (long long)z * n) + i);
-            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        // four splits per batch, the four loads in flight together; splits beyond the last add zero
+        for (int z0 = zl; z0 < splits; z0 += 32) {
+            float4 v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int z = z0 + 8 * j;
+                v[j] = z < splits ? __ldcg(reinterpret_cast<const float4*>(partials + (long long)z * n) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { s.x += v[j].x; s.y += v[j].y; s.z += v[j].z; s.w += v[j].w; }
         }
     }
     sh[zl][lane] = s;

@@ -198,12 +198,21 @@ bn_reduce_kernel(const float* __restrict__ x, const float* __restrict__ dy, cons
         const int cg = pass * cgt + my_cg;
         double acc[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
         if (my_rl < rl && cg < cg_total) {
-#pragma unroll 2
-            for (int k = my_rl; k < nb; k += rl) {
-                const float4 va = __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 0) * C) + cg);
-                const float4 vb = __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 1) * C) + cg);
-                acc[0] += (double)va.x; acc[1] += (double)va.y; acc[2] += (double)va.z; acc[3] += (double)va.w;
-                acc[4] += (double)vb.x; acc[5] += (double)vb.y; acc[6] += (double)vb.z; acc[7] += (double)vb.w;
+            // four partial rows per batch, their eight loads in flight together
+            for (int k0 = my_rl; k0 < nb; k0 += 4 * rl) {
+                float4 va[4], vb[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int k = k0 + j * rl;
+                    const bool in = k < nb;
+                    va[j] = in ? __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 0) * C) + cg) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    vb[j] = in ? __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 1) * C) + cg) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    acc[0] += (double)va[j].x; acc[1] += (double)va[j].y; acc[2] += (double)va[j].z; acc[3] += (double)va[j].w;
+                    acc[4] += (double)vb[j].x; acc[5] += (double)vb[j].y; acc[6] += (double)vb[j].z; acc[7] += (double)vb[j].w;
+                }
             }
         }
         __syncthreads();
@@ -733,12 +742,21 @@ __device__ __forceinline__ void bn_big_finalise(const float* __restrict__ partia
     const int t = threadIdx.x;
     const int my_rl = t / cgt, my_cg = t % cgt;
     double acc[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
-#pragma unroll 4
-    for (int k = my_rl; k < n_part; k += rl) {
-        const float4 va = __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 0) * C) + my_cg);
-        const float4 vb = __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 1) * C) + my_cg);
-        acc[0] += (double)va.x; acc[1] += (double)va.y; acc[2] += (double)va.z; acc[3] += (double)va.w;
-        acc[4] += (double)vb.x; acc[5] += (double)vb.y; acc[6] += (double)vb.z; acc[7] += (double)vb.w;
+    // four partial rows per batch, their eight loads in flight together
+    for (int k0 = my_rl; k0 < n_part; k0 += 4 * rl) {
+        float4 va[4], vb[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int k = k0 + j * rl;
+            const bool in = k < n_part;
+            va[j] = in ? __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 0) * C) + my_cg) : make_float4(0.f, 0.f, 0.f, 0.f);
+            vb[j] = in ? __ldcg(reinterpret_cast<const float4*>(partials + ((int64_t)k * 2 + 1) * C) + my_cg) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            acc[0] += (double)va[j].x; acc[1] += (double)va[j].y; acc[2] += (double)va[j].z; acc[3] += (double)va[j].w;
+            acc[4] += (double)vb[j].x; acc[5] += (double)vb[j].y; acc[6] += (double)vb[j].z; acc[7] += (double)vb[j].w;
+        }
     }
     if (cgt <= 16) {
         for (int off = 16; off >= cgt; off >>= 1) {
@@ -1048,12 +1066,26 @@ grad_average_kernel(const float* __restrict__ slots, float* __restrict__ out, in
         float s[VEC];
 #pragma unroll
         for (int e = 0; e < VEC; ++e) s[e] = 0.f;
-#pragma unroll 8
-        for (int m = 0; m < M; ++m) {
-            const float* src = slots + (int64_t)m * G + i * VEC;
-            if (VEC == 4) { const float4 v = __ldcs(reinterpret_cast<const float4*>(src)); s[0] += v.x; s[1] += v.y; s[2 % VEC] += v.z; s[3 % VEC] += v.w; }
-            else if (VEC == 2) { const float2 v = __ldcs(reinterpret_cast<const float2*>(src)); s[0] += v.x; s[1 % VEC] += v.y; }
-            else s[0] += __ldcs(src);
+        // eight slots per batch, the loads of a batch in flight together whatever M is (a partially unrolled loop would
+        // run its remainder one load at a time); the sum stays in ascending slot order
+        for (int m0 = 0; m0 < M; m0 += 8) {
+            float q[8][VEC];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (m0 + j < M) {
+                    const float* src = slots + (int64_t)(m0 + j) * G + i * VEC;
+                    if (VEC == 4) { const float4 v = __ldcs(reinterpret_cast<const float4*>(src)); q[j][0] = v.x; q[j][1 % VEC] = v.y; q[j][2 % VEC] = v.z; q[j][3 % VEC] = v.w; }
+                    else if (VEC == 2) { const float2 v = __ldcs(reinterpret_cast<const float2*>(src)); q[j][0] = v.x; q[j][1 % VEC] = v.y; }
+                    else q[j][0] = __ldcs(src);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (m0 + j < M) {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) s[e] += q[j][e];
+                }
+            }
         }
         float* dst = out + i * VEC;
         if (VEC == 4) *reinterpret_cast<float4*>(dst) = make_float4(s[0] * inv_m, s[1 % VEC] * inv_m, s[2 % VEC] * inv_m, s[3 % VEC] * inv_m);
@@ -1076,11 +1108,23 @@ sgd_momentum_kernel(const float* __restrict__ slots, float* __restrict__ gavg, f
         float s[VEC], th[VEC], v[VEC];
 #pragma unroll
         for (int e = 0; e < VEC; ++e) s[e] = 0.f;
-#pragma unroll 8
-        for (int m = 0; m < M; ++m) {
-            const float* src = slots + (int64_t)m * G + i * VEC;
-            if (VEC == 4) { const float4 q = __ldcs(reinterpret_cast<const float4*>(src)); s[0] += q.x; s[1 % VEC] += q.y; s[2 % VEC] += q.z; s[3 % VEC] += q.w; }
-            else s[0] += __ldcs(src);
+        for (int m0 = 0; m0 < M; m0 += 8) {          // batches of eight slots, as in grad_average_kernel
+            float q[8][VEC];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (m0 + j < M) {
+                    const float* src = slots + (int64_t)(m0 + j) * G + i * VEC;
+                    if (VEC == 4) { const float4 w4 = __ldcs(reinterpret_cast<const float4*>(src)); q[j][0] = w4.x; q[j][1 % VEC] = w4.y; q[j][2 % VEC] = w4.z; q[j][3 % VEC] = w4.w; }
+                    else q[j][0] = __ldcs(src);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (m0 + j < M) {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) s[e] += q[j][e];
+                }
+            }
         }
         if (VEC == 4) {
             const float4 a = *reinterpret_cast<const float4*>(theta + i * 4), b = *reinterpret_cast<const float4*>(vel + i * 4);
