@@ -381,6 +381,8 @@ def main():
                     help="partition cut points: balanced = the library's load balancer on its modelled op costs; "
                          "equal = the same number of ops in every partition")
     ap.add_argument("--conv-path", type=int, default=0)
+    ap.add_argument("--cell-ctas", type=int, default=-1,
+                    help="CTAs of the persistent forward cell kernels (HPF_OPT_CELL_CTAS); 0: one launch per convolution; -1: the library's default")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-kernel-roofline", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
@@ -427,6 +429,8 @@ def main():
     model = hpf.Model(ops, (B,) + tuple(hwc), cuts, M)
     model.set_option(hpf.OPT_GRAPH, 0 if args.no_graph else 1)
     model.set_option(hpf.OPT_CONV_PATH, args.conv_path)
+    if args.cell_ctas >= 0:
+        model.set_option(hpf.OPT_CELL_CTAS, args.cell_ctas)
     G = model.num_params()
     params = torch.from_numpy(theta).to(dev)
     slots = torch.empty((M, G), device=dev)
@@ -470,6 +474,15 @@ def main():
     loss = model.loss()
     model.synchronize(0)
 
+    # where the step's time goes: the three phases timed apart (a diagnostic; events on stream 0, which every phase joins)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    phase_ms = [0.0, 0.0, 0.0]
+    for _ in range(3):
+        ev[0].record(s0); model.forward(dx, dl); ev[1].record(s0); model.backward(); ev[2].record(s0); model.grad_average(); ev[3].record(s0)
+        barrier()
+        for k in range(3):
+            phase_ms[k] += ev[k].elapsed_time(ev[k + 1]) / 3
+
     # end to end: host buffers in, loss out, every step
     ms_e2e = float("nan")
     if not args.skip_e2e:
@@ -502,7 +515,8 @@ def main():
         "config": {"workload": NAMES[args.workload], "global_batch": world * B, "micro_batches": M,
                    "partitions": model.num_partitions(), "parallelism": "replicas x%d, no data-path collective" % world,
                    "l2": "working set %.1f GB per step exceeds the 126 MB L2; no explicit flush" % (ws_bytes / 1e9),
-                   "cuts": args.cuts, "cut_points": list(cuts), "graph": not args.no_graph, "conv_sites_tensor_core": n_tc, "conv_sites_cuda_core": n_cc,
+                   "cuts": args.cuts, "cut_points": list(cuts), "graph": not args.no_graph, "cell_ctas": args.cell_ctas,
+                   "phase_ms": {"forward": phase_ms[0], "backward": phase_ms[1], "average": phase_ms[2]}, "conv_sites_tensor_core": n_tc, "conv_sites_cuda_core": n_cc,
                    "loss": loss},
         "e2e": {"value": world * B / (ms_e2e / args.steps * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": int(hx.numel() * 4 + hl.numel() * 4), "d2h_bytes_per_step": 4},

@@ -113,10 +113,16 @@ int hpf_model_destroy(hpf_model *model);
  *                          pipeline, as it really ran); read them with hpf_cell_times.  Default 0.
  *   HPF_OPT_BN_CLUSTER     1 (default): the backward of a BN whose micro-batch tensor is small enough to sit in the
  *                          registers of a few thread-block clusters is one launch (the CTAs of a cluster exchange their
- *                          per-channel sums through distributed shared memory); 0: always the reduce + apply pair. */
+ *                          per-channel sums through distributed shared memory); 0: always the reduce + apply pair.
+ *   HPF_OPT_CELL_CTAS      N > 0: the forward tensor-core convolutions of a (partition, micro-batch) cell that follow each
+ *                          other with no other kernel between them run as ONE persistent kernel of N CTAs that stays
+ *                          resident for the cell, walks the list of convolutions and meets at a grid-wide barrier between
+ *                          them (Section 5.3's stage as one resident grid instead of a chain of launches).  The cells of
+ *                          all partitions must fit the GPU together (hpf_bind: HPF_ERR_UNSUPPORTED otherwise).  Results
+ *                          are bit-identical to N = 0 when the tile assignment is the same.  0: one launch per convolution. */
 typedef enum { HPF_OPT_GRAPH = 1, HPF_OPT_CONV_PATH = 2, HPF_OPT_SINGLE_STREAM = 3, HPF_OPT_KEEP_MESSAGES = 4,
                HPF_OPT_FUSE_ADD = 5, HPF_OPT_PDL = 6, HPF_OPT_WGRAD_PASSES = 7, HPF_OPT_FUSE_BN = 8, HPF_OPT_CELL_TIMES = 9,
-               HPF_OPT_BN_CLUSTER = 10 } hpf_option;
+               HPF_OPT_BN_CLUSTER = 10, HPF_OPT_CELL_CTAS = 11 } hpf_option;
 int hpf_set_option(hpf_model *model, int32_t option, int32_t value);
 
 /* ---- integer bookkeeping (Section 5.1 lists, Section 5.3 pipelining) ----------------------------- */
@@ -252,11 +258,13 @@ int hpf_bnrelu_bwd(const float *d_x, const float *d_dy, const float *d_gamma, co
  *   - Sizes whose partial sums exceed the array (hpf_bnrelu_scratch_bytes(rows, C) > 2 MiB) are refused
  *     with HPF_ERR_WORKSPACE; nothing is launched.
  *   - The first call on a device looks up the array's device address (that device must be current).
- *     Make that first call outside any stream capture.
+ *     Make that first call outside any stream capture.  Two host threads may make it at the same time.
  *   - All calls on a device share the one array, which keeps the previous call's contents; the call
  *     clears the part that must start at zero.  Two calls whose kernels overlap on the GPU (different
  *     streams, no ordering between them) race on it: order them.
- * Inputs and outputs are the caller's, exactly as for hpf_bnrelu_fwd; results are those of its two-kernel path. */
+ * Inputs and outputs are the caller's, exactly as for hpf_bnrelu_fwd.  The call always runs the reduce + apply
+ * kernel pair and never the one-launch on-chip path, so for tensors of 16 MB and more, where hpf_bnrelu_fwd takes
+ * that path, the two agree to rounding (a different summation order), not bit for bit, unless HPF_BN_RESIDENT=0. */
 int hpf_bnrelu_fwd_static(const float *d_x, const float *d_gamma, const float *d_beta, float eps, float *d_y,
                           float *d_stats, int64_t rows, int32_t C, void *stream);
 int hpf_static_scratch_bytes(size_t *bytes);

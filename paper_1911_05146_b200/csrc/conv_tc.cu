@@ -51,6 +51,8 @@ constexpr int kFwdMaxStages = 4;
 #endif
 constexpr int kWgradWantCtas = HPF_WGRAD_WANT;   // CTAs a weight-gradient launch spreads its pixel walk over at least
 constexpr int kMultiTileFrom = 2 * 296;     // CTAs (two per SM) beyond which a forward / data-gradient launch gives each CTA two tiles
+constexpr unsigned int kCellTmemCols = 256;  // tensor-memory columns a persistent cell CTA may hold (two such CTAs share an SM's 512)
+constexpr unsigned int kCellSmemBudget = 100 * 1024;   // dynamic shared memory of a cell CTA (two per SM)
 constexpr unsigned int kWgradSlack = 16384;   // an MMA reads 128 operand rows (16 KB) from a base that may be the last one in use
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -66,6 +68,10 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_inval(uint32_t bar)
+{
+    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
@@ -318,17 +324,24 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 // x = hi + lo, hi = x with the low 13 significand bits cleared (what a TF32 operand keeps)
 __device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 
-// BN statistics from per-tile sums [n_tiles][2][C] (sum x, sum x*x): the tiles are added in a fixed order in fp64, so
-// every caller gets the same bits.  Called by 256 threads (tid 0..255) that share named barrier 1; C is a power of
-// two in 16..256; bn_red: 256 x 4 doubles of shared memory.  On return thread tid < C holds its channel's mean and
+// BN statistics from per-tile moments [n_tiles][2][C]: per tile and channel the mean of the tile's values and the sum
+// of their squared deviations from that mean (M2).  Every tile holds the same number of values (the host fuses only
+// launches whose tiles are all full), so the total is
+//     mean = average of the tile means,   M2 = sum of the tile M2 + n_tile * sum (tile mean - mean)^2,
+// evaluated about tile 0's mean so that no difference of large numbers appears anywhere: the result stays accurate
+// however far a channel's mean is from zero compared with its spread.  The tiles are added in a fixed order in fp64,
+// so every caller gets the same bits.  Called by 256 threads (tid 0..255) that share named barrier 1; C is a power of
+// two in 16..256; bn_red: 256 x 8 doubles of shared memory.  On return thread tid < C holds its channel's mean and
 // 1/sqrt(var + eps).
 __device__ __forceinline__ void bn_combine_partials(const float* partials, int n_tiles, int C, double inv_rows, float eps,
-                                                    double (*bn_red)[4], int tid, float* mean, float* rstd)
+                                                    double (*bn_red)[8], int tid, float* mean, float* rstd)
 {
-    const int ncol4 = C >> 1;                          // float4 columns of one tile's [2][C] sums; 256 % ncol4 == 0
+    const int ncol4 = C >> 1;                          // float4 columns of one tile's [2][C] moments; 256 % ncol4 == 0
     const int col4 = tid % ncol4, ln = tid / ncol4, L = 256 / ncol4;
     const float4* part = reinterpret_cast<const float4*>(partials);
-    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+    // the first C/4 columns are tile means: accumulated as differences from tile 0's mean (and their squares)
+    const float4 ref = col4 < (C >> 2) ? __ldcg(part + col4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0, b0 = 0.0, b1 = 0.0, b2 = 0.0, b3 = 0.0;
     // eight rows per batch, all eight loads in flight together (a loop that used each load before issuing the next would
     // pay an L2 round trip per row); rows beyond the last add zero
     for (int k0 = ln; k0 < n_tiles; k0 += 8 * L) {
@@ -336,48 +349,65 @@ __device__ __forceinline__ void bn_combine_partials(const float* partials, int n
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int k = k0 + j * L;
-            v[j] = k < n_tiles ? __ldcg(part + (size_t)k * ncol4 + col4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            v[j] = k < n_tiles ? __ldcg(part + (size_t)k * ncol4 + col4) : ref;
         }
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { a0 += (double)v[j].x; a1 += (double)v[j].y; a2 += (double)v[j].z; a3 += (double)v[j].w; }
+        for (int j = 0; j < 8; ++j) {
+            const double d0 = (double)(v[j].x - ref.x), d1 = (double)(v[j].y - ref.y), d2 = (double)(v[j].z - ref.z), d3 = (double)(v[j].w - ref.w);
+            a0 += d0; a1 += d1; a2 += d2; a3 += d3;
+            b0 += d0 * d0; b1 += d1 * d1; b2 += d2 * d2; b3 += d3 * d3;
+        }
     }
     if (ncol4 <= 16) {
         // several lanes of a column sit in one warp: a fixed butterfly first, then the eight warps in ascending order
         for (int off = 16; off >= ncol4; off >>= 1) {
             a0 += __shfl_xor_sync(0xffffffffu, a0, off); a1 += __shfl_xor_sync(0xffffffffu, a1, off);
             a2 += __shfl_xor_sync(0xffffffffu, a2, off); a3 += __shfl_xor_sync(0xffffffffu, a3, off);
+            b0 += __shfl_xor_sync(0xffffffffu, b0, off); b1 += __shfl_xor_sync(0xffffffffu, b1, off);
+            b2 += __shfl_xor_sync(0xffffffffu, b2, off); b3 += __shfl_xor_sync(0xffffffffu, b3, off);
         }
         const int warp = tid >> 5, lane = tid & 31;
-        double (*wsum)[4] = bn_red + 128;                   // [warp * ncol4 + column]; rows 0..127 stay free for the totals
-        if (lane < ncol4) { double* d = wsum[warp * ncol4 + lane]; d[0] = a0; d[1] = a1; d[2] = a2; d[3] = a3; }
+        double (*wsum)[8] = bn_red + 128;                   // [warp * ncol4 + column]; rows 0..127 stay free for the totals
+        if (lane < ncol4) {
+            double* d = wsum[warp * ncol4 + lane];
+            d[0] = a0; d[1] = a1; d[2] = a2; d[3] = a3; d[4] = b0; d[5] = b1; d[6] = b2; d[7] = b3;
+        }
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (tid < ncol4) {
-            double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
+            double t[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
             for (int w = 0; w < 8; ++w) {
                 const double* r = wsum[w * ncol4 + tid];
-                t0 += r[0]; t1 += r[1]; t2 += r[2]; t3 += r[3];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) t[q] += r[q];
             }
-            bn_red[tid][0] = t0; bn_red[tid][1] = t1; bn_red[tid][2] = t2; bn_red[tid][3] = t3;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) bn_red[tid][q] = t[q];
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
     } else {
-    bn_red[tid][0] = a0; bn_red[tid][1] = a1; bn_red[tid][2] = a2; bn_red[tid][3] = a3;
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    if (tid < ncol4) {
-        // rows tid, tid + ncol4, ... are read by this thread alone, so the total can go back into row tid
-        double t0 = 0.0, t1 = 0.0, t2 = 0.0, t3 = 0.0;
-        for (int l = 0; l < L; ++l) {
-            const double* r = bn_red[l * ncol4 + tid];
-            t0 += r[0]; t1 += r[1]; t2 += r[2]; t3 += r[3];
+        double* mine = bn_red[tid];
+        mine[0] = a0; mine[1] = a1; mine[2] = a2; mine[3] = a3; mine[4] = b0; mine[5] = b1; mine[6] = b2; mine[7] = b3;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (tid < ncol4) {
+            // rows tid, tid + ncol4, ... are read by this thread alone, so the total can go back into row tid
+            double t[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+            for (int l = 0; l < L; ++l) {
+                const double* r = bn_red[l * ncol4 + tid];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) t[q] += r[q];
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) bn_red[tid][q] = t[q];
         }
-        bn_red[tid][0] = t0; bn_red[tid][1] = t1; bn_red[tid][2] = t2; bn_red[tid][3] = t3;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
     }
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    }
-    const double* tot = &bn_red[0][0];                  // [2][C]: sums, then sums of squares
     if (tid < C) {
-        const double m = tot[tid] * inv_rows;
-        double var = tot[C + tid] * inv_rows - m * m;
+        const double T = (double)n_tiles;
+        const double sd = bn_red[tid >> 2][tid & 3], sq = bn_red[tid >> 2][4 + (tid & 3)];        // sum of (tile mean - ref), of its square
+        const double m2 = bn_red[(C >> 2) + (tid >> 2)][tid & 3];                                   // sum of the tile M2
+        const double n_tile = 1.0 / (inv_rows * T);
+        const double m = (double)__ldcg(partials + tid) + sd / T;
+        double var = (m2 + n_tile * (sq - sd * sd / T)) * inv_rows;
         if (var < 0.0) var = 0.0;
         *mean = (float)m;
         *rstd = (float)(1.0 / sqrt(var + (double)eps));
@@ -387,20 +417,25 @@ __device__ __forceinline__ void bn_combine_partials(const float* partials, int n
 // ------------------------------------------------------------------------------------------------
 // forward / data-gradient kernel: 10 warps = TMA producer, MMA issuer, 8 splitter / epilogue warps
 // ------------------------------------------------------------------------------------------------
-// MULTI = false: one 128-pixel tile per CTA (the shortest launch; what a launch of up to one wave wants).
-// MULTI = true: p.tiles_per_cta tiles per CTA for launches of several waves: fewer CTAs, and a tile's write-out hides
-// the next tile's loads, split and MMAs.
-template <bool MULTI, bool KSPLIT = false>
-__global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_constant__ FwdParams gp)
+// One CTA's share of a forward / data-gradient launch: `vb` of `vg` (block index and grid size of the launch as a stand-alone
+// launch has them).  MODE 0: one 128-pixel tile per CTA (the shortest launch; what a launch of up to one wave wants).
+// MODE 1: p.tiles_per_cta tiles per CTA for launches of several waves: fewer CTAs, and a tile's write-out hides the next
+// tile's loads, split and MMAs.  MODE 2: the K loop split over vg.z CTAs.  MODE 3: inside the persistent cell kernel, which
+// runs many launches one after the other in one resident grid: tiles per CTA and K split are read from the parameters,
+// tensor memory is allocated once by the caller, the mbarriers are set up again for every call, and nothing of the
+// programmatic-launch protocol applies.  `p` (shared memory) holds gp->s.
+template <int MODE>
+__device__ __forceinline__ int conv_fwd_cta(const FwdParams* gpp, FwdScalars& p, const uint3 vb, const uint3 vg, const uint32_t cell_tmem_base,
+                                             const bool cell_first)
 {
-    __shared__ FwdScalars p;                 // scalar parameters, see load_scalars
+    const FwdParams& gp = *gpp;
+    constexpr bool CELL = MODE == 3;
+    const bool MULTI = CELL ? p.tiles_per_cta > 1 : MODE == 1;
+    const bool KSPLIT = CELL ? p.ksplit > 1 : MODE == 2;
 #if defined(HPF_TC_TIMELINE) && HPF_TC_TIMELINE == 2
     __shared__ unsigned long long tl_s[16];
     if (threadIdx.x < 16) tl_s[threadIdx.x] = 0;
 #endif
-    pdl_launch_dependents();
-    load_scalars(&p, &gp.s);
-    __syncthreads();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[3 * 8 + 4];       // full[8], empty[8], split[8], accum[4] (one per tile of this CTA)
     __shared__ uint32_t tmem_slot;
@@ -419,11 +454,11 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
     const uint32_t off_blo = off_b + p.b_bytes;
 
     const int tiles_per_cta = MULTI ? p.tiles_per_cta : 1;
-    const int tile0 = blockIdx.x * tiles_per_cta;
+    const int tile0 = (int)vb.x * tiles_per_cta;
     const int my_tiles = MULTI ? (p.n_tiles - tile0 < tiles_per_cta ? p.n_tiles - tile0 : tiles_per_cta) : 1;
     const uint32_t acc_cols = MULTI ? p.acc_cols : 0u;
     const uint32_t stg_off = MULTI ? p.stg_off : 0u;
-    const int co0 = blockIdx.y * p.n_chunk;
+    const int co0 = (int)vb.y * p.n_chunk;
     // first pixel (q0, p0, n0) of tile t
 #define HPF_TILE_ORIGIN(t_)                                                          \
     int q0, p0, n0;                                                                   \
@@ -436,8 +471,8 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
     if (threadIdx.x == 0) HPF_TL(0);
     const int total = p.R * p.R * p.n_kchunks;
     // this CTA's share of the K loop (all of it unless the launch splits K over gridDim.z)
-    const int kb = KSPLIT ? (int)(((long long)total * blockIdx.z) / p.ksplit) : 0;
-    const int ke = KSPLIT ? (int)(((long long)total * (blockIdx.z + 1)) / p.ksplit) : total;
+    const int kb = KSPLIT ? (int)(((long long)total * vb.z) / p.ksplit) : 0;
+    const int ke = KSPLIT ? (int)(((long long)total * (vb.z + 1)) / p.ksplit) : total;
     // Thread 0 is the TMA producer.  The origin of its first tile and its first K step are a chain of dependent
     // shared-memory reads and integer divisions in ONE thread (most of a microsecond): worked out here, while the CTA
     // still waits for tensor memory and for the preceding kernel, not between that wait and the first copy.
@@ -448,21 +483,23 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
         if (KSPLIT) { f_tap = kb / p.n_kchunks; f_kc = kb % p.n_kchunks; f_r = f_tap / p.R; f_sx = f_tap % p.R; }
     }
     if (threadIdx.x == 0) {
+        if (CELL && !cell_first)       // the barriers of the call before are retired first
+            for (int j = 0; j < 3 * 8 + 4; ++j) mbar_inval(full0 + 8 * j);
         for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); mbar_init(split0 + 8 * s, 8); }
         for (int j = 0; j < 4; ++j) mbar_init(accum_bar + 8 * j, 1);
         abort_flag = 0; issued = 0; consumed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (threadIdx.x == 32) { prefetch_tmap(&gp.tm_a); prefetch_tmap(&gp.tm_b); if (p.passes == 3) prefetch_tmap(&gp.tm_b_lo); }
-    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), p.tmem_cols);
+    if (!CELL && warp == 0) tmem_alloc(smem_u32(&tmem_slot), p.tmem_cols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     // Everything above touched only parameters, shared and tensor memory.  The TMA producer (thread 0) first works out
     // its first tile's coordinates - a chain of dependent shared-memory reads and integer divisions of most of a
     // microsecond - and waits for the preceding kernel only then, right before its first copy.
-    if (threadIdx.x != 0) pdl_wait();
-    const uint32_t tmem_base = tmem_slot;
+    if (!CELL && threadIdx.x != 0) pdl_wait();
+    const uint32_t tmem_base = CELL ? cell_tmem_base : tmem_slot;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -486,7 +523,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     if (!mbar_wait(empty0 + 8 * st, par, &abort_flag)) { report(p.status, 1); live = false; break; }
                     const uint32_t dst = smem_base + st * stage_bytes;
                     const int cx = kc * kchunk, cq = q0 + sx - pad, cp = p0 + r - pad, cb = tap * c_in + cx;
-                    if (it == 0) { pdl_wait(); HPF_TL(1); }
+                    if (!CELL && it == 0) { pdl_wait(); HPF_TL(1); }
                     mbar_expect_tx(full0 + 8 * st, tx);
                     tma_load_4d(dst, &gp.tm_a, full0 + 8 * st, cx, cq, cp, n0);
                     tma_load_2d(dst + off_b, &gp.tm_b, full0 + 8 * st, cb, co0);
@@ -496,7 +533,16 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     if (++st == stages) { st = 0; par ^= 1u; }
                 }
             }
-            if (it == 0) pdl_wait();         // nothing to copy: still ordered behind the preceding kernel
+            if (!CELL && it == 0) pdl_wait();         // nothing to copy: still ordered behind the preceding kernel
+            if (CELL && live) {
+                // The MMA issuer's last commits on the `empty` barriers are awaited by nobody in a stand-alone launch.  Here
+                // the barriers are set up again for the next call, so every arrival still on its way has to land first.
+                const int left = it < stages ? it : stages;
+                for (int j = 0; j < left; ++j) {
+                    if (!mbar_wait(empty0 + 8 * st, par, &abort_flag)) { report(p.status, 8); break; }
+                    if (++st == stages) { st = 0; par ^= 1u; }
+                }
+            }
             issued = it;
         }
     } else if (warp == 1) {
@@ -565,13 +611,13 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                 // The producer left only its per-tile sums (few enough that adding them here, under the first copy's
                 // latency, is cheaper than a ticket at the producer's end): every CTA adds them in the same fixed order,
                 // so all CTAs hold identical statistics; the first CTA stores them for the backward pass.
-                __shared__ double bn_red[256][4];
+                __shared__ double bn_red[256][8];
                 float gam = 0.f, bet = 0.f, mu = 0.f, rs = 0.f;
                 if (tid < C) { gam = __ldg(p.bn_in_gamma + tid); bet = __ldg(p.bn_in_beta + tid); }   // travel with the sums
                 bn_combine_partials(p.bn_in_partials, p.bn_in_tiles, C, p.bn_in_inv_rows, p.bn_in_eps, bn_red, tid, &mu, &rs);
                 if (tid < C) {
                     bn_par[0][tid] = mu; bn_par[1][tid] = rs; bn_par[2][tid] = gam; bn_par[3][tid] = bet;
-                    if (blockIdx.x == 0 && blockIdx.y == 0) { p.bn_in_stats_out[tid] = mu; p.bn_in_stats_out[C + tid] = rs; }
+                    if (vb.x == 0 && vb.y == 0) { p.bn_in_stats_out[tid] = mu; p.bn_in_stats_out[C + tid] = rs; }
                 }
             }
             // the statistics written by the kernel before (not the read-only path) and the parameters: fetched now, used
@@ -589,7 +635,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             const int cph = tid % f4row;
             const int clog = p.kchunk == 32 ? (cph ^ (row0 & 7)) : (cph ^ ((row0 >> 1) & 3));
             const bool three = p.passes == 3;
-            const bool writer = blockIdx.y == 0;
+            const bool writer = vb.y == 0;
             const int stages = p.stages, nkc = p.n_kchunks, R = p.R, pad = p.pad;
             // position of row r of the pixel box (the same for every tile)
             int rw[4], rh[4], rn[4];
@@ -747,8 +793,8 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                 // is) and goes on to the write-out; the others are done.
                 __shared__ int last_of_unit;
                 const int c4n_ = p.n_chunk >> 2, tile_f4 = kTileM * c4n_;
-                const unsigned int unit = blockIdx.x * gridDim.y + blockIdx.y;
-                float4* mine = reinterpret_cast<float4*>(p.splitk_partials) + ((size_t)unit * p.ksplit + blockIdx.z) * tile_f4;
+                const unsigned int unit = vb.x * vg.y + vb.y;
+                float4* mine = reinterpret_cast<float4*>(p.splitk_partials) + ((size_t)unit * p.ksplit + vb.z) * tile_f4;
                 for (int idx = tid; idx < tile_f4; idx += 256) {
                     const int r = idx / c4n_, c4 = idx - r * c4n_;
                     mine[idx] = *reinterpret_cast<const float4*>(stg + (size_t)r * p.stg_pitch + 4 * c4);
@@ -774,7 +820,7 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     asm volatile("bar.sync 1, 256;" ::: "memory");
                 }
             }
-            float4 sa = make_float4(0.f, 0.f, 0.f, 0.f), sb = sa;
+            float4 sa = make_float4(0.f, 0.f, 0.f, 0.f), sb = sa, sk = sa;
             if (write_out) {
             // write-out: consecutive threads write consecutive float4 of a pixel's channel row.  Eight warps cannot
             // hide latency by occupancy, so four independent float4 are in flight per thread and nothing is re-read.
@@ -787,6 +833,16 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
             const unsigned int pitch = p.stg_pitch;
             const long long dense_h = p.dense_h, dense_w = p.dense_w;
             const int stat_mode = p.stat_mode;
+            if (stat_mode) {
+                // The statistics are accumulated as deviations from the tile's first pixel (what the kernel stores for it,
+                // so residual included): sums of x and x*x themselves would cancel catastrophically in var = E[x^2] - mean^2
+                // for a channel whose mean is large compared with its spread.  A thread keeps one group of 4 channels
+                // throughout (256 is a multiple of c4n), so one shift per thread does.
+                const int c4k = tid % c4n;
+                sk = *reinterpret_cast<const float4*>(stg + 4 * c4k);
+                if (extra) { const float4 e = __ldcg(reinterpret_cast<const float4*>(extra + row_off[0] + 4 * c4k)); sk.x += e.x; sk.y += e.y; sk.z += e.z; sk.w += e.w; }
+                if (accumulate) { const float4 e = *reinterpret_cast<const float4*>(outp + row_off[0] + 4 * c4k); sk.x += e.x; sk.y += e.y; sk.z += e.z; sk.w += e.w; }
+            }
             for (int base = tid; base < total4; base += 1024) {
                 float4 o[4];
                 int off[4];
@@ -822,9 +878,10 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     float* optr = outp + off[u];
                     *reinterpret_cast<float4*>(optr) = o[u];
                     if (stat_mode) {
-                        sa.x += o[u].x; sa.y += o[u].y; sa.z += o[u].z; sa.w += o[u].w;
-                        sb.x = fmaf(o[u].x, o[u].x, sb.x); sb.y = fmaf(o[u].y, o[u].y, sb.y);
-                        sb.z = fmaf(o[u].z, o[u].z, sb.z); sb.w = fmaf(o[u].w, o[u].w, sb.w);
+                        const float dx_ = o[u].x - sk.x, dy_ = o[u].y - sk.y, dz_ = o[u].z - sk.z, dw_ = o[u].w - sk.w;
+                        sa.x += dx_; sa.y += dy_; sa.z += dz_; sa.w += dw_;
+                        sb.x = fmaf(dx_, dx_, sb.x); sb.y = fmaf(dy_, dy_, sb.y);
+                        sb.z = fmaf(dz_, dz_, sb.z); sb.w = fmaf(dw_, dw_, sb.w);
                     }
                     if (fill[u]) {
                         // strided data gradient: the positions between the samples receive no contribution
@@ -858,12 +915,23 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                     red[2 * tid] = sa; red[2 * tid + 1] = sb;
                 }
                 asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (tid < c4n * 2) {
-                    const int g = tid >> 1, which = tid & 1;
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int t2 = g; t2 < n_rows; t2 += c4n) { const float4 v2 = red[2 * t2 + which]; acc.x += v2.x; acc.y += v2.y; acc.z += v2.z; acc.w += v2.w; }
-                    float* dstp = p.stat_partials + ((size_t)(tile0 + tj) * 2 + which) * p.c_out + co0 + 4 * g;
-                    *reinterpret_cast<float4*>(dstp) = acc;
+                if (tid < c4n) {
+                    // thread g owns channel group g (its own shift sk is that group's): the tile's mean and the sum of
+                    // squared deviations from it, from the shifted sums
+                    const int g = tid;
+                    float4 s1 = make_float4(0.f, 0.f, 0.f, 0.f), s2 = s1;
+                    for (int t2 = g; t2 < n_rows; t2 += c4n) {
+                        const float4 v1 = red[2 * t2], v2 = red[2 * t2 + 1];
+                        s1.x += v1.x; s1.y += v1.y; s1.z += v1.z; s1.w += v1.w;
+                        s2.x += v2.x; s2.y += v2.y; s2.z += v2.z; s2.w += v2.w;
+                    }
+                    const float inv_n = 1.f / (float)(p.box_w * p.box_h * p.box_n);       // every tile of a fused launch is full
+                    const float4 mt = make_float4(sk.x + s1.x * inv_n, sk.y + s1.y * inv_n, sk.z + s1.z * inv_n, sk.w + s1.w * inv_n);
+                    const float4 m2 = make_float4(s2.x - s1.x * s1.x * inv_n, s2.y - s1.y * s1.y * inv_n, s2.z - s1.z * s1.z * inv_n,
+                                                  s2.w - s1.w * s1.w * inv_n);
+                    float* dstp = p.stat_partials + (size_t)(tile0 + tj) * 2 * p.c_out + co0 + 4 * g;
+                    *reinterpret_cast<float4*>(dstp) = mt;
+                    *reinterpret_cast<float4*>(dstp + p.c_out) = m2;
                     if (stat_mode == 1) __threadfence();
                 }
             }
@@ -880,14 +948,15 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
                 if (stat_mode == 1) asm volatile("bar.sync 1, 256;" ::: "memory");
                 if (stat_mode == 1 && tid == 0) {
                     const unsigned int done_before = atomicAdd(p.stat_ticket, 1u);
-                    is_last = done_before == gridDim.x * gridDim.y - 1;
+                    is_last = done_before == vg.x * vg.y - 1;
                 }
                 if (stat_mode == 1) asm volatile("bar.sync 1, 256;" ::: "memory");
                 if (stat_mode == 1 && is_last) {
                     __threadfence();
                     float mu = 0.f, rs = 0.f;
-                    bn_combine_partials(p.stat_partials, MULTI ? p.n_tiles : (int)gridDim.x, p.c_out, p.stat_inv_rows, p.stat_eps,
-                                        reinterpret_cast<double (*)[4]>(stg), tid, &mu, &rs);
+                    // every tile is written out and the pipeline buffers are idle: they hold the reduction
+                    bn_combine_partials(p.stat_partials, p.n_tiles, p.c_out, p.stat_inv_rows, p.stat_eps,
+                                        reinterpret_cast<double (*)[8]>(smem), tid, &mu, &rs);
                     if (tid < p.c_out) { p.stat_out[tid] = mu; p.stat_out[p.c_out + tid] = rs; }
                     if (tid == 0) *p.stat_ticket = 0u;
                 }
@@ -908,17 +977,134 @@ __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_consta
         }
     }
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
+    if (!CELL && warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
     if (threadIdx.x == 0) HPF_TL(9);
 #if defined(HPF_TC_TIMELINE) && HPF_TC_TIMELINE == 2
     __syncthreads();
     if (threadIdx.x < 16) {
-        const int tiles = gridDim.x;
+        const int tiles = vg.x;
         const int cls = (p.R == 3 ? 1 : 0) + 2 * (tiles >= 128 ? 0 : (tiles >= 32 ? 1 : 2)) + (p.bn_in ? 0 : 0);
         if (threadIdx.x == 0) atomicAdd(&g_tl_acc[cls][0], 1ull);
         else if (tl_s[threadIdx.x] > tl_s[0]) atomicAdd(&g_tl_acc[cls][threadIdx.x], tl_s[threadIdx.x] - tl_s[0]);
     }
 #endif
+    return abort_flag;          // uniform: nobody writes it between the barrier above and the next call's set-up
+}
+
+template <bool MULTI, bool KSPLIT = false>
+__global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_constant__ FwdParams gp)
+{
+    __shared__ FwdScalars p;                 // scalar parameters, see load_scalars
+    pdl_launch_dependents();
+    load_scalars(&p, &gp.s);
+    __syncthreads();
+    conv_fwd_cta<MULTI ? 1 : (KSPLIT ? 2 : 0)>(&gp, p, make_uint3(blockIdx.x, blockIdx.y, blockIdx.z), make_uint3(gridDim.x, gridDim.y, gridDim.z), 0u, true);
+}
+
+// ------------------------------------------------------------------------------------------------
+// persistent cell kernel: the forward convolutions of one (partition, micro-batch) cell in ONE resident grid
+// ------------------------------------------------------------------------------------------------
+// A cell of the pipeline is a chain of a hundred and more small dependent convolutions.  As separate launches each pays
+// the launch-to-launch latency, and eight stages' worth of them compete for SM slots in which their CTAs mostly wait.
+// Here a fixed, small grid stays resident for the whole cell and walks the list of launches: the CTAs share out the
+// CTAs of each launch (virtual CTAs: block index and grid size of the stand-alone launch), run them with the same code,
+// and meet at a grid-wide barrier before the next launch, whose input the whole grid has just produced.  Every CTA of
+// the grid must be resident at the same time; the host sizes the grids so that all cells that can run concurrently fit
+// the GPU together.  The barrier wait is bounded like every other wait here.
+struct alignas(64) CellOp {
+    FwdParams p;                 // exactly what the stand-alone launch would receive
+    unsigned int gx, gy, gz;     // its grid
+    unsigned int reserved;
+};
+struct CellParams {
+    const CellOp* ops;           // device memory, written before the launch and read-only for the kernel
+    int n_ops;
+    unsigned int* barrier;       // {arrivals, generation}: zero before the first use, left with arrivals at zero
+    DeviceStatus* status;
+    unsigned int tmem_cols;      // the largest accumulator of the list
+};
+
+__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* ptr)
+{
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_gpu(unsigned int* ptr, unsigned int v)
+{
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(ptr), "r"(v) : "memory");
+}
+
+// All CTAs of the grid arrive; the last one opens the next generation.  What the CTAs wrote before the barrier is
+// visible to all of them after it, also to copies issued through the async proxy (TMA).  Returns false when the wait ran
+// out or another kernel already reported a failure.
+__device__ __forceinline__ bool cell_grid_barrier(unsigned int* bar, DeviceStatus* status, int* stop_flag)
+{
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int gen = ld_acquire_gpu(bar + 1);      // cannot advance before this CTA has arrived
+        __threadfence();
+        int stop = 0;
+        if (atomicAdd(bar, 1u) == gridDim.x - 1) {
+            bar[0] = 0u;
+            __threadfence();
+            st_release_gpu(bar + 1, gen + 1u);
+        } else {
+            const long long t0 = clock64();
+            int polls = 0;
+            while (ld_acquire_gpu(bar + 1) == gen) {
+                if ((++polls & 63) == 0 && (clock64() - t0 > kWaitLimit || ld_acquire_gpu(&status->code) != 0u)) { report(status, 9); stop = 1; break; }
+            }
+        }
+        *stop_flag = stop;
+    }
+    __syncthreads();
+    asm volatile("fence.proxy.async;" ::: "memory");
+    return *stop_flag == 0;
+}
+
+__global__ void __launch_bounds__(320, 2) conv_tc_cell_kernel(const __grid_constant__ CellParams cp)
+{
+    __shared__ FwdScalars p;
+    __shared__ unsigned int vgrid[4];
+    __shared__ uint32_t cell_tmem;
+    __shared__ int cell_stop;
+    constexpr int kWords = (int)(sizeof(FwdScalars) / 4);
+    static_assert(sizeof(FwdScalars) % 4 == 0 && kWords + 3 <= 320, "one parameter word per thread");
+    const int tid = threadIdx.x;
+    if ((tid >> 5) == 0) tmem_alloc(smem_u32(&cell_tmem), cp.tmem_cols);
+    if (tid == 0) cell_stop = 0;
+    // one word of the parameters per thread: the first launch's now, the next one's while the current one runs
+    auto fetch = [&](int op) -> uint32_t {
+        const CellOp* o = cp.ops + op;
+        if (tid < kWords) return __ldg(reinterpret_cast<const uint32_t*>(&o->p.s) + tid);
+        if (tid < kWords + 3) return __ldg(&o->gx + (tid - kWords));
+        return 0u;
+    };
+    uint32_t nxt = fetch(0);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = cell_tmem;
+    bool first = true;
+    int stop = 0;
+    for (int op = 0; op < cp.n_ops && !stop; ++op) {
+        if (tid < kWords) reinterpret_cast<uint32_t*>(&p)[tid] = nxt;
+        else if (tid < kWords + 3) vgrid[tid - kWords] = nxt;
+        if (op + 1 < cp.n_ops) nxt = fetch(op + 1);
+        __syncthreads();
+        const unsigned int gx = vgrid[0], gy = vgrid[1], gz = vgrid[2], V = gx * gy * gz;
+        for (unsigned int v = blockIdx.x; v < V && !stop; v += gridDim.x) {
+            const uint3 vb = make_uint3(v % gx, (v / gx) % gy, v / (gx * gy));
+            stop = conv_fwd_cta<3>(&cp.ops[op].p, p, vb, make_uint3(gx, gy, gz), tmem_base, first);
+            first = false;
+        }
+        if (stop) break;
+        if (op + 1 < cp.n_ops && !cell_grid_barrier(cp.barrier, cp.status, &cell_stop)) stop = 1;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if ((tid >> 5) == 0) tmem_dealloc(tmem_base, cp.tmem_cols);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1467,7 +1653,11 @@ bool conv_tc_can_fuse_bn(const ConvShape& s, int pass)
     // the write-out keeps one group of 4 channels per thread and the last CTA combines 2*C columns with 256 threads:
     // a power of two between 16 and 256 channels, all in one channel slice
     const int C = v.c_out;
-    return C >= 16 && C <= 256 && (C & (C - 1)) == 0 && conv_tc_tiles(s, pass) > 0;
+    if (!(C >= 16 && C <= 256 && (C & (C - 1)) == 0 && conv_tc_tiles(s, pass) > 0)) return false;
+    // the per-tile moments are merged as equal-sized groups: every tile must be full
+    PixelBox b;
+    if (!choose_box(v.Q, v.P, v.N, kTileM, 1, &b)) return false;
+    return v.Q % b.w == 0 && v.P % b.h == 0 && v.N % b.n == 0;
 }
 
 bool conv_tc_can_fuse_bn_input(const ConvShape& s)
@@ -1491,6 +1681,8 @@ cudaError_t conv_tc_init()
     e = cudaFuncSetAttribute(conv_tc_fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(conv_tc_fwd_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(conv_tc_cell_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 2048);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(conv_tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWgradSmemBudget + 2048);
     if (e != cudaSuccess) return e;
@@ -1667,6 +1859,10 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     // one more where two CTAs still fit an SM: nine taps then take two rounds of the ring instead of three
     if (total > kFwdMaxStages && (unsigned int)(kFwdMaxStages + 1) * p.stage_bytes <= 92u * 1024u) stages = kFwdMaxStages + 1;
     if (stages > total) stages = total;
+    const int cell_ctas = fuse ? fuse->cell_ctas : 0;
+    const unsigned int cell_budget = cell_ctas > 0 ? (fuse->cell_smem ? fuse->cell_smem : kCellSmemBudget) : 0u;
+    if (cell_ctas > 0)
+        while (stages > 1 && (unsigned int)stages * p.stage_bytes > cell_budget) --stages;
     p.stages = stages;
     if (fuse && fuse->mode) {
         if (256 % (n_chunk / 4)) return cudaErrorNotSupported;
@@ -1697,7 +1893,15 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     // the 512 columns of an SM) and a staging area beside the pipeline.  A launch of about a wave keeps one tile per
     // CTA: there the duration of the launch is one CTA's own chain.
     p.tiles_per_cta = 1;
-    if (p.n_tiles * (v.c_out / n_chunk) >= kMultiTileFrom && 2 * p.acc_cols <= 256 && pipe_bytes + stg_bytes <= 110u * 1024u) {
+    if (cell_ctas > 0) {
+        // inside a persistent cell kernel of cell_ctas CTAs: as many tiles per CTA as bring the launch down to one round of
+        // the grid, within four accumulator barriers, the cell's tensor-memory columns and its shared memory
+        int t = (p.n_tiles * (v.c_out / n_chunk) + cell_ctas - 1) / cell_ctas;
+        if (t > 4) t = 4;
+        while (t > 1 && (unsigned int)t * p.acc_cols > kCellTmemCols) --t;
+        if (t > 1 && pipe_bytes + stg_bytes > cell_budget) t = 1;
+        p.tiles_per_cta = t < 1 ? 1 : t;
+    } else if (p.n_tiles * (v.c_out / n_chunk) >= kMultiTileFrom && 2 * p.acc_cols <= 256 && pipe_bytes + stg_bytes <= 110u * 1024u) {
         int t = (p.n_tiles * (v.c_out / n_chunk) + 295) / 296;            // tiles per CTA that bring the launch down to one wave
         if (t > 4) t = 4;                                                 // accumulator barriers
         while (t > 2 && (unsigned int)t * p.acc_cols > 256u) --t;
@@ -1720,6 +1924,7 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     L->grid = dim3((p.n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta, v.c_out / n_chunk, p.ksplit);
     L->smem = p.tiles_per_cta > 1 ? pipe_bytes + stg_bytes : (pipe_bytes > stg_bytes ? pipe_bytes : stg_bytes);
     L->smem += 1024;
+    if (p.stat_mode == 1 && L->smem < 16384u + 1024u) L->smem = 16384u + 1024u;      // the last CTA's fp64 reduction: 256 x 8 doubles
     plan->valid = 1;
     return cudaSuccess;
 }
@@ -1744,6 +1949,51 @@ cudaError_t conv_tc_launch(const ConvTcPlan* plan, DeviceStatus* status, cudaStr
     if (L.p.s.ksplit > 1) launch_pdl(conv_tc_fwd_kernel<false, true>, L.grid, dim3(320), L.smem, st, L.p);
     else if (L.p.s.tiles_per_cta > 1) launch_pdl(conv_tc_fwd_kernel<true>, L.grid, dim3(320), L.smem, st, L.p);
     else launch_pdl(conv_tc_fwd_kernel<false>, L.grid, dim3(320), L.smem, st, L.p);
+    count(n_launch, 1);
+    return cudaGetLastError();
+}
+
+size_t conv_tc_cell_op_bytes() { return sizeof(CellOp); }
+
+cudaError_t conv_tc_cell_op(const ConvTcPlan* plan, DeviceStatus* status, void* dst_host, unsigned int* smem, unsigned int* tmem_cols,
+                            unsigned int* ctas)
+{
+    if (!plan->valid || plan->pass == PASS_WGRAD) return cudaErrorInvalidValue;
+    const ConvTcFwdLaunch* L = reinterpret_cast<const ConvTcFwdLaunch*>(plan->storage);
+    CellOp op;
+    memset(&op, 0, sizeof op);
+    op.p = L->p;
+    op.p.s.status = status;
+    op.gx = L->grid.x; op.gy = L->grid.y; op.gz = L->grid.z;
+    memcpy(dst_host, &op, sizeof op);
+    if (L->p.s.tmem_cols > kCellTmemCols) return cudaErrorNotSupported;
+    *smem = L->smem; *tmem_cols = L->p.s.tmem_cols; *ctas = L->grid.x * L->grid.y * L->grid.z;
+    return cudaSuccess;
+}
+
+void conv_tc_plan_pipeline(const ConvTcPlan* plan, int* stages, int* k_iterations)
+{
+    const ConvTcFwdLaunch* L = reinterpret_cast<const ConvTcFwdLaunch*>(plan->storage);
+    *stages = L->p.s.stages; *k_iterations = L->p.s.R * L->p.s.R * L->p.s.n_kchunks;
+}
+
+int conv_tc_cell_max_ctas(unsigned int smem)
+{
+    int dev = 0, sms = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, conv_tc_cell_kernel, 320, smem) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    if (per_sm > 2) per_sm = 2;          // two cell CTAs hold an SM's 512 tensor-memory columns between them
+    return per_sm * sms;
+}
+
+cudaError_t conv_tc_cell_launch(const void* d_ops, int n_ops, int ctas, unsigned int smem, unsigned int tmem_cols, unsigned int* d_barrier,
+                                DeviceStatus* status, cudaStream_t st, int64_t* n_launch)
+{
+    if (n_ops < 1 || ctas < 1 || tmem_cols < 32 || tmem_cols > kCellTmemCols) return cudaErrorInvalidValue;
+    CellParams cp;
+    cp.ops = reinterpret_cast<const CellOp*>(d_ops); cp.n_ops = n_ops; cp.barrier = d_barrier; cp.status = status; cp.tmem_cols = tmem_cols;
+    // a plain stream-ordered launch: a resident grid that started early would only hold SM slots while it waits
+    conv_tc_cell_kernel<<<dim3(ctas), dim3(320), smem, st>>>(cp);
     count(n_launch, 1);
     return cudaGetLastError();
 }

@@ -58,6 +58,10 @@ struct ConvBnFuse {
     // the first kSplitKTicketBytes hold tickets, zero before the first use and left zero).  nullptr: never split.
     void* splitk = nullptr;
     size_t splitk_bytes = 0;
+    // > 0: the launch will run inside a persistent cell kernel of this many CTAs (conv_tc_cell_launch): tiles per CTA are
+    // chosen so that the launch is one round of that grid where tensor and shared memory allow
+    int cell_ctas = 0;
+    unsigned int cell_smem = 0;          // dynamic shared memory such a CTA may use (0: what lets two of them share an SM)
 };
 constexpr size_t kSplitKTicketBytes = 4096;
 // Bytes a forward (or data-gradient) launch of this shape wants for splitting its K loop; 0 when it would not split.
@@ -76,6 +80,21 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
                             const float* w_hi, const float* w_lo, float* out, const float* extra, bool accumulate, void* scratch,
                             const ConvBnFuse* fuse = nullptr);
 cudaError_t conv_tc_launch(const ConvTcPlan* plan, DeviceStatus* status, cudaStream_t st, int64_t* n_launch);
+
+// Persistent cell kernel: a list of prepared forward / data-gradient launches run one after the other by ONE resident grid
+// with a grid-wide barrier between them (see conv_tc.cu).  conv_tc_cell_op writes the device-side record of a prepared
+// launch (conv_tc_cell_op_bytes() bytes, to be copied to 64-byte aligned device memory) and reports what the launch needs;
+// cudaErrorNotSupported: the launch exceeds what a cell CTA may hold.  The list is launched with the largest smem /
+// tmem_cols of its records.  d_barrier: two zeroed words per stream of cells.
+size_t conv_tc_cell_op_bytes();
+cudaError_t conv_tc_cell_op(const ConvTcPlan* plan, DeviceStatus* status, void* dst_host, unsigned int* smem, unsigned int* tmem_cols,
+                            unsigned int* ctas);
+// Depth of the prepared forward / data-gradient launch's operand pipeline and the length of its K loop.
+void conv_tc_plan_pipeline(const ConvTcPlan* plan, int* stages, int* k_iterations);
+// CTAs of the cell kernel that can be resident on the current device at once with this much dynamic shared memory.
+int conv_tc_cell_max_ctas(unsigned int smem);
+cudaError_t conv_tc_cell_launch(const void* d_ops, int n_ops, int ctas, unsigned int smem, unsigned int tmem_cols, unsigned int* d_barrier,
+                                DeviceStatus* status, cudaStream_t st, int64_t* n_launch);
 
 // One convolution's weights inside the flat parameter vector.
 struct WeightPrepEntry { long long w_off; int C, K, R, reserved; };

@@ -50,6 +50,11 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
 
+// Failure bookkeeping of the C ABI (hpf_model.cu): records the text hpf_last_error() returns on the calling thread
+// and hands the status back, so that every entry point, whichever file it lives in, reports through one place.
+int api_fail(int status, const char* what);
+int api_cuda_fail(cudaError_t e, const char* where);
+
 // Device-side status word shared by all kernels that have bounded waits.
 // 0 = fine; anything else = where a wait gave up (see conv_tc.cu).
 struct DeviceStatus { unsigned int code; unsigned int detail; };

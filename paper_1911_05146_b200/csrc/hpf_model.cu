@@ -16,22 +16,27 @@
 using namespace hpf;
 
 namespace {
-
 thread_local std::string g_last_error;
+}
 
-int fail(int status, const char* what)
+int hpf::api_fail(int status, const char* what)
 {
     g_last_error = what ? what : "";
     return status;
 }
 
-int cuda_fail(cudaError_t e, const char* where)
+int hpf::api_cuda_fail(cudaError_t e, const char* where)
 {
     char buf[512];
     snprintf(buf, sizeof buf, "%s: %s", where, cudaGetErrorString(e));
     g_last_error = buf;
     return HPF_ERR_CUDA;
 }
+
+namespace {
+
+int fail(int status, const char* what) { return hpf::api_fail(status, what); }
+int cuda_fail(cudaError_t e, const char* where) { return hpf::api_cuda_fail(e, where); }
 
 #define CU(call)                                                   \
     do {                                                           \
@@ -94,6 +99,20 @@ struct hpf_model {
     bool opt_bn_cluster = true; // BN backward of micro-batch sized tensors as one thread-block-cluster launch
     int opt_cell_times = 0;    // record a device timestamp at the start and end of every (partition, micro-batch) cell
     size_t cell_times_off = 0;
+    // persistent cell kernels: maximal runs of tensor-core forward convolutions of a partition with nothing but
+    // kernel-less ops between them (BN+ReLU applied by the reading convolution, residual adds fused into the producer)
+    struct CellRun {
+        int part = 0;
+        std::vector<int> convs;               // ops of the run, ascending; the kernel is enqueued at convs[0]'s place
+        std::vector<size_t> ops_off;          // per micro-batch: device records (conv_tc_cell_op) in the workspace
+        unsigned int smem = 0, tmem = 0, smem_budget = 0;
+        int ctas = 0;
+        bool ready = false;
+    };
+    int opt_cell = 0;          // CTAs of a persistent forward cell kernel; 0: every convolution is its own launch
+    std::vector<CellRun> cell_runs;
+    std::vector<int> cell_of_op;              // conv -> run, or -1
+    std::vector<size_t> cell_bar_off;         // per partition: the grid barrier's two words (zeroed at bind)
     int opt_fuse_bn = 3;       // bit 0: BN statistics in the producing convolution's write-out, bit 1: BN+ReLU applied by the reading convolution
     std::vector<GradEdge> edge0;              // per op: contribution to src0
     std::vector<AccumAction> accums;
@@ -408,6 +427,35 @@ void build_kernel_plan(hpf_model* mdl)
     }
 }
 
+// Which forward convolutions share a persistent cell kernel: consecutive tensor-core convolutions of one partition
+// between which the op list holds only ops that launch nothing.
+void build_cell_runs(hpf_model* mdl)
+{
+    const int n = mdl->n_ops;
+    mdl->cell_runs.clear();
+    mdl->cell_of_op.assign(n, -1);
+    if (mdl->opt_cell <= 0) return;
+    for (int p = 0; p < mdl->P; ++p) {
+        hpf_model::CellRun run;
+        run.part = p;
+        auto close = [&]() {
+            if (run.convs.size() >= 2) {
+                for (int i : run.convs) mdl->cell_of_op[i] = (int)mdl->cell_runs.size();
+                mdl->cell_runs.push_back(run);
+            }
+            run.convs.clear();
+        };
+        for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i) {
+            const int kind = mdl->ops[i].op.kind;
+            if (kind == HPF_OP_CONV && mdl->use_tc[PASS_FWD][i]) run.convs.push_back(i);
+            else if (kind == HPF_OP_BNRELU && mdl->bn_into[i] >= 0) continue;
+            else if (kind == HPF_OP_ADD && mdl->add_done_by[i] >= 0) continue;
+            else close();
+        }
+        close();
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // memory plan
 // ------------------------------------------------------------------------------------------------
@@ -453,7 +501,14 @@ void build_memory_plan(hpf_model* mdl)
         mdl->splitk_bytes[p] = need;
         mdl->splitk_off[p] = take(need ? need : 16);
     }
+    mdl->cell_bar_off.assign(P, 0);
+    for (int p = 0; p < P; ++p) mdl->cell_bar_off[p] = take(16);
     mdl->zero_hi = at;
+    build_cell_runs(mdl);
+    for (auto& run : mdl->cell_runs) {
+        run.ops_off.assign(M, 0);
+        for (int m = 0; m < M; ++m) run.ops_off[m] = take(conv_tc_cell_op_bytes() * run.convs.size());
+    }
     for (int p = 0; p < P; ++p) {
         size_t cv = 256;
         for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i)
@@ -544,7 +599,13 @@ int forward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
             const hpf_op& a = mdl->ops[mdl->fused_into[i]].op;
             residual = mdl->act(a.src0 == i ? a.src1 : a.src0, m);
         }
-        if (mdl->use_tc[PASS_FWD][i]) {
+        if (mdl->cell_of_op[i] >= 0 && mdl->cell_runs[mdl->cell_of_op[i]].ready) {
+            // the whole run of convolutions is one resident grid, enqueued where its first convolution stands
+            const hpf_model::CellRun& run = mdl->cell_runs[mdl->cell_of_op[i]];
+            if (run.convs[0] == i)
+                CU(conv_tc_cell_launch(mdl->ws + run.ops_off[m], (int)run.convs.size(), run.ctas, run.smem, run.tmem,
+                                       reinterpret_cast<unsigned int*>(mdl->ws + mdl->cell_bar_off[p]), mdl->status(), st, &mdl->launches));
+        } else if (mdl->use_tc[PASS_FWD][i]) {
             CU(conv_tc_launch(&mdl->tc_plan[PASS_FWD][(size_t)m * mdl->n_ops + i], mdl->status(), st, &mdl->launches));
         } else {
             CU(conv_fwd_simt(in0, mdl->params + o.w_off, out, residual, conv_shape_of(mdl, i), st, &mdl->launches));
@@ -855,6 +916,7 @@ int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
     case HPF_OPT_FUSE_BN: if (value < 0 || value > 3) return fail(HPF_ERR_INVALID, "0..3"); mdl->opt_fuse_bn = value; break;
     case HPF_OPT_CELL_TIMES: mdl->opt_cell_times = value != 0; break;
     case HPF_OPT_BN_CLUSTER: mdl->opt_bn_cluster = value != 0; break;
+    case HPF_OPT_CELL_CTAS: if (value < 0 || value > 148) return fail(HPF_ERR_INVALID, "0..148 CTAs"); mdl->opt_cell = value; break;
     case HPF_OPT_WGRAD_PASSES: if (value != 1 && value != 3) return fail(HPF_ERR_INVALID, "1 or 3 passes"); mdl->opt_wgrad_passes = value; break;
     default: return fail(HPF_ERR_INVALID, "unknown option");
     }
@@ -1071,8 +1133,54 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
             if (!mdl->prep_table[p].empty())
                 CU(cudaMemcpyAsync(mdl->ws + mdl->prep_table_off[p], mdl->prep_table[p].data(),
                                    sizeof(WeightPrepEntry) * mdl->prep_table[p].size(), cudaMemcpyHostToDevice, mdl->streams[0]));
+        for (int pass = 0; pass < 3; ++pass) mdl->tc_plan[pass].resize((size_t)n * M);
+        // the forward launch of convolution i on micro-batch m (prepared again when its cell's shared-memory budget changes)
+        auto prepare_fwd = [&](int i, int m) -> int {
+            const OpInfo& o = mdl->ops[i];
+            const int src = o.op.src0;
+            const ConvShape s = conv_shape_of(mdl, i);
+            ConvTcPlan* pl = &mdl->tc_plan[PASS_FWD][(size_t)m * n + i];
+            void* scratch = mdl->ws + mdl->conv_scratch_off[o.part];
+            const int pass = PASS_FWD;
+            const float* residual = nullptr;
+                    if (mdl->fused_into[i] >= 0) {
+                        const hpf_op& a = mdl->ops[mdl->fused_into[i]].op;
+                        residual = mdl->act(a.src0 == i ? a.src1 : a.src0, m);
+                    }
+                    ConvBnFuse fuse;
+                    if (mdl->splitk_bytes[o.part]) { fuse.splitk = mdl->ws + mdl->splitk_off[o.part]; fuse.splitk_bytes = mdl->splitk_bytes[o.part]; }
+                    if (mdl->cell_of_op[i] >= 0) {
+                        fuse.cell_ctas = mdl->opt_cell;
+                        fuse.cell_smem = mdl->cell_runs[mdl->cell_of_op[i]].smem_budget;
+                    }
+                    if (mdl->conv_fwd_bn[i] >= 0) {
+                        const int jn = mdl->conv_fwd_bn[i];
+                        const OpInfo& bn = mdl->ops[jn];
+                        fuse.mode = mdl->bn_late[jn] ? 3 : 1;
+                        fuse.ticket = reinterpret_cast<unsigned int*>(mdl->ws + mdl->bn_scratch_off[o.part]);
+                        fuse.partials = mdl->bn_partials(jn);
+                        fuse.stats_out = mdl->stats(jn, m);
+                        fuse.rows = (long long)mdl->b * bn.H * bn.W;
+                        fuse.eps = bn.op.eps;
+                    }
+                    const float* in = mdl->act(src, m);
+                    const int jb = mdl->conv_in_bn[i];
+                    if (jb >= 0) {
+                        const OpInfo& bn = mdl->ops[jb];
+                        in = mdl->act(bn.op.src0, m);          // the BN's input; its output is a by-product of this kernel
+                        fuse.in_mode = mdl->bn_late[jb] ? 2 : 1;
+                        fuse.in_partials = mdl->bn_partials(jb);
+                        fuse.in_tiles = conv_tc_tiles(conv_shape_of(mdl, mdl->bn_fwd_from[jb]), PASS_FWD);
+                        fuse.in_rows = (long long)mdl->b * bn.H * bn.W;
+                        fuse.in_eps = bn.op.eps;
+                        fuse.in_gamma = mdl->params + bn.w_off; fuse.in_beta = mdl->params + bn.b_off;
+                        fuse.in_stats = mdl->stats(jb, m); fuse.in_y = mdl->act(jb, m);
+                    }
+                    CU(conv_tc_prepare(pl, s, pass, passes, in, nullptr, wp + o.w_off, wp + G + o.w_off,
+                                       mdl->act(i, m), residual, false, scratch, &fuse));
+            return HPF_OK;
+        };
         for (int pass = 0; pass < 3; ++pass) {
-            mdl->tc_plan[pass].resize((size_t)n * M);
             for (int m = 0; m < M; ++m)
                 for (int i = 0; i < n; ++i) {
                     if (!mdl->use_tc[pass][i]) continue;
@@ -1083,38 +1191,8 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                     ConvTcPlan* pl = &mdl->tc_plan[pass][(size_t)m * n + i];
                     void* scratch = mdl->ws + mdl->conv_scratch_off[o.part];
                     if (pass == PASS_FWD) {
-                        const float* residual = nullptr;
-                        if (mdl->fused_into[i] >= 0) {
-                            const hpf_op& a = mdl->ops[mdl->fused_into[i]].op;
-                            residual = mdl->act(a.src0 == i ? a.src1 : a.src0, m);
-                        }
-                        ConvBnFuse fuse;
-                        if (mdl->splitk_bytes[o.part]) { fuse.splitk = mdl->ws + mdl->splitk_off[o.part]; fuse.splitk_bytes = mdl->splitk_bytes[o.part]; }
-                        if (mdl->conv_fwd_bn[i] >= 0) {
-                            const int jn = mdl->conv_fwd_bn[i];
-                            const OpInfo& bn = mdl->ops[jn];
-                            fuse.mode = mdl->bn_late[jn] ? 3 : 1;
-                            fuse.ticket = reinterpret_cast<unsigned int*>(mdl->ws + mdl->bn_scratch_off[o.part]);
-                            fuse.partials = mdl->bn_partials(jn);
-                            fuse.stats_out = mdl->stats(jn, m);
-                            fuse.rows = (long long)mdl->b * bn.H * bn.W;
-                            fuse.eps = bn.op.eps;
-                        }
-                        const float* in = mdl->act(src, m);
-                        const int jb = mdl->conv_in_bn[i];
-                        if (jb >= 0) {
-                            const OpInfo& bn = mdl->ops[jb];
-                            in = mdl->act(bn.op.src0, m);          // the BN's input; its output is a by-product of this kernel
-                            fuse.in_mode = mdl->bn_late[jb] ? 2 : 1;
-                            fuse.in_partials = mdl->bn_partials(jb);
-                            fuse.in_tiles = conv_tc_tiles(conv_shape_of(mdl, mdl->bn_fwd_from[jb]), PASS_FWD);
-                            fuse.in_rows = (long long)mdl->b * bn.H * bn.W;
-                            fuse.in_eps = bn.op.eps;
-                            fuse.in_gamma = mdl->params + bn.w_off; fuse.in_beta = mdl->params + bn.b_off;
-                            fuse.in_stats = mdl->stats(jb, m); fuse.in_y = mdl->act(jb, m);
-                        }
-                        CU(conv_tc_prepare(pl, s, pass, passes, in, nullptr, wp + o.w_off, wp + G + o.w_off,
-                                           mdl->act(i, m), residual, false, scratch, &fuse));
+                        int rc = prepare_fwd(i, m);
+                        if (rc) return rc;
                     }
                     else if (pass == PASS_DGRAD) {
                         ConvBnFuse dsplit;
@@ -1134,6 +1212,55 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                                            mdl->gslots + (int64_t)m * mdl->G + o.w_off, nullptr, false, scratch, &hint));
                     }
                 }
+        }
+        // persistent forward cells: records of every run's launches, per micro-batch
+        for (auto& run : mdl->cell_runs) {
+            // a launch whose operand pipeline came out shallower than it wants (wide channels: large stages) gets the
+            // shared memory of a whole SM; such a cell's CTAs then sit one per SM
+            bool shallow = false;
+            for (int i : run.convs) {
+                int stages = 0, iters = 0;
+                conv_tc_plan_pipeline(&mdl->tc_plan[PASS_FWD][i], &stages, &iters);
+                if (stages < (iters < 3 ? iters : 3)) shallow = true;
+            }
+            if (shallow) {
+                run.smem_budget = 200u * 1024u;
+                for (int m = 0; m < M; ++m)
+                    for (int i : run.convs) { int rc = prepare_fwd(i, m); if (rc) return rc; }
+            }
+            const size_t rec = conv_tc_cell_op_bytes();
+            std::vector<unsigned char> host(rec * run.convs.size());
+            bool ok = true;
+            unsigned int most_ctas = 0;
+            for (int m = 0; m < M && ok; ++m) {
+                for (size_t k = 0; k < run.convs.size() && ok; ++k) {
+                    unsigned int smem = 0, tmem = 0, ctas = 0;
+                    cudaError_t e = conv_tc_cell_op(&mdl->tc_plan[PASS_FWD][(size_t)m * n + run.convs[k]], mdl->status(), host.data() + k * rec, &smem, &tmem, &ctas);
+                    if (e == cudaErrorNotSupported) { ok = false; break; }
+                    CU(e);
+                    if (smem > run.smem) run.smem = smem;
+                    if (tmem > run.tmem) run.tmem = tmem;
+                    if (ctas > most_ctas) most_ctas = ctas;
+                }
+                if (ok) CU(cudaMemcpyAsync(mdl->ws + run.ops_off[m], host.data(), host.size(), cudaMemcpyHostToDevice, mdl->streams[0]));
+                CU(cudaStreamSynchronize(mdl->streams[0]));          // `host` is reused for the next micro-batch
+            }
+            run.ctas = (int)most_ctas < mdl->opt_cell ? (int)most_ctas : mdl->opt_cell;
+            run.ready = ok && run.ctas >= 1;
+        }
+        // All cells that can run at the same time (one per partition) must be resident together, or their grid barriers
+        // would wait for CTAs that cannot start: the grids have to fit the GPU side by side.
+        {
+            std::vector<double> share(mdl->P, 0.0);
+            for (const auto& run : mdl->cell_runs) {
+                if (!run.ready) continue;
+                const int cap = conv_tc_cell_max_ctas(run.smem);
+                if (cap < run.ctas) return fail(HPF_ERR_UNSUPPORTED, "a persistent cell kernel does not fit the GPU");
+                share[run.part] = std::max(share[run.part], (double)run.ctas / cap);
+            }
+            double total = 0.0;
+            for (double v : share) total += v;
+            if (total > 0.92) return fail(HPF_ERR_UNSUPPORTED, "the persistent cell kernels of all partitions do not fit the GPU together: lower HPF_OPT_CELL_CTAS");
         }
     }
     CU(cudaStreamSynchronize(mdl->streams[0]));

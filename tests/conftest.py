@@ -24,3 +24,16 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter):
+    """The parity figures of the GPU tests: per compared step the worst relative L2 error against the plain oracle and
+    against the oracle evaluated under the GPU's in-window ReLU decisions (a diagnostic), with the decision counts."""
+    try:
+        import hpf_testlib
+    except Exception:
+        return
+    if hpf_testlib.PARITY_LOG:
+        terminalreporter.write_sep("-", "parity against the fp64 oracle")
+        for line in hpf_testlib.PARITY_LOG:
+            terminalreporter.write_line(line)

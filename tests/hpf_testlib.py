@@ -7,13 +7,21 @@ import workloads as wl
 
 TOL_TENSOR = 1e-2     # relative L2 per activation and gradient tensor
 TOL_LOSS = 1e-3       # relative, on the loss
-# ReLU decisions: the gradient is a discontinuous function of the forward values, so both sides must take
-# the decision z > 0 on the same side wherever the forward tolerance leaves it open.  The oracle keeps its own
-# decision where |z| >= TAU*|gamma| (a GPU disagreement there fails the test) and evaluates the gradient under
-# the GPU's decision inside that window.  The window follows the forward accuracy of the convolution path:
-# fp32-class (three-pass TF32, CUDA cores) or one TF32 pass.
-TAU = 2e-3
+# The judge of every comparison is the PLAIN oracle: it takes nothing from the GPU.  The gradient is a discontinuous
+# function of the forward values (the derivative of ReLU is a step), so an implementation whose pre-activation z
+# differs from the oracle's by a rounding error takes the other branch where |z| is below that error, and a handful
+# of such flips per tensor can add up, through a thousand layers, to more than the tolerance.  Only for a backward
+# tensor that misses the tolerance against the plain oracle is a second, diagnostic oracle run consulted, in which
+# the oracle evaluates its gradient under the decisions z > 0 the GPU took - and only inside the window
+# |z| < TAU*|gamma| (a GPU decision that differs outside it fails the test), and only if those decisions are a
+# vanishing fraction of all decisions.  The window follows the forward accuracy of the convolution path: measured
+# max |z| at a differing decision on ResNet-1001 is 3e-5 for the fp32-class paths (three-pass TF32, CUDA cores).
+TAU = 1e-4
 TAU_ONE_PASS = 0.02
+MAX_DECISION_FRACTION = 2e-5          # of all ReLU decisions of the micro-batch (fp32-class paths)
+MAX_DECISION_FRACTION_ONE_PASS = 5e-3
+
+PARITY_LOG = []       # one line per compared step; the test session prints them in its summary
 
 
 def rel_l2(a, ref):
@@ -91,12 +99,88 @@ def seeded(ops, in_hwc, B, seed=0, bn_jitter=0.0):
 
 
 def matched_oracle(bd, m, theta, x, labels, cuts=None, want=None, tau=TAU):
-    """The oracle's micro-batch m with the GPU's in-window ReLU decisions; fails on any decision the
-    forward tolerance does not leave open."""
+    """DIAGNOSTIC: the oracle's micro-batch m evaluated under the GPU's in-window ReLU decisions; fails on any
+    decision the forward tolerance does not leave open.  Never the first judge of a comparison (see compare_microbatch)."""
     from oracle import reference as ora
     b = bd.B // bd.M
     dec = {i: (bd.tensor(i, m) > 0).astype(np.uint8) for i, o in enumerate(bd.ops) if o.kind in (wl.BNRELU, wl.RELU)}
     r = ora.microbatch(bd.ops, bd.in_hwc, theta, x[m * b:(m + 1) * b], labels[m * b:(m + 1) * b], cuts=cuts, want=want,
                        decisions=dec, tau=tau)
     assert r["decision_violations"] == 0, r["decision_violations"]
+    r["decisions_total"] = int(sum(d.size for d in dec.values()))
     return r
+
+
+def _tensor_errors(bd, m, slots, offs, r, tensors):
+    """rel-L2 of every stored activation, every activation gradient and every parameter-gradient tensor of
+    micro-batch m against oracle result r."""
+    err = {}
+    if tensors:
+        for i in range(len(bd.ops)):
+            a = bd.tensor_or_none(i, m)          # None: a convolution whose output lives only inside the fused residual add
+            if a is not None:
+                err[("act", i)] = rel_l2(a, r["act"][i])
+            err[("dact", i)] = rel_l2(bd.tensor(i, m, grad=True), r["dact"][i])
+    for i, (w_off, w_cnt, b_off, b_cnt) in enumerate(offs):
+        for which, off, cnt in (("w", w_off, w_cnt), ("b", b_off, b_cnt)):
+            if cnt:
+                err[("g", i, which)] = rel_l2(slots[m, off:off + cnt], r["g"][off:off + cnt])
+    return err
+
+
+def compare_microbatch(bd, m, theta, x, labels, slots, offs, loss_m, cuts=None, tau=TAU, max_fraction=MAX_DECISION_FRACTION,
+                       tensors=True, diagnostic=True, skip=()):
+    """Micro-batch m of the GPU step against the oracle.
+
+    1. The plain oracle (no input from the GPU) judges the loss, every activation, and every gradient tensor.
+    `skip`: keys of tensors left out (a gradient that is zero analytically has no relative error to speak of).
+    2. A gradient tensor beyond the tolerance there is named, and must then hold the tolerance against the oracle
+       evaluated under the GPU's in-window ReLU decisions, with no decision outside the window and at most
+       max(8, max_fraction * decisions) decisions taken from the GPU.
+    Returns the worst figures of both comparisons (the second one is also run when nothing failed, as a diagnostic,
+    unless diagnostic=False)."""
+    from oracle import reference as ora
+    b = bd.B // bd.M
+    plain = ora.microbatch(bd.ops, bd.in_hwc, theta, x[m * b:(m + 1) * b], labels[m * b:(m + 1) * b], cuts=cuts,
+                           want=None if tensors else [])
+    assert abs(loss_m - plain["loss"]) <= TOL_LOSS * abs(plain["loss"]), ("loss", m, loss_m, plain["loss"])
+    e_plain = {k: e for k, e in _tensor_errors(bd, m, slots, offs, plain, tensors).items() if k not in skip}
+    for k, e in e_plain.items():
+        if k[0] == "act":
+            assert e <= TOL_TENSOR, (k, m, e)          # forward values are continuous: the plain oracle alone decides
+    over = {k: e for k, e in e_plain.items() if k[0] != "act" and not e <= TOL_TENSOR}
+    out = {"m": m, "plain": {kind: max([e for k, e in e_plain.items() if k[0] == kind] or [0.0]) for kind in ("act", "dact", "g")},
+           "over": over, "matched": None, "decisions_used": None, "decisions_total": None, "plain_result": plain}
+    if over or diagnostic:
+        r = matched_oracle(bd, m, theta, x, labels, cuts=cuts, want=None if tensors else [], tau=tau)
+        e_m = _tensor_errors(bd, m, slots, offs, r, tensors)
+        out["matched"] = {kind: max([e for k, e in e_m.items() if k[0] == kind] or [0.0]) for kind in ("act", "dact", "g")}
+        out["decisions_used"], out["decisions_total"] = int(r["decisions_used"]), r["decisions_total"]
+        out["matched_result"] = r
+        for k in over:
+            assert e_m[k] <= TOL_TENSOR, ("beyond the tolerance against the plain oracle AND under matched decisions", k, m, over[k], e_m[k])
+        if over:
+            allowed = max(8, int(max_fraction * r["decisions_total"]))
+            assert r["decisions_used"] <= allowed, ("too many ReLU decisions taken from the GPU", r["decisions_used"], allowed)
+    return out
+
+
+def log_parity(name, results):
+    """One summary line for the comparisons of a test (printed at the end of the test session)."""
+    worst_p = {k: max(r["plain"][k] for r in results) for k in ("act", "dact", "g")}
+    have_m = [r for r in results if r["matched"] is not None]
+    worst_m = {k: max(r["matched"][k] for r in have_m) for k in ("act", "dact", "g")} if have_m else None
+    over = sorted({k for r in results for k in r["over"]})
+    over_worst = max([e for r in results for e in r["over"].values()] or [0.0])
+    used = sum(r["decisions_used"] or 0 for r in results)
+    total = sum(r["decisions_total"] or 0 for r in results)
+    line = ("%s: micro-batches %s | plain oracle worst rel-L2 act %.2e dact %.2e g %.2e | " %
+            (name, [r["m"] for r in results], worst_p["act"], worst_p["dact"], worst_p["g"]))
+    if worst_m:
+        line += "GPU-decision oracle (diagnostic) worst dact %.2e g %.2e, decisions_used %d of %d | " % (worst_m["dact"], worst_m["g"], used, total)
+    line += ("every tensor within %.0e of the plain oracle" % TOL_TENSOR) if not over else \
+            ("%d gradient tensors beyond %.0e against the plain oracle (worst %.2e, first %s): judged under GPU decisions" %
+             (len(over), TOL_TENSOR, over_worst, over[:4]))
+    PARITY_LOG.append(line)
+    print(line)
+    return line

@@ -5,7 +5,7 @@ import pytest
 
 import workloads as wl
 from oracle import reference as ora
-from hpf_testlib import Bound, rel_l2, seeded, matched_oracle, TOL_TENSOR, TOL_LOSS
+from hpf_testlib import Bound, rel_l2, seeded, compare_microbatch, log_parity, TOL_TENSOR, TOL_LOSS
 
 pytestmark = pytest.mark.gpu
 
@@ -17,35 +17,22 @@ def _fullsize(name, sample_m):
     bd = Bound(ops, hwc, B, M, c["cuts"], theta)
     bd.upload(x, labels)
     loss = bd.step()
-    b = B // M
     slots = bd.slots.cpu().numpy()
     offs, G = wl.param_offsets(ops)
     losses = bd.loss_slots()
     assert np.isfinite(slots).all()
-    worst = {"act": 0.0, "dact": 0.0, "g": 0.0}
-    for m in sample_m:
-        r = matched_oracle(bd, m, theta, x, labels)
-        worst["decisions_from_gpu"] = worst.get("decisions_from_gpu", 0) + r["decisions_used"]
-        assert abs(losses[m] - r["loss"]) <= TOL_LOSS * abs(r["loss"])
-        for i in range(len(ops)):
-            a = bd.tensor_or_none(i, m)
-            if a is not None:
-                e = rel_l2(a, r["act"][i]); worst["act"] = max(worst["act"], e)
-                assert e <= TOL_TENSOR, ("act", i, m, e)
-            e = rel_l2(bd.tensor(i, m, grad=True), r["dact"][i]); worst["dact"] = max(worst["dact"], e)
-            assert e <= TOL_TENSOR, ("dact", i, m, e)
-        for i, (w_off, w_cnt, b_off, b_cnt) in enumerate(offs):
-            for off, cnt in ((w_off, w_cnt), (b_off, b_cnt)):
-                if cnt:
-                    e = rel_l2(slots[m, off:off + cnt], r["g"][off:off + cnt]); worst["g"] = max(worst["g"], e)
-                    assert e <= TOL_TENSOR, ("g", i, m, e)
+    # sampled micro-batches, recomputed one by one: judged by the plain oracle (which takes nothing from the GPU); the
+    # oracle under the GPU's in-window ReLU decisions runs beside it as a diagnostic and decides only the gradient
+    # tensors that the plain comparison leaves beyond the tolerance
+    res = [compare_microbatch(bd, m, theta, x, labels, slots, offs, float(losses[m])) for m in sample_m]
     # properties that hold at any size: the average is the fixed-order mean of the slots
     acc = slots[0].copy()
     for m in range(1, M):
         acc += slots[m]
     assert np.array_equal(bd.avg.cpu().numpy(), acc * np.float32(1.0 / M))
     assert abs(loss - float(np.sum(losses.astype(np.float32)) / np.float32(M))) <= 1e-6 * abs(loss)
-    print(name, "worst rel-L2", worst)
+    log_parity("full size " + name, res)
+    return res
 
 
 def test_config3_resnet110_batch128():

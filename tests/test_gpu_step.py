@@ -6,13 +6,17 @@ import torch
 import paper_1911_05146_b200 as hpf
 import workloads as wl
 from oracle import reference as ora
-from hpf_testlib import Bound, rel_l2, seeded, matched_oracle, TOL_TENSOR, TOL_LOSS, TAU, TAU_ONE_PASS
+from hpf_testlib import (Bound, rel_l2, seeded, matched_oracle, compare_microbatch, log_parity, TOL_TENSOR, TOL_LOSS, TAU, TAU_ONE_PASS,
+                         MAX_DECISION_FRACTION, MAX_DECISION_FRACTION_ONE_PASS)
 
 pytestmark = pytest.mark.gpu
 
 
-def check_step(ops, in_hwc, B, M, cuts, options=None, seed=0, bn_jitter=0.0, microbatches=None, tensors=True):
+def check_step(ops, in_hwc, B, M, cuts, options=None, seed=0, bn_jitter=0.0, microbatches=None, tensors=True, name=None, edit_theta=None,
+               skip=()):
     x, labels, theta = seeded(ops, in_hwc, B, seed, bn_jitter)
+    if edit_theta is not None:
+        theta = edit_theta(theta)
     bd = Bound(ops, in_hwc, B, M, cuts, theta, options)
     bd.upload(x, labels)
     loss = bd.step()
@@ -28,33 +32,25 @@ def check_step(ops, in_hwc, B, M, cuts, options=None, seed=0, bn_jitter=0.0, mic
         acc += slots[m]
     assert np.array_equal(avg, acc * np.float32(1.0 / M))
     offs, G = wl.param_offsets(ops)
-    worst = 0.0
-    used = 0
-    tau = TAU_ONE_PASS if (options or {}).get(hpf.OPT_CONV_PATH) == 2 else TAU
-    mbs = [matched_oracle(bd, m, theta, x, labels, cuts=list(cuts), tau=tau) for m in range(M)]
-    g_avg_ref = ora.grad_average(np.stack([r["g"] for r in mbs]))
+    one_pass = (options or {}).get(hpf.OPT_CONV_PATH) == 2
+    tau = TAU_ONE_PASS if one_pass else TAU
+    frac = MAX_DECISION_FRACTION_ONE_PASS if one_pass else MAX_DECISION_FRACTION
+    losses = bd.loss_slots()
+    want_m = set(range(M) if microbatches is None else microbatches)
+    # every micro-batch: the plain oracle first, the oracle under the GPU's in-window decisions as a diagnostic
+    res = [compare_microbatch(bd, m, theta, x, labels, slots, offs, float(losses[m]), cuts=list(cuts), tau=tau, max_fraction=frac,
+                              tensors=tensors and m in want_m, skip=skip) for m in range(M)]
+    # the averaged gradient against the plain oracle's step; where slots needed the GPU's decisions, against their average
+    need_matched = any(r["over"] for r in res)
+    g_avg_ref = ref["g_avg"] if not need_matched else ora.grad_average(np.stack([r["matched_result"]["g"] for r in res]))
     for i, (w_off, w_cnt, b_off, b_cnt) in enumerate(offs):
-        for off, cnt in ((w_off, w_cnt), (b_off, b_cnt)):
-            if cnt == 0:
-                continue
-            for m in range(M):
-                e = rel_l2(slots[m, off:off + cnt], mbs[m]["g"][off:off + cnt])
-                worst = max(worst, e)
-                assert e <= TOL_TENSOR, ("slot", m, "op", i, e)
-            e = rel_l2(avg[off:off + cnt], g_avg_ref[off:off + cnt])
-            assert e <= TOL_TENSOR, ("avg op", i, e)
-    if tensors:
-        for m in (range(M) if microbatches is None else microbatches):
-            mb = mbs[m]
-            used += mb["decisions_used"]
-            for i in range(len(ops)):
-                a = bd.tensor_or_none(i, m)          # None: a convolution whose output lives only inside the fused residual add
-                if a is not None:
-                    e = rel_l2(a, mb["act"][i]); worst = max(worst, e)
-                    assert e <= TOL_TENSOR, ("act", i, m, e)
-                e = rel_l2(bd.tensor(i, m, grad=True), mb["dact"][i]); worst = max(worst, e)
-                assert e <= TOL_TENSOR, ("dact", i, m, e)
-    print("worst rel-L2 %.3e, in-window ReLU decisions taken from the GPU: %d" % (worst, used))
+        for which, off, cnt in (("w", w_off, w_cnt), ("b", b_off, b_cnt)):
+            if cnt and ("g", i, which) not in skip:
+                e = rel_l2(avg[off:off + cnt], g_avg_ref[off:off + cnt])
+                assert e <= TOL_TENSOR, ("avg op", i, e)
+    import inspect
+    log_parity(name or inspect.stack()[1].function, res)
+    worst = max(max(r["plain"].values()) for r in res)
     return bd, ref, worst
 
 
@@ -123,6 +119,74 @@ def test_large_microbatch_uses_the_multi_tile_convolutions_with_the_bn_fusions()
     check_step(c["ops"], c["in_hwc"], 80, 1, c["cuts"], seed=9, bn_jitter=0.1, microbatches=[0])
 
 
+@pytest.mark.parametrize("fuse_bn", [0, 1, 3])
+def test_bn_statistics_of_channels_whose_mean_dwarfs_their_spread(fuse_bn):
+    """BN shifts of ten and scales of a tenth: the activations a convolution reads are then ten +- 0.1, and its output,
+    the next BN's input, has per-channel means of a hundred and more standard deviations.  The statistics must come out
+    right whether the BN runs its own kernels (0), takes its moments from the producing convolution's write-out (1) or is
+    applied by the reading convolution (3)."""
+    ops = wl.resnet_v2_cifar(1)
+    offs, G = wl.param_offsets(ops)
+
+    def shifted(theta):
+        theta = theta.copy()
+        for i, o in enumerate(ops):
+            if o.kind == wl.BNRELU:
+                w_off, w_cnt, b_off, b_cnt = offs[i]
+                theta[w_off:w_off + w_cnt] *= np.float32(0.1)
+                theta[b_off:b_off + b_cnt] += np.float32(10.0)
+        return theta
+
+    # With shifts this large no activation is ever clipped, so a BN's shift only adds a constant per channel to the
+    # convolution that follows (but for the padding ring of a 3x3 window), which the next BN removes again: its gradient
+    # is zero analytically, or a sum that cancels to almost nothing (both sides compute rounding noise there), and a
+    # relative error of it means nothing.
+    zero_grad = {("g", i, "b") for i, o in enumerate(ops) if o.kind == wl.BNRELU and ops[i + 1].kind == wl.CONV}
+    bd, _, _ = check_step(ops, (32, 32, 3), 8, 2, [9], {hpf.OPT_FUSE_BN: fuse_bn}, seed=21, bn_jitter=0.2, edit_theta=shifted,
+                          name="mean >> sigma, fuse_bn=%d" % fuse_bn, skip=zero_grad)
+    # the premise: some BN input really is that badly centred
+    ratios = []
+    for i, o in enumerate(ops):
+        if o.kind == wl.BNRELU and ops[o.src0].kind == wl.CONV and ops[o.src0].src0 >= 0:
+            t = bd.tensor_or_none(o.src0, 0)
+            if t is not None:
+                t = t.reshape(-1, t.shape[-1]).astype(np.float64)
+                ratios.append(float(np.max(np.abs(t.mean(0)) / t.std(0))))
+    assert max(ratios) > 50, ratios
+
+
+@pytest.mark.parametrize("ctas", [3, 16, 40])
+def test_persistent_forward_cells_give_the_same_bits_as_one_launch_per_convolution(ctas):
+    """Section 5.3's stage as one resident grid: the forward convolutions of a cell run inside ONE persistent kernel that
+    walks the list with grid-wide barriers.  Fewer CTAs than tiles (several rounds and several tiles per CTA), about as many,
+    and more than any launch has; against the oracle, and bit for bit against the step made of single launches."""
+    ops = wl.resnet_v2_cifar(2)
+    cuts = wl.default_cuts(len(ops), 3)
+    bd, _, _ = check_step(ops, (32, 32, 3), 8, 2, cuts, {hpf.OPT_CELL_CTAS: ctas}, seed=12, bn_jitter=0.2, name="persistent cells, %d CTAs" % ctas)
+    x, labels, theta = seeded(ops, (32, 32, 3), 8, 12, 0.2)
+    ref = Bound(ops, (32, 32, 3), 8, 2, cuts, theta, {hpf.OPT_CELL_CTAS: 0})
+    ref.upload(x, labels)
+    loss = ref.step()
+    assert bd.model.launch_count() < ref.model.launch_count()          # the cells replaced launches
+    assert loss == bd.model.loss()
+    assert torch.equal(ref.slots, bd.slots) and torch.equal(ref.avg, bd.avg)
+    for i in range(len(ops)):
+        a, b2 = ref.tensor_or_none(i, 1), bd.tensor_or_none(i, 1)
+        assert (a is None) == (b2 is None)
+        if a is not None:
+            assert np.array_equal(a, b2), i
+
+
+def test_persistent_forward_cells_on_wide_channels_and_repeated_steps():
+    """ImageNet-layout block with 256..1024 channels (stages too large for two CTAs per SM, channel slices) inside cells; the
+    second step must find the grid barrier as the first one left it."""
+    ops = wl.resnet_v2_imagenet(blocks=(2, 1), widths=(128, 256), n_classes=9)
+    bd, _, _ = check_step(ops, (32, 32, 3), 4, 2, [9, 20], {hpf.OPT_CELL_CTAS: 12}, seed=3, bn_jitter=0.2, name="persistent cells, wide channels")
+    s1 = bd.slots.clone()
+    l1 = bd.model.loss()
+    assert bd.step() == l1 and torch.equal(s1, bd.slots)
+
+
 def test_odd_widths_run_on_cuda_cores():
     ops = wl.resnet_v2_cifar(1, widths=(4, 8, 12), n_classes=5)
     bd, _, _ = check_step(ops, (8, 8, 3), 6, 3, [9], seed=1, bn_jitter=0.2)
@@ -170,7 +234,6 @@ def test_second_step_and_new_inputs_reuse_the_model():
     l3 = bd.step()
     ref = ora.step(ops, c["in_hwc"], theta, x2, labels2, c["M"], cuts=c["cuts"])
     assert abs(l3 - ref["loss"]) <= TOL_LOSS * abs(ref["loss"])
-    ref["g_avg"] = ora.grad_average(np.stack([matched_oracle(bd, m, theta, x2, labels2, want=[])["g"] for m in range(c["M"])]))
     assert rel_l2(bd.avg.cpu().numpy(), ref["g_avg"]) <= TOL_TENSOR
     # the host-buffer entry point gives the same numbers
     hx = torch.from_numpy(x2).pin_memory(); hl = torch.from_numpy(labels2).pin_memory()
@@ -207,11 +270,16 @@ def test_messages_across_cuts_match_the_oracle():
     bd.step()
     b = B // M
     for m in range(M):
-        r = matched_oracle(bd, m, theta, x, labels, cuts=cuts)
+        r = ora.microbatch(ops, (32, 32, 3), theta, x[m * b:(m + 1) * b], labels[m * b:(m + 1) * b], cuts=cuts)     # the plain oracle
         for (j, k), msg in r["fwd_msg"].items():
             assert rel_l2(bd.message(j, k, m), msg) <= TOL_TENSOR, ("fwd", j, k, m)
-        for (j, k), msg in r["bwd_msg"].items():
-            assert rel_l2(bd.message(j, k, m, grad=True), msg) <= TOL_TENSOR, ("bwd", j, k, m)
+        over = [(j, k) for (j, k), msg in r["bwd_msg"].items() if not rel_l2(bd.message(j, k, m, grad=True), msg) <= TOL_TENSOR]
+        if over:      # a flipped ReLU decision upstream: those messages are judged under the GPU's in-window decisions
+            rm = matched_oracle(bd, m, theta, x, labels, cuts=cuts)
+            assert rm["decisions_used"] <= 8, rm["decisions_used"]
+            for (j, k) in over:
+                assert rel_l2(bd.message(j, k, m, grad=True), rm["bwd_msg"][(j, k)]) <= TOL_TENSOR, ("bwd", j, k, m)
+        print("micro-batch %d: partial-error messages beyond the tolerance against the plain oracle: %s" % (m, over))
 
 
 def test_state_machine_on_a_bound_model():
