@@ -47,6 +47,51 @@ def peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
+def measure_tf32_peak(torch, seconds=2.0):
+    """Dense TF32 tensor throughput of this GPU, measured in this run: torch.matmul (a library GEMM: a probe for the
+    roofline's denominator, not a product path) on 8192^3 fp32 operands with TF32 allowed; best of 10 single calls
+    (burst: for a kernel timed alone) and back to back for `seconds` (sustained, under the power cap)."""
+    old = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = True
+    try:
+        n = 8192
+        a = torch.randn(n, n, device="cuda"); b = torch.randn(n, n, device="cuda"); c = torch.empty(n, n, device="cuda")
+        for _ in range(3):
+            torch.matmul(a, b, out=c)
+        torch.cuda.synchronize()
+        flop = 2.0 * n ** 3
+        best = 0.0
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); torch.matmul(a, b, out=c); e1.record(); torch.cuda.synchronize()
+            best = max(best, flop / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+        reps = max(10, int(seconds * best * 1e12 / flop))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            torch.matmul(a, b, out=c)
+        e1.record(); torch.cuda.synchronize()
+        sustained = reps * flop / (e0.elapsed_time(e1) * 1e-3) / 1e12
+        del a, b, c
+        return {"burst_tflops": best, "sustained_tflops": sustained, "how": "torch.matmul fp32 operands, TF32 allowed, 8192^3: best of 10 "
+                "(burst) and %d back to back (sustained); measured in this run" % reps}
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = old
+
+
+def dram_traffic_table():
+    """DRAM bytes of the convolution kernel per launch as ncu counted them, from the tracked summary
+    profiles/conv_tc_fwd_dram_traffic.txt: rows `ksize stride c_in c_out H batch read_bytes write_bytes`."""
+    table = {}
+    path = os.path.join(ROOT, "profiles", "conv_tc_fwd_dram_traffic.txt")
+    if os.path.exists(path):
+        for line in open(path):
+            f = line.split("#")[0].split()
+            if len(f) >= 8:
+                table[tuple(int(v) for v in f[:5])] = (int(f[5]), float(f[6]) + float(f[7]))
+    return table
+
+
 # ----------------------------------------------------------------------------------------------------
 # algorithmic byte / flop model of one step (unfused op model: every op reads its inputs and writes
 # its outputs once; conv counted for forward, data gradient and weight gradient)
@@ -230,11 +275,13 @@ def kernel_roofline(torch, hpf, cfg, pk):
     torch.cuda.synchronize()
     sec = e0.elapsed_time(e1) * 1e-3 / (3 * reps)
     achieved = alg / sec / 1e9
+    cap = dram_traffic_table().get((ks, st, ci, co, H))
+    traffic = cap[1] * b / cap[0] if cap else None
     return {"bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"],
-            # dram__bytes_read + dram__bytes_write of this kernel in the ncu captures of the same shape at batch 128
-            # (profiles/conv_tc_fwd_1x1_*_at32_batch128.md: the input is read once, 33.62 MB / 8.47 MB, and the output is
-            # still in L2 when the kernel ends), scaled by the pixels per launch
-            "traffic": {(1, 1, 64, 16, 32): 33.62e6, (1, 1, 16, 64, 32): 8.47e6}.get((ks, st, ci, co, H), 0.0) * b / 128.0 or None,
+            # dram__bytes_read + dram__bytes_write of this kernel in the ncu capture of the same shape (tracked table under
+            # profiles/, captured at a batch whose operands exceed L2), scaled by the pixels per launch: traffic grows in
+            # proportion to the pixels (the input is read once, nothing is re-read); null when no capture covers the shape
+            "traffic": traffic,
             "peak_source": pk["source"],
             "kernel": "conv_tc_fwd_kernel (tcgen05 implicit GEMM, three-pass TF32), %dx%d stride %d, %d->%d channels, %dx%d "
                       "pixels, micro-batch %d; %d rotating operand sets, kernel nodes only, launched with programmatic dependent launch as in the step"
@@ -253,7 +300,8 @@ def conv_sweep(args):
     import paper_1911_05146_b200 as hpf
     torch.cuda.set_device(0)
     pk = peaks()
-    tf32_peak = pk["bf16_tflops"] / 2.0            # dense TF32 = half the measured dense BF16 rate
+    tf32 = measure_tf32_peak(torch)
+    tf32_peak = tf32["burst_tflops"]               # the kernels of the sweep are timed alone: the burst figure
     N, rows_out = 128, []
     dev = "cuda"
     for (ks, st, ci, co, H) in wl.conv_sweep_shapes():
@@ -299,7 +347,8 @@ def conv_sweep(args):
     best = max(r["tflops"] for r in rows_out)
     print(json.dumps({"metric": "conv sweep (configuration 2), batch 128", "unit": "TFLOP/s", "value": best, "n_gpus": 1,
                       "dtype": "tf32", "data": "synthetic", "config": {"workload": "28 bottleneck conv shapes x {fwd, dgrad, wgrad}",
-                      "conv_path": args.conv_path, "tf32_peak_tflops": tf32_peak, "hbm_gbs": pk["hbm_gbs"], "peak_source": pk["source"]},
+                      "conv_path": args.conv_path, "tf32_peak_tflops": tf32_peak, "tf32_peak": tf32,
+                      "tf32_from_bf16_over_2_tflops": pk["bf16_tflops"] / 2.0, "hbm_gbs": pk["hbm_gbs"], "peak_source": pk["source"]},
                       "rows": rows_out}), flush=True)
 
 
@@ -334,6 +383,18 @@ def membound_sweep(args):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) * 1e-3 / (3 * reps)
 
+    # Latency floor of each kernel: the same entry point on a tensor of a few rows of the same width, where nothing but the
+    # launch, the statistics exchange (block reduction, cluster or ticket hand-off) and the dependent second phase is left.
+    floors = {}
+    for C in (16, 64, 128, 256):
+        rows0 = 512
+        x0 = torch.randn(rows0, C, device=dev); y0 = torch.empty_like(x0); d0 = torch.randn_like(x0)
+        g0 = torch.ones(C, device=dev); b0 = torch.zeros(C, device=dev); st0 = torch.empty(2 * C, device=dev)
+        dg0 = torch.empty(C, device=dev); db0 = torch.empty(C, device=dev)
+        sc0 = torch.zeros(hpf.bnrelu_scratch_bytes(rows0, C), dtype=torch.uint8, device=dev)
+        floors[("bnrelu_fwd", C)] = timed(lambda k: hpf.bnrelu_fwd(x0, g0, b0, 1e-5, y0, st0, rows0, C, sc0), 1, 50)
+        floors[("bnrelu_bwd", C)] = timed(lambda k: hpf.bnrelu_bwd(x0, d0, g0, b0, st0, y0, None, 0, dg0, db0, rows0, C, sc0), 1, 50)
+    l2_mb = 126.0
     shapes = [(N, H, C) for N in (128, 16) for (H, C) in ((32, 64), (16, 128), (8, 256), (32, 16))] + [(64, 56, 256)]
     for (N, H, C) in shapes:
         rows = N * H * H
@@ -352,8 +413,19 @@ def membound_sweep(args):
         tc = timed(lambda k: torch.relu_(xs[k]), nset, reps)
         for name, t, bpe in (("bnrelu_fwd", tf, 8.0), ("bnrelu_bwd", tb, 12.0), ("one-pass elementwise (torch.relu_, context)", tc, 8.0)):
             gbs = bpe * rows * C / t / 1e9
-            out.append({"kernel": name, "shape": "N=%d %dx%d C=%d" % (N, H, H, C), "mb": rows * C * 4 / 1e6, "us": t * 1e6,
-                        "gbs": gbs, "frac_hbm": gbs / pk["hbm_gbs"]})
+            row = {"kernel": name, "shape": "N=%d %dx%d C=%d" % (N, H, H, C), "mb": rows * C * 4 / 1e6, "us": t * 1e6,
+                   "gbs": gbs, "frac_hbm": gbs / pk["hbm_gbs"]}
+            if name.startswith("bnrelu"):
+                # beyond L2 the statistics pass and the apply pass both read the input from HBM: 12 B (forward) / 16 B
+                # (backward) per element is what such a tensor has to move, the 8 / 12 B model is unreachable there
+                mb = rows * C * 4 / 1e6
+                bpe2 = bpe + 4.0 if mb > l2_mb else bpe
+                t_hbm = bpe2 * rows * C / (pk["hbm_gbs"] * 1e9)
+                t_lat = floors[(name, C)]
+                row.update({"bytes_per_element_model": bpe2, "frac_hbm_model": bpe2 * rows * C / t / 1e9 / pk["hbm_gbs"],
+                            "latency_floor_us": t_lat * 1e6, "hbm_floor_us": t_hbm * 1e6,
+                            "bound": "latency" if t_lat > t_hbm else "hbm", "frac_of_floor": max(t_lat, t_hbm) / t})
+            out.append(row)
         del xs, dys, outs
     for (M, G) in ((8, 10327706), (4, 60185128)):
         nset = 2
@@ -377,8 +449,10 @@ def main():
     ap.add_argument("--impl", default="hpf", choices=["hpf", "reference"])
     ap.add_argument("--workload", default="r1001", choices=sorted(wl.CONFIGS) + ["conv_sweep", "membound_sweep"])
     ap.add_argument("--no-graph", action="store_true")
-    ap.add_argument("--cuts", default="equal", choices=["balanced", "equal"],
+    ap.add_argument("--cuts", default="equal", choices=["balanced", "equal", "measured"],
                     help="partition cut points: balanced = the library's load balancer on its modelled op costs; "
+                         "measured = the load balancer on per-op costs apportioned from the measured, loaded cell times "
+                         "(tuner.balance_by_measurement; its history, equal cuts first, goes into the line); "
                          "equal = the same number of ops in every partition")
     ap.add_argument("--conv-path", type=int, default=0)
     ap.add_argument("--cell-ctas", type=int, default=-1,
@@ -424,8 +498,16 @@ def main():
     ops, hwc, B, M = cfg["ops"], cfg["in_hwc"], cfg["B"], cfg["M"]
     x, labels, theta = replica_inputs(cfg, rank)          # each replica its own batch, shared parameters
     cuts = cfg["cuts"]
+    balance_history = None
     if args.cuts == "balanced":
         cuts = hpf.balance_cuts(hpf.estimate_op_costs(ops, (B // M,) + tuple(hwc)), cfg["P"])
+    elif args.cuts == "measured":
+        # the load balancer by measurement (outside the timed region): loaded per-cell times -> per-op costs -> cuts
+        from paper_1911_05146_b200.tuner import balance_by_measurement
+        opts = {hpf.OPT_CONV_PATH: args.conv_path}
+        if args.cell_ctas >= 0:
+            opts[hpf.OPT_CELL_CTAS] = args.cell_ctas
+        cuts, balance_history = balance_by_measurement(ops, (B,) + tuple(hwc), cfg["P"], M, torch.from_numpy(theta), cfg["cuts"], options=opts)
     model = hpf.Model(ops, (B,) + tuple(hwc), cuts, M)
     model.set_option(hpf.OPT_GRAPH, 0 if args.no_graph else 1)
     model.set_option(hpf.OPT_CONV_PATH, args.conv_path)
@@ -508,6 +590,7 @@ def main():
     by, flops = step_model(ops, hwc, B)
     step_bytes = sum(by.values())
     n_tc, n_cc = model.conv_path_counts()
+    fused_bytes = model.step_bytes()
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -515,7 +598,7 @@ def main():
         "config": {"workload": NAMES[args.workload], "global_batch": world * B, "micro_batches": M,
                    "partitions": model.num_partitions(), "parallelism": "replicas x%d, no data-path collective" % world,
                    "l2": "working set %.1f GB per step exceeds the 126 MB L2; no explicit flush" % (ws_bytes / 1e9),
-                   "cuts": args.cuts, "cut_points": list(cuts), "graph": not args.no_graph, "cell_ctas": args.cell_ctas,
+                   "cuts": args.cuts, "cut_points": list(cuts), "balance_history": balance_history, "graph": not args.no_graph, "cell_ctas": args.cell_ctas,
                    "phase_ms": {"forward": phase_ms[0], "backward": phase_ms[1], "average": phase_ms[2]}, "conv_sites_tensor_core": n_tc, "conv_sites_cuda_core": n_cc,
                    "loss": loss},
         "e2e": {"value": world * B / (ms_e2e / args.steps * 1e-3), "unit": UNIT,
@@ -526,6 +609,12 @@ def main():
                           "conv_flops_per_step": flops, "achieved": step_bytes / (ms_step * 1e-3) / 1e9,
                           "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": step_bytes / (ms_step * 1e-3) / 1e9 / pk["hbm_gbs"],
                           "peak_source": pk["source"],
+                          # what the step has to move with the fusions it runs with (BN+ReLU applied by the reading convolution,
+                          # residual adds in the write-out): fewer bytes for the same time, so a lower fraction of the roof
+                          "fused_algorithmic_bytes_per_step": fused_bytes,
+                          "fused_achieved": fused_bytes / (ms_step * 1e-3) / 1e9,
+                          "fused_frac": fused_bytes / (ms_step * 1e-3) / 1e9 / pk["hbm_gbs"],
+                          "hbm_floor_ms": {"unfused_model": step_bytes / (pk["hbm_gbs"] * 1e9) * 1e3, "fused_model": fused_bytes / (pk["hbm_gbs"] * 1e9) * 1e3},
                           "conv_tflops": flops / (ms_step * 1e-3) / 1e12},
     }
     if not args.skip_kernel_roofline:

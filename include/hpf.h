@@ -205,6 +205,11 @@ int hpf_loss_slots_ptr(const hpf_model *model, const float **d_ptr);
  * backward (phase 1).  h_ns: host, 2*P*M values.  Synchronises.  HPF_ERR_STATE if the option is off. */
 int hpf_cell_times(hpf_model *model, int32_t phase, int64_t *h_ns);
 
+/* Bytes one step (forward + backward + average) has to move between the kernels under the fusions the model's options
+ * select: per op what its kernels read and write once (a BN+ReLU applied by the reading convolution and a residual add
+ * computed in a convolution's write-out move nothing of their own; the by-products those convolutions store are
+ * counted with them), times M, plus the once-per-step weight preparation and the gradient average.  Host only. */
+int hpf_step_bytes(const hpf_model *model, double *fused_bytes);
 /* Kernel launches (graph kernel nodes count as launches) issued by the step calls since bind. */
 int hpf_launch_count(const hpf_model *model, int64_t *n);
 /* How many convolution launch sites per phase use the tensor-core path / the CUDA-core path. */

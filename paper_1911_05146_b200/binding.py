@@ -56,6 +56,7 @@ _SIGNATURES = {
     "hpf_sgd_momentum_step": [_vp, _vp, _f32, _f32, _f32],
     "hpf_sgd_momentum_flat": [_vp, _vp, _vp, _vp, _i32, _i64, _f32, _f32, _f32, _vp],
     "hpf_launch_count": [_vp, _pi64],
+    "hpf_step_bytes": [_vp, C.POINTER(C.c_double)],
     "hpf_cell_times": [_vp, _i32, _pi64],
     "hpf_conv_path_counts": [_vp, _pi64, _pi64],
     "hpf_conv_scratch_bytes": [_i32] * 8 + [C.POINTER(C.c_size_t)],
@@ -245,6 +246,9 @@ class Model:
         P = self.num_partitions()
         buf = (_i64 * (P * self.M * 2))(); _check(lib().hpf_cell_times(self._h, int(phase), buf))
         return [[(buf[(p * self.M + m) * 2], buf[(p * self.M + m) * 2 + 1]) for m in range(self.M)] for p in range(P)]
+
+    def step_bytes(self):
+        v = C.c_double(); _check(lib().hpf_step_bytes(self._h, C.byref(v))); return v.value
 
     def launch_count(self):
         n = _i64(); _check(lib().hpf_launch_count(self._h, C.byref(n))); return n.value

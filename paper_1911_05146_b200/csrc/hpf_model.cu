@@ -1401,6 +1401,52 @@ int hpf_cell_times(hpf_model* mdl, int32_t phase, int64_t* h_ns)
     return HPF_OK;
 }
 
+int hpf_step_bytes(const hpf_model* mdl_c, double* fused_bytes)
+{
+    if (!mdl_c || !fused_bytes) return fail(HPF_ERR_INVALID, "null");
+    hpf_model* mdl = const_cast<hpf_model*>(mdl_c);
+    if (!mdl->planned) build_memory_plan(mdl);
+    double total = 0.0;
+    double conv_weights = 0.0;
+    for (int i = 0; i < mdl->n_ops; ++i) {
+        const OpInfo& o = mdl->ops[i];
+        const hpf_op& q = o.op;
+        const double out_el = (double)mdl->b * o.H * o.W * o.C, in_el = (double)mdl->b * o.iH * o.iW * o.iC;
+        const GradEdge& e = mdl->edge0[i];
+        const double extra_in = (e.addend >= 0 ? in_el : 0.0) + (e.accumulate ? in_el : 0.0);
+        double f = 0.0, bw = 0.0;
+        switch (q.kind) {
+        case HPF_OP_CONV: {
+            const double w = (double)q.c_out * q.ksize * q.ksize * q.c_in;
+            const double read_in = q.stride > 1 && q.ksize == 1 ? (double)mdl->b * o.H * o.W * o.iC : in_el;   // a strided 1x1 samples
+            conv_weights += w;
+            f = read_in + w + out_el;
+            if (mdl->fused_into[i] >= 0) f += out_el;                       // the residual rides in the write-out
+            if (mdl->conv_in_bn[i] >= 0) f += in_el;                        // the BN+ReLU output is stored as a by-product
+            if (q.src0 >= 0) bw += out_el + w + in_el + extra_in;           // data gradient
+            bw += read_in + out_el + w;                                     // weight gradient
+            break;
+        }
+        case HPF_OP_BNRELU:
+        case HPF_OP_BN:
+            f = mdl->bn_into[i] >= 0 ? 0.0 : 2.0 * out_el;                 // applied by the reading convolution: no traffic of its own
+            bw = 3.0 * out_el + extra_in;
+            break;
+        case HPF_OP_RELU: f = 2.0 * out_el; bw = 3.0 * out_el + extra_in; break;
+        case HPF_OP_ADD: f = mdl->add_done_by[i] >= 0 ? 0.0 : 3.0 * out_el; break;   // its gradient is an alias or an on-the-fly addend
+        case HPF_OP_MAXPOOL: f = in_el + out_el; bw = in_el + out_el + in_el + (e.accumulate ? in_el : 0.0); break;
+        case HPF_OP_HEAD: f = in_el; bw = in_el; break;
+        }
+        total += 4.0 * (f + bw);
+    }
+    for (const AccumAction& a : mdl->accums) total += 4.0 * 3.0 * (double)mdl->numel(a.dst);
+    total *= mdl->M;
+    total += 4.0 * 5.0 * conv_weights;                                      // once per step: weights read, four prepared copies written
+    total += 4.0 * (mdl->M + 1.0) * (double)mdl->G;                         // the gradient average
+    *fused_bytes = total;
+    return HPF_OK;
+}
+
 int hpf_launch_count(const hpf_model* mdl, int64_t* n)
 {
     if (!mdl || !n) return fail(HPF_ERR_INVALID, "null");
