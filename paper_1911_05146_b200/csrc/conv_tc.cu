@@ -252,6 +252,7 @@ struct FwdScalars {
     unsigned int* stat_ticket;   // counts finished CTAs; zero between launches
     float* stat_out;             // mean[c_out], rstd[c_out], written by the CTA that finishes last
     float stat_eps;
+    float stat_inv_tile_rows;    // 1 / (pixels of one tile)
     double stat_inv_rows;        // 1 / (pixels the statistics run over)
     // BN+ReLU applied to the activation operand on its way to the tensor core (see ConvBnFuse::in_mode)
     // several tiles per CTA (MULTI kernel; tile j of CTA b is tile b*tiles_per_cta + j): tile j+1's loads, split and MMAs
@@ -329,19 +330,23 @@ __device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__flo
 // launches whose tiles are all full), so the total is
 //     mean = average of the tile means,   M2 = sum of the tile M2 + n_tile * sum (tile mean - mean)^2,
 // evaluated about tile 0's mean so that no difference of large numbers appears anywhere: the result stays accurate
-// however far a channel's mean is from zero compared with its spread.  The tiles are added in a fixed order in fp64,
-// so every caller gets the same bits.  Called by 256 threads (tid 0..255) that share named barrier 1; C is a power of
-// two in 16..256; bn_red: 256 x 8 doubles of shared memory.  On return thread tid < C holds its channel's mean and
-// 1/sqrt(var + eps).
+// however far a channel's mean is from zero compared with its spread.  What is added up are small differences of tile
+// means, their squares and the non-negative tile M2, at most a few hundred terms: fp32 sums in a fixed order (every
+// caller gets the same bits), the final combination in fp64.  Called by 256 threads (tid 0..255) that share named
+// barrier 1; C is a power of two in 16..256; bn_ws: 8 x 32 x 8 floats of shared memory.  On return thread tid < C holds
+// its channel's mean and 1/sqrt(var + eps).
+// Consecutive threads read consecutive float4 of a tile's row (coalesced: every CTA of a launch reads these same few
+// lines); the lanes of a warp that share a column are added by a butterfly, the warps through shared memory.
 __device__ __forceinline__ void bn_combine_partials(const float* partials, int n_tiles, int C, double inv_rows, float eps,
-                                                    double (*bn_red)[8], int tid, float* mean, float* rstd)
+                                                    float (*bn_ws)[32][8], int tid, float* mean, float* rstd)
 {
-    const int ncol4 = C >> 1;                          // float4 columns of one tile's [2][C] moments; 256 % ncol4 == 0
+    const int ncol4 = C >> 1;                          // float4 columns of one tile's [2][C] moments: 8..128
     const int col4 = tid % ncol4, ln = tid / ncol4, L = 256 / ncol4;
     const float4* part = reinterpret_cast<const float4*>(partials);
     // the first C/4 columns are tile means: accumulated as differences from tile 0's mean (and their squares)
-    const float4 ref = col4 < (C >> 2) ? __ldcg(part + col4) : make_float4(0.f, 0.f, 0.f, 0.f);
-    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0, b0 = 0.0, b1 = 0.0, b2 = 0.0, b3 = 0.0;
+    const bool mean_col = col4 < (C >> 2);
+    const float4 ref = mean_col ? __ldcg(part + col4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f, b0 = 0.f, b1 = 0.f, b2 = 0.f, b3 = 0.f;
     // eight rows per batch, all eight loads in flight together (a loop that used each load before issuing the next would
     // pay an L2 round trip per row); rows beyond the last add zero
     for (int k0 = ln; k0 < n_tiles; k0 += 8 * L) {
@@ -353,64 +358,47 @@ __device__ __forceinline__ void bn_combine_partials(const float* partials, int n
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const double d0 = (double)(v[j].x - ref.x), d1 = (double)(v[j].y - ref.y), d2 = (double)(v[j].z - ref.z), d3 = (double)(v[j].w - ref.w);
-            a0 += d0; a1 += d1; a2 += d2; a3 += d3;
-            b0 += d0 * d0; b1 += d1 * d1; b2 += d2 * d2; b3 += d3 * d3;
+            const float f0 = v[j].x - ref.x, f1 = v[j].y - ref.y, f2 = v[j].z - ref.z, f3 = v[j].w - ref.w;
+            a0 += f0; a1 += f1; a2 += f2; a3 += f3;
+            b0 = fmaf(f0, f0, b0); b1 = fmaf(f1, f1, b1); b2 = fmaf(f2, f2, b2); b3 = fmaf(f3, f3, b3);
         }
     }
-    if (ncol4 <= 16) {
-        // several lanes of a column sit in one warp: a fixed butterfly first, then the eight warps in ascending order
-        for (int off = 16; off >= ncol4; off >>= 1) {
-            a0 += __shfl_xor_sync(0xffffffffu, a0, off); a1 += __shfl_xor_sync(0xffffffffu, a1, off);
-            a2 += __shfl_xor_sync(0xffffffffu, a2, off); a3 += __shfl_xor_sync(0xffffffffu, a3, off);
-            b0 += __shfl_xor_sync(0xffffffffu, b0, off); b1 += __shfl_xor_sync(0xffffffffu, b1, off);
-            b2 += __shfl_xor_sync(0xffffffffu, b2, off); b3 += __shfl_xor_sync(0xffffffffu, b3, off);
-        }
-        const int warp = tid >> 5, lane = tid & 31;
-        double (*wsum)[8] = bn_red + 128;                   // [warp * ncol4 + column]; rows 0..127 stay free for the totals
-        if (lane < ncol4) {
-            double* d = wsum[warp * ncol4 + lane];
-            d[0] = a0; d[1] = a1; d[2] = a2; d[3] = a3; d[4] = b0; d[5] = b1; d[6] = b2; d[7] = b3;
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (tid < ncol4) {
-            double t[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
-            for (int w = 0; w < 8; ++w) {
-                const double* r = wsum[w * ncol4 + tid];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) t[q] += r[q];
-            }
-#pragma unroll
-            for (int q = 0; q < 8; ++q) bn_red[tid][q] = t[q];
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-    } else {
-        double* mine = bn_red[tid];
-        mine[0] = a0; mine[1] = a1; mine[2] = a2; mine[3] = a3; mine[4] = b0; mine[5] = b1; mine[6] = b2; mine[7] = b3;
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (tid < ncol4) {
-            // rows tid, tid + ncol4, ... are read by this thread alone, so the total can go back into row tid
-            double t[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
-            for (int l = 0; l < L; ++l) {
-                const double* r = bn_red[l * ncol4 + tid];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) t[q] += r[q];
-            }
-#pragma unroll
-            for (int q = 0; q < 8; ++q) bn_red[tid][q] = t[q];
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
+    // lanes of one warp that share a column (fewer than 32 columns): a fixed butterfly
+    for (int off = 16; off >= ncol4; off >>= 1) {
+        a0 += __shfl_xor_sync(0xffffffffu, a0, off); a1 += __shfl_xor_sync(0xffffffffu, a1, off);
+        a2 += __shfl_xor_sync(0xffffffffu, a2, off); a3 += __shfl_xor_sync(0xffffffffu, a3, off);
+        b0 += __shfl_xor_sync(0xffffffffu, b0, off); b1 += __shfl_xor_sync(0xffffffffu, b1, off);
+        b2 += __shfl_xor_sync(0xffffffffu, b2, off); b3 += __shfl_xor_sync(0xffffffffu, b3, off);
     }
+    const int warp = tid >> 5, lane = tid & 31;
+    if (lane < ncol4) {
+        float* d = bn_ws[warp][lane];
+        *reinterpret_cast<float4*>(d) = make_float4(a0, a1, a2, a3);
+        if (mean_col) *reinterpret_cast<float4*>(d + 4) = make_float4(b0, b1, b2, b3);
+    }
+    // tile 0's means travel in the half of an M2 column's slot that nothing else uses (that of the channel's M2 column in
+    // the first warp that holds it), so that nothing has to be fetched again after the barrier
+    if (mean_col && ln == 0) {
+        const int qv0 = (C >> 2) + col4;
+        *reinterpret_cast<float4*>(bn_ws[ncol4 > 32 ? qv0 >> 5 : 0][qv0 & 31] + 4) = ref;
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
     if (tid < C) {
-        const double T = (double)n_tiles;
-        const double sd = bn_red[tid >> 2][tid & 3], sq = bn_red[tid >> 2][4 + (tid & 3)];        // sum of (tile mean - ref), of its square
-        const double m2 = bn_red[(C >> 2) + (tid >> 2)][tid & 3];                                   // sum of the tile M2
-        const double n_tile = 1.0 / (inv_rows * T);
-        const double m = (double)__ldcg(partials + tid) + sd / T;
-        double var = (m2 + n_tile * (sq - sd * sd / T)) * inv_rows;
+        // column q sits in lane q % 32 of the warps q / 32, q / 32 + ncol4 / 32, ... (of every warp when there are at most
+        // 32 columns): added in ascending warp order
+        const int qm = tid >> 2, qv = (C >> 2) + (tid >> 2), comp = tid & 3;
+        const int wstep = ncol4 > 32 ? ncol4 >> 5 : 1;
+        float sd = 0.f, sq = 0.f, m2 = 0.f;
+        for (int w = (ncol4 > 32 ? qm >> 5 : 0); w < 8; w += wstep) { sd += bn_ws[w][qm & 31][comp]; sq += bn_ws[w][qm & 31][4 + comp]; }
+        for (int w = (ncol4 > 32 ? qv >> 5 : 0); w < 8; w += wstep) m2 += bn_ws[w][qv & 31][comp];
+        // (no fp64 division: mean = ref + sd / T and var = M2 / rows + (sq - sd^2 / T) / T with 1 / T in fp32-exact steps)
+        const double inv_tiles = (double)(1.0f / (float)n_tiles);
+        const double dsd = (double)sd;
+        const double m = (double)bn_ws[ncol4 > 32 ? qv >> 5 : 0][qv & 31][4 + comp] + dsd * inv_tiles;
+        double var = (double)m2 * inv_rows + ((double)sq - dsd * dsd * inv_tiles) * inv_tiles;
         if (var < 0.0) var = 0.0;
         *mean = (float)m;
-        *rstd = (float)(1.0 / sqrt(var + (double)eps));
+        *rstd = 1.0f / sqrtf((float)(var + (double)eps));          // correctly rounded fp32 operations: within an ulp or two of the fp64 result
     }
 }
 
@@ -611,7 +599,7 @@ __device__ __forceinline__ int conv_fwd_cta(const FwdParams* gpp, FwdScalars& p,
                 // The producer left only its per-tile sums (few enough that adding them here, under the first copy's
                 // latency, is cheaper than a ticket at the producer's end): every CTA adds them in the same fixed order,
                 // so all CTAs hold identical statistics; the first CTA stores them for the backward pass.
-                __shared__ double bn_red[256][8];
+                __shared__ __align__(16) float bn_red[8][32][8];
                 float gam = 0.f, bet = 0.f, mu = 0.f, rs = 0.f;
                 if (tid < C) { gam = __ldg(p.bn_in_gamma + tid); bet = __ldg(p.bn_in_beta + tid); }   // travel with the sums
                 bn_combine_partials(p.bn_in_partials, p.bn_in_tiles, C, p.bn_in_inv_rows, p.bn_in_eps, bn_red, tid, &mu, &rs);
@@ -737,6 +725,7 @@ __device__ __forceinline__ int conv_fwd_cta(const FwdParams* gpp, FwdScalars& p,
         // stores would touch 32 lines each).  With one tile per CTA the staging area is the pipeline itself, idle once
         // the accumulator is complete; with several tiles it is a region of its own, because the next tile's loads and
         // MMAs are in flight while this tile is written out.
+        __shared__ float4 shift_s[64];                 // per group of 4 output channels: the shift of the tile's statistics
         __shared__ int row_off[kTileM];                // offset (floats) of the pixel's channel row in the output, or -1
         __shared__ int row_fill[kTileM];               // strided data gradient: which neighbours of the sample exist
         float* const stg = reinterpret_cast<float*>(smem + stg_off);
@@ -842,6 +831,7 @@ __device__ __forceinline__ int conv_fwd_cta(const FwdParams* gpp, FwdScalars& p,
                 sk = *reinterpret_cast<const float4*>(stg + 4 * c4k);
                 if (extra) { const float4 e = __ldcg(reinterpret_cast<const float4*>(extra + row_off[0] + 4 * c4k)); sk.x += e.x; sk.y += e.y; sk.z += e.z; sk.w += e.w; }
                 if (accumulate) { const float4 e = *reinterpret_cast<const float4*>(outp + row_off[0] + 4 * c4k); sk.x += e.x; sk.y += e.y; sk.z += e.z; sk.w += e.w; }
+                if (tid < c4n) shift_s[tid] = sk;          // read again when the tile's moments are formed
             }
             for (int base = tid; base < total4; base += 1024) {
                 float4 o[4];
@@ -915,24 +905,32 @@ __device__ __forceinline__ int conv_fwd_cta(const FwdParams* gpp, FwdScalars& p,
                     red[2 * tid] = sa; red[2 * tid + 1] = sb;
                 }
                 asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (tid < c4n) {
-                    // thread g owns channel group g (its own shift sk is that group's): the tile's mean and the sum of
-                    // squared deviations from it, from the shifted sums
-                    const int g = tid;
-                    float4 s1 = make_float4(0.f, 0.f, 0.f, 0.f), s2 = s1;
-                    for (int t2 = g; t2 < n_rows; t2 += c4n) {
-                        const float4 v1 = red[2 * t2], v2 = red[2 * t2 + 1];
-                        s1.x += v1.x; s1.y += v1.y; s1.z += v1.z; s1.w += v1.w;
-                        s2.x += v2.x; s2.y += v2.y; s2.z += v2.z; s2.w += v2.w;
+                if (tid < ((c4n * 2 + 31) & ~31)) {          // whole warps: the swap below is a warp shuffle
+                    // threads 2g and 2g+1 add group g's rows of shifted sums and of shifted squares, swap the totals, and store
+                    // the tile's mean (from the sums and the group's shift, which thread g keeps: fetched through shared memory)
+                    // and the sum of squared deviations from it
+                    const int g = tid >> 1, which = tid & 1;
+                    const bool mine = tid < c4n * 2;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {                       // n_rows / c4n <= 8
+                        const int t2 = g + j * c4n;
+                        if (mine && t2 < n_rows) { const float4 v2 = red[2 * t2 + which]; acc.x += v2.x; acc.y += v2.y; acc.z += v2.z; acc.w += v2.w; }
                     }
-                    const float inv_n = 1.f / (float)(p.box_w * p.box_h * p.box_n);       // every tile of a fused launch is full
-                    const float4 mt = make_float4(sk.x + s1.x * inv_n, sk.y + s1.y * inv_n, sk.z + s1.z * inv_n, sk.w + s1.w * inv_n);
-                    const float4 m2 = make_float4(s2.x - s1.x * s1.x * inv_n, s2.y - s1.y * s1.y * inv_n, s2.z - s1.z * s1.z * inv_n,
-                                                  s2.w - s1.w * s1.w * inv_n);
-                    float* dstp = p.stat_partials + (size_t)(tile0 + tj) * 2 * p.c_out + co0 + 4 * g;
-                    *reinterpret_cast<float4*>(dstp) = mt;
-                    *reinterpret_cast<float4*>(dstp + p.c_out) = m2;
-                    if (stat_mode == 1) __threadfence();
+                    float4 oth;
+                    oth.x = __shfl_xor_sync(0xffffffffu, acc.x, 1); oth.y = __shfl_xor_sync(0xffffffffu, acc.y, 1);
+                    oth.z = __shfl_xor_sync(0xffffffffu, acc.z, 1); oth.w = __shfl_xor_sync(0xffffffffu, acc.w, 1);
+                    const float4 s1 = which ? oth : acc, s2 = which ? acc : oth;
+                    const float4 kg = shift_s[mine ? g : 0];
+                    const float inv_n = p.stat_inv_tile_rows;       // every tile of a fused launch is full
+                    float4 r;
+                    if (which == 0) r = make_float4(kg.x + s1.x * inv_n, kg.y + s1.y * inv_n, kg.z + s1.z * inv_n, kg.w + s1.w * inv_n);
+                    else r = make_float4(s2.x - s1.x * s1.x * inv_n, s2.y - s1.y * s1.y * inv_n, s2.z - s1.z * s1.z * inv_n, s2.w - s1.w * s1.w * inv_n);
+                    if (mine) {
+                        float* dstp = p.stat_partials + ((size_t)(tile0 + tj) * 2 + which) * p.c_out + co0 + 4 * g;
+                        *reinterpret_cast<float4*>(dstp) = r;
+                        if (stat_mode == 1) __threadfence();
+                    }
                 }
             }
         }
@@ -956,7 +954,7 @@ __device__ __forceinline__ int conv_fwd_cta(const FwdParams* gpp, FwdScalars& p,
                     float mu = 0.f, rs = 0.f;
                     // every tile is written out and the pipeline buffers are idle: they hold the reduction
                     bn_combine_partials(p.stat_partials, p.n_tiles, p.c_out, p.stat_inv_rows, p.stat_eps,
-                                        reinterpret_cast<double (*)[8]>(smem), tid, &mu, &rs);
+                                        reinterpret_cast<float (*)[32][8]>(smem), tid, &mu, &rs);
                     if (tid < p.c_out) { p.stat_out[tid] = mu; p.stat_out[p.c_out + tid] = rs; }
                     if (tid == 0) *p.stat_ticket = 0u;
                 }
@@ -1869,6 +1867,7 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
         if ((fuse->mode != 1 && fuse->mode != 3) || pass != PASS_FWD || !conv_tc_can_fuse_bn(s, pass) || fuse->rows < 1) return cudaErrorNotSupported;
         p.stat_mode = fuse->mode; p.stat_partials = fuse->partials;
         p.stat_ticket = fuse->ticket; p.stat_out = fuse->stats_out; p.stat_eps = fuse->eps; p.stat_inv_rows = 1.0 / (double)fuse->rows;
+        p.stat_inv_tile_rows = 1.0f / (float)b.rows;
     }
     if (fuse && fuse->in_mode) {
         if (pass != PASS_FWD || !conv_tc_can_fuse_bn_input(s)) return cudaErrorNotSupported;
@@ -1924,7 +1923,7 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
     L->grid = dim3((p.n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta, v.c_out / n_chunk, p.ksplit);
     L->smem = p.tiles_per_cta > 1 ? pipe_bytes + stg_bytes : (pipe_bytes > stg_bytes ? pipe_bytes : stg_bytes);
     L->smem += 1024;
-    if (p.stat_mode == 1 && L->smem < 16384u + 1024u) L->smem = 16384u + 1024u;      // the last CTA's fp64 reduction: 256 x 8 doubles
+    if (p.stat_mode == 1 && L->smem < 8192u + 1024u) L->smem = 8192u + 1024u;      // the last CTA's reduction: 8 x 32 x 8 floats
     plan->valid = 1;
     return cudaSuccess;
 }
