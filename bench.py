@@ -460,6 +460,8 @@ def main():
     ap.add_argument("--conv-path", type=int, default=0)
     ap.add_argument("--cell-ctas", type=int, default=-1,
                     help="CTAs of the persistent forward cell kernels (HPF_OPT_CELL_CTAS); 0: one launch per convolution; -1: the library's default")
+    ap.add_argument("--two-phases", action="store_true",
+                    help="hpf_forward then hpf_backward (backward after the forward drain) instead of hpf_forward_backward")
     ap.add_argument("--opt", action="append", default=[], help="library option as NUMBER=VALUE (hpf_set_option), repeatable")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-kernel-roofline", action="store_true")
@@ -526,7 +528,8 @@ def main():
     avg = torch.empty(G, device=dev)
     ws_bytes = model.workspace_bytes()
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
-    streams = [torch.cuda.Stream(device=dev) for _ in range(2 * model.num_partitions())]     # stage streams + weight-gradient side streams
+    # stage streams + weight-gradient side streams + backward streams (the one-graph schedule)
+    streams = [torch.cuda.Stream(device=dev) for _ in range((2 if args.two_phases else 3) * model.num_partitions())]
     torch.cuda.synchronize()
     model.bind(params, slots, avg, ws, streams)
     dx, dl = torch.from_numpy(x).to(dev), torch.from_numpy(labels).to(dev)
@@ -534,8 +537,11 @@ def main():
     s0 = streams[0]
 
     def step():
-        model.forward(dx, dl)
-        model.backward()
+        if args.two_phases:
+            model.forward(dx, dl)
+            model.backward()
+        else:
+            model.forward_backward(dx, dl)
         model.grad_average()
 
     def barrier():
@@ -566,6 +572,8 @@ def main():
     # where the step's time goes: the three phases timed apart (a diagnostic; events on stream 0, which every phase joins)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
     phase_ms = [0.0, 0.0, 0.0]
+    model.forward(dx, dl); model.backward(); model.grad_average()          # untimed: the two-phase graphs may not exist yet
+    barrier()
     for _ in range(3):
         ev[0].record(s0); model.forward(dx, dl); ev[1].record(s0); model.backward(); ev[2].record(s0); model.grad_average(); ev[3].record(s0)
         barrier()
@@ -606,6 +614,8 @@ def main():
                    "partitions": model.num_partitions(), "parallelism": "replicas x%d, no data-path collective" % world,
                    "l2": "working set %.1f GB per step exceeds the 126 MB L2; no explicit flush" % (ws_bytes / 1e9),
                    "cuts": args.cuts, "cut_points": list(cuts), "balance_history": balance_history, "graph": not args.no_graph, "cell_ctas": args.cell_ctas, "options": args.opt,
+                   "schedule": "forward then backward, two graphs (fill / drain twice)" if args.two_phases else
+                               "hpf_forward_backward: one graph, a backward cell starts when the cell that feeds it is done",
                    "phase_ms": {"forward": phase_ms[0], "backward": phase_ms[1], "average": phase_ms[2]}, "conv_sites_tensor_core": n_tc, "conv_sites_cuda_core": n_cc,
                    "loss": loss},
         "e2e": {"value": world * B / (ms_e2e / args.steps * 1e-3), "unit": UNIT,

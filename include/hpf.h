@@ -159,7 +159,8 @@ int hpf_workspace_bytes(const hpf_model *model, size_t *bytes);
  * aligned, >= hpf_workspace_bytes): all caller-owned device memory that must outlive the model.
  * cuda_streams: n_streams >= P cudaStream_t handles (stage p runs on stream p; stream 0 is the one
  * the phases fork from and join to).  With n_streams >= 2P, stream P+p carries stage p's weight-gradient
- * kernels, which feed only the final average and so leave the chain of dependent kernels.  Creates
+ * kernels, which feed only the final average and so leave the chain of dependent kernels; with n_streams >= 3P,
+ * stream 2P+p carries stage p's backward cells in hpf_forward_backward.  Creates
  * events and tensor-map descriptors; allocates nothing on the device.  Errors: HPF_ERR_WORKSPACE, HPF_ERR_INVALID, HPF_ERR_CUDA. */
 int hpf_bind(hpf_model *model, float *d_params, float *d_grad_slots, float *d_grad_avg, void *d_workspace,
              size_t ws_bytes, void *const *cuda_streams, int32_t n_streams);
@@ -171,6 +172,14 @@ int hpf_bind(hpf_model *model, float *d_params, float *d_grad_slots, float *d_gr
 int hpf_forward(hpf_model *model, const float *d_x, const int32_t *d_labels);
 /* Section 5.2 Eq. 5-7: reverse sweep, last partition first; writes slot m of d_grad_slots. */
 int hpf_backward(hpf_model *model);
+/* hpf_forward and hpf_backward as ONE set of dependencies (Section 5.3: a stage works as soon as what it needs has
+ * arrived): the backward cell (p, m) starts when the cell that feeds it has finished - backward (p+1, m), or forward
+ * (P-1, m) for the last partition - instead of after the whole forward pass, so the backward pipeline fills while the
+ * forward pipeline drains.  The same kernels run on the same data: every result is bit-identical to hpf_forward followed
+ * by hpf_backward.  With n_streams >= 3P at hpf_bind, stream 2P+p carries partition p's backward cells, beside its
+ * forward cells on stream p; with fewer streams the call is hpf_forward followed by hpf_backward in one graph.
+ * Leaves the model where hpf_backward does (hpf_grad_average / hpf_sgd_momentum_step next; hpf_loss any time after). */
+int hpf_forward_backward(hpf_model *model, const float *d_x, const int32_t *d_labels);
 /* d_grad_avg = (sum over m ascending of slot m) / M  (Section 5.3: gradients accumulated/averaged). */
 int hpf_grad_average(hpf_model *model);
 /* The gradient average fused with the parameter update that closes the training step (Section 5.3: the averaged

@@ -46,6 +46,7 @@ _SIGNATURES = {
     "hpf_bind": [_vp, _vp, _vp, _vp, _vp, C.c_size_t, C.POINTER(_vp), _i32],
     "hpf_forward": [_vp, _vp, _vp],
     "hpf_backward": [_vp],
+    "hpf_forward_backward": [_vp, _vp, _vp],
     "hpf_grad_average": [_vp],
     "hpf_loss": [_vp, C.POINTER(_f32)],
     "hpf_step_host": [_vp, _vp, _vp, C.POINTER(_f32)],
@@ -214,6 +215,10 @@ class Model:
 
     def backward(self):
         _check(lib().hpf_backward(self._h))
+
+    def forward_backward(self, x, labels):
+        self._keep_inputs = (x, labels)
+        _check(lib().hpf_forward_backward(self._h, _ptr(x), _ptr(labels)))
 
     def grad_average(self):
         _check(lib().hpf_grad_average(self._h))

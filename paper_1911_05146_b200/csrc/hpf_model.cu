@@ -46,7 +46,7 @@ int cuda_fail(cudaError_t e, const char* where) { return hpf::api_cuda_fail(e, w
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-enum Phase { PH_FWD = 0, PH_BWD = 1, PH_AVG = 2, PH_COUNT = 3 };
+enum Phase { PH_FWD = 0, PH_BWD = 1, PH_AVG = 2, PH_COUNT = 3, PH_FB = 4 };
 enum State { ST_CREATED = 0, ST_BOUND = 1, ST_FWD = 2, ST_BWD = 3 };
 
 struct OpInfo {
@@ -121,6 +121,9 @@ struct hpf_model {
     std::vector<size_t> act_off, grad_off, stats_off;   // [m * n_ops + op]
     std::vector<size_t> bn_scratch_off, conv_scratch_off;   // per stream
     std::vector<size_t> splitk_off, splitk_bytes;            // per stream: tickets + partial tiles of K-split convolutions (zeroed at bind)
+    // the backward kernels of a partition have scratch of their own: in the one-graph schedule (hpf_forward_backward) a
+    // partition's backward cells run while its forward cells of later micro-batches are still under way
+    std::vector<size_t> bn_scratch_bwd_off, splitk_bwd_off;
     std::vector<size_t> pooled_off, persample_off;      // per m
     std::vector<std::vector<size_t>> fmsg_off, bmsg_off;  // [cut][i*M + m]
     size_t loss_slots_off = 0, loss_avg_off = 0, wprep_off = 0, stage_x_off = 0, stage_lab_off = 0, status_off = 0;
@@ -136,6 +139,8 @@ struct hpf_model {
     std::vector<cudaEvent_t> ev_fwd, ev_bwd;  // [cut * M + m]
     std::vector<cudaEvent_t> ev_join;         // per stream
     std::vector<cudaStream_t> side;           // per partition: weight-gradient stream (empty: none)
+    std::vector<cudaStream_t> bwd_streams;    // per partition: the backward cells' stream in the one-graph schedule (empty: none)
+    std::vector<cudaEvent_t> ev_fdone, ev_bjoin;   // forward (P-1, m) done; backward stream p done
     std::vector<cudaEvent_t> ev_side, ev_side_join;   // per partition: gradient ready -> side stream; side stream done
     cudaEvent_t ev_fork = nullptr, ev_sync = nullptr;
     // tensor-core plans [m * n_ops + op] per pass
@@ -145,6 +150,8 @@ struct hpf_model {
     struct FwdGraph { const float* x = nullptr; const int32_t* labels = nullptr; cudaGraphExec_t exec = nullptr; int64_t nodes = 0; };
     FwdGraph fwd_graph[2];
     int fwd_graph_next = 0;
+    FwdGraph fb_graph[2];                     // forward + backward as one graph (hpf_forward_backward)
+    int fb_graph_next = 0;
     cudaGraphExec_t graph[PH_COUNT] = {nullptr, nullptr, nullptr};
     int64_t graph_nodes[PH_COUNT] = {0, 0, 0};
     const float* cur_x = nullptr;
@@ -501,6 +508,15 @@ void build_memory_plan(hpf_model* mdl)
         mdl->splitk_bytes[p] = need;
         mdl->splitk_off[p] = take(need ? need : 16);
     }
+    mdl->bn_scratch_bwd_off.assign(P, 0); mdl->splitk_bwd_off.assign(P, 0);
+    for (int p = 0; p < P; ++p) {
+        size_t bn = 256;
+        for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i)
+            if (mdl->ops[i].op.kind == HPF_OP_BNRELU || mdl->ops[i].op.kind == HPF_OP_BN)
+                bn = std::max(bn, bn_scratch_bytes((int64_t)mdl->b * mdl->ops[i].H * mdl->ops[i].W, mdl->ops[i].C));
+        mdl->bn_scratch_bwd_off[p] = take(bn);
+        mdl->splitk_bwd_off[p] = take(mdl->splitk_bytes[p] ? mdl->splitk_bytes[p] : 16);
+    }
     mdl->cell_bar_off.assign(P, 0);
     for (int p = 0; p < P; ++p) mdl->cell_bar_off[p] = take(16);
     mdl->zero_hi = at;
@@ -685,12 +701,12 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
     case HPF_OP_BNRELU:
         CU(bnrelu_bwd(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m), addend,
                       e.accumulate != 0, slot + o.w_off, slot + o.b_off, (int64_t)mdl->b * o.H * o.W, o.C,
-                      mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches, true, true));
+                      mdl->ws + mdl->bn_scratch_bwd_off[p], st, &mdl->launches, true, true));
         break;
     case HPF_OP_BN:
         CU(bnrelu_bwd(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m), addend,
                       e.accumulate != 0, slot + o.w_off, slot + o.b_off, (int64_t)mdl->b * o.H * o.W, o.C,
-                      mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches, false, true));
+                      mdl->ws + mdl->bn_scratch_bwd_off[p], st, &mdl->launches, false, true));
         break;
     case HPF_OP_RELU:
         CU(relu_bwd(in0, dout, mdl->grad(q.src0, m), addend, e.accumulate != 0, mdl->numel(i), st, &mdl->launches));
@@ -710,6 +726,11 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
     return HPF_OK;
 }
 
+// phase PH_FWD / PH_BWD / PH_AVG: one phase, forked from and joined into stream 0.  PH_FB: forward and backward as ONE
+// set of dependencies (hpf_forward_backward): the backward cell (p, m) runs on partition p's backward stream as soon as
+// the cell that feeds it has finished - backward (p+1, m), or forward (P-1, m) for the last partition - while the
+// partition's forward stream may still be busy with later micro-batches.  Same kernels on the same data as the two
+// phases, so the results are bit-identical; only the idle slots of the forward drain and the backward fill get used.
 int enqueue_phase(hpf_model* mdl, int phase)
 {
     const PdlScope pdl_scope(mdl->opt_pdl);
@@ -717,11 +738,16 @@ int enqueue_phase(hpf_model* mdl, int phase)
     const int P = mdl->P, M = mdl->M;
     cudaStream_t s0 = mdl->streams[0];
     const bool multi = !mdl->opt_single && P > 1;
-    if (multi) {
+    const bool merged = phase == PH_FB;
+    const bool do_fwd = phase == PH_FWD || merged, do_bwd = phase == PH_BWD || merged;
+    const bool own_bwd_streams = merged && !mdl->bwd_streams.empty() && !mdl->opt_single;
+    auto bwd_stream = [&](int p) { return own_bwd_streams ? mdl->bwd_streams[p] : mdl->stream_of(p); };
+    if (multi || own_bwd_streams) {
         CU(cudaEventRecord(mdl->ev_fork, s0));
-        for (int p = 1; p < P; ++p) CU(cudaStreamWaitEvent(mdl->streams[p], mdl->ev_fork, 0));
+        if (multi) for (int p = 1; p < P; ++p) CU(cudaStreamWaitEvent(mdl->streams[p], mdl->ev_fork, 0));
+        if (own_bwd_streams) for (int p = 0; p < P; ++p) CU(cudaStreamWaitEvent(mdl->bwd_streams[p], mdl->ev_fork, 0));
     }
-    if (phase == PH_FWD) {
+    if (do_fwd) {
         // the tensor-core convolutions read split (and, for the data gradient, rearranged) weights: once per step
         for (int p = 0; p < P; ++p)
             if (!mdl->prep_table[p].empty()) {
@@ -753,15 +779,17 @@ int enqueue_phase(hpf_model* mdl, int phase)
                 }
                 if (mdl->opt_cell_times) CU(stamp_time(mdl->cell_time_slot(PH_FWD, p, m) + 1, st, &mdl->launches));
                 if (p < P - 1 && multi) CU(cudaEventRecord(mdl->ev_fwd[(size_t)p * M + m], st));          // send
+                if (p == P - 1 && own_bwd_streams) CU(cudaEventRecord(mdl->ev_fdone[m], st));            // the loss of micro-batch m stands
             }
-    } else if (phase == PH_BWD) {
+    }
+    if (do_bwd) {
         for (int t = 0; t < P + M - 1; ++t)
             for (int p = P - 1; p >= 0; --p) {
                 const int m = t - (P - 1 - p);
                 if (m < 0 || m >= M) continue;
-                cudaStream_t st = mdl->stream_of(p);
+                cudaStream_t st = bwd_stream(p);
                 if (p < P - 1) {
-                    if (multi) CU(cudaStreamWaitEvent(st, mdl->ev_bwd[(size_t)p * M + m], 0));           // recv partial errors
+                    if (multi || own_bwd_streams) CU(cudaStreamWaitEvent(st, mdl->ev_bwd[(size_t)p * M + m], 0));           // recv partial errors
                     if (mdl->opt_messages)
                         for (size_t k = 0; k < mdl->msg_plan[p].size(); ++k) {
                             const MessagePlan& mp = mdl->msg_plan[p][k];
@@ -769,6 +797,8 @@ int enqueue_phase(hpf_model* mdl, int phase)
                             if (mp.from_buffer) CU(grad_accumulate(dst, mdl->grad(mp.tensor, m), mdl->numel(mp.tensor), false, st, &mdl->launches));
                             if (mp.pending >= 0) CU(grad_accumulate(dst, mdl->grad(mp.pending, m), mdl->numel(mp.tensor), mp.from_buffer != 0, st, &mdl->launches));
                         }
+                } else if (own_bwd_streams) {
+                    CU(cudaStreamWaitEvent(st, mdl->ev_fdone[m], 0));      // the last partition turns around: forward (P-1, m) is done
                 }
                 if (mdl->opt_cell_times) CU(stamp_time(mdl->cell_time_slot(PH_BWD, p, m), st, &mdl->launches));
                 for (int i = mdl->part_hi[p] - 1; i >= mdl->part_lo[p]; --i) {
@@ -776,23 +806,28 @@ int enqueue_phase(hpf_model* mdl, int phase)
                     if (rc) return rc;
                 }
                 if (mdl->opt_cell_times) CU(stamp_time(mdl->cell_time_slot(PH_BWD, p, m) + 1, st, &mdl->launches));
-                if (p > 0 && multi) CU(cudaEventRecord(mdl->ev_bwd[(size_t)(p - 1) * M + m], st));       // send partial errors
+                if (p > 0 && (multi || own_bwd_streams)) CU(cudaEventRecord(mdl->ev_bwd[(size_t)(p - 1) * M + m], st));       // send partial errors
             }
     }
-    if (phase == PH_BWD && !mdl->side.empty() && !mdl->opt_single)
+    if (do_bwd && !mdl->side.empty() && !mdl->opt_single)
         for (int p = 0; p < P; ++p) {
             // the side stream holds work only if it was forked during this phase; joining an unforked stream is harmless
-            CU(cudaEventRecord(mdl->ev_side[p], mdl->stream_of(p)));
+            CU(cudaEventRecord(mdl->ev_side[p], bwd_stream(p)));
             CU(cudaStreamWaitEvent(mdl->side[p], mdl->ev_side[p], 0));
             CU(cudaEventRecord(mdl->ev_side_join[p], mdl->side[p]));
             CU(cudaStreamWaitEvent(s0, mdl->ev_side_join[p], 0));
+        }
+    if (own_bwd_streams)
+        for (int p = 0; p < P; ++p) {
+            CU(cudaEventRecord(mdl->ev_bjoin[p], mdl->bwd_streams[p]));
+            CU(cudaStreamWaitEvent(s0, mdl->ev_bjoin[p], 0));
         }
     if (multi)
         for (int p = 1; p < P; ++p) {
             CU(cudaEventRecord(mdl->ev_join[p], mdl->streams[p]));
             CU(cudaStreamWaitEvent(s0, mdl->ev_join[p], 0));
         }
-    if (phase == PH_FWD)
+    if (do_fwd)
         CU(loss_average(reinterpret_cast<float*>(mdl->ws + mdl->loss_slots_off), reinterpret_cast<float*>(mdl->ws + mdl->loss_avg_off), M, s0, &mdl->launches));
     if (phase == PH_AVG)
         CU(grad_average(mdl->gslots, mdl->gavg, M, mdl->G, s0, &mdl->launches));
@@ -822,13 +857,16 @@ int run_phase(hpf_model* mdl, int phase)
     if (!mdl->opt_graph) return enqueue_phase(mdl, phase);
     cudaGraphExec_t exec = nullptr;
     int64_t nodes = 0;
-    if (phase == PH_FWD) {
+    if (phase == PH_FWD || phase == PH_FB) {
+        // the captured graph reads the input and the labels it was captured with: one graph per (x, labels) pair, two kept
+        hpf_model::FwdGraph* slots = phase == PH_FWD ? mdl->fwd_graph : mdl->fb_graph;
+        int& next = phase == PH_FWD ? mdl->fwd_graph_next : mdl->fb_graph_next;
         hpf_model::FwdGraph* slot = nullptr;
-        for (auto& g : mdl->fwd_graph)
-            if (g.exec && g.x == mdl->cur_x && g.labels == mdl->cur_labels) slot = &g;
+        for (int k = 0; k < 2; ++k)
+            if (slots[k].exec && slots[k].x == mdl->cur_x && slots[k].labels == mdl->cur_labels) slot = &slots[k];
         if (!slot) {
-            slot = &mdl->fwd_graph[mdl->fwd_graph_next];
-            mdl->fwd_graph_next ^= 1;
+            slot = &slots[next];
+            next ^= 1;
             if (slot->exec) { cudaGraphExecDestroy(slot->exec); slot->exec = nullptr; }
             int rc = capture_phase(mdl, phase, &slot->exec, &slot->nodes);
             if (rc) return rc;
@@ -855,6 +893,10 @@ int run_phase(hpf_model* mdl, int phase)
 void release_device_objects(hpf_model* mdl)
 {
     for (auto& g : mdl->fwd_graph) if (g.exec) { cudaGraphExecDestroy(g.exec); g.exec = nullptr; }
+    for (auto& g : mdl->fb_graph) if (g.exec) { cudaGraphExecDestroy(g.exec); g.exec = nullptr; }
+    for (auto e : mdl->ev_fdone) if (e) cudaEventDestroy(e);
+    for (auto e : mdl->ev_bjoin) if (e) cudaEventDestroy(e);
+    mdl->ev_fdone.clear(); mdl->ev_bjoin.clear();
     for (auto& g : mdl->graph) if (g) { cudaGraphExecDestroy(g); g = nullptr; }
     for (auto e : mdl->ev_fwd) cudaEventDestroy(e);
     for (auto e : mdl->ev_bwd) cudaEventDestroy(e);
@@ -1105,6 +1147,14 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
             CU(cudaEventCreateWithFlags(&mdl->ev_side_join[p], cudaEventDisableTiming));
         }
     }
+    mdl->bwd_streams.clear();
+    if (n_streams >= 3 * mdl->P) {
+        mdl->bwd_streams.resize(mdl->P);
+        for (int p = 0; p < mdl->P; ++p) mdl->bwd_streams[p] = reinterpret_cast<cudaStream_t>(cuda_streams[2 * mdl->P + p]);
+        mdl->ev_fdone.assign(mdl->M, nullptr); mdl->ev_bjoin.assign(mdl->P, nullptr);
+        for (auto& ev : mdl->ev_fdone) CU(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+        for (auto& ev : mdl->ev_bjoin) CU(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+    }
     const int M = mdl->M, n = mdl->n_ops;
     CU(cudaEventCreateWithFlags(&mdl->ev_fork, cudaEventDisableTiming));
     CU(cudaEventCreateWithFlags(&mdl->ev_sync, cudaEventDisableTiming));
@@ -1196,7 +1246,7 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                     }
                     else if (pass == PASS_DGRAD) {
                         ConvBnFuse dsplit;
-                        if (mdl->splitk_bytes[o.part]) { dsplit.splitk = mdl->ws + mdl->splitk_off[o.part]; dsplit.splitk_bytes = mdl->splitk_bytes[o.part]; }
+                        if (mdl->splitk_bytes[o.part]) { dsplit.splitk = mdl->ws + mdl->splitk_bwd_off[o.part]; dsplit.splitk_bytes = mdl->splitk_bytes[o.part]; }
                         CU(conv_tc_prepare(pl, s, pass, passes, mdl->grad(i, m), nullptr, wp + 2 * G + o.w_off, wp + 3 * G + o.w_off,
                                            mdl->grad(src, m), ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch,
                                            &dsplit));
@@ -1279,6 +1329,17 @@ int hpf_forward(hpf_model* mdl, const float* d_x, const int32_t* d_labels)
     return HPF_OK;
 }
 
+int hpf_forward_backward(hpf_model* mdl, const float* d_x, const int32_t* d_labels)
+{
+    if (!mdl || !d_x || !d_labels) return fail(HPF_ERR_INVALID, "null argument");
+    if (mdl->state < ST_BOUND) return fail(HPF_ERR_STATE, "hpf_bind first");
+    mdl->cur_x = d_x; mdl->cur_labels = d_labels;
+    int rc = run_phase(mdl, PH_FB);
+    if (rc) return rc;
+    mdl->state = ST_BWD;
+    return HPF_OK;
+}
+
 int hpf_backward(hpf_model* mdl)
 {
     if (!mdl) return fail(HPF_ERR_INVALID, "null model");
@@ -1325,8 +1386,7 @@ int hpf_step_host(hpf_model* mdl, const float* h_x, const int32_t* h_labels, flo
     int32_t* dl = reinterpret_cast<int32_t*>(mdl->ws + mdl->stage_lab_off);
     CU(cudaMemcpyAsync(dx, h_x, sizeof(float) * (size_t)mdl->B * mdl->inH * mdl->inW * mdl->inC, cudaMemcpyHostToDevice, s0));
     CU(cudaMemcpyAsync(dl, h_labels, sizeof(int32_t) * (size_t)mdl->B, cudaMemcpyHostToDevice, s0));
-    int rc = hpf_forward(mdl, dx, dl);
-    if (!rc) rc = hpf_backward(mdl);
+    int rc = hpf_forward_backward(mdl, dx, dl);
     if (!rc) rc = hpf_grad_average(mdl);
     if (rc) return rc;
     return hpf_loss(mdl, h_loss);

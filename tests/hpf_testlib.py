@@ -36,7 +36,7 @@ def rel_l2(a, ref):
 class Bound:
     """A model bound to torch-owned device memory."""
 
-    def __init__(self, ops, in_hwc, B, M, cuts, theta, options=None, device="cuda:0", side_streams=True):
+    def __init__(self, ops, in_hwc, B, M, cuts, theta, options=None, device="cuda:0", side_streams=True, backward_streams=False):
         self.ops, self.in_hwc, self.B, self.M, self.cuts = ops, tuple(in_hwc), B, M, list(cuts)
         self.dev = torch.device(device)
         torch.cuda.set_device(self.dev)
@@ -48,7 +48,7 @@ class Bound:
         self.slots = torch.full((M, self.G), float("nan"), dtype=torch.float32, device=self.dev)
         self.avg = torch.full((self.G,), float("nan"), dtype=torch.float32, device=self.dev)
         self.ws = torch.empty(self.model.workspace_bytes(), dtype=torch.uint8, device=self.dev)
-        n_streams = self.model.num_partitions() * (2 if side_streams else 1)
+        n_streams = self.model.num_partitions() * (3 if backward_streams else (2 if side_streams else 1))
         self.streams = [torch.cuda.Stream(device=self.dev) for _ in range(n_streams)]
         torch.cuda.synchronize()
         self.model.bind(self.params, self.slots, self.avg, self.ws, self.streams)
@@ -58,9 +58,12 @@ class Bound:
         self.labels = torch.from_numpy(np.ascontiguousarray(labels, dtype=np.int32)).to(self.dev)
         torch.cuda.synchronize()
 
-    def step(self):
-        self.model.forward(self.x, self.labels)
-        self.model.backward()
+    def step(self, one_graph=False):
+        if one_graph:
+            self.model.forward_backward(self.x, self.labels)
+        else:
+            self.model.forward(self.x, self.labels)
+            self.model.backward()
         self.model.grad_average()
         loss = self.model.loss()
         self.model.synchronize(60000)

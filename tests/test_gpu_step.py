@@ -261,6 +261,37 @@ def test_single_stream_equals_multi_stream_bitwise():
         assert torch.equal(outs[0][1], o[1]) and torch.equal(outs[0][2], o[2])
 
 
+@pytest.mark.parametrize("streams", ["3P", "2P", "P"])
+def test_forward_and_backward_as_one_graph_give_the_same_bits(streams):
+    """hpf_forward_backward: the backward pipeline fills while the forward pipeline drains (a cell starts as soon as the
+    cell that feeds it is done).  Same kernels on the same data, so every bit must equal the two-phase step - also when
+    the caller gave no streams for the backward cells (then the call is the two phases in one graph)."""
+    ops = wl.resnet_v2_cifar(2)
+    x, labels, theta = seeded(ops, (32, 32, 3), 8, seed=4, bn_jitter=0.1)
+    cuts = wl.default_cuts(len(ops), 4)
+    ref = Bound(ops, (32, 32, 3), 8, 4, cuts, theta)
+    ref.upload(x, labels)
+    l_ref = ref.step()
+    bd = Bound(ops, (32, 32, 3), 8, 4, cuts, theta, {hpf.OPT_CELL_TIMES: 1}, side_streams=streams != "P", backward_streams=streams == "3P")
+    bd.upload(x, labels)
+    for _ in range(2):                           # the second replay must find every ticket and barrier as the first left it
+        assert bd.step(one_graph=True) == l_ref
+        assert torch.equal(ref.slots, bd.slots) and torch.equal(ref.avg, bd.avg)
+    for i in range(len(ops)):
+        assert np.array_equal(ref.tensor(i, 3, grad=True), bd.tensor(i, 3, grad=True)), i
+    if streams == "3P":
+        # the point of it: some backward cell starts before the last forward cell has ended
+        fwd, bwd = bd.model.cell_times(0), bd.model.cell_times(1)
+        assert min(s for row in bwd for s, _ in row) < max(e for row in fwd for _, e in row)
+        P, M = 4, 4
+        for m in range(M):
+            assert bwd[P - 1][m][0] >= fwd[P - 1][m][1]          # the last partition turns around only after its forward cell
+            for p in range(P - 1):
+                assert bwd[p][m][0] >= bwd[p + 1][m][1]          # partial errors arrive from the partition above
+    with pytest.raises(hpf.HpfError):
+        bd.model.backward()                      # the step is complete: a second backward needs a fresh forward
+
+
 def test_messages_across_cuts_match_the_oracle():
     """Activations sent forward and partial errors sent back (Eq. 7) per cut and micro-batch."""
     ops = wl.resnet_v2_cifar(1)
