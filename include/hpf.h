@@ -180,6 +180,32 @@ int hpf_backward(hpf_model *model);
  * forward cells on stream p; with fewer streams the call is hpf_forward followed by hpf_backward in one graph.
  * Leaves the model where hpf_backward does (hpf_grad_average / hpf_sgd_momentum_step next; hpf_loss any time after). */
 int hpf_forward_backward(hpf_model *model, const float *d_x, const int32_t *d_labels);
+/* ---- one cell at a time (Section 5.3: one process per model-partition) ---------------------------------------------
+ * The calls a stage-per-GPU run is made of: every GPU binds the same model (same op list, cuts, micro-batch count, hence
+ * the same memory plan) and runs only the cells of the partition it owns; what crosses a cut is copied between the GPUs'
+ * workspaces, where it lives at the same offset on both sides (hpf_tensor_ptr), by the caller (a peer copy or an NCCL
+ * send / recv into the consumer's own memory).  All calls enqueue on partition p's stream (weight gradients on its side
+ * stream) without a CUDA graph and without waiting for any other partition: the caller orders the cells.
+ *   hpf_prepare_partition  once per step before the partition's first cell: the split / rearranged weights.
+ *   hpf_forward_cell       ops of partition p on micro-batch m.  d_x [B][H][W][C]: needed by partition 0 (NULL otherwise);
+ *                          d_labels [B]: needed by the last partition.  Reads the activations of the live set of cut p-1
+ *                          for micro-batch m (hpf_boundary_desc), which must be in place.
+ *   hpf_backward_cell      reverse sweep of partition p on micro-batch m; for p < P-1 the gradient buffers listed by
+ *                          hpf_backward_message_desc(cut p) must hold what the partition above computed (Eq. 7).
+ *   hpf_join_partition     orders partition p's weight-gradient side stream before what follows on its stream.
+ *   hpf_partition_param_range   partition p's contiguous slice of the flat parameter / gradient vectors: the message
+ *                          of the per-partition allreduce across replicas (Section 5.3, one communicator per partition).
+ *   hpf_backward_message_count / _desc   the gradient buffers (by op: hpf_tensor_ptr(op, m, 1)) that partition p+1 hands
+ *                          down across cut p: for every tensor of the live set the buffer that holds the sum over its
+ *                          consumers at or above the cut, plus the gradient of a residual add that a kernel below the cut
+ *                          folds in on the fly. */
+int hpf_prepare_partition(hpf_model *model, int32_t p);
+int hpf_forward_cell(hpf_model *model, int32_t p, int32_t m, const float *d_x, const int32_t *d_labels);
+int hpf_backward_cell(hpf_model *model, int32_t p, int32_t m);
+int hpf_join_partition(hpf_model *model, int32_t p);
+int hpf_partition_param_range(const hpf_model *model, int32_t p, int64_t *first, int64_t *count);
+int hpf_backward_message_count(const hpf_model *model, int32_t cut, int32_t *n);
+int hpf_backward_message_desc(const hpf_model *model, int32_t cut, int32_t j, int32_t *op, int32_t shape[4] /* b,H,W,C */);
 /* d_grad_avg = (sum over m ascending of slot m) / M  (Section 5.3: gradients accumulated/averaged). */
 int hpf_grad_average(hpf_model *model);
 /* The gradient average fused with the parameter update that closes the training step (Section 5.3: the averaged

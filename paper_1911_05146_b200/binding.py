@@ -47,6 +47,13 @@ _SIGNATURES = {
     "hpf_forward": [_vp, _vp, _vp],
     "hpf_backward": [_vp],
     "hpf_forward_backward": [_vp, _vp, _vp],
+    "hpf_prepare_partition": [_vp, _i32],
+    "hpf_forward_cell": [_vp, _i32, _i32, _vp, _vp],
+    "hpf_backward_cell": [_vp, _i32, _i32],
+    "hpf_join_partition": [_vp, _i32],
+    "hpf_partition_param_range": [_vp, _i32, _pi64, _pi64],
+    "hpf_backward_message_count": [_vp, _i32, _pi32],
+    "hpf_backward_message_desc": [_vp, _i32, _i32, _pi32, _pi32],
     "hpf_grad_average": [_vp],
     "hpf_loss": [_vp, C.POINTER(_f32)],
     "hpf_step_host": [_vp, _vp, _vp, C.POINTER(_f32)],
@@ -215,6 +222,33 @@ class Model:
 
     def backward(self):
         _check(lib().hpf_backward(self._h))
+
+    # ---- one cell at a time (stage-per-GPU runs) ----
+    def prepare_partition(self, p):
+        _check(lib().hpf_prepare_partition(self._h, int(p)))
+
+    def forward_cell(self, p, m, x=None, labels=None):
+        self._keep_inputs = (x, labels) if x is not None or labels is not None else getattr(self, "_keep_inputs", None)
+        _check(lib().hpf_forward_cell(self._h, int(p), int(m), _ptr(x), _ptr(labels)))
+
+    def backward_cell(self, p, m):
+        _check(lib().hpf_backward_cell(self._h, int(p), int(m)))
+
+    def join_partition(self, p):
+        _check(lib().hpf_join_partition(self._h, int(p)))
+
+    def partition_param_range(self, p):
+        a, b = _i64(), _i64(); _check(lib().hpf_partition_param_range(self._h, int(p), C.byref(a), C.byref(b))); return a.value, b.value
+
+    def backward_messages(self, cut):
+        """Ops whose gradient buffers partition cut+1 hands down across `cut`, with their shapes (b, H, W, C)."""
+        n = _i32(); _check(lib().hpf_backward_message_count(self._h, int(cut), C.byref(n)))
+        out = []
+        for j in range(n.value):
+            op = _i32(); shape = (_i32 * 4)()
+            _check(lib().hpf_backward_message_desc(self._h, int(cut), j, C.byref(op), shape))
+            out.append((op.value, tuple(shape)))
+        return out
 
     def forward_backward(self, x, labels):
         self._keep_inputs = (x, labels)

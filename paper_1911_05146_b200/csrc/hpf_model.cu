@@ -1340,6 +1340,113 @@ int hpf_forward_backward(hpf_model* mdl, const float* d_x, const int32_t* d_labe
     return HPF_OK;
 }
 
+// ---- one cell at a time: the building blocks of a stage-per-GPU run (each GPU owns one partition) ----------------
+int hpf_prepare_partition(hpf_model* mdl, int32_t p)
+{
+    if (!mdl) return fail(HPF_ERR_INVALID, "null model");
+    if (mdl->state < ST_BOUND) return fail(HPF_ERR_STATE, "hpf_bind first");
+    if (p < 0 || p >= mdl->P) return fail(HPF_ERR_INVALID, "partition out of range");
+    if (mdl->prep_table[p].empty()) return HPF_OK;
+    float* wp = reinterpret_cast<float*>(mdl->ws + mdl->wprep_off);
+    const int64_t G4 = (mdl->G + 3) / 4 * 4;
+    int max_tiles = 1;
+    for (const WeightPrepEntry& e : mdl->prep_table[p]) max_tiles = std::max(max_tiles, conv_weight_prep_tiles(e.C, e.K, e.R));
+    CU(conv_weight_prep(mdl->params, wp, wp + G4, wp + 2 * G4, wp + 3 * G4,
+                        reinterpret_cast<const WeightPrepEntry*>(mdl->ws + mdl->prep_table_off[p]),
+                        (int)mdl->prep_table[p].size(), max_tiles, mdl->stream_of(p), &mdl->launches));
+    return HPF_OK;
+}
+
+int hpf_forward_cell(hpf_model* mdl, int32_t p, int32_t m, const float* d_x, const int32_t* d_labels)
+{
+    if (!mdl) return fail(HPF_ERR_INVALID, "null model");
+    if (mdl->state < ST_BOUND) return fail(HPF_ERR_STATE, "hpf_bind first");
+    if (p < 0 || p >= mdl->P || m < 0 || m >= mdl->M) return fail(HPF_ERR_INVALID, "cell out of range");
+    if (p == 0 && !d_x) return fail(HPF_ERR_INVALID, "the first partition reads the network input");
+    if (p == mdl->P - 1 && !d_labels) return fail(HPF_ERR_INVALID, "the last partition reads the labels");
+    if (d_x) mdl->cur_x = d_x;
+    if (d_labels) mdl->cur_labels = d_labels;
+    const PdlScope pdl_scope(mdl->opt_pdl);
+    const BnClusterScope bn_cluster_scope(mdl->opt_bn_cluster);
+    for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i) {
+        int rc = forward_op(mdl, i, m, mdl->stream_of(p), p);
+        if (rc) return rc;
+    }
+    if (mdl->state < ST_FWD) mdl->state = ST_FWD;
+    return HPF_OK;
+}
+
+int hpf_backward_cell(hpf_model* mdl, int32_t p, int32_t m)
+{
+    if (!mdl) return fail(HPF_ERR_INVALID, "null model");
+    if (mdl->state < ST_FWD) return fail(HPF_ERR_STATE, "the cell's forward has not run");
+    if (p < 0 || p >= mdl->P || m < 0 || m >= mdl->M) return fail(HPF_ERR_INVALID, "cell out of range");
+    if (p == mdl->P - 1 && !mdl->cur_labels) return fail(HPF_ERR_STATE, "the last partition needs the labels of its forward cell");
+    const PdlScope pdl_scope(mdl->opt_pdl);
+    const BnClusterScope bn_cluster_scope(mdl->opt_bn_cluster);
+    for (int i = mdl->part_hi[p] - 1; i >= mdl->part_lo[p]; --i) {
+        int rc = backward_op(mdl, i, m, mdl->stream_of(p), p);
+        if (rc) return rc;
+    }
+    mdl->state = ST_BWD;
+    return HPF_OK;
+}
+
+int hpf_join_partition(hpf_model* mdl, int32_t p)
+{
+    if (!mdl) return fail(HPF_ERR_INVALID, "null model");
+    if (mdl->state < ST_BOUND) return fail(HPF_ERR_STATE, "hpf_bind first");
+    if (p < 0 || p >= mdl->P) return fail(HPF_ERR_INVALID, "partition out of range");
+    if (!mdl->side.empty() && !mdl->opt_single) {
+        cudaStream_t st = mdl->stream_of(p);
+        CU(cudaEventRecord(mdl->ev_side[p], st));
+        CU(cudaStreamWaitEvent(mdl->side[p], mdl->ev_side[p], 0));
+        CU(cudaEventRecord(mdl->ev_side_join[p], mdl->side[p]));
+        CU(cudaStreamWaitEvent(st, mdl->ev_side_join[p], 0));
+    }
+    return HPF_OK;
+}
+
+int hpf_partition_param_range(const hpf_model* mdl, int32_t p, int64_t* first, int64_t* count)
+{
+    if (!mdl || !first || !count) return fail(HPF_ERR_INVALID, "null");
+    if (p < 0 || p >= mdl->P) return fail(HPF_ERR_INVALID, "partition out of range");
+    const OpInfo& a = mdl->ops[mdl->part_lo[p]];
+    const OpInfo& z = mdl->ops[mdl->part_hi[p] - 1];
+    *first = a.w_off;
+    *count = z.b_off + z.b_cnt - a.w_off;
+    return HPF_OK;
+}
+
+int hpf_backward_message_count(const hpf_model* mdl, int32_t cut, int32_t* n)
+{
+    if (!mdl || !n) return fail(HPF_ERR_INVALID, "null");
+    if (cut < 0 || cut >= (int)mdl->cuts.size()) return fail(HPF_ERR_INVALID, "cut out of range");
+    int k = 0;
+    for (const MessagePlan& mp : mdl->msg_plan[cut]) k += (mp.from_buffer ? 1 : 0) + (mp.pending >= 0 ? 1 : 0);
+    *n = k;
+    return HPF_OK;
+}
+
+int hpf_backward_message_desc(const hpf_model* mdl, int32_t cut, int32_t j, int32_t* op, int32_t shape[4])
+{
+    if (!mdl || !op || !shape) return fail(HPF_ERR_INVALID, "null");
+    if (cut < 0 || cut >= (int)mdl->cuts.size()) return fail(HPF_ERR_INVALID, "cut out of range");
+    int k = 0;
+    for (const MessagePlan& mp : mdl->msg_plan[cut]) {
+        const int cand[2] = {mp.from_buffer ? mp.tensor : -1, mp.pending};
+        for (int c = 0; c < 2; ++c) {
+            if (cand[c] < 0) continue;
+            if (k++ == j) {
+                *op = cand[c];
+                shape[0] = mdl->b; shape[1] = mdl->ops[cand[c]].H; shape[2] = mdl->ops[cand[c]].W; shape[3] = mdl->ops[cand[c]].C;
+                return HPF_OK;
+            }
+        }
+    }
+    return fail(HPF_ERR_INVALID, "message out of range");
+}
+
 int hpf_backward(hpf_model* mdl)
 {
     if (!mdl) return fail(HPF_ERR_INVALID, "null model");

@@ -292,6 +292,53 @@ def test_forward_and_backward_as_one_graph_give_the_same_bits(streams):
         bd.model.backward()                      # the step is complete: a second backward needs a fresh forward
 
 
+@pytest.mark.parametrize("P,R,cuts", [(2, 1, [12]), (3, 1, [9, 30]), (2, 2, [25])], ids=["two_stages_mid_block_cut", "three_stages", "two_stages_two_replicas"])
+def test_stage_per_gpu_hand_offs_emulated_on_one_gpu(P, R, cuts):
+    """Hybrid parallelism (Section 5.3): every rank binds the same model and runs only its partition's cells; what crosses
+    a cut is copied between the ranks' workspaces.  All ranks are emulated in one process on this GPU (cell by cell, device
+    copies for the hand-offs, a mean over the replicas for the per-partition allreduce): the averaged gradient must equal,
+    bit for bit, what ordinary single-model steps give, and match the oracle."""
+    from paper_1911_05146_b200.hybrid import HybridLayout, Stage, emulate_step
+    ops = wl.resnet_v2_cifar(2)
+    B, M, hwc = 4, 2, (32, 32, 3)
+    theta = wl.draw_params(ops, seed=wl.inputs.SEED_PARAMS + 17, bn_jitter=0.2)
+    layout = HybridLayout(P * R, P)
+    data = [wl.draw_inputs(B, hwc, 10, seed_x=wl.inputs.SEED_X + 30 + r, seed_labels=wl.inputs.SEED_LABELS + 30 + r) for r in range(R)]
+    dev = torch.device("cuda:0")
+    batches = [(torch.from_numpy(x).to(dev), torch.from_numpy(l).to(dev)) for x, l in data]
+    stages = [Stage(ops, (B,) + hwc, cuts, M, torch.from_numpy(theta), layout.coords(rank)[1], dev) for rank in range(layout.world)]
+    slices = emulate_step(stages, layout, batches)
+    # the same batches through ordinary single-model steps, averaged over the replicas the same way
+    singles, losses = [], []
+    for x, l in data:
+        bd = Bound(ops, hwc, B, M, cuts, theta, {hpf.OPT_GRAPH: 0})
+        bd.upload(x, l)
+        losses.append(bd.step())
+        singles.append(bd.avg.clone())
+    mean = singles[0].clone()
+    for g in singles[1:]:
+        mean += g
+    mean /= R
+    for rank, st in enumerate(stages):
+        a, n = st.plan.param_first, st.plan.param_count
+        assert torch.equal(slices[rank], mean[a:a + n]), (rank, float((slices[rank] - mean[a:a + n]).abs().max()))
+    covered = sorted((st.plan.param_first, st.plan.param_count) for st in stages[:P])
+    assert covered[0][0] == 0 and all(covered[k][0] + covered[k][1] == covered[k + 1][0] for k in range(P - 1))
+    assert covered[-1][0] + covered[-1][1] == theta.size
+    # the last partition of every replica holds that replica's losses
+    for r in range(R):
+        got = stages[layout.rank_of(r, P - 1)].losses().cpu().numpy()
+        assert abs(float(got.astype(np.float32).sum() / np.float32(M)) - losses[r]) <= 1e-6 * abs(losses[r])
+    # and against the oracle: the mean over replicas of the oracle's averaged gradients
+    g_ref = np.mean([ora.step(ops, hwc, theta, x, l, M)["g_avg"] for x, l in data], axis=0)
+    full = torch.cat([slices[layout.rank_of(0, p)] for p in range(P)]).cpu().numpy()
+    offs, G = wl.param_offsets(ops)
+    for i, (w_off, w_cnt, b_off, b_cnt) in enumerate(offs):
+        for off, cnt in ((w_off, w_cnt), (b_off, b_cnt)):
+            if cnt:
+                assert rel_l2(full[off:off + cnt], g_ref[off:off + cnt]) <= TOL_TENSOR, ("op", i)
+
+
 def test_messages_across_cuts_match_the_oracle():
     """Activations sent forward and partial errors sent back (Eq. 7) per cut and micro-batch."""
     ops = wl.resnet_v2_cifar(1)
