@@ -1258,6 +1258,7 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                         // fall behind the chain; with four stages the uncapped launch measured faster).
                         ConvBnFuse hint;
                         hint.wgrad_max_ctas = (mdl->P >= 6 && !mdl->side.empty()) ? 32 : 0;
+                        if (const char* v = getenv("HPF_WGRAD_MAX_CTAS")) hint.wgrad_max_ctas = atoi(v);      // experiments
                         CU(conv_tc_prepare(pl, s, pass, mdl->opt_conv_path == 2 ? 1 : mdl->opt_wgrad_passes, mdl->grad(i, m), mdl->act(src, m), nullptr, nullptr,
                                            mdl->gslots + (int64_t)m * mdl->G + o.w_off, nullptr, false, scratch, &hint));
                     }

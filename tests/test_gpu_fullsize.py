@@ -5,18 +5,22 @@ import pytest
 
 import workloads as wl
 from oracle import reference as ora
-from hpf_testlib import Bound, rel_l2, seeded, compare_microbatch, log_parity, TOL_TENSOR, TOL_LOSS
+import paper_1911_05146_b200 as hpf
+from hpf_testlib import (Bound, rel_l2, seeded, compare_microbatch, log_parity, TOL_TENSOR, TOL_LOSS, TAU, TAU_ONE_PASS,
+                         MAX_DECISION_FRACTION, MAX_DECISION_FRACTION_ONE_PASS)
 
 pytestmark = pytest.mark.gpu
 
 
-def _fullsize(name, sample_m):
+def _fullsize(name, sample_m, options=None, one_graph=True):
     c = wl.config(name)
     ops, hwc, B, M = c["ops"], c["in_hwc"], c["B"], c["M"]
     x, labels, theta = seeded(ops, hwc, B)
-    bd = Bound(ops, hwc, B, M, c["cuts"], theta)
+    # the launch configuration the benchmark times: three streams per partition, forward and backward as one graph
+    bd = Bound(ops, hwc, B, M, c["cuts"], theta, options, backward_streams=one_graph)
     bd.upload(x, labels)
-    loss = bd.step()
+    loss = bd.step(one_graph=one_graph)
+    one_pass = (options or {}).get(hpf.OPT_CONV_PATH) == 2
     slots = bd.slots.cpu().numpy()
     offs, G = wl.param_offsets(ops)
     losses = bd.loss_slots()
@@ -24,14 +28,15 @@ def _fullsize(name, sample_m):
     # sampled micro-batches, recomputed one by one: judged by the plain oracle (which takes nothing from the GPU); the
     # oracle under the GPU's in-window ReLU decisions runs beside it as a diagnostic and decides only the gradient
     # tensors that the plain comparison leaves beyond the tolerance
-    res = [compare_microbatch(bd, m, theta, x, labels, slots, offs, float(losses[m])) for m in sample_m]
+    res = [compare_microbatch(bd, m, theta, x, labels, slots, offs, float(losses[m]), tau=TAU_ONE_PASS if one_pass else TAU,
+                              max_fraction=MAX_DECISION_FRACTION_ONE_PASS if one_pass else MAX_DECISION_FRACTION) for m in sample_m]
     # properties that hold at any size: the average is the fixed-order mean of the slots
     acc = slots[0].copy()
     for m in range(1, M):
         acc += slots[m]
     assert np.array_equal(bd.avg.cpu().numpy(), acc * np.float32(1.0 / M))
     assert abs(loss - float(np.sum(losses.astype(np.float32)) / np.float32(M))) <= 1e-6 * abs(loss)
-    log_parity("full size " + name, res)
+    log_parity("full size " + name + (" (one TF32 pass)" if one_pass else ""), res)
     return res
 
 
@@ -64,3 +69,13 @@ def test_resnet110_v1_batch128():
 
 def test_vgg16_batch128():
     _fullsize("vgg16", sample_m=[2])
+
+
+def test_one_tf32_pass_at_depth_110():
+    """HPF_OPT_CONV_PATH = 2: a single TF32 pass (11-bit operands) in the forward and data-gradient convolutions.  At depth
+    110 the forward values hold the tolerance (worst activation 4e-3) and the gradients do under the wider decision window
+    of that path.  Measured at full size on the two workloads whose wide 3x3 convolutions are bound by the tensor pipe, it
+    does NOT: VGG-16's loss is off by 2.1e-3 relative (no batch norm renormalises the error) and the ImageNet-layout
+    ResNet-152 takes 40 ReLU decisions on pre-activations beyond 2 % of the channel's scale.  Three passes stay the default
+    everywhere."""
+    _fullsize("r110", [1], {hpf.OPT_CONV_PATH: 2})
