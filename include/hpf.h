@@ -279,9 +279,11 @@ int hpf_conv_wgrad(const float *d_x, const float *d_dy, float *d_dw, int32_t N, 
  * are processed by ONE cooperative launch that keeps the tensor on chip between the statistics and the apply step; it
  * occupies every SM while it runs.  That launch synchronises its CTAs through words 0-1 of the scratch; the wait is
  * bounded (2 s): if it ever gives up, word 2 of the scratch becomes 1, d_stats (forward) or d_dgamma / d_dbeta
- * (backward) are NaN and the output is not written.  HPF_BN_RESIDENT=0 in the environment keeps all sizes on the
- * two-kernel path. */
+ * (backward) are NaN and the output is not written; the CTAs that arrived are still counted in word 0, so the caller
+ * must zero the first 256 bytes of the scratch again before its next use.  hpf_bnrelu_status copies that flag to the
+ * host (it waits for the device).  HPF_BN_RESIDENT=0 in the environment keeps all sizes on the two-kernel path. */
 int hpf_bnrelu_scratch_bytes(int64_t rows, int32_t C, size_t *bytes);
+int hpf_bnrelu_status(const void *d_scratch, int32_t *h_gave_up);
 int hpf_bnrelu_fwd(const float *d_x, const float *d_gamma, const float *d_beta, float eps, float *d_y,
                    float *d_stats, int64_t rows, int32_t C, void *d_scratch, void *stream);
 /* dx (+= if accumulate) = BN+ReLU backward of dy; d_addend (may be NULL) is added to dx as well

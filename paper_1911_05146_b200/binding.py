@@ -64,6 +64,7 @@ _SIGNATURES = {
     "hpf_sgd_momentum_step": [_vp, _vp, _f32, _f32, _f32],
     "hpf_sgd_momentum_flat": [_vp, _vp, _vp, _vp, _i32, _i64, _f32, _f32, _f32, _vp],
     "hpf_launch_count": [_vp, _pi64],
+    "hpf_bnrelu_status": [_vp, _pi32],
     "hpf_step_bytes": [_vp, C.POINTER(C.c_double)],
     "hpf_cell_times": [_vp, _i32, _pi64],
     "hpf_conv_path_counts": [_vp, _pi64, _pi64],
@@ -297,6 +298,11 @@ class Model:
 
 
 # ---- single kernels on caller buffers -------------------------------------------------------------
+def bnrelu_status(scratch):
+    """True if a bounded wait of a single-op BN call on this scratch gave up (the scratch head must then be zeroed again)."""
+    v = _i32(); _check(lib().hpf_bnrelu_status(_ptr(scratch), C.byref(v))); return bool(v.value)
+
+
 def conv_scratch_bytes(N, H, W, Cc, K, R, stride, pad):
     n = C.c_size_t(); _check(lib().hpf_conv_scratch_bytes(N, H, W, Cc, K, R, stride, pad, C.byref(n))); return n.value
 

@@ -1768,6 +1768,15 @@ int hpf_bnrelu_bwd(const float* d_x, const float* d_dy, const float* d_gamma, co
     return HPF_OK;
 }
 
+int hpf_bnrelu_status(const void* d_scratch, int32_t* h_gave_up)
+{
+    if (!d_scratch || !h_gave_up) return fail(HPF_ERR_INVALID, "null argument");
+    unsigned int words[3] = {0, 0, 0};
+    CU(cudaMemcpy(words, d_scratch, sizeof words, cudaMemcpyDeviceToHost));
+    *h_gave_up = words[2] != 0u;
+    return HPF_OK;
+}
+
 int hpf_sgd_momentum_flat(const float* d_slots, float* d_grad_avg, float* d_params, float* d_velocity, int32_t M, int64_t G,
                           float lr, float momentum, float weight_decay, void* stream)
 {

@@ -917,8 +917,12 @@ struct BnBigPlan { bool ok; int n_clusters, nblk_apply, stream_out; int64_t rows
 template <bool BWD>
 int bn_big_max_clusters()
 {
-    static int cached = -1;
-    if (cached >= 0) return cached;
+    // per device: a process may drive several GPUs, and the answer (like the attributes set below) belongs to one of them
+    static int cached_by_device[64];
+    static bool have[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { (void)cudaGetLastError(); return 0; }
+    if (have[dev]) return cached_by_device[dev];
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(kBnBigCluster * kBnBigMaxPartials); cfg.blockDim = dim3(kBnThreads);
     cudaLaunchAttribute attr[1];
@@ -927,7 +931,7 @@ int bn_big_max_clusters()
     cfg.attrs = attr; cfg.numAttrs = 1;
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, bn_reduce_big_kernel<BWD>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
-    cached = n;
+    cached_by_device[dev] = n; have[dev] = true;
     return n;
 }
 
@@ -1547,6 +1551,26 @@ size_t bn_scratch_bytes(int64_t rows, int C)
     return 256 + ((size_t)p.nblk * 2 * C + 2 * (size_t)C) * sizeof(float);
 }
 
+// The large-tensor apply kernels keep up to 2048 channels of coefficients in dynamic shared memory beyond the default limit.
+// The attribute is set once per device; if that fails the callers stay on the ticket path, which needs none.
+bool big_apply_attributes_set()
+{
+    static signed char state[64];        // 0 not tried, 1 set, -1 failed
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { (void)cudaGetLastError(); return false; }
+    if (state[dev] == 0) {
+        const int mx = (int)bn_big_apply_smem(2048);
+        bool ok = cudaFuncSetAttribute(bn_apply_big_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, mx) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(bn_apply_big_bwd_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(bn_apply_big_bwd_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(bn_apply_big_bwd_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(bn_apply_big_bwd_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx) == cudaSuccess;
+        if (!ok) (void)cudaGetLastError();
+        state[dev] = ok ? 1 : -1;
+    }
+    return state[dev] == 1;
+}
+
 cudaError_t bnrelu_fwd(const float* x, const float* gamma, const float* beta, float eps, float* y, float* stats,
                        int64_t rows, int C, void* scratch, cudaStream_t st, int64_t* n_launch, bool relu)
 {
@@ -1568,10 +1592,8 @@ cudaError_t bnrelu_fwd(const float* x, const float* gamma, const float* beta, fl
         return e;
     }
     const BnBigPlan bp = bn_big_plan<false>(rows, C, p);
-    if (bp.ok) {
-        static bool attr_set = false;
+    if (bp.ok && big_apply_attributes_set()) {
         const size_t smem = bn_big_apply_smem(C);
-        if (!attr_set) { cudaFuncSetAttribute(bn_apply_big_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bn_big_apply_smem(2048)); attr_set = true; }
         launch_cluster_pdl(bn_reduce_big_kernel<false>, bp.n_clusters * kBnBigCluster, kBnThreads, kBnBigCluster, st,
                            reinterpret_cast<const float4*>(x), (const float4*)nullptr, gamma, beta, (const float*)nullptr, rows, C,
                            p.cgt, p.rl, bp.rows_per_blk, partials, floor);
@@ -1626,17 +1648,8 @@ cudaError_t bnrelu_bwd(const float* x, const float* dy, const float* gamma, cons
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + 256);
     float* coef = partials + (size_t)p.nblk * 2 * C;
     const BnBigPlan bp = bn_big_plan<true>(rows, C, p);
-    if (bp.ok) {
-        static bool attr_set = false;
+    if (bp.ok && big_apply_attributes_set()) {
         const size_t smem = bn_big_apply_smem(C);
-        if (!attr_set) {
-            const int mx = (int)bn_big_apply_smem(2048);
-            cudaFuncSetAttribute(bn_apply_big_bwd_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx);
-            cudaFuncSetAttribute(bn_apply_big_bwd_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx);
-            cudaFuncSetAttribute(bn_apply_big_bwd_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx);
-            cudaFuncSetAttribute(bn_apply_big_bwd_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx);
-            attr_set = true;
-        }
         const float4* x4 = reinterpret_cast<const float4*>(x);
         const float4* dy4 = reinterpret_cast<const float4*>(dy);
         const float4* ad4 = reinterpret_cast<const float4*>(addend);

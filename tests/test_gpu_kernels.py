@@ -139,6 +139,7 @@ def test_bnrelu_fwd_bwd(rows, C):
     hpf.bnrelu_bwd(dx_, ddy, dg, db, stats, gx, dadd, 1, ggam, gbet, rows, C, scratch)
     torch.cuda.synchronize()
     assert torch.allclose(gx, base + base + dadd, rtol=1e-5, atol=1e-5)
+    assert hpf.bnrelu_status(scratch) is False           # no bounded wait gave up; the scratch is fit for the next call
 
 
 def test_bnrelu_rejects_odd_channels():
