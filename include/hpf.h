@@ -114,6 +114,11 @@ int hpf_model_destroy(hpf_model *model);
  *   HPF_OPT_BN_CLUSTER     1 (default): the backward of a BN whose micro-batch tensor is small enough to sit in the
  *                          registers of a few thread-block clusters is one launch (the CTAs of a cluster exchange their
  *                          per-channel sums through distributed shared memory); 0: always the reduce + apply pair.
+ *   HPF_OPT_PDL_LATE_FROM  N (default 8): with programmatic dependent launch, the forward convolutions of a cell that runs while at
+ *                          least N cells of the one-graph schedule are under way let their successor be scheduled only when
+ *                          their accumulator is complete, not at their first instruction: a successor scheduled early sits in
+ *                          its SM slots for the whole life of its predecessor, which shortens a lone stage's chain of kernels
+ *                          but costs throughput once every stage is busy.  0: always late; a large N: always early.
  *   HPF_OPT_CELL_CTAS      N > 0: the forward tensor-core convolutions of a (partition, micro-batch) cell that follow each
  *                          other with no other kernel between them run as ONE persistent kernel of N CTAs that stays
  *                          resident for the cell, walks the list of convolutions and meets at a grid-wide barrier between
@@ -122,7 +127,7 @@ int hpf_model_destroy(hpf_model *model);
  *                          are bit-identical to N = 0 when the tile assignment is the same.  0: one launch per convolution. */
 typedef enum { HPF_OPT_GRAPH = 1, HPF_OPT_CONV_PATH = 2, HPF_OPT_SINGLE_STREAM = 3, HPF_OPT_KEEP_MESSAGES = 4,
                HPF_OPT_FUSE_ADD = 5, HPF_OPT_PDL = 6, HPF_OPT_WGRAD_PASSES = 7, HPF_OPT_FUSE_BN = 8, HPF_OPT_CELL_TIMES = 9,
-               HPF_OPT_BN_CLUSTER = 10, HPF_OPT_CELL_CTAS = 11 } hpf_option;
+               HPF_OPT_BN_CLUSTER = 10, HPF_OPT_CELL_CTAS = 11, HPF_OPT_PDL_LATE_FROM = 12 } hpf_option;
 int hpf_set_option(hpf_model *model, int32_t option, int32_t value);
 
 /* ---- integer bookkeeping (Section 5.1 lists, Section 5.3 pipelining) ----------------------------- */

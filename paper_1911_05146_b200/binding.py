@@ -5,7 +5,7 @@ import os
 from . import build as _build
 
 CONV, BNRELU, ADD, MAXPOOL, HEAD, BN, RELU = 1, 2, 3, 4, 5, 6, 7
-OPT_GRAPH, OPT_CONV_PATH, OPT_SINGLE_STREAM, OPT_KEEP_MESSAGES, OPT_FUSE_ADD, OPT_PDL, OPT_WGRAD_PASSES, OPT_FUSE_BN, OPT_CELL_TIMES, OPT_BN_CLUSTER, OPT_CELL_CTAS = 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11
+OPT_GRAPH, OPT_CONV_PATH, OPT_SINGLE_STREAM, OPT_KEEP_MESSAGES, OPT_FUSE_ADD, OPT_PDL, OPT_WGRAD_PASSES, OPT_FUSE_BN, OPT_CELL_TIMES, OPT_BN_CLUSTER, OPT_CELL_CTAS, OPT_PDL_LATE_FROM = 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12
 
 
 class HpfError(RuntimeError):

@@ -275,6 +275,7 @@ struct FwdScalars {
     float* bn_in_y;              // relu(bn(x)), dense [N][in_h][in_w][c_in], written by the CTAs of the first channel slice
     // K loop split over gridDim.z CTAs (launches of a few tiles with a long K loop): every CTA stores its partial tile, the
     // one that takes the last ticket of its (tile, channel slice) adds them in split order and writes the output
+    int pdl_late;                // see the kernel's first statement
     int ksplit;
     float* splitk_partials;      // [(tile * slices + slice) * ksplit + z][128][n_chunk]
     unsigned int* splitk_ticket; // one per (tile, slice); zero between launches
@@ -745,6 +746,7 @@ __device__ __forceinline__ int conv_fwd_cta(const FwdParams* gpp, FwdScalars& p,
             row_fill[tid] = (valid && p.zero_fill > 1 && p.zero_fill <= 4) ? fill : 0;
         }
         mbar_wait(accum_bar + 8 * tj, 0, &abort_flag);
+        if (!CELL && tj == 0 && p.pdl_late) pdl_launch_dependents();
         asm volatile("bar.sync 1, 256;" ::: "memory");
         const bool done = abort_flag == 0;             // uniform over the 8 warps after the barrier
         all_done = all_done && done;
@@ -993,7 +995,11 @@ template <bool MULTI, bool KSPLIT = false>
 __global__ void __launch_bounds__(320, 2) conv_tc_fwd_kernel(const __grid_constant__ FwdParams gp)
 {
     __shared__ FwdScalars p;                 // scalar parameters, see load_scalars
-    pdl_launch_dependents();
+    // Programmatic launch: the next kernel of the stream may be scheduled once every CTA of this one has said so.  Early (here):
+    // the successor's set-up hides under this kernel, which shortens a lone stage's chain of kernels.  Late (when the first
+    // accumulator is complete, see below): the successor's CTAs do not sit in SM slots for the whole life of this kernel,
+    // which is what counts when every stage is busy and slots are what the stages compete for.  The host chooses per launch.
+    if (!gp.s.pdl_late) pdl_launch_dependents();
     load_scalars(&p, &gp.s);
     __syncthreads();
     conv_fwd_cta<MULTI ? 1 : (KSPLIT ? 2 : 0)>(&gp, p, make_uint3(blockIdx.x, blockIdx.y, blockIdx.z), make_uint3(gridDim.x, gridDim.y, gridDim.z), 0u, true);
@@ -1906,6 +1912,7 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
         while (t > 2 && (unsigned int)t * p.acc_cols > 256u) --t;
         p.tiles_per_cta = t < 2 ? 2 : t;
     }
+    p.pdl_late = fuse && fuse->pdl_late ? 1 : 0;
     p.ksplit = 1;
     if (fuse && fuse->splitk && !fuse->mode && !fuse->in_mode && p.tiles_per_cta == 1) {
         const int S = splitk_factor(p.n_tiles, v.c_out / n_chunk, total, kchunk / 8);

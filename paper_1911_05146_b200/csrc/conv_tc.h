@@ -60,6 +60,9 @@ struct ConvBnFuse {
     size_t splitk_bytes = 0;
     // > 0: the launch will run inside a persistent cell kernel of this many CTAs (conv_tc_cell_launch): tiles per CTA are
     // chosen so that the launch is one round of that grid where tensor and shared memory allow
+    // forward / data gradient: programmatic launch of the kernel's successor when the first accumulator is complete
+    // instead of at the kernel's first instruction
+    int pdl_late = 0;
     int cell_ctas = 0;
     unsigned int cell_smem = 0;          // dynamic shared memory such a CTA may use (0: what lets two of them share an SM)
 };

@@ -110,6 +110,7 @@ struct hpf_model {
         bool ready = false;
     };
     int opt_cell = 0;          // CTAs of a persistent forward cell kernel; 0: every convolution is its own launch
+    int opt_pdl_late_from = 8;   // forward cells that run while at least this many cells are under way trigger their successors late
     std::vector<CellRun> cell_runs;
     std::vector<int> cell_of_op;              // conv -> run, or -1
     std::vector<size_t> cell_bar_off;         // per partition: the grid barrier's two words (zeroed at bind)
@@ -731,6 +732,23 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
 // the cell that feeds it has finished - backward (p+1, m), or forward (P-1, m) for the last partition - while the
 // partition's forward stream may still be busy with later micro-batches.  Same kernels on the same data as the two
 // phases, so the results are bit-identical; only the idle slots of the forward drain and the backward fill get used.
+// Cells under way, roughly, while cell (p, m) of the forward (bwd = false) or backward phase runs in the one-graph schedule:
+// the stages busy at its own tick plus those of the other phase at the tick that runs at the same time (the backward
+// pipeline starts when the first micro-batch has passed all P stages).
+int cells_under_way(int P, int M, int p, int m, bool bwd)
+{
+    auto busy = [&](int t) {
+        if (t < 0 || t > P + M - 2) return 0;
+        int n = t + 1;
+        if (n > P) n = P;
+        if (n > M) n = M;
+        if (n > P + M - 1 - t) n = P + M - 1 - t;
+        return n;
+    };
+    const int t = bwd ? (P - 1 - p) + m : p + m;
+    return bwd ? busy(t) + busy(t + P) : busy(t) + busy(t - P);
+}
+
 int enqueue_phase(hpf_model* mdl, int phase)
 {
     const PdlScope pdl_scope(mdl->opt_pdl);
@@ -958,6 +976,7 @@ int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
     case HPF_OPT_FUSE_BN: if (value < 0 || value > 3) return fail(HPF_ERR_INVALID, "0..3"); mdl->opt_fuse_bn = value; break;
     case HPF_OPT_CELL_TIMES: mdl->opt_cell_times = value != 0; break;
     case HPF_OPT_BN_CLUSTER: mdl->opt_bn_cluster = value != 0; break;
+    case HPF_OPT_PDL_LATE_FROM: if (value < 0) return fail(HPF_ERR_INVALID, ">= 0"); mdl->opt_pdl_late_from = value; break;
     case HPF_OPT_CELL_CTAS: if (value < 0 || value > 148) return fail(HPF_ERR_INVALID, "0..148 CTAs"); mdl->opt_cell = value; break;
     case HPF_OPT_WGRAD_PASSES: if (value != 1 && value != 3) return fail(HPF_ERR_INVALID, "1 or 3 passes"); mdl->opt_wgrad_passes = value; break;
     default: return fail(HPF_ERR_INVALID, "unknown option");
@@ -1199,6 +1218,7 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                     }
                     ConvBnFuse fuse;
                     if (mdl->splitk_bytes[o.part]) { fuse.splitk = mdl->ws + mdl->splitk_off[o.part]; fuse.splitk_bytes = mdl->splitk_bytes[o.part]; }
+                    fuse.pdl_late = cells_under_way(mdl->P, M, o.part, m, false) >= mdl->opt_pdl_late_from;
                     if (mdl->cell_of_op[i] >= 0) {
                         fuse.cell_ctas = mdl->opt_cell;
                         fuse.cell_smem = mdl->cell_runs[mdl->cell_of_op[i]].smem_budget;
@@ -1258,7 +1278,6 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                         // fall behind the chain; with four stages the uncapped launch measured faster).
                         ConvBnFuse hint;
                         hint.wgrad_max_ctas = (mdl->P >= 6 && !mdl->side.empty()) ? 32 : 0;
-                        if (const char* v = getenv("HPF_WGRAD_MAX_CTAS")) hint.wgrad_max_ctas = atoi(v);      // experiments
                         CU(conv_tc_prepare(pl, s, pass, mdl->opt_conv_path == 2 ? 1 : mdl->opt_wgrad_passes, mdl->grad(i, m), mdl->act(src, m), nullptr, nullptr,
                                            mdl->gslots + (int64_t)m * mdl->G + o.w_off, nullptr, false, scratch, &hint));
                     }
