@@ -572,9 +572,10 @@ def main():
     # where the step's time goes: the three phases timed apart (a diagnostic; events on stream 0, which every phase joins)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
     phase_ms = [0.0, 0.0, 0.0]
-    model.forward(dx, dl); model.backward(); model.grad_average()          # untimed: the two-phase graphs may not exist yet
-    barrier()
-    for _ in range(3):
+    if not args.profile:
+        model.forward(dx, dl); model.backward(); model.grad_average()          # untimed: the two-phase graphs may not exist yet
+        barrier()
+    for _ in range(0 if args.profile else 3):
         ev[0].record(s0); model.forward(dx, dl); ev[1].record(s0); model.backward(); ev[2].record(s0); model.grad_average(); ev[3].record(s0)
         barrier()
         for k in range(3):
