@@ -291,6 +291,51 @@ def kernel_roofline(torch, hpf, cfg, pk):
                     "the batch-128 sweep (--workload conv_sweep) gives the bandwidth-bound figures" % ((b * P * P + 127) // 128)}
 
 
+def run_hybrid(args, cfg, torch, hpf, dist, rank, local, world, dev):
+    """Hybrid parallelism across the GPUs of the job: rank = replica * P + partition.  One step = every rank's cells of its
+    partition for all micro-batches, the hand-offs, the micro-batch average and the per-partition allreduce over replicas."""
+    from paper_1911_05146_b200.hybrid import HybridLayout, Stage, TorchDistComm, SingleRankComm, run_step
+    P = args.hybrid_partitions
+    layout = HybridLayout(world, P)
+    replica, part = layout.coords(rank)
+    ops, hwc, B, M = cfg["ops"], cfg["in_hwc"], cfg["B"], cfg["M"]
+    x, labels, theta = replica_inputs(cfg, replica)
+    cuts = wl.default_cuts(len(ops), P)
+    stage = Stage(ops, (B,) + tuple(hwc), cuts, M, torch.from_numpy(theta), part, dev)
+    comm = TorchDistComm(layout, rank) if world > 1 else SingleRankComm()
+    dx, dl = torch.from_numpy(x).to(dev), torch.from_numpy(labels).to(dev)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        run_step(stage, layout, rank, comm, dx, dl)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        run_step(stage, layout, rank, comm, dx, dl)          # ends with a host wait for this rank's slice
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        ms, = max_over_ranks(dist, [ms], dev)
+    if rank == 0:
+        ms_step = ms / args.steps
+        print(json.dumps({"metric": METRIC, "value": layout.R * B / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                          "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                          "dtype": "tf32", "data": "synthetic",
+                          "config": {"workload": NAMES[args.workload], "global_batch": layout.R * B, "micro_batches": M, "partitions": P,
+                                     "parallelism": "hybrid: %d replica(s) x %d partitions, one partition per GPU; NCCL send / recv across "
+                                                    "cuts, one allreduce group per partition" % (layout.R, P),
+                                     "cut_points": list(cuts), "graph": False}}), flush=True)
+    if dist is not None:
+        dist.barrier(); dist.destroy_process_group()
+
+
 def conv_sweep(args):
     """Configuration 2: the bottleneck convolution shapes at batch 128, forward / data gradient / weight
     gradient each, through the C ABI on rotating operand sets that together exceed L2.  One JSON line with
@@ -460,6 +505,10 @@ def main():
     ap.add_argument("--conv-path", type=int, default=0)
     ap.add_argument("--cell-ctas", type=int, default=-1,
                     help="CTAs of the persistent forward cell kernels (HPF_OPT_CELL_CTAS); 0: one launch per convolution; -1: the library's default")
+    ap.add_argument("--hybrid-partitions", type=int, default=0,
+                    help="N GPUs as N / P replicas of a P-stage pipeline, one partition per GPU (paper_1911_05146_b200.hybrid): "
+                         "activations and partial errors by NCCL send / recv, one allreduce group per partition.  Not the default "
+                         "(the default for N > 1 is independent replicas) and not yet measured on hardware.")
     ap.add_argument("--two-phases", action="store_true",
                     help="hpf_forward then hpf_backward (backward after the forward drain) instead of hpf_forward_backward")
     ap.add_argument("--opt", action="append", default=[], help="library option as NUMBER=VALUE (hpf_set_option), repeatable")
@@ -501,6 +550,9 @@ def main():
     dev = torch.device("cuda", local)
     pk = peaks()
 
+    if args.hybrid_partitions > 0:
+        run_hybrid(args, cfg, torch, hpf, dist, rank, local, world, dev)
+        return
     ops, hwc, B, M = cfg["ops"], cfg["in_hwc"], cfg["B"], cfg["M"]
     x, labels, theta = replica_inputs(cfg, rank)          # each replica its own batch, shared parameters
     cuts = cfg["cuts"]

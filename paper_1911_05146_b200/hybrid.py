@@ -144,10 +144,15 @@ class TorchDistComm:
             self.groups[p] = dist.new_group(ranks) if len(ranks) > 1 else None
 
     def send(self, tensor, dst):
+        # the caller has waited for the producing kernels; the copy engine / NCCL reads a finished tensor
         self.dist.send(tensor.contiguous(), dst)
 
     def recv(self, tensor, src):
         self.dist.recv(tensor, src)
+        if tensor.is_cuda:
+            # NCCL completes on its own stream: the cell that reads the tensor is enqueued on the stage's stream only
+            # after the data has landed
+            torch.cuda.current_stream(tensor.device).synchronize()
 
     def all_reduce_mean(self, tensor, partition):
         g = self.groups[partition]
@@ -158,6 +163,19 @@ class TorchDistComm:
         else:
             self.dist.all_reduce(tensor, op=self.dist.ReduceOp.SUM, group=g)     # gloo (CPU tests) has no averaging reduction
             tensor /= self.layout.R
+
+
+class SingleRankComm:
+    """The communicator of a world of one rank: nothing to send, nothing to average."""
+
+    def send(self, tensor, dst):
+        raise RuntimeError("a single rank has no neighbour")
+
+    def recv(self, tensor, src):
+        raise RuntimeError("a single rank has no neighbour")
+
+    def all_reduce_mean(self, tensor, partition):
+        pass
 
 
 def run_step(stage, layout, rank, comm, x=None, labels=None):

@@ -339,6 +339,22 @@ def test_stage_per_gpu_hand_offs_emulated_on_one_gpu(P, R, cuts):
                 assert rel_l2(full[off:off + cnt], g_ref[off:off + cnt]) <= TOL_TENSOR, ("op", i)
 
 
+def test_one_rank_of_the_hybrid_step_is_the_ordinary_step():
+    """hybrid.run_step on a world of one rank (one replica, one partition): the same cells, the library's average, no
+    neighbour and no allreduce; bit for bit the ordinary step without a CUDA graph."""
+    from paper_1911_05146_b200.hybrid import HybridLayout, Stage, SingleRankComm, run_step
+    c = wl.config("r11")
+    ops, hwc, B, M = c["ops"], c["in_hwc"], c["B"], c["M"]
+    x, labels, theta = seeded(ops, hwc, B, seed=2)
+    dev = torch.device("cuda:0")
+    stage = Stage(ops, (B,) + tuple(hwc), [], M, torch.from_numpy(theta), 0, dev)
+    g = run_step(stage, HybridLayout(1, 1), 0, SingleRankComm(), torch.from_numpy(x).to(dev), torch.from_numpy(labels).to(dev))
+    bd = Bound(ops, hwc, B, M, [], theta, {hpf.OPT_GRAPH: 0})
+    bd.upload(x, labels)
+    bd.step()
+    assert g.numel() == theta.size and torch.equal(g, bd.avg)
+
+
 def test_messages_across_cuts_match_the_oracle():
     """Activations sent forward and partial errors sent back (Eq. 7) per cut and micro-batch."""
     ops = wl.resnet_v2_cifar(1)
