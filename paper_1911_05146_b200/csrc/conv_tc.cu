@@ -835,6 +835,7 @@ __device__ __forceinline__ int conv_fwd_cta(const FwdParams* gpp, FwdScalars& p,
                 if (accumulate) { const float4 e = *reinterpret_cast<const float4*>(outp + row_off[0] + 4 * c4k); sk.x += e.x; sk.y += e.y; sk.z += e.z; sk.w += e.w; }
                 if (tid < c4n) shift_s[tid] = sk;          // read again when the tile's moments are formed
             }
+            if (tid == 0 && tj == 0) HPF_TL(12);
             for (int base = tid; base < total4; base += 1024) {
                 float4 o[4];
                 int off[4];
@@ -885,6 +886,7 @@ __device__ __forceinline__ int conv_fwd_cta(const FwdParams* gpp, FwdScalars& p,
                 }
             }
             }   // write_out
+            if (tid == 0 && tj == 0) HPF_TL(13);
             if (p.stat_mode) {
                 const int c4n = p.n_chunk >> 2;
                 const int stat_mode = p.stat_mode;
@@ -907,6 +909,7 @@ __device__ __forceinline__ int conv_fwd_cta(const FwdParams* gpp, FwdScalars& p,
                     red[2 * tid] = sa; red[2 * tid + 1] = sb;
                 }
                 asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (tid == 0 && tj == 0) HPF_TL(14);
                 if (tid < ((c4n * 2 + 31) & ~31)) {          // whole warps: the swap below is a warp shuffle
                     // threads 2g and 2g+1 add group g's rows of shifted sums and of shifted squares, swap the totals, and store
                     // the tile's mean (from the sums and the group's shift, which thread g keeps: fetched through shared memory)

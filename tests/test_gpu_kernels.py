@@ -71,6 +71,41 @@ def test_conv_launches_of_several_waves_use_two_tiles_per_cta(shape):
     assert max(e) <= 2e-5, e
 
 
+@pytest.mark.parametrize("shape", wl.conv_sweep_shapes(), ids=lambda s: "k%d_s%d_%dto%d_at%d" % s)
+def test_conv_sweep_at_batch_128_sampled_against_the_oracle(shape):
+    """Configuration 2 in the launch configuration the sweep benchmark times (batch 128, three-pass path: several tiles per
+    CTA, K splits and channel slices as the planner chooses them at that size).  Forward and data gradient are independent
+    per image, so the oracle recomputes three sampled images; the weight gradient sums over the batch, so the oracle
+    recomputes it whole."""
+    ks, st, ci, co, H = shape
+    N, pad = 128, (1 if ks == 3 else 0)
+    rng = np.random.Generator(np.random.PCG64(4242 + ks * 1000 + ci + 7 * co + H))
+    x = rng.standard_normal((N, H, H, ci)).astype(np.float32)
+    w = (rng.standard_normal((co, ks, ks, ci)) * np.sqrt(2.0 / (ci * ks * ks))).astype(np.float32)
+    P = (H + 2 * pad - ks) // st + 1
+    dy = rng.standard_normal((N, P, P, co)).astype(np.float32)
+    dx_, dw_, dy_ = _dev(x), _dev(w), _dev(dy)
+    scratch = torch.zeros(hpf.conv_scratch_bytes(N, H, H, ci, co, ks, st, pad), dtype=torch.uint8, device=DEV)
+    y = torch.full((N, P, P, co), float("nan"), device=DEV)
+    gx = torch.full((N, H, H, ci), float("nan"), device=DEV)
+    gw = torch.full((co, ks, ks, ci), float("nan"), device=DEV)
+    wprep = torch.empty(4 * dw_.numel(), device=DEV)
+    args = (N, H, H, ci, co, ks, st, pad, 0)
+    hpf.conv_prepare_weights(dw_, wprep, ci, co, ks)
+    for _ in range(2):                      # twice: tickets of K-split launches must be left clean
+        hpf.conv_fwd(dx_, dw_, wprep, y, *args, scratch)
+        hpf.conv_dgrad(dy_, dw_, wprep, gx, *args, scratch)
+        hpf.conv_wgrad(dx_, dy_, gw, *args, scratch)
+    torch.cuda.synchronize()
+    assert scratch[-256:-248].view(torch.int32).cpu().tolist() == [0, 0]
+    yh, gxh = y.cpu().numpy(), gx.cpu().numpy()
+    assert np.isfinite(yh).all() and np.isfinite(gxh).all()
+    for n in (0, 77, 127):
+        assert rel_l2(yh[n:n + 1], ora.conv_fwd(x[n:n + 1], w, st, pad)) <= 2e-5, ("fwd", n)
+        assert rel_l2(gxh[n:n + 1], ora.conv_dgrad(dy[n:n + 1], w, (1, H, H, ci), st, pad)) <= 2e-5, ("dgrad", n)
+    assert rel_l2(gw.cpu().numpy(), ora.conv_wgrad(x, dy, ks, st, pad)) <= 5e-5
+
+
 @pytest.mark.parametrize("shape", [(3, 1, 64, 64, 56), (1, 1, 256, 64, 56), (1, 2, 256, 128, 56), (3, 1, 128, 128, 28),
                                    (1, 1, 128, 512, 28), (3, 1, 256, 256, 14), (1, 2, 1024, 512, 14), (3, 1, 512, 512, 7),
                                    (1, 1, 512, 2048, 7), (1, 1, 2048, 512, 7)],
