@@ -581,7 +581,7 @@ def main():
     ws_bytes = model.workspace_bytes()
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     # stage streams + weight-gradient side streams + backward streams (the one-graph schedule)
-    streams = [torch.cuda.Stream(device=dev) for _ in range((2 if args.two_phases else 3) * model.num_partitions())]
+    streams = [torch.cuda.Stream(device=dev) for _ in range((2 if args.two_phases else 3) * model.num_stream_slots())]
     torch.cuda.synchronize()
     model.bind(params, slots, avg, ws, streams)
     dx, dl = torch.from_numpy(x).to(dev), torch.from_numpy(labels).to(dev)

@@ -119,6 +119,18 @@ int hpf_model_destroy(hpf_model *model);
  *                          their accumulator is complete, not at their first instruction: a successor scheduled early sits in
  *                          its SM slots for the whole life of its predecessor, which shortens a lone stage's chain of kernels
  *                          but costs throughput once every stage is busy.  0: always late; a large N: always early.
+ *   HPF_OPT_STAGE_LANES    L (default 1): a stage keeps up to L of its micro-batches under way at once, micro-batch m on lane
+ *                          m mod L, every lane with its own streams and scratch memory.  L = 1 is the schedule of Section 5.3
+ *                          as the paper's one-process-per-partition runs it: a stage works through its micro-batches one
+ *                          after the other, and P + M - 1 ticks pass before the last cell ends.  On one GPU the stages share
+ *                          the same SMs, so nothing forces that order: with L > 1 the cells (p, m) and (p, m + 1) may run side
+ *                          by side, the hand-offs between stages are unchanged, and the idle slots of the pipeline's fill and
+ *                          drain get used.  Every cell computes on the same data with the same kernels: results are
+ *                          bit-identical for every L.  hpf_bind then wants its streams per (partition, lane).
+ *   HPF_OPT_WGRAD_DIRECT   1 (default): the tensor-core weight gradient hands its TMA tiles (pixels x channels, channels
+ *                          innermost) to the tensor core as MN-major operands, as they land in shared memory; 0: the earlier
+ *                          kernel, which transposes every tile in shared memory first (kept as a cross-check; also used for
+ *                          channel counts that are neither 16 nor a multiple of 32).
  *   HPF_OPT_CELL_CTAS      N > 0: the forward tensor-core convolutions of a (partition, micro-batch) cell that follow each
  *                          other with no other kernel between them run as ONE persistent kernel of N CTAs that stays
  *                          resident for the cell, walks the list of convolutions and meets at a grid-wide barrier between
@@ -127,12 +139,15 @@ int hpf_model_destroy(hpf_model *model);
  *                          are bit-identical to N = 0 when the tile assignment is the same.  0: one launch per convolution. */
 typedef enum { HPF_OPT_GRAPH = 1, HPF_OPT_CONV_PATH = 2, HPF_OPT_SINGLE_STREAM = 3, HPF_OPT_KEEP_MESSAGES = 4,
                HPF_OPT_FUSE_ADD = 5, HPF_OPT_PDL = 6, HPF_OPT_WGRAD_PASSES = 7, HPF_OPT_FUSE_BN = 8, HPF_OPT_CELL_TIMES = 9,
-               HPF_OPT_BN_CLUSTER = 10, HPF_OPT_CELL_CTAS = 11, HPF_OPT_PDL_LATE_FROM = 12 } hpf_option;
+               HPF_OPT_BN_CLUSTER = 10, HPF_OPT_CELL_CTAS = 11, HPF_OPT_PDL_LATE_FROM = 12,
+               HPF_OPT_STAGE_LANES = 13, HPF_OPT_WGRAD_DIRECT = 14 } hpf_option;
 int hpf_set_option(hpf_model *model, int32_t option, int32_t value);
 
 /* ---- integer bookkeeping (Section 5.1 lists, Section 5.3 pipelining) ----------------------------- */
 int hpf_num_ops(const hpf_model *model, int32_t *n_ops);
 int hpf_num_partitions(const hpf_model *model, int32_t *P);
+/* S = P * min(HPF_OPT_STAGE_LANES, M): hpf_bind takes S, 2S or 3S streams */
+int hpf_num_stream_slots(const hpf_model *model, int32_t *S);
 int hpf_num_params(const hpf_model *model, int64_t *G);
 /* Offsets (in floats) into the flat parameter / gradient vectors: ops in list order; CONV weights
  * [c_out][r][s][c_in]; BNRELU gamma[C] then beta[C]; HEAD W[classes][C] then bias[classes]. */
@@ -165,7 +180,8 @@ int hpf_workspace_bytes(const hpf_model *model, size_t *bytes);
  * cuda_streams: n_streams >= P cudaStream_t handles (stage p runs on stream p; stream 0 is the one
  * the phases fork from and join to).  With n_streams >= 2P, stream P+p carries stage p's weight-gradient
  * kernels, which feed only the final average and so leave the chain of dependent kernels; with n_streams >= 3P,
- * stream 2P+p carries stage p's backward cells in hpf_forward_backward.  Creates
+ * stream 2P+p carries stage p's backward cells in hpf_forward_backward.  With HPF_OPT_STAGE_LANES = L > 1 read
+ * S = P * min(L, M) for P throughout: lane l of stage p is stream slot p * min(L, M) + l.  Creates
  * events and tensor-map descriptors; allocates nothing on the device.  Errors: HPF_ERR_WORKSPACE, HPF_ERR_INVALID, HPF_ERR_CUDA. */
 int hpf_bind(hpf_model *model, float *d_params, float *d_grad_slots, float *d_grad_avg, void *d_workspace,
              size_t ws_bytes, void *const *cuda_streams, int32_t n_streams);
@@ -259,7 +275,8 @@ int hpf_conv_path_counts(const hpf_model *model, int64_t *n_tensor, int64_t *n_c
  * All pointers are device pointers, `stream` is a cudaStream_t.  x [N][H][W][C], w [K][R][R][C],
  * y/dy [N][P][Q][K] with P = (H+2*pad-R)/stride+1.  path: 0 = tensor cores, three-pass TF32;
  * 2 = tensor cores, one TF32 pass (both HPF_ERR_UNSUPPORTED when the shape is outside their reach);
- * 1 = CUDA cores.  d_scratch: caller-owned scratch of at least hpf_conv_scratch_bytes(), zeroed ONCE by the caller (e.g.
+ * 1 = CUDA cores; hpf_conv_wgrad also takes 3 and 4: as 0 and 2 with the kernel that transposes its tiles in shared
+ * memory instead of handing them to the tensor core as MN-major operands (a cross-check).  d_scratch: caller-owned scratch of at least hpf_conv_scratch_bytes(), zeroed ONCE by the caller (e.g.
  * allocated zeroed) and used by one stream at a time.  Its last 256 bytes are the device status of the tensor-core
  * kernels: a kernel whose bounded wait gives up stores a non-zero code there (first failure wins) and nothing ever
  * clears it.  Launches that split a long K loop over several CTAs keep their tickets in it and leave them at zero.

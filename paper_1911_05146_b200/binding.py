@@ -5,7 +5,7 @@ import os
 from . import build as _build
 
 CONV, BNRELU, ADD, MAXPOOL, HEAD, BN, RELU = 1, 2, 3, 4, 5, 6, 7
-OPT_GRAPH, OPT_CONV_PATH, OPT_SINGLE_STREAM, OPT_KEEP_MESSAGES, OPT_FUSE_ADD, OPT_PDL, OPT_WGRAD_PASSES, OPT_FUSE_BN, OPT_CELL_TIMES, OPT_BN_CLUSTER, OPT_CELL_CTAS, OPT_PDL_LATE_FROM = 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12
+OPT_GRAPH, OPT_CONV_PATH, OPT_SINGLE_STREAM, OPT_KEEP_MESSAGES, OPT_FUSE_ADD, OPT_PDL, OPT_WGRAD_PASSES, OPT_FUSE_BN, OPT_CELL_TIMES, OPT_BN_CLUSTER, OPT_CELL_CTAS, OPT_PDL_LATE_FROM, OPT_STAGE_LANES, OPT_WGRAD_DIRECT = 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14
 
 
 class HpfError(RuntimeError):
@@ -31,6 +31,7 @@ _SIGNATURES = {
     "hpf_set_option": [_vp, _i32, _i32],
     "hpf_num_ops": [_vp, _pi32],
     "hpf_num_partitions": [_vp, _pi32],
+    "hpf_num_stream_slots": [_vp, _pi32],
     "hpf_num_params": [_vp, _pi64],
     "hpf_param_layout": [_vp, _i32, _pi64, _pi64, _pi64, _pi64],
     "hpf_op_shape": [_vp, _i32, _pi32],
@@ -176,6 +177,9 @@ class Model:
 
     def num_partitions(self):
         p = _i32(); _check(lib().hpf_num_partitions(self._h, C.byref(p))); return p.value
+
+    def num_stream_slots(self):
+        s = _i32(); _check(lib().hpf_num_stream_slots(self._h, C.byref(s))); return s.value
 
     def param_layout(self, op):
         a, b, c, d = _i64(), _i64(), _i64(), _i64()

@@ -185,6 +185,17 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
            ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (layout << 61);
 }
 
+// MN-major TF32 operand (the reduction index runs over the rows of the tile, channels are contiguous): the one layout
+// the tensor core accepts for 32-bit MN-major operands is rows of 128 bytes whose 32-byte chunks are XOR-swizzled by
+// (row % 4) (layout type 1, what a TMA box with CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B delivers).  One MMA of K = 8 reads
+// 8 consecutive rows (two groups of 4, `stride` = 512 bytes apart) of every 32-channel block; `block_bytes` is the
+// distance between consecutive 32-channel blocks (the leading-dimension offset).
+__device__ __forceinline__ uint64_t smem_desc_mn(uint32_t addr, uint32_t block_bytes)
+{
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)((block_bytes >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((512u >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (1ull << 61);
+}
+
 // Instruction descriptor: fp32 accumulator, TF32 A and B, M = 128, N = n; major bits select MN-major operands.
 inline uint32_t instr_desc(int n, bool a_mn_major, bool b_mn_major)
 {
@@ -307,6 +318,27 @@ struct alignas(64) WgradParams {
     CUtensorMap tm_a;            // dy {c_out, Q, P, N}, box {m_chunk, w, h, n}, no swizzle
     CUtensorMap tm_b;            // x {C, Wv, Hv, N}, box {n_cols, w, h, n}, no swizzle
     WgradScalars s;
+};
+
+struct WgradDirectScalars {
+    float* out;                  // dw or partials [splits][c_out*taps*c_in]
+    DeviceStatus* status;
+    int box_w, box_h, box_n, tiles_w, tiles_h, n_tiles, tiles_per_split;
+    int rows;                    // pixel rows of a tile in shared memory (a multiple of 8)
+    int box_rows;                // pixels the copy delivers (<= rows); the rest stays zero
+    int c_out, c_in, R, pad;
+    int m_chunk, n_cols;         // output / input channels per CTA
+    int m_blocks, n_blocks;      // 32-channel blocks of the dy tile / of one tap's x tile (a 16-channel tensor fills half a block)
+    int m_box, n_box;            // channels per TMA box: 32, or 16 for a 16-channel tensor
+    int taps_per_cta, taps_per_mma;
+    int stages, passes;
+    unsigned int stage_bytes, lo_off, tx_bytes_a, tx_per_tap, tmem_cols, idesc, idesc_tail;
+    long long split_stride;      // floats between partials
+};
+struct alignas(64) WgradDirectParams {
+    CUtensorMap tm_a;            // dy {c_out, Q, P, N}, box {m_box, w, h, n}, 128-byte swizzle with 32-byte atoms
+    CUtensorMap tm_b;            // x {C, Wv, Hv, N}, box {n_box, w, h, n}, same swizzle
+    WgradDirectScalars s;
 };
 
 template <class T>
@@ -1356,6 +1388,225 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
     if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
 }
 
+// ------------------------------------------------------------------------------------------------
+// weight-gradient kernel without the transposition: the tensor core reads the TMA tiles as they land
+// ------------------------------------------------------------------------------------------------
+// dW[co][tap][ci] = sum over pixels of dy[pixel][co] * x[pixel + tap][ci]: the reduction runs over pixels, and both
+// tensors keep channels innermost in memory, so both operands are MN-major.  A TMA box of 32 channels x `rows` pixels with
+// the 32-byte-atom swizzle is exactly the tile the tensor core wants (smem_desc_mn): 6 warps = TMA producer, MMA issuer and
+// 4 warps that only read the accumulators at the end (with three passes they also split every tile into hi and lo, in
+// place and position by position - no transposition either).  A 16-channel tensor is copied with 16-channel boxes: the
+// copy still gives every pixel a 128-byte row and leaves its second half alone; those columns and lanes of the
+// accumulator hold products of whatever the shared memory held and are never read.  An MMA always reads 128 operand
+// rows = 4 blocks from the dy tile's base: blocks beyond the tile's own are the x tile or what follows it, and land in
+// accumulator lanes nobody reads.
+__global__ void __launch_bounds__(192) conv_tc_wgrad_direct_kernel(const __grid_constant__ WgradDirectParams gp)
+{
+    __shared__ WgradDirectScalars p;
+    pdl_launch_dependents();
+    load_scalars(&p, &gp.s);
+    __syncthreads();
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[3 * 8 + 1];       // full[8], empty[8], split[8], accum
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ int issued, consumed;
+
+    const uint32_t base_off = ((smem_u32(smem_raw) + 1023u) & ~1023u) - smem_u32(smem_raw);
+    uint8_t* smem = smem_raw + base_off;
+    const uint32_t smem_base = smem_u32(smem);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[8]), split0 = smem_u32(&bars[16]), accum_bar = smem_u32(&bars[24]);
+
+    const int split = blockIdx.x;
+    const int tap0 = blockIdx.y * p.taps_per_cta;
+    const int m_chunks = p.c_out / p.m_chunk;
+    const int m0 = (blockIdx.z % m_chunks) * p.m_chunk;
+    const int cn0 = (blockIdx.z / m_chunks) * p.n_cols;
+    int ntaps = p.R * p.R - tap0;
+    if (ntaps > p.taps_per_cta) ntaps = p.taps_per_cta;
+    const int tile_begin = split * p.tiles_per_split;
+    int tile_end = tile_begin + p.tiles_per_split;
+    if (tile_end > p.n_tiles) tile_end = p.n_tiles;
+    const int total = tile_end - tile_begin;
+    const uint32_t block_bytes = (uint32_t)p.rows * 128u;                 // one 32-channel block of a tile
+    const uint32_t a_bytes = (uint32_t)p.m_blocks * block_bytes;          // the dy tile
+    const uint32_t tap_bytes = (uint32_t)p.n_blocks * block_bytes;        // one tap's x tile
+    const int slot = p.n_blocks * 32;                                     // accumulator columns of one tap
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 8; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); mbar_init(split0 + 8 * s, 4); }
+        mbar_init(accum_bar, 1);
+        abort_flag = 0; issued = 0; consumed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), p.tmem_cols);
+    if (p.box_rows < p.rows) {
+        // A pixel box that is not a multiple of 8 pixels leaves the last rows of every block untouched by the copies:
+        // zeroed once, they add nothing to the sums over pixels.
+        const int pad_rows = p.rows - p.box_rows;
+        const int blocks = p.m_blocks + ntaps * p.n_blocks;
+        for (int s = 0; s < p.stages; ++s)
+            for (int part = 0; part < (p.passes == 3 ? 2 : 1); ++part)
+                for (int b = 0; b < blocks; ++b) {
+                    float* blk = reinterpret_cast<float*>(smem + s * p.stage_bytes + part * p.lo_off + b * block_bytes) + p.box_rows * 32;
+                    for (int i = threadIdx.x; i < pad_rows * 32; i += blockDim.x) blk[i] = 0.f;
+                }
+        fence_async_smem();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    pdl_wait();              // everything above touched only parameters, shared and tensor memory
+    const uint32_t tmem_base = tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- TMA producer ----
+            const int stages = p.stages, tiles_w = p.tiles_w, tiles_h = p.tiles_h, R = p.R, pad = p.pad;
+            const int box_w = p.box_w, box_h = p.box_h, box_n = p.box_n, m_blocks = p.m_blocks, n_blocks = p.n_blocks;
+            const int m_box = p.m_box, n_box = p.n_box;
+            const uint32_t stage_bytes = p.stage_bytes, tx = p.tx_bytes_a + (uint32_t)ntaps * p.tx_per_tap;
+            int tw, th, tn;
+            { int t = tile_begin; tw = t % tiles_w; t /= tiles_w; th = t % tiles_h; tn = t / tiles_h; }
+            const int r_first = tap0 / R, sx_first = tap0 - r_first * R;
+            int it = 0, s = 0;
+            uint32_t par = 1u;
+            for (; it < total; ++it) {
+                if (!mbar_wait(empty0 + 8 * s, par, &abort_flag)) { report(p.status, 3); break; }
+                const int q0 = tw * box_w, p0 = th * box_h, n0 = tn * box_n;
+                uint32_t dst = smem_base + s * stage_bytes;
+                const uint32_t bar = full0 + 8 * s;
+                mbar_expect_tx(bar, tx);
+                for (int b = 0; b < m_blocks; ++b, dst += block_bytes) tma_load_4d(dst, &gp.tm_a, bar, m0 + b * m_box, q0, p0, n0);
+                int r = r_first, sx = sx_first;
+                for (int tp = 0; tp < ntaps; ++tp) {
+                    for (int b = 0; b < n_blocks; ++b, dst += block_bytes)
+                        tma_load_4d(dst, &gp.tm_b, bar, cn0 + b * n_box, q0 + sx - pad, p0 + r - pad, n0);
+                    if (++sx == R) { sx = 0; ++r; }
+                }
+                if (++tw == tiles_w) { tw = 0; if (++th == tiles_h) { th = 0; ++tn; } }
+                if (++s == stages) { s = 0; par ^= 1u; }
+            }
+            issued = it;
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- MMA issuer ----
+            const int stages = p.stages, k8n = p.rows >> 3;
+            const bool three = p.passes == 3;
+            const uint32_t ready0 = three ? split0 : full0;
+            int it = 0, s = 0;
+            uint32_t par = 0;
+            for (; it < total; ++it) {
+                if (!mbar_wait(ready0 + 8 * s, par, &abort_flag)) { report(p.status, 4); break; }
+                tc_fence_after();
+                const uint32_t a_src = smem_base + s * p.stage_bytes, b_src = a_src + a_bytes;
+                // taps are consecutive blocks of the x operand: groups of up to 256 accumulator columns per MMA
+                for (int tg = 0; tg < ntaps; tg += p.taps_per_mma) {
+                    const int nt = ntaps - tg < p.taps_per_mma ? ntaps - tg : p.taps_per_mma;
+                    const uint32_t idesc = nt == p.taps_per_mma ? p.idesc : p.idesc_tail;
+                    const uint32_t acc = tmem_base + (uint32_t)(tg * slot);
+                    const uint32_t b_tg = b_src + (uint32_t)tg * tap_bytes;
+                    for (int k8 = 0; k8 < k8n; ++k8) {
+                        const uint64_t ad = smem_desc_mn(a_src + 1024u * k8, block_bytes);
+                        const uint64_t bd = smem_desc_mn(b_tg + 1024u * k8, block_bytes);
+                        umma_tf32(acc, ad, bd, idesc, (it | k8) ? 1u : 0u);
+                        if (three) {
+                            const uint64_t adl = smem_desc_mn(a_src + p.lo_off + 1024u * k8, block_bytes);
+                            const uint64_t bdl = smem_desc_mn(b_tg + p.lo_off + 1024u * k8, block_bytes);
+                            umma_tf32(acc, adl, bd, idesc, 1u);
+                            umma_tf32(acc, ad, bdl, idesc, 1u);
+                        }
+                    }
+                }
+                umma_commit(empty0 + 8 * s);
+                if (++s == stages) { s = 0; par ^= 1u; }
+            }
+            if (!three) consumed = it;
+            if (it == total) umma_commit(accum_bar);
+        }
+    } else {
+        const int tid = threadIdx.x - 64;
+        bool ok = true;
+        if (p.passes == 3) {
+            // ---- splitters: hi stays where the copy put it, lo goes to the stage's second half, same position ----
+            const int stages = p.stages;
+            // 16-byte pieces of the dy tile and of the x tiles.  A tile of a 16-channel tensor holds data in one half of
+            // every 128-byte row only (which half: bit 1 of the row number, the swizzle's doing): 4 pieces per row then.
+            const int a_half = p.m_box == 16, b_half = p.n_box == 16;
+            const int a4 = (int)(a_bytes >> 4) >> a_half;
+            const int n4 = a4 + ((int)(((uint32_t)(ntaps * p.n_blocks) * block_bytes) >> 4) >> b_half);
+            int it = 0, s = 0;
+            uint32_t par = 0;
+            for (; it < total && ok; ++it) {
+                ok = mbar_wait(full0 + 8 * s, par, &abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) { if (lane == 0) report(p.status, 5); break; }
+                float4* hi = reinterpret_cast<float4*>(smem + s * p.stage_bytes);
+                float4* lo = reinterpret_cast<float4*>(smem + s * p.stage_bytes + p.lo_off);
+                for (int i = tid; i < n4; i += 128) {
+                    int j;                                  // the piece's place among the stage's 16-byte pieces
+                    if (i < a4) j = a_half ? ((i >> 2) << 3) + ((i >> 3) & 1) * 4 + (i & 3) : i;
+                    else {
+                        const int k = i - a4;
+                        j = (int)(a_bytes >> 4) + (b_half ? ((k >> 2) << 3) + ((k >> 3) & 1) * 4 + (k & 3) : k);
+                    }
+                    const float4 v = hi[j];
+                    const float4 h = make_float4(tf32_hi(v.x), tf32_hi(v.y), tf32_hi(v.z), tf32_hi(v.w));
+                    hi[j] = h;
+                    lo[j] = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
+                }
+                fence_async_smem();     // generic-proxy writes -> tensor-core reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(split0 + 8 * s);
+                if (++s == stages) { s = 0; par ^= 1u; }
+            }
+            if (tid == 0) consumed = it;
+        }
+        // ---- epilogue ----
+        bool done = ok && mbar_wait(accum_bar, 0, &abort_flag);
+        done = __all_sync(0xffffffffu, done);
+        if (done) {
+            tc_fence_after();
+            const int row = (warp & 3) * 32 + lane;          // TMEM lane = output channel within the chunk
+            const bool valid = row < p.m_chunk;
+            const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+            float* obase = p.out + (long long)split * p.split_stride + ((long long)(m0 + row) * p.R * p.R) * p.c_in + cn0;
+            if ((warp & 3) * 32 < p.m_chunk)                 // a whole warp of lanes beyond the chunk has nothing to read
+                for (int tp = 0; tp < ntaps; ++tp)
+                    for (int c0 = 0; c0 < p.n_cols; c0 += 16) {
+                        float v[16];
+                        tmem_ld16(lane_addr + (uint32_t)(tp * slot + c0), v);
+                        if (valid) {
+                            // a gradient slot starts at m*G floats: 16-byte aligned only if G is a multiple of 4
+                            float* o = obase + (long long)(tap0 + tp) * p.c_in + c0;
+                            if ((reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
+#pragma unroll
+                                for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(o + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) o[j] = v[j];
+                            }
+                        }
+                    }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (abort_flag && threadIdx.x == 0) {
+        // copies in flight must land before the shared memory is given back
+        for (int it = consumed; it < issued; ++it) {
+            const int s = it % p.stages;
+            const long long t0 = clock64();
+            while (!mbar_try_wait(full0 + 8 * s, (it / p.stages) & 1) && clock64() - t0 < kWaitLimit) {}
+        }
+    }
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, p.tmem_cols);
+}
+
 // dw[i] = sum over splits of partials[z][i], in an order fixed by the launch shape: thread (lane, zl) adds the
 // splits zl, zl+8, ... ascending, then the 8 partial sums are added ascending.  32 float4 per block.
 __global__ void __launch_bounds__(256)
@@ -1539,6 +1790,7 @@ bool fwd_view(const ConvShape& s, int pass, FwdView* v)
     return true;
 }
 
+constexpr int kSwizzle128Atom32 = 1;      // encode(): rows of 128 bytes, 32-byte chunks XOR-swizzled by (row % 4)
 cudaError_t encode(CUtensorMap* tm, const float* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
                    const cuuint32_t* box, int swizzle_bytes)
 {
@@ -1547,9 +1799,36 @@ cudaError_t encode(CUtensorMap* tm, const float* base, int rank, const cuuint64_
     CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<float*>(base), dims, strides_bytes, box,
                           ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
                           swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
-                          : (swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE),
+                          : (swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                             : (swizzle_bytes == kSwizzle128Atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_NONE)),
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+// How many pixel splits (CTAs along x) a weight-gradient launch of n_tiles pixel tiles gets.
+void wgrad_splits(const ConvShape& s, int n_tiles, int ctas_per_split, int max_ctas, int* splits_out, int* tiles_per_split_out)
+{
+    const int taps = s.R * s.R;
+    // enough CTAs to spread the pixel walk, few enough that the partials stay a fraction of the operand bytes
+    const double operand_bytes = 4.0 * ((double)s.N * s.P * s.Q * s.K + (double)s.N * s.P * s.Q * s.C);
+    const double dw_bytes = 4.0 * (double)s.K * taps * s.C;
+    int splits = n_tiles / 4;
+    int cap = (int)(operand_bytes / (4.0 * dw_bytes));
+    // small problems are latency bound, not byte bound: spread the pixel walk over several dozen CTAs
+    const int want = (kWgradWantCtas + ctas_per_split - 1) / ctas_per_split;
+    if (cap < want) cap = want;
+    if (splits > cap) splits = cap;
+    if (splits > 296) splits = 296;          // two CTAs per SM
+    if (max_ctas > 0) {
+        // the caller wants the launch to take little SM time (CTAs x (fixed cost + tiles)) rather than to be short
+        int ms = max_ctas / ctas_per_split;
+        if (ms < 1) ms = 1;
+        if (splits > ms) splits = ms;
+    }
+    if (splits > n_tiles / 2) splits = n_tiles / 2;
+    if (splits < 1) splits = 1;
+    *tiles_per_split_out = (n_tiles + splits - 1) / splits;
+    *splits_out = (n_tiles + *tiles_per_split_out - 1) / *tiles_per_split_out;
 }
 
 struct WgradGeom {
@@ -1605,27 +1884,84 @@ bool wgrad_geom(const ConvShape& s, int passes, WgradGeom* g, int max_ctas = 0)
     g->tmem_cols = pow2_cols(g->taps_per_cta * g->n_cols);
     const int tiles_w = (s.Q + g->box.w - 1) / g->box.w, tiles_h = (s.P + g->box.h - 1) / g->box.h, tiles_n = (s.N + g->box.n - 1) / g->box.n;
     g->n_tiles = tiles_w * tiles_h * tiles_n;
-    // splits: enough CTAs to spread the pixel walk, few enough that the partials stay a fraction of the operand bytes
-    const double operand_bytes = 4.0 * ((double)s.N * s.P * s.Q * s.K + (double)s.N * s.P * s.Q * s.C);
-    const double dw_bytes = 4.0 * (double)s.K * taps * s.C;
-    int splits = g->n_tiles / 4;
-    int cap = (int)(operand_bytes / (4.0 * dw_bytes));
-    // small problems are latency bound, not byte bound: spread the pixel walk over several dozen CTAs
-    const int ctas_per_split = g->tap_groups * (s.K / g->m_chunk) * (s.C / g->n_cols);
-    const int want = (kWgradWantCtas + ctas_per_split - 1) / ctas_per_split;
-    if (cap < want) cap = want;
-    if (splits > cap) splits = cap;
-    if (splits > 296) splits = 296;          // two CTAs per SM
-    if (max_ctas > 0) {
-        // the caller wants the launch to take little SM time (CTAs x (fixed cost + tiles)) rather than to be short
-        int ms = max_ctas / ctas_per_split;
-        if (ms < 1) ms = 1;
-        if (splits > ms) splits = ms;
+    wgrad_splits(s, g->n_tiles, g->tap_groups * (s.K / g->m_chunk) * (s.C / g->n_cols), max_ctas, &g->splits, &g->tiles_per_split);
+    return true;
+}
+
+struct WgradDirectGeom {
+    PixelBox box;
+    int m_chunk, n_cols, m_blocks, n_blocks, m_box, n_box, taps_per_cta, tap_groups, stages, splits, tiles_per_split, n_tiles, rows_padded;
+    unsigned int stage_bytes, lo_off, slack, tmem_cols;
+};
+
+// Geometry of the kernel that reads its TMA tiles directly: output channels per CTA (up to 128), input channels per CTA
+// (all up to 256, else 128 or 64), taps per CTA (all, one row of the window, or one) and pixels per tile (128, 64 or 32):
+// the first combination whose accumulators take at most half of an SM's tensor memory (other kernels' CTAs share the
+// SM) and that gets at least three pipeline stages into 100 KB of shared memory - failing that two stages, failing
+// that two stages into 200 KB with all of the tensor memory.
+bool wgrad_direct_geom(const ConvShape& s, int passes, WgradDirectGeom* g, int max_ctas = 0)
+{
+    if (s.C % 16 || s.K % 16) return false;
+    if ((s.C > 16 && s.C % 32) || (s.K > 16 && s.K % 32)) return false;
+    if (s.R != 1 && s.R != 3) return false;
+    if (s.R == 3 && (s.stride != 1 || s.pad != 1)) return false;
+    if (s.R == 1 && s.pad != 0) return false;
+    if (s.stride < 1 || s.stride > 2) return false;
+    // measured: nine taps of a 16-channel tensor, split into hi and lo, are faster through the transposing kernel (its
+    // tiles of such a tensor are dense; here every pixel of it takes a 128-byte row)
+    if (passes == 3 && s.R == 3 && (s.C == 16 || s.K == 16)) return false;
+    g->m_chunk = s.K < 128 ? s.K : 128;
+    if (s.K % g->m_chunk) return false;
+    g->m_blocks = (g->m_chunk + 31) / 32;
+    g->m_box = g->m_chunk < 32 ? g->m_chunk : 32;
+    const int taps = s.R * s.R;
+    const unsigned int parts = passes == 3 ? 2u : 1u;
+    bool found = false;
+    const int ncand[3] = {s.C < 256 ? s.C : 256, 128, 64};
+    const int cand[3] = {taps, taps == 9 ? 3 : 1, 1};
+    const unsigned int budgets[3] = {100u * 1024u, 100u * 1024u, 200u * 1024u};
+    const unsigned int tmem_caps[3] = {256u, 256u, 512u};
+    const int min_stages[3] = {3, 2, 2};
+    for (int tier = 0; tier < 3 && !found; ++tier) {
+        // three passes double every stage and put the hi / lo split on the four spare warps: two stages are then too few
+        // to keep the tensor core fed, and the launch does better alone on an SM with long tiles
+        if (tier == 1 && passes == 3) continue;
+        for (int ni = 0; ni < 3 && !found; ++ni) {
+            const int n_cols = ncand[ni];
+            if (n_cols > s.C || s.C % n_cols || (ni > 0 && n_cols >= ncand[0])) continue;
+            const int n_blocks = (n_cols + 31) / 32;
+            for (int ci = 0; ci < 3 && !found; ++ci) {
+                const int tpc = cand[ci];
+                if (ci > 0 && tpc >= cand[0]) continue;
+                if ((unsigned int)(tpc * n_blocks * 32) > tmem_caps[tier]) continue;
+                for (int rows = 128; rows >= 32 && !found; rows >>= 1) {
+                    PixelBox b;
+                    if (!choose_box(s.Q, s.P, s.N, rows, 1, &b)) continue;
+                    const int padded = (b.rows + 7) / 8 * 8;
+                    const unsigned int half = (unsigned int)padded * 128u * (unsigned int)(g->m_blocks + tpc * n_blocks);
+                    const unsigned int stage = parts * half;
+                    // the dy operand is read as 4 blocks whatever it holds; in the last stage what follows the x tile is
+                    // read too: room for that behind the last stage
+                    const int stage_blocks = g->m_blocks + tpc * n_blocks;
+                    const unsigned int slack = stage_blocks < 4 ? (unsigned int)(4 - stage_blocks) * (unsigned int)padded * 128u : 0u;
+                    const int want_stages = min_stages[tier];
+                    if ((unsigned int)want_stages * stage + slack > budgets[tier]) continue;
+                    int st = (int)((budgets[tier] - slack) / stage);
+                    if (st > 4) st = 4;
+                    g->n_cols = n_cols; g->n_blocks = n_blocks; g->n_box = n_cols < 32 ? n_cols : 32;
+                    g->taps_per_cta = tpc;
+                    g->box = b; g->rows_padded = padded; g->stage_bytes = stage; g->lo_off = half; g->slack = slack; g->stages = st;
+                    found = true;
+                }
+            }
+        }
     }
-    if (splits > g->n_tiles / 2) splits = g->n_tiles / 2;
-    if (splits < 1) splits = 1;
-    g->tiles_per_split = (g->n_tiles + splits - 1) / splits;
-    g->splits = (g->n_tiles + g->tiles_per_split - 1) / g->tiles_per_split;
+    if (!found) return false;
+    g->tap_groups = (taps + g->taps_per_cta - 1) / g->taps_per_cta;
+    g->tmem_cols = pow2_cols(g->taps_per_cta * g->n_blocks * 32);
+    const int tiles_w = (s.Q + g->box.w - 1) / g->box.w, tiles_h = (s.P + g->box.h - 1) / g->box.h, tiles_n = (s.N + g->box.n - 1) / g->box.n;
+    g->n_tiles = tiles_w * tiles_h * tiles_n;
+    wgrad_splits(s, g->n_tiles, g->tap_groups * (s.K / g->m_chunk) * (s.C / g->n_cols), max_ctas, &g->splits, &g->tiles_per_split);
     return true;
 }
 
@@ -1693,6 +2029,8 @@ cudaError_t conv_tc_init()
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(conv_tc_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWgradSmemBudget + 2048);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(conv_tc_wgrad_direct_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWgradSmemBudget + 2048);
+    if (e != cudaSuccess) return e;
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
     return cudaSuccess;
 }
@@ -1748,12 +2086,18 @@ size_t conv_tc_scratch_bytes(const ConvShape& s)
         if (!wgrad_geom(s, passes, &g)) continue;
         const size_t b = g.splits > 1 ? (size_t)g.splits * s.K * s.R * s.R * s.C * sizeof(float) : 0;
         if (b > need) need = b;
+        WgradDirectGeom d;
+        if (!wgrad_direct_geom(s, passes, &d)) continue;
+        const size_t bd = d.splits > 1 ? (size_t)d.splits * s.K * s.R * s.R * s.C * sizeof(float) : 0;
+        if (bd > need) need = bd;
     }
     return need;
 }
 
 struct ConvTcFwdLaunch { FwdParams p; dim3 grid; unsigned int smem; };
 struct ConvTcWgradLaunch { WgradParams p; dim3 grid; unsigned int smem; int splits; float* dw; long long n_out; };
+struct ConvTcWgradDirectLaunch { WgradDirectParams p; dim3 grid; unsigned int smem; int splits; float* dw; long long n_out; };
+static_assert(sizeof(ConvTcWgradDirectLaunch) <= sizeof(((ConvTcPlan*)0)->storage), "plan storage too small");
 static_assert(sizeof(ConvTcFwdLaunch) <= sizeof(((ConvTcPlan*)0)->storage) && sizeof(ConvTcWgradLaunch) <= sizeof(((ConvTcPlan*)0)->storage),
               "plan storage too small");
 
@@ -1761,8 +2105,52 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
                             const float* w_hi, const float* w_lo, float* out, const float* extra, bool accumulate, void* scratch,
                             const ConvBnFuse* fuse)
 {
-    plan->valid = 0; plan->s = s; plan->pass = pass;
+    plan->valid = 0; plan->s = s; plan->pass = pass; plan->direct = 0;
     if (passes != 1 && passes != 3) return cudaErrorInvalidValue;
+    WgradDirectGeom dg;
+    if (pass == PASS_WGRAD && !(fuse && fuse->wgrad_transposing) && wgrad_direct_geom(s, passes, &dg, fuse ? fuse->wgrad_max_ctas : 0)) {
+        ConvTcWgradDirectLaunch* L = reinterpret_cast<ConvTcWgradDirectLaunch*>(plan->storage);
+        WgradDirectParams& P = L->p;
+        memset(&P, 0, sizeof P);
+        WgradDirectScalars& p = P.s;
+        {   // dy {K, Q, P, N}
+            cuuint64_t dims[4] = {(cuuint64_t)s.K, (cuuint64_t)s.Q, (cuuint64_t)s.P, (cuuint64_t)s.N};
+            cuuint64_t str[3] = {(cuuint64_t)s.K * 4, (cuuint64_t)s.Q * s.K * 4, (cuuint64_t)s.P * s.Q * s.K * 4};
+            cuuint32_t box[4] = {(cuuint32_t)dg.m_box, (cuuint32_t)dg.box.w, (cuuint32_t)dg.box.h, (cuuint32_t)dg.box.n};
+            cudaError_t e = encode(&P.tm_a, in, 4, dims, str, box, kSwizzle128Atom32);
+            if (e != cudaSuccess) return e;
+        }
+        {   // x {C, Wv, Hv, N}: a strided 1x1 convolution samples every stride-th pixel
+            const int wv = s.stride == 1 ? s.W : s.Q, hv = s.stride == 1 ? s.H : s.P;
+            cuuint64_t dims[4] = {(cuuint64_t)s.C, (cuuint64_t)wv, (cuuint64_t)hv, (cuuint64_t)s.N};
+            cuuint64_t str[3] = {(cuuint64_t)s.stride * s.C * 4, (cuuint64_t)s.stride * s.W * s.C * 4, (cuuint64_t)s.H * s.W * s.C * 4};
+            cuuint32_t box[4] = {(cuuint32_t)dg.n_box, (cuuint32_t)dg.box.w, (cuuint32_t)dg.box.h, (cuuint32_t)dg.box.n};
+            cudaError_t e = encode(&P.tm_b, in2, 4, dims, str, box, kSwizzle128Atom32);
+            if (e != cudaSuccess) return e;
+        }
+        const long long n_out = (long long)s.K * s.R * s.R * s.C;
+        p.out = dg.splits > 1 ? reinterpret_cast<float*>(scratch) : out;
+        p.box_w = dg.box.w; p.box_h = dg.box.h; p.box_n = dg.box.n;
+        p.tiles_w = (s.Q + dg.box.w - 1) / dg.box.w; p.tiles_h = (s.P + dg.box.h - 1) / dg.box.h;
+        p.n_tiles = dg.n_tiles; p.tiles_per_split = dg.tiles_per_split; p.rows = dg.rows_padded; p.box_rows = dg.box.rows;
+        p.c_out = s.K; p.c_in = s.C; p.R = s.R; p.pad = s.pad;
+        p.m_chunk = dg.m_chunk; p.n_cols = dg.n_cols; p.m_blocks = dg.m_blocks; p.n_blocks = dg.n_blocks; p.m_box = dg.m_box; p.n_box = dg.n_box;
+        p.taps_per_cta = dg.taps_per_cta; p.stages = dg.stages; p.passes = passes;
+        p.stage_bytes = dg.stage_bytes; p.lo_off = dg.lo_off;
+        p.tx_bytes_a = (unsigned int)dg.box.rows * dg.m_chunk * 4u; p.tx_per_tap = (unsigned int)dg.box.rows * dg.n_cols * 4u;
+        p.tmem_cols = dg.tmem_cols;
+        const int slot = dg.n_blocks * 32;
+        p.taps_per_mma = 256 / slot < dg.taps_per_cta ? 256 / slot : dg.taps_per_cta;
+        p.idesc = instr_desc(slot * p.taps_per_mma, true, true);
+        p.idesc_tail = instr_desc(slot * (dg.taps_per_cta % p.taps_per_mma ? dg.taps_per_cta % p.taps_per_mma : p.taps_per_mma), true, true);
+        p.split_stride = n_out;
+        L->grid = dim3(dg.splits, dg.tap_groups, (s.K / dg.m_chunk) * (s.C / dg.n_cols));
+        L->smem = (unsigned int)dg.stages * dg.stage_bytes + dg.slack + 1024;
+        L->splits = dg.splits; L->dw = out; L->n_out = n_out;
+        plan->direct = 1;
+        plan->valid = 1;
+        return cudaSuccess;
+    }
     if (pass == PASS_WGRAD) {
         WgradGeom g;
         if (!wgrad_geom(s, passes, &g, fuse ? fuse->wgrad_max_ctas : 0)) return cudaErrorNotSupported;
@@ -1941,6 +2329,18 @@ cudaError_t conv_tc_prepare(ConvTcPlan* plan, const ConvShape& s, int pass, int 
 cudaError_t conv_tc_launch(const ConvTcPlan* plan, DeviceStatus* status, cudaStream_t st, int64_t* n_launch)
 {
     if (!plan->valid) return cudaErrorInvalidValue;
+    if (plan->pass == PASS_WGRAD && plan->direct) {
+        ConvTcWgradDirectLaunch L = *reinterpret_cast<const ConvTcWgradDirectLaunch*>(plan->storage);
+        L.p.s.status = status;
+        launch_pdl(conv_tc_wgrad_direct_kernel, L.grid, dim3(192), L.smem, st, L.p);
+        count(n_launch, 1);
+        if (L.splits > 1) {
+            const int nb = (int)((L.n_out / 4 + 31) / 32);
+            launch_pdl(wgrad_partials_reduce_kernel, dim3(nb), dim3(256), 0, st, (const float*)L.p.s.out, L.dw, L.n_out, L.splits);
+            count(n_launch, 1);
+        }
+        return cudaGetLastError();
+    }
     if (plan->pass == PASS_WGRAD) {
         ConvTcWgradLaunch L = *reinterpret_cast<const ConvTcWgradLaunch*>(plan->storage);
         L.p.s.status = status;

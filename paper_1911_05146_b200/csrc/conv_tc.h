@@ -20,6 +20,7 @@ struct ConvTcPlan {
     ConvShape s;
     int pass;
     int valid;
+    int direct;          // weight gradient: the kernel that feeds the TMA tiles to the tensor core as they land
     alignas(64) unsigned char storage[896];
 };
 
@@ -50,6 +51,8 @@ struct ConvBnFuse {
     // weight gradient only: > 0 caps the CTAs of the launch (fewer pixel splits, each walking more tiles): less SM time
     // at a longer duration, for launches that run beside a chain of latency-bound kernels
     int wgrad_max_ctas = 0;
+    // weight gradient only: 1 keeps the kernel that transposes its tiles in shared memory (a cross-check)
+    int wgrad_transposing = 0;
     const float* in_partials = nullptr;
     int in_tiles = 0;
     long long in_rows = 0;

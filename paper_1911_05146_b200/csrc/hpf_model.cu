@@ -110,6 +110,14 @@ struct hpf_model {
         bool ready = false;
     };
     int opt_cell = 0;          // CTAs of a persistent forward cell kernel; 0: every convolution is its own launch
+    // Stage lanes: a stage keeps up to `lanes` of its micro-batches under way at once, micro-batch m on lane m % lanes; every
+    // lane has its own streams and its own scratch, so cells of different lanes share nothing but the parameters.  One
+    // lane is the paper's schedule (a stage works through its micro-batches one after the other).
+    int opt_wgrad_direct = 1;   // weight gradients read their TMA tiles as MN-major operands (0: the kernel that transposes them)
+    int opt_lanes = 1;
+    int lanes() const { return opt_lanes < M ? opt_lanes : M; }
+    int n_slots() const { return P * lanes(); }
+    int slot_of(int p, int m) const { return p * lanes() + m % lanes(); }
     int opt_pdl_late_from = 8;   // forward cells that run while at least this many cells are under way trigger their successors late
     std::vector<CellRun> cell_runs;
     std::vector<int> cell_of_op;              // conv -> run, or -1
@@ -120,7 +128,7 @@ struct hpf_model {
     std::vector<std::vector<MessagePlan>> msg_plan;   // per cut
     // memory plan (byte offsets into the workspace)
     std::vector<size_t> act_off, grad_off, stats_off;   // [m * n_ops + op]
-    std::vector<size_t> bn_scratch_off, conv_scratch_off;   // per stream
+    std::vector<size_t> bn_scratch_off, conv_scratch_off;   // per stream slot (partition, lane)
     std::vector<size_t> splitk_off, splitk_bytes;            // per stream: tickets + partial tiles of K-split convolutions (zeroed at bind)
     // the backward kernels of a partition have scratch of their own: in the one-graph schedule (hpf_forward_backward) a
     // partition's backward cells run while its forward cells of later micro-batches are still under way
@@ -138,7 +146,8 @@ struct hpf_model {
     char* ws = nullptr;
     std::vector<cudaStream_t> streams;
     std::vector<cudaEvent_t> ev_fwd, ev_bwd;  // [cut * M + m]
-    std::vector<cudaEvent_t> ev_join;         // per stream
+    std::vector<cudaEvent_t> ev_join;         // per stream slot
+    std::vector<cudaEvent_t> ev_prep;         // per partition: prepared weights ready (the other lanes wait for lane 0)
     std::vector<cudaStream_t> side;           // per partition: weight-gradient stream (empty: none)
     std::vector<cudaStream_t> bwd_streams;    // per partition: the backward cells' stream in the one-graph schedule (empty: none)
     std::vector<cudaEvent_t> ev_fdone, ev_bjoin;   // forward (P-1, m) done; backward stream p done
@@ -165,17 +174,17 @@ struct hpf_model {
     float* act(int op, int m) const { return reinterpret_cast<float*>(ws + act_off[(size_t)m * n_ops + op]); }
     float* grad(int op, int m) const { return reinterpret_cast<float*>(ws + grad_off[(size_t)m * n_ops + op]); }
     float* stats(int op, int m) const { return reinterpret_cast<float*>(ws + stats_off[(size_t)m * n_ops + op]); }
-    float* bn_partials(int bn) const
+    float* bn_partials(int bn, int m) const
     {
         const int p = ops[bn].part;
-        return reinterpret_cast<float*>(ws + bn_scratch_off[p] + 256 + (size_t)bn_buf[bn] * bn_part_bytes[p]);
+        return reinterpret_cast<float*>(ws + bn_scratch_off[slot_of(p, m)] + 256 + (size_t)bn_buf[bn] * bn_part_bytes[p]);
     }
     unsigned long long* cell_time_slot(int phase, int p, int m) const
     {
         return reinterpret_cast<unsigned long long*>(ws + cell_times_off) + 2 * (((size_t)(phase == PH_BWD) * P + p) * M + m);
     }
     int64_t numel(int op) const { const OpInfo& o = ops[op]; return (int64_t)b * o.H * o.W * o.C; }
-    cudaStream_t stream_of(int p) const { return opt_single ? streams[0] : streams[p]; }
+    cudaStream_t stream_of(int p, int m = 0) const { return opt_single ? streams[0] : streams[slot_of(p, m)]; }
     DeviceStatus* status() const { return reinterpret_cast<DeviceStatus*>(ws + status_off); }
 };
 
@@ -477,8 +486,9 @@ void build_memory_plan(hpf_model* mdl)
     // region that must start as zeros: status word and BN tickets (with their partials)
     mdl->zero_lo = at;
     mdl->status_off = take(sizeof(DeviceStatus));
-    mdl->bn_scratch_off.assign(P, 0);
-    mdl->conv_scratch_off.assign(P, 0);
+    const int L = mdl->lanes(), S = P * L;
+    mdl->bn_scratch_off.assign(S, 0);
+    mdl->conv_scratch_off.assign(S, 0);
     mdl->bn_part_bytes.assign(P, 0);
     for (int p = 0; p < P; ++p) {
         size_t bn = 256, part = 0;
@@ -495,9 +505,9 @@ void build_memory_plan(hpf_model* mdl)
             }
         mdl->bn_part_bytes[p] = part;
         if (256 + 2 * part > bn) bn = 256 + 2 * part;
-        mdl->bn_scratch_off[p] = take(bn);
+        for (int l = 0; l < L; ++l) mdl->bn_scratch_off[p * L + l] = take(bn);
     }
-    mdl->splitk_off.assign(P, 0); mdl->splitk_bytes.assign(P, 0);
+    mdl->splitk_off.assign(S, 0); mdl->splitk_bytes.assign(P, 0);
     for (int p = 0; p < P; ++p) {
         size_t need = 0;
         if (mdl->opt_conv_path != 1)
@@ -507,19 +517,21 @@ void build_memory_plan(hpf_model* mdl)
                     need = std::max(need, std::max(conv_tc_splitk_bytes(s, PASS_FWD, 3), conv_tc_splitk_bytes(s, PASS_DGRAD, 3)));
                 }
         mdl->splitk_bytes[p] = need;
-        mdl->splitk_off[p] = take(need ? need : 16);
+        for (int l = 0; l < L; ++l) mdl->splitk_off[p * L + l] = take(need ? need : 16);
     }
-    mdl->bn_scratch_bwd_off.assign(P, 0); mdl->splitk_bwd_off.assign(P, 0);
+    mdl->bn_scratch_bwd_off.assign(S, 0); mdl->splitk_bwd_off.assign(S, 0);
     for (int p = 0; p < P; ++p) {
         size_t bn = 256;
         for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i)
             if (mdl->ops[i].op.kind == HPF_OP_BNRELU || mdl->ops[i].op.kind == HPF_OP_BN)
                 bn = std::max(bn, bn_scratch_bytes((int64_t)mdl->b * mdl->ops[i].H * mdl->ops[i].W, mdl->ops[i].C));
-        mdl->bn_scratch_bwd_off[p] = take(bn);
-        mdl->splitk_bwd_off[p] = take(mdl->splitk_bytes[p] ? mdl->splitk_bytes[p] : 16);
+        for (int l = 0; l < L; ++l) {
+            mdl->bn_scratch_bwd_off[p * L + l] = take(bn);
+            mdl->splitk_bwd_off[p * L + l] = take(mdl->splitk_bytes[p] ? mdl->splitk_bytes[p] : 16);
+        }
     }
-    mdl->cell_bar_off.assign(P, 0);
-    for (int p = 0; p < P; ++p) mdl->cell_bar_off[p] = take(16);
+    mdl->cell_bar_off.assign(S, 0);
+    for (int k = 0; k < S; ++k) mdl->cell_bar_off[k] = take(16);
     mdl->zero_hi = at;
     build_cell_runs(mdl);
     for (auto& run : mdl->cell_runs) {
@@ -536,7 +548,7 @@ void build_memory_plan(hpf_model* mdl)
                 if (need2 > need) need = need2;
                 if (need > cv) cv = need;
             }
-        mdl->conv_scratch_off[p] = take(cv);
+        for (int l = 0; l < L; ++l) mdl->conv_scratch_off[p * L + l] = take(cv);
     }
     mdl->cell_times_off = take(sizeof(unsigned long long) * 2 * 2 * (size_t)P * M);
     mdl->loss_slots_off = take(sizeof(float) * M);
@@ -602,7 +614,8 @@ const float* src_act(const hpf_model* mdl, int src, int m)
     return mdl->act(src, m);
 }
 
-int forward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
+// sl: the stream slot (partition, lane) whose scratch and side stream the op uses
+int forward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int sl)
 {
     const OpInfo& o = mdl->ops[i];
     const hpf_op& q = o.op;
@@ -621,7 +634,7 @@ int forward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
             const hpf_model::CellRun& run = mdl->cell_runs[mdl->cell_of_op[i]];
             if (run.convs[0] == i)
                 CU(conv_tc_cell_launch(mdl->ws + run.ops_off[m], (int)run.convs.size(), run.ctas, run.smem, run.tmem,
-                                       reinterpret_cast<unsigned int*>(mdl->ws + mdl->cell_bar_off[p]), mdl->status(), st, &mdl->launches));
+                                       reinterpret_cast<unsigned int*>(mdl->ws + mdl->cell_bar_off[sl]), mdl->status(), st, &mdl->launches));
         } else if (mdl->use_tc[PASS_FWD][i]) {
             CU(conv_tc_launch(&mdl->tc_plan[PASS_FWD][(size_t)m * mdl->n_ops + i], mdl->status(), st, &mdl->launches));
         } else {
@@ -636,11 +649,11 @@ int forward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
                                 (int64_t)mdl->b * o.H * o.W, o.C, st, &mdl->launches));
         else
             CU(bnrelu_fwd(in0, mdl->params + o.w_off, mdl->params + o.b_off, q.eps, out, mdl->stats(i, m),
-                          (int64_t)mdl->b * o.H * o.W, o.C, mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches));
+                          (int64_t)mdl->b * o.H * o.W, o.C, mdl->ws + mdl->bn_scratch_off[sl], st, &mdl->launches));
         break;
     case HPF_OP_BN:                        // batch normalisation without the activation
         CU(bnrelu_fwd(in0, mdl->params + o.w_off, mdl->params + o.b_off, q.eps, out, mdl->stats(i, m),
-                      (int64_t)mdl->b * o.H * o.W, o.C, mdl->ws + mdl->bn_scratch_off[p], st, &mdl->launches, false));
+                      (int64_t)mdl->b * o.H * o.W, o.C, mdl->ws + mdl->bn_scratch_off[sl], st, &mdl->launches, false));
         break;
     case HPF_OP_RELU:
         CU(relu_fwd(in0, out, mdl->numel(i), st, &mdl->launches));
@@ -662,7 +675,7 @@ int forward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
     return HPF_OK;
 }
 
-int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
+int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int sl)
 {
     const OpInfo& o = mdl->ops[i];
     const hpf_op& q = o.op;
@@ -681,14 +694,14 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
         // it runs on the partition's side stream once dL/d(output) is ready (everything before this point on st).
         cudaStream_t wst = st;
         if (!mdl->side.empty() && !mdl->opt_single) {
-            wst = mdl->side[p];
-            CU(cudaEventRecord(mdl->ev_side[p], st));
-            CU(cudaStreamWaitEvent(wst, mdl->ev_side[p], 0));
+            wst = mdl->side[sl];
+            CU(cudaEventRecord(mdl->ev_side[sl], st));
+            CU(cudaStreamWaitEvent(wst, mdl->ev_side[sl], 0));
         }
         if (mdl->use_tc[PASS_WGRAD][i]) {
             CU(conv_tc_launch(&mdl->tc_plan[PASS_WGRAD][(size_t)m * mdl->n_ops + i], mdl->status(), wst, &mdl->launches));
         } else {
-            CU(conv_wgrad_simt(in0, dout, slot + o.w_off, s, mdl->ws + mdl->conv_scratch_off[p], wst, &mdl->launches));
+            CU(conv_wgrad_simt(in0, dout, slot + o.w_off, s, mdl->ws + mdl->conv_scratch_off[sl], wst, &mdl->launches));
         }
         if (q.src0 >= 0) {
             if (mdl->use_tc[PASS_DGRAD][i]) {
@@ -702,12 +715,12 @@ int backward_op(hpf_model* mdl, int i, int m, cudaStream_t st, int p)
     case HPF_OP_BNRELU:
         CU(bnrelu_bwd(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m), addend,
                       e.accumulate != 0, slot + o.w_off, slot + o.b_off, (int64_t)mdl->b * o.H * o.W, o.C,
-                      mdl->ws + mdl->bn_scratch_bwd_off[p], st, &mdl->launches, true, true));
+                      mdl->ws + mdl->bn_scratch_bwd_off[sl], st, &mdl->launches, true, true));
         break;
     case HPF_OP_BN:
         CU(bnrelu_bwd(in0, dout, mdl->params + o.w_off, mdl->params + o.b_off, mdl->stats(i, m), mdl->grad(q.src0, m), addend,
                       e.accumulate != 0, slot + o.w_off, slot + o.b_off, (int64_t)mdl->b * o.H * o.W, o.C,
-                      mdl->ws + mdl->bn_scratch_bwd_off[p], st, &mdl->launches, false, true));
+                      mdl->ws + mdl->bn_scratch_bwd_off[sl], st, &mdl->launches, false, true));
         break;
     case HPF_OP_RELU:
         CU(relu_bwd(in0, dout, mdl->grad(q.src0, m), addend, e.accumulate != 0, mdl->numel(i), st, &mdl->launches));
@@ -755,15 +768,16 @@ int enqueue_phase(hpf_model* mdl, int phase)
     const BnClusterScope bn_cluster_scope(mdl->opt_bn_cluster);
     const int P = mdl->P, M = mdl->M;
     cudaStream_t s0 = mdl->streams[0];
-    const bool multi = !mdl->opt_single && P > 1;
     const bool merged = phase == PH_FB;
     const bool do_fwd = phase == PH_FWD || merged, do_bwd = phase == PH_BWD || merged;
+    const int S = mdl->n_slots();
+    const bool multi = !mdl->opt_single && S > 1;
     const bool own_bwd_streams = merged && !mdl->bwd_streams.empty() && !mdl->opt_single;
-    auto bwd_stream = [&](int p) { return own_bwd_streams ? mdl->bwd_streams[p] : mdl->stream_of(p); };
+    auto bwd_stream = [&](int p, int m) { return own_bwd_streams ? mdl->bwd_streams[mdl->slot_of(p, m)] : mdl->stream_of(p, m); };
     if (multi || own_bwd_streams) {
         CU(cudaEventRecord(mdl->ev_fork, s0));
-        if (multi) for (int p = 1; p < P; ++p) CU(cudaStreamWaitEvent(mdl->streams[p], mdl->ev_fork, 0));
-        if (own_bwd_streams) for (int p = 0; p < P; ++p) CU(cudaStreamWaitEvent(mdl->bwd_streams[p], mdl->ev_fork, 0));
+        if (multi) for (int k = 1; k < S; ++k) CU(cudaStreamWaitEvent(mdl->streams[k], mdl->ev_fork, 0));
+        if (own_bwd_streams) for (int k = 0; k < S; ++k) CU(cudaStreamWaitEvent(mdl->bwd_streams[k], mdl->ev_fork, 0));
     }
     if (do_fwd) {
         // the tensor-core convolutions read split (and, for the data gradient, rearranged) weights: once per step
@@ -776,13 +790,18 @@ int enqueue_phase(hpf_model* mdl, int phase)
                 CU(conv_weight_prep(mdl->params, wp, wp + G4, wp + 2 * G4, wp + 3 * G4,
                                     reinterpret_cast<const WeightPrepEntry*>(mdl->ws + mdl->prep_table_off[p]),
                                     (int)mdl->prep_table[p].size(), max_tiles, mdl->stream_of(p), &mdl->launches));
+                // the partition's other lanes read the same prepared weights
+                if (multi && mdl->lanes() > 1) {
+                    CU(cudaEventRecord(mdl->ev_prep[p], mdl->stream_of(p)));
+                    for (int l = 1; l < mdl->lanes(); ++l) CU(cudaStreamWaitEvent(mdl->streams[p * mdl->lanes() + l], mdl->ev_prep[p], 0));
+                }
             }
         // tick t: every (p, m) with p + m = t
         for (int t = 0; t < P + M - 1; ++t)
             for (int p = 0; p < P; ++p) {
                 const int m = t - p;
                 if (m < 0 || m >= M) continue;
-                cudaStream_t st = mdl->stream_of(p);
+                cudaStream_t st = mdl->stream_of(p, m);
                 if (p > 0) {
                     if (multi) CU(cudaStreamWaitEvent(st, mdl->ev_fwd[(size_t)(p - 1) * M + m], 0));     // recv
                     if (mdl->opt_messages)
@@ -792,7 +811,7 @@ int enqueue_phase(hpf_model* mdl, int phase)
                 }
                 if (mdl->opt_cell_times) CU(stamp_time(mdl->cell_time_slot(PH_FWD, p, m), st, &mdl->launches));
                 for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i) {
-                    int rc = forward_op(mdl, i, m, st, p);
+                    int rc = forward_op(mdl, i, m, st, mdl->slot_of(p, m));
                     if (rc) return rc;
                 }
                 if (mdl->opt_cell_times) CU(stamp_time(mdl->cell_time_slot(PH_FWD, p, m) + 1, st, &mdl->launches));
@@ -805,7 +824,7 @@ int enqueue_phase(hpf_model* mdl, int phase)
             for (int p = P - 1; p >= 0; --p) {
                 const int m = t - (P - 1 - p);
                 if (m < 0 || m >= M) continue;
-                cudaStream_t st = bwd_stream(p);
+                cudaStream_t st = bwd_stream(p, m);
                 if (p < P - 1) {
                     if (multi || own_bwd_streams) CU(cudaStreamWaitEvent(st, mdl->ev_bwd[(size_t)p * M + m], 0));           // recv partial errors
                     if (mdl->opt_messages)
@@ -820,7 +839,7 @@ int enqueue_phase(hpf_model* mdl, int phase)
                 }
                 if (mdl->opt_cell_times) CU(stamp_time(mdl->cell_time_slot(PH_BWD, p, m), st, &mdl->launches));
                 for (int i = mdl->part_hi[p] - 1; i >= mdl->part_lo[p]; --i) {
-                    int rc = backward_op(mdl, i, m, st, p);
+                    int rc = backward_op(mdl, i, m, st, mdl->slot_of(p, m));
                     if (rc) return rc;
                 }
                 if (mdl->opt_cell_times) CU(stamp_time(mdl->cell_time_slot(PH_BWD, p, m) + 1, st, &mdl->launches));
@@ -828,22 +847,23 @@ int enqueue_phase(hpf_model* mdl, int phase)
             }
     }
     if (do_bwd && !mdl->side.empty() && !mdl->opt_single)
-        for (int p = 0; p < P; ++p) {
+        for (int k = 0; k < S; ++k) {
             // the side stream holds work only if it was forked during this phase; joining an unforked stream is harmless
-            CU(cudaEventRecord(mdl->ev_side[p], bwd_stream(p)));
-            CU(cudaStreamWaitEvent(mdl->side[p], mdl->ev_side[p], 0));
-            CU(cudaEventRecord(mdl->ev_side_join[p], mdl->side[p]));
-            CU(cudaStreamWaitEvent(s0, mdl->ev_side_join[p], 0));
+            cudaStream_t from = own_bwd_streams ? mdl->bwd_streams[k] : mdl->streams[k];
+            CU(cudaEventRecord(mdl->ev_side[k], from));
+            CU(cudaStreamWaitEvent(mdl->side[k], mdl->ev_side[k], 0));
+            CU(cudaEventRecord(mdl->ev_side_join[k], mdl->side[k]));
+            CU(cudaStreamWaitEvent(s0, mdl->ev_side_join[k], 0));
         }
     if (own_bwd_streams)
-        for (int p = 0; p < P; ++p) {
-            CU(cudaEventRecord(mdl->ev_bjoin[p], mdl->bwd_streams[p]));
-            CU(cudaStreamWaitEvent(s0, mdl->ev_bjoin[p], 0));
+        for (int k = 0; k < S; ++k) {
+            CU(cudaEventRecord(mdl->ev_bjoin[k], mdl->bwd_streams[k]));
+            CU(cudaStreamWaitEvent(s0, mdl->ev_bjoin[k], 0));
         }
     if (multi)
-        for (int p = 1; p < P; ++p) {
-            CU(cudaEventRecord(mdl->ev_join[p], mdl->streams[p]));
-            CU(cudaStreamWaitEvent(s0, mdl->ev_join[p], 0));
+        for (int k = 1; k < S; ++k) {
+            CU(cudaEventRecord(mdl->ev_join[k], mdl->streams[k]));
+            CU(cudaStreamWaitEvent(s0, mdl->ev_join[k], 0));
         }
     if (do_fwd)
         CU(loss_average(reinterpret_cast<float*>(mdl->ws + mdl->loss_slots_off), reinterpret_cast<float*>(mdl->ws + mdl->loss_avg_off), M, s0, &mdl->launches));
@@ -919,6 +939,8 @@ void release_device_objects(hpf_model* mdl)
     for (auto e : mdl->ev_fwd) cudaEventDestroy(e);
     for (auto e : mdl->ev_bwd) cudaEventDestroy(e);
     for (auto e : mdl->ev_join) if (e) cudaEventDestroy(e);
+    for (auto e : mdl->ev_prep) if (e) cudaEventDestroy(e);
+    mdl->ev_prep.clear();
     for (auto e : mdl->ev_side) if (e) cudaEventDestroy(e);
     for (auto e : mdl->ev_side_join) if (e) cudaEventDestroy(e);
     mdl->ev_side.clear(); mdl->ev_side_join.clear();
@@ -976,6 +998,8 @@ int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
     case HPF_OPT_FUSE_BN: if (value < 0 || value > 3) return fail(HPF_ERR_INVALID, "0..3"); mdl->opt_fuse_bn = value; break;
     case HPF_OPT_CELL_TIMES: mdl->opt_cell_times = value != 0; break;
     case HPF_OPT_BN_CLUSTER: mdl->opt_bn_cluster = value != 0; break;
+    case HPF_OPT_WGRAD_DIRECT: mdl->opt_wgrad_direct = value != 0; break;
+    case HPF_OPT_STAGE_LANES: if (value < 1 || value > 64) return fail(HPF_ERR_INVALID, "1..64 lanes"); mdl->opt_lanes = value; break;
     case HPF_OPT_PDL_LATE_FROM: if (value < 0) return fail(HPF_ERR_INVALID, ">= 0"); mdl->opt_pdl_late_from = value; break;
     case HPF_OPT_CELL_CTAS: if (value < 0 || value > 148) return fail(HPF_ERR_INVALID, "0..148 CTAs"); mdl->opt_cell = value; break;
     case HPF_OPT_WGRAD_PASSES: if (value != 1 && value != 3) return fail(HPF_ERR_INVALID, "1 or 3 passes"); mdl->opt_wgrad_passes = value; break;
@@ -987,6 +1011,7 @@ int hpf_set_option(hpf_model* mdl, int32_t option, int32_t value)
 
 int hpf_num_ops(const hpf_model* mdl, int32_t* n) { if (!mdl || !n) return fail(HPF_ERR_INVALID, "null"); *n = mdl->n_ops; return HPF_OK; }
 int hpf_num_partitions(const hpf_model* mdl, int32_t* P) { if (!mdl || !P) return fail(HPF_ERR_INVALID, "null"); *P = mdl->P; return HPF_OK; }
+int hpf_num_stream_slots(const hpf_model* mdl, int32_t* S) { if (!mdl || !S) return fail(HPF_ERR_INVALID, "null"); *S = mdl->n_slots(); return HPF_OK; }
 int hpf_num_params(const hpf_model* mdl, int64_t* G) { if (!mdl || !G) return fail(HPF_ERR_INVALID, "null"); *G = mdl->G; return HPF_OK; }
 
 int hpf_param_layout(const hpf_model* mdl, int32_t op, int64_t* w_off, int64_t* w_cnt, int64_t* b_off, int64_t* b_cnt)
@@ -1143,7 +1168,8 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
 {
     if (!mdl || !d_params || !d_grad_slots || !d_grad_avg || !d_workspace || !cuda_streams) return fail(HPF_ERR_INVALID, "null argument");
     if (mdl->state != ST_CREATED) return fail(HPF_ERR_STATE, "already bound");
-    if (n_streams < mdl->P) return fail(HPF_ERR_INVALID, "one stream per partition is required");
+    const int S = mdl->n_slots();
+    if (n_streams < S) return fail(HPF_ERR_INVALID, "one stream per partition and stage lane is required");
     if (!mdl->planned) build_memory_plan(mdl);
     if (ws_bytes < mdl->ws_bytes) return fail(HPF_ERR_WORKSPACE, "workspace too small");
     if (reinterpret_cast<uintptr_t>(d_workspace) % 256) return fail(HPF_ERR_WORKSPACE, "workspace must be 256-byte aligned");
@@ -1154,31 +1180,33 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
     if (e != cudaSuccess || ndev < 1) { cudaGetLastError(); return cuda_fail(e != cudaSuccess ? e : cudaErrorNoDevice, "cudaGetDeviceCount"); }
     mdl->params = d_params; mdl->gslots = d_grad_slots; mdl->gavg = d_grad_avg;
     mdl->ws = reinterpret_cast<char*>(d_workspace);
-    mdl->streams.resize(mdl->P);
-    for (int p = 0; p < mdl->P; ++p) mdl->streams[p] = reinterpret_cast<cudaStream_t>(cuda_streams[p]);
+    mdl->streams.resize(S);
+    for (int k = 0; k < S; ++k) mdl->streams[k] = reinterpret_cast<cudaStream_t>(cuda_streams[k]);
     mdl->side.clear();
-    if (n_streams >= 2 * mdl->P) {
-        mdl->side.resize(mdl->P);
-        for (int p = 0; p < mdl->P; ++p) mdl->side[p] = reinterpret_cast<cudaStream_t>(cuda_streams[mdl->P + p]);
-        mdl->ev_side.assign(mdl->P, nullptr); mdl->ev_side_join.assign(mdl->P, nullptr);
-        for (int p = 0; p < mdl->P; ++p) {
-            CU(cudaEventCreateWithFlags(&mdl->ev_side[p], cudaEventDisableTiming));
-            CU(cudaEventCreateWithFlags(&mdl->ev_side_join[p], cudaEventDisableTiming));
+    if (n_streams >= 2 * S) {
+        mdl->side.resize(S);
+        for (int k = 0; k < S; ++k) mdl->side[k] = reinterpret_cast<cudaStream_t>(cuda_streams[S + k]);
+        mdl->ev_side.assign(S, nullptr); mdl->ev_side_join.assign(S, nullptr);
+        for (int k = 0; k < S; ++k) {
+            CU(cudaEventCreateWithFlags(&mdl->ev_side[k], cudaEventDisableTiming));
+            CU(cudaEventCreateWithFlags(&mdl->ev_side_join[k], cudaEventDisableTiming));
         }
     }
     mdl->bwd_streams.clear();
-    if (n_streams >= 3 * mdl->P) {
-        mdl->bwd_streams.resize(mdl->P);
-        for (int p = 0; p < mdl->P; ++p) mdl->bwd_streams[p] = reinterpret_cast<cudaStream_t>(cuda_streams[2 * mdl->P + p]);
-        mdl->ev_fdone.assign(mdl->M, nullptr); mdl->ev_bjoin.assign(mdl->P, nullptr);
+    if (n_streams >= 3 * S) {
+        mdl->bwd_streams.resize(S);
+        for (int k = 0; k < S; ++k) mdl->bwd_streams[k] = reinterpret_cast<cudaStream_t>(cuda_streams[2 * S + k]);
+        mdl->ev_fdone.assign(mdl->M, nullptr); mdl->ev_bjoin.assign(S, nullptr);
         for (auto& ev : mdl->ev_fdone) CU(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
         for (auto& ev : mdl->ev_bjoin) CU(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
     }
     const int M = mdl->M, n = mdl->n_ops;
     CU(cudaEventCreateWithFlags(&mdl->ev_fork, cudaEventDisableTiming));
     CU(cudaEventCreateWithFlags(&mdl->ev_sync, cudaEventDisableTiming));
-    mdl->ev_join.assign(mdl->P, nullptr);
-    for (int p = 1; p < mdl->P; ++p) CU(cudaEventCreateWithFlags(&mdl->ev_join[p], cudaEventDisableTiming));
+    mdl->ev_join.assign(S, nullptr);
+    for (int k = 1; k < S; ++k) CU(cudaEventCreateWithFlags(&mdl->ev_join[k], cudaEventDisableTiming));
+    mdl->ev_prep.assign(mdl->P, nullptr);
+    for (auto& ev : mdl->ev_prep) CU(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
     mdl->ev_fwd.resize(mdl->cuts.size() * M); mdl->ev_bwd.resize(mdl->cuts.size() * M);
     for (auto& ev : mdl->ev_fwd) CU(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
     for (auto& ev : mdl->ev_bwd) CU(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
@@ -1209,7 +1237,8 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
             const int src = o.op.src0;
             const ConvShape s = conv_shape_of(mdl, i);
             ConvTcPlan* pl = &mdl->tc_plan[PASS_FWD][(size_t)m * n + i];
-            void* scratch = mdl->ws + mdl->conv_scratch_off[o.part];
+            const int sl = mdl->slot_of(o.part, m);
+            void* scratch = mdl->ws + mdl->conv_scratch_off[sl];
             const int pass = PASS_FWD;
             const float* residual = nullptr;
                     if (mdl->fused_into[i] >= 0) {
@@ -1217,8 +1246,8 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                         residual = mdl->act(a.src0 == i ? a.src1 : a.src0, m);
                     }
                     ConvBnFuse fuse;
-                    if (mdl->splitk_bytes[o.part]) { fuse.splitk = mdl->ws + mdl->splitk_off[o.part]; fuse.splitk_bytes = mdl->splitk_bytes[o.part]; }
-                    fuse.pdl_late = cells_under_way(mdl->P, M, o.part, m, false) >= mdl->opt_pdl_late_from;
+                    if (mdl->splitk_bytes[o.part]) { fuse.splitk = mdl->ws + mdl->splitk_off[sl]; fuse.splitk_bytes = mdl->splitk_bytes[o.part]; }
+                    fuse.pdl_late = cells_under_way(mdl->P, M, o.part, m, false) * mdl->lanes() >= mdl->opt_pdl_late_from;
                     if (mdl->cell_of_op[i] >= 0) {
                         fuse.cell_ctas = mdl->opt_cell;
                         fuse.cell_smem = mdl->cell_runs[mdl->cell_of_op[i]].smem_budget;
@@ -1227,8 +1256,8 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                         const int jn = mdl->conv_fwd_bn[i];
                         const OpInfo& bn = mdl->ops[jn];
                         fuse.mode = mdl->bn_late[jn] ? 3 : 1;
-                        fuse.ticket = reinterpret_cast<unsigned int*>(mdl->ws + mdl->bn_scratch_off[o.part]);
-                        fuse.partials = mdl->bn_partials(jn);
+                        fuse.ticket = reinterpret_cast<unsigned int*>(mdl->ws + mdl->bn_scratch_off[sl]);
+                        fuse.partials = mdl->bn_partials(jn, m);
                         fuse.stats_out = mdl->stats(jn, m);
                         fuse.rows = (long long)mdl->b * bn.H * bn.W;
                         fuse.eps = bn.op.eps;
@@ -1239,7 +1268,7 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                         const OpInfo& bn = mdl->ops[jb];
                         in = mdl->act(bn.op.src0, m);          // the BN's input; its output is a by-product of this kernel
                         fuse.in_mode = mdl->bn_late[jb] ? 2 : 1;
-                        fuse.in_partials = mdl->bn_partials(jb);
+                        fuse.in_partials = mdl->bn_partials(jb, m);
                         fuse.in_tiles = conv_tc_tiles(conv_shape_of(mdl, mdl->bn_fwd_from[jb]), PASS_FWD);
                         fuse.in_rows = (long long)mdl->b * bn.H * bn.W;
                         fuse.in_eps = bn.op.eps;
@@ -1259,14 +1288,15 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                     const ConvShape s = conv_shape_of(mdl, i);
                     const GradEdge& ed = mdl->edge0[i];
                     ConvTcPlan* pl = &mdl->tc_plan[pass][(size_t)m * n + i];
-                    void* scratch = mdl->ws + mdl->conv_scratch_off[o.part];
+                    const int sl = mdl->slot_of(o.part, m);
+                    void* scratch = mdl->ws + mdl->conv_scratch_off[sl];
                     if (pass == PASS_FWD) {
                         int rc = prepare_fwd(i, m);
                         if (rc) return rc;
                     }
                     else if (pass == PASS_DGRAD) {
                         ConvBnFuse dsplit;
-                        if (mdl->splitk_bytes[o.part]) { dsplit.splitk = mdl->ws + mdl->splitk_bwd_off[o.part]; dsplit.splitk_bytes = mdl->splitk_bytes[o.part]; }
+                        if (mdl->splitk_bytes[o.part]) { dsplit.splitk = mdl->ws + mdl->splitk_bwd_off[sl]; dsplit.splitk_bytes = mdl->splitk_bytes[o.part]; }
                         CU(conv_tc_prepare(pl, s, pass, passes, mdl->grad(i, m), nullptr, wp + 2 * G + o.w_off, wp + 3 * G + o.w_off,
                                            mdl->grad(src, m), ed.addend >= 0 ? mdl->grad(ed.addend, m) : nullptr, ed.accumulate != 0, scratch,
                                            &dsplit));
@@ -1277,7 +1307,8 @@ int hpf_bind(hpf_model* mdl, float* d_params, float* d_grad_slots, float* d_grad
                         // duration: about 32 CTAs is the measured optimum for eight stages (fewer and the weight gradients
                         // fall behind the chain; with four stages the uncapped launch measured faster).
                         ConvBnFuse hint;
-                        hint.wgrad_max_ctas = (mdl->P >= 6 && !mdl->side.empty()) ? 32 : 0;
+                        hint.wgrad_max_ctas = (mdl->n_slots() >= 6 && !mdl->side.empty()) ? 32 : 0;
+                        hint.wgrad_transposing = mdl->opt_wgrad_direct ? 0 : 1;
                         CU(conv_tc_prepare(pl, s, pass, mdl->opt_conv_path == 2 ? 1 : mdl->opt_wgrad_passes, mdl->grad(i, m), mdl->act(src, m), nullptr, nullptr,
                                            mdl->gslots + (int64_t)m * mdl->G + o.w_off, nullptr, false, scratch, &hint));
                     }
@@ -1374,6 +1405,10 @@ int hpf_prepare_partition(hpf_model* mdl, int32_t p)
     CU(conv_weight_prep(mdl->params, wp, wp + G4, wp + 2 * G4, wp + 3 * G4,
                         reinterpret_cast<const WeightPrepEntry*>(mdl->ws + mdl->prep_table_off[p]),
                         (int)mdl->prep_table[p].size(), max_tiles, mdl->stream_of(p), &mdl->launches));
+    if (mdl->lanes() > 1 && !mdl->opt_single) {
+        CU(cudaEventRecord(mdl->ev_prep[p], mdl->stream_of(p)));
+        for (int l = 1; l < mdl->lanes(); ++l) CU(cudaStreamWaitEvent(mdl->streams[p * mdl->lanes() + l], mdl->ev_prep[p], 0));
+    }
     return HPF_OK;
 }
 
@@ -1389,7 +1424,7 @@ int hpf_forward_cell(hpf_model* mdl, int32_t p, int32_t m, const float* d_x, con
     const PdlScope pdl_scope(mdl->opt_pdl);
     const BnClusterScope bn_cluster_scope(mdl->opt_bn_cluster);
     for (int i = mdl->part_lo[p]; i < mdl->part_hi[p]; ++i) {
-        int rc = forward_op(mdl, i, m, mdl->stream_of(p), p);
+        int rc = forward_op(mdl, i, m, mdl->stream_of(p, m), mdl->slot_of(p, m));
         if (rc) return rc;
     }
     if (mdl->state < ST_FWD) mdl->state = ST_FWD;
@@ -1405,7 +1440,7 @@ int hpf_backward_cell(hpf_model* mdl, int32_t p, int32_t m)
     const PdlScope pdl_scope(mdl->opt_pdl);
     const BnClusterScope bn_cluster_scope(mdl->opt_bn_cluster);
     for (int i = mdl->part_hi[p] - 1; i >= mdl->part_lo[p]; --i) {
-        int rc = backward_op(mdl, i, m, mdl->stream_of(p), p);
+        int rc = backward_op(mdl, i, m, mdl->stream_of(p, m), mdl->slot_of(p, m));
         if (rc) return rc;
     }
     mdl->state = ST_BWD;
@@ -1418,11 +1453,15 @@ int hpf_join_partition(hpf_model* mdl, int32_t p)
     if (mdl->state < ST_BOUND) return fail(HPF_ERR_STATE, "hpf_bind first");
     if (p < 0 || p >= mdl->P) return fail(HPF_ERR_INVALID, "partition out of range");
     if (!mdl->side.empty() && !mdl->opt_single) {
+        // every lane's weight gradients and cells join the partition's first stream
         cudaStream_t st = mdl->stream_of(p);
-        CU(cudaEventRecord(mdl->ev_side[p], st));
-        CU(cudaStreamWaitEvent(mdl->side[p], mdl->ev_side[p], 0));
-        CU(cudaEventRecord(mdl->ev_side_join[p], mdl->side[p]));
-        CU(cudaStreamWaitEvent(st, mdl->ev_side_join[p], 0));
+        for (int l = 0; l < mdl->lanes(); ++l) {
+            const int k = p * mdl->lanes() + l;
+            CU(cudaEventRecord(mdl->ev_side[k], mdl->streams[k]));
+            CU(cudaStreamWaitEvent(mdl->side[k], mdl->ev_side[k], 0));
+            CU(cudaEventRecord(mdl->ev_side_join[k], mdl->side[k]));
+            CU(cudaStreamWaitEvent(st, mdl->ev_side_join[k], 0));
+        }
     }
     return HPF_OK;
 }
@@ -1693,6 +1732,8 @@ static int conv_single(int pass, const float* in, const float* in2, const float*
         else CU(conv_wgrad_simt(in2, in, out, s, d_scratch, st, nullptr));
         return HPF_OK;
     }
+    const bool transposing = pass == PASS_WGRAD && (path == 3 || path == 4);
+    if (transposing) path = path == 3 ? 0 : 2;
     if (path != 0 && path != 2) return fail(HPF_ERR_INVALID, "bad path");
     if (pass != PASS_WGRAD && !wprep) return fail(HPF_ERR_INVALID, "the tensor-core paths need prepared weights");
     if (!conv_tc_supported(s, pass)) return fail(HPF_ERR_UNSUPPORTED, "shape outside the tensor-core kernels' reach");
@@ -1706,6 +1747,7 @@ static int conv_single(int pass, const float* in, const float* in2, const float*
     const int64_t nw = (int64_t)K * R * R * C;
     const float* hi = wprep ? wprep + (pass == PASS_DGRAD ? 2 * nw : 0) : nullptr;
     ConvBnFuse split;
+    split.wgrad_transposing = transposing ? 1 : 0;
     if (pass != PASS_WGRAD) {
         const size_t a = conv_simt_scratch_bytes(s), b = conv_tc_scratch_bytes(s);
         split.splitk_bytes = conv_tc_splitk_bytes(s, pass, 3);

@@ -83,7 +83,7 @@ class Stage:
             self.slots = torch.zeros((n_microbatches, G), device=self.dev)
             self.avg = torch.zeros(G, device=self.dev)
             self.ws = torch.empty(self.model.workspace_bytes(), dtype=torch.uint8, device=self.dev)
-            self.streams = [torch.cuda.Stream(device=self.dev) for _ in range(2 * self.P)]
+            self.streams = [torch.cuda.Stream(device=self.dev) for _ in range(2 * self.model.num_stream_slots())]
             torch.cuda.synchronize(self.dev)
             self.model.bind(self.params, self.slots, self.avg, self.ws, self.streams)
         self.stream = self.streams[p]

@@ -44,7 +44,7 @@ def time_step(ops, in_shape, cuts, n_microbatches, params, steps=3, warmup=2, de
         slots = torch.empty((n_microbatches, G), device=dev)
         avg = torch.empty(G, device=dev)
         ws = torch.empty(model.workspace_bytes(), dtype=torch.uint8, device=dev)
-        streams = [torch.cuda.Stream(device=dev) for _ in range(3 * model.num_partitions())]      # stage, weight-gradient, backward
+        streams = [torch.cuda.Stream(device=dev) for _ in range(3 * model.num_stream_slots())]      # stage, weight-gradient, backward
         x = torch.randn(tuple(in_shape), device=dev)
         labels = torch.zeros(in_shape[0], dtype=torch.int32, device=dev)
         torch.cuda.synchronize(dev)

@@ -50,7 +50,7 @@ class Bound:
         self.slots = torch.full((M, self.G), float("nan"), dtype=torch.float32, device=self.dev)
         self.avg = torch.full((self.G,), float("nan"), dtype=torch.float32, device=self.dev)
         self.ws = torch.empty(self.model.workspace_bytes(), dtype=torch.uint8, device=self.dev)
-        n_streams = self.model.num_partitions() * (3 if backward_streams else (2 if side_streams else 1))
+        n_streams = self.model.num_stream_slots() * (3 if backward_streams else (2 if side_streams else 1))
         self.streams = [torch.cuda.Stream(device=self.dev) for _ in range(n_streams)]
         torch.cuda.synchronize()
         self.model.bind(self.params, self.slots, self.avg, self.ws, self.streams)

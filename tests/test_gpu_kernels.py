@@ -61,6 +61,39 @@ def test_conv_sweep_tensor_core_path(shape, path):
         assert min(e) > 1e-5          # it really is the 11-bit path
 
 
+def _wgrad_case(ks, st, ci, co, H, N, path, seed=0):
+    pad = 1 if ks == 3 else 0
+    rng = np.random.Generator(np.random.PCG64(2000 + seed))
+    x = rng.standard_normal((N, H, H, ci)).astype(np.float32)
+    P = (H + 2 * pad - ks) // st + 1
+    dy = rng.standard_normal((N, P, P, co)).astype(np.float32)
+    scratch = torch.zeros(hpf.conv_scratch_bytes(N, H, H, ci, co, ks, st, pad), dtype=torch.uint8, device=DEV)
+    gw = torch.full((co, ks, ks, ci), float("nan"), device=DEV)
+    hpf.conv_wgrad(_dev(x), _dev(dy), gw, N, H, H, ci, co, ks, st, pad, path, scratch)
+    torch.cuda.synchronize()
+    assert scratch[-256:-248].view(torch.int32).cpu().tolist() == [0, 0]
+    return rel_l2(gw.cpu().numpy(), ora.conv_wgrad(x, dy, ks, st, pad)), gw
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 64, 16, 32), (3, 1, 16, 16, 32), (3, 1, 64, 64, 8), (1, 2, 64, 32, 32), (3, 1, 128, 128, 14), (1, 1, 48, 16, 8)],
+                         ids=lambda s: "k%d_s%d_%dto%d_at%d" % s)
+@pytest.mark.parametrize("passes", [3, 1])
+def test_weight_gradient_kernels_agree(shape, passes):
+    """The weight gradient has two tensor-core kernels: one hands the TMA tiles (pixels x channels) to the tensor core as
+    MN-major operands as they land, the other transposes them in shared memory first (kept as a cross-check, and for
+    channel counts like 48 that the first does not take).  Both against the oracle; with three passes they agree to
+    fp32 rounding with each other."""
+    ks, st, ci, co, H = shape
+    e_direct, g_direct = _wgrad_case(ks, st, ci, co, H, 6, 0 if passes == 3 else 2)
+    e_transp, g_transp = _wgrad_case(ks, st, ci, co, H, 6, 3 if passes == 3 else 4)
+    tol = 2e-5 if passes == 3 else TOL_TENSOR
+    assert e_direct <= tol and e_transp <= tol, (e_direct, e_transp)
+    if passes == 3:
+        assert rel_l2(g_direct.cpu().numpy(), g_transp.cpu().numpy()) <= 1e-5
+    else:
+        assert e_direct > 1e-5 and e_transp > 1e-5          # both really are 11-bit paths
+
+
 @pytest.mark.parametrize("shape", [(1, 1, 64, 16, 32), (3, 1, 16, 16, 32), (1, 1, 16, 64, 32), (1, 2, 64, 32, 32)],
                          ids=lambda s: "k%d_s%d_%dto%d_at%d" % s)
 def test_conv_launches_of_several_waves_use_two_tiles_per_cta(shape):

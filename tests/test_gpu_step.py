@@ -144,8 +144,17 @@ def test_bn_statistics_of_channels_whose_mean_dwarfs_their_spread(fuse_bn):
     zero_grad = {("g", i, "b") for i, o in enumerate(ops) if o.kind == wl.BNRELU and ops[i + 1].kind == wl.CONV}
     # (three-pass weight gradients: with activations of ten +- 0.1 a single TF32 pass keeps too little of the +- 0.1, which
     # is all that survives the sum against a gradient whose channel sums vanish)
-    bd, _, _ = check_step(ops, (32, 32, 3), 8, 2, [9], {hpf.OPT_FUSE_BN: fuse_bn, hpf.OPT_WGRAD_PASSES: 3}, seed=21, bn_jitter=0.2, edit_theta=shifted,
-                          name="mean >> sigma, fuse_bn=%d" % fuse_bn, skip=zero_grad)
+    # The weight gradient of a convolution that reads such a BN's output sums dy * (10 +- 0.1) over the pixels against a dy
+    # whose channel sums all but vanish: two digits cancel in any fp32 evaluation (the two weight-gradient kernels, fed the
+    # same bits, differ from each other by as much as either differs from the oracle).  Those tensors are held to 5e-2 here;
+    # everything else, the BN statistics and activations above all, to the usual tolerance.
+    shifted_input = {("g", i, "w") for i, o in enumerate(ops) if o.kind == wl.CONV and o.src0 >= 0 and ops[o.src0].kind == wl.BNRELU}
+    bd, ref, _ = check_step(ops, (32, 32, 3), 8, 2, [9], {hpf.OPT_FUSE_BN: fuse_bn, hpf.OPT_WGRAD_PASSES: 3}, seed=21, bn_jitter=0.2, edit_theta=shifted,
+                            name="mean >> sigma, fuse_bn=%d" % fuse_bn, skip=zero_grad | shifted_input)
+    avg = bd.avg.cpu().numpy()
+    for _, i, _ in sorted(shifted_input):
+        w_off, w_cnt, _, _ = offs[i]
+        assert rel_l2(avg[w_off:w_off + w_cnt], ref["g_avg"][w_off:w_off + w_cnt]) <= 5e-2, i
     # the premise: some BN input really is that badly centred
     ratios = []
     for i, o in enumerate(ops):
@@ -290,6 +299,53 @@ def test_forward_and_backward_as_one_graph_give_the_same_bits(streams):
                 assert bwd[p][m][0] >= bwd[p + 1][m][1]          # partial errors arrive from the partition above
     with pytest.raises(hpf.HpfError):
         bd.model.backward()                      # the step is complete: a second backward needs a fresh forward
+
+
+@pytest.mark.parametrize("lanes,one_graph", [(2, True), (3, True), (4, True), (8, True), (2, False)])
+def test_stage_lanes_give_the_same_bits_and_fill_the_bubble(lanes, one_graph):
+    """HPF_OPT_STAGE_LANES: a stage keeps several of its micro-batches under way at once, each lane on its own streams and
+    scratch.  Every cell runs the same kernels on the same data, so every bit must equal the one-lane schedule; the hand-offs
+    between stages still order the cells of one micro-batch; and cells of one stage really do overlap."""
+    ops = wl.resnet_v2_cifar(2)
+    x, labels, theta = seeded(ops, (32, 32, 3), 8, seed=6, bn_jitter=0.1)
+    P, M = 3, 4
+    cuts = wl.default_cuts(len(ops), P)
+    ref = Bound(ops, (32, 32, 3), 8, M, cuts, theta)
+    ref.upload(x, labels)
+    l_ref = ref.step()
+    bd = Bound(ops, (32, 32, 3), 8, M, cuts, theta, {hpf.OPT_STAGE_LANES: lanes, hpf.OPT_CELL_TIMES: 1}, backward_streams=one_graph)
+    assert bd.model.num_stream_slots() == P * min(lanes, M)
+    bd.upload(x, labels)
+    for _ in range(2):
+        assert bd.step(one_graph=one_graph) == l_ref
+        assert torch.equal(ref.slots, bd.slots) and torch.equal(ref.avg, bd.avg)
+    for i in range(len(ops)):
+        assert np.array_equal(ref.tensor(i, M - 1, grad=True), bd.tensor(i, M - 1, grad=True)), i
+    fwd, bwd = bd.model.cell_times(0), bd.model.cell_times(1)
+    for m in range(M):
+        for p in range(1, P):
+            assert fwd[p][m][0] >= fwd[p - 1][m][1]              # activations arrive from the partition below
+        for p in range(P - 1):
+            assert bwd[p][m][0] >= bwd[p + 1][m][1]              # partial errors arrive from the partition above
+        assert bwd[P - 1][m][0] >= fwd[P - 1][m][1]
+    L = min(lanes, M)
+    for p in range(P):
+        for m in range(L, M):
+            assert fwd[p][m][0] >= fwd[p][m - L][1]              # a lane works through its micro-batches in order
+    # the point of it: micro-batches 0 and 1 of the first stage run side by side
+    assert fwd[0][1][0] < fwd[0][0][1]
+
+
+def test_too_few_streams_for_the_lanes_are_refused():
+    ops = wl.resnet_v2_cifar(1)
+    model = hpf.Model(ops, (4, 32, 32, 3), wl.default_cuts(len(ops), 2), 2)
+    model.set_option(hpf.OPT_STAGE_LANES, 2)
+    assert model.num_stream_slots() == 4
+    G = model.num_params()
+    params = torch.zeros(G, device="cuda"); slots = torch.zeros((2, G), device="cuda"); avg = torch.zeros(G, device="cuda")
+    ws = torch.empty(model.workspace_bytes(), dtype=torch.uint8, device="cuda")
+    with pytest.raises(hpf.HpfError):
+        model.bind(params, slots, avg, ws, [torch.cuda.Stream() for _ in range(2)])
 
 
 @pytest.mark.parametrize("P,R,cuts", [(2, 1, [12]), (3, 1, [9, 30]), (2, 2, [25])], ids=["two_stages_mid_block_cut", "three_stages", "two_stages_two_replicas"])
