@@ -368,6 +368,10 @@ def conv_sweep(args):
             "dgrad": lambda k: hpf.conv_dgrad(ys[k], w, wprep, xs[k], *geo, scratch),
             "wgrad": lambda k: hpf.conv_wgrad(xs[k], ys[k], dw, *geo, scratch),
         }
+        if args.conv_path == 0:
+            # what the training step runs: the weight gradient with ONE TF32 pass (its error does not compound with depth)
+            geo1 = geo[:-1] + (2,)
+            calls["wgrad, one pass"] = lambda k: hpf.conv_wgrad(xs[k], ys[k], dw, *geo1, scratch)
         flops = 2.0 * N * P * P * ci * co * ks * ks
         nbytes = 4.0 * (in_el + y_el + w_el)
         for name, fn in calls.items():

@@ -577,7 +577,10 @@ __device__ __forceinline__ int conv_fwd_cta(const FwdParams* gpp, FwdScalars& p,
             const bool stacked = p.stacked != 0;
             const int stages = p.stages, k8n = p.kchunk / 8;
             const bool three = p.passes == 3;
-            const bool split_first = three || p.bn_in != 0;   // the splitter warps rewrite the tile before it is read
+            // the splitter warps write the lo part (and with BN+ReLU on the way in rewrite the tile) before the MMAs of the
+            // stage are issued.  (Issuing the MMAs that read only the tile as copied ahead of the splitters' barrier was
+            // measured: the step got 1.7 ms slower.)
+            const bool split_first = three || p.bn_in != 0;
             int it = 0, s = 0;
             uint32_t par = 0;
             bool live = true;
@@ -742,8 +745,9 @@ __device__ __forceinline__ int conv_fwd_cta(const FwdParams* gpp, FwdScalars& p,
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
                     if (j < per) {
+                        // The tile itself stays as copied: the tensor core ignores the 13 low mantissa bits of a 32-bit
+                        // operand, which is the very truncation the hi part is defined by.
                         const float4 h = make_float4(tf32_hi(v[j].x), tf32_hi(v[j].y), tf32_hi(v[j].z), tf32_hi(v[j].w));
-                        a[tid + 256 * j] = h;
                         alo[tid + 256 * j] = make_float4(v[j].x - h.x, v[j].y - h.y, v[j].z - h.z, v[j].w - h.w);
                     }
                 fence_async_smem();               // generic-proxy writes -> tensor-core reads
@@ -1394,8 +1398,8 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_kernel(const __grid_constan
 // dW[co][tap][ci] = sum over pixels of dy[pixel][co] * x[pixel + tap][ci]: the reduction runs over pixels, and both
 // tensors keep channels innermost in memory, so both operands are MN-major.  A TMA box of 32 channels x `rows` pixels with
 // the 32-byte-atom swizzle is exactly the tile the tensor core wants (smem_desc_mn): 6 warps = TMA producer, MMA issuer and
-// 4 warps that only read the accumulators at the end (with three passes they also split every tile into hi and lo, in
-// place and position by position - no transposition either).  A 16-channel tensor is copied with 16-channel boxes: the
+// 4 warps that only read the accumulators at the end (with three passes they also write every tile's lo part, position
+// by position - no transposition either).  A 16-channel tensor is copied with 16-channel boxes: the
 // copy still gives every pixel a 128-byte row and leaves its second half alone; those columns and lanes of the
 // accumulator hold products of whatever the shared memory held and are never read.  An MMA always reads 128 operand
 // rows = 4 blocks from the dy tile's base: blocks beyond the tile's own are the x tile or what follows it, and land in
@@ -1530,7 +1534,7 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_direct_kernel(const __grid_
         const int tid = threadIdx.x - 64;
         bool ok = true;
         if (p.passes == 3) {
-            // ---- splitters: hi stays where the copy put it, lo goes to the stage's second half, same position ----
+            // ---- splitters: the tile stays where the copy put it, its lo part goes to the stage's second half, same position ----
             const int stages = p.stages;
             // 16-byte pieces of the dy tile and of the x tiles.  A tile of a 16-channel tensor holds data in one half of
             // every 128-byte row only (which half: bit 1 of the row number, the swizzle's doing): 4 pieces per row then.
@@ -1552,9 +1556,9 @@ __global__ void __launch_bounds__(192) conv_tc_wgrad_direct_kernel(const __grid_
                         const int k = i - a4;
                         j = (int)(a_bytes >> 4) + (b_half ? ((k >> 2) << 3) + ((k >> 3) & 1) * 4 + (k & 3) : k);
                     }
+                    // the tile stays as copied: the tensor core's truncation of a 32-bit operand is the hi part
                     const float4 v = hi[j];
                     const float4 h = make_float4(tf32_hi(v.x), tf32_hi(v.y), tf32_hi(v.z), tf32_hi(v.w));
-                    hi[j] = h;
                     lo[j] = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
                 }
                 fence_async_smem();     // generic-proxy writes -> tensor-core reads
