@@ -380,12 +380,30 @@ def conv_sweep(args):
             reps = 2 if args.profile else max(10, 3 * nset)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             torch.cuda.synchronize()
-            e0.record()
-            for i in range(reps):
-                fn(i % nset)
-            e1.record()
-            torch.cuda.synchronize()
-            sec = e0.elapsed_time(e1) * 1e-3 / reps
+            if args.profile:
+                e0.record()
+                for i in range(reps):
+                    fn(i % nset)
+                e1.record()
+                torch.cuda.synchronize()
+                sec = e0.elapsed_time(e1) * 1e-3 / reps
+            else:
+                # the calls are captured once into a CUDA graph and the replay is timed: the figure is the kernels'
+                # launch-to-launch duration, not the host's call overhead (about 5 us per launch through ctypes)
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph):
+                    for i in range(reps):
+                        fn(i % nset)
+                graph.replay()
+                torch.cuda.synchronize()
+                cur = torch.cuda.current_stream()
+                e0.record(cur)
+                for _ in range(3):
+                    graph.replay()
+                e1.record(cur)
+                torch.cuda.synchronize()
+                sec = e0.elapsed_time(e1) * 1e-3 / (3 * reps)
+                del graph
             rows_out.append({"shape": "%dx%d s%d %d->%d @%d" % (ks, ks, st, ci, co, H), "pass": name, "us": sec * 1e6,
                              "tflops": flops / sec / 1e12, "gbs": nbytes / sec / 1e9, "ai": flops / nbytes})
         del xs, ys
