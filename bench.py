@@ -525,6 +525,8 @@ def main():
                          "(tuner.balance_by_measurement; its history, equal cuts first, goes into the line); "
                          "equal = the same number of ops in every partition")
     ap.add_argument("--conv-path", type=int, default=0)
+    ap.add_argument("--lanes", type=int, default=1,
+                    help="stage lanes (HPF_OPT_STAGE_LANES): micro-batches a stage keeps under way at once; 1 = the paper's schedule")
     ap.add_argument("--cell-ctas", type=int, default=-1,
                     help="CTAs of the persistent forward cell kernels (HPF_OPT_CELL_CTAS); 0: one launch per convolution; -1: the library's default")
     ap.add_argument("--hybrid-partitions", type=int, default=0,
@@ -593,6 +595,8 @@ def main():
     model.set_option(hpf.OPT_CONV_PATH, args.conv_path)
     if args.cell_ctas >= 0:
         model.set_option(hpf.OPT_CELL_CTAS, args.cell_ctas)
+    if args.lanes != 1:
+        model.set_option(hpf.OPT_STAGE_LANES, args.lanes)
     for kv in args.opt:
         k, v = kv.split("=")
         model.set_option(int(k), int(v))
@@ -688,7 +692,7 @@ def main():
         "config": {"workload": NAMES[args.workload], "global_batch": world * B, "micro_batches": M,
                    "partitions": model.num_partitions(), "parallelism": "replicas x%d, no data-path collective" % world,
                    "l2": "working set %.1f GB per step exceeds the 126 MB L2; no explicit flush" % (ws_bytes / 1e9),
-                   "cuts": args.cuts, "cut_points": list(cuts), "balance_history": balance_history, "graph": not args.no_graph, "cell_ctas": args.cell_ctas, "options": args.opt,
+                   "cuts": args.cuts, "cut_points": list(cuts), "balance_history": balance_history, "graph": not args.no_graph, "cell_ctas": args.cell_ctas, "stage_lanes": args.lanes, "options": args.opt,
                    "schedule": "forward then backward, two graphs (fill / drain twice)" if args.two_phases else
                                "hpf_forward_backward: one graph, a backward cell starts when the cell that feeds it is done",
                    "phase_ms": {"forward": phase_ms[0], "backward": phase_ms[1], "average": phase_ms[2]}, "conv_sites_tensor_core": n_tc, "conv_sites_cuda_core": n_cc,
