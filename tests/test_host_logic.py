@@ -128,6 +128,27 @@ def test_workspace_grows_with_message_buffers():
     assert b.workspace_bytes() > a.workspace_bytes()
 
 
+def test_stage_lanes_multiply_the_stream_slots_and_the_scratch():
+    """HPF_OPT_STAGE_LANES: S = P * min(L, M) stream slots, each with scratch of its own, so the workspace grows with L;
+    values outside 1..64 are refused.  Host only."""
+    c = wl.config("r11")
+    B = c["B"]
+    m = hpf.Model(c["ops"], (B,) + tuple(c["in_hwc"]), c["cuts"], c["M"])
+    P, M = m.num_partitions(), c["M"]
+    assert m.num_stream_slots() == P
+    one_lane = m.workspace_bytes()
+    m.set_option(hpf.OPT_STAGE_LANES, 2)
+    assert m.num_stream_slots() == P * min(2, M)
+    assert m.workspace_bytes() > one_lane
+    m.set_option(hpf.OPT_STAGE_LANES, 64)
+    assert m.num_stream_slots() == P * M                   # never more lanes than micro-batches
+    for bad in (0, -1, 65):
+        with pytest.raises(hpf.HpfError) as e:
+            m.set_option(hpf.OPT_STAGE_LANES, bad)
+        assert e.value.status == -1
+    m.close()
+
+
 def test_load_balancer_cuts():
     """Section 5.4's load balancer: contiguous partitions minimising the largest modelled partition cost."""
     import itertools
